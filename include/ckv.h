@@ -1,0 +1,191 @@
+/*
+ * ckv.h -- C ABI of the CollectiveKV decode-stage library for NVIDIA B200 (sm_100a).
+ *
+ * The library keeps, on one GPU, the learnable global K/V pool and the compressed
+ * per-user caches of the paper (Sec. 4.2), and attends users' queries over the K/V it
+ * rebuilds on chip:
+ *
+ *     K_c[i] = P_k[I_k[i]],  V_c[i] = P_v[I_v[i]]                    (Eq. Kc, inference branch)
+ *     K = concat(K_u, K_c),  V = concat(V_u, V_c),  d_a = d_u + d_g   (Eq. K; user part first)
+ *     out = attention(q, K, V)                                        (Sec. 4.2, last sentence)
+ *
+ * Full-width K/V never exist in device memory except through the test-only
+ * ckv_materialize.
+ *
+ * Conventions
+ *   - A "group" is one (layer, head) pair; every group has its own pool pair and its own
+ *     index pair.  n_groups = layers * heads.
+ *   - Indices are 0-based int32 at this boundary (the paper counts from 1).
+ *   - Pointers marked [host] must be host memory.  Pointers marked [any] may be device
+ *     memory or host memory (pinned or pageable); the library detects which and stages
+ *     host data through its own device buffers on `stream`.  With host *output* memory the
+ *     call returns after the copy has been enqueued; synchronise the stream before reading.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *     Calls enqueue work on it and return; ckv_cache_put* additionally wait for their own
+ *     index validation (one 4-byte read-back).
+ *   - The library copies what it is given: inputs may be released once the stream has
+ *     passed the call.  Outputs are caller-owned.
+ *   - Errors are return codes.  Nothing aborts, traps or throws across the boundary.  After
+ *     any error the context is unchanged and stays usable (CKV_ERR_CUDA excepted: the CUDA
+ *     context may be lost).
+ *   - A context belongs to one device and may be used by one host thread at a time.
+ */
+#ifndef CKV_H_
+#define CKV_H_
+
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define CKV_API __attribute__((visibility("default")))
+#else
+#define CKV_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ckv_ctx ckv_ctx;
+
+typedef enum {
+    CKV_OK = 0,
+    CKV_ERR_INVALID_ARG = 1,  /* NULL pointer, negative size, bad enum, offsets not monotone   */
+    CKV_ERR_SHAPE = 2,        /* d_shared + d_user != head_dim, or a size that contradicts the
+                                 pool already loaded                                           */
+    CKV_ERR_STATE = 3,        /* call needs a pool and none is loaded                          */
+    CKV_ERR_INDEX_RANGE = 4,  /* some pool index outside [0, n_entries)                        */
+    CKV_ERR_UNKNOWN_USER = 5, /* user id has no cache entry                                    */
+    CKV_ERR_OOM = 6,          /* device or host allocation failed                              */
+    CKV_ERR_CUDA = 7,         /* a CUDA call failed; see ckv_last_cuda_error                   */
+    CKV_ERR_UNSUPPORTED = 8   /* configuration outside what the kernels were built for         */
+} ckv_status;
+
+typedef enum { CKV_F32 = 0, CKV_BF16 = 1 } ckv_dtype;
+
+typedef enum {
+    CKV_SOFTMAX = 0,      /* p = softmax_i(scale * <q, K[i]>),  out = sum_i p_i V[i]            */
+    CKV_SILU_OVER_L = 1   /* out = (1/L_u) sum_i silu(scale * <q, K[i]>) V[i]  (HSTU-style)     */
+} ckv_mode;
+
+typedef struct {
+    int32_t n_groups;     /* >= 1                                                               */
+    int32_t head_dim;     /* d_a = d_shared + d_user; one of 16, 32, 64, 128                    */
+    int32_t dtype;        /* ckv_dtype of pool, user K/V and queries                            */
+    int32_t out_dtype;    /* ckv_dtype of the outputs (fp32 accumulator, rounded once, RNE)     */
+    int32_t mode;         /* ckv_mode                                                           */
+    float scale;          /* multiplies <q, K[i]>; <= 0 selects the default:
+                             1/sqrt(head_dim) for CKV_SOFTMAX, 1 for CKV_SILU_OVER_L            */
+    int32_t device;       /* CUDA device ordinal                                                */
+} ckv_config;
+
+/* Create / destroy a context on cfg->device.  ckv_destroy(NULL) is a no-op.
+ * Errors: INVALID_ARG, UNSUPPORTED (head_dim), CUDA, OOM. */
+CKV_API ckv_status ckv_create(const ckv_config* cfg, ckv_ctx** out);
+CKV_API ckv_status ckv_destroy(ckv_ctx* ctx);
+
+/*
+ * Global K/V pool P_k, P_v (Sec. 4.2: learnable tables shared by all users that stay in GPU
+ * memory at inference).
+ *   pool_K, pool_V [any] : [n_groups][n_entries][d_shared], contiguous, ctx dtype.
+ * The pool is copied into the library's own row layout (full head_dim-wide rows whose first
+ * d_user slots are zero) and asked to persist in L2.  Fixes d_user = head_dim - d_shared and
+ * the stored index width (16 bit when n_entries <= 65536, else 32 bit).  May be called again
+ * with the same n_entries and d_shared to refresh the values; any other reload while users
+ * are cached is CKV_ERR_SHAPE.
+ * Errors: INVALID_ARG (NULL, n_entries < 1), SHAPE (d_shared outside [1, head_dim]), OOM, CUDA.
+ */
+CKV_API ckv_status ckv_pool_load(ckv_ctx* ctx, const void* pool_K, const void* pool_V,
+                         int32_t n_entries, int32_t d_shared, void* stream);
+
+/*
+ * Store one user's compressed cache (Sec. 4.2, prefill output: global K/V indices plus
+ * user-specific K/V), replacing any earlier entry of `user`.
+ *   idx_K, idx_V   [any] : int32 [L][n_groups]  (may alias each other)
+ *   user_K, user_V [any] : [L][n_groups][d_user], ctx dtype; may be NULL iff d_user == 0
+ *   L >= 0 (a user with an empty history is legal and attends to a zero output).
+ * Errors: STATE (no pool), SHAPE (d_user != head_dim - d_shared), INVALID_ARG,
+ *         INDEX_RANGE (cache unchanged), OOM, CUDA.
+ */
+CKV_API ckv_status ckv_cache_put(ckv_ctx* ctx, int64_t user, int32_t L,
+                         const int32_t* idx_K, const int32_t* idx_V,
+                         const void* user_K, const void* user_V, int32_t d_user, void* stream);
+
+/*
+ * Bulk form: n users whose histories are concatenated along the position axis.
+ *   users [host] : int64 [n], distinct;  hist_off [host] : int64 [n+1], non-decreasing,
+ *   hist_off[0] = 0;  arrays as in ckv_cache_put with L = hist_off[n].
+ * All-or-nothing: on any error no user of the batch is stored.
+ */
+CKV_API ckv_status ckv_cache_put_batch(ckv_ctx* ctx, int32_t n, const int64_t* users,
+                               const int64_t* hist_off,
+                               const int32_t* idx_K, const int32_t* idx_V,
+                               const void* user_K, const void* user_V, int32_t d_user,
+                               void* stream);
+
+/* Forget one user / all users (the pool stays).  Unknown user: CKV_ERR_UNKNOWN_USER. */
+CKV_API ckv_status ckv_cache_evict(ckv_ctx* ctx, int64_t user);
+CKV_API ckv_status ckv_cache_clear(ckv_ctx* ctx);
+
+/*
+ * Decode: rebuild each listed user's K/V (Eq. Kc, Eq. K) on chip and attend the user's
+ * queries over it, in the context's mode.  Candidates are independent target-attention
+ * queries (Sec. 2.1: Q in R^{1 x d} per target item); there is no mask.
+ *   users   [host] : int64 [n]   (a user may appear more than once)
+ *   q_off   [host] : int32 [n+1], non-decreasing, q_off[0] = 0; user k owns query rows
+ *                    q_off[k] .. q_off[k+1]-1
+ *   queries [any]  : [q_off[n]][n_groups][head_dim], ctx dtype
+ *   out     [any]  : [q_off[n]][n_groups][head_dim], ctx out_dtype, caller-allocated
+ * A user with an empty history produces zero rows.  Results do not depend on how the
+ * library splits long histories across thread blocks beyond fp32 rounding, and are bitwise
+ * reproducible from call to call for the same context settings.
+ * Errors: STATE, INVALID_ARG, UNKNOWN_USER, OOM (workspace), CUDA.
+ */
+CKV_API ckv_status ckv_attend(ckv_ctx* ctx, int32_t n, const int64_t* users, const int32_t* q_off,
+                      const void* queries, void* out, void* stream);
+
+/*
+ * TEST ONLY -- the single path that writes full-width K/V to device memory: Eq. (Kc) and
+ * Eq. (K) for one user.  K_out, V_out [any] : [L][n_groups][head_dim], ctx dtype.  The result
+ * is a pure copy of input bits.
+ */
+CKV_API ckv_status ckv_materialize(ckv_ctx* ctx, int64_t user, void* K_out, void* V_out, void* stream);
+
+/* History length of a cached user.  Errors: UNKNOWN_USER. */
+CKV_API ckv_status ckv_user_length(ckv_ctx* ctx, int64_t user, int64_t* L);
+
+/*
+ * Storage accounting over all cached users (Sec. 5.1 compression rate, Sec. 4.4 load size):
+ *   compressed = bytes of stored indices + user-specific K/V (padding excluded)
+ *   full_width = bytes a classical cache would hold: 2 * positions * n_groups * head_dim * e
+ */
+CKV_API ckv_status ckv_cache_bytes(ckv_ctx* ctx, int64_t* compressed, int64_t* full_width);
+
+/*
+ * Tuning and test knobs (integers).  Unknown name: INVALID_ARG.
+ *   "split_len"    positions per history chunk for the split-along-history reduction;
+ *                  0 = choose automatically (default)
+ *   "kernel"       0 = choose by queries per user (default); 1 = CUDA-core kernel;
+ *                  2 = warp-level tensor-core kernel; 3 = tcgen05 kernel
+ *   "l2_persist"   1 = ask for the pool to persist in L2 on the streams used (default), 0 = off
+ */
+CKV_API ckv_status ckv_set_option(ckv_ctx* ctx, const char* name, int64_t value);
+CKV_API ckv_status ckv_get_option(ckv_ctx* ctx, const char* name, int64_t* value);
+
+/*
+ * Introspection for tests and the benchmark.  Counters describe the most recent
+ * ckv_attend: "launches" (kernels enqueued), "work_items", "split_items" (items that went
+ * through the partial-result workspace), "kernel" (family that ran: 1, 2 or 3),
+ * "workspace_bytes", "plan_cache_hit".
+ */
+CKV_API ckv_status ckv_last_stat(ckv_ctx* ctx, const char* name, int64_t* value);
+
+CKV_API const char* ckv_strerror(ckv_status s);
+/* Text of the last CUDA error seen by this context ("" if none). */
+CKV_API const char* ckv_last_cuda_error(ckv_ctx* ctx);
+/* Library version as major*10000 + minor*100 + patch. */
+CKV_API int32_t ckv_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CKV_H_ */

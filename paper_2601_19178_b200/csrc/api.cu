@@ -1,0 +1,705 @@
+// Host side of the library: context, pool and compressed-cache management, attend
+// planning (history chunking for the split-along-history reduction) and kernel dispatch.
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <string>
+#include <unordered_map>
+#include <vector>
+
+#include "ckv_internal.h"
+
+using namespace ckv;
+
+namespace {
+
+struct UserEntry {
+    int64_t base;
+    int32_t L;
+    int32_t Lpad;
+};
+
+struct DevBuf {  // grow-only device buffer
+    void* p = nullptr;
+    size_t cap = 0;
+};
+
+struct Plan {
+    std::vector<int64_t> users;
+    std::vector<int32_t> q_off;
+    uint64_t generation = 0;
+    int64_t opt_split = 0, opt_kernel = 0;
+    void* dev = nullptr;  // one allocation: reqs | items | split list
+    Req* d_reqs = nullptr;
+    Item* d_items = nullptr;
+    int32_t* d_split = nullptr;
+    int32_t n_items = 0, n_split = 0, split_items = 0, max_M = 0, family = 1;
+    int64_t part_rows = 0;
+    uint64_t last_use = 0;
+};
+
+constexpr int kMaxPlans = 4;
+constexpr int kNumSMs = 148;
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok;
+    explicit DeviceGuard(int dev)
+    {
+        ok = cudaGetDevice(&prev) == cudaSuccess;
+        if (ok && prev != dev) ok = cudaSetDevice(dev) == cudaSuccess;
+    }
+    ~DeviceGuard()
+    {
+        int cur = -1;
+        if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+    }
+};
+
+}  // namespace
+
+struct ckv_ctx {
+    ckv_config cfg{};
+    float scale = 1.f;
+    int elem = 2;  // bytes per element of cfg.dtype
+    // pool
+    int n_entries = 0, d_shared = 0, d_user = 0, idx_bytes = 0;
+    void* pool = nullptr;  // K rows then V rows, each [G][m][D]
+    size_t pool_half = 0;  // bytes of one of them
+    // arena of compressed caches (units = (position, group) slots)
+    void *a_idxK = nullptr, *a_idxV = nullptr, *a_userK = nullptr, *a_userV = nullptr;
+    int64_t cap_units = 0, used_units = 0, live_positions = 0;
+    std::unordered_map<int64_t, UserEntry> users;
+    uint64_t generation = 1;
+    // scratch
+    DevBuf stage_q, stage_out, partials;
+    int* d_flag = nullptr;
+    std::vector<Plan> plans;
+    uint64_t tick = 0;
+    // options
+    int64_t opt_split = 0, opt_kernel = 0, opt_l2 = 1;
+    // statistics of the last attend
+    int64_t st_launches = 0, st_items = 0, st_split = 0, st_kernel = 0, st_ws = 0, st_hit = 0;
+    std::string cuda_err;
+
+    ckv_status fail(cudaError_t e)
+    {
+        cuda_err = std::string(cudaGetErrorName(e)) + ": " + cudaGetErrorString(e);
+        cudaGetLastError();  // clear the sticky-free error state
+        return e == cudaErrorMemoryAllocation ? CKV_ERR_OOM : CKV_ERR_CUDA;
+    }
+};
+
+#define CK(call)                                        \
+    do {                                                \
+        cudaError_t e_ = (call);                        \
+        if (e_ != cudaSuccess) return ctx->fail(e_);    \
+    } while (0)
+
+namespace {
+
+bool is_device_ptr(const void* p)
+{
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, p) != cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    return at.type == cudaMemoryTypeDevice || at.type == cudaMemoryTypeManaged;
+}
+
+// A temporary device copy of host input, freed by the destructor.
+struct Staged {
+    const void* dev = nullptr;
+    void* owned = nullptr;
+    ~Staged()
+    {
+        if (owned) cudaFree(owned);
+    }
+    cudaError_t init(const void* src, size_t bytes, cudaStream_t s)
+    {
+        if (bytes == 0 || src == nullptr || is_device_ptr(src)) {
+            dev = src;
+            return cudaSuccess;
+        }
+        cudaError_t e = cudaMalloc(&owned, bytes);
+        if (e != cudaSuccess) return e;
+        dev = owned;
+        return cudaMemcpyAsync(owned, src, bytes, cudaMemcpyHostToDevice, s);
+    }
+};
+
+cudaError_t grow(DevBuf& b, size_t bytes)
+{
+    if (bytes <= b.cap) return cudaSuccess;
+    if (b.p) {
+        cudaError_t e = cudaFree(b.p);  // waits for work that may still use it
+        b.p = nullptr;
+        b.cap = 0;
+        if (e != cudaSuccess) return e;
+    }
+    size_t want = bytes + bytes / 4;
+    cudaError_t e = cudaMalloc(&b.p, want);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        want = bytes;
+        e = cudaMalloc(&b.p, want);
+        if (e != cudaSuccess) return e;
+    }
+    b.cap = want;
+    return cudaSuccess;
+}
+
+void free_plan(Plan& p)
+{
+    if (p.dev) cudaFree(p.dev);
+    p.dev = nullptr;
+}
+
+void drop_plans(ckv_ctx* ctx)
+{
+    for (auto& p : ctx->plans) free_plan(p);
+    ctx->plans.clear();
+}
+
+CacheView view_of(const ckv_ctx* ctx)
+{
+    CacheView v;
+    v.poolK = ctx->pool;
+    v.poolV = (const char*)ctx->pool + ctx->pool_half;
+    v.idxK = ctx->a_idxK;
+    v.idxV = ctx->a_idxV;
+    v.userK = ctx->a_userK;
+    v.userV = ctx->a_userV;
+    v.n_groups = ctx->cfg.n_groups;
+    v.n_entries = ctx->n_entries;
+    v.d_user = ctx->d_user;
+    v.idx_bytes = ctx->idx_bytes;
+    return v;
+}
+
+// Make room for `need` more units, keeping what is stored.
+ckv_status ensure_arena(ckv_ctx* ctx, int64_t need, cudaStream_t s)
+{
+    if (ctx->used_units + need <= ctx->cap_units) return CKV_OK;
+    int64_t cap = std::max<int64_t>(ctx->cap_units * 2, ctx->used_units + need);
+    cap = (cap + 1023) / 1024 * 1024;
+    const size_t ub = (size_t)std::max(ctx->d_user, 1) * ctx->elem;
+    void* n[4] = {nullptr, nullptr, nullptr, nullptr};
+    const size_t bytes[4] = {(size_t)cap * ctx->idx_bytes, (size_t)cap * ctx->idx_bytes, (size_t)cap * ub,
+                             (size_t)cap * ub};
+    void* old[4] = {ctx->a_idxK, ctx->a_idxV, ctx->a_userK, ctx->a_userV};
+    for (int i = 0; i < 4; ++i) {
+        cudaError_t e = cudaMalloc(&n[i], bytes[i]);
+        if (e != cudaSuccess) {
+            for (int j = 0; j < i; ++j) cudaFree(n[j]);
+            return ctx->fail(e);
+        }
+    }
+    const size_t used[4] = {(size_t)ctx->used_units * ctx->idx_bytes, (size_t)ctx->used_units * ctx->idx_bytes,
+                            (size_t)ctx->used_units * ub, (size_t)ctx->used_units * ub};
+    for (int i = 0; i < 4; ++i)
+        if (used[i]) {
+            cudaError_t e = cudaMemcpyAsync(n[i], old[i], used[i], cudaMemcpyDeviceToDevice, s);
+            if (e != cudaSuccess) {
+                for (int j = 0; j < 4; ++j) cudaFree(n[j]);
+                return ctx->fail(e);
+            }
+        }
+    CK(cudaStreamSynchronize(s));
+    for (int i = 0; i < 4; ++i)
+        if (old[i]) cudaFree(old[i]);
+    ctx->a_idxK = n[0];
+    ctx->a_idxV = n[1];
+    ctx->a_userK = n[2];
+    ctx->a_userV = n[3];
+    ctx->cap_units = cap;
+    return CKV_OK;
+}
+
+int64_t auto_split_len(const ckv_ctx* ctx, int64_t total_positions, int family)
+{
+    // Enough (chunk, group) blocks to fill the SMs several times over, but chunks long
+    // enough that the merge of partial results stays a small fraction of the work.
+    (void)family;
+    int64_t c = total_positions * ctx->cfg.n_groups / (kNumSMs * 16);
+    c = (c + 63) / 64 * 64;
+    return std::min<int64_t>(std::max<int64_t>(c, 256), 2048);
+}
+
+ckv_status build_plan(ckv_ctx* ctx, Plan& pl, int32_t n, const int64_t* users, const int32_t* q_off,
+                      cudaStream_t s)
+{
+    std::vector<Req> reqs((size_t)n);
+    int64_t total_pos = 0;
+    int32_t max_M = 0;
+    for (int32_t k = 0; k < n; ++k) {
+        auto f = ctx->users.find(users[k]);
+        if (f == ctx->users.end()) return CKV_ERR_UNKNOWN_USER;
+        Req& r = reqs[k];
+        r.base = f->second.base;
+        r.L = f->second.L;
+        r.Lpad = f->second.Lpad;
+        r.q0 = q_off[k];
+        r.M = q_off[k + 1] - q_off[k];
+        r.part0 = -1;
+        r.n_chunks = 1;
+        if (r.M > 0) total_pos += r.L;
+        max_M = std::max(max_M, r.M);
+    }
+    pl.max_M = max_M;
+    pl.family = 1;
+    const int64_t C = ctx->opt_split > 0 ? ctx->opt_split : auto_split_len(ctx, total_pos, pl.family);
+    std::vector<Item> items;
+    std::vector<int32_t> split;
+    items.reserve((size_t)n);
+    int64_t part_rows = 0;
+    for (int32_t k = 0; k < n; ++k) {
+        Req& r = reqs[k];
+        if (r.M <= 0) continue;
+        const int64_t nc = r.L == 0 ? 1 : (r.L + C - 1) / C;
+        r.n_chunks = (int32_t)nc;
+        if (nc == 1) {
+            items.push_back(Item{k, 0, r.L, -1});
+            continue;
+        }
+        if (part_rows + nc * r.M > INT32_MAX) return CKV_ERR_UNSUPPORTED;
+        r.part0 = (int32_t)part_rows;
+        split.push_back(k);
+        for (int64_t c = 0; c < nc; ++c) {
+            const int32_t b = (int32_t)(c * C);
+            items.push_back(Item{k, b, (int32_t)std::min<int64_t>(C, r.L - b), (int32_t)(part_rows + c * r.M)});
+        }
+        part_rows += nc * r.M;
+    }
+    // longest chunks first: the tail of the grid is made of short ones
+    std::stable_sort(items.begin(), items.end(), [](const Item& x, const Item& y) { return x.len > y.len; });
+    pl.n_items = (int32_t)items.size();
+    pl.n_split = (int32_t)split.size();
+    pl.split_items = 0;
+    for (const Item& it : items) pl.split_items += it.part_row >= 0;
+    pl.part_rows = part_rows;
+
+    const size_t b_req = sizeof(Req) * reqs.size(), b_item = sizeof(Item) * items.size(),
+                 b_split = sizeof(int32_t) * split.size();
+    const size_t o_item = (b_req + 255) / 256 * 256, o_split = o_item + (b_item + 255) / 256 * 256;
+    CK(cudaMalloc(&pl.dev, o_split + b_split + 256));
+    pl.d_reqs = (Req*)pl.dev;
+    pl.d_items = (Item*)((char*)pl.dev + o_item);
+    pl.d_split = (int32_t*)((char*)pl.dev + o_split);
+    if (b_req) CK(cudaMemcpyAsync(pl.d_reqs, reqs.data(), b_req, cudaMemcpyHostToDevice, s));
+    if (b_item) CK(cudaMemcpyAsync(pl.d_items, items.data(), b_item, cudaMemcpyHostToDevice, s));
+    if (b_split) CK(cudaMemcpyAsync(pl.d_split, split.data(), b_split, cudaMemcpyHostToDevice, s));
+    // the host vectors die at return: pageable copies have been staged by then
+    pl.users.assign(users, users + n);
+    pl.q_off.assign(q_off, q_off + n + 1);
+    pl.generation = ctx->generation;
+    pl.opt_split = ctx->opt_split;
+    pl.opt_kernel = ctx->opt_kernel;
+    return CKV_OK;
+}
+
+ckv_status get_plan(ckv_ctx* ctx, int32_t n, const int64_t* users, const int32_t* q_off, cudaStream_t s,
+                    Plan** out)
+{
+    ctx->tick++;
+    for (auto& p : ctx->plans) {
+        if (p.generation == ctx->generation && p.opt_split == ctx->opt_split &&
+            p.opt_kernel == ctx->opt_kernel && (int32_t)p.users.size() == n &&
+            std::memcmp(p.users.data(), users, sizeof(int64_t) * (size_t)n) == 0 &&
+            std::memcmp(p.q_off.data(), q_off, sizeof(int32_t) * ((size_t)n + 1)) == 0) {
+            p.last_use = ctx->tick;
+            ctx->st_hit = 1;
+            *out = &p;
+            return CKV_OK;
+        }
+    }
+    ctx->st_hit = 0;
+    // drop stale plans, then the least recently used one if the cache is full
+    for (size_t i = 0; i < ctx->plans.size();) {
+        if (ctx->plans[i].generation != ctx->generation) {
+            free_plan(ctx->plans[i]);
+            ctx->plans.erase(ctx->plans.begin() + i);
+        } else {
+            ++i;
+        }
+    }
+    if ((int)ctx->plans.size() >= kMaxPlans) {
+        size_t lru = 0;
+        for (size_t i = 1; i < ctx->plans.size(); ++i)
+            if (ctx->plans[i].last_use < ctx->plans[lru].last_use) lru = i;
+        free_plan(ctx->plans[lru]);
+        ctx->plans.erase(ctx->plans.begin() + lru);
+    }
+    Plan pl;
+    ckv_status st = build_plan(ctx, pl, n, users, q_off, s);
+    if (st != CKV_OK) {
+        free_plan(pl);
+        return st;
+    }
+    pl.last_use = ctx->tick;
+    ctx->plans.push_back(std::move(pl));
+    *out = &ctx->plans.back();
+    return CKV_OK;
+}
+
+bool offsets_ok32(const int32_t* off, int32_t n)
+{
+    if (off[0] != 0) return false;
+    for (int32_t k = 0; k < n; ++k)
+        if (off[k + 1] < off[k]) return false;
+    return true;
+}
+
+}  // namespace
+
+extern "C" {
+
+ckv_status ckv_create(const ckv_config* cfg, ckv_ctx** out)
+{
+    if (!cfg || !out) return CKV_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (cfg->n_groups < 1 || cfg->n_groups > 65535) return CKV_ERR_INVALID_ARG;
+    if ((cfg->dtype != CKV_F32 && cfg->dtype != CKV_BF16) ||
+        (cfg->out_dtype != CKV_F32 && cfg->out_dtype != CKV_BF16) ||
+        (cfg->mode != CKV_SOFTMAX && cfg->mode != CKV_SILU_OVER_L) || cfg->device < 0)
+        return CKV_ERR_INVALID_ARG;
+    if (cfg->head_dim != 16 && cfg->head_dim != 32 && cfg->head_dim != 64 && cfg->head_dim != 128)
+        return CKV_ERR_UNSUPPORTED;
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || cfg->device >= ndev) {
+        cudaGetLastError();
+        return CKV_ERR_CUDA;
+    }
+    ckv_ctx* ctx = new (std::nothrow) ckv_ctx();
+    if (!ctx) return CKV_ERR_OOM;
+    ctx->cfg = *cfg;
+    ctx->elem = cfg->dtype == CKV_BF16 ? 2 : 4;
+    ctx->scale = cfg->scale > 0.f ? cfg->scale
+                                  : (cfg->mode == CKV_SOFTMAX ? 1.0f / std::sqrt((float)cfg->head_dim) : 1.0f);
+    DeviceGuard dg(cfg->device);
+    if (!dg.ok || cudaMalloc((void**)&ctx->d_flag, sizeof(int)) != cudaSuccess) {
+        cudaGetLastError();
+        delete ctx;
+        return CKV_ERR_CUDA;
+    }
+    *out = ctx;
+    return CKV_OK;
+}
+
+ckv_status ckv_destroy(ckv_ctx* ctx)
+{
+    if (!ctx) return CKV_OK;
+    DeviceGuard dg(ctx->cfg.device);
+    drop_plans(ctx);
+    void* bufs[] = {ctx->pool,    ctx->a_idxK,     ctx->a_idxV,      ctx->a_userK,   ctx->a_userV,
+                    ctx->d_flag,  ctx->stage_q.p,  ctx->stage_out.p, ctx->partials.p};
+    for (void* b : bufs)
+        if (b) cudaFree(b);
+    cudaGetLastError();
+    delete ctx;
+    return CKV_OK;
+}
+
+ckv_status ckv_pool_load(ckv_ctx* ctx, const void* pool_K, const void* pool_V, int32_t n_entries,
+                         int32_t d_shared, void* stream)
+{
+    if (!ctx || !pool_K || !pool_V || n_entries < 1) return CKV_ERR_INVALID_ARG;
+    const int D = ctx->cfg.head_dim, G = ctx->cfg.n_groups;
+    if (d_shared < 1 || d_shared > D) return CKV_ERR_SHAPE;
+    if (!ctx->users.empty() && (n_entries != ctx->n_entries || d_shared != ctx->d_shared)) return CKV_ERR_SHAPE;
+    DeviceGuard dg(ctx->cfg.device);
+    cudaStream_t s = (cudaStream_t)stream;
+    const size_t half = (size_t)G * n_entries * D * ctx->elem;
+    const size_t src_bytes = (size_t)G * n_entries * d_shared * ctx->elem;
+    Staged sk, sv;
+    CK(sk.init(pool_K, src_bytes, s));
+    CK(sv.init(pool_V, src_bytes, s));
+    if (!ctx->pool || half != ctx->pool_half) {
+        void* np = nullptr;
+        CK(cudaMalloc(&np, 2 * half));
+        if (ctx->pool) cudaFree(ctx->pool);
+        ctx->pool = np;
+        ctx->pool_half = half;
+    }
+    CK(launch_pool_layout(ctx->cfg.dtype, G, n_entries, d_shared, D, sk.dev, ctx->pool, s));
+    CK(launch_pool_layout(ctx->cfg.dtype, G, n_entries, d_shared, D, sv.dev, (char*)ctx->pool + half, s));
+    if (sk.owned || sv.owned) CK(cudaStreamSynchronize(s));
+    if (ctx->users.empty() && (ctx->n_entries != n_entries || ctx->d_shared != d_shared)) {
+        // index width or user width may change: restart the (empty) arena
+        void* old[4] = {ctx->a_idxK, ctx->a_idxV, ctx->a_userK, ctx->a_userV};
+        for (void* b : old)
+            if (b) cudaFree(b);
+        ctx->a_idxK = ctx->a_idxV = ctx->a_userK = ctx->a_userV = nullptr;
+        ctx->cap_units = ctx->used_units = 0;
+    }
+    ctx->n_entries = n_entries;
+    ctx->d_shared = d_shared;
+    ctx->d_user = D - d_shared;
+    ctx->idx_bytes = n_entries <= 65536 ? 2 : 4;
+    return CKV_OK;
+}
+
+ckv_status ckv_cache_put_batch(ckv_ctx* ctx, int32_t n, const int64_t* users, const int64_t* hist_off,
+                               const int32_t* idx_K, const int32_t* idx_V, const void* user_K,
+                               const void* user_V, int32_t d_user, void* stream)
+{
+    if (!ctx || n < 0 || (n > 0 && (!users || !hist_off))) return CKV_ERR_INVALID_ARG;
+    if (!ctx->pool) return CKV_ERR_STATE;
+    if (d_user != ctx->d_user) return CKV_ERR_SHAPE;
+    if (n == 0) return CKV_OK;
+    if (hist_off[0] != 0) return CKV_ERR_INVALID_ARG;
+    const int G = ctx->cfg.n_groups;
+    std::vector<int64_t> unit_off((size_t)n + 1);
+    unit_off[0] = 0;
+    for (int32_t k = 0; k < n; ++k) {
+        const int64_t L = hist_off[k + 1] - hist_off[k];
+        if (L < 0 || L > INT32_MAX - 8) return CKV_ERR_INVALID_ARG;
+        unit_off[k + 1] = unit_off[k] + (int64_t)G * ((L + 7) / 8 * 8);
+    }
+    const int64_t P = hist_off[n], total_units = unit_off[n];
+    if (P > 0 && (!idx_K || !idx_V || (d_user > 0 && (!user_K || !user_V)))) return CKV_ERR_INVALID_ARG;
+
+    DeviceGuard dg(ctx->cfg.device);
+    cudaStream_t s = (cudaStream_t)stream;
+    if (total_units > 0) {
+        Staged sik, siv, suk, suv, sho, suo;
+        const size_t ib = (size_t)P * G * sizeof(int32_t), ubytes = (size_t)P * G * d_user * ctx->elem;
+        CK(sik.init(idx_K, ib, s));
+        if (idx_V == idx_K) siv.dev = sik.dev; else CK(siv.init(idx_V, ib, s));
+        CK(suk.init(user_K, ubytes, s));
+        CK(suv.init(user_V, ubytes, s));
+        CK(sho.init(hist_off, sizeof(int64_t) * ((size_t)n + 1), s));
+        CK(suo.init(unit_off.data(), sizeof(int64_t) * ((size_t)n + 1), s));
+        ckv_status st = ensure_arena(ctx, total_units, s);
+        if (st != CKV_OK) return st;
+        CK(cudaMemsetAsync(ctx->d_flag, 0, sizeof(int), s));
+        CK(launch_pack(ctx->cfg.dtype, G, ctx->n_entries, d_user, ctx->idx_bytes, n, (const int64_t*)sho.dev,
+                       (const int64_t*)suo.dev, total_units, ctx->used_units, (const int32_t*)sik.dev,
+                       (const int32_t*)siv.dev, suk.dev, suv.dev, ctx->a_idxK, ctx->a_idxV, ctx->a_userK,
+                       ctx->a_userV, ctx->d_flag, s));
+        int bad = 0;
+        CK(cudaMemcpyAsync(&bad, ctx->d_flag, sizeof(int), cudaMemcpyDeviceToHost, s));
+        CK(cudaStreamSynchronize(s));
+        if (bad) return CKV_ERR_INDEX_RANGE;  // used_units not advanced: nothing was stored
+    }
+    for (int32_t k = 0; k < n; ++k) {
+        const int64_t L = hist_off[k + 1] - hist_off[k];
+        auto f = ctx->users.find(users[k]);
+        if (f != ctx->users.end()) ctx->live_positions -= f->second.L;
+        ctx->users[users[k]] = UserEntry{ctx->used_units + unit_off[k], (int32_t)L, (int32_t)((L + 7) / 8 * 8)};
+        ctx->live_positions += L;
+    }
+    ctx->used_units += total_units;
+    ctx->generation++;
+    return CKV_OK;
+}
+
+ckv_status ckv_cache_put(ckv_ctx* ctx, int64_t user, int32_t L, const int32_t* idx_K, const int32_t* idx_V,
+                         const void* user_K, const void* user_V, int32_t d_user, void* stream)
+{
+    if (L < 0) return CKV_ERR_INVALID_ARG;
+    const int64_t off[2] = {0, L};
+    return ckv_cache_put_batch(ctx, 1, &user, off, idx_K, idx_V, user_K, user_V, d_user, stream);
+}
+
+ckv_status ckv_cache_evict(ckv_ctx* ctx, int64_t user)
+{
+    if (!ctx) return CKV_ERR_INVALID_ARG;
+    auto f = ctx->users.find(user);
+    if (f == ctx->users.end()) return CKV_ERR_UNKNOWN_USER;
+    ctx->live_positions -= f->second.L;
+    ctx->users.erase(f);
+    ctx->generation++;
+    if (ctx->users.empty()) ctx->used_units = 0;
+    return CKV_OK;
+}
+
+ckv_status ckv_cache_clear(ckv_ctx* ctx)
+{
+    if (!ctx) return CKV_ERR_INVALID_ARG;
+    ctx->users.clear();
+    ctx->live_positions = 0;
+    ctx->used_units = 0;
+    ctx->generation++;
+    return CKV_OK;
+}
+
+ckv_status ckv_attend(ckv_ctx* ctx, int32_t n, const int64_t* users, const int32_t* q_off,
+                      const void* queries, void* out, void* stream)
+{
+    if (!ctx || n < 0 || (n > 0 && (!users || !q_off))) return CKV_ERR_INVALID_ARG;
+    if (!ctx->pool) return CKV_ERR_STATE;
+    if (n == 0) return CKV_OK;
+    if (!offsets_ok32(q_off, n)) return CKV_ERR_INVALID_ARG;
+    const int64_t Q = q_off[n];
+    if (Q > 0 && (!queries || !out)) return CKV_ERR_INVALID_ARG;
+    DeviceGuard dg(ctx->cfg.device);
+    cudaStream_t s = (cudaStream_t)stream;
+    ctx->st_launches = 0;
+    Plan* pl = nullptr;
+    ckv_status st = get_plan(ctx, n, users, q_off, s, &pl);
+    if (st != CKV_OK) return st;
+    ctx->st_items = pl->n_items;
+    ctx->st_split = pl->split_items;
+    ctx->st_kernel = pl->family;
+    if (Q == 0) return CKV_OK;
+
+    const int D = ctx->cfg.head_dim, G = ctx->cfg.n_groups;
+    const size_t q_bytes = (size_t)Q * G * D * ctx->elem;
+    const size_t o_bytes = (size_t)Q * G * D * (ctx->cfg.out_dtype == CKV_BF16 ? 2 : 4);
+    const void* d_q = queries;
+    void* d_out = out;
+    const bool q_host = !is_device_ptr(queries), o_host = !is_device_ptr(out);
+    if (q_host) {
+        CK(grow(ctx->stage_q, q_bytes));
+        CK(cudaMemcpyAsync(ctx->stage_q.p, queries, q_bytes, cudaMemcpyHostToDevice, s));
+        d_q = ctx->stage_q.p;
+    }
+    if (o_host) {
+        CK(grow(ctx->stage_out, o_bytes));
+        d_out = ctx->stage_out.p;
+    }
+    const size_t ws = (size_t)pl->part_rows * G * (D + 2) * sizeof(float);
+    if (ws) CK(grow(ctx->partials, ws));
+    ctx->st_ws = (int64_t)ws;
+
+    AttendArgs a;
+    a.cv = view_of(ctx);
+    a.reqs = pl->d_reqs;
+    a.items = pl->d_items;
+    a.n_items = pl->n_items;
+    a.queries = d_q;
+    a.out = d_out;
+    a.partials = (float*)ctx->partials.p;
+    a.out_dtype = ctx->cfg.out_dtype;
+    a.mode = ctx->cfg.mode;
+    a.scale = ctx->scale;
+    if (pl->n_items > 0) {
+        CK(launch_attend_simt(ctx->cfg.dtype, D, pl->max_M, a, s));
+        ctx->st_launches++;
+    }
+    if (pl->n_split > 0) {
+        CK(launch_combine(D, a, pl->d_split, pl->n_split, s));
+        ctx->st_launches++;
+    }
+    if (o_host) CK(cudaMemcpyAsync(out, d_out, o_bytes, cudaMemcpyDeviceToHost, s));
+    return CKV_OK;
+}
+
+ckv_status ckv_materialize(ckv_ctx* ctx, int64_t user, void* K_out, void* V_out, void* stream)
+{
+    if (!ctx || !K_out || !V_out) return CKV_ERR_INVALID_ARG;
+    if (!ctx->pool) return CKV_ERR_STATE;
+    auto f = ctx->users.find(user);
+    if (f == ctx->users.end()) return CKV_ERR_UNKNOWN_USER;
+    const UserEntry& e = f->second;
+    if (e.L == 0) return CKV_OK;
+    DeviceGuard dg(ctx->cfg.device);
+    cudaStream_t s = (cudaStream_t)stream;
+    const int D = ctx->cfg.head_dim;
+    const size_t bytes = (size_t)e.L * ctx->cfg.n_groups * D * ctx->elem;
+    const bool kh = !is_device_ptr(K_out), vh = !is_device_ptr(V_out);
+    void *dk = K_out, *dv = V_out, *tk = nullptr, *tv = nullptr;
+    if (kh) {
+        CK(cudaMalloc(&tk, bytes));
+        dk = tk;
+    }
+    if (vh) {
+        cudaError_t er = cudaMalloc(&tv, bytes);
+        if (er != cudaSuccess) {
+            if (tk) cudaFree(tk);
+            return ctx->fail(er);
+        }
+        dv = tv;
+    }
+    cudaError_t er = launch_materialize(ctx->cfg.dtype, D, view_of(ctx), e.base, e.L, e.Lpad, dk, dv, s);
+    if (er == cudaSuccess && kh) er = cudaMemcpyAsync(K_out, dk, bytes, cudaMemcpyDeviceToHost, s);
+    if (er == cudaSuccess && vh) er = cudaMemcpyAsync(V_out, dv, bytes, cudaMemcpyDeviceToHost, s);
+    if (er == cudaSuccess && (kh || vh)) er = cudaStreamSynchronize(s);
+    if (tk) cudaFree(tk);
+    if (tv) cudaFree(tv);
+    if (er != cudaSuccess) return ctx->fail(er);
+    return CKV_OK;
+}
+
+ckv_status ckv_user_length(ckv_ctx* ctx, int64_t user, int64_t* L)
+{
+    if (!ctx || !L) return CKV_ERR_INVALID_ARG;
+    auto f = ctx->users.find(user);
+    if (f == ctx->users.end()) return CKV_ERR_UNKNOWN_USER;
+    *L = f->second.L;
+    return CKV_OK;
+}
+
+ckv_status ckv_cache_bytes(ckv_ctx* ctx, int64_t* compressed, int64_t* full_width)
+{
+    if (!ctx || !compressed || !full_width) return CKV_ERR_INVALID_ARG;
+    const int64_t pg = ctx->live_positions * ctx->cfg.n_groups;
+    *compressed = pg * (2 * (int64_t)ctx->idx_bytes + 2 * (int64_t)ctx->d_user * ctx->elem);
+    *full_width = pg * 2 * (int64_t)ctx->cfg.head_dim * ctx->elem;
+    return CKV_OK;
+}
+
+ckv_status ckv_set_option(ckv_ctx* ctx, const char* name, int64_t value)
+{
+    if (!ctx || !name) return CKV_ERR_INVALID_ARG;
+    if (!std::strcmp(name, "split_len")) {
+        if (value < 0) return CKV_ERR_INVALID_ARG;
+        ctx->opt_split = value == 0 ? 0 : (value + 7) / 8 * 8;
+    } else if (!std::strcmp(name, "kernel")) {
+        if (value < 0 || value > 3) return CKV_ERR_INVALID_ARG;
+        ctx->opt_kernel = value;
+    } else if (!std::strcmp(name, "l2_persist")) {
+        ctx->opt_l2 = value != 0;
+    } else {
+        return CKV_ERR_INVALID_ARG;
+    }
+    return CKV_OK;
+}
+
+ckv_status ckv_get_option(ckv_ctx* ctx, const char* name, int64_t* value)
+{
+    if (!ctx || !name || !value) return CKV_ERR_INVALID_ARG;
+    if (!std::strcmp(name, "split_len")) *value = ctx->opt_split;
+    else if (!std::strcmp(name, "kernel")) *value = ctx->opt_kernel;
+    else if (!std::strcmp(name, "l2_persist")) *value = ctx->opt_l2;
+    else return CKV_ERR_INVALID_ARG;
+    return CKV_OK;
+}
+
+ckv_status ckv_last_stat(ckv_ctx* ctx, const char* name, int64_t* value)
+{
+    if (!ctx || !name || !value) return CKV_ERR_INVALID_ARG;
+    if (!std::strcmp(name, "launches")) *value = ctx->st_launches;
+    else if (!std::strcmp(name, "work_items")) *value = ctx->st_items;
+    else if (!std::strcmp(name, "split_items")) *value = ctx->st_split;
+    else if (!std::strcmp(name, "kernel")) *value = ctx->st_kernel;
+    else if (!std::strcmp(name, "workspace_bytes")) *value = ctx->st_ws;
+    else if (!std::strcmp(name, "plan_cache_hit")) *value = ctx->st_hit;
+    else return CKV_ERR_INVALID_ARG;
+    return CKV_OK;
+}
+
+const char* ckv_strerror(ckv_status s)
+{
+    switch (s) {
+        case CKV_OK: return "ok";
+        case CKV_ERR_INVALID_ARG: return "invalid argument";
+        case CKV_ERR_SHAPE: return "shape mismatch";
+        case CKV_ERR_STATE: return "no pool loaded";
+        case CKV_ERR_INDEX_RANGE: return "pool index out of range";
+        case CKV_ERR_UNKNOWN_USER: return "unknown user";
+        case CKV_ERR_OOM: return "out of memory";
+        case CKV_ERR_CUDA: return "CUDA error";
+        case CKV_ERR_UNSUPPORTED: return "unsupported configuration";
+    }
+    return "unknown status";
+}
+
+const char* ckv_last_cuda_error(ckv_ctx* ctx) { return ctx ? ctx->cuda_err.c_str() : ""; }
+
+int32_t ckv_version(void) { return 100; }
+
+}  // extern "C"

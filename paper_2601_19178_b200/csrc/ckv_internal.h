@@ -1,0 +1,77 @@
+// Internal declarations shared by the host side of the library and its kernels.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "ckv.h"
+
+namespace ckv {
+
+// One request row of an attend plan: where the user's compressed history lives in the
+// arena and which query rows belong to it.
+struct Req {
+    int64_t base;      // first arena unit of the user; unit(g, i) = base + g * Lpad + i
+    int32_t L;         // history length
+    int32_t Lpad;      // L rounded up to a multiple of 8
+    int32_t q0;        // first query row
+    int32_t M;         // number of query rows
+    int32_t part0;     // first partial-result row block (split requests), else -1
+    int32_t n_chunks;  // history chunks this request was cut into (>= 1)
+};
+
+// One unit of kernel work: a contiguous chunk of one request's history, for every group.
+struct Item {
+    int32_t req;
+    int32_t begin;     // first position of the chunk
+    int32_t len;       // positions in the chunk (0 only for an empty history)
+    int32_t part_row;  // first row of this chunk's partial results, or -1: write `out`
+};
+
+// Everything a kernel needs to find the compressed cache and the pool.
+struct CacheView {
+    const void* poolK;   // [G][m][D] rows, first d_user slots zero
+    const void* poolV;
+    const void* idxK;    // arena, idx_bytes per unit
+    const void* idxV;
+    const void* userK;   // arena, d_user elements per unit
+    const void* userV;
+    int32_t n_groups;
+    int32_t n_entries;
+    int32_t d_user;
+    int32_t idx_bytes;   // 2 or 4
+};
+
+struct AttendArgs {
+    CacheView cv;
+    const Req* reqs;
+    const Item* items;
+    int32_t n_items;
+    const void* queries;   // [Q][G][D]
+    void* out;             // [Q][G][D]
+    float* partials;       // [part rows][G][D + 2]  (m, l, acc[D])
+    int32_t out_dtype;     // ckv_dtype
+    int32_t mode;          // ckv_mode
+    float scale;
+};
+
+// ---- kernels_pack.cu
+cudaError_t launch_pool_layout(int dtype, int G, int m, int d_shared, int D, const void* src,
+                               void* dst, cudaStream_t s);
+// Packs n users' [P][G] indices and [P][G][d_user] user parts into arena units and
+// validates index range; *bad_flag (device int) is OR-ed with 1 on a bad index.
+cudaError_t launch_pack(int dtype, int G, int n_entries, int d_user, int idx_bytes, int n_users,
+                        const int64_t* hist_off_dev, const int64_t* unit_off_dev,
+                        int64_t total_units, int64_t arena_base, const int32_t* idxK,
+                        const int32_t* idxV, const void* userK, const void* userV, void* a_idxK,
+                        void* a_idxV, void* a_userK, void* a_userV, int* bad_flag, cudaStream_t s);
+cudaError_t launch_materialize(int dtype, int D, const CacheView& cv, int64_t base, int L, int Lpad,
+                               void* K_out, void* V_out, cudaStream_t s);
+
+// ---- kernels_simt.cu : CUDA-core family (any number of queries, best for few)
+cudaError_t launch_attend_simt(int dtype, int D, int max_M, const AttendArgs& a, cudaStream_t s);
+// Merges the partial results of split requests into `out`.
+cudaError_t launch_combine(int D, const AttendArgs& a, const int32_t* split_reqs, int n_split,
+                           cudaStream_t s);
+
+}  // namespace ckv

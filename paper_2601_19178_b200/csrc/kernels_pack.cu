@@ -1,0 +1,165 @@
+// Data-movement kernels: pool row layout, compressed-cache packing with index
+// validation, and the test-only full-width materialisation (Eq. Kc + Eq. K).
+// All of them copy bits; none does arithmetic on values.
+#include "ckv_internal.h"
+
+namespace ckv {
+namespace {
+
+// dst[g][j][c] = c < d_user ? 0 : src[g][j][c - d_user]      (rows padded to the head width)
+template <typename E>
+__global__ void pool_layout_kernel(const E* __restrict__ src, E* __restrict__ dst, int64_t rows,
+                                   int d_shared, int D)
+{
+    const int d_user = D - d_shared;
+    const int64_t total = rows * D;
+    for (int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; t < total;
+         t += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = t / D;
+        const int c = (int)(t - r * D);
+        dst[t] = c < d_user ? E(0) : src[r * d_shared + (c - d_user)];
+    }
+}
+
+// One thread per arena unit of the batch.  unit_off[u] = sum over earlier users of
+// G * Lpad; the unit of (user u, group g, position i) is unit_off[u] + g * Lpad_u + i.
+template <typename E, typename I>
+__global__ void pack_kernel(int G, int n_entries, int d_user, int n_users,
+                            const int64_t* __restrict__ hist_off,
+                            const int64_t* __restrict__ unit_off, int64_t total_units,
+                            int64_t arena_base, const int32_t* __restrict__ idxK,
+                            const int32_t* __restrict__ idxV, const E* __restrict__ userK,
+                            const E* __restrict__ userV, I* __restrict__ a_idxK,
+                            I* __restrict__ a_idxV, E* __restrict__ a_userK,
+                            E* __restrict__ a_userV, int* __restrict__ bad_flag)
+{
+    for (int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; t < total_units;
+         t += (int64_t)gridDim.x * blockDim.x) {
+        int lo = 0, hi = n_users;  // last u with unit_off[u] <= t
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (unit_off[mid] <= t) lo = mid; else hi = mid;
+        }
+        const int u = lo;
+        const int64_t local = t - unit_off[u];
+        const int64_t Lpad = (unit_off[u + 1] - unit_off[u]) / G;
+        const int g = (int)(local / Lpad);
+        const int64_t i = local - g * Lpad;
+        const int64_t L = hist_off[u + 1] - hist_off[u];
+        const int64_t dst = arena_base + t;
+        int32_t ik = 0, iv = 0;
+        if (i < L) {
+            const int64_t src = (hist_off[u] + i) * G + g;
+            ik = idxK[src];
+            iv = idxV[src];
+            if (ik < 0 || ik >= n_entries || iv < 0 || iv >= n_entries) {
+                atomicOr(bad_flag, 1);
+                ik = iv = 0;
+            }
+            for (int c = 0; c < d_user; ++c) {
+                a_userK[dst * d_user + c] = userK[src * d_user + c];
+                a_userV[dst * d_user + c] = userV[src * d_user + c];
+            }
+        } else {  // padding: a valid row index and a zero user part
+            for (int c = 0; c < d_user; ++c) {
+                a_userK[dst * d_user + c] = E(0);
+                a_userV[dst * d_user + c] = E(0);
+            }
+        }
+        a_idxK[dst] = (I)ik;
+        a_idxV[dst] = (I)iv;
+    }
+}
+
+template <typename E, typename I>
+__global__ void materialize_kernel(int G, int n_entries, int d_user, int D,
+                                   const E* __restrict__ poolK, const E* __restrict__ poolV,
+                                   const I* __restrict__ idxK, const I* __restrict__ idxV,
+                                   const E* __restrict__ userK, const E* __restrict__ userV,
+                                   int64_t base, int L, int Lpad, E* __restrict__ K_out,
+                                   E* __restrict__ V_out)
+{
+    const int64_t total = (int64_t)L * G * D;
+    for (int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; t < total;
+         t += (int64_t)gridDim.x * blockDim.x) {
+        const int c = (int)(t % D);
+        const int64_t ig = t / D;
+        const int g = (int)(ig % G);
+        const int64_t i = ig / G;
+        const int64_t unit = base + (int64_t)g * Lpad + i;
+        if (c < d_user) {
+            K_out[t] = userK[unit * d_user + c];
+            V_out[t] = userV[unit * d_user + c];
+        } else {
+            K_out[t] = poolK[((int64_t)g * n_entries + (int64_t)idxK[unit]) * D + c];
+            V_out[t] = poolV[((int64_t)g * n_entries + (int64_t)idxV[unit]) * D + c];
+        }
+    }
+}
+
+inline int grid_for(int64_t total, int block)
+{
+    int64_t g = (total + block - 1) / block;
+    if (g < 1) g = 1;
+    if (g > 148 * 32) g = 148 * 32;
+    return (int)g;
+}
+
+}  // namespace
+
+cudaError_t launch_pool_layout(int dtype, int G, int m, int d_shared, int D, const void* src,
+                               void* dst, cudaStream_t s)
+{
+    const int64_t rows = (int64_t)G * m;
+    const int grid = grid_for(rows * D, 256);
+    if (dtype == CKV_BF16)
+        pool_layout_kernel<uint16_t><<<grid, 256, 0, s>>>((const uint16_t*)src, (uint16_t*)dst, rows,
+                                                          d_shared, D);
+    else
+        pool_layout_kernel<uint32_t><<<grid, 256, 0, s>>>((const uint32_t*)src, (uint32_t*)dst, rows,
+                                                          d_shared, D);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_pack(int dtype, int G, int n_entries, int d_user, int idx_bytes, int n_users,
+                        const int64_t* hist_off_dev, const int64_t* unit_off_dev,
+                        int64_t total_units, int64_t arena_base, const int32_t* idxK,
+                        const int32_t* idxV, const void* userK, const void* userV, void* a_idxK,
+                        void* a_idxV, void* a_userK, void* a_userV, int* bad_flag, cudaStream_t s)
+{
+    if (total_units == 0) return cudaSuccess;
+    const int grid = grid_for(total_units, 256);
+#define CKV_PACK(E, I)                                                                          \
+    pack_kernel<E, I><<<grid, 256, 0, s>>>(G, n_entries, d_user, n_users, hist_off_dev,          \
+                                           unit_off_dev, total_units, arena_base, idxK, idxV,    \
+                                           (const E*)userK, (const E*)userV, (I*)a_idxK,         \
+                                           (I*)a_idxV, (E*)a_userK, (E*)a_userV, bad_flag)
+    if (dtype == CKV_BF16) {
+        if (idx_bytes == 2) CKV_PACK(uint16_t, uint16_t); else CKV_PACK(uint16_t, int32_t);
+    } else {
+        if (idx_bytes == 2) CKV_PACK(uint32_t, uint16_t); else CKV_PACK(uint32_t, int32_t);
+    }
+#undef CKV_PACK
+    return cudaGetLastError();
+}
+
+cudaError_t launch_materialize(int dtype, int D, const CacheView& cv, int64_t base, int L, int Lpad,
+                               void* K_out, void* V_out, cudaStream_t s)
+{
+    if (L == 0) return cudaSuccess;
+    const int grid = grid_for((int64_t)L * cv.n_groups * D, 256);
+#define CKV_MAT(E, I)                                                                            \
+    materialize_kernel<E, I><<<grid, 256, 0, s>>>(                                               \
+        cv.n_groups, cv.n_entries, cv.d_user, D, (const E*)cv.poolK, (const E*)cv.poolV,         \
+        (const I*)cv.idxK, (const I*)cv.idxV, (const E*)cv.userK, (const E*)cv.userV, base, L,   \
+        Lpad, (E*)K_out, (E*)V_out)
+    if (dtype == CKV_BF16) {
+        if (cv.idx_bytes == 2) CKV_MAT(uint16_t, uint16_t); else CKV_MAT(uint16_t, int32_t);
+    } else {
+        if (cv.idx_bytes == 2) CKV_MAT(uint32_t, uint16_t); else CKV_MAT(uint32_t, int32_t);
+    }
+#undef CKV_MAT
+    return cudaGetLastError();
+}
+
+}  // namespace ckv

@@ -1,0 +1,68 @@
+"""A small convenience wrapper over the C-ABI calls for torch users: owns the context
+handle and converts between torch dtypes and the library's enums.  No arithmetic here."""
+from __future__ import annotations
+
+from typing import Optional
+
+import numpy as np
+import torch
+
+from . import binding as B
+
+_DT = {torch.float32: B.CKV_F32, torch.bfloat16: B.CKV_BF16}
+_MODE = {"softmax": B.CKV_SOFTMAX, "silu_over_l": B.CKV_SILU_OVER_L}
+
+
+def as_device_tensor(a: np.ndarray, dtype: str, device="cuda") -> torch.Tensor:
+    """numpy array (float32, or uint16 bf16 bit patterns, or integers) -> device tensor."""
+    if dtype == "bf16" and a.dtype == np.uint16:
+        return torch.from_numpy(a.view(np.int16)).to(device).view(torch.bfloat16)
+    return torch.from_numpy(a).to(device)
+
+
+class CollectiveKV:
+    def __init__(self, n_groups: int, head_dim: int, dtype: torch.dtype, mode: str = "softmax",
+                 scale: float = 0.0, out_dtype: Optional[torch.dtype] = None, device: int = 0):
+        self.n_groups, self.head_dim, self.dtype = n_groups, head_dim, dtype
+        self.out_dtype = out_dtype or dtype
+        self.device = torch.device("cuda", device)
+        self.d_user = None
+        self.ctx = B.ckv_create(n_groups, head_dim, _DT[dtype], _MODE[mode], scale, _DT[self.out_dtype], device)
+
+    def close(self):
+        if self.ctx:
+            B.ckv_destroy(self.ctx)
+            self.ctx = None
+
+    __del__ = close
+
+    def pool_load(self, pool_K: torch.Tensor, pool_V: torch.Tensor):
+        G, m, dg = pool_K.shape
+        assert G == self.n_groups and pool_V.shape == pool_K.shape and pool_K.dtype == self.dtype
+        B.ckv_pool_load(self.ctx, pool_K, pool_V, m, dg)
+        self.d_user = self.head_dim - dg
+
+    def cache_put(self, user: int, idx_K, idx_V, user_K, user_V):
+        B.ckv_cache_put(self.ctx, user, idx_K.shape[0], idx_K, idx_V, user_K, user_V, self.d_user)
+
+    def cache_put_batch(self, users, hist_off, idx_K, idx_V, user_K, user_V):
+        B.ckv_cache_put_batch(self.ctx, users, hist_off, idx_K, idx_V, user_K, user_V, self.d_user)
+
+    def attend(self, users, q_off, queries: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        if out is None:
+            out = torch.empty(queries.shape, dtype=self.out_dtype, device=queries.device)
+        B.ckv_attend(self.ctx, users, q_off, queries, out)
+        return out
+
+    def materialize(self, user: int):
+        L = B.ckv_user_length(self.ctx, user)
+        K = torch.empty((L, self.n_groups, self.head_dim), dtype=self.dtype, device=self.device)
+        V = torch.empty_like(K)
+        B.ckv_materialize(self.ctx, user, K, V)
+        return K, V
+
+    def set_option(self, name: str, value: int):
+        B.ckv_set_option(self.ctx, name, value)
+
+    def stat(self, name: str) -> int:
+        return B.ckv_last_stat(self.ctx, name)

@@ -1,0 +1,187 @@
+"""CUDA path vs CPU oracle, through the C ABI, on seeded synthetic inputs."""
+import numpy as np
+import pytest
+import torch
+
+import synth
+from ckv_testlib import assert_close, gpu_attend, make_session, oracle_attend, to_dev
+from oracle import ckv_oracle as O
+
+pytestmark = pytest.mark.gpu
+
+W = synth.WORKLOADS
+
+# scaled-down copies of the five benchmark workloads: several tiles and a ragged tail each
+SMALL = {
+    "cfg1": synth.scaled(W["cfg1"], n_users=64),                                        # full size
+    "cfg2": synth.scaled(W["cfg2"], n_users=6, hist_len=(1024, 1024)),
+    "cfg2_ragged": synth.scaled(W["cfg2"], n_users=9, hist_len=(1, 700), n_queries=37),
+    "cfg3": synth.scaled(W["cfg3"], n_users=3, hist_len=(1100, 1100)),
+    "cfg3_ragged": synth.scaled(W["cfg3"], n_users=7, hist_len=(3, 333), n_queries=50),
+    "cfg4": synth.scaled(W["cfg4"], n_users=12, hist_len=(1000, 9000)),
+    "cfg5": synth.scaled(W["cfg5"], n_users=300, hist_len=(512, 512)),
+    "cfg5_ragged": synth.scaled(W["cfg5"], n_users=80, hist_len=(1, 130)),
+}
+
+
+@pytest.mark.parametrize("name", sorted(SMALL))
+def test_attend_matches_oracle(name):
+    w = SMALL[name]
+    d = synth.generate(w)
+    got = gpu_attend(w, d)
+    want = oracle_attend(w, d)
+    assert_close(got, want, w.dtype, name)
+
+
+@pytest.mark.parametrize("name", ["cfg1", "cfg2_ragged", "cfg4", "cfg5_ragged"])
+@pytest.mark.parametrize("scale_mul", [1.0, 4.0])
+def test_attend_sharper_softmax(name, scale_mul):
+    """The default logits are nearly flat (std ~0.2); a larger scale makes the softmax matter."""
+    w = synth.scaled(SMALL[name], n_users=min(SMALL[name].n_users, 8))
+    d = synth.generate(w)
+    scale = scale_mul * 4.0 / np.sqrt(w.head_dim)
+    assert_close(gpu_attend(w, d, scale=scale), oracle_attend(w, d, scale=scale), w.dtype, name)
+
+
+@pytest.mark.parametrize("name", ["cfg1", "cfg2_ragged", "cfg3_ragged", "cfg4"])
+def test_materialize_is_bit_exact(name):
+    w = synth.scaled(SMALL[name], n_users=min(SMALL[name].n_users, 5))
+    d = synth.generate(w)
+    s = make_session(w, d)
+    for u in range(w.n_users):
+        K, V = s.materialize(int(d["users"][u]))
+        p0, L = int(d["hist_off"][u]), int(d["hist_off"][u + 1] - d["hist_off"][u])
+        Ko, Vo = O.materialize(w.dtype, d["pool_K"], d["pool_V"], d["idx_K"], d["idx_V"], d["user_K"],
+                               d["user_V"], p0, L)
+        view = torch.int16 if w.dtype == "bf16" else torch.int32
+        npv = np.int16 if w.dtype == "bf16" else np.int32
+        assert np.array_equal(K.view(view).cpu().numpy(), Ko.view(npv))
+        assert np.array_equal(V.view(view).cpu().numpy(), Vo.view(npv))
+    s.close()
+
+
+@pytest.mark.parametrize("mode", ["softmax", "silu_over_l"])
+@pytest.mark.parametrize("split_len", [8, 64, 1000, 100000])
+def test_split_count_does_not_change_the_result(mode, split_len):
+    w = synth.scaled(W["cfg4"], n_users=6, hist_len=(1, 1500), n_queries=3, mode=mode)
+    d = synth.generate(w)
+    want = oracle_attend(w, d)
+    s = make_session(w, d, split_len=split_len)
+    a = gpu_attend(w, d, session=s)
+    b = gpu_attend(w, d, session=s)
+    assert np.array_equal(a, b), "run-to-run bitwise reproducibility"
+    if split_len >= 100000:
+        assert s.stat("split_items") == 0
+    else:
+        assert s.stat("split_items") > 0
+    s.close()
+    assert_close(a, want, w.dtype, f"split_len={split_len}")
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("head", [(16, 0), (14, 2), (31, 1), (28, 4), (56, 8), (120, 8), (10, 22)])
+@pytest.mark.parametrize("mode", ["softmax", "silu_over_l"])
+def test_head_shapes(dtype, head, mode):
+    dg, du = head
+    w = synth.Workload("shape", 3, dg, du, 97, 5, (1, 90), 5, mode, dtype, None, 1.0 / (dg + du),
+                       1.0 / (dg + du), 77)
+    d = synth.generate(w)
+    assert_close(gpu_attend(w, d), oracle_attend(w, d), dtype, f"{head}")
+
+
+def test_degenerate_one_entry_pool_and_no_user_part():
+    w = synth.Workload("deg", 2, 32, 0, 1, 4, (1, 300), 2, "softmax", "bf16", None, 1 / 32, 1 / 32, 5)
+    d = synth.generate(w)
+    got = gpu_attend(w, d, out_dtype="f32")
+    pv = synth.bf16_bits_to_f32(d["pool_V"])[:, 0].astype(np.float64)
+    assert np.abs(got - pv[None]).max() <= 1e-6 * np.abs(pv).max() + 1e-7
+    assert_close(got, oracle_attend(w, d), "bf16")
+
+
+def test_wide_pool_uses_32_bit_indices():
+    w = synth.Workload("wide", 1, 30, 2, 70000, 3, (50, 400), 2, "softmax", "bf16", None, 1 / 32, 1 / 32, 6)
+    d = synth.generate(w)
+    d["idx_K"][0, 0] = 69999
+    d["idx_V"][1, 0] = 65536
+    assert_close(gpu_attend(w, d), oracle_attend(w, d), "bf16")
+
+
+def test_empty_history_empty_query_list_and_repeated_user():
+    w = synth.Workload("edge", 2, 30, 2, 64, 4, (40, 40), 3, "softmax", "bf16", None, 1 / 32, 1 / 32, 8)
+    d = synth.generate(w)
+    # user 1: empty history; request list: [u0, u1, u2 (no queries), u3, u0 again]
+    keep = np.r_[0:40, 80:160]
+    for k in ("idx_K", "idx_V", "user_K", "user_V"):
+        d[k] = np.ascontiguousarray(d[k][keep])
+    d["hist_off"] = np.array([0, 40, 40, 80, 120], dtype=np.int64)
+    s = make_session(w, d)
+    req_users = d["users"][[0, 1, 2, 3, 0]]
+    q_off = np.array([0, 3, 6, 6, 9, 12], dtype=np.int32)
+    q = d["queries"]
+    out = s.attend(req_users, q_off, to_dev(q, "bf16")).float().cpu().numpy().astype(np.float64)
+    s.close()
+    # oracle on the equivalent explicit layout
+    o_all = O.attend("bf16", "softmax", w.default_scale, d["pool_K"], d["pool_V"], d["hist_off"], d["idx_K"],
+                     d["idx_V"], d["user_K"], d["user_V"], np.array([0, 3, 6, 6, 9]), d["queries"][:9])
+    assert np.all(out[3:6] == 0.0)                       # empty history -> zero rows
+    assert_close(out[0:3], o_all[0:3], "bf16")
+    assert_close(out[6:9], o_all[6:9], "bf16")
+    # the repeated user sees queries 9..11: compare against the oracle fed with those rows
+    d2 = dict(d, queries=np.ascontiguousarray(d["queries"][9:12]))
+    o_rep = O.attend("bf16", "softmax", w.default_scale, d["pool_K"], d["pool_V"], d["hist_off"], d["idx_K"],
+                     d["idx_V"], d["user_K"], d["user_V"], np.array([0, 3, 3, 3, 3]), d2["queries"])
+    assert_close(out[9:12], o_rep, "bf16")
+
+
+def test_host_buffers_go_through_the_same_path():
+    w = SMALL["cfg5_ragged"]
+    d = synth.generate(w)
+    s = make_session(w, d)
+    dev = gpu_attend(w, d, session=s)
+    q_host = torch.from_numpy(d["queries"].view(np.int16)).view(torch.bfloat16).pin_memory()
+    o_host = torch.empty(q_host.shape, dtype=torch.bfloat16).pin_memory()
+    s.attend(d["users"], d["q_off"], q_host, o_host)
+    torch.cuda.synchronize()
+    s.close()
+    assert np.array_equal(o_host.float().numpy().astype(np.float64), dev)
+
+
+def test_permuting_a_history_keeps_the_output():
+    w = synth.scaled(W["cfg4"], n_users=1, hist_len=(777, 777), n_queries=2)
+    d = synth.generate(w)
+    a = gpu_attend(w, d, out_dtype="f32")
+    perm = np.random.default_rng(3).permutation(777)
+    d2 = dict(d)
+    for k in ("idx_K", "idx_V", "user_K", "user_V"):
+        d2[k] = np.ascontiguousarray(d[k][perm])
+    b = gpu_attend(w, d2, out_dtype="f32")
+    assert np.abs(a - b).max() <= 1e-5 * np.abs(a).max()
+
+
+def test_replacing_and_evicting_users():
+    import paper_2601_19178_b200 as ckv
+    w = synth.scaled(W["cfg1"], n_users=3, hist_len=(20, 60))
+    d = synth.generate(w)
+    s = make_session(w, d)
+    first = gpu_attend(w, d, session=s)
+    # replace user 1 by user 0's history: its output must now equal what user 0's history gives
+    p0, p1 = int(d["hist_off"][0]), int(d["hist_off"][1])
+    s.cache_put(int(d["users"][1]), to_dev(d["idx_K"][p0:p1], "i"), to_dev(d["idx_V"][p0:p1], "i"),
+                to_dev(d["user_K"][p0:p1], "f32"), to_dev(d["user_V"][p0:p1], "f32"))
+    d2 = dict(d)
+    sel = np.r_[p0:p1, p0:p1, int(d["hist_off"][2]):int(d["hist_off"][3])]
+    for k in ("idx_K", "idx_V", "user_K", "user_V"):
+        d2[k] = np.ascontiguousarray(d[k][sel])
+    L0, L2 = p1 - p0, int(d["hist_off"][3] - d["hist_off"][2])
+    d2["hist_off"] = np.array([0, L0, 2 * L0, 2 * L0 + L2], dtype=np.int64)
+    second = gpu_attend(w, d, session=s)
+    assert_close(second, oracle_attend(w, d2), "f32")
+    assert np.array_equal(first[0], second[0])
+    ckv.ckv_cache_evict(s.ctx, int(d["users"][2]))
+    with pytest.raises(ckv.CkvError) as e:
+        gpu_attend(w, d, session=s)
+    assert e.value.status == ckv.CKV_ERR_UNKNOWN_USER
+    comp, full = ckv.ckv_cache_bytes(s.ctx)
+    assert full == 2 * (2 * L0) * w.n_groups * w.head_dim * 4
+    assert comp == (2 * L0) * w.n_groups * (2 * 2 + 2 * w.d_user * 4)
+    s.close()

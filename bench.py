@@ -1,0 +1,354 @@
+#!/usr/bin/env python
+"""Benchmark of the CollectiveKV decode path (one `ckv_attend` over all users of a workload).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--impl ours|reference]
+
+Prints ONE JSON line.  A step = one pass of the whole hot path (compressed-cache read, pool
+gather, concat, scores, normalisation, weighted sum, split merge, store) over the workload,
+with pool and caches resident in HBM.  `value` is cached history positions per second over all
+ranks (device time, max over ranks); `e2e` is the same call fed with host buffers (query
+upload and output download inside the timed region).  Under torchrun each rank serves its own
+users (weak scaling, no collective on the data path).
+
+`--impl reference` times the CPU oracle, as it stands, on this machine's host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import synth  # noqa: E402
+
+METRIC = "cached_history_positions_per_sec"
+UNIT = "positions/s"
+HBM_FALLBACK_GBS = 6650.0
+# users of the workload the CPU oracle is timed on (about 10-30 s of host work)
+CPU_SAMPLE_USERS = {"cfg1": 64, "cfg2": 1024, "cfg3": 256, "cfg4": 512, "cfg5": 32768}
+
+
+def _peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return HBM_FALLBACK_GBS, "fallback"
+
+
+def _traffic(workload: str):
+    """DRAM bytes per launch of the dominant kernel from the committed ncu summary, if any."""
+    p = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    try:
+        return json.load(open(p)).get(workload)
+    except Exception:
+        return None
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons of one GPU through NVML while the bench runs."""
+
+    def __init__(self, uuid: str, period: float = 0.005):
+        super().__init__(daemon=True)
+        self.period, self.samples, self.reasons, self.max_mhz = period, [], set(), None
+        self._stop_evt, self._on = threading.Event(), threading.Event()
+        self.h = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + uuid).encode() if not uuid.startswith("GPU-") else uuid.encode())
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.h = None
+
+    def run(self):
+        if self.h is None:
+            return
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4): "sw_power_cap",
+        }
+        while not self._stop_evt.is_set():
+            if self._on.is_set():
+                try:
+                    self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                    r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                    for bit, name in names.items():
+                        if r & bit:
+                            self.reasons.add(name)
+                except Exception:
+                    pass
+            time.sleep(self.period)
+
+    def on(self):
+        self._on.set()
+
+    def off(self):
+        self._on.clear()
+
+    def finish(self):
+        self._stop_evt.set()
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def _oracle_rate(w, data, n_users: int, n_threads: int = 0):
+    """Times the CPU oracle on the first n_users users; returns (positions/s, seconds, cores)."""
+    from oracle import ckv_oracle as O
+    n_users = min(n_users, w.n_users)
+    sel = np.arange(n_users, dtype=np.int64)
+    t0 = time.perf_counter()
+    O.attend(w.dtype, w.mode, w.default_scale, data["pool_K"], data["pool_V"], data["hist_off"], data["idx_K"],
+             data["idx_V"], data["user_K"], data["user_V"], data["q_off"], data["queries"], sel=sel,
+             n_threads=n_threads)
+    dt = time.perf_counter() - t0
+    pos = int(data["hist_off"][n_users])
+    return pos / dt, dt, O.max_threads(), n_users, pos
+
+
+def run_reference(args, w):
+    """The oracle, as it stands, on the host cores: each step is a bounded sample of users."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    data = synth.generate(w)
+    # size the per-step sample from a short probe so the whole run stays within ~2 minutes
+    probe_users = max(1, min(w.n_users, 8))
+    _, probe_dt, cores, _, _ = _oracle_rate(w, data, probe_users)
+    per_user = probe_dt / probe_users
+    budget = 100.0 / max(1, args.steps + args.warmup)
+    n_users = int(max(1, min(w.n_users, budget / max(per_user, 1e-9))))
+    for _ in range(args.warmup):
+        _oracle_rate(w, data, n_users)
+    times, pos = [], 0
+    for _ in range(args.steps):
+        _, dt, cores, _, pos = _oracle_rate(w, data, n_users)
+        times.append(dt)
+    total = sum(times)
+    value = pos * args.steps / total
+    sample = f"first {n_users} of {w.n_users} users ({pos} positions) per step"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": w.name, "describe": w.describe, "sample": sample},
+        "users_per_sec": n_users * args.steps / total,
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(args, w):
+    import torch
+    import paper_2601_19178_b200 as ckv
+    from paper_2601_19178_b200.session import as_device_tensor as dev
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    # weak scaling: every rank serves its own users of the same workload shape
+    data = synth.generate(w, seed=w.seed + 1000 * rank)
+    tdt = torch.float32 if w.dtype == "f32" else torch.bfloat16
+    s = ckv.CollectiveKV(w.n_groups, w.head_dim, tdt, w.mode, device=local)
+    s.pool_load(dev(data["pool_K"], w.dtype), dev(data["pool_V"], w.dtype))
+    ik, iv = dev(data["idx_K"], "i"), dev(data["idx_V"], "i")
+    uk, uv = dev(data["user_K"], w.dtype), dev(data["user_V"], w.dtype)
+    s.cache_put_batch(data["users"], data["hist_off"], ik, iv, uk, uv)
+    del ik, iv, uk, uv
+    torch.cuda.empty_cache()
+    if args.kernel:
+        s.set_option("kernel", args.kernel)
+    if args.split_len:
+        s.set_option("split_len", args.split_len)
+    s.set_option("time_kernels", 1)
+    users, q_off = data["users"], data["q_off"]
+    q = dev(data["queries"], w.dtype)
+    out = torch.empty_like(q)
+    positions = int(data["hist_off"][-1])
+    comp_bytes, full_bytes = ckv.ckv_cache_bytes(s.ctx)
+    qo_bytes = q.numel() * q.element_size() + out.numel() * out.element_size()
+    algo_bytes = comp_bytes + qo_bytes
+
+    # L2 flush between timed iterations: overwrite a buffer twice the size of L2
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def step():
+        s.attend(users, q_off, q, out)
+
+    for _ in range(max(args.warmup, 3)):
+        flush.zero_()
+        step()
+    torch.cuda.synchronize()
+
+    # parity spot check on sampled users, in the launch configuration that is timed
+    parity = None
+    if rank == 0 and not args.no_check:
+        from oracle import ckv_oracle as O
+        rng = np.random.default_rng(0)
+        lens = np.diff(data["hist_off"])
+        sel = sorted(set([0, w.n_users - 1, int(np.argmax(lens)), int(np.argmin(lens))] +
+                         rng.integers(0, w.n_users, size=4).tolist()))
+        want = O.attend(w.dtype, w.mode, w.default_scale, data["pool_K"], data["pool_V"], data["hist_off"],
+                        data["idx_K"], data["idx_V"], data["user_K"], data["user_V"], data["q_off"],
+                        data["queries"], sel=sel)
+        rows = np.concatenate([np.arange(q_off[u], q_off[u + 1]) for u in sel])
+        got = out[torch.from_numpy(rows).cuda()].float().cpu().numpy().astype(np.float64)
+        atol, rtol = (1e-5, 1e-5) if w.dtype == "f32" else (2e-3, 1e-2)
+        err = np.abs(got - want)
+        ok = bool((err <= atol + rtol * np.abs(want)).all())
+        rown = float((err.max(axis=-1) / np.maximum(np.abs(want).max(axis=-1), 1e-30)).max())
+        parity = {"users_checked": len(sel), "ok": ok, "max_abs_err": float(err.max()), "row_norm_err": rown}
+
+    sampler = None
+    if rank == 0:
+        try:
+            sampler = ClockSampler(str(torch.cuda.get_device_properties(local).uuid))
+            sampler.start()
+        except Exception:
+            sampler = None
+
+    ev0 = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    ev1 = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    kern_ns, comb_ns, launches = [], [], 0
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    if sampler:
+        sampler.on()
+    for i in range(args.steps):
+        flush.zero_()
+        ev0[i].record(stream)
+        step()
+        ev1[i].record(stream)
+        launches += s.stat("launches")
+        if i % 8 == 7 or i == args.steps - 1:   # keep the queue shallow; read the library's own events
+            kern_ns.append(s.stat("main_kernel_ns"))
+            comb_ns.append(s.stat("combine_kernel_ns"))
+    torch.cuda.synchronize()
+    if sampler:
+        sampler.off()
+    if dist is not None:
+        dist.barrier()
+    step_ms = [a.elapsed_time(b) for a, b in zip(ev0, ev1)]
+    total_ms = float(sum(step_ms))
+    if dist is not None:
+        t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+
+    # end to end: host query buffer in, host output buffer out, through the same C-ABI call
+    q_host = torch.empty(q.shape, dtype=q.dtype).pin_memory()
+    q_host.copy_(q)
+    o_host = torch.empty(out.shape, dtype=out.dtype).pin_memory()
+    e2e_steps = max(3, min(args.steps, 20))
+    for _ in range(2):
+        s.attend(users, q_off, q_host, o_host)
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        s.attend(users, q_off, q_host, o_host)
+        torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+    if dist is not None:
+        t = torch.tensor([e2e_s], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    clocks = sampler.finish() if sampler else None
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = _peaks()
+    kern_s = statistics.mean(kern_ns) * 1e-9
+    achieved = algo_bytes / kern_s / 1e9
+    value = positions * world * args.steps / (total_ms * 1e-3)
+    cpu = None
+    if not args.no_cpu:
+        rate, dt, cores, n_u, pos = _oracle_rate(w, data, CPU_SAMPLE_USERS.get(w.name, w.n_users))
+        cpu = {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle",
+               "sample": f"first {n_u} of {w.n_users} users ({pos} positions), {dt:.1f} s"}
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32" if w.dtype == "f32" else "bf16_f32acc",
+        "data": "synthetic",
+        "config": {"workload": w.name, "describe": w.describe, "users": w.n_users, "positions": positions,
+                   "l2": "flushed between timed steps (256 MiB overwrite)",
+                   "kernel_family": s.stat("kernel"), "work_items": s.stat("work_items"),
+                   "split_items": s.stat("split_items")},
+        "users_per_sec": w.n_users * world * args.steps / (total_ms * 1e-3),
+        "clocks": clocks,
+        "e2e": {"value": positions * world * e2e_steps / e2e_s, "unit": UNIT,
+                "h2d_bytes_per_step": q_host.numel() * q_host.element_size() + users.nbytes + q_off.nbytes,
+                "d2h_bytes_per_step": o_host.numel() * o_host.element_size(), "ms_per_step": 1e3 * e2e_s / e2e_steps},
+        "gpu_launches": launches,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": _traffic(w.name), "peak_kind": peak_kind, "algorithmic_bytes": algo_bytes,
+                     "kernel_us": kern_s * 1e6, "combine_us": statistics.mean(comb_ns) * 1e-3,
+                     "frac_of_nominal_8TBs": achieved / 8000.0},
+        "cpu_baseline": cpu,
+        "parity": parity,
+        "compression": {"compressed_bytes": comp_bytes, "full_width_bytes": full_bytes,
+                        "ratio": comp_bytes / max(full_bytes, 1)},
+    }
+    print(json.dumps(line), flush=True)
+    s.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="cfg2", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--users", type=int, default=0, help="override the user count (smaller captures)")
+    ap.add_argument("--kernel", type=int, default=0)
+    ap.add_argument("--split-len", type=int, default=0)
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
+    ap.add_argument("--no-check", action="store_true", help="skip the sampled parity check")
+    args = ap.parse_args()
+    w = synth.WORKLOADS[args.workload]
+    if args.users:
+        w = synth.scaled(w, n_users=args.users)
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

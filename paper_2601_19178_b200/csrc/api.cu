@@ -78,7 +78,9 @@ struct ckv_ctx {
     std::vector<Plan> plans;
     uint64_t tick = 0;
     // options
-    int64_t opt_split = 0, opt_kernel = 0, opt_l2 = 1;
+    int64_t opt_split = 0, opt_kernel = 0, opt_l2 = 1, opt_time = 0;
+    cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};  // around the main kernel and the combine
+    bool ev_valid = false;
     // statistics of the last attend
     int64_t st_launches = 0, st_items = 0, st_split = 0, st_kernel = 0, st_ws = 0, st_hit = 0;
     std::string cuda_err;
@@ -397,6 +399,8 @@ ckv_status ckv_destroy(ckv_ctx* ctx)
                     ctx->d_flag,  ctx->stage_q.p,  ctx->stage_out.p, ctx->partials.p};
     for (void* b : bufs)
         if (b) cudaFree(b);
+    for (auto& e : ctx->ev)
+        if (e) cudaEventDestroy(e);
     cudaGetLastError();
     delete ctx;
     return CKV_OK;
@@ -576,13 +580,24 @@ ckv_status ckv_attend(ckv_ctx* ctx, int32_t n, const int64_t* users, const int32
     a.out_dtype = ctx->cfg.out_dtype;
     a.mode = ctx->cfg.mode;
     a.scale = ctx->scale;
+    ctx->ev_valid = false;
+    if (ctx->opt_time) {
+        for (auto& e : ctx->ev)
+            if (!e) CK(cudaEventCreate(&e));
+        CK(cudaEventRecord(ctx->ev[0], s));
+    }
     if (pl->n_items > 0) {
         CK(launch_attend_simt(ctx->cfg.dtype, D, pl->max_M, a, s));
         ctx->st_launches++;
     }
+    if (ctx->opt_time) CK(cudaEventRecord(ctx->ev[1], s));
     if (pl->n_split > 0) {
         CK(launch_combine(D, a, pl->d_split, pl->n_split, s));
         ctx->st_launches++;
+    }
+    if (ctx->opt_time) {
+        CK(cudaEventRecord(ctx->ev[2], s));
+        ctx->ev_valid = true;
     }
     if (o_host) CK(cudaMemcpyAsync(out, d_out, o_bytes, cudaMemcpyDeviceToHost, s));
     return CKV_OK;
@@ -653,6 +668,8 @@ ckv_status ckv_set_option(ckv_ctx* ctx, const char* name, int64_t value)
         ctx->opt_kernel = value;
     } else if (!std::strcmp(name, "l2_persist")) {
         ctx->opt_l2 = value != 0;
+    } else if (!std::strcmp(name, "time_kernels")) {
+        ctx->opt_time = value != 0;
     } else {
         return CKV_ERR_INVALID_ARG;
     }
@@ -665,6 +682,7 @@ ckv_status ckv_get_option(ckv_ctx* ctx, const char* name, int64_t* value)
     if (!std::strcmp(name, "split_len")) *value = ctx->opt_split;
     else if (!std::strcmp(name, "kernel")) *value = ctx->opt_kernel;
     else if (!std::strcmp(name, "l2_persist")) *value = ctx->opt_l2;
+    else if (!std::strcmp(name, "time_kernels")) *value = ctx->opt_time;
     else return CKV_ERR_INVALID_ARG;
     return CKV_OK;
 }
@@ -678,6 +696,15 @@ ckv_status ckv_last_stat(ckv_ctx* ctx, const char* name, int64_t* value)
     else if (!std::strcmp(name, "kernel")) *value = ctx->st_kernel;
     else if (!std::strcmp(name, "workspace_bytes")) *value = ctx->st_ws;
     else if (!std::strcmp(name, "plan_cache_hit")) *value = ctx->st_hit;
+    else if (!std::strcmp(name, "main_kernel_ns") || !std::strcmp(name, "combine_kernel_ns")) {
+        if (!ctx->ev_valid) return CKV_ERR_STATE;
+        DeviceGuard dg(ctx->cfg.device);
+        const bool main = name[0] == 'm';
+        float ms = 0.f;
+        CK(cudaEventSynchronize(ctx->ev[2]));
+        CK(cudaEventElapsedTime(&ms, ctx->ev[main ? 0 : 1], ctx->ev[main ? 1 : 2]));
+        *value = (int64_t)(ms * 1e6);
+    }
     else return CKV_ERR_INVALID_ARG;
     return CKV_OK;
 }

@@ -65,7 +65,8 @@ struct ckv_ctx {
     int elem = 2;  // bytes per element of cfg.dtype
     // pool
     int n_entries = 0, d_shared = 0, d_user = 0, idx_bytes = 0;
-    void* pool = nullptr;  // K rows then V rows, each [G][m][D]
+    void* pool = nullptr;  // K rows then V rows, each [G][m][D]; then the two MMA-ordered copies
+    bool has_mma_pool = false;
     size_t pool_half = 0;  // bytes of one of them
     // arena of compressed caches (units = (position, group) slots)
     void *a_idxK = nullptr, *a_idxV = nullptr, *a_userK = nullptr, *a_userV = nullptr;
@@ -220,12 +221,18 @@ ckv_status ensure_arena(ckv_ctx* ctx, int64_t need, cudaStream_t s)
     return CKV_OK;
 }
 
-int64_t auto_split_len(const ckv_ctx* ctx, int64_t total_positions, int family)
+int64_t auto_split_len(const ckv_ctx* ctx, int64_t total_positions, int family, int max_M)
 {
     // Enough (chunk, group) blocks to fill the SMs several times over, but chunks long
     // enough that the merge of partial results stays a small fraction of the work.
-    (void)family;
-    int64_t c = total_positions * ctx->cfg.n_groups / (kNumSMs * 16);
+    int64_t c;
+    if (family == 2) {
+        const int qpw = mma_queries_per_warp(max_M);
+        c = total_positions * ctx->cfg.n_groups * ((max_M + qpw - 1) / qpw) / (kNumSMs * 32);
+        c = (c + 63) / 64 * 64;
+        return std::min<int64_t>(std::max<int64_t>(c, 256), 4096);
+    }
+    c = total_positions * ctx->cfg.n_groups / (kNumSMs * 16);
     c = (c + 63) / 64 * 64;
     return std::min<int64_t>(std::max<int64_t>(c, 256), 2048);
 }
@@ -251,8 +258,12 @@ ckv_status build_plan(ckv_ctx* ctx, Plan& pl, int32_t n, const int64_t* users, c
         max_M = std::max(max_M, r.M);
     }
     pl.max_M = max_M;
-    pl.family = 1;
-    const int64_t C = ctx->opt_split > 0 ? ctx->opt_split : auto_split_len(ctx, total_pos, pl.family);
+    const bool can_mma = ctx->has_mma_pool;
+    if (ctx->opt_kernel == 0) pl.family = can_mma && max_M >= 9 ? 2 : 1;
+    else if (ctx->opt_kernel == 1) pl.family = 1;
+    else if (ctx->opt_kernel == 2 && can_mma) pl.family = 2;
+    else return CKV_ERR_UNSUPPORTED;
+    const int64_t C = ctx->opt_split > 0 ? ctx->opt_split : auto_split_len(ctx, total_pos, pl.family, max_M);
     std::vector<Item> items;
     std::vector<int32_t> split;
     items.reserve((size_t)n);
@@ -420,15 +431,20 @@ ckv_status ckv_pool_load(ckv_ctx* ctx, const void* pool_K, const void* pool_V, i
     Staged sk, sv;
     CK(sk.init(pool_K, src_bytes, s));
     CK(sv.init(pool_V, src_bytes, s));
-    if (!ctx->pool || half != ctx->pool_half) {
+    const bool mma = mma_supported(ctx->cfg.dtype, D, D - d_shared);
+    if (!ctx->pool || half != ctx->pool_half || mma != ctx->has_mma_pool) {
         void* np = nullptr;
-        CK(cudaMalloc(&np, 2 * half));
+        CK(cudaMalloc(&np, (mma ? 4 : 2) * half));
         if (ctx->pool) cudaFree(ctx->pool);
         ctx->pool = np;
         ctx->pool_half = half;
+        ctx->has_mma_pool = mma;
     }
     CK(launch_pool_layout(ctx->cfg.dtype, G, n_entries, d_shared, D, sk.dev, ctx->pool, s));
     CK(launch_pool_layout(ctx->cfg.dtype, G, n_entries, d_shared, D, sv.dev, (char*)ctx->pool + half, s));
+    if (mma)
+        CK(launch_pool_permute(G, n_entries, ctx->pool, (char*)ctx->pool + half, (char*)ctx->pool + 2 * half,
+                               (char*)ctx->pool + 3 * half, s));
     if (sk.owned || sv.owned) CK(cudaStreamSynchronize(s));
     if (ctx->users.empty() && (ctx->n_entries != n_entries || ctx->d_shared != d_shared)) {
         // index width or user width may change: restart the (empty) arena
@@ -459,8 +475,8 @@ ckv_status ckv_cache_put_batch(ckv_ctx* ctx, int32_t n, const int64_t* users, co
     unit_off[0] = 0;
     for (int32_t k = 0; k < n; ++k) {
         const int64_t L = hist_off[k + 1] - hist_off[k];
-        if (L < 0 || L > INT32_MAX - 8) return CKV_ERR_INVALID_ARG;
-        unit_off[k + 1] = unit_off[k] + (int64_t)G * ((L + 7) / 8 * 8);
+        if (L < 0 || L > INT32_MAX - 32) return CKV_ERR_INVALID_ARG;
+        unit_off[k + 1] = unit_off[k] + (int64_t)G * ((L + 31) / 32 * 32);
     }
     const int64_t P = hist_off[n], total_units = unit_off[n];
     if (P > 0 && (!idx_K || !idx_V || (d_user > 0 && (!user_K || !user_V)))) return CKV_ERR_INVALID_ARG;
@@ -492,7 +508,7 @@ ckv_status ckv_cache_put_batch(ckv_ctx* ctx, int32_t n, const int64_t* users, co
         const int64_t L = hist_off[k + 1] - hist_off[k];
         auto f = ctx->users.find(users[k]);
         if (f != ctx->users.end()) ctx->live_positions -= f->second.L;
-        ctx->users[users[k]] = UserEntry{ctx->used_units + unit_off[k], (int32_t)L, (int32_t)((L + 7) / 8 * 8)};
+        ctx->users[users[k]] = UserEntry{ctx->used_units + unit_off[k], (int32_t)L, (int32_t)((L + 31) / 32 * 32)};
         ctx->live_positions += L;
     }
     ctx->used_units += total_units;
@@ -587,7 +603,11 @@ ckv_status ckv_attend(ckv_ctx* ctx, int32_t n, const int64_t* users, const int32
         CK(cudaEventRecord(ctx->ev[0], s));
     }
     if (pl->n_items > 0) {
-        CK(launch_attend_simt(ctx->cfg.dtype, D, pl->max_M, a, s));
+        if (pl->family == 2)
+            CK(launch_attend_mma(pl->max_M, a, (const char*)ctx->pool + 2 * ctx->pool_half,
+                                 (const char*)ctx->pool + 3 * ctx->pool_half, s));
+        else
+            CK(launch_attend_simt(ctx->cfg.dtype, D, pl->max_M, a, s));
         ctx->st_launches++;
     }
     if (ctx->opt_time) CK(cudaEventRecord(ctx->ev[1], s));
@@ -662,7 +682,7 @@ ckv_status ckv_set_option(ckv_ctx* ctx, const char* name, int64_t value)
     if (!ctx || !name) return CKV_ERR_INVALID_ARG;
     if (!std::strcmp(name, "split_len")) {
         if (value < 0) return CKV_ERR_INVALID_ARG;
-        ctx->opt_split = value == 0 ? 0 : (value + 7) / 8 * 8;
+        ctx->opt_split = value == 0 ? 0 : (value + 63) / 64 * 64;
     } else if (!std::strcmp(name, "kernel")) {
         if (value < 0 || value > 3) return CKV_ERR_INVALID_ARG;
         ctx->opt_kernel = value;

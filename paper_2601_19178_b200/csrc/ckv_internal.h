@@ -13,7 +13,7 @@ namespace ckv {
 struct Req {
     int64_t base;      // first arena unit of the user; unit(g, i) = base + g * Lpad + i
     int32_t L;         // history length
-    int32_t Lpad;      // L rounded up to a multiple of 8
+    int32_t Lpad;      // L rounded up to a multiple of 32
     int32_t q0;        // first query row
     int32_t M;         // number of query rows
     int32_t part0;     // first partial-result row block (split requests), else -1
@@ -73,5 +73,14 @@ cudaError_t launch_attend_simt(int dtype, int D, int max_M, const AttendArgs& a,
 // Merges the partial results of split requests into `out`.
 cudaError_t launch_combine(int D, const AttendArgs& a, const int32_t* split_reqs, int n_split,
                            cudaStream_t s);
+
+// ---- kernels_mma.cu : warp-level tensor-core family (bf16, head_dim 32, d_user <= 8)
+bool mma_supported(int dtype, int head_dim, int d_user);
+int mma_queries_per_warp(int max_M);
+// Builds the two pool copies whose row-internal element order matches the MMA B fragments.
+cudaError_t launch_pool_permute(int G, int m, const void* poolK, const void* poolV, void* poolKp, void* poolVp,
+                                cudaStream_t s);
+cudaError_t launch_attend_mma(int max_M, const AttendArgs& a, const void* poolKp, const void* poolVp,
+                              cudaStream_t s);
 
 }  // namespace ckv

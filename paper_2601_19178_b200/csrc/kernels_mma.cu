@@ -1,0 +1,359 @@
+// Warp-level tensor-core gather-concat-attention kernel (bf16, head_dim 32) for a moderate
+// number of queries per user.
+//
+// One warp owns (work item, group, block of 16*MT queries) and walks the history chunk 32
+// positions at a time.  K and V rows never pass through shared memory: the pool is kept in
+// two extra copies whose element order inside a row matches the m16n8k16 B-operand register
+// layout, so that
+//   - for S = Q K^T a lane reads 16 contiguous bytes of "its" K row and has both k-steps'
+//     B fragments,
+//   - for O += P V a lane reads 8 contiguous bytes of four V rows and builds the B
+//     fragments with byte permutes.
+// Which history position sits in which MMA slot is free (attention does not depend on the
+// order of positions): slot (n-tile nt, column n) of a 32-block holds position 4n + nt, which
+// makes a lane's four K positions (4g..4g+3) and eight V positions (8t..8t+7) contiguous in
+// the compressed cache -- one 8-byte and one 16-byte index load per 32 positions.
+// The user-specific leading elements (Eq. K) are patched into the owning register.
+#include <cuda_bf16.h>
+#include <math_constants.h>
+
+#include "ckv_internal.h"
+
+namespace ckv {
+namespace {
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr int D = 32;
+constexpr int NTD = D / 8;   // n-tiles of the output
+constexpr int KS = D / 16;   // k-steps of Q K^T
+
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+{
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+        "{%0,%1,%2,%3};\n"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
+{
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+__device__ __forceinline__ float ex2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+__device__ __forceinline__ float tanh_fast(float x)
+{
+    float y;
+    asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+template <bool IDX16, int N>
+__device__ __forceinline__ void load_indices(const void* base, int64_t unit, int (&out)[N])
+{
+    if constexpr (IDX16) {
+        if constexpr (N == 4) {
+            const uint2 r = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const uint16_t*>(base) + unit));
+            out[0] = r.x & 0xffff; out[1] = r.x >> 16; out[2] = r.y & 0xffff; out[3] = r.y >> 16;
+        } else {
+            const uint4 r = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const uint16_t*>(base) + unit));
+            out[0] = r.x & 0xffff; out[1] = r.x >> 16; out[2] = r.y & 0xffff; out[3] = r.y >> 16;
+            out[4] = r.z & 0xffff; out[5] = r.z >> 16; out[6] = r.w & 0xffff; out[7] = r.w >> 16;
+        }
+    } else {
+        const int4* p = reinterpret_cast<const int4*>(reinterpret_cast<const int32_t*>(base) + unit);
+#pragma unroll
+        for (int i = 0; i < N / 4; ++i) {
+            const int4 r = __ldg(p + i);
+            out[4 * i] = r.x; out[4 * i + 1] = r.y; out[4 * i + 2] = r.z; out[4 * i + 3] = r.w;
+        }
+    }
+}
+
+template <int MT, int MODE, bool IDX16>
+__global__ void __launch_bounds__(128) attend_mma_kernel(const AttendArgs a, const void* poolKp,
+                                                         const void* poolVp, int n_mb)
+{
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = lane >> 2, t = lane & 3;
+    const int64_t wid = (int64_t)blockIdx.x * 4 + warp;
+    if (wid >= (int64_t)a.n_items * n_mb) return;
+    const Item it = a.items[wid / n_mb];
+    const int mb = (int)(wid % n_mb);
+    const Req rq = a.reqs[it.req];
+    const int row0 = mb * 16 * MT;
+    if (row0 >= rq.M) return;
+    const int grp = blockIdx.y, G = a.cv.n_groups, d_user = a.cv.d_user;
+
+    // Q as A fragments (row-major m16 x k16): rows g and g+8, columns 2t.. and 2t+8..
+    uint32_t qa[MT][KS][4];
+    const uint16_t* Q = reinterpret_cast<const uint16_t*>(a.queries);
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) {
+        const int r_lo = row0 + 16 * mt + g, r_hi = r_lo + 8;
+        const uint16_t* q_lo = Q + ((int64_t)(rq.q0 + r_lo) * G + grp) * D;
+        const uint16_t* q_hi = Q + ((int64_t)(rq.q0 + r_hi) * G + grp) * D;
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+            const int c = 16 * ks + 2 * t;
+            qa[mt][ks][0] = r_lo < rq.M ? __ldg(reinterpret_cast<const uint32_t*>(q_lo + c)) : 0u;
+            qa[mt][ks][1] = r_hi < rq.M ? __ldg(reinterpret_cast<const uint32_t*>(q_hi + c)) : 0u;
+            qa[mt][ks][2] = r_lo < rq.M ? __ldg(reinterpret_cast<const uint32_t*>(q_lo + c + 8)) : 0u;
+            qa[mt][ks][3] = r_hi < rq.M ? __ldg(reinterpret_cast<const uint32_t*>(q_hi + c + 8)) : 0u;
+        }
+    }
+
+    float o[MT][NTD][4];
+    float m_run[MT][2], l_run[MT][2];
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) {
+        m_run[mt][0] = m_run[mt][1] = -CUDART_INF_F;
+        l_run[mt][0] = l_run[mt][1] = 0.f;
+#pragma unroll
+        for (int j = 0; j < NTD; ++j)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) o[mt][j][e] = 0.f;
+    }
+
+    const char* pK = reinterpret_cast<const char*>(poolKp) + (int64_t)grp * a.cv.n_entries * (D * 2) + t * 16;
+    const char* pV = reinterpret_cast<const char*>(poolVp) + (int64_t)grp * a.cv.n_entries * (D * 2) + g * 8;
+    const int64_t unit0 = rq.base + (int64_t)grp * rq.Lpad;
+    const uint16_t* uK = reinterpret_cast<const uint16_t*>(a.cv.userK);
+    const uint16_t* uV = reinterpret_cast<const uint16_t*>(a.cv.userV);
+    const int end = it.begin + it.len;
+    const float sc = a.scale * (MODE == CKV_SOFTMAX ? kLog2e : 0.5f);
+    const bool patchK0 = 2 * t < d_user, patchK1 = 2 * t + 1 < d_user, patchV = g < d_user;
+
+    for (int p0 = it.begin; p0 < end; p0 += 32) {
+        int ik[4], iv[8];
+        const int64_t unitK = unit0 + p0 + 4 * g;   // this lane's four K positions
+        const int64_t unitV = unit0 + p0 + 8 * t;   // this lane's eight V positions
+        load_indices<IDX16, 4>(a.cv.idxK, unitK, ik);
+        load_indices<IDX16, 8>(a.cv.idxV, unitV, iv);
+        uint4 kf[4];
+        uint2 vr[8];
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) kf[nt] = __ldg(reinterpret_cast<const uint4*>(pK + (int64_t)ik[nt] * (D * 2)));
+#pragma unroll
+        for (int j = 0; j < 8; ++j) vr[j] = __ldg(reinterpret_cast<const uint2*>(pV + (int64_t)iv[j] * (D * 2)));
+        if (patchK0) {  // Eq. K: dims [0, d_user) come from the user-specific part
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt) {
+                const uint16_t* u = uK + (unitK + nt) * d_user + 2 * t;
+                uint32_t w = __ldg(u);
+                w |= patchK1 ? (uint32_t)__ldg(u + 1) << 16 : (kf[nt].x & 0xffff0000u);
+                kf[nt].x = w;
+            }
+        }
+        if (patchV) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                vr[j].x = (vr[j].x & 0xffff0000u) | (uint32_t)__ldg(uV + (unitV + j) * d_user + g);
+        }
+        // V B-fragments: k-slots (2t, 2t+1, 2t+8, 2t+9) of block b are positions
+        // 8t + (2b, 4+2b, 2b+1, 5+2b)
+        uint32_t vb[2][NTD][2];
+#pragma unroll
+        for (int b = 0; b < 2; ++b) {
+            vb[b][0][0] = __byte_perm(vr[2 * b].x, vr[4 + 2 * b].x, 0x5410);
+            vb[b][1][0] = __byte_perm(vr[2 * b].x, vr[4 + 2 * b].x, 0x7632);
+            vb[b][2][0] = __byte_perm(vr[2 * b].y, vr[4 + 2 * b].y, 0x5410);
+            vb[b][3][0] = __byte_perm(vr[2 * b].y, vr[4 + 2 * b].y, 0x7632);
+            vb[b][0][1] = __byte_perm(vr[2 * b + 1].x, vr[5 + 2 * b].x, 0x5410);
+            vb[b][1][1] = __byte_perm(vr[2 * b + 1].x, vr[5 + 2 * b].x, 0x7632);
+            vb[b][2][1] = __byte_perm(vr[2 * b + 1].y, vr[5 + 2 * b].y, 0x5410);
+            vb[b][3][1] = __byte_perm(vr[2 * b + 1].y, vr[5 + 2 * b].y, 0x7632);
+        }
+        const bool tail = p0 + 32 > end;
+
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+            float s[4][4];
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt) {
+                s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
+                mma_bf16(s[nt], qa[mt][0], kf[nt].x, kf[nt].y);
+                mma_bf16(s[nt], qa[mt][1], kf[nt].z, kf[nt].w);
+            }
+            // element (nt, e): column 2t + (e & 1) -> position p0 + 8t + 4 (e & 1) + nt
+            uint32_t pa[2][4];
+            if constexpr (MODE == CKV_SOFTMAX) {
+                if (tail) {
+#pragma unroll
+                    for (int nt = 0; nt < 4; ++nt) {
+                        if (p0 + 8 * t + nt >= end) s[nt][0] = s[nt][2] = -CUDART_INF_F;
+                        if (p0 + 8 * t + 4 + nt >= end) s[nt][1] = s[nt][3] = -CUDART_INF_F;
+                    }
+                }
+                float mx0 = s[0][0], mx1 = s[0][2];
+#pragma unroll
+                for (int nt = 0; nt < 4; ++nt) {
+                    mx0 = fmaxf(mx0, fmaxf(s[nt][0], s[nt][1]));
+                    mx1 = fmaxf(mx1, fmaxf(s[nt][2], s[nt][3]));
+                }
+                mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+                mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+                mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+                mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+                // the first position of a block is always valid, so mx is finite
+                const float mn0 = fmaxf(m_run[mt][0], mx0 * sc), mn1 = fmaxf(m_run[mt][1], mx1 * sc);
+                const float c0 = ex2(m_run[mt][0] - mn0), c1 = ex2(m_run[mt][1] - mn1);
+                m_run[mt][0] = mn0;
+                m_run[mt][1] = mn1;
+                float ps0 = 0.f, ps1 = 0.f;
+#pragma unroll
+                for (int nt = 0; nt < 4; ++nt) {
+                    const float p0v = ex2(fmaf(s[nt][0], sc, -mn0)), p1v = ex2(fmaf(s[nt][1], sc, -mn0));
+                    const float p2v = ex2(fmaf(s[nt][2], sc, -mn1)), p3v = ex2(fmaf(s[nt][3], sc, -mn1));
+                    ps0 += p0v + p1v;
+                    ps1 += p2v + p3v;
+                    pa[nt >> 1][(nt & 1) * 2] = pack_bf16(p0v, p1v);
+                    pa[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(p2v, p3v);
+                }
+                l_run[mt][0] = l_run[mt][0] * c0 + ps0;
+                l_run[mt][1] = l_run[mt][1] * c1 + ps1;
+#pragma unroll
+                for (int j = 0; j < NTD; ++j) {
+                    o[mt][j][0] *= c0; o[mt][j][1] *= c0;
+                    o[mt][j][2] *= c1; o[mt][j][3] *= c1;
+                }
+            } else {
+                // silu(x) = x sigmoid(x) = h (1 + tanh(h)), h = x / 2   (sc = scale / 2)
+#pragma unroll
+                for (int nt = 0; nt < 4; ++nt) {
+                    float w[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float h = s[nt][e] * sc;
+                        w[e] = fmaf(h, tanh_fast(h), h);
+                    }
+                    if (tail) {
+                        if (p0 + 8 * t + nt >= end) w[0] = w[2] = 0.f;
+                        if (p0 + 8 * t + 4 + nt >= end) w[1] = w[3] = 0.f;
+                    }
+                    pa[nt >> 1][(nt & 1) * 2] = pack_bf16(w[0], w[1]);
+                    pa[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(w[2], w[3]);
+                }
+            }
+#pragma unroll
+            for (int b = 0; b < 2; ++b)
+#pragma unroll
+                for (int j = 0; j < NTD; ++j) mma_bf16(o[mt][j], pa[b], vb[b][j][0], vb[b][j][1]);
+        }
+    }
+
+    // epilogue: finish the row sums over the quad, then store outputs or partials
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            float l = l_run[mt][h];
+            l += __shfl_xor_sync(0xffffffffu, l, 1);
+            l += __shfl_xor_sync(0xffffffffu, l, 2);
+            const int r = row0 + 16 * mt + g + 8 * h;
+            if (r >= rq.M) continue;
+            if (it.part_row < 0) {
+                float inv;
+                if constexpr (MODE == CKV_SOFTMAX) inv = l > 0.f ? 1.0f / l : 0.f;
+                else inv = rq.L > 0 ? 1.0f / (float)rq.L : 0.f;
+                const int64_t base = ((int64_t)(rq.q0 + r) * G + grp) * D;
+#pragma unroll
+                for (int j = 0; j < NTD; ++j) {
+                    const float x = o[mt][j][2 * h] * inv, y = o[mt][j][2 * h + 1] * inv;
+                    if (a.out_dtype == CKV_BF16)
+                        *reinterpret_cast<uint32_t*>(reinterpret_cast<uint16_t*>(a.out) + base + 8 * j + 2 * t) =
+                            pack_bf16(x, y);
+                    else
+                        *reinterpret_cast<float2*>(reinterpret_cast<float*>(a.out) + base + 8 * j + 2 * t) =
+                            make_float2(x, y);
+                }
+            } else {
+                float* pr = a.partials + ((int64_t)(it.part_row + r) * G + grp) * (D + 2);
+                if (t == 0) {
+                    pr[0] = m_run[mt][h];
+                    pr[1] = l;
+                }
+#pragma unroll
+                for (int j = 0; j < NTD; ++j)
+                    *reinterpret_cast<float2*>(pr + 2 + 8 * j + 2 * t) =
+                        make_float2(o[mt][j][2 * h], o[mt][j][2 * h + 1]);
+            }
+        }
+    }
+}
+
+// Row-internal element orders of the two extra pool copies (see the header comment).
+//   K copy: 16-byte chunk t holds, per k-step ks, elements 16ks + {2t, 2t+1, 2t+8, 2t+9}
+//   V copy:  8-byte chunk g holds elements g, g+8, g+16, g+24
+__global__ void pool_permute_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dstK,
+                                    uint16_t* __restrict__ dstV, const uint16_t* __restrict__ srcV, int64_t rows)
+{
+    const int64_t total = rows * D;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = i / D;
+        const int c = (int)(i - r * D);
+        const int ks = c >> 4, rem = c & 15, hi = rem >> 3, tt = (rem & 7) >> 1, lo = rem & 1;
+        dstK[r * D + tt * (D / 4) + ks * 4 + hi * 2 + lo] = src[i];
+        dstV[r * D + (c & 7) * NTD + (c >> 3)] = srcV[i];
+    }
+}
+
+template <int MT>
+cudaError_t launch_mt(const AttendArgs& a, const void* pKp, const void* pVp, int n_mb, cudaStream_t s)
+{
+    const int64_t warps = (int64_t)a.n_items * n_mb;
+    const dim3 grid((unsigned)((warps + 3) / 4), a.cv.n_groups);
+    const bool i16 = a.cv.idx_bytes == 2;
+    if (a.mode == CKV_SOFTMAX) {
+        if (i16) attend_mma_kernel<MT, CKV_SOFTMAX, true><<<grid, 128, 0, s>>>(a, pKp, pVp, n_mb);
+        else attend_mma_kernel<MT, CKV_SOFTMAX, false><<<grid, 128, 0, s>>>(a, pKp, pVp, n_mb);
+    } else {
+        if (i16) attend_mma_kernel<MT, CKV_SILU_OVER_L, true><<<grid, 128, 0, s>>>(a, pKp, pVp, n_mb);
+        else attend_mma_kernel<MT, CKV_SILU_OVER_L, false><<<grid, 128, 0, s>>>(a, pKp, pVp, n_mb);
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+bool mma_supported(int dtype, int head_dim, int d_user)
+{
+    return dtype == CKV_BF16 && head_dim == D && d_user <= 8;
+}
+
+cudaError_t launch_pool_permute(int G, int m, const void* poolK, const void* poolV, void* poolKp, void* poolVp,
+                                cudaStream_t s)
+{
+    const int64_t rows = (int64_t)G * m;
+    int grid = (int)((rows * D + 255) / 256);
+    if (grid > 148 * 16) grid = 148 * 16;
+    pool_permute_kernel<<<grid, 256, 0, s>>>((const uint16_t*)poolK, (uint16_t*)poolKp, (uint16_t*)poolVp,
+                                             (const uint16_t*)poolV, rows);
+    return cudaGetLastError();
+}
+
+int mma_queries_per_warp(int max_M) { return max_M <= 16 ? 16 : (max_M <= 32 ? 32 : 64); }
+
+cudaError_t launch_attend_mma(int max_M, const AttendArgs& a, const void* poolKp, const void* poolVp,
+                              cudaStream_t s)
+{
+    if (a.n_items == 0) return cudaSuccess;
+    const int qpw = mma_queries_per_warp(max_M);
+    const int n_mb = (max_M + qpw - 1) / qpw;
+    switch (qpw) {
+        case 16: return launch_mt<1>(a, poolKp, poolVp, n_mb, s);
+        case 32: return launch_mt<2>(a, poolKp, poolVp, n_mb, s);
+        default: return launch_mt<4>(a, poolKp, poolVp, n_mb, s);
+    }
+}
+
+}  // namespace ckv

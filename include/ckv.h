@@ -57,7 +57,8 @@ typedef enum {
     CKV_ERR_UNKNOWN_USER = 5, /* user id has no cache entry                                    */
     CKV_ERR_OOM = 6,          /* device or host allocation failed                              */
     CKV_ERR_CUDA = 7,         /* a CUDA call failed; see ckv_last_cuda_error                   */
-    CKV_ERR_UNSUPPORTED = 8   /* configuration outside what the kernels were built for         */
+    CKV_ERR_UNSUPPORTED = 8,  /* configuration outside what the kernels were built for         */
+    CKV_ERR_TOO_LARGE = 9     /* request beyond a fixed capacity (ckv_attend_static only)      */
 } ckv_status;
 
 typedef enum { CKV_F32 = 0, CKV_BF16 = 1 } ckv_dtype;
@@ -142,6 +143,41 @@ CKV_API ckv_status ckv_cache_clear(ckv_ctx* ctx);
  */
 CKV_API ckv_status ckv_attend(ckv_ctx* ctx, int32_t n, const int64_t* users, const int32_t* q_off,
                       const void* queries, void* out, void* stream);
+
+/*
+ * Decode without any allocation.  (The paper has no counterpart: this is a deployment variant of
+ * ckv_attend, not a different computation.)
+ *
+ * ckv_attend may call cudaMalloc/cudaFree: it grows a workspace for the partial results of
+ * the split-along-history reduction and keeps per-request tables in device memory it
+ * allocates.  Some callers cannot tolerate that: a serving thread inside a latency-critical
+ * section (cudaMalloc and cudaFree synchronise the device), a process whose memory was handed
+ * in full to another allocator, code running between cudaStreamBeginCapture and EndCapture
+ * where allocation is not permitted.  For them this entry point computes exactly what
+ * ckv_attend computes, with the same kernels, but keeps those tables and partial results in a
+ * fixed array that is part of the library's device image:
+ *   - CKV_STATIC_SCRATCH_BYTES (8 MiB) per GPU that loads the library, held until the
+ *     process exits, shared by every context and every call on that GPU;
+ *   - limits: n <= CKV_STATIC_MAX_USERS (256) users per call, at most 4096 history chunks, and
+ *     partial results (chunks x queries of every split user x n_groups x (head_dim + 2) floats)
+ *     that fit the rest of the array.  Anything larger returns CKV_ERR_TOO_LARGE and
+ *     enqueues nothing.  ("split_len" controls the chunk count; 0 = automatic.)
+ *   - queries and out must be device memory (staging host buffers would need an allocation);
+ *     host pointers return CKV_ERR_INVALID_ARG.
+ * It calls no cudaMalloc, cudaFree or other allocating routine.  The first call on a device
+ * looks up the array's device address (once per device, with that device current); make that
+ * first call outside any stream capture.
+ * The array keeps the previous call's contents.  Nothing in it needs clearing: every entry
+ * a call reads it has written itself.  Because all calls on a GPU share the array, two
+ * calls whose kernels may overlap on the GPU (different streams, or different host threads)
+ * race on it: serialise them (one stream, or events between streams).
+ * Other arguments, results and errors are those of ckv_attend.
+ */
+#define CKV_STATIC_SCRATCH_BYTES (8u << 20)
+#define CKV_STATIC_MAX_USERS 256
+CKV_API ckv_status ckv_attend_static(ckv_ctx* ctx, int32_t n, const int64_t* users,
+                                     const int32_t* q_off, const void* queries, void* out,
+                                     void* stream);
 
 /*
  * TEST ONLY -- the single path that writes full-width K/V to device memory: Eq. (Kc) and

@@ -17,12 +17,13 @@ LIB_PATH = os.path.join(_HERE, "libckv.so")
 CKV_F32, CKV_BF16 = 0, 1
 CKV_SOFTMAX, CKV_SILU_OVER_L = 0, 1
 (CKV_OK, CKV_ERR_INVALID_ARG, CKV_ERR_SHAPE, CKV_ERR_STATE, CKV_ERR_INDEX_RANGE,
- CKV_ERR_UNKNOWN_USER, CKV_ERR_OOM, CKV_ERR_CUDA, CKV_ERR_UNSUPPORTED) = range(9)
+ CKV_ERR_UNKNOWN_USER, CKV_ERR_OOM, CKV_ERR_CUDA, CKV_ERR_UNSUPPORTED, CKV_ERR_TOO_LARGE) = range(10)
 
 # every symbol include/ckv.h declares
 EXPORTS = (
     "ckv_create", "ckv_destroy", "ckv_pool_load", "ckv_cache_put", "ckv_cache_put_batch",
-    "ckv_cache_evict", "ckv_cache_clear", "ckv_attend", "ckv_materialize", "ckv_user_length",
+    "ckv_cache_evict", "ckv_cache_clear", "ckv_attend", "ckv_attend_static", "ckv_materialize",
+    "ckv_user_length",
     "ckv_cache_bytes", "ckv_set_option", "ckv_get_option", "ckv_last_stat", "ckv_strerror",
     "ckv_last_cuda_error", "ckv_version",
 )
@@ -44,7 +45,7 @@ class CkvError(RuntimeError):
 def _load() -> ctypes.CDLL:
     if not os.path.exists(LIB_PATH):
         raise ImportError(
-            f"{LIB_PATH} is missing: build it with `python -m paper_2601_19178_b200.build` "
+            f"{LIB_PATH} is missing: build it with `python paper_2601_19178_b200/build.py` "
             "(there is no fallback implementation)")
     L = ctypes.CDLL(LIB_PATH)
     vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
@@ -58,6 +59,7 @@ def _load() -> ctypes.CDLL:
         "ckv_cache_evict": (i32, [vp, i64]),
         "ckv_cache_clear": (i32, [vp]),
         "ckv_attend": (i32, [vp, i32, vp, vp, vp, vp, vp]),
+        "ckv_attend_static": (i32, [vp, i32, vp, vp, vp, vp, vp]),
         "ckv_materialize": (i32, [vp, i64, vp, vp, vp]),
         "ckv_user_length": (i32, [vp, i64, p64]),
         "ckv_cache_bytes": (i32, [vp, p64, p64]),
@@ -163,6 +165,20 @@ def ckv_attend(ctx, users, q_off, queries, out, stream=None) -> None:
         raise ValueError("q_off must have len(users) + 1 entries")
     _check(ctx, lib.ckv_attend(ctx, users.shape[0], users.ctypes.data, q_off.ctypes.data, _ptr(queries),
                                _ptr(out), _stream(stream)), "ckv_attend")
+
+
+def ckv_attend_static(ctx, users, q_off, queries, out, stream=None) -> None:
+    """ckv_attend for callers that must not allocate device memory (a latency-critical
+    serving section, a process whose memory belongs to another allocator): same result, but
+    the work tables and split-reduction partials live in a fixed 8 MiB array inside the
+    library.  queries/out must be device buffers; raises CkvError(CKV_ERR_TOO_LARGE) beyond
+    256 users per call or when the partial results do not fit.  Calls that may overlap on the
+    GPU race on that array."""
+    users, q_off = _host_i64(users), _host_i32(q_off)
+    if q_off.shape[0] != users.shape[0] + 1:
+        raise ValueError("q_off must have len(users) + 1 entries")
+    _check(ctx, lib.ckv_attend_static(ctx, users.shape[0], users.ctypes.data, q_off.ctypes.data,
+                                      _ptr(queries), _ptr(out), _stream(stream)), "ckv_attend_static")
 
 
 def ckv_materialize(ctx, user: int, K_out, V_out, stream=None) -> None:

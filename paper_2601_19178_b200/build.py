@@ -1,6 +1,6 @@
 """Builds libckv.so (sm_100a) next to this file with nvcc.  No GPU is needed to build.
 
-    python -m paper_2601_19178_b200.build [--force] [--verbose]
+    python paper_2601_19178_b200/build.py [--force] [--verbose]     (or: python __graft_entry__.py)
 """
 from __future__ import annotations
 

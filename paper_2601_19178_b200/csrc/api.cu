@@ -3,6 +3,7 @@
 #include <algorithm>
 #include <cmath>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <string>
 #include <unordered_map>
@@ -741,6 +742,7 @@ const char* ckv_strerror(ckv_status s)
         case CKV_ERR_OOM: return "out of memory";
         case CKV_ERR_CUDA: return "CUDA error";
         case CKV_ERR_UNSUPPORTED: return "unsupported configuration";
+        case CKV_ERR_TOO_LARGE: return "request exceeds the fixed capacity of this entry point";
     }
     return "unknown status";
 }
@@ -750,3 +752,140 @@ const char* ckv_last_cuda_error(ckv_ctx* ctx) { return ctx ? ctx->cuda_err.c_str
 int32_t ckv_version(void) { return 100; }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------------------------------
+// ckv_attend_static: the decode call for callers that must not allocate.
+//
+// Everything ckv_attend would put into freshly allocated or grown device memory -- the
+// request/work-item tables and the partial results of the split-along-history reduction --
+// lives in one fixed array in the library's device image instead.  The array exists once per
+// GPU that loads the library and is shared by every call on that GPU.
+// ------------------------------------------------------------------------------------------
+namespace {
+
+constexpr size_t kStaticBytes = size_t(8) << 20;  // CKV_STATIC_SCRATCH_BYTES
+constexpr int kStaticMaxReqs = 256;                // CKV_STATIC_MAX_USERS
+constexpr int kStaticMaxItems = 4096;
+constexpr int kStaticMaxDevices = 64;
+constexpr size_t kOffItems = sizeof(Req) * kStaticMaxReqs;
+constexpr size_t kOffSplit = kOffItems + sizeof(Item) * kStaticMaxItems;
+constexpr size_t kOffPartials = (kOffSplit + sizeof(int32_t) * kStaticMaxReqs + 255) / 256 * 256;
+
+static __device__ __align__(256) unsigned char ckv_static_scratch[kStaticBytes];
+
+// In host code `ckv_static_scratch` is only a handle for the runtime, not a device address.
+// The address a kernel can use is looked up once per device, with that device current.
+void* g_static_addr[kStaticMaxDevices];
+std::mutex g_static_mu;
+
+cudaError_t static_scratch_address(int device, void** out)
+{
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (!g_static_addr[device]) {
+        void* p = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&p, ckv_static_scratch);
+        if (e != cudaSuccess) return e;
+        g_static_addr[device] = p;
+    }
+    *out = g_static_addr[device];
+    return cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" ckv_status ckv_attend_static(ckv_ctx* ctx, int32_t n, const int64_t* users, const int32_t* q_off,
+                                        const void* queries, void* out, void* stream)
+{
+    if (!ctx || n < 0 || (n > 0 && (!users || !q_off))) return CKV_ERR_INVALID_ARG;
+    if (!ctx->pool) return CKV_ERR_STATE;
+    if (n == 0) return CKV_OK;
+    if (n > kStaticMaxReqs) return CKV_ERR_TOO_LARGE;
+    if (!offsets_ok32(q_off, n)) return CKV_ERR_INVALID_ARG;
+    if (ctx->cfg.device >= kStaticMaxDevices) return CKV_ERR_UNSUPPORTED;
+    const int64_t Q = q_off[n];
+    if (Q == 0) return CKV_OK;
+    if (!queries || !out) return CKV_ERR_INVALID_ARG;
+    DeviceGuard dg(ctx->cfg.device);
+    if (!is_device_ptr(queries) || !is_device_ptr(out)) return CKV_ERR_INVALID_ARG;  // staging would allocate
+    cudaStream_t s = (cudaStream_t)stream;
+    void* scratch = nullptr;
+    CK(static_scratch_address(ctx->cfg.device, &scratch));
+
+    // the plan, in fixed-size host arrays
+    Req reqs[kStaticMaxReqs];
+    Item items[kStaticMaxItems];
+    int32_t split[kStaticMaxReqs];
+    const int D = ctx->cfg.head_dim, G = ctx->cfg.n_groups;
+    int64_t total_pos = 0;
+    int32_t max_M = 0;
+    for (int32_t k = 0; k < n; ++k) {
+        auto f = ctx->users.find(users[k]);
+        if (f == ctx->users.end()) return CKV_ERR_UNKNOWN_USER;
+        Req& r = reqs[k];
+        r.base = f->second.base;
+        r.L = f->second.L;
+        r.Lpad = f->second.Lpad;
+        r.q0 = q_off[k];
+        r.M = q_off[k + 1] - q_off[k];
+        r.part0 = -1;
+        r.n_chunks = 1;
+        if (r.M > 0) total_pos += r.L;
+        max_M = std::max(max_M, r.M);
+    }
+    int family;
+    if (ctx->opt_kernel == 0) family = ctx->has_mma_pool && max_M >= 9 ? 2 : 1;
+    else if (ctx->opt_kernel == 1) family = 1;
+    else if (ctx->opt_kernel == 2 && ctx->has_mma_pool) family = 2;
+    else return CKV_ERR_UNSUPPORTED;
+    const int64_t C = ctx->opt_split > 0 ? ctx->opt_split : auto_split_len(ctx, total_pos, family, max_M);
+    const int64_t row_floats = (int64_t)G * (D + 2);
+    const int64_t cap_rows = (int64_t)((kStaticBytes - kOffPartials) / sizeof(float)) / row_floats;
+    int32_t n_items = 0, n_split = 0;
+    int64_t part_rows = 0;
+    for (int32_t k = 0; k < n; ++k) {
+        Req& r = reqs[k];
+        if (r.M <= 0) continue;
+        const int64_t nc = r.L == 0 ? 1 : (r.L + C - 1) / C;
+        if (n_items + nc > kStaticMaxItems) return CKV_ERR_TOO_LARGE;
+        r.n_chunks = (int32_t)nc;
+        if (nc == 1) {
+            items[n_items++] = Item{k, 0, r.L, -1};
+            continue;
+        }
+        if (part_rows + nc * r.M > cap_rows) return CKV_ERR_TOO_LARGE;
+        r.part0 = (int32_t)part_rows;
+        split[n_split++] = k;
+        for (int64_t c = 0; c < nc; ++c) {
+            const int32_t b = (int32_t)(c * C);
+            items[n_items++] = Item{k, b, (int32_t)std::min<int64_t>(C, r.L - b), (int32_t)(part_rows + c * r.M)};
+        }
+        part_rows += nc * r.M;
+    }
+    std::stable_sort(items, items + n_items, [](const Item& x, const Item& y) { return x.len > y.len; });
+
+    char* base = (char*)scratch;
+    CK(cudaMemcpyAsync(base, reqs, sizeof(Req) * (size_t)n, cudaMemcpyHostToDevice, s));
+    if (n_items) CK(cudaMemcpyAsync(base + kOffItems, items, sizeof(Item) * (size_t)n_items, cudaMemcpyHostToDevice, s));
+    if (n_split) CK(cudaMemcpyAsync(base + kOffSplit, split, sizeof(int32_t) * (size_t)n_split, cudaMemcpyHostToDevice, s));
+
+    AttendArgs a;
+    a.cv = view_of(ctx);
+    a.reqs = (const Req*)base;
+    a.items = (const Item*)(base + kOffItems);
+    a.n_items = n_items;
+    a.queries = queries;
+    a.out = out;
+    a.partials = (float*)(base + kOffPartials);  // every entry that is read was written by this call
+    a.out_dtype = ctx->cfg.out_dtype;
+    a.mode = ctx->cfg.mode;
+    a.scale = ctx->scale;
+    if (n_items > 0) {
+        if (family == 2)
+            CK(launch_attend_mma(max_M, a, (const char*)ctx->pool + 2 * ctx->pool_half,
+                                 (const char*)ctx->pool + 3 * ctx->pool_half, s));
+        else
+            CK(launch_attend_simt(ctx->cfg.dtype, D, max_M, a, s));
+    }
+    if (n_split > 0) CK(launch_combine(D, a, (const int32_t*)(base + kOffSplit), n_split, s));
+    return CKV_OK;
+}

@@ -215,6 +215,8 @@ CKV_API ckv_status ckv_get_option(ckv_ctx* ctx, const char* name, int64_t* value
  * "workspace_bytes", "plan_cache_hit"; with option "time_kernels" also "main_kernel_ns" and
  * "combine_kernel_ns" (device time of the attend kernel and of the split-merge kernel; the
  * query waits for that attend to finish; CKV_ERR_STATE if nothing was timed).
+ * "device_errors" (not tied to the last call): non-zero once a kernel of this context gave up
+ * on one of its internal bounded waits -- its outputs are then invalid; synchronises the device.
  */
 CKV_API ckv_status ckv_last_stat(ckv_ctx* ctx, const char* name, int64_t* value);
 

@@ -68,6 +68,8 @@ struct ckv_ctx {
     int n_entries = 0, d_shared = 0, d_user = 0, idx_bytes = 0;
     void* pool = nullptr;  // K rows then V rows, each [G][m][D]; then the two MMA-ordered copies
     bool has_mma_pool = false;
+    bool has_umma = false;
+    int* d_err = nullptr;  // OR of error codes from kernels whose bounded waits ran out
     size_t pool_half = 0;  // bytes of one of them
     // arena of compressed caches (units = (position, group) slots)
     void *a_idxK = nullptr, *a_idxV = nullptr, *a_userK = nullptr, *a_userV = nullptr;
@@ -227,6 +229,11 @@ int64_t auto_split_len(const ckv_ctx* ctx, int64_t total_positions, int family, 
     // Enough (chunk, group) blocks to fill the SMs several times over, but chunks long
     // enough that the merge of partial results stays a small fraction of the work.
     int64_t c;
+    if (family == 3) {  // one CTA per (chunk, group, 128 queries), two CTAs per SM, 128-position tiles
+        c = total_positions * ctx->cfg.n_groups * ((max_M + 127) / 128) / (kNumSMs * 2 * 4);
+        c = (c + 127) / 128 * 128;
+        return std::min<int64_t>(std::max<int64_t>(c, 512), 8192);
+    }
     if (family == 2) {
         const int qpw = mma_queries_per_warp(max_M);
         c = total_positions * ctx->cfg.n_groups * ((max_M + qpw - 1) / qpw) / (kNumSMs * 32);
@@ -260,9 +267,10 @@ ckv_status build_plan(ckv_ctx* ctx, Plan& pl, int32_t n, const int64_t* users, c
     }
     pl.max_M = max_M;
     const bool can_mma = ctx->has_mma_pool;
-    if (ctx->opt_kernel == 0) pl.family = can_mma && max_M >= 9 ? 2 : 1;
+    if (ctx->opt_kernel == 0) pl.family = ctx->has_umma && max_M >= 48 ? 3 : (can_mma && max_M >= 9 ? 2 : 1);
     else if (ctx->opt_kernel == 1) pl.family = 1;
     else if (ctx->opt_kernel == 2 && can_mma) pl.family = 2;
+    else if (ctx->opt_kernel == 3 && ctx->has_umma) pl.family = 3;
     else return CKV_ERR_UNSUPPORTED;
     const int64_t C = ctx->opt_split > 0 ? ctx->opt_split : auto_split_len(ctx, total_pos, pl.family, max_M);
     std::vector<Item> items;
@@ -393,11 +401,13 @@ ckv_status ckv_create(const ckv_config* cfg, ckv_ctx** out)
     ctx->scale = cfg->scale > 0.f ? cfg->scale
                                   : (cfg->mode == CKV_SOFTMAX ? 1.0f / std::sqrt((float)cfg->head_dim) : 1.0f);
     DeviceGuard dg(cfg->device);
-    if (!dg.ok || cudaMalloc((void**)&ctx->d_flag, sizeof(int)) != cudaSuccess) {
+    if (!dg.ok || cudaMalloc((void**)&ctx->d_flag, 2 * sizeof(int)) != cudaSuccess ||
+        cudaMemset(ctx->d_flag, 0, 2 * sizeof(int)) != cudaSuccess) {
         cudaGetLastError();
         delete ctx;
         return CKV_ERR_CUDA;
     }
+    ctx->d_err = ctx->d_flag + 1;
     *out = ctx;
     return CKV_OK;
 }
@@ -441,6 +451,7 @@ ckv_status ckv_pool_load(ckv_ctx* ctx, const void* pool_K, const void* pool_V, i
         ctx->pool_half = half;
         ctx->has_mma_pool = mma;
     }
+    ctx->has_umma = umma_supported(ctx->cfg.dtype, D, D - d_shared);
     CK(launch_pool_layout(ctx->cfg.dtype, G, n_entries, d_shared, D, sk.dev, ctx->pool, s));
     CK(launch_pool_layout(ctx->cfg.dtype, G, n_entries, d_shared, D, sv.dev, (char*)ctx->pool + half, s));
     if (mma)
@@ -604,7 +615,9 @@ ckv_status ckv_attend(ckv_ctx* ctx, int32_t n, const int64_t* users, const int32
         CK(cudaEventRecord(ctx->ev[0], s));
     }
     if (pl->n_items > 0) {
-        if (pl->family == 2)
+        if (pl->family == 3)
+            CK(launch_attend_umma(pl->max_M, a, ctx->d_err, s));
+        else if (pl->family == 2)
             CK(launch_attend_mma(pl->max_M, a, (const char*)ctx->pool + 2 * ctx->pool_half,
                                  (const char*)ctx->pool + 3 * ctx->pool_half, s));
         else
@@ -717,6 +730,12 @@ ckv_status ckv_last_stat(ckv_ctx* ctx, const char* name, int64_t* value)
     else if (!std::strcmp(name, "kernel")) *value = ctx->st_kernel;
     else if (!std::strcmp(name, "workspace_bytes")) *value = ctx->st_ws;
     else if (!std::strcmp(name, "plan_cache_hit")) *value = ctx->st_hit;
+    else if (!std::strcmp(name, "device_errors")) {
+        DeviceGuard dg(ctx->cfg.device);
+        int v = 0;
+        CK(cudaMemcpy(&v, ctx->d_err, sizeof(int), cudaMemcpyDeviceToHost));
+        *value = v;
+    }
     else if (!std::strcmp(name, "main_kernel_ns") || !std::strcmp(name, "combine_kernel_ns")) {
         if (!ctx->ev_valid) return CKV_ERR_STATE;
         DeviceGuard dg(ctx->cfg.device);

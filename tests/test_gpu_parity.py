@@ -33,6 +33,51 @@ def test_attend_matches_oracle(name):
     assert_close(got, want, w.dtype, name)
 
 
+@pytest.mark.parametrize("kernel", [1, 2, 3])
+@pytest.mark.parametrize("name", ["cfg2", "cfg2_ragged", "cfg3", "cfg3_ragged", "cfg5_ragged"])
+def test_every_kernel_family_matches_oracle(name, kernel):
+    """1 = CUDA cores, 2 = warp-level MMA, 3 = tcgen05; all must agree with the oracle."""
+    w = SMALL[name]
+    d = synth.generate(w)
+    s = make_session(w, d, kernel=kernel)
+    got = gpu_attend(w, d, session=s)
+    assert s.stat("kernel") == kernel
+    assert s.stat("device_errors") == 0
+    s.close()
+    assert_close(got, oracle_attend(w, d), w.dtype, f"{name} kernel {kernel}")
+
+
+@pytest.mark.parametrize("kernel", [2, 3])
+@pytest.mark.parametrize("mode", ["softmax", "silu_over_l"])
+@pytest.mark.parametrize("d_user", [0, 1, 2, 4, 8])
+def test_tensor_core_kernels_user_widths_and_sharp_softmax(kernel, mode, d_user):
+    w = synth.Workload("tc", 3, 32 - d_user, d_user, 300, 5, (1, 700), 70, mode, "bf16", 1.1, 1 / 32, 1 / 32, 21)
+    d = synth.generate(w)
+    scale = 8.0 / np.sqrt(32) if mode == "softmax" else 1.0
+    s = make_session(w, d, scale=scale, kernel=kernel, split_len=256)
+    got = gpu_attend(w, d, session=s)
+    assert s.stat("split_items") > 0 and s.stat("device_errors") == 0
+    s.close()
+    assert_close(got, oracle_attend(w, d, scale=scale), "bf16", f"d_user={d_user}")
+
+
+def test_growing_maximum_triggers_rescale_in_tcgen05_kernel():
+    """Keys sorted by increasing score make every tile raise the running maximum."""
+    w = synth.Workload("grow", 1, 30, 2, 512, 2, (1024, 1024), 128, "softmax", "bf16", None, 1.0, 1.0, 33)
+    d = synth.generate(w)
+    # history = pool rows in an order of growing norm along one direction: scale the user part
+    ramp = np.linspace(-40.0, 40.0, 1024, dtype=np.float32)
+    for u in range(2):
+        d["user_K"][u * 1024:(u + 1) * 1024, 0, 0] = synth.f32_to_bf16_bits(ramp)
+    d["queries"][:, 0, 0] = synth.f32_to_bf16_bits(np.full(d["queries"].shape[0], 1.0, np.float32))
+    for kernel in (2, 3):
+        s = make_session(w, d, scale=1.0, kernel=kernel)
+        got = gpu_attend(w, d, session=s)
+        assert s.stat("device_errors") == 0
+        s.close()
+        assert_close(got, oracle_attend(w, d, scale=1.0), "bf16", f"kernel {kernel}")
+
+
 @pytest.mark.parametrize("name", ["cfg1", "cfg2_ragged", "cfg4", "cfg5_ragged"])
 @pytest.mark.parametrize("scale_mul", [1.0, 4.0])
 def test_attend_sharper_softmax(name, scale_mul):
@@ -106,7 +151,8 @@ def test_wide_pool_uses_32_bit_indices():
     assert_close(gpu_attend(w, d), oracle_attend(w, d), "bf16")
 
 
-def test_empty_history_empty_query_list_and_repeated_user():
+@pytest.mark.parametrize("kernel", [1, 2, 3])
+def test_empty_history_empty_query_list_and_repeated_user(kernel):
     w = synth.Workload("edge", 2, 30, 2, 64, 4, (40, 40), 3, "softmax", "bf16", None, 1 / 32, 1 / 32, 8)
     d = synth.generate(w)
     # user 1: empty history; request list: [u0, u1, u2 (no queries), u3, u0 again]
@@ -114,7 +160,7 @@ def test_empty_history_empty_query_list_and_repeated_user():
     for k in ("idx_K", "idx_V", "user_K", "user_V"):
         d[k] = np.ascontiguousarray(d[k][keep])
     d["hist_off"] = np.array([0, 40, 40, 80, 120], dtype=np.int64)
-    s = make_session(w, d)
+    s = make_session(w, d, kernel=kernel)
     req_users = d["users"][[0, 1, 2, 3, 0]]
     q_off = np.array([0, 3, 6, 6, 9, 12], dtype=np.int32)
     q = d["queries"]

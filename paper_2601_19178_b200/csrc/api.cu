@@ -41,7 +41,6 @@ struct Plan {
 };
 
 constexpr int kMaxPlans = 4;
-constexpr int kNumSMs = 148;
 
 struct DeviceGuard {
     int prev = -1;
@@ -64,6 +63,7 @@ struct ckv_ctx {
     ckv_config cfg{};
     float scale = 1.f;
     int elem = 2;  // bytes per element of cfg.dtype
+    int n_sms = 148;
     // pool
     int n_entries = 0, d_shared = 0, d_user = 0, idx_bytes = 0;
     void* pool = nullptr;  // K rows then V rows, each [G][m][D]; then the two MMA-ordered copies
@@ -229,18 +229,18 @@ int64_t auto_split_len(const ckv_ctx* ctx, int64_t total_positions, int family, 
     // Enough (chunk, group) blocks to fill the SMs several times over, but chunks long
     // enough that the merge of partial results stays a small fraction of the work.
     int64_t c;
-    if (family == 3) {  // one CTA per (chunk, group, 128 queries), two CTAs per SM, 128-position tiles
-        c = total_positions * ctx->cfg.n_groups * ((max_M + 127) / 128) / (kNumSMs * 2 * 4);
+    if (family == 3) {  // persistent CTAs share (chunk, group, 128 queries) units round-robin: a few units per SM
+        c = total_positions * ctx->cfg.n_groups * ((max_M + 127) / 128) / (ctx->n_sms * 4);
         c = (c + 127) / 128 * 128;
-        return std::min<int64_t>(std::max<int64_t>(c, 512), 8192);
+        return std::min<int64_t>(std::max<int64_t>(c, 1024), 16384);
     }
     if (family == 2) {
         const int qpw = mma_queries_per_warp(max_M);
-        c = total_positions * ctx->cfg.n_groups * ((max_M + qpw - 1) / qpw) / (kNumSMs * 32);
+        c = total_positions * ctx->cfg.n_groups * ((max_M + qpw - 1) / qpw) / (ctx->n_sms * 32);
         c = (c + 63) / 64 * 64;
         return std::min<int64_t>(std::max<int64_t>(c, 256), 4096);
     }
-    c = total_positions * ctx->cfg.n_groups / (kNumSMs * 16);
+    c = total_positions * ctx->cfg.n_groups / (ctx->n_sms * 16);
     c = (c + 63) / 64 * 64;
     return std::min<int64_t>(std::max<int64_t>(c, 256), 2048);
 }
@@ -408,6 +408,10 @@ ckv_status ckv_create(const ckv_config* cfg, ckv_ctx** out)
         return CKV_ERR_CUDA;
     }
     ctx->d_err = ctx->d_flag + 1;
+    if (cudaDeviceGetAttribute(&ctx->n_sms, cudaDevAttrMultiProcessorCount, cfg->device) != cudaSuccess || ctx->n_sms < 1) {
+        cudaGetLastError();
+        ctx->n_sms = 148;
+    }
     *out = ctx;
     return CKV_OK;
 }
@@ -616,7 +620,7 @@ ckv_status ckv_attend(ckv_ctx* ctx, int32_t n, const int64_t* users, const int32
     }
     if (pl->n_items > 0) {
         if (pl->family == 3)
-            CK(launch_attend_umma(pl->max_M, a, ctx->d_err, s));
+            CK(launch_attend_umma(pl->max_M, a, ctx->n_sms, ctx->d_err, s));
         else if (pl->family == 2)
             CK(launch_attend_mma(pl->max_M, a, (const char*)ctx->pool + 2 * ctx->pool_half,
                                  (const char*)ctx->pool + 3 * ctx->pool_half, s));

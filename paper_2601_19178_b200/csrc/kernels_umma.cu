@@ -1,27 +1,38 @@
 // tcgen05 gather-concat-attention kernel (bf16, head_dim 32) for many queries per user.
 //
-// One CTA owns (work item, group, block of up to 128 queries) and walks the history chunk
-// in tiles of 128 positions.  Roles (warp-specialised, 7 warps):
-//   warps 0-3  softmax / SiLU: thread i owns query row i = TMEM lane i
-//   warp  4    issues tcgen05.mma (one elected thread), owns the TMEM allocation
-//   warps 5-6  producers: gather pool rows into shared memory with 16-byte cp.async,
-//              patch the user-specific leading elements (Eq. K), publish the tile
+// Persistent: one CTA per SM walks a static round-robin share of the work units, where a unit
+// is (work item = history chunk of one user, group, block of up to 128 queries).  The history
+// chunk is processed in tiles of 128 positions.  Roles (warp-specialised, 13 warps):
+//   warps 0-3   normalisation group 0: thread i owns query row i = TMEM lane i, even tiles
+//   warps 4-7   normalisation group 1: the same rows, odd tiles
+//   warp  8     issues tcgen05.mma (one thread), owns the TMEM allocation
+//   warps 9-12  producers: gather pool rows into shared memory with 16-byte cp.async, patch the
+//               user-specific leading elements (Eq. K), publish the tile; also stage Q
 //
-// Per tile j:   S_j = Q K_j^T   (UMMA 128 x 128 x 32, A = Q smem, B = K tile smem, K-major)
-//               P_j = exp2(S_j c - m) or silu(S_j c)    (softmax warps: tcgen05.ld -> math ->
-//                                                         bf16 -> tcgen05.st)
-//               O  += P_j V_j   (UMMA 128 x 32 x 128, A = P from TMEM, B = V tile smem, MN-major)
-// O stays in TMEM for the whole chunk.  The softmax keeps a reference maximum m per row and
-// only rescales O (a TMEM read-modify-write) when a tile raises the maximum by more than 2^8;
-// otherwise p may exceed 1 by at most that factor, which fp32/bf16 hold easily.
+// Tile t of the CTA's tile stream uses score buffer b = t mod 2:
+//   S_b  = Q K_t^T                    UMMA 128 x 128 x 32, A = Q smem, B = K tile smem (K-major)
+//   P_b  = exp2(S_b c - m) | silu     group b: tcgen05.ld -> math -> bf16 -> tcgen05.st
+//   O_b += P_b [V_t | 1]              UMMA 128 x 48 x 128, A = P from TMEM, B = V tile (MN-major)
+// While group b normalises tile t the tensor core already works on tile t+1 for the other
+// group, and the producers gather tiles t+2...; nothing drains between work units.  The two
+// groups keep separate accumulators O_0, O_1 with separate reference maxima and merge them
+// through shared memory when a unit ends.
 //
-// Shared-memory tiles use the no-swizzle UMMA canonical layout: 8-row groups of 512 bytes,
-// inside a group four 128-byte core matrices (one per 16-byte row chunk), inside a core
-// matrix row r%8 at 16 r.  A gathered 64-byte row therefore lands as four 16-byte pieces;
-// the same physical layout serves K (K-major B operand) and V (MN-major B operand).
+// Softmax bookkeeping.  The V tile carries sixteen extra columns of which the first is all
+// ones, so column 32 of O_b accumulates the row sum l of exactly the bf16-rounded P that
+// multiplies V.  The reference maximum m of a row is the exact maximum of the group's first
+// tile of the unit and stays fixed: later scores may exceed it by up to 2^64 (fp32
+// accumulators and bf16 P have the exponent range for that); only when a tile exceeds that
+// bound is O_b rescaled (TMEM read-modify-write) and the tile redone.
 //
-// Every wait in this kernel is bounded: on time-out the CTA records an error code, drains its
-// own copies, frees its TMEM and returns.
+// Shared-memory tiles use the no-swizzle UMMA canonical layout: groups of 8 rows, inside a
+// group one 128-byte core matrix per 16-byte row chunk, inside a core matrix row r%8 at 16 r.
+// K tiles and Q use 512-byte groups (4 chunks); V tiles 768-byte groups (4 data chunks + 2
+// chunks holding the ones column).
+//
+// Every wait in this kernel is bounded: on time-out the CTA records an error code, raises a
+// CTA-wide abort flag that ends every other wait, drains its own copies, frees its TMEM and
+// returns.
 #include <cuda_bf16.h>
 #include <math_constants.h>
 
@@ -31,32 +42,46 @@ namespace ckv {
 namespace {
 
 constexpr int D = 32;
-constexpr int TK = 128;                 // positions per tile
-constexpr int NS = 4;                   // shared-memory stages
-constexpr int kSoftmaxThreads = 128;
-constexpr int kProducerThreads = 64;
-constexpr int kThreads = kSoftmaxThreads + 32 + kProducerThreads;  // 224
-constexpr int kMmaWarp = 4;
-constexpr int kTileBytes = TK * D * 2;  // 8 KB
-constexpr int kMaxDu = 8;
-constexpr int kSideBytes = TK * kMaxDu * 2;  // user part of one tile, K or V: up to 2 KB
-constexpr uint32_t kTmemCols = 256;
-constexpr uint32_t kColS = 0, kColP = 128, kColO = 192;
+constexpr int TK = 128;                  // positions per tile
+constexpr int NS = 6;                    // K/V stages
+constexpr int LAG = 3;                   // tiles whose copies are in flight per producer thread
+constexpr int NQ = 3;                    // Q buffers
+// A producer publishes tile t - LAG before it issues tile t.  Q buffer reuse waits for the unit
+// NQ units back, whose last tile is at most t - NQ: published already iff NQ >= LAG.
+static_assert(NQ >= LAG, "Q buffer reuse would wait for a tile that is not published yet");
+constexpr int kGroupThreads = 128;       // one normalisation group
+constexpr int kMmaWarp = 8;
+constexpr int kProducerWarp0 = 9;
+constexpr int kProducerThreads = 128;
+constexpr int kThreads = 2 * kGroupThreads + 32 + kProducerThreads;  // 416
+constexpr int kTileK = TK * D * 2;       // 8 KB, also the Q tile
+constexpr int kVGroup = 768;             // bytes of one 8-row group of a V tile
+constexpr int kTileV = (TK / 8) * kVGroup;  // 12 KB
+constexpr int kNV = 48;                  // columns of [V | 1 | 0...]
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kColS = 0, kColP = 256, kColO = 384;  // S_b at kColS + 128 b, P_b at kColP + 64 b, O_b at kColO + 48 b
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr float kRescaleThreshold = 8.0f;  // log2 units
+constexpr float kHeadroom = 64.0f;       // log2 units a score may exceed the reference maximum
 constexpr uint32_t kSpinLimit = 1u << 20;
 
 // dynamic shared memory map
 constexpr int kOffQ = 0;
-constexpr int kOffK = kOffQ + kTileBytes;
-constexpr int kOffV = kOffK + NS * kTileBytes;
-constexpr int kOffSideK = kOffV + NS * kTileBytes;
-constexpr int kOffSideV = kOffSideK + NS * kSideBytes;
-constexpr int kOffBar = kOffSideV + NS * kSideBytes;
-constexpr int kSmemBytes = kOffBar + 256;  // 8 KB + 64 KB + 16 KB + barriers
+constexpr int kOffK = kOffQ + NQ * kTileK;
+constexpr int kOffV = kOffK + NS * kTileK;
+constexpr int kOffX = kOffV + NS * kTileV;          // exchange between the groups: [34][128] floats
+constexpr int kOffBar = kOffX + 34 * 128 * 4;
+constexpr int kOffAbort = kOffBar + 256;
+constexpr int kSmemBytes = kOffAbort + 16;
 
 // barrier slots (8 bytes each) behind kOffBar
-enum { BAR_FULL = 0, BAR_EMPTY = NS, BAR_S = 2 * NS, BAR_P, BAR_PV, BAR_DRAIN, BAR_COUNT };
+enum {
+    BAR_FULL = 0, BAR_EMPTY = NS, BAR_QEMPTY = 2 * NS, BAR_SFULL = 2 * NS + NQ, BAR_PREADY = BAR_SFULL + 2,
+    BAR_PFREE = BAR_SFULL + 4, BAR_OFULL = BAR_SFULL + 6, BAR_XFULL = BAR_SFULL + 8, BAR_XEMPTY, BAR_DRAIN, BAR_COUNT
+};
+static_assert(BAR_COUNT * 8 <= 256, "barrier area");
+
+// error codes OR-ed into the context's device error word
+enum { ERR_NORMALISE = 1, ERR_MMA = 2, ERR_DRAIN = 4, ERR_PRODUCER = 8 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -68,8 +93,8 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-// Bounded wait on a phase parity.  Returns false on time-out.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+// Bounded wait on a phase parity.  Returns false on time-out or when the CTA is aborting.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const volatile int* abort_flag)
 {
     for (uint32_t i = 0; i < kSpinLimit; ++i) {
         uint32_t ok;
@@ -81,12 +106,14 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
             : "r"(bar), "r"(parity)
             : "memory");
         if (ok) return true;
+        if ((i & 63u) == 63u && *abort_flag) return false;
     }
     return false;
 }
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src)
+// 16-byte copy global -> shared; src_bytes = 0 fills the destination with zeros instead
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes)
 {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
@@ -98,7 +125,6 @@ __device__ __forceinline__ void tc_commit(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 // D[tmem] (+)= A[smem] * B[smem]
@@ -134,6 +160,8 @@ __host__ __device__ constexpr uint32_t make_idesc(int M, int N, bool b_mn_major)
            ((uint32_t)(M >> 4) << 24);
 }
 
+// 32 consecutive columns of this thread's TMEM lane.  The load is asynchronous: its registers
+// hold the data only after tmem_wait_ld32 on the same array.
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
 {
     asm volatile(
@@ -146,6 +174,30 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
           "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr)
         : "memory");
+}
+// Waits for every tcgen05.ld of this thread.  Naming the registers as in/out operands keeps the
+// compiler from scheduling their consumers ahead of the wait.
+__device__ __forceinline__ void tmem_wait_ld32(uint32_t (&r)[32])
+{
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                   "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]),
+                   "+r"(r[15]), "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]),
+                   "+r"(r[22]), "+r"(r[23]), "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]),
+                   "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+                 :
+                 : "memory");
+}
+__device__ __forceinline__ uint32_t tmem_ld1(uint32_t taddr)
+{
+    uint32_t r;
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(r) : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" : "+r"(r) : : "memory");
+    return r;
+}
+__device__ __forceinline__ void tmem_st1(uint32_t taddr, uint32_t r)
+{
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x1.b32 [%0], {%1};" ::"r"(taddr), "r"(r) : "memory");
 }
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32])
 {
@@ -187,37 +239,114 @@ __device__ __forceinline__ float tanh_fast(float x)
     asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+__device__ __forceinline__ float max3(float a, float b, float c)
+{
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
 
-// byte offset of (row r, 16-byte chunk c) inside a tile
-__device__ __forceinline__ uint32_t tile_off(int r, int c) { return (uint32_t)((r >> 3) * 512 + c * 128 + (r & 7) * 16); }
+// byte offset of (row r, 16-byte chunk c) inside a K/Q tile and inside a V tile
+__device__ __forceinline__ uint32_t k_off(int r, int c) { return (uint32_t)((r >> 3) * 512 + c * 128 + (r & 7) * 16); }
+__device__ __forceinline__ uint32_t v_off(int r, int c) { return (uint32_t)((r >> 3) * kVGroup + c * 128 + (r & 7) * 16); }
+
+// One work unit of the CTA's share.
+struct Unit {
+    Item it;
+    Req rq;
+    int grp;
+    int row0;        // first query row of the block
+    int n_tiles;     // > 0: tiles to process; 0: empty history (zero output rows); < 0: nothing at all
+    int last_valid;  // real positions in the last tile
+};
+
+__device__ __forceinline__ void load_unit(const AttendArgs& a, int n_mb, int64_t w, Unit& u)
+{
+    const int G = a.cv.n_groups;
+    const int mb = (int)(w % n_mb);
+    const int64_t t = w / n_mb;
+    u.grp = (int)(t % G);
+    u.it = a.items[t / G];
+    u.rq = a.reqs[u.it.req];
+    u.row0 = mb * 128;
+    u.n_tiles = u.row0 < u.rq.M ? (u.it.len + TK - 1) / TK : -1;
+    u.last_valid = u.it.len - (u.n_tiles - 1) * TK;
+}
+
+// The CTA's tile stream: units blockIdx.x, blockIdx.x + gridDim.x, ... that have tiles, tile by
+// tile.  Every role walks an identical copy, so stage and buffer indices need no communication.
+struct Stream {
+    const AttendArgs* a;
+    int n_mb;
+    int64_t w, n_work;
+    Unit u;
+    int j;       // tile inside the unit
+    int g;       // tiles before this one in the stream
+    int useq;    // units with tiles before this one
+    bool valid;
+    __device__ __forceinline__ void seek()
+    {
+        valid = false;
+        while (w < n_work) {
+            load_unit(*a, n_mb, w, u);
+            if (u.n_tiles > 0) {
+                valid = true;
+                j = 0;
+                return;
+            }
+            w += gridDim.x;
+        }
+    }
+    __device__ __forceinline__ void init(const AttendArgs* args, int n_mb_, int64_t n_work_)
+    {
+        a = args;
+        n_mb = n_mb_;
+        n_work = n_work_;
+        w = blockIdx.x;
+        g = 0;
+        useq = 0;
+        seek();
+    }
+    __device__ __forceinline__ void advance()
+    {
+        ++g;
+        if (++j == u.n_tiles) {
+            w += gridDim.x;
+            ++useq;
+            seek();
+        }
+    }
+};
 
 template <int MODE, bool IDX16>
-__global__ void __launch_bounds__(kThreads, 2) attend_umma_kernel(const AttendArgs a, int n_mb, int* err_flag)
+__global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendArgs a, int n_mb, int64_t n_work, int* err_flag)
 {
     extern __shared__ __align__(1024) unsigned char smem[];
     __shared__ uint32_t tmem_base_slot;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const Item it = a.items[blockIdx.x / n_mb];
-    const int mb = blockIdx.x % n_mb;
-    const Req rq = a.reqs[it.req];
-    const int row0 = mb * 128;
-    if (row0 >= rq.M) return;  // uniform per CTA
-    const int grp = blockIdx.y, G = a.cv.n_groups, d_user = a.cv.d_user;
-    const int n_tiles = (it.len + TK - 1) / TK;
     const uint32_t sbase = smem_u32(smem);
     const uint32_t bar0 = sbase + kOffBar;
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kOffAbort);
+    const int G = a.cv.n_groups;
 
     if (tid == 0) {
         for (int s = 0; s < NS; ++s) {
             mbar_init(bar(BAR_FULL + s), kProducerThreads);
             mbar_init(bar(BAR_EMPTY + s), 1);
         }
-        mbar_init(bar(BAR_S), 1);
-        mbar_init(bar(BAR_P), kSoftmaxThreads);
-        mbar_init(bar(BAR_PV), 1);
+        for (int q = 0; q < NQ; ++q) mbar_init(bar(BAR_QEMPTY + q), 1);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(bar(BAR_SFULL + b), 1);
+            mbar_init(bar(BAR_PREADY + b), kGroupThreads);
+            mbar_init(bar(BAR_PFREE + b), 1);
+            mbar_init(bar(BAR_OFULL + b), 1);
+        }
+        mbar_init(bar(BAR_XFULL), kGroupThreads);
+        mbar_init(bar(BAR_XEMPTY), kGroupThreads);
         mbar_init(bar(BAR_DRAIN), 1);
+        *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == kMmaWarp) {
@@ -226,16 +355,10 @@ __global__ void __launch_bounds__(kThreads, 2) attend_umma_kernel(const AttendAr
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    // Q tile: rows row0 .. row0+127 of this (user, group), zero beyond M
-    {
-        const uint16_t* Q = reinterpret_cast<const uint16_t*>(a.queries);
-        for (int i = tid; i < 128 * 4; i += kThreads) {
-            const int r = i >> 2, c = i & 3;
-            uint4 v = make_uint4(0, 0, 0, 0);
-            if (row0 + r < rq.M)
-                v = __ldg(reinterpret_cast<const uint4*>(Q + ((int64_t)(rq.q0 + row0 + r) * G + grp) * D + c * 8));
-            *reinterpret_cast<uint4*>(smem + kOffQ + tile_off(r, c)) = v;
-        }
+    // the constant chunks 4 and 5 of every V stage: column 32 is one, columns 33..47 are zero
+    for (int i = tid; i < NS * TK * 2; i += kThreads) {
+        const int s = i / (TK * 2), r = (i >> 1) & (TK - 1), c = 4 + (i & 1);
+        *reinterpret_cast<uint4*>(smem + kOffV + s * kTileV + v_off(r, c)) = make_uint4(c == 4 ? 0x3f80u : 0u, 0u, 0u, 0u);
     }
     fence_proxy_async();
     tc_fence_before();
@@ -243,270 +366,426 @@ __global__ void __launch_bounds__(kThreads, 2) attend_umma_kernel(const AttendAr
     tc_fence_after();
     const uint32_t tmem = tmem_base_slot;
 
-    if (n_tiles > 0) {
-        if (warp < 4) {
-            // ------------------------------------------------------------- softmax / SiLU
-            const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
-            const float sc = a.scale * (MODE == CKV_SOFTMAX ? kLog2e : 0.5f);
-            float m_ref = -CUDART_INF_F, l_run = 0.f;
-            bool ok = true;
-            for (int j = 0; j < n_tiles && ok; ++j) {
-                ok = mbar_wait(bar(BAR_S), j & 1);
+    if (warp < 8) {
+        // --------------------------------------------------------------- normalisation groups
+        const int b = warp >> 2;                  // group = score buffer
+        const int row = tid & (kGroupThreads - 1);  // query row inside the block = TMEM lane
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t tS = tmem + lane_base + kColS + 128u * b, tP = tmem + lane_base + kColP + 64u * b,
+                       tO = tmem + lane_base + kColO + (uint32_t)kNV * b;
+        const float sc = a.scale * (MODE == CKV_SOFTMAX ? kLog2e : 0.5f);
+        float* xch = reinterpret_cast<float*>(smem + kOffX);
+        int cnt = 0;    // tiles this group has normalised
+        int ocnt = 0;   // units in which this group had tiles
+        int xcnt = 0;   // units exchanged between the groups
+        int g = 0;      // tiles of the stream before the current unit
+        bool ok = true;
+        for (int64_t w = blockIdx.x; w < n_work && ok; w += gridDim.x) {
+            Unit u;
+            load_unit(a, n_mb, w, u);
+            if (u.n_tiles < 0) continue;
+            const int r = u.row0 + row;
+            const int64_t out_base = ((int64_t)(u.rq.q0 + r) * G + u.grp) * D;
+            if (u.n_tiles == 0) {  // empty history: zero output rows
+                if (b == 0 && r < u.rq.M && u.it.part_row < 0) {
+                    if (a.out_dtype == CKV_BF16) {
+                        uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(a.out) + out_base);
+                        for (int q4 = 0; q4 < 4; ++q4) dst[q4] = make_uint4(0, 0, 0, 0);
+                    } else {
+                        float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(a.out) + out_base);
+                        for (int q4 = 0; q4 < 8; ++q4) dst[q4] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+                }
+                continue;
+            }
+            float m_ref = -CUDART_INF_F;
+            int mine = 0;  // tiles of this unit normalised by this group
+            for (int j = 0; j < u.n_tiles && ok; ++j) {
+                if (((g + j) & 1) != b) continue;
+                ok = mbar_wait(bar(BAR_SFULL + b), cnt & 1, abort_flag);
+                if (ok && cnt > 0) ok = mbar_wait(bar(BAR_PFREE + b), (cnt - 1) & 1, abort_flag);  // P_b and O_b are quiet
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 tc_fence_after();
-                const int valid = min(TK, it.len - j * TK);  // columns of this tile that are real positions
-                bool waited_pv = false;
+                const int valid = j == u.n_tiles - 1 ? u.last_valid : TK;
+                const bool tail = valid < TK;
                 if constexpr (MODE == CKV_SOFTMAX) {
-                    float tmax = -CUDART_INF_F;
+                    if (mine == 0) {  // the reference maximum: exact maximum of the first tile
+                        float tmax = -CUDART_INF_F;
 #pragma unroll 1
-                    for (int c = 0; c < 4; ++c) {
-                        uint32_t r[32];
-                        tmem_ld32(tmem + lane_base + kColS + 32 * c, r);
-                        tc_wait_ld();
-                        if (valid >= 32 * (c + 1)) {
+                        for (int c = 0; c < 4; ++c) {
+                            uint32_t s[32];
+                            tmem_ld32(tS + 32 * c, s);
+                            tmem_wait_ld32(s);
 #pragma unroll
-                            for (int e = 0; e < 32; ++e) tmax = fmaxf(tmax, __uint_as_float(r[e]));
-                        } else {
-#pragma unroll
-                            for (int e = 0; e < 32; ++e)
-                                if (32 * c + e < valid) tmax = fmaxf(tmax, __uint_as_float(r[e]));
+                            for (int e = 0; e < 32; e += 2) {
+                                float x0 = __uint_as_float(s[e]), x1 = __uint_as_float(s[e + 1]);
+                                if (tail) {
+                                    if (32 * c + e >= valid) x0 = -CUDART_INF_F;
+                                    if (32 * c + e + 1 >= valid) x1 = -CUDART_INF_F;
+                                }
+                                tmax = max3(tmax, x0, x1);
+                            }
                         }
+                        m_ref = tmax * sc;  // valid >= 1, so finite
                     }
-                    const float m_new = fmaxf(m_ref, tmax * sc);  // valid >= 1, so finite
-                    if (__any_sync(0xffffffffu, m_new > m_ref + kRescaleThreshold)) {
-                        if (j > 0) {
-                            ok = mbar_wait(bar(BAR_PV), (j - 1) & 1);
-                            ok = __all_sync(0xffffffffu, ok);
-                            if (!ok) break;
-                            waited_pv = true;
-                            tc_fence_after();
-                            const float f = ex2(m_ref - m_new);
+                    for (int attempt = 0; attempt < 2; ++attempt) {
+                        const float nm = -m_ref;
+                        float mx = -CUDART_INF_F;
+                        uint32_t sa[32], sb[32];
+                        tmem_ld32(tS, sa);
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            uint32_t(&cur)[32] = (c & 1) ? sb : sa;
+                            uint32_t(&nxt)[32] = (c & 1) ? sa : sb;
+                            tmem_wait_ld32(cur);
+                            if (c < 3) tmem_ld32(tS + 32 * (c + 1), nxt);
+                            uint32_t p[16];
+#pragma unroll
+                            for (int e = 0; e < 32; e += 2) {
+                                float x0 = fmaf(__uint_as_float(cur[e]), sc, nm), x1 = fmaf(__uint_as_float(cur[e + 1]), sc, nm);
+                                if (tail) {
+                                    if (32 * c + e >= valid) x0 = -CUDART_INF_F;
+                                    if (32 * c + e + 1 >= valid) x1 = -CUDART_INF_F;
+                                }
+                                mx = max3(mx, x0, x1);
+                                p[e >> 1] = pack_bf16(ex2(x0), ex2(x1));
+                            }
+                            tmem_st16(tP + 16 * c, p);
+                        }
+                        if (!__any_sync(0xffffffffu, mx > kHeadroom)) break;
+                        // some row of this warp left the headroom: move its reference, rescale what
+                        // O_b holds so far (its MMAs have finished, see the PFREE wait) and redo the tile
+                        const float shift = mx > kHeadroom ? mx : 0.f;
+                        const float f = ex2(-shift);
+                        m_ref += shift;
+                        if (mine > 0) {
                             uint32_t o[32];
-                            tmem_ld32(tmem + lane_base + kColO, o);
-                            tc_wait_ld();
+                            tmem_ld32(tO, o);
+                            tmem_wait_ld32(o);
 #pragma unroll
                             for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * f);
-                            tmem_st32(tmem + lane_base + kColO, o);
-                            l_run *= f;
+                            tmem_st32(tO, o);
+                            const uint32_t l = tmem_ld1(tO + 32);
+                            tmem_st1(tO + 32, __float_as_uint(__uint_as_float(l) * f));
                         }
-                        m_ref = m_new;
+                        tc_wait_st();
                     }
-                }
-                if (j > 0 && !waited_pv) {  // P buffer is free once PV of the previous tile has finished
-                    ok = mbar_wait(bar(BAR_PV), (j - 1) & 1);
-                    ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) break;
-                    tc_fence_after();
-                }
-#pragma unroll 1
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t r[32];
-                    tmem_ld32(tmem + lane_base + kColS + 32 * c, r);
-                    tc_wait_ld();
-                    uint32_t p[16];
-                    const bool full = valid >= 32 * (c + 1);
+                } else {
+                    // silu(x) = x sigmoid(x) = h (1 + tanh(h)), h = x / 2   (sc = scale / 2)
+                    uint32_t sa[32], sb[32];
+                    tmem_ld32(tS, sa);
 #pragma unroll
-                    for (int e = 0; e < 32; e += 2) {
-                        float w0, w1;
-                        if constexpr (MODE == CKV_SOFTMAX) {
-                            w0 = ex2(fmaf(__uint_as_float(r[e]), sc, -m_ref));
-                            w1 = ex2(fmaf(__uint_as_float(r[e + 1]), sc, -m_ref));
-                        } else {
-                            const float h0 = __uint_as_float(r[e]) * sc, h1 = __uint_as_float(r[e + 1]) * sc;
-                            w0 = fmaf(h0, tanh_fast(h0), h0);
-                            w1 = fmaf(h1, tanh_fast(h1), h1);
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t(&cur)[32] = (c & 1) ? sb : sa;
+                        uint32_t(&nxt)[32] = (c & 1) ? sa : sb;
+                        tmem_wait_ld32(cur);
+                        if (c < 3) tmem_ld32(tS + 32 * (c + 1), nxt);
+                        uint32_t p[16];
+#pragma unroll
+                        for (int e = 0; e < 32; e += 2) {
+                            const float h0 = __uint_as_float(cur[e]) * sc, h1 = __uint_as_float(cur[e + 1]) * sc;
+                            float w0 = fmaf(h0, tanh_fast(h0), h0), w1 = fmaf(h1, tanh_fast(h1), h1);
+                            if (tail) {
+                                if (32 * c + e >= valid) w0 = 0.f;
+                                if (32 * c + e + 1 >= valid) w1 = 0.f;
+                            }
+                            p[e >> 1] = pack_bf16(w0, w1);
                         }
-                        if (!full) {
-                            if (32 * c + e >= valid) w0 = 0.f;
-                            if (32 * c + e + 1 >= valid) w1 = 0.f;
-                        }
-                        if constexpr (MODE == CKV_SOFTMAX) l_run += w0 + w1;
-                        p[e >> 1] = pack_bf16(w0, w1);
+                        tmem_st16(tP + 16 * c, p);
                     }
-                    tmem_st16(tmem + lane_base + kColP + 16 * c, p);
                 }
                 tc_wait_st();
                 tc_fence_before();
-                mbar_arrive(bar(BAR_P));
+                mbar_arrive(bar(BAR_PREADY + b));
+                ++cnt;
+                ++mine;
             }
-            // epilogue: O is final once the last PV has finished
-            if (ok) {
-                ok = mbar_wait(bar(BAR_PV), (n_tiles - 1) & 1);
+            g += u.n_tiles;
+            if (!ok) break;
+
+            // ---- the unit's epilogue: fetch O_b, merge the two groups, store
+            float o[32], l = 0.f;
+            if (mine > 0) {
+                ok = mbar_wait(bar(BAR_OFULL + b), ocnt & 1, abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
-            }
-            if (ok) {
+                if (!ok) break;
+                ++ocnt;
                 tc_fence_after();
-                uint32_t o[32];
-                tmem_ld32(tmem + lane_base + kColO, o);
-                tc_wait_ld();
-                const int r = row0 + tid;
-                if (r < rq.M) {
-                    if (it.part_row < 0) {
+                uint32_t raw[32];
+                tmem_ld32(tO, raw);
+                tmem_wait_ld32(raw);
+#pragma unroll
+                for (int e = 0; e < 32; ++e) o[e] = __uint_as_float(raw[e]);
+                if constexpr (MODE == CKV_SOFTMAX) l = __uint_as_float(tmem_ld1(tO + 32));
+                tc_fence_before();
+            } else {
+#pragma unroll
+                for (int e = 0; e < 32; ++e) o[e] = 0.f;
+            }
+            if (b == 1) {
+                if (xcnt > 0) ok = mbar_wait(bar(BAR_XEMPTY), (xcnt - 1) & 1, abort_flag);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                xch[row] = m_ref;
+                xch[128 + row] = l;
+#pragma unroll
+                for (int e = 0; e < 32; ++e) xch[(2 + e) * 128 + row] = o[e];
+                mbar_arrive(bar(BAR_XFULL));
+                ++xcnt;
+            } else {
+                ok = mbar_wait(bar(BAR_XFULL), xcnt & 1, abort_flag);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                ++xcnt;
+                const float m1 = xch[row], l1 = xch[128 + row];
+                if constexpr (MODE == CKV_SOFTMAX) {
+                    const float mt = fmaxf(m_ref, m1);
+                    const float ms = mt == -CUDART_INF_F ? 0.f : mt;
+                    const float c0 = ex2(m_ref - ms), c1 = ex2(m1 - ms);
+                    l = l * c0 + l1 * c1;
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) o[e] = o[e] * c0 + xch[(2 + e) * 128 + row] * c1;
+                    m_ref = mt;
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) o[e] += xch[(2 + e) * 128 + row];
+                }
+                mbar_arrive(bar(BAR_XEMPTY));
+                if (r < u.rq.M) {
+                    if (u.it.part_row < 0) {
                         float inv;
-                        if constexpr (MODE == CKV_SOFTMAX) inv = l_run > 0.f ? 1.0f / l_run : 0.f;
-                        else inv = 1.0f / (float)rq.L;
-                        const int64_t base = ((int64_t)(rq.q0 + r) * G + grp) * D;
+                        if constexpr (MODE == CKV_SOFTMAX) inv = l > 0.f ? 1.0f / l : 0.f;
+                        else inv = 1.0f / (float)u.rq.L;
                         if (a.out_dtype == CKV_BF16) {
-                            uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(a.out) + base);
+                            uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(a.out) + out_base);
 #pragma unroll
                             for (int q4 = 0; q4 < 4; ++q4) {
                                 uint4 v;
-                                v.x = pack_bf16(__uint_as_float(o[8 * q4 + 0]) * inv, __uint_as_float(o[8 * q4 + 1]) * inv);
-                                v.y = pack_bf16(__uint_as_float(o[8 * q4 + 2]) * inv, __uint_as_float(o[8 * q4 + 3]) * inv);
-                                v.z = pack_bf16(__uint_as_float(o[8 * q4 + 4]) * inv, __uint_as_float(o[8 * q4 + 5]) * inv);
-                                v.w = pack_bf16(__uint_as_float(o[8 * q4 + 6]) * inv, __uint_as_float(o[8 * q4 + 7]) * inv);
+                                v.x = pack_bf16(o[8 * q4 + 0] * inv, o[8 * q4 + 1] * inv);
+                                v.y = pack_bf16(o[8 * q4 + 2] * inv, o[8 * q4 + 3] * inv);
+                                v.z = pack_bf16(o[8 * q4 + 4] * inv, o[8 * q4 + 5] * inv);
+                                v.w = pack_bf16(o[8 * q4 + 6] * inv, o[8 * q4 + 7] * inv);
                                 dst[q4] = v;
                             }
                         } else {
-                            float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(a.out) + base);
+                            float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(a.out) + out_base);
 #pragma unroll
                             for (int q4 = 0; q4 < 8; ++q4)
-                                dst[q4] = make_float4(__uint_as_float(o[4 * q4]) * inv, __uint_as_float(o[4 * q4 + 1]) * inv,
-                                                      __uint_as_float(o[4 * q4 + 2]) * inv, __uint_as_float(o[4 * q4 + 3]) * inv);
+                                dst[q4] = make_float4(o[4 * q4] * inv, o[4 * q4 + 1] * inv, o[4 * q4 + 2] * inv,
+                                                      o[4 * q4 + 3] * inv);
                         }
                     } else {
-                        float* pr = a.partials + ((int64_t)(it.part_row + r) * G + grp) * (D + 2);
+                        float* pr = a.partials + ((int64_t)(u.it.part_row + r) * G + u.grp) * (D + 2);
                         pr[0] = m_ref;
-                        pr[1] = l_run;
+                        pr[1] = l;
 #pragma unroll
-                        for (int e = 0; e < 32; ++e) pr[2 + e] = __uint_as_float(o[e]);
+                        for (int e = 0; e < 32; ++e) pr[2 + e] = o[e];
                     }
                 }
             }
-            if (!ok && lane == 0) atomicOr(err_flag, 1);
-        } else if (warp == kMmaWarp) {
-            // ------------------------------------------------------------- MMA issue
-            if (lane == 0) {
-                constexpr uint32_t idesc_s = make_idesc(128, TK, false);
-                constexpr uint32_t idesc_pv = make_idesc(128, D, true);
-                const uint32_t q_addr = sbase + kOffQ;
-                bool ok = true;
-                auto issue_pv = [&](int j) {  // O += P_j V_j, sixteen positions per instruction
-                    const uint32_t v_addr = sbase + kOffV + (j % NS) * kTileBytes;
-#pragma unroll
-                    for (int kk = 0; kk < TK / 16; ++kk)
-                        umma_ts(tmem + kColO, tmem + kColP + 8 * kk, smem_desc(v_addr + kk * 1024, 512, 128), idesc_pv,
-                                (j > 0 || kk > 0) ? 1u : 0u);
-                    tc_commit(bar(BAR_PV));
-                    tc_commit(bar(BAR_EMPTY + j % NS));
-                };
-                for (int j = 0; j < n_tiles; ++j) {
-                    ok = mbar_wait(bar(BAR_FULL + j % NS), (j / NS) & 1);
-                    if (ok && j > 0) ok = mbar_wait(bar(BAR_P), (j - 1) & 1);  // S free, P_{j-1} written
-                    if (!ok) break;
-                    tc_fence_after();
-                    const uint32_t k_addr = sbase + kOffK + (j % NS) * kTileBytes;
-#pragma unroll
-                    for (int ks = 0; ks < D / 16; ++ks)
-                        umma_ss(tmem + kColS, smem_desc(q_addr + ks * 256, 128, 512), smem_desc(k_addr + ks * 256, 128, 512),
-                                idesc_s, ks > 0 ? 1u : 0u);
-                    tc_commit(bar(BAR_S));
-                    if (j > 0) issue_pv(j - 1);
-                }
-                if (ok) ok = mbar_wait(bar(BAR_P), (n_tiles - 1) & 1);
-                if (ok) {
-                    tc_fence_after();
-                    issue_pv(n_tiles - 1);
-                } else {
-                    atomicOr(err_flag, 2);
-                }
-                // nothing of this CTA may still be running on the tensor core at teardown
-                tc_commit(bar(BAR_DRAIN));
-                if (!mbar_wait(bar(BAR_DRAIN), 0)) atomicOr(err_flag, 4);
-            }
-            __syncwarp();
-        } else {
-            // ------------------------------------------------------------- producers
-            const int p = tid - (kSoftmaxThreads + 32);  // 0..63
-            const char* poolK = reinterpret_cast<const char*>(a.cv.poolK) + (int64_t)grp * a.cv.n_entries * (D * 2);
-            const char* poolV = reinterpret_cast<const char*>(a.cv.poolV) + (int64_t)grp * a.cv.n_entries * (D * 2);
-            const int64_t unit0 = rq.base + (int64_t)grp * rq.Lpad + it.begin;
-            const int side_granules = (TK * d_user * 2) / 16;  // 16-byte pieces of one tile's user part
+        }
+        if (!ok) {
+            *abort_flag = 1;
+            if (lane == 0) atomicOr(err_flag, ERR_NORMALISE);
+        }
+    } else if (warp == kMmaWarp) {
+        // --------------------------------------------------------------------- MMA issue
+        if (lane == 0) {
+            constexpr uint32_t idesc_s = make_idesc(128, TK, false);
+            constexpr uint32_t idesc_pv = make_idesc(128, MODE == CKV_SOFTMAX ? kNV : D, true);
+            Stream ss, sp;  // next tile whose S / whose PV is to be issued
+            ss.init(&a, n_mb, n_work);
+            sp = ss;
+            int pcnt[2] = {0, 0};
             bool ok = true;
-            constexpr int LAG = 2;
-            for (int j = 0; j < n_tiles + LAG; ++j) {
-                // after a time-out nothing more is copied, but the loop keeps its shape so that
-                // every producer thread meets the same named barriers
-                if (j < n_tiles && ok && j >= NS) ok = mbar_wait(bar(BAR_EMPTY + (j % NS)), ((j / NS) - 1) & 1);
-                if (j < n_tiles && ok) {
-                    const int s = j % NS;
-                    const int valid = min(TK, it.len - j * TK);
+            auto issue_s = [&]() {
+                const int s = ss.g % NS, b = ss.g & 1;
+                if (!mbar_wait(bar(BAR_FULL + s), (ss.g / NS) & 1, abort_flag)) return false;
+                tc_fence_after();
+                const uint32_t q_addr = sbase + kOffQ + (ss.useq % NQ) * kTileK, k_addr = sbase + kOffK + s * kTileK;
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        const int r = p + 64 * h;
-                        int ik = 0, iv = 0;
-                        if (r < valid) {
-                            const int64_t u = unit0 + (int64_t)j * TK + r;
-                            if constexpr (IDX16) {
-                                ik = __ldg(reinterpret_cast<const uint16_t*>(a.cv.idxK) + u);
-                                iv = __ldg(reinterpret_cast<const uint16_t*>(a.cv.idxV) + u);
-                            } else {
-                                ik = __ldg(reinterpret_cast<const int32_t*>(a.cv.idxK) + u);
-                                iv = __ldg(reinterpret_cast<const int32_t*>(a.cv.idxV) + u);
-                            }
-                        }
-                        const char* ksrc = poolK + (int64_t)ik * (D * 2);
-                        const char* vsrc = poolV + (int64_t)iv * (D * 2);
-                        const uint32_t kdst = sbase + kOffK + s * kTileBytes, vdst = sbase + kOffV + s * kTileBytes;
+                for (int ks = 0; ks < D / 16; ++ks)
+                    umma_ss(tmem + kColS + 128u * b, smem_desc(q_addr + ks * 256, 128, 512),
+                            smem_desc(k_addr + ks * 256, 128, 512), idesc_s, ks > 0 ? 1u : 0u);
+                tc_commit(bar(BAR_SFULL + b));
+                if (ss.j == ss.u.n_tiles - 1) tc_commit(bar(BAR_QEMPTY + ss.useq % NQ));  // Q buffer no longer read
+                ss.advance();
+                return true;
+            };
+            auto issue_pv = [&]() {  // O_b += P_b [V | 1], sixteen positions per instruction
+                const int s = sp.g % NS, b = sp.g & 1;
+                if (!mbar_wait(bar(BAR_PREADY + b), pcnt[b] & 1, abort_flag)) return false;
+                ++pcnt[b];
+                tc_fence_after();
+                const uint32_t v_addr = sbase + kOffV + s * kTileV;
 #pragma unroll
-                        for (int c = 0; c < 4; ++c) {
-                            cp_async16(kdst + tile_off(r, c), ksrc + 16 * c);
-                            cp_async16(vdst + tile_off(r, c), vsrc + 16 * c);
-                        }
-                    }
-                    // the tile's user-specific parts: contiguous in the cache, copied as they are
-                    const int64_t pos0 = (int64_t)it.begin + (int64_t)j * TK;
-                    for (int gr = p; gr < side_granules; gr += kProducerThreads) {
-                        const int64_t first_pos = pos0 + (int64_t)gr * 8 / d_user;
-                        if (first_pos < rq.Lpad) {
-                            const int64_t byte = ((unit0 + (int64_t)j * TK) * d_user) * 2 + (int64_t)gr * 16;
-                            cp_async16(sbase + kOffSideK + s * kSideBytes + gr * 16, reinterpret_cast<const char*>(a.cv.userK) + byte);
-                            cp_async16(sbase + kOffSideV + s * kSideBytes + gr * 16, reinterpret_cast<const char*>(a.cv.userV) + byte);
-                        }
-                    }
+                for (int kk = 0; kk < TK / 16; ++kk)
+                    umma_ts(tmem + kColO + (uint32_t)kNV * b, tmem + kColP + 64u * b + 8 * kk,
+                            smem_desc(v_addr + kk * 2 * kVGroup, kVGroup, 128), idesc_pv, (sp.j >= 2 || kk > 0) ? 1u : 0u);
+                tc_commit(bar(BAR_EMPTY + s));
+                tc_commit(bar(BAR_PFREE + b));
+                if (sp.j >= sp.u.n_tiles - 2) tc_commit(bar(BAR_OFULL + b));  // last tile of its group in the unit
+                sp.advance();
+                return true;
+            };
+            if (ss.valid) ok = issue_s();
+            if (ok && ss.valid) ok = issue_s();
+            while (ok && sp.valid) {
+                ok = issue_pv();
+                if (ok && ss.valid) ok = issue_s();
+            }
+            if (!ok) {
+                *abort_flag = 1;
+                atomicOr(err_flag, ERR_MMA);
+            }
+            // nothing of this CTA may still be running on the tensor core at teardown
+            tc_commit(bar(BAR_DRAIN));
+            volatile int never = 0;
+            if (!mbar_wait(bar(BAR_DRAIN), 0, &never)) atomicOr(err_flag, ERR_DRAIN);
+        }
+        __syncwarp();
+    } else {
+        // --------------------------------------------------------------------- producers
+        const int p = tid - kProducerWarp0 * 32;  // 0..127 = the tile row this thread owns
+        const int pw = p >> 5;
+        const int du_bytes = a.cv.d_user * 2;
+        const int src_lane0 = lane >> 2, chunk = lane & 3;
+        Stream st;
+        st.init(&a, n_mb, n_work);
+        bool ok = true;
+        // per tile in flight: where it went and this thread's user-specific leading elements
+        uint4 uk[LAG], uv[LAG];
+        int stage_of[LAG];
+        bool patch[LAG], live[LAG];
+#pragma unroll
+        for (int u = 0; u < LAG; ++u) {
+            live[u] = false;
+            patch[u] = false;
+            stage_of[u] = 0;
+            uk[u] = uv[u] = make_uint4(0, 0, 0, 0);
+        }
+        // indices of the next tile to issue, loaded one iteration ahead
+        int ik = 0, iv = 0;
+        int64_t my_unit = 0;
+        bool my_valid = false;
+        auto prefetch = [&]() {
+            if (!st.valid) return;
+            const int valid = st.j == st.u.n_tiles - 1 ? st.u.last_valid : TK;
+            my_valid = p < valid;
+            my_unit = st.u.rq.base + (int64_t)st.u.grp * st.u.rq.Lpad + st.u.it.begin + (int64_t)st.j * TK + p;
+            ik = iv = 0;
+            if (my_valid) {
+                if constexpr (IDX16) {
+                    ik = __ldg(reinterpret_cast<const uint16_t*>(a.cv.idxK) + my_unit);
+                    iv = __ldg(reinterpret_cast<const uint16_t*>(a.cv.idxV) + my_unit);
+                } else {
+                    ik = __ldg(reinterpret_cast<const int32_t*>(a.cv.idxK) + my_unit);
+                    iv = __ldg(reinterpret_cast<const int32_t*>(a.cv.idxV) + my_unit);
                 }
-                cp_async_commit();
-                if (j >= LAG) {
-                    const int jj = j - LAG, s = jj % NS;
-                    cp_async_wait<LAG>();
-                    asm volatile("bar.sync 1, %0;" ::"n"(kProducerThreads) : "memory");  // side buffers are shared work
-                    if (d_user > 0) {
-                        const int valid = min(TK, it.len - jj * TK);
+            }
+        };
+        prefetch();
+        bool more = true;
+        while (more) {
+            more = false;
 #pragma unroll
-                        for (int h = 0; h < 2; ++h) {
-                            const int r = p + 64 * h;
-                            if (r < valid) {  // Eq. K: dims [0, d_user) come from the user part
-                                const uint16_t* sk = reinterpret_cast<const uint16_t*>(smem + kOffSideK + s * kSideBytes) + r * d_user;
-                                const uint16_t* sv = reinterpret_cast<const uint16_t*>(smem + kOffSideV + s * kSideBytes) + r * d_user;
-                                uint16_t* kd = reinterpret_cast<uint16_t*>(smem + kOffK + s * kTileBytes + tile_off(r, 0));
-                                uint16_t* vd = reinterpret_cast<uint16_t*>(smem + kOffV + s * kTileBytes + tile_off(r, 0));
-                                for (int e = 0; e < d_user; ++e) {
-                                    kd[e] = sk[e];
-                                    vd[e] = sv[e];
-                                }
-                            }
+            for (int u = 0; u < LAG; ++u) {
+                // (1) the tile issued LAG iterations ago has landed: patch and publish it
+                if (live[u]) {
+                    cp_async_wait<LAG - 1>();
+                    __syncwarp();  // a row's chunks were copied by four other lanes of this warp
+                    if (patch[u]) {  // Eq. K: dims [0, d_user) come from the user part
+                        unsigned char* kd = smem + kOffK + stage_of[u] * kTileK + k_off(p, 0);
+                        unsigned char* vd = smem + kOffV + stage_of[u] * kTileV + v_off(p, 0);
+                        if (du_bytes == 4) {
+                            *reinterpret_cast<uint32_t*>(kd) = uk[u].x;
+                            *reinterpret_cast<uint32_t*>(vd) = uv[u].x;
+                        } else if (du_bytes == 2) {
+                            *reinterpret_cast<uint16_t*>(kd) = (uint16_t)uk[u].x;
+                            *reinterpret_cast<uint16_t*>(vd) = (uint16_t)uv[u].x;
+                        } else if (du_bytes == 8) {
+                            *reinterpret_cast<uint2*>(kd) = make_uint2(uk[u].x, uk[u].y);
+                            *reinterpret_cast<uint2*>(vd) = make_uint2(uv[u].x, uv[u].y);
+                        } else {
+                            *reinterpret_cast<uint4*>(kd) = uk[u];
+                            *reinterpret_cast<uint4*>(vd) = uv[u];
                         }
                     }
                     fence_proxy_async();
-                    mbar_arrive(bar(BAR_FULL + s));
+                    mbar_arrive(bar(BAR_FULL + stage_of[u]));
+                    live[u] = false;
                 }
+                // (2) issue the copies of the next tile of the stream
+                if (st.valid && ok) {
+                    const int s = st.g % NS;
+                    if (st.g >= NS) ok = mbar_wait(bar(BAR_EMPTY + s), ((st.g / NS) - 1) & 1, abort_flag);
+                    if (ok && st.j == 0) {  // a new unit: stage its Q block (rows beyond M are zero)
+                        if (st.useq >= NQ) ok = mbar_wait(bar(BAR_QEMPTY + st.useq % NQ), ((st.useq / NQ) - 1) & 1, abort_flag);
+                        if (ok) {
+                            const uint32_t qdst = sbase + kOffQ + (st.useq % NQ) * kTileK;
+                            const uint16_t* Q = reinterpret_cast<const uint16_t*>(a.queries);
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                const int r = 32 * pw + 8 * i + src_lane0;
+                                const bool in = st.u.row0 + r < st.u.rq.M;
+                                const uint16_t* src = Q + ((int64_t)(st.u.rq.q0 + st.u.row0 + (in ? r : 0)) * G + st.u.grp) * D + chunk * 8;
+                                cp_async16(qdst + k_off(r, chunk), src, in ? 16u : 0u);
+                            }
+                        }
+                    }
+                    if (ok) {
+                        const char* poolK = reinterpret_cast<const char*>(a.cv.poolK) + (int64_t)st.u.grp * a.cv.n_entries * (D * 2);
+                        const char* poolV = reinterpret_cast<const char*>(a.cv.poolV) + (int64_t)st.u.grp * a.cv.n_entries * (D * 2);
+                        const uint32_t kdst = sbase + kOffK + s * kTileK, vdst = sbase + kOffV + s * kTileV;
+                        const uint32_t vbits = __ballot_sync(0xffffffffu, my_valid);
+                        // four lanes fetch the four 16-byte chunks of one row: 64 contiguous bytes per row
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const int sl = 8 * i + src_lane0;
+                            const int rk = __shfl_sync(0xffffffffu, ik, sl), rv = __shfl_sync(0xffffffffu, iv, sl);
+                            const uint32_t nb = (vbits >> sl) & 1u ? 16u : 0u;  // rows beyond the history are zero
+                            const int r = 32 * pw + sl;
+                            cp_async16(kdst + k_off(r, chunk), poolK + (int64_t)rk * (D * 2) + chunk * 16, nb);
+                            cp_async16(vdst + v_off(r, chunk), poolV + (int64_t)rv * (D * 2) + chunk * 16, nb);
+                        }
+                        patch[u] = my_valid && du_bytes > 0;
+                        if (patch[u]) {
+                            const char* ku = reinterpret_cast<const char*>(a.cv.userK) + my_unit * du_bytes;
+                            const char* vu = reinterpret_cast<const char*>(a.cv.userV) + my_unit * du_bytes;
+                            if (du_bytes == 4) {
+                                uk[u].x = __ldg(reinterpret_cast<const uint32_t*>(ku));
+                                uv[u].x = __ldg(reinterpret_cast<const uint32_t*>(vu));
+                            } else if (du_bytes == 2) {
+                                uk[u].x = __ldg(reinterpret_cast<const uint16_t*>(ku));
+                                uv[u].x = __ldg(reinterpret_cast<const uint16_t*>(vu));
+                            } else if (du_bytes == 8) {
+                                const uint2 x = __ldg(reinterpret_cast<const uint2*>(ku)), y = __ldg(reinterpret_cast<const uint2*>(vu));
+                                uk[u] = make_uint4(x.x, x.y, 0, 0);
+                                uv[u] = make_uint4(y.x, y.y, 0, 0);
+                            } else {
+                                uk[u] = __ldg(reinterpret_cast<const uint4*>(ku));
+                                uv[u] = __ldg(reinterpret_cast<const uint4*>(vu));
+                            }
+                        }
+                        stage_of[u] = s;
+                        live[u] = true;
+                        st.advance();
+                        prefetch();
+                    }
+                }
+                cp_async_commit();  // one group per iteration, also when nothing was issued
+                more = more || live[u];
             }
-            if (!ok) atomicOr(err_flag, 8);
-            cp_async_wait<0>();
+            more = more || (st.valid && ok);
+        }
+        cp_async_wait<0>();
+        if (!ok) {
+            *abort_flag = 1;
+            if (lane == 0) atomicOr(err_flag, ERR_PRODUCER);
         }
     }
 
-    if (n_tiles == 0 && warp < 4 && row0 + tid < rq.M && it.part_row < 0) {  // empty history: zero output row
-        const int64_t base = ((int64_t)(rq.q0 + row0 + tid) * G + grp) * D;
-        if (a.out_dtype == CKV_BF16) {
-            uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(a.out) + base);
-            for (int q4 = 0; q4 < 4; ++q4) dst[q4] = make_uint4(0, 0, 0, 0);
-        } else {
-            float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(a.out) + base);
-            for (int q4 = 0; q4 < 8; ++q4) dst[q4] = make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-    }
     tc_fence_before();
     __syncthreads();
     if (warp == kMmaWarp) {
@@ -519,19 +798,20 @@ __global__ void __launch_bounds__(kThreads, 2) attend_umma_kernel(const AttendAr
 
 bool umma_supported(int dtype, int head_dim, int d_user)
 {
-    return dtype == CKV_BF16 && head_dim == D && d_user <= kMaxDu && (d_user == 0 || 8 % d_user == 0);
+    return dtype == CKV_BF16 && head_dim == D && (d_user == 0 || d_user == 1 || d_user == 2 || d_user == 4 || d_user == 8);
 }
 
-cudaError_t launch_attend_umma(int max_M, const AttendArgs& a, int* err_flag, cudaStream_t s)
+cudaError_t launch_attend_umma(int max_M, const AttendArgs& a, int n_sms, int* err_flag, cudaStream_t s)
 {
     if (a.n_items == 0) return cudaSuccess;
     const int n_mb = (max_M + 127) / 128;
-    const dim3 grid((unsigned)((int64_t)a.n_items * n_mb), a.cv.n_groups);
+    const int64_t n_work = (int64_t)a.n_items * n_mb * a.cv.n_groups;
+    const unsigned grid = (unsigned)(n_work < n_sms ? n_work : n_sms);
     const bool i16 = a.cv.idx_bytes == 2;
     auto go = [&](auto kernel) {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (e != cudaSuccess) return e;
-        kernel<<<grid, kThreads, kSmemBytes, s>>>(a, n_mb, err_flag);
+        kernel<<<grid, kThreads, kSmemBytes, s>>>(a, n_mb, n_work, err_flag);
         return cudaGetLastError();
     };
     if (a.mode == CKV_SOFTMAX)

@@ -61,6 +61,22 @@ def test_tensor_core_kernels_user_widths_and_sharp_softmax(kernel, mode, d_user)
     assert_close(got, oracle_attend(w, d, scale=scale), "bf16", f"d_user={d_user}")
 
 
+@pytest.mark.parametrize("mode", ["softmax", "silu_over_l"])
+@pytest.mark.parametrize("n_queries", [70, 150])
+def test_persistent_tcgen05_kernel_many_units_per_sm(mode, n_queries):
+    """More work units than SMs, one to six tiles each: every buffer of the kernel is reused
+    across unit boundaries (tile stages, Q buffers, both accumulators)."""
+    w = synth.Workload("many", 8, 30, 2, 500, 110, (1, 700), n_queries, mode, "bf16", 1.1, 1 / 32, 1 / 32, 41)
+    d = synth.generate(w)
+    s = make_session(w, d, kernel=3)
+    got = gpu_attend(w, d, session=s)
+    again = gpu_attend(w, d, session=s)
+    assert s.stat("kernel") == 3 and s.stat("device_errors") == 0
+    s.close()
+    assert np.array_equal(got, again), "run-to-run bitwise reproducibility"
+    assert_close(got, oracle_attend(w, d), "bf16", f"{mode} M={n_queries}")
+
+
 def test_growing_maximum_triggers_rescale_in_tcgen05_kernel():
     """Keys sorted by increasing score make every tile raise the running maximum."""
     w = synth.Workload("grow", 1, 30, 2, 512, 2, (1024, 1024), 128, "softmax", "bf16", None, 1.0, 1.0, 33)

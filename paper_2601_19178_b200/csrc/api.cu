@@ -31,10 +31,11 @@ struct Plan {
     std::vector<int32_t> q_off;
     uint64_t generation = 0;
     int64_t opt_split = 0, opt_kernel = 0;
-    void* dev = nullptr;  // one allocation: reqs | items | split list
+    void* dev = nullptr;  // one allocation: reqs | items | split list | works
     Req* d_reqs = nullptr;
     Item* d_items = nullptr;
     int32_t* d_split = nullptr;
+    Work* d_works = nullptr;
     int32_t n_items = 0, n_split = 0, split_items = 0, max_M = 0, family = 1;
     int64_t part_rows = 0;
     uint64_t last_use = 0;
@@ -303,13 +304,25 @@ ckv_status build_plan(ckv_ctx* ctx, Plan& pl, int32_t n, const int64_t* users, c
     for (const Item& it : items) pl.split_items += it.part_row >= 0;
     pl.part_rows = part_rows;
 
+    std::vector<Work> works;
+    if (pl.family == 3) {
+        works.resize(items.size());
+        for (size_t i = 0; i < items.size(); ++i) {
+            const Item& it = items[i];
+            const Req& r = reqs[it.req];
+            works[i] = Work{r.base, r.L, r.Lpad, r.q0, r.M, it.begin, it.len, it.part_row, {0, 0, 0}};
+        }
+    }
     const size_t b_req = sizeof(Req) * reqs.size(), b_item = sizeof(Item) * items.size(),
-                 b_split = sizeof(int32_t) * split.size();
-    const size_t o_item = (b_req + 255) / 256 * 256, o_split = o_item + (b_item + 255) / 256 * 256;
-    CK(cudaMalloc(&pl.dev, o_split + b_split + 256));
+                 b_split = sizeof(int32_t) * split.size(), b_work = sizeof(Work) * works.size();
+    const size_t o_item = (b_req + 255) / 256 * 256, o_split = o_item + (b_item + 255) / 256 * 256,
+                 o_work = o_split + (b_split + 255) / 256 * 256;
+    CK(cudaMalloc(&pl.dev, o_work + b_work + 256));
     pl.d_reqs = (Req*)pl.dev;
     pl.d_items = (Item*)((char*)pl.dev + o_item);
     pl.d_split = (int32_t*)((char*)pl.dev + o_split);
+    pl.d_works = (Work*)((char*)pl.dev + o_work);
+    if (b_work) CK(cudaMemcpyAsync(pl.d_works, works.data(), b_work, cudaMemcpyHostToDevice, s));
     if (b_req) CK(cudaMemcpyAsync(pl.d_reqs, reqs.data(), b_req, cudaMemcpyHostToDevice, s));
     if (b_item) CK(cudaMemcpyAsync(pl.d_items, items.data(), b_item, cudaMemcpyHostToDevice, s));
     if (b_split) CK(cudaMemcpyAsync(pl.d_split, split.data(), b_split, cudaMemcpyHostToDevice, s));
@@ -605,6 +618,7 @@ ckv_status ckv_attend(ckv_ctx* ctx, int32_t n, const int64_t* users, const int32
     a.cv = view_of(ctx);
     a.reqs = pl->d_reqs;
     a.items = pl->d_items;
+    a.works = pl->d_works;
     a.n_items = pl->n_items;
     a.queries = d_q;
     a.out = d_out;
@@ -895,6 +909,7 @@ extern "C" ckv_status ckv_attend_static(ckv_ctx* ctx, int32_t n, const int64_t* 
     a.cv = view_of(ctx);
     a.reqs = (const Req*)base;
     a.items = (const Item*)(base + kOffItems);
+    a.works = nullptr;
     a.n_items = n_items;
     a.queries = queries;
     a.out = out;

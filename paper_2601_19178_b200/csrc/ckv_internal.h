@@ -28,6 +28,16 @@ struct Item {
     int32_t part_row;  // first row of this chunk's partial results, or -1: write `out`
 };
 
+// An Item merged with its request row, for kernels that read their work list once per unit
+// with plain 16-byte loads (48 bytes, 16-byte aligned).
+struct Work {
+    int64_t base;      // Req::base
+    int32_t L, Lpad;   // Req::L, Req::Lpad
+    int32_t q0, M;     // Req::q0, Req::M
+    int32_t begin, len, part_row;  // Item::begin, Item::len, Item::part_row
+    int32_t pad[3];
+};
+
 // Everything a kernel needs to find the compressed cache and the pool.
 struct CacheView {
     const void* poolK;   // [G][m][D] rows, first d_user slots zero
@@ -46,6 +56,7 @@ struct AttendArgs {
     CacheView cv;
     const Req* reqs;
     const Item* items;
+    const Work* works;     // one per item, same order (tcgen05 family only, else null)
     int32_t n_items;
     const void* queries;   // [Q][G][D]
     void* out;             // [Q][G][D]

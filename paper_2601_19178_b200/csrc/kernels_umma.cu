@@ -2,12 +2,14 @@
 //
 // Persistent: one CTA per SM walks a static round-robin share of the work units, where a unit
 // is (work item = history chunk of one user, group, block of up to 128 queries).  The history
-// chunk is processed in tiles of 128 positions.  Roles (warp-specialised, 13 warps):
+// chunk is processed in tiles of 128 positions.  Roles (warp-specialised, 15 warps):
 //   warps 0-3   normalisation group 0: thread i owns query row i = TMEM lane i, even tiles
 //   warps 4-7   normalisation group 1: the same rows, odd tiles
-//   warp  8     issues tcgen05.mma (one thread), owns the TMEM allocation
-//   warps 9-12  producers: gather pool rows into shared memory with 16-byte cp.async, patch the
-//               user-specific leading elements (Eq. K), publish the tile; also stage Q
+//   warp  8     issues the score MMAs (one thread), owns the TMEM allocation
+//   warps 9-10  issue the weighted-sum MMAs of score buffer 0 and 1 (one thread each)
+//   warps 11-14 producers, one tile each in turn: gather pool rows into shared memory with
+//               16-byte cp.async, patch the user-specific leading elements (Eq. K), publish the
+//               tile; the owner of a unit's first tile also stages Q
 //
 // Tile t of the CTA's tile stream uses score buffer b = t mod 2:
 //   S_b  = Q K_t^T                    UMMA 128 x 128 x 32, A = Q smem, B = K tile smem (K-major)
@@ -18,12 +20,18 @@
 // groups keep separate accumulators O_0, O_1 with separate reference maxima and merge them
 // through shared memory when a unit ends.
 //
+// Why three issuing warps: one thread hands a tcgen05.mma to the tensor core about every
+// hundred cycles whatever the instruction's size, and a tile needs ten of these small ones
+// (K = 16 per instruction).  Why one producer warp per tile: the bookkeeping of a tile (stream
+// position, waits, index and user-part loads) is a serial chain of a few hundred instructions;
+// paid by every producer warp for every tile it was the bottleneck of the whole pipeline.
+//
 // Softmax bookkeeping.  The V tile carries sixteen extra columns of which the first is all
 // ones, so column 32 of O_b accumulates the row sum l of exactly the bf16-rounded P that
-// multiplies V.  The reference maximum m of a row is the exact maximum of the group's first
-// tile of the unit and stays fixed: later scores may exceed it by up to 2^64 (fp32
-// accumulators and bf16 P have the exponent range for that); only when a tile exceeds that
-// bound is O_b rescaled (TMEM read-modify-write) and the tile redone.
+// multiplies V.  The reference maximum m of a row is the largest of the first 32 scores of the
+// group's first tile of the unit and stays fixed: later scores may exceed it by up to 2^64
+// (fp32 accumulators and bf16 P have the exponent range for that); only when a tile exceeds
+// that bound is O_b rescaled (TMEM read-modify-write) and the tile redone.
 //
 // Shared-memory tiles use the no-swizzle UMMA canonical layout: groups of 8 rows, inside a
 // group one 128-byte core matrix per 16-byte row chunk, inside a core matrix row r%8 at 16 r.
@@ -35,6 +43,9 @@
 // returns.
 #include <cuda_bf16.h>
 #include <math_constants.h>
+#ifdef CKV_STAGE_TIMERS
+#include <cstdio>
+#endif
 
 #include "ckv_internal.h"
 
@@ -44,16 +55,13 @@ namespace {
 constexpr int D = 32;
 constexpr int TK = 128;                  // positions per tile
 constexpr int NS = 6;                    // K/V stages
-constexpr int LAG = 3;                   // tiles whose copies are in flight per producer thread
 constexpr int NQ = 3;                    // Q buffers
-// A producer publishes tile t - LAG before it issues tile t.  Q buffer reuse waits for the unit
-// NQ units back, whose last tile is at most t - NQ: published already iff NQ >= LAG.
-static_assert(NQ >= LAG, "Q buffer reuse would wait for a tile that is not published yet");
 constexpr int kGroupThreads = 128;       // one normalisation group
-constexpr int kMmaWarp = 8;
-constexpr int kProducerWarp0 = 9;
-constexpr int kProducerThreads = 128;
-constexpr int kThreads = 2 * kGroupThreads + 32 + kProducerThreads;  // 416
+constexpr int kMmaWarp = 8;              // issues S = Q K^T, owns the TMEM allocation
+constexpr int kPvWarp0 = 9;              // warps 9, 10 issue the weighted sums of buffer 0, 1
+constexpr int kProducerWarp0 = 11;
+constexpr int kProducerWarps = 4;        // each owns every fourth tile of the stream
+constexpr int kThreads = 2 * kGroupThreads + 3 * 32 + kProducerWarps * 32;  // 480
 constexpr int kTileK = TK * D * 2;       // 8 KB, also the Q tile
 constexpr int kVGroup = 768;             // bytes of one 8-row group of a V tile
 constexpr int kTileV = (TK / 8) * kVGroup;  // 12 KB
@@ -62,7 +70,9 @@ constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColS = 0, kColP = 256, kColO = 384;  // S_b at kColS + 128 b, P_b at kColP + 64 b, O_b at kColO + 48 b
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kHeadroom = 64.0f;       // log2 units a score may exceed the reference maximum
-constexpr uint32_t kSpinLimit = 1u << 20;
+constexpr uint32_t kSpinLimit = 1u << 16;  // polls of a wait before the CTA gives up
+constexpr uint32_t kSuspendNs = 20000;     // how long one poll may stay suspended in hardware
+static_assert(NS > kProducerWarps, "every producer warp holds one stage while it copies");
 
 // dynamic shared memory map
 constexpr int kOffQ = 0;
@@ -76,7 +86,8 @@ constexpr int kSmemBytes = kOffAbort + 16;
 // barrier slots (8 bytes each) behind kOffBar
 enum {
     BAR_FULL = 0, BAR_EMPTY = NS, BAR_QEMPTY = 2 * NS, BAR_SFULL = 2 * NS + NQ, BAR_PREADY = BAR_SFULL + 2,
-    BAR_PFREE = BAR_SFULL + 4, BAR_OFULL = BAR_SFULL + 6, BAR_XFULL = BAR_SFULL + 8, BAR_XEMPTY, BAR_DRAIN, BAR_COUNT
+    BAR_PFREE = BAR_SFULL + 4, BAR_OFULL = BAR_SFULL + 6, BAR_XFULL = BAR_SFULL + 8, BAR_XEMPTY, BAR_DRAIN,
+    BAR_COUNT = BAR_DRAIN + 3
 };
 static_assert(BAR_COUNT * 8 <= 256, "barrier area");
 
@@ -100,13 +111,13 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const v
         uint32_t ok;
         asm volatile(
             "{\n.reg .pred p;\n"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
             "selp.u32 %0, 1, 0, p;\n}\n"
             : "=r"(ok)
-            : "r"(bar), "r"(parity)
+            : "r"(bar), "r"(parity), "r"(kSuspendNs)
             : "memory");
         if (ok) return true;
-        if ((i & 63u) == 63u && *abort_flag) return false;
+        if (*abort_flag) return false;
     }
     return false;
 }
@@ -246,66 +257,215 @@ __device__ __forceinline__ float max3(float a, float b, float c)
     return r;
 }
 
+// Optional stage timers (debug builds with -DCKV_STAGE_TIMERS): one thread per role of CTA 0
+// accumulates clock64 intervals per stage and prints them when the kernel ends.
+#ifdef CKV_STAGE_TIMERS
+#define T_DECL(n) long long tmr_[n] = {}; long long tmr_last_ = clock64(); const long long tmr_start_ = tmr_last_
+#define T_ACC(i) do { const long long t_now_ = clock64(); tmr_[i] += t_now_ - tmr_last_; tmr_last_ = t_now_; } while (0)
+#define T_TOTAL() (clock64() - tmr_start_)
+#else
+#define T_DECL(n) do {} while (0)
+#define T_ACC(i) do {} while (0)
+#endif
+
 // byte offset of (row r, 16-byte chunk c) inside a K/Q tile and inside a V tile
 __device__ __forceinline__ uint32_t k_off(int r, int c) { return (uint32_t)((r >> 3) * 512 + c * 128 + (r & 7) * 16); }
 __device__ __forceinline__ uint32_t v_off(int r, int c) { return (uint32_t)((r >> 3) * kVGroup + c * 128 + (r & 7) * 16); }
 
-// One work unit of the CTA's share.
+// Inside a tile the producers place history position 32 c + 4 q + i (q < 8, i < 4) in row
+// 32 c + 8 i + q: a lane then reads the indices of four consecutive positions with one load and
+// its four 16-byte copies of an instruction still fall into different shared-memory banks.
+// Attention does not depend on the order of positions; only the tail mask has to know which
+// position a score column belongs to.
+__device__ __forceinline__ int pos_of_col(int c, int e) { return 32 * c + 4 * (e & 7) + (e >> 3); }
+
+// ---- normalisation of one 128 x 128 score tile by its group (thread = query row = TMEM lane) ----
+// TAIL = false: all 128 columns are real positions; the 32-column chunks are double-buffered
+// in registers so that the next tcgen05.ld is in flight during the arithmetic.
+// TAIL = true (last tile of a history, at most once per unit): compact code, masked columns.
+
+// p = exp2(s c - m) as bf16 into P; returns the largest exponent argument of the row.  With
+// `first` the row's reference m is set from its first 32 scores (column 0 is position 0, always
+// a real one).
+template <bool TAIL>
+__device__ __forceinline__ float softmax_tile(uint32_t tS, uint32_t tP, float sc, int valid, bool first, float& m_ref)
+{
+    float nm = -m_ref;
+    float mx = -CUDART_INF_F, mx2 = -CUDART_INF_F;
+    auto chunk = [&](const uint32_t (&cur)[32], int c) {
+        if (c == 0 && first) {
+            float t0 = -CUDART_INF_F, t1 = -CUDART_INF_F;
+#pragma unroll
+            for (int e = 0; e < 32; e += 4) {
+                float x[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    x[i] = (TAIL && pos_of_col(0, e + i) >= valid) ? -CUDART_INF_F : __uint_as_float(cur[e + i]);
+                t0 = max3(t0, x[0], x[1]);
+                t1 = max3(t1, x[2], x[3]);
+            }
+            m_ref = fmaxf(t0, t1) * sc;
+            nm = -m_ref;
+        }
+        uint32_t p[16];
+#pragma unroll
+        for (int e = 0; e < 32; e += 2) {
+            float x0 = fmaf(__uint_as_float(cur[e]), sc, nm), x1 = fmaf(__uint_as_float(cur[e + 1]), sc, nm);
+            if (TAIL) {
+                if (pos_of_col(c, e) >= valid) x0 = -CUDART_INF_F;
+                if (pos_of_col(c, e + 1) >= valid) x1 = -CUDART_INF_F;
+            }
+            if (e & 2) mx = max3(mx, x0, x1);
+            else mx2 = max3(mx2, x0, x1);
+            p[e >> 1] = pack_bf16(ex2(x0), ex2(x1));
+        }
+        tmem_st16(tP + 16 * c, p);
+    };
+    if constexpr (TAIL) {
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+            uint32_t cur[32];
+            tmem_ld32(tS + 32 * c, cur);
+            tmem_wait_ld32(cur);
+            chunk(cur, c);
+        }
+    } else {
+        uint32_t sa[32], sb[32];
+        tmem_ld32(tS, sa);
+        tmem_wait_ld32(sa);
+        tmem_ld32(tS + 32, sb);
+        chunk(sa, 0);
+        tmem_wait_ld32(sb);
+        tmem_ld32(tS + 64, sa);
+        chunk(sb, 1);
+        tmem_wait_ld32(sa);
+        tmem_ld32(tS + 96, sb);
+        chunk(sa, 2);
+        tmem_wait_ld32(sb);
+        chunk(sb, 3);
+    }
+    return fmaxf(mx, mx2);
+}
+
+// p = silu(x) = x sigmoid(x) = h (1 + tanh(h)), h = x / 2, as bf16 into P   (sc = scale / 2)
+template <bool TAIL>
+__device__ __forceinline__ void silu_tile(uint32_t tS, uint32_t tP, float sc, int valid)
+{
+    auto chunk = [&](const uint32_t (&cur)[32], int c) {
+        uint32_t p[16];
+#pragma unroll
+        for (int e = 0; e < 32; e += 2) {
+            const float h0 = __uint_as_float(cur[e]) * sc, h1 = __uint_as_float(cur[e + 1]) * sc;
+            float w0 = fmaf(h0, tanh_fast(h0), h0), w1 = fmaf(h1, tanh_fast(h1), h1);
+            if (TAIL) {
+                if (pos_of_col(c, e) >= valid) w0 = 0.f;
+                if (pos_of_col(c, e + 1) >= valid) w1 = 0.f;
+            }
+            p[e >> 1] = pack_bf16(w0, w1);
+        }
+        tmem_st16(tP + 16 * c, p);
+    };
+    if constexpr (TAIL) {
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+            uint32_t cur[32];
+            tmem_ld32(tS + 32 * c, cur);
+            tmem_wait_ld32(cur);
+            chunk(cur, c);
+        }
+    } else {
+        uint32_t sa[32], sb[32];
+        tmem_ld32(tS, sa);
+        tmem_wait_ld32(sa);
+        tmem_ld32(tS + 32, sb);
+        chunk(sa, 0);
+        tmem_wait_ld32(sb);
+        tmem_ld32(tS + 64, sa);
+        chunk(sb, 1);
+        tmem_wait_ld32(sa);
+        tmem_ld32(tS + 96, sb);
+        chunk(sa, 2);
+        tmem_wait_ld32(sb);
+        chunk(sb, 3);
+    }
+}
+
+// One work unit of the CTA's share, decoded from its Work record.
 struct Unit {
-    Item it;
-    Req rq;
+    Work wk;
     int grp;
     int row0;        // first query row of the block
     int n_tiles;     // > 0: tiles to process; 0: empty history (zero output rows); < 0: nothing at all
     int last_valid;  // real positions in the last tile
 };
 
-__device__ __forceinline__ void load_unit(const AttendArgs& a, int n_mb, int64_t w, Unit& u)
+__device__ __forceinline__ Work load_work(const Work* p)
 {
-    const int G = a.cv.n_groups;
-    const int mb = (int)(w % n_mb);
-    const int64_t t = w / n_mb;
-    u.grp = (int)(t % G);
-    u.it = a.items[t / G];
-    u.rq = a.reqs[u.it.req];
-    u.row0 = mb * 128;
-    u.n_tiles = u.row0 < u.rq.M ? (u.it.len + TK - 1) / TK : -1;
-    u.last_valid = u.it.len - (u.n_tiles - 1) * TK;
+    static_assert(sizeof(Work) == 48, "Work is read as three 16-byte words");
+    union {
+        Work w;
+        uint4 q[3];
+    } u;
+    const uint4* src = reinterpret_cast<const uint4*>(p);
+    u.q[0] = __ldg(src);
+    u.q[1] = __ldg(src + 1);
+    u.q[2] = __ldg(src + 2);
+    return u.w;
 }
 
-// The CTA's tile stream: units blockIdx.x, blockIdx.x + gridDim.x, ... that have tiles, tile by
-// tile.  Every role walks an identical copy, so stage and buffer indices need no communication.
+// The CTA's tile stream: units blockIdx.x, blockIdx.x + gridDim.x, ... tile by tile.  Every role
+// walks an identical copy, so stage and buffer indices need no communication.  The record of
+// the following unit is always in flight while the current one is processed.
+// KEEP_EMPTY: also stop at units with an empty history (the role that writes their zero rows).
+template <bool KEEP_EMPTY>
 struct Stream {
-    const AttendArgs* a;
-    int n_mb;
-    int64_t w, n_work;
+    const Work* works;
+    uint32_t n_mb, n_groups;
+    uint32_t w, n_work;  // the host keeps n_work + gridDim.x below 2^32
     Unit u;
+    Work nxt;    // record of unit w + gridDim.x (valid if that is < n_work)
     int j;       // tile inside the unit
     int g;       // tiles before this one in the stream
     int useq;    // units with tiles before this one
     bool valid;
-    __device__ __forceinline__ void seek()
+    __device__ __forceinline__ void take()
     {
         valid = false;
         while (w < n_work) {
-            load_unit(*a, n_mb, w, u);
-            if (u.n_tiles > 0) {
+            u.wk = nxt;
+            const uint32_t wn = w + gridDim.x;
+            if (wn < n_work) nxt = load_work(works + (wn / n_mb) / n_groups);
+            const uint32_t t = w / n_mb;
+            u.grp = (int)(t % n_groups);
+            u.row0 = (int)(w - t * n_mb) * 128;
+            u.n_tiles = u.row0 < u.wk.M ? (u.wk.len + TK - 1) / TK : -1;
+            u.last_valid = u.wk.len - (u.n_tiles - 1) * TK;
+            if (u.n_tiles > 0 || (KEEP_EMPTY && u.n_tiles == 0)) {
                 valid = true;
                 j = 0;
                 return;
             }
-            w += gridDim.x;
+            w = wn;
         }
     }
-    __device__ __forceinline__ void init(const AttendArgs* args, int n_mb_, int64_t n_work_)
+    __device__ __forceinline__ void init(const AttendArgs& a, int n_mb_, int64_t n_work_)
     {
-        a = args;
-        n_mb = n_mb_;
-        n_work = n_work_;
+        works = a.works;
+        n_mb = (uint32_t)n_mb_;
+        n_groups = (uint32_t)a.cv.n_groups;
+        n_work = (uint32_t)n_work_;
         w = blockIdx.x;
         g = 0;
         useq = 0;
-        seek();
+        if (w < n_work) nxt = load_work(works + (w / n_mb) / n_groups);
+        take();
+    }
+    __device__ __forceinline__ void next_unit()
+    {
+        g += u.n_tiles > 0 ? u.n_tiles : 0;
+        useq += u.n_tiles > 0;
+        w += gridDim.x;
+        take();
     }
     __device__ __forceinline__ void advance()
     {
@@ -313,7 +473,7 @@ struct Stream {
         if (++j == u.n_tiles) {
             w += gridDim.x;
             ++useq;
-            seek();
+            take();
         }
     }
 };
@@ -333,7 +493,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
 
     if (tid == 0) {
         for (int s = 0; s < NS; ++s) {
-            mbar_init(bar(BAR_FULL + s), kProducerThreads);
+            mbar_init(bar(BAR_FULL + s), 1);  // lane 0 of the producer warp that owns the tile
             mbar_init(bar(BAR_EMPTY + s), 1);
         }
         for (int q = 0; q < NQ; ++q) mbar_init(bar(BAR_QEMPTY + q), 1);
@@ -345,7 +505,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
         }
         mbar_init(bar(BAR_XFULL), kGroupThreads);
         mbar_init(bar(BAR_XEMPTY), kGroupThreads);
-        mbar_init(bar(BAR_DRAIN), 1);
+        for (int i = 0; i < 3; ++i) mbar_init(bar(BAR_DRAIN + i), 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -368,7 +528,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
 
     if (warp < 8) {
         // --------------------------------------------------------------- normalisation groups
-        const int b = warp >> 2;                  // group = score buffer
+        const int b = warp >> 2;                    // group = score buffer
         const int row = tid & (kGroupThreads - 1);  // query row inside the block = TMEM lane
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t tS = tmem + lane_base + kColS + 128u * b, tP = tmem + lane_base + kColP + 64u * b,
@@ -378,16 +538,16 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
         int cnt = 0;    // tiles this group has normalised
         int ocnt = 0;   // units in which this group had tiles
         int xcnt = 0;   // units exchanged between the groups
-        int g = 0;      // tiles of the stream before the current unit
         bool ok = true;
-        for (int64_t w = blockIdx.x; w < n_work && ok; w += gridDim.x) {
-            Unit u;
-            load_unit(a, n_mb, w, u);
-            if (u.n_tiles < 0) continue;
+        T_DECL(8);  // 0 other, 1 wait S, 2 wait PFREE, 3 unused, 4 tile, 5 wait O, 6 exchange wait, 7 rest
+        Stream<true> sn;
+        for (sn.init(a, n_mb, n_work); sn.valid && ok; sn.next_unit()) {
+            const Unit& u = sn.u;
+            const int g = sn.g;
             const int r = u.row0 + row;
-            const int64_t out_base = ((int64_t)(u.rq.q0 + r) * G + u.grp) * D;
+            const int64_t out_base = ((int64_t)(u.wk.q0 + r) * G + u.grp) * D;
             if (u.n_tiles == 0) {  // empty history: zero output rows
-                if (b == 0 && r < u.rq.M && u.it.part_row < 0) {
+                if (b == 0 && r < u.wk.M && u.wk.part_row < 0) {
                     if (a.out_dtype == CKV_BF16) {
                         uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(a.out) + out_base);
                         for (int q4 = 0; q4 < 4; ++q4) dst[q4] = make_uint4(0, 0, 0, 0);
@@ -402,57 +562,21 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
             int mine = 0;  // tiles of this unit normalised by this group
             for (int j = 0; j < u.n_tiles && ok; ++j) {
                 if (((g + j) & 1) != b) continue;
+                T_ACC(0);
                 ok = mbar_wait(bar(BAR_SFULL + b), cnt & 1, abort_flag);
+                T_ACC(1);
                 if (ok && cnt > 0) ok = mbar_wait(bar(BAR_PFREE + b), (cnt - 1) & 1, abort_flag);  // P_b and O_b are quiet
                 ok = __all_sync(0xffffffffu, ok);
+                T_ACC(2);
                 if (!ok) break;
                 tc_fence_after();
                 const int valid = j == u.n_tiles - 1 ? u.last_valid : TK;
                 const bool tail = valid < TK;
                 if constexpr (MODE == CKV_SOFTMAX) {
-                    if (mine == 0) {  // the reference maximum: exact maximum of the first tile
-                        float tmax = -CUDART_INF_F;
-#pragma unroll 1
-                        for (int c = 0; c < 4; ++c) {
-                            uint32_t s[32];
-                            tmem_ld32(tS + 32 * c, s);
-                            tmem_wait_ld32(s);
-#pragma unroll
-                            for (int e = 0; e < 32; e += 2) {
-                                float x0 = __uint_as_float(s[e]), x1 = __uint_as_float(s[e + 1]);
-                                if (tail) {
-                                    if (32 * c + e >= valid) x0 = -CUDART_INF_F;
-                                    if (32 * c + e + 1 >= valid) x1 = -CUDART_INF_F;
-                                }
-                                tmax = max3(tmax, x0, x1);
-                            }
-                        }
-                        m_ref = tmax * sc;  // valid >= 1, so finite
-                    }
                     for (int attempt = 0; attempt < 2; ++attempt) {
-                        const float nm = -m_ref;
-                        float mx = -CUDART_INF_F;
-                        uint32_t sa[32], sb[32];
-                        tmem_ld32(tS, sa);
-#pragma unroll
-                        for (int c = 0; c < 4; ++c) {
-                            uint32_t(&cur)[32] = (c & 1) ? sb : sa;
-                            uint32_t(&nxt)[32] = (c & 1) ? sa : sb;
-                            tmem_wait_ld32(cur);
-                            if (c < 3) tmem_ld32(tS + 32 * (c + 1), nxt);
-                            uint32_t p[16];
-#pragma unroll
-                            for (int e = 0; e < 32; e += 2) {
-                                float x0 = fmaf(__uint_as_float(cur[e]), sc, nm), x1 = fmaf(__uint_as_float(cur[e + 1]), sc, nm);
-                                if (tail) {
-                                    if (32 * c + e >= valid) x0 = -CUDART_INF_F;
-                                    if (32 * c + e + 1 >= valid) x1 = -CUDART_INF_F;
-                                }
-                                mx = max3(mx, x0, x1);
-                                p[e >> 1] = pack_bf16(ex2(x0), ex2(x1));
-                            }
-                            tmem_st16(tP + 16 * c, p);
-                        }
+                        const bool first = mine == 0 && attempt == 0;
+                        const float mx = tail ? softmax_tile<true>(tS, tP, sc, valid, first, m_ref)
+                                              : softmax_tile<false>(tS, tP, sc, valid, first, m_ref);
                         if (!__any_sync(0xffffffffu, mx > kHeadroom)) break;
                         // some row of this warp left the headroom: move its reference, rescale what
                         // O_b holds so far (its MMAs have finished, see the PFREE wait) and redo the tile
@@ -472,43 +596,25 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                         tc_wait_st();
                     }
                 } else {
-                    // silu(x) = x sigmoid(x) = h (1 + tanh(h)), h = x / 2   (sc = scale / 2)
-                    uint32_t sa[32], sb[32];
-                    tmem_ld32(tS, sa);
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        uint32_t(&cur)[32] = (c & 1) ? sb : sa;
-                        uint32_t(&nxt)[32] = (c & 1) ? sa : sb;
-                        tmem_wait_ld32(cur);
-                        if (c < 3) tmem_ld32(tS + 32 * (c + 1), nxt);
-                        uint32_t p[16];
-#pragma unroll
-                        for (int e = 0; e < 32; e += 2) {
-                            const float h0 = __uint_as_float(cur[e]) * sc, h1 = __uint_as_float(cur[e + 1]) * sc;
-                            float w0 = fmaf(h0, tanh_fast(h0), h0), w1 = fmaf(h1, tanh_fast(h1), h1);
-                            if (tail) {
-                                if (32 * c + e >= valid) w0 = 0.f;
-                                if (32 * c + e + 1 >= valid) w1 = 0.f;
-                            }
-                            p[e >> 1] = pack_bf16(w0, w1);
-                        }
-                        tmem_st16(tP + 16 * c, p);
-                    }
+                    if (tail) silu_tile<true>(tS, tP, sc, valid);
+                    else silu_tile<false>(tS, tP, sc, valid);
                 }
                 tc_wait_st();
                 tc_fence_before();
                 mbar_arrive(bar(BAR_PREADY + b));
+                T_ACC(4);
                 ++cnt;
                 ++mine;
             }
-            g += u.n_tiles;
             if (!ok) break;
 
             // ---- the unit's epilogue: fetch O_b, merge the two groups, store
             float o[32], l = 0.f;
+            T_ACC(0);
             if (mine > 0) {
                 ok = mbar_wait(bar(BAR_OFULL + b), ocnt & 1, abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
+                T_ACC(5);
                 if (!ok) break;
                 ++ocnt;
                 tc_fence_after();
@@ -524,8 +630,10 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                 for (int e = 0; e < 32; ++e) o[e] = 0.f;
             }
             if (b == 1) {
+                T_ACC(0);
                 if (xcnt > 0) ok = mbar_wait(bar(BAR_XEMPTY), (xcnt - 1) & 1, abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
+                T_ACC(6);
                 if (!ok) break;
                 xch[row] = m_ref;
                 xch[128 + row] = l;
@@ -534,8 +642,10 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                 mbar_arrive(bar(BAR_XFULL));
                 ++xcnt;
             } else {
+                T_ACC(0);
                 ok = mbar_wait(bar(BAR_XFULL), xcnt & 1, abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
+                T_ACC(6);
                 if (!ok) break;
                 ++xcnt;
                 const float m1 = xch[row], l1 = xch[128 + row];
@@ -552,11 +662,11 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                     for (int e = 0; e < 32; ++e) o[e] += xch[(2 + e) * 128 + row];
                 }
                 mbar_arrive(bar(BAR_XEMPTY));
-                if (r < u.rq.M) {
-                    if (u.it.part_row < 0) {
+                if (r < u.wk.M) {
+                    if (u.wk.part_row < 0) {
                         float inv;
                         if constexpr (MODE == CKV_SOFTMAX) inv = l > 0.f ? 1.0f / l : 0.f;
-                        else inv = 1.0f / (float)u.rq.L;
+                        else inv = 1.0f / (float)u.wk.L;
                         if (a.out_dtype == CKV_BF16) {
                             uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(a.out) + out_base);
 #pragma unroll
@@ -576,7 +686,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                                                       o[4 * q4 + 3] * inv);
                         }
                     } else {
-                        float* pr = a.partials + ((int64_t)(u.it.part_row + r) * G + u.grp) * (D + 2);
+                        float* pr = a.partials + ((int64_t)(u.wk.part_row + r) * G + u.grp) * (D + 2);
                         pr[0] = m_ref;
                         pr[1] = l;
 #pragma unroll
@@ -585,23 +695,35 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                 }
             }
         }
+        T_ACC(7);
+#ifdef CKV_STAGE_TIMERS
+        if (blockIdx.x == 0 && row == 0)
+            printf("group %d: total %lld | other %lld waitS %lld waitPfree %lld tile %lld waitO %lld xchg %lld rest %lld | tiles %d\n", b,
+                   T_TOTAL(), tmr_[0], tmr_[1], tmr_[2], tmr_[4], tmr_[5], tmr_[6], tmr_[7], cnt);
+#endif
         if (!ok) {
             *abort_flag = 1;
             if (lane == 0) atomicOr(err_flag, ERR_NORMALISE);
         }
     } else if (warp == kMmaWarp) {
-        // --------------------------------------------------------------------- MMA issue
+        // --------------------------------------------------------------------- S = Q K^T issue
         if (lane == 0) {
             constexpr uint32_t idesc_s = make_idesc(128, TK, false);
-            constexpr uint32_t idesc_pv = make_idesc(128, MODE == CKV_SOFTMAX ? kNV : D, true);
-            Stream ss, sp;  // next tile whose S / whose PV is to be issued
-            ss.init(&a, n_mb, n_work);
-            sp = ss;
-            int pcnt[2] = {0, 0};
+            Stream<false> ss;
+            ss.init(a, n_mb, n_work);
+            int cnt[2] = {0, 0};  // tiles issued per score buffer
             bool ok = true;
-            auto issue_s = [&]() {
+            T_DECL(3);  // 0 issue, 1 wait FULL, 2 wait PREADY
+            while (ok && ss.valid) {
                 const int s = ss.g % NS, b = ss.g & 1;
-                if (!mbar_wait(bar(BAR_FULL + s), (ss.g / NS) & 1, abort_flag)) return false;
+                T_ACC(0);
+                ok = mbar_wait(bar(BAR_FULL + s), (ss.g / NS) & 1, abort_flag);
+                T_ACC(1);
+                // S_b is free once group b has read the previous tile that used it
+                if (ok && cnt[b] > 0) ok = mbar_wait(bar(BAR_PREADY + b), (cnt[b] - 1) & 1, abort_flag);
+                T_ACC(2);
+                if (!ok) break;
+                ++cnt[b];
                 tc_fence_after();
                 const uint32_t q_addr = sbase + kOffQ + (ss.useq % NQ) * kTileK, k_addr = sbase + kOffK + s * kTileK;
 #pragma unroll
@@ -611,30 +733,12 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                 tc_commit(bar(BAR_SFULL + b));
                 if (ss.j == ss.u.n_tiles - 1) tc_commit(bar(BAR_QEMPTY + ss.useq % NQ));  // Q buffer no longer read
                 ss.advance();
-                return true;
-            };
-            auto issue_pv = [&]() {  // O_b += P_b [V | 1], sixteen positions per instruction
-                const int s = sp.g % NS, b = sp.g & 1;
-                if (!mbar_wait(bar(BAR_PREADY + b), pcnt[b] & 1, abort_flag)) return false;
-                ++pcnt[b];
-                tc_fence_after();
-                const uint32_t v_addr = sbase + kOffV + s * kTileV;
-#pragma unroll
-                for (int kk = 0; kk < TK / 16; ++kk)
-                    umma_ts(tmem + kColO + (uint32_t)kNV * b, tmem + kColP + 64u * b + 8 * kk,
-                            smem_desc(v_addr + kk * 2 * kVGroup, kVGroup, 128), idesc_pv, (sp.j >= 2 || kk > 0) ? 1u : 0u);
-                tc_commit(bar(BAR_EMPTY + s));
-                tc_commit(bar(BAR_PFREE + b));
-                if (sp.j >= sp.u.n_tiles - 2) tc_commit(bar(BAR_OFULL + b));  // last tile of its group in the unit
-                sp.advance();
-                return true;
-            };
-            if (ss.valid) ok = issue_s();
-            if (ok && ss.valid) ok = issue_s();
-            while (ok && sp.valid) {
-                ok = issue_pv();
-                if (ok && ss.valid) ok = issue_s();
             }
+            T_ACC(0);
+#ifdef CKV_STAGE_TIMERS
+            if (blockIdx.x == 0)
+                printf("S issue: total %lld | issue %lld waitFULL %lld waitPREADY %lld | tiles %d\n", T_TOTAL(), tmr_[0], tmr_[1], tmr_[2], ss.g);
+#endif
             if (!ok) {
                 *abort_flag = 1;
                 atomicOr(err_flag, ERR_MMA);
@@ -645,141 +749,215 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
             if (!mbar_wait(bar(BAR_DRAIN), 0, &never)) atomicOr(err_flag, ERR_DRAIN);
         }
         __syncwarp();
+    } else if (warp < kProducerWarp0) {
+        // --------------------------------------------------------------------- O_b += P_b [V | 1] issue
+        if (lane == 0) {
+            const int b = warp - kPvWarp0;
+            constexpr uint32_t idesc_pv = make_idesc(128, MODE == CKV_SOFTMAX ? kNV : D, true);
+            Stream<false> sp;
+            sp.init(a, n_mb, n_work);
+            int cnt = 0;
+            bool ok = true;
+            T_DECL(2);  // 0 issue, 1 wait PREADY
+            for (; ok && sp.valid; sp.advance()) {
+                if ((sp.g & 1) != b) continue;
+                const int s = sp.g % NS;
+                T_ACC(0);
+                ok = mbar_wait(bar(BAR_PREADY + b), cnt & 1, abort_flag);
+                if (ok) ok = mbar_wait(bar(BAR_FULL + s), (sp.g / NS) & 1, abort_flag);  // completed long ago: makes the V tile visible here
+                T_ACC(1);
+                if (!ok) break;
+                ++cnt;
+                tc_fence_after();
+                const uint32_t v_addr = sbase + kOffV + s * kTileV;
+#pragma unroll
+                for (int kk = 0; kk < TK / 16; ++kk)  // sixteen positions per instruction
+                    umma_ts(tmem + kColO + (uint32_t)kNV * b, tmem + kColP + 64u * b + 8 * kk,
+                            smem_desc(v_addr + kk * 2 * kVGroup, kVGroup, 128), idesc_pv, (sp.j >= 2 || kk > 0) ? 1u : 0u);
+                tc_commit(bar(BAR_EMPTY + s));
+                tc_commit(bar(BAR_PFREE + b));
+                if (sp.j >= sp.u.n_tiles - 2) tc_commit(bar(BAR_OFULL + b));  // last tile of its group in the unit
+            }
+            T_ACC(0);
+#ifdef CKV_STAGE_TIMERS
+            if (blockIdx.x == 0)
+                printf("PV issue %d: total %lld | issue %lld waitPREADY %lld | tiles %d\n", b, T_TOTAL(), tmr_[0], tmr_[1], cnt);
+#endif
+            if (!ok) {
+                *abort_flag = 1;
+                atomicOr(err_flag, ERR_MMA);
+            }
+            tc_commit(bar(BAR_DRAIN + 1 + b));
+            volatile int never = 0;
+            if (!mbar_wait(bar(BAR_DRAIN + 1 + b), 0, &never)) atomicOr(err_flag, ERR_DRAIN);
+        }
+        __syncwarp();
     } else {
         // --------------------------------------------------------------------- producers
-        const int p = tid - kProducerWarp0 * 32;  // 0..127 = the tile row this thread owns
-        const int pw = p >> 5;
+        // Producer warp pw owns every kProducerWarps-th tile of the stream and does all of its
+        // copies, so the per-tile bookkeeping is paid by one warp while the others work on their own
+        // tiles.  Lane (q = lane / 4, chunk = lane % 4) copies chunk `chunk` of the pool rows of
+        // positions 32 rb + 4 q + i (rb, i < 4) into tile rows 32 rb + 8 i + q, and patches the
+        // user-specific leading elements of tile rows 32 rb + lane.
+        const int pw = warp - kProducerWarp0, q = lane >> 2, chunk = lane & 3;
         const int du_bytes = a.cv.d_user * 2;
-        const int src_lane0 = lane >> 2, chunk = lane & 3;
-        Stream st;
-        st.init(&a, n_mb, n_work);
+        const int patch_pos = 4 * (lane & 7) + (lane >> 3);  // position (inside a 32-block) held by row `lane`
+        const uint32_t kv_lane = (uint32_t)(chunk * 128 + q * 16);
+        const int64_t pool_stride = (int64_t)a.cv.n_entries * (D * 2);
+        const char* poolK0 = reinterpret_cast<const char*>(a.cv.poolK) + chunk * 16;
+        const char* poolV0 = reinterpret_cast<const char*>(a.cv.poolV) + chunk * 16;
+        const uint16_t* Q = reinterpret_cast<const uint16_t*>(a.queries);
+        Stream<false> st;
+        st.init(a, n_mb, n_work);
+        for (int i = 0; i < pw && st.valid; ++i) st.advance();
         bool ok = true;
-        // per tile in flight: where it went and this thread's user-specific leading elements
-        uint4 uk[LAG], uv[LAG];
-        int stage_of[LAG];
-        bool patch[LAG], live[LAG];
-#pragma unroll
-        for (int u = 0; u < LAG; ++u) {
-            live[u] = false;
-            patch[u] = false;
-            stage_of[u] = 0;
-            uk[u] = uv[u] = make_uint4(0, 0, 0, 0);
-        }
-        // indices of the next tile to issue, loaded one iteration ahead
-        int ik = 0, iv = 0;
-        int64_t my_unit = 0;
-        bool my_valid = false;
-        auto prefetch = [&]() {
+        uint4 xk[4], xv[4];  // row indices of this lane's positions of the next tile (16-bit: packed in .x .y)
+        int64_t unit0 = 0;   // arena unit of that tile's position 0
+        auto fetch = [&]() {
             if (!st.valid) return;
-            const int valid = st.j == st.u.n_tiles - 1 ? st.u.last_valid : TK;
-            my_valid = p < valid;
-            my_unit = st.u.rq.base + (int64_t)st.u.grp * st.u.rq.Lpad + st.u.it.begin + (int64_t)st.j * TK + p;
-            ik = iv = 0;
-            if (my_valid) {
-                if constexpr (IDX16) {
-                    ik = __ldg(reinterpret_cast<const uint16_t*>(a.cv.idxK) + my_unit);
-                    iv = __ldg(reinterpret_cast<const uint16_t*>(a.cv.idxV) + my_unit);
-                } else {
-                    ik = __ldg(reinterpret_cast<const int32_t*>(a.cv.idxK) + my_unit);
-                    iv = __ldg(reinterpret_cast<const int32_t*>(a.cv.idxV) + my_unit);
+            const int pos0 = st.u.wk.begin + st.j * TK;
+            unit0 = st.u.wk.base + (int64_t)st.u.grp * st.u.wk.Lpad + pos0;
+#pragma unroll
+            for (int rb = 0; rb < 4; ++rb) {
+                xk[rb] = xv[rb] = make_uint4(0, 0, 0, 0);
+                if (pos0 + 32 * rb + 4 * q < st.u.wk.Lpad) {  // the arena is padded to 32 positions per user
+                    const int64_t un = unit0 + 32 * rb + 4 * q;
+                    if constexpr (IDX16) {
+                        const uint2 a2 = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const uint16_t*>(a.cv.idxK) + un));
+                        const uint2 b2 = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const uint16_t*>(a.cv.idxV) + un));
+                        xk[rb] = make_uint4(a2.x, a2.y, 0, 0);
+                        xv[rb] = make_uint4(b2.x, b2.y, 0, 0);
+                    } else {
+                        xk[rb] = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const int32_t*>(a.cv.idxK) + un));
+                        xv[rb] = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const int32_t*>(a.cv.idxV) + un));
+                    }
                 }
             }
         };
-        prefetch();
-        bool more = true;
-        while (more) {
-            more = false;
-#pragma unroll
-            for (int u = 0; u < LAG; ++u) {
-                // (1) the tile issued LAG iterations ago has landed: patch and publish it
-                if (live[u]) {
-                    cp_async_wait<LAG - 1>();
-                    __syncwarp();  // a row's chunks were copied by four other lanes of this warp
-                    if (patch[u]) {  // Eq. K: dims [0, d_user) come from the user part
-                        unsigned char* kd = smem + kOffK + stage_of[u] * kTileK + k_off(p, 0);
-                        unsigned char* vd = smem + kOffV + stage_of[u] * kTileV + v_off(p, 0);
-                        if (du_bytes == 4) {
-                            *reinterpret_cast<uint32_t*>(kd) = uk[u].x;
-                            *reinterpret_cast<uint32_t*>(vd) = uv[u].x;
-                        } else if (du_bytes == 2) {
-                            *reinterpret_cast<uint16_t*>(kd) = (uint16_t)uk[u].x;
-                            *reinterpret_cast<uint16_t*>(vd) = (uint16_t)uv[u].x;
-                        } else if (du_bytes == 8) {
-                            *reinterpret_cast<uint2*>(kd) = make_uint2(uk[u].x, uk[u].y);
-                            *reinterpret_cast<uint2*>(vd) = make_uint2(uv[u].x, uv[u].y);
-                        } else {
-                            *reinterpret_cast<uint4*>(kd) = uk[u];
-                            *reinterpret_cast<uint4*>(vd) = uv[u];
-                        }
-                    }
-                    fence_proxy_async();
-                    mbar_arrive(bar(BAR_FULL + stage_of[u]));
-                    live[u] = false;
-                }
-                // (2) issue the copies of the next tile of the stream
-                if (st.valid && ok) {
-                    const int s = st.g % NS;
-                    if (st.g >= NS) ok = mbar_wait(bar(BAR_EMPTY + s), ((st.g / NS) - 1) & 1, abort_flag);
-                    if (ok && st.j == 0) {  // a new unit: stage its Q block (rows beyond M are zero)
-                        if (st.useq >= NQ) ok = mbar_wait(bar(BAR_QEMPTY + st.useq % NQ), ((st.useq / NQ) - 1) & 1, abort_flag);
-                        if (ok) {
-                            const uint32_t qdst = sbase + kOffQ + (st.useq % NQ) * kTileK;
-                            const uint16_t* Q = reinterpret_cast<const uint16_t*>(a.queries);
-#pragma unroll
-                            for (int i = 0; i < 4; ++i) {
-                                const int r = 32 * pw + 8 * i + src_lane0;
-                                const bool in = st.u.row0 + r < st.u.rq.M;
-                                const uint16_t* src = Q + ((int64_t)(st.u.rq.q0 + st.u.row0 + (in ? r : 0)) * G + st.u.grp) * D + chunk * 8;
-                                cp_async16(qdst + k_off(r, chunk), src, in ? 16u : 0u);
-                            }
-                        }
-                    }
-                    if (ok) {
-                        const char* poolK = reinterpret_cast<const char*>(a.cv.poolK) + (int64_t)st.u.grp * a.cv.n_entries * (D * 2);
-                        const char* poolV = reinterpret_cast<const char*>(a.cv.poolV) + (int64_t)st.u.grp * a.cv.n_entries * (D * 2);
-                        const uint32_t kdst = sbase + kOffK + s * kTileK, vdst = sbase + kOffV + s * kTileV;
-                        const uint32_t vbits = __ballot_sync(0xffffffffu, my_valid);
-                        // four lanes fetch the four 16-byte chunks of one row: 64 contiguous bytes per row
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const int sl = 8 * i + src_lane0;
-                            const int rk = __shfl_sync(0xffffffffu, ik, sl), rv = __shfl_sync(0xffffffffu, iv, sl);
-                            const uint32_t nb = (vbits >> sl) & 1u ? 16u : 0u;  // rows beyond the history are zero
-                            const int r = 32 * pw + sl;
-                            cp_async16(kdst + k_off(r, chunk), poolK + (int64_t)rk * (D * 2) + chunk * 16, nb);
-                            cp_async16(vdst + v_off(r, chunk), poolV + (int64_t)rv * (D * 2) + chunk * 16, nb);
-                        }
-                        patch[u] = my_valid && du_bytes > 0;
-                        if (patch[u]) {
-                            const char* ku = reinterpret_cast<const char*>(a.cv.userK) + my_unit * du_bytes;
-                            const char* vu = reinterpret_cast<const char*>(a.cv.userV) + my_unit * du_bytes;
-                            if (du_bytes == 4) {
-                                uk[u].x = __ldg(reinterpret_cast<const uint32_t*>(ku));
-                                uv[u].x = __ldg(reinterpret_cast<const uint32_t*>(vu));
-                            } else if (du_bytes == 2) {
-                                uk[u].x = __ldg(reinterpret_cast<const uint16_t*>(ku));
-                                uv[u].x = __ldg(reinterpret_cast<const uint16_t*>(vu));
-                            } else if (du_bytes == 8) {
-                                const uint2 x = __ldg(reinterpret_cast<const uint2*>(ku)), y = __ldg(reinterpret_cast<const uint2*>(vu));
-                                uk[u] = make_uint4(x.x, x.y, 0, 0);
-                                uv[u] = make_uint4(y.x, y.y, 0, 0);
-                            } else {
-                                uk[u] = __ldg(reinterpret_cast<const uint4*>(ku));
-                                uv[u] = __ldg(reinterpret_cast<const uint4*>(vu));
-                            }
-                        }
-                        stage_of[u] = s;
-                        live[u] = true;
-                        st.advance();
-                        prefetch();
-                    }
-                }
-                cp_async_commit();  // one group per iteration, also when nothing was issued
-                more = more || live[u];
+        auto row_index = [](const uint4& x, int i) -> uint32_t {
+            if constexpr (IDX16) {
+                const uint32_t w = i < 2 ? x.x : x.y;
+                return (i & 1) ? w >> 16 : w & 0xffffu;
+            } else {
+                return i == 0 ? x.x : (i == 1 ? x.y : (i == 2 ? x.z : x.w));
             }
-            more = more || (st.valid && ok);
+        };
+        fetch();
+        T_DECL(6);  // 0 other, 1 wait copies, 2 wait EMPTY, 3 wait QEMPTY, 4 patch+publish, 5 copy issue
+        while (st.valid && ok) {
+            const int s = st.g % NS;
+            T_ACC(0);
+            if (st.g >= NS) {
+                if (lane == 0) ok = mbar_wait(bar(BAR_EMPTY + s), ((st.g / NS) - 1) & 1, abort_flag);
+                ok = __all_sync(0xffffffffu, ok);
+            }
+            T_ACC(2);
+            if (!ok) break;
+            if (st.j == 0) {  // a new unit: stage its Q block (rows beyond M are zero)
+                if (st.useq >= NQ) {
+                    if (lane == 0) ok = mbar_wait(bar(BAR_QEMPTY + st.useq % NQ), ((st.useq / NQ) - 1) & 1, abort_flag);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                }
+                T_ACC(3);
+                const uint32_t qdst = sbase + kOffQ + (st.useq % NQ) * kTileK;
+#pragma unroll 4
+                for (int rr = 0; rr < 16; ++rr) {
+                    const int r = 8 * rr + q;
+                    const bool in = st.u.row0 + r < st.u.wk.M;
+                    const uint16_t* src = Q + ((int64_t)(st.u.wk.q0 + st.u.row0 + (in ? r : 0)) * G + st.u.grp) * D + chunk * 8;
+                    cp_async16(qdst + k_off(r, chunk), src, in ? 16u : 0u);
+                }
+            }
+            const char* pk = poolK0 + st.u.grp * pool_stride;
+            const char* pv = poolV0 + st.u.grp * pool_stride;
+            const uint32_t kdst = sbase + kOffK + s * kTileK + kv_lane, vdst = sbase + kOffV + s * kTileV + kv_lane;
+            const int valid = st.j == st.u.n_tiles - 1 ? st.u.last_valid : TK;
+            if (valid == TK) {
+#pragma unroll
+                for (int rb = 0; rb < 4; ++rb)
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        cp_async16(kdst + 2048 * rb + 512 * i, pk + (size_t)row_index(xk[rb], i) * (D * 2), 16u);
+                        cp_async16(vdst + 4 * kVGroup * rb + kVGroup * i, pv + (size_t)row_index(xv[rb], i) * (D * 2), 16u);
+                    }
+            } else {  // rows of positions beyond the history are zero
+#pragma unroll
+                for (int rb = 0; rb < 4; ++rb)
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const uint32_t nb = 32 * rb + 4 * q + i < valid ? 16u : 0u;
+                        cp_async16(kdst + 2048 * rb + 512 * i, pk + (size_t)row_index(xk[rb], i) * (D * 2), nb);
+                        cp_async16(vdst + 4 * kVGroup * rb + kVGroup * i, pv + (size_t)row_index(xv[rb], i) * (D * 2), nb);
+                    }
+            }
+            cp_async_commit();
+            T_ACC(5);
+            // this lane's user-specific leading elements (Eq. K: dims [0, d_user)) of tile rows 32 rb + lane
+            uint4 uk[4], uv[4];
+#pragma unroll
+            for (int rb = 0; rb < 4; ++rb) {
+                uk[rb] = uv[rb] = make_uint4(0, 0, 0, 0);
+                if (du_bytes > 0 && 32 * rb + patch_pos < valid) {
+                    const char* ku = reinterpret_cast<const char*>(a.cv.userK) + (unit0 + 32 * rb + patch_pos) * du_bytes;
+                    const char* vu = reinterpret_cast<const char*>(a.cv.userV) + (unit0 + 32 * rb + patch_pos) * du_bytes;
+                    if (du_bytes == 4) {
+                        uk[rb].x = __ldg(reinterpret_cast<const uint32_t*>(ku));
+                        uv[rb].x = __ldg(reinterpret_cast<const uint32_t*>(vu));
+                    } else if (du_bytes == 2) {
+                        uk[rb].x = __ldg(reinterpret_cast<const uint16_t*>(ku));
+                        uv[rb].x = __ldg(reinterpret_cast<const uint16_t*>(vu));
+                    } else if (du_bytes == 8) {
+                        const uint2 x = __ldg(reinterpret_cast<const uint2*>(ku)), y = __ldg(reinterpret_cast<const uint2*>(vu));
+                        uk[rb] = make_uint4(x.x, x.y, 0, 0);
+                        uv[rb] = make_uint4(y.x, y.y, 0, 0);
+                    } else {
+                        uk[rb] = __ldg(reinterpret_cast<const uint4*>(ku));
+                        uv[rb] = __ldg(reinterpret_cast<const uint4*>(vu));
+                    }
+                }
+            }
+            // the indices of this warp's next tile travel while the copies land
+            for (int i = 0; i < kProducerWarps && st.valid; ++i) st.advance();
+            fetch();
+            T_ACC(0);
+            cp_async_wait<0>();
+            __syncwarp();  // a row's chunks were copied by four lanes of this warp
+            T_ACC(1);
+            if (du_bytes > 0) {
+#pragma unroll
+                for (int rb = 0; rb < 4; ++rb) {
+                    if (32 * rb + patch_pos < valid) {  // zero rows beyond the history stay zero
+                        unsigned char* kd = smem + kOffK + s * kTileK + k_off(32 * rb + lane, 0);
+                        unsigned char* vd = smem + kOffV + s * kTileV + v_off(32 * rb + lane, 0);
+                        if (du_bytes == 4) {
+                            *reinterpret_cast<uint32_t*>(kd) = uk[rb].x;
+                            *reinterpret_cast<uint32_t*>(vd) = uv[rb].x;
+                        } else if (du_bytes == 2) {
+                            *reinterpret_cast<uint16_t*>(kd) = (uint16_t)uk[rb].x;
+                            *reinterpret_cast<uint16_t*>(vd) = (uint16_t)uv[rb].x;
+                        } else if (du_bytes == 8) {
+                            *reinterpret_cast<uint2*>(kd) = make_uint2(uk[rb].x, uk[rb].y);
+                            *reinterpret_cast<uint2*>(vd) = make_uint2(uv[rb].x, uv[rb].y);
+                        } else {
+                            *reinterpret_cast<uint4*>(kd) = uk[rb];
+                            *reinterpret_cast<uint4*>(vd) = uv[rb];
+                        }
+                    }
+                }
+            }
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(BAR_FULL + s));
+            T_ACC(4);
         }
         cp_async_wait<0>();
+        T_ACC(0);
+#ifdef CKV_STAGE_TIMERS
+        if (blockIdx.x == 0 && lane == 0)
+            printf("producer %d: total %lld | other %lld waitcopies %lld waitEMPTY %lld waitQEMPTY %lld publish %lld copies %lld\n", pw, T_TOTAL(),
+                   tmr_[0], tmr_[1], tmr_[2], tmr_[3], tmr_[4], tmr_[5]);
+#endif
         if (!ok) {
             *abort_flag = 1;
             if (lane == 0) atomicOr(err_flag, ERR_PRODUCER);
@@ -806,6 +984,7 @@ cudaError_t launch_attend_umma(int max_M, const AttendArgs& a, int n_sms, int* e
     if (a.n_items == 0) return cudaSuccess;
     const int n_mb = (max_M + 127) / 128;
     const int64_t n_work = (int64_t)a.n_items * n_mb * a.cv.n_groups;
+    if (n_work + n_sms >= (int64_t)1 << 32) return cudaErrorInvalidValue;  // the kernel counts units in 32 bits
     const unsigned grid = (unsigned)(n_work < n_sms ? n_work : n_sms);
     const bool i16 = a.cv.idx_bytes == 2;
     auto go = [&](auto kernel) {

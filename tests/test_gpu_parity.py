@@ -78,8 +78,11 @@ def test_persistent_tcgen05_kernel_many_units_per_sm(mode, n_queries):
 
 
 def test_growing_maximum_triggers_rescale_in_tcgen05_kernel():
-    """Keys sorted by increasing score make every tile raise the running maximum."""
-    w = synth.Workload("grow", 1, 30, 2, 512, 2, (1024, 1024), 128, "softmax", "bf16", None, 1.0, 1.0, 33)
+    """Keys sorted by increasing score: the scores climb by about 115 log2 units along the
+    history, so every kernel has to move its running / reference maximum several times.
+    Pool and user values keep the workloads' scale (variance 1/32): with unit-variance V the
+    bf16 rounding of the weights alone leaves well under 1e-3 of margin to the tolerance."""
+    w = synth.Workload("grow", 1, 30, 2, 512, 2, (1024, 1024), 128, "softmax", "bf16", None, 1 / 32, 1 / 32, 33)
     d = synth.generate(w)
     # history = pool rows in an order of growing norm along one direction: scale the user part
     ramp = np.linspace(-40.0, 40.0, 1024, dtype=np.float32)

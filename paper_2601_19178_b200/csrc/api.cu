@@ -468,7 +468,7 @@ ckv_status ckv_pool_load(ckv_ctx* ctx, const void* pool_K, const void* pool_V, i
         ctx->pool_half = half;
         ctx->has_mma_pool = mma;
     }
-    ctx->has_umma = umma_supported(ctx->cfg.dtype, D, D - d_shared);
+    ctx->has_umma = umma_supported(ctx->cfg.dtype, D, D - d_shared, n_entries <= 65536 ? 2 : 4);
     CK(launch_pool_layout(ctx->cfg.dtype, G, n_entries, d_shared, D, sk.dev, ctx->pool, s));
     CK(launch_pool_layout(ctx->cfg.dtype, G, n_entries, d_shared, D, sv.dev, (char*)ctx->pool + half, s));
     if (mma)

@@ -94,8 +94,8 @@ cudaError_t launch_pool_permute(int G, int m, const void* poolK, const void* poo
 cudaError_t launch_attend_mma(int max_M, const AttendArgs& a, const void* poolKp, const void* poolVp,
                               cudaStream_t s);
 
-// ---- kernels_umma.cu : tcgen05 family (bf16, head_dim 32, d_user in {0, 1, 2, 4, 8})
-bool umma_supported(int dtype, int head_dim, int d_user);
+// ---- kernels_umma.cu : tcgen05 family (bf16, head_dim 32, d_user in {0, 1, 2, 4, 8}, 16-bit stored indices)
+bool umma_supported(int dtype, int head_dim, int d_user, int idx_bytes);
 // err_flag: device int, OR-ed with a non-zero code if a bounded wait inside the kernel ran out.
 // Persistent: one CTA per SM (n_sms of them at most).
 cudaError_t launch_attend_umma(int max_M, const AttendArgs& a, int n_sms, int* err_flag, cudaStream_t s);

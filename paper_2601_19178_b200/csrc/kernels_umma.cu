@@ -2,27 +2,29 @@
 //
 // Persistent: one CTA per SM walks a static round-robin share of the work units, where a unit
 // is (work item = history chunk of one user, group, block of up to 128 queries).  The history
-// chunk is processed in tiles of 128 positions.  Roles (warp-specialised, 15 warps):
-//   warps 0-3   normalisation group 0: thread i owns query row i = TMEM lane i, even tiles
-//   warps 4-7   normalisation group 1: the same rows, odd tiles
-//   warp  8     issues the score MMAs (one thread), owns the TMEM allocation
-//   warps 9-10  issue the weighted-sum MMAs of score buffer 0 and 1 (one thread each)
-//   warps 11-14 producers, one tile each in turn: gather pool rows into shared memory with
+// chunk is processed in tiles of 128 positions.  Roles (warp-specialised, 16 warps):
+//   warps 0-3   normalisation group 0: thread i owns query row i = TMEM lane i, first half of every tile
+//   warps 4-7   normalisation group 1: the same rows, second half of every tile
+//   warps 8-9   issue the score MMAs of group 0 and 1 (one thread each); warp 8 owns the TMEM allocation
+//   warps 10-11 issue the weighted-sum MMAs of group 0 and 1 (one thread each)
+//   warps 12-15 producers, one tile each in turn: gather pool rows into shared memory with
 //               16-byte cp.async, patch the user-specific leading elements (Eq. K), publish the
 //               tile; the owner of a unit's first tile also stages Q
 //
-// Tile t of the CTA's tile stream uses score buffer b = t mod 2:
-//   S_b  = Q K_t^T                    UMMA 128 x 128 x 32, A = Q smem, B = K tile smem (K-major)
-//   P_b  = exp2(S_b c - m) | silu     group b: tcgen05.ld -> math -> bf16 -> tcgen05.st
-//   O_b += P_b [V_t | 1]              UMMA 128 x 48 x 128, A = P from TMEM, B = V tile (MN-major)
-// While group b normalises tile t the tensor core already works on tile t+1 for the other
-// group, and the producers gather tiles t+2...; nothing drains between work units.  The two
-// groups keep separate accumulators O_0, O_1 with separate reference maxima and merge them
-// through shared memory when a unit ends.
+// A tile (128 positions) is split into two halves of 64 positions; half b belongs to group b,
+// which has two score buffers and two weight buffers in TMEM and uses them alternately:
+//   S_bi  = Q K_half^T                UMMA 128 x 64 x 32, A = Q smem, B = half K tile smem (K-major)
+//   P_bi  = exp2(S_bi c - m) | silu   group b: tcgen05.ld -> math -> bf16 -> tcgen05.st
+//   O_b  += P_bi [V_half | 1]         UMMA 128 x 48 x 64, A = P from TMEM, B = half V tile (MN-major)
+// While group b normalises its half of tile t, its scores of tile t+1 are already being
+// computed into the other buffer, the other group works on its own half, and the producers
+// gather tiles t+2...; nothing drains between work units.  The two groups keep separate
+// accumulators O_0, O_1 with separate reference maxima and merge them through shared memory
+// when a unit ends.
 //
-// Why three issuing warps: one thread hands a tcgen05.mma to the tensor core about every
+// Why four issuing warps: one thread hands a tcgen05.mma to the tensor core about every
 // hundred cycles whatever the instruction's size, and a tile needs ten of these small ones
-// (K = 16 per instruction).  Why one producer warp per tile: the bookkeeping of a tile (stream
+// (K = 16 per instruction), twelve with the halves.  Why one producer warp per tile: the bookkeeping of a tile (stream
 // position, waits, index and user-part loads) is a serial chain of a few hundred instructions;
 // paid by every producer warp for every tile it was the bottleneck of the whole pipeline.
 //
@@ -53,25 +55,25 @@ namespace ckv {
 namespace {
 
 constexpr int D = 32;
-constexpr int TK = 128;                  // positions per tile
+constexpr int TK = 128;                  // positions per tile (one shared-memory stage)
+constexpr int TH = 64;                   // positions per half tile = one MMA / normalisation step of a group
 constexpr int NS = 6;                    // K/V stages
 constexpr int NQ = 3;                    // Q buffers
 constexpr int kGroupThreads = 128;       // one normalisation group
-constexpr int kMmaWarp = 8;              // issues S = Q K^T, owns the TMEM allocation
-constexpr int kPvWarp0 = 9;              // warps 9, 10 issue the weighted sums of buffer 0, 1
-constexpr int kProducerWarp0 = 11;
+constexpr int kMmaWarp = 8;              // warps 8, 9 issue S = Q K^T of group 0, 1; warp 8 owns the TMEM allocation
+constexpr int kPvWarp0 = 10;             // warps 10, 11 issue the weighted sums of group 0, 1
+constexpr int kProducerWarp0 = 12;
 constexpr int kProducerWarps = 4;        // each owns every fourth tile of the stream
-constexpr int kThreads = 2 * kGroupThreads + 3 * 32 + kProducerWarps * 32;  // 480
+constexpr int kThreads = 2 * kGroupThreads + 4 * 32 + kProducerWarps * 32;  // 512
 constexpr int kTileK = TK * D * 2;       // 8 KB, also the Q tile
 constexpr int kVGroup = 768;             // bytes of one 8-row group of a V tile
 constexpr int kTileV = (TK / 8) * kVGroup;  // 12 KB
 constexpr int kNV = 48;                  // columns of [V | 1 | 0...]
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kColS = 0, kColP = 256, kColO = 384;  // S_b at kColS + 128 b, P_b at kColP + 64 b, O_b at kColO + 48 b
+constexpr uint32_t kColS = 0, kColP = 256, kColO = 384;  // S_bi at kColS + 64 (2b+i), P_bi at kColP + 32 (2b+i), O_b at kColO + 48 b
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kHeadroom = 64.0f;       // log2 units a score may exceed the reference maximum
-constexpr uint32_t kSpinLimit = 1u << 16;  // polls of a wait before the CTA gives up
-constexpr uint32_t kSuspendNs = 20000;     // how long one poll may stay suspended in hardware
+constexpr uint32_t kSpinLimit = 1u << 20;  // polls of a wait before the CTA gives up
 static_assert(NS > kProducerWarps, "every producer warp holds one stage while it copies");
 
 // dynamic shared memory map
@@ -79,17 +81,22 @@ constexpr int kOffQ = 0;
 constexpr int kOffK = kOffQ + NQ * kTileK;
 constexpr int kOffV = kOffK + NS * kTileK;
 constexpr int kOffX = kOffV + NS * kTileV;          // exchange between the groups: [34][128] floats
-constexpr int kOffBar = kOffX + 34 * 128 * 4;
-constexpr int kOffAbort = kOffBar + 256;
+constexpr int kOffIdx = kOffX + 34 * 128 * 4;        // per producer warp: K and V row indices of its tile, 16 bit
+constexpr int kOffBar = kOffIdx + kProducerWarps * 2 * TK * 2;
+constexpr int kOffAbort = kOffBar + 320;
 constexpr int kSmemBytes = kOffAbort + 16;
 
 // barrier slots (8 bytes each) behind kOffBar
 enum {
-    BAR_FULL = 0, BAR_EMPTY = NS, BAR_QEMPTY = 2 * NS, BAR_SFULL = 2 * NS + NQ, BAR_PREADY = BAR_SFULL + 2,
-    BAR_PFREE = BAR_SFULL + 4, BAR_OFULL = BAR_SFULL + 6, BAR_XFULL = BAR_SFULL + 8, BAR_XEMPTY, BAR_DRAIN,
-    BAR_COUNT = BAR_DRAIN + 3
+    BAR_FULL = 0, BAR_EMPTY = NS, BAR_QEMPTY = 2 * NS,
+    BAR_SFULL = 2 * NS + NQ,      // [2b + i]
+    BAR_PREADY = BAR_SFULL + 4,   // [2b + i]
+    BAR_PFREE = BAR_SFULL + 8,    // [2b + i]
+    BAR_OFULL = BAR_SFULL + 12,   // [b]
+    BAR_XFULL = BAR_SFULL + 14, BAR_XEMPTY, BAR_DRAIN,
+    BAR_COUNT = BAR_DRAIN + 4
 };
-static_assert(BAR_COUNT * 8 <= 256, "barrier area");
+static_assert(BAR_COUNT * 8 <= 320, "barrier area");
 
 // error codes OR-ed into the context's device error word
 enum { ERR_NORMALISE = 1, ERR_MMA = 2, ERR_DRAIN = 4, ERR_PRODUCER = 8 };
@@ -105,19 +112,19 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar)
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 // Bounded wait on a phase parity.  Returns false on time-out or when the CTA is aborting.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const volatile int* abort_flag)
+__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const volatile int* abort_flag)
 {
     for (uint32_t i = 0; i < kSpinLimit; ++i) {
         uint32_t ok;
         asm volatile(
             "{\n.reg .pred p;\n"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
             "selp.u32 %0, 1, 0, p;\n}\n"
             : "=r"(ok)
-            : "r"(bar), "r"(parity), "r"(kSuspendNs)
+            : "r"(bar), "r"(parity)
             : "memory");
         if (ok) return true;
-        if (*abort_flag) return false;
+        if ((i & 31u) == 31u && *abort_flag) return false;
     }
     return false;
 }
@@ -279,14 +286,16 @@ __device__ __forceinline__ uint32_t v_off(int r, int c) { return (uint32_t)((r >
 // position a score column belongs to.
 __device__ __forceinline__ int pos_of_col(int c, int e) { return 32 * c + 4 * (e & 7) + (e >> 3); }
 
-// ---- normalisation of one 128 x 128 score tile by its group (thread = query row = TMEM lane) ----
-// TAIL = false: all 128 columns are real positions; the 32-column chunks are double-buffered
-// in registers so that the next tcgen05.ld is in flight during the arithmetic.
-// TAIL = true (last tile of a history, at most once per unit): compact code, masked columns.
+// ---- normalisation of one 128 x 64 score half tile by its group (thread = query row = TMEM lane) ----
+// `valid` counts the real positions of the half (1..64); column (c, e) of the half holds position
+// pos_of_col(c, e) of the half.
+// TAIL = false: all 64 columns are real positions; the two 32-column chunks are double-buffered
+// in registers so that the second tcgen05.ld is in flight during the arithmetic of the first.
+// TAIL = true (end of a history, at most once per unit and group): compact code, masked columns.
 
 // p = exp2(s c - m) as bf16 into P; returns the largest exponent argument of the row.  With
-// `first` the row's reference m is set from its first 32 scores (column 0 is position 0, always
-// a real one).
+// `first` the row's reference m is set from its first 32 scores (column 0 is the half's position 0,
+// always a real one).
 template <bool TAIL>
 __device__ __forceinline__ float softmax_tile(uint32_t tS, uint32_t tP, float sc, int valid, bool first, float& m_ref)
 {
@@ -323,7 +332,7 @@ __device__ __forceinline__ float softmax_tile(uint32_t tS, uint32_t tP, float sc
     };
     if constexpr (TAIL) {
 #pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
+        for (int c = 0; c < 2; ++c) {
             uint32_t cur[32];
             tmem_ld32(tS + 32 * c, cur);
             tmem_wait_ld32(cur);
@@ -336,15 +345,22 @@ __device__ __forceinline__ float softmax_tile(uint32_t tS, uint32_t tP, float sc
         tmem_ld32(tS + 32, sb);
         chunk(sa, 0);
         tmem_wait_ld32(sb);
-        tmem_ld32(tS + 64, sa);
         chunk(sb, 1);
-        tmem_wait_ld32(sa);
-        tmem_ld32(tS + 96, sb);
-        chunk(sa, 2);
-        tmem_wait_ld32(sb);
-        chunk(sb, 3);
     }
     return fmaxf(mx, mx2);
+}
+
+// Multiplies this thread's row of O (32 columns and the row sum in column 32) by f.
+__device__ __noinline__ void rescale_row(uint32_t tO, float f)
+{
+    uint32_t o[32];
+    tmem_ld32(tO, o);
+    tmem_wait_ld32(o);
+#pragma unroll
+    for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * f);
+    tmem_st32(tO, o);
+    const uint32_t l = tmem_ld1(tO + 32);
+    tmem_st1(tO + 32, __float_as_uint(__uint_as_float(l) * f));
 }
 
 // p = silu(x) = x sigmoid(x) = h (1 + tanh(h)), h = x / 2, as bf16 into P   (sc = scale / 2)
@@ -367,7 +383,7 @@ __device__ __forceinline__ void silu_tile(uint32_t tS, uint32_t tP, float sc, in
     };
     if constexpr (TAIL) {
 #pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
+        for (int c = 0; c < 2; ++c) {
             uint32_t cur[32];
             tmem_ld32(tS + 32 * c, cur);
             tmem_wait_ld32(cur);
@@ -380,15 +396,34 @@ __device__ __forceinline__ void silu_tile(uint32_t tS, uint32_t tP, float sc, in
         tmem_ld32(tS + 32, sb);
         chunk(sa, 0);
         tmem_wait_ld32(sb);
-        tmem_ld32(tS + 64, sa);
         chunk(sb, 1);
-        tmem_wait_ld32(sa);
-        tmem_ld32(tS + 96, sb);
-        chunk(sa, 2);
-        tmem_wait_ld32(sb);
-        chunk(sb, 3);
     }
 }
+
+// The user-specific leading elements of one row (DUB = 2 d_user bytes), as the producers carry
+// them from the compressed cache to a shared-memory tile.
+template <int DUB> struct UserPart;
+template <> struct UserPart<0> {};
+template <> struct UserPart<2> {
+    uint16_t v;
+    __device__ __forceinline__ void load(const char* p) { v = __ldg(reinterpret_cast<const uint16_t*>(p)); }
+    __device__ __forceinline__ void store(unsigned char* p) const { *reinterpret_cast<uint16_t*>(p) = v; }
+};
+template <> struct UserPart<4> {
+    uint32_t v;
+    __device__ __forceinline__ void load(const char* p) { v = __ldg(reinterpret_cast<const uint32_t*>(p)); }
+    __device__ __forceinline__ void store(unsigned char* p) const { *reinterpret_cast<uint32_t*>(p) = v; }
+};
+template <> struct UserPart<8> {
+    uint2 v;
+    __device__ __forceinline__ void load(const char* p) { v = __ldg(reinterpret_cast<const uint2*>(p)); }
+    __device__ __forceinline__ void store(unsigned char* p) const { *reinterpret_cast<uint2*>(p) = v; }
+};
+template <> struct UserPart<16> {
+    uint4 v;
+    __device__ __forceinline__ void load(const char* p) { v = __ldg(reinterpret_cast<const uint4*>(p)); }
+    __device__ __forceinline__ void store(unsigned char* p) const { *reinterpret_cast<uint4*>(p) = v; }
+};
 
 // One work unit of the CTA's share, decoded from its Work record.
 struct Unit {
@@ -415,29 +450,48 @@ __device__ __forceinline__ Work load_work(const Work* p)
 
 // The CTA's tile stream: units blockIdx.x, blockIdx.x + gridDim.x, ... tile by tile.  Every role
 // walks an identical copy, so stage and buffer indices need no communication.  The record of
-// the following unit is always in flight while the current one is processed.
+// the following unit is always in flight while the current one is processed.  Unit w stands for
+// (item, group, query block) = (w / n_mb / G, w / n_mb % G, w % n_mb); the coordinates are
+// stepped with carries instead of divided out each time.
 // KEEP_EMPTY: also stop at units with an empty history (the role that writes their zero rows).
 template <bool KEEP_EMPTY>
 struct Stream {
     const Work* works;
     uint32_t n_mb, n_groups;
-    uint32_t w, n_work;  // the host keeps n_work + gridDim.x below 2^32
+    uint32_t w, n_work;          // the host keeps n_work + gridDim.x below 2^32
+    uint32_t item, grp, mb;      // coordinates of unit w
+    uint32_t d_item, d_grp, d_mb;  // gridDim.x in the same mixed radix
     Unit u;
     Work nxt;    // record of unit w + gridDim.x (valid if that is < n_work)
     int j;       // tile inside the unit
     int g;       // tiles before this one in the stream
     int useq;    // units with tiles before this one
     bool valid;
+    __device__ __forceinline__ void step(uint32_t& it, uint32_t& gr, uint32_t& m) const
+    {
+        m += d_mb;
+        gr += d_grp;
+        it += d_item;
+        if (m >= n_mb) {
+            m -= n_mb;
+            ++gr;
+        }
+        if (gr >= n_groups) {
+            gr -= n_groups;
+            ++it;
+        }
+    }
     __device__ __forceinline__ void take()
     {
         valid = false;
         while (w < n_work) {
             u.wk = nxt;
+            u.grp = (int)grp;
+            u.row0 = (int)mb * 128;
             const uint32_t wn = w + gridDim.x;
-            if (wn < n_work) nxt = load_work(works + (wn / n_mb) / n_groups);
-            const uint32_t t = w / n_mb;
-            u.grp = (int)(t % n_groups);
-            u.row0 = (int)(w - t * n_mb) * 128;
+            uint32_t ni = item, ng = grp, nm = mb;
+            step(ni, ng, nm);
+            if (wn < n_work) nxt = load_work(works + ni);
             u.n_tiles = u.row0 < u.wk.M ? (u.wk.len + TK - 1) / TK : -1;
             u.last_valid = u.wk.len - (u.n_tiles - 1) * TK;
             if (u.n_tiles > 0 || (KEEP_EMPTY && u.n_tiles == 0)) {
@@ -446,7 +500,16 @@ struct Stream {
                 return;
             }
             w = wn;
+            item = ni;
+            grp = ng;
+            mb = nm;
         }
+    }
+    __device__ __forceinline__ void to_next_unit()
+    {
+        w += gridDim.x;
+        step(item, grp, mb);
+        take();
     }
     __device__ __forceinline__ void init(const AttendArgs& a, int n_mb_, int64_t n_work_)
     {
@@ -455,30 +518,34 @@ struct Stream {
         n_groups = (uint32_t)a.cv.n_groups;
         n_work = (uint32_t)n_work_;
         w = blockIdx.x;
+        mb = w % n_mb;
+        grp = (w / n_mb) % n_groups;
+        item = (w / n_mb) / n_groups;
+        d_mb = gridDim.x % n_mb;
+        d_grp = (gridDim.x / n_mb) % n_groups;
+        d_item = (gridDim.x / n_mb) / n_groups;
         g = 0;
         useq = 0;
-        if (w < n_work) nxt = load_work(works + (w / n_mb) / n_groups);
+        if (w < n_work) nxt = load_work(works + item);
         take();
     }
     __device__ __forceinline__ void next_unit()
     {
         g += u.n_tiles > 0 ? u.n_tiles : 0;
         useq += u.n_tiles > 0;
-        w += gridDim.x;
-        take();
+        to_next_unit();
     }
     __device__ __forceinline__ void advance()
     {
         ++g;
         if (++j == u.n_tiles) {
-            w += gridDim.x;
             ++useq;
-            take();
+            to_next_unit();
         }
     }
 };
 
-template <int MODE, bool IDX16>
+template <int MODE, int DUB>
 __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendArgs a, int n_mb, int64_t n_work, int* err_flag)
 {
     extern __shared__ __align__(1024) unsigned char smem[];
@@ -494,18 +561,18 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
     if (tid == 0) {
         for (int s = 0; s < NS; ++s) {
             mbar_init(bar(BAR_FULL + s), 1);  // lane 0 of the producer warp that owns the tile
-            mbar_init(bar(BAR_EMPTY + s), 1);
+            mbar_init(bar(BAR_EMPTY + s), 2);  // one arrival per half
         }
-        for (int q = 0; q < NQ; ++q) mbar_init(bar(BAR_QEMPTY + q), 1);
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(bar(BAR_SFULL + b), 1);
-            mbar_init(bar(BAR_PREADY + b), kGroupThreads);
-            mbar_init(bar(BAR_PFREE + b), 1);
-            mbar_init(bar(BAR_OFULL + b), 1);
+        for (int q = 0; q < NQ; ++q) mbar_init(bar(BAR_QEMPTY + q), 2);  // both score issuers
+        for (int bi = 0; bi < 4; ++bi) {
+            mbar_init(bar(BAR_SFULL + bi), 1);
+            mbar_init(bar(BAR_PREADY + bi), kGroupThreads);
+            mbar_init(bar(BAR_PFREE + bi), 1);
         }
+        for (int b = 0; b < 2; ++b) mbar_init(bar(BAR_OFULL + b), 1);
         mbar_init(bar(BAR_XFULL), kGroupThreads);
         mbar_init(bar(BAR_XEMPTY), kGroupThreads);
-        for (int i = 0; i < 3; ++i) mbar_init(bar(BAR_DRAIN + i), 1);
+        for (int i = 0; i < 4; ++i) mbar_init(bar(BAR_DRAIN + i), 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -531,19 +598,20 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
         const int b = warp >> 2;                    // group = score buffer
         const int row = tid & (kGroupThreads - 1);  // query row inside the block = TMEM lane
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t tS = tmem + lane_base + kColS + 128u * b, tP = tmem + lane_base + kColP + 64u * b,
+        const uint32_t tS0 = tmem + lane_base + kColS + 128u * b, tP0 = tmem + lane_base + kColP + 64u * b,
                        tO = tmem + lane_base + kColO + (uint32_t)kNV * b;
         const float sc = a.scale * (MODE == CKV_SOFTMAX ? kLog2e : 0.5f);
         float* xch = reinterpret_cast<float*>(smem + kOffX);
-        int cnt = 0;    // tiles this group has normalised
+        int cnt = 0;    // half tiles this group has normalised
         int ocnt = 0;   // units in which this group had tiles
         int xcnt = 0;   // units exchanged between the groups
         bool ok = true;
-        T_DECL(8);  // 0 other, 1 wait S, 2 wait PFREE, 3 unused, 4 tile, 5 wait O, 6 exchange wait, 7 rest
+        T_DECL(8);  // 0 other, 1 wait S, 2 wait PFREE, 3 read O, 4 tile, 5 wait O, 6 exchange wait, 7 next unit
         Stream<true> sn;
-        for (sn.init(a, n_mb, n_work); sn.valid && ok; sn.next_unit()) {
+        sn.init(a, n_mb, n_work);
+        for (; sn.valid && ok; sn.next_unit()) {
+            T_ACC(7);  // (time since the end of the previous unit's body: next_unit)
             const Unit& u = sn.u;
-            const int g = sn.g;
             const int r = u.row0 + row;
             const int64_t out_base = ((int64_t)(u.wk.q0 + r) * G + u.grp) * D;
             if (u.n_tiles == 0) {  // empty history: zero output rows
@@ -559,19 +627,22 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                 continue;
             }
             float m_ref = -CUDART_INF_F;
-            int mine = 0;  // tiles of this unit normalised by this group
+            int mine = 0;  // half tiles of this unit normalised by this group
             for (int j = 0; j < u.n_tiles && ok; ++j) {
-                if (((g + j) & 1) != b) continue;
+                const int valid = (j == u.n_tiles - 1 ? u.last_valid : TK) - TH * b;  // real positions of this group's half
+                if (valid <= 0) continue;  // only the second half of a unit's last tile can be empty
+                const int i = cnt & 1;     // buffer pair of this step
+                const uint32_t tS = tS0 + 64u * i, tP = tP0 + 32u * i;
                 T_ACC(0);
-                ok = mbar_wait(bar(BAR_SFULL + b), cnt & 1, abort_flag);
+                ok = mbar_wait(bar(BAR_SFULL + 2 * b + i), (cnt >> 1) & 1, abort_flag);
                 T_ACC(1);
-                if (ok && cnt > 0) ok = mbar_wait(bar(BAR_PFREE + b), (cnt - 1) & 1, abort_flag);  // P_b and O_b are quiet
+                // P_bi is free once the weighted sum of two steps ago has been computed
+                if (ok && cnt >= 2) ok = mbar_wait(bar(BAR_PFREE + 2 * b + i), ((cnt >> 1) - 1) & 1, abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
                 T_ACC(2);
                 if (!ok) break;
                 tc_fence_after();
-                const int valid = j == u.n_tiles - 1 ? u.last_valid : TK;
-                const bool tail = valid < TK;
+                const bool tail = valid < TH;
                 if constexpr (MODE == CKV_SOFTMAX) {
                     for (int attempt = 0; attempt < 2; ++attempt) {
                         const bool first = mine == 0 && attempt == 0;
@@ -579,29 +650,27 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                                               : softmax_tile<false>(tS, tP, sc, valid, first, m_ref);
                         if (!__any_sync(0xffffffffu, mx > kHeadroom)) break;
                         // some row of this warp left the headroom: move its reference, rescale what
-                        // O_b holds so far (its MMAs have finished, see the PFREE wait) and redo the tile
+                        // O_b holds so far (once the previous step's MMAs have finished too) and redo
                         const float shift = mx > kHeadroom ? mx : 0.f;
                         const float f = ex2(-shift);
                         m_ref += shift;
                         if (mine > 0) {
-                            uint32_t o[32];
-                            tmem_ld32(tO, o);
-                            tmem_wait_ld32(o);
-#pragma unroll
-                            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * f);
-                            tmem_st32(tO, o);
-                            const uint32_t l = tmem_ld1(tO + 32);
-                            tmem_st1(tO + 32, __float_as_uint(__uint_as_float(l) * f));
+                            ok = mbar_wait(bar(BAR_PFREE + 2 * b + (i ^ 1)), ((cnt - 1) >> 1) & 1, abort_flag);
+                            ok = __all_sync(0xffffffffu, ok);
+                            if (!ok) break;
+                            tc_fence_after();
+                            rescale_row(tO, f);
                         }
                         tc_wait_st();
                     }
+                    if (!ok) break;
                 } else {
                     if (tail) silu_tile<true>(tS, tP, sc, valid);
                     else silu_tile<false>(tS, tP, sc, valid);
                 }
                 tc_wait_st();
                 tc_fence_before();
-                mbar_arrive(bar(BAR_PREADY + b));
+                mbar_arrive(bar(BAR_PREADY + 2 * b + i));
                 T_ACC(4);
                 ++cnt;
                 ++mine;
@@ -625,6 +694,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                 for (int e = 0; e < 32; ++e) o[e] = __uint_as_float(raw[e]);
                 if constexpr (MODE == CKV_SOFTMAX) l = __uint_as_float(tmem_ld1(tO + 32));
                 tc_fence_before();
+                T_ACC(3);
             } else {
 #pragma unroll
                 for (int e = 0; e < 32; ++e) o[e] = 0.f;
@@ -694,59 +764,72 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                     }
                 }
             }
+            T_ACC(0);
         }
-        T_ACC(7);
+        T_ACC(0);
 #ifdef CKV_STAGE_TIMERS
         if (blockIdx.x == 0 && row == 0)
-            printf("group %d: total %lld | other %lld waitS %lld waitPfree %lld tile %lld waitO %lld xchg %lld rest %lld | tiles %d\n", b,
-                   T_TOTAL(), tmr_[0], tmr_[1], tmr_[2], tmr_[4], tmr_[5], tmr_[6], tmr_[7], cnt);
+            printf("group %d: total %lld | other %lld waitS %lld waitPfree %lld tile %lld waitO %lld readO %lld xchg %lld nextunit %lld | tiles %d\n", b,
+                   T_TOTAL(), tmr_[0], tmr_[1], tmr_[2], tmr_[4], tmr_[5], tmr_[3], tmr_[6], tmr_[7], cnt);
 #endif
         if (!ok) {
             *abort_flag = 1;
             if (lane == 0) atomicOr(err_flag, ERR_NORMALISE);
         }
-    } else if (warp == kMmaWarp) {
-        // --------------------------------------------------------------------- S = Q K^T issue
+    } else if (warp < kPvWarp0) {
+        // --------------------------------------------------------------------- S_bi = Q K_half^T issue
         if (lane == 0) {
-            constexpr uint32_t idesc_s = make_idesc(128, TK, false);
+            const int b = warp - kMmaWarp;
+            constexpr uint32_t idesc_s = make_idesc(128, TH, false);
             Stream<false> ss;
             ss.init(a, n_mb, n_work);
-            int cnt[2] = {0, 0};  // tiles issued per score buffer
+            int cnt = 0;  // half tiles issued
             bool ok = true;
             T_DECL(3);  // 0 issue, 1 wait FULL, 2 wait PREADY
-            while (ok && ss.valid) {
-                const int s = ss.g % NS, b = ss.g & 1;
-                T_ACC(0);
-                ok = mbar_wait(bar(BAR_FULL + s), (ss.g / NS) & 1, abort_flag);
-                T_ACC(1);
-                // S_b is free once group b has read the previous tile that used it
-                if (ok && cnt[b] > 0) ok = mbar_wait(bar(BAR_PREADY + b), (cnt[b] - 1) & 1, abort_flag);
-                T_ACC(2);
-                if (!ok) break;
-                ++cnt[b];
-                tc_fence_after();
-                const uint32_t q_addr = sbase + kOffQ + (ss.useq % NQ) * kTileK, k_addr = sbase + kOffK + s * kTileK;
+            for (; ok && ss.valid; ss.advance()) {
+                const int s = ss.g % NS;
+                const bool last = ss.j == ss.u.n_tiles - 1;
+                if ((last ? ss.u.last_valid : TK) > TH * b) {  // else: empty second half
+                    const int i = cnt & 1;
+                    T_ACC(0);
+                    ok = mbar_wait(bar(BAR_FULL + s), (ss.g / NS) & 1, abort_flag);
+                    T_ACC(1);
+                    // S_bi is free once the group has read the half tile of two steps ago
+                    if (ok && cnt >= 2) ok = mbar_wait(bar(BAR_PREADY + 2 * b + i), ((cnt >> 1) - 1) & 1, abort_flag);
+                    T_ACC(2);
+                    if (!ok) break;
+                    tc_fence_after();
+                    ++cnt;
+                    const uint32_t q_addr = sbase + kOffQ + (ss.useq % NQ) * kTileK,
+                                   k_addr = sbase + kOffK + s * kTileK + b * (TH / 8) * 512;
 #pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks)
-                    umma_ss(tmem + kColS + 128u * b, smem_desc(q_addr + ks * 256, 128, 512),
-                            smem_desc(k_addr + ks * 256, 128, 512), idesc_s, ks > 0 ? 1u : 0u);
-                tc_commit(bar(BAR_SFULL + b));
-                if (ss.j == ss.u.n_tiles - 1) tc_commit(bar(BAR_QEMPTY + ss.useq % NQ));  // Q buffer no longer read
-                ss.advance();
+                    for (int ks = 0; ks < D / 16; ++ks)
+                        umma_ss(tmem + kColS + 64u * (2 * b + i), smem_desc(q_addr + ks * 256, 128, 512),
+                                smem_desc(k_addr + ks * 256, 128, 512), idesc_s, ks > 0 ? 1u : 0u);
+                    tc_commit(bar(BAR_SFULL + 2 * b + i));
+                }
+                if (last) {
+                    // This issuer no longer reads the unit's Q buffer.  It must have seen the unit's last
+                    // tile published even if it issued nothing for it, or it could run units ahead of
+                    // the other issuer and complete a later use of the same barrier in its place.
+                    ok = mbar_wait(bar(BAR_FULL + s), (ss.g / NS) & 1, abort_flag);
+                    if (!ok) break;
+                    tc_commit(bar(BAR_QEMPTY + ss.useq % NQ));
+                }
             }
             T_ACC(0);
 #ifdef CKV_STAGE_TIMERS
             if (blockIdx.x == 0)
-                printf("S issue: total %lld | issue %lld waitFULL %lld waitPREADY %lld | tiles %d\n", T_TOTAL(), tmr_[0], tmr_[1], tmr_[2], ss.g);
+                printf("S issue %d: total %lld | issue %lld waitFULL %lld waitPREADY %lld | tiles %d\n", b, T_TOTAL(), tmr_[0], tmr_[1], tmr_[2], cnt);
 #endif
             if (!ok) {
                 *abort_flag = 1;
                 atomicOr(err_flag, ERR_MMA);
             }
             // nothing of this CTA may still be running on the tensor core at teardown
-            tc_commit(bar(BAR_DRAIN));
+            tc_commit(bar(BAR_DRAIN + b));
             volatile int never = 0;
-            if (!mbar_wait(bar(BAR_DRAIN), 0, &never)) atomicOr(err_flag, ERR_DRAIN);
+            if (!mbar_wait(bar(BAR_DRAIN + b), 0, &never)) atomicOr(err_flag, ERR_DRAIN);
         }
         __syncwarp();
     } else if (warp < kProducerWarp0) {
@@ -760,23 +843,30 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
             bool ok = true;
             T_DECL(2);  // 0 issue, 1 wait PREADY
             for (; ok && sp.valid; sp.advance()) {
-                if ((sp.g & 1) != b) continue;
                 const int s = sp.g % NS;
+                const int valid = (sp.j == sp.u.n_tiles - 1 ? sp.u.last_valid : TK) - TH * b;
+                if (valid <= 0) {  // empty second half: nothing to add, but the stage still needs this half's release
+                    ok = mbar_wait(bar(BAR_FULL + s), (sp.g / NS) & 1, abort_flag);
+                    if (ok) mbar_arrive(bar(BAR_EMPTY + s));
+                    continue;
+                }
+                const int i = cnt & 1;
                 T_ACC(0);
-                ok = mbar_wait(bar(BAR_PREADY + b), cnt & 1, abort_flag);
+                ok = mbar_wait(bar(BAR_PREADY + 2 * b + i), (cnt >> 1) & 1, abort_flag);
                 if (ok) ok = mbar_wait(bar(BAR_FULL + s), (sp.g / NS) & 1, abort_flag);  // completed long ago: makes the V tile visible here
                 T_ACC(1);
                 if (!ok) break;
                 ++cnt;
                 tc_fence_after();
-                const uint32_t v_addr = sbase + kOffV + s * kTileV;
+                const uint32_t v_addr = sbase + kOffV + s * kTileV + b * (TH / 8) * kVGroup;
+                const bool last = sp.j == sp.u.n_tiles - 1 || (sp.j == sp.u.n_tiles - 2 && sp.u.last_valid <= TH * b);
 #pragma unroll
-                for (int kk = 0; kk < TK / 16; ++kk)  // sixteen positions per instruction
-                    umma_ts(tmem + kColO + (uint32_t)kNV * b, tmem + kColP + 64u * b + 8 * kk,
-                            smem_desc(v_addr + kk * 2 * kVGroup, kVGroup, 128), idesc_pv, (sp.j >= 2 || kk > 0) ? 1u : 0u);
+                for (int kk = 0; kk < TH / 16; ++kk)  // sixteen positions per instruction
+                    umma_ts(tmem + kColO + (uint32_t)kNV * b, tmem + kColP + 32u * (2 * b + i) + 8 * kk,
+                            smem_desc(v_addr + kk * 2 * kVGroup, kVGroup, 128), idesc_pv, (sp.j > 0 || kk > 0) ? 1u : 0u);
                 tc_commit(bar(BAR_EMPTY + s));
-                tc_commit(bar(BAR_PFREE + b));
-                if (sp.j >= sp.u.n_tiles - 2) tc_commit(bar(BAR_OFULL + b));  // last tile of its group in the unit
+                tc_commit(bar(BAR_PFREE + 2 * b + i));
+                if (last) tc_commit(bar(BAR_OFULL + b));  // the group's last step of the unit
             }
             T_ACC(0);
 #ifdef CKV_STAGE_TIMERS
@@ -787,9 +877,9 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                 *abort_flag = 1;
                 atomicOr(err_flag, ERR_MMA);
             }
-            tc_commit(bar(BAR_DRAIN + 1 + b));
+            tc_commit(bar(BAR_DRAIN + 2 + b));
             volatile int never = 0;
-            if (!mbar_wait(bar(BAR_DRAIN + 1 + b), 0, &never)) atomicOr(err_flag, ERR_DRAIN);
+            if (!mbar_wait(bar(BAR_DRAIN + 2 + b), 0, &never)) atomicOr(err_flag, ERR_DRAIN);
         }
         __syncwarp();
     } else {
@@ -798,54 +888,57 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
         // copies, so the per-tile bookkeeping is paid by one warp while the others work on their own
         // tiles.  Lane (q = lane / 4, chunk = lane % 4) copies chunk `chunk` of the pool rows of
         // positions 32 rb + 4 q + i (rb, i < 4) into tile rows 32 rb + 8 i + q, and patches the
-        // user-specific leading elements of tile rows 32 rb + lane.
+        // user-specific leading elements of tile rows 32 rb + lane.  The loops are kept rolled on
+        // purpose: the kernel's speed depends on how little code its roles execute.
         const int pw = warp - kProducerWarp0, q = lane >> 2, chunk = lane & 3;
-        const int du_bytes = a.cv.d_user * 2;
         const int patch_pos = 4 * (lane & 7) + (lane >> 3);  // position (inside a 32-block) held by row `lane`
         const uint32_t kv_lane = (uint32_t)(chunk * 128 + q * 16);
         const int64_t pool_stride = (int64_t)a.cv.n_entries * (D * 2);
         const char* poolK0 = reinterpret_cast<const char*>(a.cv.poolK) + chunk * 16;
         const char* poolV0 = reinterpret_cast<const char*>(a.cv.poolV) + chunk * 16;
         const uint16_t* Q = reinterpret_cast<const uint16_t*>(a.queries);
+        uint16_t* sidxK = reinterpret_cast<uint16_t*>(smem + kOffIdx) + pw * 2 * TK;  // this warp's row indices of a tile
+        uint16_t* sidxV = sidxK + TK;
         Stream<false> st;
         st.init(a, n_mb, n_work);
         for (int i = 0; i < pw && st.valid; ++i) st.advance();
         bool ok = true;
-        uint4 xk[4], xv[4];  // row indices of this lane's positions of the next tile (16-bit: packed in .x .y)
-        int64_t unit0 = 0;   // arena unit of that tile's position 0
+        // Everything a tile needs from the compressed cache is requested one tile of this warp ahead:
+        uint2 xk, xv;                     // pool rows of positions 4 lane .. 4 lane + 3
+        UserPart<DUB> uk_n[4], uv_n[4];   // user-specific leading elements (Eq. K: dims [0, d_user)) of tile rows 32 rb + lane
         auto fetch = [&]() {
             if (!st.valid) return;
             const int pos0 = st.u.wk.begin + st.j * TK;
-            unit0 = st.u.wk.base + (int64_t)st.u.grp * st.u.wk.Lpad + pos0;
+            const int64_t unit0 = st.u.wk.base + (int64_t)st.u.grp * st.u.wk.Lpad + pos0;  // arena unit of the tile's position 0
+            const int valid = st.j == st.u.n_tiles - 1 ? st.u.last_valid : TK;
+            xk = xv = make_uint2(0, 0);
+            if (pos0 + 4 * lane < st.u.wk.Lpad) {  // the arena is padded to 32 positions per user
+                xk = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const uint16_t*>(a.cv.idxK) + unit0 + 4 * lane));
+                xv = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const uint16_t*>(a.cv.idxV) + unit0 + 4 * lane));
+            }
+            if constexpr (DUB > 0) {
 #pragma unroll
-            for (int rb = 0; rb < 4; ++rb) {
-                xk[rb] = xv[rb] = make_uint4(0, 0, 0, 0);
-                if (pos0 + 32 * rb + 4 * q < st.u.wk.Lpad) {  // the arena is padded to 32 positions per user
-                    const int64_t un = unit0 + 32 * rb + 4 * q;
-                    if constexpr (IDX16) {
-                        const uint2 a2 = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const uint16_t*>(a.cv.idxK) + un));
-                        const uint2 b2 = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const uint16_t*>(a.cv.idxV) + un));
-                        xk[rb] = make_uint4(a2.x, a2.y, 0, 0);
-                        xv[rb] = make_uint4(b2.x, b2.y, 0, 0);
-                    } else {
-                        xk[rb] = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const int32_t*>(a.cv.idxK) + un));
-                        xv[rb] = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const int32_t*>(a.cv.idxV) + un));
+                for (int rb = 0; rb < 4; ++rb) {
+                    if (32 * rb + patch_pos < valid) {
+                        uk_n[rb].load(reinterpret_cast<const char*>(a.cv.userK) + (unit0 + 32 * rb + patch_pos) * DUB);
+                        uv_n[rb].load(reinterpret_cast<const char*>(a.cv.userV) + (unit0 + 32 * rb + patch_pos) * DUB);
                     }
                 }
-            }
-        };
-        auto row_index = [](const uint4& x, int i) -> uint32_t {
-            if constexpr (IDX16) {
-                const uint32_t w = i < 2 ? x.x : x.y;
-                return (i & 1) ? w >> 16 : w & 0xffffu;
-            } else {
-                return i == 0 ? x.x : (i == 1 ? x.y : (i == 2 ? x.z : x.w));
             }
         };
         fetch();
         T_DECL(6);  // 0 other, 1 wait copies, 2 wait EMPTY, 3 wait QEMPTY, 4 patch+publish, 5 copy issue
         while (st.valid && ok) {
             const int s = st.g % NS;
+            UserPart<DUB> uk[4], uv[4];
+#pragma unroll
+            for (int rb = 0; rb < 4; ++rb) {
+                uk[rb] = uk_n[rb];
+                uv[rb] = uv_n[rb];
+            }
+            *reinterpret_cast<uint2*>(sidxK + 4 * lane) = xk;
+            *reinterpret_cast<uint2*>(sidxV + 4 * lane) = xv;
+            __syncwarp();
             T_ACC(0);
             if (st.g >= NS) {
                 if (lane == 0) ok = mbar_wait(bar(BAR_EMPTY + s), ((st.g / NS) - 1) & 1, abort_flag);
@@ -860,93 +953,45 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                     if (!ok) break;
                 }
                 T_ACC(3);
-                const uint32_t qdst = sbase + kOffQ + (st.useq % NQ) * kTileK;
-#pragma unroll 4
-                for (int rr = 0; rr < 16; ++rr) {
-                    const int r = 8 * rr + q;
-                    const bool in = st.u.row0 + r < st.u.wk.M;
-                    const uint16_t* src = Q + ((int64_t)(st.u.wk.q0 + st.u.row0 + (in ? r : 0)) * G + st.u.grp) * D + chunk * 8;
-                    cp_async16(qdst + k_off(r, chunk), src, in ? 16u : 0u);
+                const uint32_t qdst = sbase + kOffQ + (st.useq % NQ) * kTileK + kv_lane;
+                const int rows_in = st.u.wk.M - st.u.row0;
+                const uint16_t* qsrc = Q + ((int64_t)(st.u.wk.q0 + st.u.row0 + q) * G + st.u.grp) * D + chunk * 8;
+#pragma unroll 2
+                for (int rr = 0; rr < 16; ++rr) {  // rows 8 rr + q
+                    const bool in = 8 * rr + q < rows_in;
+                    cp_async16(qdst + 512 * rr, in ? qsrc + (int64_t)8 * rr * G * D : Q, in ? 16u : 0u);
                 }
             }
             const char* pk = poolK0 + st.u.grp * pool_stride;
             const char* pv = poolV0 + st.u.grp * pool_stride;
             const uint32_t kdst = sbase + kOffK + s * kTileK + kv_lane, vdst = sbase + kOffV + s * kTileV + kv_lane;
             const int valid = st.j == st.u.n_tiles - 1 ? st.u.last_valid : TK;
-            if (valid == TK) {
-#pragma unroll
-                for (int rb = 0; rb < 4; ++rb)
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        cp_async16(kdst + 2048 * rb + 512 * i, pk + (size_t)row_index(xk[rb], i) * (D * 2), 16u);
-                        cp_async16(vdst + 4 * kVGroup * rb + kVGroup * i, pv + (size_t)row_index(xv[rb], i) * (D * 2), 16u);
-                    }
-            } else {  // rows of positions beyond the history are zero
-#pragma unroll
-                for (int rb = 0; rb < 4; ++rb)
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const uint32_t nb = 32 * rb + 4 * q + i < valid ? 16u : 0u;
-                        cp_async16(kdst + 2048 * rb + 512 * i, pk + (size_t)row_index(xk[rb], i) * (D * 2), nb);
-                        cp_async16(vdst + 4 * kVGroup * rb + kVGroup * i, pv + (size_t)row_index(xv[rb], i) * (D * 2), nb);
-                    }
+#pragma unroll 2
+            for (int it = 0; it < 16; ++it) {  // rb = it / 4, i = it % 4: position 32 rb + 4 q + i -> tile row 32 rb + 8 i + q
+                const int pos = 32 * (it >> 2) + 4 * q + (it & 3);
+                const uint32_t nb = pos < valid ? 16u : 0u;  // rows of positions beyond the history are zero
+                cp_async16(kdst + 512 * it, pk + (size_t)sidxK[pos] * (D * 2), nb);
+                cp_async16(vdst + kVGroup * it, pv + (size_t)sidxV[pos] * (D * 2), nb);
             }
             cp_async_commit();
             T_ACC(5);
-            // this lane's user-specific leading elements (Eq. K: dims [0, d_user)) of tile rows 32 rb + lane
-            uint4 uk[4], uv[4];
-#pragma unroll
-            for (int rb = 0; rb < 4; ++rb) {
-                uk[rb] = uv[rb] = make_uint4(0, 0, 0, 0);
-                if (du_bytes > 0 && 32 * rb + patch_pos < valid) {
-                    const char* ku = reinterpret_cast<const char*>(a.cv.userK) + (unit0 + 32 * rb + patch_pos) * du_bytes;
-                    const char* vu = reinterpret_cast<const char*>(a.cv.userV) + (unit0 + 32 * rb + patch_pos) * du_bytes;
-                    if (du_bytes == 4) {
-                        uk[rb].x = __ldg(reinterpret_cast<const uint32_t*>(ku));
-                        uv[rb].x = __ldg(reinterpret_cast<const uint32_t*>(vu));
-                    } else if (du_bytes == 2) {
-                        uk[rb].x = __ldg(reinterpret_cast<const uint16_t*>(ku));
-                        uv[rb].x = __ldg(reinterpret_cast<const uint16_t*>(vu));
-                    } else if (du_bytes == 8) {
-                        const uint2 x = __ldg(reinterpret_cast<const uint2*>(ku)), y = __ldg(reinterpret_cast<const uint2*>(vu));
-                        uk[rb] = make_uint4(x.x, x.y, 0, 0);
-                        uv[rb] = make_uint4(y.x, y.y, 0, 0);
-                    } else {
-                        uk[rb] = __ldg(reinterpret_cast<const uint4*>(ku));
-                        uv[rb] = __ldg(reinterpret_cast<const uint4*>(vu));
-                    }
-                }
-            }
-            // the indices of this warp's next tile travel while the copies land
+            // what this warp's next tile needs travels while the copies land
             for (int i = 0; i < kProducerWarps && st.valid; ++i) st.advance();
             fetch();
             T_ACC(0);
             cp_async_wait<0>();
             __syncwarp();  // a row's chunks were copied by four lanes of this warp
             T_ACC(1);
-            if (du_bytes > 0) {
+            if constexpr (DUB > 0) {
 #pragma unroll
                 for (int rb = 0; rb < 4; ++rb) {
                     if (32 * rb + patch_pos < valid) {  // zero rows beyond the history stay zero
-                        unsigned char* kd = smem + kOffK + s * kTileK + k_off(32 * rb + lane, 0);
-                        unsigned char* vd = smem + kOffV + s * kTileV + v_off(32 * rb + lane, 0);
-                        if (du_bytes == 4) {
-                            *reinterpret_cast<uint32_t*>(kd) = uk[rb].x;
-                            *reinterpret_cast<uint32_t*>(vd) = uv[rb].x;
-                        } else if (du_bytes == 2) {
-                            *reinterpret_cast<uint16_t*>(kd) = (uint16_t)uk[rb].x;
-                            *reinterpret_cast<uint16_t*>(vd) = (uint16_t)uv[rb].x;
-                        } else if (du_bytes == 8) {
-                            *reinterpret_cast<uint2*>(kd) = make_uint2(uk[rb].x, uk[rb].y);
-                            *reinterpret_cast<uint2*>(vd) = make_uint2(uv[rb].x, uv[rb].y);
-                        } else {
-                            *reinterpret_cast<uint4*>(kd) = uk[rb];
-                            *reinterpret_cast<uint4*>(vd) = uv[rb];
-                        }
+                        uk[rb].store(smem + kOffK + s * kTileK + k_off(32 * rb + lane, 0));
+                        uv[rb].store(smem + kOffV + s * kTileV + v_off(32 * rb + lane, 0));
                     }
                 }
             }
-            fence_proxy_async();
+            fence_proxy_async();  // by the writing threads themselves: a fence on the reading side alone is not enough
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(BAR_FULL + s));
             T_ACC(4);
@@ -974,9 +1019,10 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
 
 }  // namespace
 
-bool umma_supported(int dtype, int head_dim, int d_user)
+bool umma_supported(int dtype, int head_dim, int d_user, int idx_bytes)
 {
-    return dtype == CKV_BF16 && head_dim == D && (d_user == 0 || d_user == 1 || d_user == 2 || d_user == 4 || d_user == 8);
+    return dtype == CKV_BF16 && head_dim == D && idx_bytes == 2 &&
+           (d_user == 0 || d_user == 1 || d_user == 2 || d_user == 4 || d_user == 8);
 }
 
 cudaError_t launch_attend_umma(int max_M, const AttendArgs& a, int n_sms, int* err_flag, cudaStream_t s)
@@ -986,16 +1032,21 @@ cudaError_t launch_attend_umma(int max_M, const AttendArgs& a, int n_sms, int* e
     const int64_t n_work = (int64_t)a.n_items * n_mb * a.cv.n_groups;
     if (n_work + n_sms >= (int64_t)1 << 32) return cudaErrorInvalidValue;  // the kernel counts units in 32 bits
     const unsigned grid = (unsigned)(n_work < n_sms ? n_work : n_sms);
-    const bool i16 = a.cv.idx_bytes == 2;
     auto go = [&](auto kernel) {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (e != cudaSuccess) return e;
         kernel<<<grid, kThreads, kSmemBytes, s>>>(a, n_mb, n_work, err_flag);
         return cudaGetLastError();
     };
-    if (a.mode == CKV_SOFTMAX)
-        return i16 ? go(attend_umma_kernel<CKV_SOFTMAX, true>) : go(attend_umma_kernel<CKV_SOFTMAX, false>);
-    return i16 ? go(attend_umma_kernel<CKV_SILU_OVER_L, true>) : go(attend_umma_kernel<CKV_SILU_OVER_L, false>);
+    const bool sm = a.mode == CKV_SOFTMAX;
+    switch (a.cv.d_user) {
+        case 0: return sm ? go(attend_umma_kernel<CKV_SOFTMAX, 0>) : go(attend_umma_kernel<CKV_SILU_OVER_L, 0>);
+        case 1: return sm ? go(attend_umma_kernel<CKV_SOFTMAX, 2>) : go(attend_umma_kernel<CKV_SILU_OVER_L, 2>);
+        case 2: return sm ? go(attend_umma_kernel<CKV_SOFTMAX, 4>) : go(attend_umma_kernel<CKV_SILU_OVER_L, 4>);
+        case 4: return sm ? go(attend_umma_kernel<CKV_SOFTMAX, 8>) : go(attend_umma_kernel<CKV_SILU_OVER_L, 8>);
+        case 8: return sm ? go(attend_umma_kernel<CKV_SOFTMAX, 16>) : go(attend_umma_kernel<CKV_SILU_OVER_L, 16>);
+    }
+    return cudaErrorInvalidValue;
 }
 
 }  // namespace ckv

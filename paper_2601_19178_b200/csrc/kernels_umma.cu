@@ -128,8 +128,14 @@ __device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const vola
     }
     return false;
 }
-// 16-byte copy global -> shared; src_bytes = 0 fills the destination with zeros instead
+// 16-byte copy global -> shared; src_bytes = 0 fills the destination with zeros instead.
+// Pool rows go through L1 (with skewed indices the hot rows then stop hammering a few L2 lines
+// from every SM at once); rows that are read once bypass it.
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async16_once(uint32_t dst, const void* src, uint32_t src_bytes)
 {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
 }
@@ -267,7 +273,9 @@ __device__ __forceinline__ float max3(float a, float b, float c)
 // Optional stage timers (debug builds with -DCKV_STAGE_TIMERS): one thread per role of CTA 0
 // accumulates clock64 intervals per stage and prints them when the kernel ends.
 #ifdef CKV_STAGE_TIMERS
-#define T_DECL(n) long long tmr_[n] = {}; long long tmr_last_ = clock64(); const long long tmr_start_ = tmr_last_
+__device__ __forceinline__ unsigned long long t_global_ns() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
+#define T_DECL(n) long long tmr_[n] = {}; long long tmr_last_ = clock64(); const long long tmr_start_ = tmr_last_; const unsigned long long tmr_ns0_ = t_global_ns()
+#define T_MHZ() (1e3 * (double)(clock64() - tmr_start_) / (double)(t_global_ns() - tmr_ns0_))
 #define T_ACC(i) do { const long long t_now_ = clock64(); tmr_[i] += t_now_ - tmr_last_; tmr_last_ = t_now_; } while (0)
 #define T_TOTAL() (clock64() - tmr_start_)
 #else
@@ -769,8 +777,8 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
         T_ACC(0);
 #ifdef CKV_STAGE_TIMERS
         if (blockIdx.x == 0 && row == 0)
-            printf("group %d: total %lld | other %lld waitS %lld waitPfree %lld tile %lld waitO %lld readO %lld xchg %lld nextunit %lld | tiles %d\n", b,
-                   T_TOTAL(), tmr_[0], tmr_[1], tmr_[2], tmr_[4], tmr_[5], tmr_[3], tmr_[6], tmr_[7], cnt);
+            printf("group %d: %.0f MHz total %lld | other %lld waitS %lld waitPfree %lld tile %lld waitO %lld readO %lld xchg %lld nextunit %lld | tiles %d\n", b,
+                   T_MHZ(), T_TOTAL(), tmr_[0], tmr_[1], tmr_[2], tmr_[4], tmr_[5], tmr_[3], tmr_[6], tmr_[7], cnt);
 #endif
         if (!ok) {
             *abort_flag = 1;
@@ -959,7 +967,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
 #pragma unroll 2
                 for (int rr = 0; rr < 16; ++rr) {  // rows 8 rr + q
                     const bool in = 8 * rr + q < rows_in;
-                    cp_async16(qdst + 512 * rr, in ? qsrc + (int64_t)8 * rr * G * D : Q, in ? 16u : 0u);
+                    cp_async16_once(qdst + 512 * rr, in ? qsrc + (int64_t)8 * rr * G * D : Q, in ? 16u : 0u);
                 }
             }
             const char* pk = poolK0 + st.u.grp * pool_stride;

@@ -80,7 +80,7 @@ __device__ __forceinline__ void load_indices(const void* base, int64_t unit, int
 }
 
 template <int MT, int MODE, bool IDX16>
-__global__ void __launch_bounds__(128) attend_mma_kernel(const AttendArgs a, const void* poolKp,
+__global__ void __launch_bounds__(128, MT == 1 ? 5 : 1) attend_mma_kernel(const AttendArgs a, const void* poolKp,
                                                          const void* poolVp, int n_mb)
 {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -137,6 +137,32 @@ __global__ void __launch_bounds__(128) attend_mma_kernel(const AttendArgs a, con
         int ik[4], iv[8];
         const int64_t unitK = unit0 + p0 + 4 * g;   // this lane's four K positions
         const int64_t unitV = unit0 + p0 + 8 * t;   // this lane's eight V positions
+        // (the user parts are requested first: they come from HBM like the indices, and a warp
+        // issues in order, so behind the gathers they would only start once the indices are back)
+        uint4 uk4[2], uv4[4];
+        if (d_user == 1) {
+            if (t == 0) {
+                const uint2 r = __ldg(reinterpret_cast<const uint2*>(uK + unitK));
+                uk4[0].x = r.x;
+                uk4[0].y = r.y;
+            }
+            if (g == 0) uv4[0] = __ldg(reinterpret_cast<const uint4*>(uV + unitV));
+        } else if (d_user == 2) {
+            if (t == 0) uk4[0] = __ldg(reinterpret_cast<const uint4*>(uK + unitK * 2));
+            if (g < 2) {
+                uv4[0] = __ldg(reinterpret_cast<const uint4*>(uV + unitV * 2));
+                uv4[1] = __ldg(reinterpret_cast<const uint4*>(uV + unitV * 2) + 1);
+            }
+        } else if (d_user == 4) {
+            if (t < 2) {
+                uk4[0] = __ldg(reinterpret_cast<const uint4*>(uK + unitK * 4));
+                uk4[1] = __ldg(reinterpret_cast<const uint4*>(uK + unitK * 4) + 1);
+            }
+            if (g < 4) {
+#pragma unroll
+                for (int jj = 0; jj < 4; ++jj) uv4[jj] = __ldg(reinterpret_cast<const uint4*>(uV + unitV * 4) + jj);
+            }
+        }
         load_indices<IDX16, 4>(a.cv.idxK, unitK, ik);
         load_indices<IDX16, 8>(a.cv.idxV, unitV, iv);
         uint4 kf[4];
@@ -145,19 +171,70 @@ __global__ void __launch_bounds__(128) attend_mma_kernel(const AttendArgs a, con
         for (int nt = 0; nt < 4; ++nt) kf[nt] = __ldg(reinterpret_cast<const uint4*>(pK + (int64_t)ik[nt] * (D * 2)));
 #pragma unroll
         for (int j = 0; j < 8; ++j) vr[j] = __ldg(reinterpret_cast<const uint2*>(pV + (int64_t)iv[j] * (D * 2)));
-        if (patchK0) {  // Eq. K: dims [0, d_user) come from the user-specific part
-#pragma unroll
-            for (int nt = 0; nt < 4; ++nt) {
-                const uint16_t* u = uK + (unitK + nt) * d_user + 2 * t;
-                uint32_t w = __ldg(u);
-                w |= patchK1 ? (uint32_t)__ldg(u + 1) << 16 : (kf[nt].x & 0xffff0000u);
-                kf[nt].x = w;
+        // Eq. K: dims [0, d_user) come from the user-specific part.  The user parts of this lane's four K
+        // positions (and of its eight V positions) are contiguous in the cache: for the common widths
+        // they are fetched with one or two wide loads instead of one 2-byte load per element.
+        if (d_user == 1) {
+            if (t == 0) {
+                const uint2 r = make_uint2(uk4[0].x, uk4[0].y);
+                kf[0].x = (kf[0].x & 0xffff0000u) | (r.x & 0xffffu);
+                kf[1].x = (kf[1].x & 0xffff0000u) | (r.x >> 16);
+                kf[2].x = (kf[2].x & 0xffff0000u) | (r.y & 0xffffu);
+                kf[3].x = (kf[3].x & 0xffff0000u) | (r.y >> 16);
             }
-        }
-        if (patchV) {
+            if (g == 0) {
+                const uint4 r = uv4[0];
+                const uint32_t w[4] = {r.x, r.y, r.z, r.w};
 #pragma unroll
-            for (int j = 0; j < 8; ++j)
-                vr[j].x = (vr[j].x & 0xffff0000u) | (uint32_t)__ldg(uV + (unitV + j) * d_user + g);
+                for (int j = 0; j < 8; ++j)
+                    vr[j].x = (vr[j].x & 0xffff0000u) | ((j & 1) ? w[j >> 1] >> 16 : w[j >> 1] & 0xffffu);
+            }
+        } else if (d_user == 2) {
+            if (t == 0) {
+                const uint4 r = uk4[0];
+                kf[0].x = r.x;
+                kf[1].x = r.y;
+                kf[2].x = r.z;
+                kf[3].x = r.w;
+            }
+            if (g < 2) {
+                const uint4 r0 = uv4[0], r1 = uv4[1];
+                const uint32_t w[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
+#pragma unroll
+                for (int j = 0; j < 8; ++j) vr[j].x = (vr[j].x & 0xffff0000u) | (g ? w[j] >> 16 : w[j] & 0xffffu);
+            }
+        } else if (d_user == 4) {
+            if (t < 2) {
+                const uint4 r0 = uk4[0], r1 = uk4[1];
+                kf[0].x = t ? r0.y : r0.x;
+                kf[1].x = t ? r0.w : r0.z;
+                kf[2].x = t ? r1.y : r1.x;
+                kf[3].x = t ? r1.w : r1.z;
+            }
+            if (g < 4) {
+#pragma unroll
+                for (int jj = 0; jj < 4; ++jj) {  // positions 2 jj and 2 jj + 1
+                    const uint4 r = uv4[jj];
+                    const uint32_t a0 = (g & 2) ? r.y : r.x, a1 = (g & 2) ? r.w : r.z;
+                    vr[2 * jj].x = (vr[2 * jj].x & 0xffff0000u) | ((g & 1) ? a0 >> 16 : a0 & 0xffffu);
+                    vr[2 * jj + 1].x = (vr[2 * jj + 1].x & 0xffff0000u) | ((g & 1) ? a1 >> 16 : a1 & 0xffffu);
+                }
+            }
+        } else {
+            if (patchK0) {
+#pragma unroll
+                for (int nt = 0; nt < 4; ++nt) {
+                    const uint16_t* u = uK + (unitK + nt) * d_user + 2 * t;
+                    uint32_t w = __ldg(u);
+                    w |= patchK1 ? (uint32_t)__ldg(u + 1) << 16 : (kf[nt].x & 0xffff0000u);
+                    kf[nt].x = w;
+                }
+            }
+            if (patchV) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    vr[j].x = (vr[j].x & 0xffff0000u) | (uint32_t)__ldg(uV + (unitV + j) * d_user + g);
+            }
         }
         // V B-fragments: k-slots (2t, 2t+1, 2t+8, 2t+9) of block b are positions
         // 8t + (2b, 4+2b, 2b+1, 5+2b)

@@ -51,6 +51,17 @@ __device__ __forceinline__ float load_elem(const void* base, int64_t i)
         return __ldg(reinterpret_cast<const float*>(base) + i);
 }
 
+// the user part of one unit (2, 4 or 8 bytes, naturally aligned) into the low end of 8 bytes
+__device__ __forceinline__ uint2 load_user(const void* base, int64_t unit, int bytes)
+{
+    const char* p = reinterpret_cast<const char*>(base) + unit * bytes;
+    uint2 r = make_uint2(0, 0);
+    if (bytes == 8) r = __ldg(reinterpret_cast<const uint2*>(p));
+    else if (bytes == 4) r.x = __ldg(reinterpret_cast<const uint32_t*>(p));
+    else r.x = __ldg(reinterpret_cast<const uint16_t*>(p));
+    return r;
+}
+
 __device__ __forceinline__ int load_idx(const void* base, int64_t unit, int idx_bytes)
 {
     return idx_bytes == 2 ? (int)__ldg(reinterpret_cast<const uint16_t*>(base) + unit)
@@ -89,6 +100,9 @@ __global__ void __launch_bounds__(kWarps * 32) attend_simt_kernel(const AttendAr
     const char* poolK = (const char*)cv.poolK + (int64_t)g * cv.n_entries * D * ES + ch * 16;
     const char* poolV = (const char*)cv.poolV + (int64_t)g * cv.n_entries * D * ES + ch * 16;
     const bool owns_user = ch * EPL < d_user;
+    // user part of a position in one load of at most 8 bytes: it fits the row's first lane and its size is a power of two
+    const int user_bytes = d_user * ES;
+    const bool wide_user = d_user <= EPL && (user_bytes == 2 || user_bytes == 4 || user_bytes == 8);
     const int end = it.begin + it.len;
     const float qscale = a.scale * (MODE == CKV_SOFTMAX ? kLog2e : 1.0f);
 
@@ -115,6 +129,27 @@ __global__ void __launch_bounds__(kWarps * 32) attend_simt_kernel(const AttendAr
             for (int e = 0; e < EPL; ++e) acc[r][e] = 0.f;
         }
 
+        // Coalesced loads of the compressed cache for the PPW * UNR positions of a step (lane l takes
+        // positions l, l + 32, ...): the indices and, where a user part is one 2..16-byte word, the user
+        // parts.  They are requested one step ahead: all of it streams from HBM, which takes several
+        // times longer than a pool row takes from L2.
+        constexpr int NL = (PPW * UNR + 31) / 32;
+        int my_ik[NL], my_iv[NL];
+        uint2 my_uk[NL], my_uv[NL];
+        auto request_indices = [&](int p0) {
+#pragma unroll
+            for (int l = 0; l < NL; ++l) {
+                const int my_p = p0 + l * 32 + lane;
+                const int64_t my_unit = unit0 + ((l * 32 + lane < PPW * UNR && my_p < end) ? my_p : it.begin);
+                my_ik[l] = load_idx(cv.idxK, my_unit, idx_bytes);
+                my_iv[l] = load_idx(cv.idxV, my_unit, idx_bytes);
+                if (wide_user) {
+                    my_uk[l] = load_user(cv.userK, my_unit, user_bytes);
+                    my_uv[l] = load_user(cv.userV, my_unit, user_bytes);
+                }
+            }
+        };
+        if (it.begin + warp * (PPW * UNR) < end) request_indices(it.begin + warp * (PPW * UNR));
         for (int p0 = it.begin + warp * (PPW * UNR); p0 < end; p0 += kWarps * PPW * UNR) {
             bool valid[UNR];
             uint4 kraw[UNR], vraw[UNR];
@@ -124,11 +159,21 @@ __global__ void __launch_bounds__(kWarps * 32) attend_simt_kernel(const AttendAr
                 const int p = p0 + j * PPW + sub;
                 valid[j] = p < end;
                 unit[j] = unit0 + (valid[j] ? p : it.begin);
-                const int ik = load_idx(cv.idxK, unit[j], idx_bytes);
-                const int iv = load_idx(cv.idxV, unit[j], idx_bytes);
+            }
+#pragma unroll
+            for (int j = 0; j < UNR; ++j) {
+                const int src = (j * PPW) % 32 + sub;
+                const int ik = __shfl_sync(0xffffffffu, my_ik[(j * PPW) / 32], src), iv = __shfl_sync(0xffffffffu, my_iv[(j * PPW) / 32], src);
                 kraw[j] = ldg16(poolK + (int64_t)ik * (D * ES));
                 vraw[j] = ldg16(poolV + (int64_t)iv * (D * ES));
             }
+            uint2 cur_uk[NL], cur_uv[NL];  // this step's user parts: the next request overwrites my_uk, my_uv
+#pragma unroll
+            for (int l = 0; l < NL; ++l) {
+                cur_uk[l] = my_uk[l];
+                cur_uv[l] = my_uv[l];
+            }
+            if (p0 + kWarps * PPW * UNR < end) request_indices(p0 + kWarps * PPW * UNR);
             float s[UNR][QB];
             float v[UNR][EPL];
 #pragma unroll
@@ -136,7 +181,29 @@ __global__ void __launch_bounds__(kWarps * 32) attend_simt_kernel(const AttendAr
                 float k[EPL];
                 unpack16<BF16>(kraw[j], k);
                 unpack16<BF16>(vraw[j], v[j]);
-                if (owns_user) {  // Eq. K: the first d_user dims come from the user part
+                if (wide_user) {  // Eq. K: the first d_user dims come from the user part
+                    // hand the position's user part to the lanes of its row (the first of them uses it)
+                    const int src = (j * PPW) % 32 + sub;
+                    uint4 ukj = make_uint4(0, 0, 0, 0), uvj = make_uint4(0, 0, 0, 0);
+                    ukj.x = __shfl_sync(0xffffffffu, cur_uk[(j * PPW) / 32].x, src);
+                    uvj.x = __shfl_sync(0xffffffffu, cur_uv[(j * PPW) / 32].x, src);
+                    if (user_bytes > 4) {
+                        ukj.y = __shfl_sync(0xffffffffu, cur_uk[(j * PPW) / 32].y, src);
+                        uvj.y = __shfl_sync(0xffffffffu, cur_uv[(j * PPW) / 32].y, src);
+                    }
+                    if (owns_user) {
+                        float ku[EPL], vu[EPL];
+                        unpack16<BF16>(ukj, ku);
+                        unpack16<BF16>(uvj, vu);
+#pragma unroll
+                        for (int e = 0; e < EPL; ++e) {
+                            if (e < d_user) {
+                                k[e] = ku[e];
+                                v[j][e] = vu[e];
+                            }
+                        }
+                    }
+                } else if (owns_user) {
 #pragma unroll
                     for (int e = 0; e < EPL; ++e) {
                         if (ch * EPL + e < d_user) {

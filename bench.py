@@ -125,9 +125,33 @@ def _oracle_rate(w, data, n_users: int, n_threads: int = 0):
     return pos / dt, dt, O.max_threads(), n_users, pos
 
 
+def rank_env():
+    """(rank, world size, local rank) of this process as torchrun exports them; (0, 1, 0) when run alone."""
+    return (int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1")),
+            int(os.environ.get("LOCAL_RANK", "0")))
+
+
+def rank_seed(w, rank: int) -> int:
+    """Weak scaling: every rank serves its own users of the same workload shape."""
+    return w.seed + 1000 * rank
+
+
+def reduce_over_ranks(elapsed, positions: int, users: int, dist=None, device="cpu"):
+    """Whole-job figures from per-rank ones: the slowest rank's time, everybody's positions and users.
+    No data of the decode path crosses ranks; this is the only communication of the benchmark."""
+    if dist is None:
+        return float(elapsed), int(positions), int(users)
+    import torch
+    t = torch.tensor([float(elapsed)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    c = torch.tensor([int(positions), int(users)], dtype=torch.int64, device=device)
+    dist.all_reduce(c, op=dist.ReduceOp.SUM)
+    return float(t.item()), int(c[0].item()), int(c[1].item())
+
+
 def run_reference(args, w):
     """The oracle, as it stands, on the host cores: each step is a bounded sample of users."""
-    rank = int(os.environ.get("RANK", "0"))
+    rank, _, _ = rank_env()
     if rank != 0:
         return
     data = synth.generate(w)
@@ -165,9 +189,7 @@ def run_ours(args, w):
     import paper_2601_19178_b200 as ckv
     from paper_2601_19178_b200.session import as_device_tensor as dev
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local = rank_env()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
     torch.cuda.set_device(local)
@@ -177,7 +199,7 @@ def run_ours(args, w):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     # weak scaling: every rank serves its own users of the same workload shape
-    data = synth.generate(w, seed=w.seed + 1000 * rank)
+    data = synth.generate(w, seed=rank_seed(w, rank))
     tdt = torch.float32 if w.dtype == "f32" else torch.bfloat16
     s = ckv.CollectiveKV(w.n_groups, w.head_dim, tdt, w.mode, device=local)
     s.pool_load(dev(data["pool_K"], w.dtype), dev(data["pool_V"], w.dtype))
@@ -261,11 +283,7 @@ def run_ours(args, w):
     if dist is not None:
         dist.barrier()
     step_ms = [a.elapsed_time(b) for a, b in zip(ev0, ev1)]
-    total_ms = float(sum(step_ms))
-    if dist is not None:
-        t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms, job_positions, job_users = reduce_over_ranks(float(sum(step_ms)), positions, w.n_users, dist, "cuda")
 
     # end to end: host query buffer in, host output buffer out, through the same C-ABI call
     q_host = torch.empty(q.shape, dtype=q.dtype).pin_memory()
@@ -281,11 +299,7 @@ def run_ours(args, w):
     for _ in range(e2e_steps):
         s.attend(users, q_off, q_host, o_host)
         torch.cuda.synchronize()
-    e2e_s = time.perf_counter() - t0
-    if dist is not None:
-        t = torch.tensor([e2e_s], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
+    e2e_s, _, _ = reduce_over_ranks(time.perf_counter() - t0, positions, w.n_users, dist, "cuda")
     clocks = sampler.finish() if sampler else None
 
     if rank != 0:
@@ -296,7 +310,7 @@ def run_ours(args, w):
     peak, peak_kind = _peaks()
     kern_s = statistics.mean(kern_ns) * 1e-9
     achieved = algo_bytes / kern_s / 1e9
-    value = positions * world * args.steps / (total_ms * 1e-3)
+    value = job_positions * args.steps / (total_ms * 1e-3)
     cpu = None
     if not args.no_cpu:
         rate, dt, cores, n_u, pos = _oracle_rate(w, data, CPU_SAMPLE_USERS.get(w.name, w.n_users))
@@ -321,9 +335,9 @@ def run_ours(args, w):
                    "l2": "flushed between timed steps (256 MiB overwrite)",
                    "kernel_family": s.stat("kernel"), "work_items": s.stat("work_items"),
                    "split_items": s.stat("split_items")},
-        "users_per_sec": w.n_users * world * args.steps / (total_ms * 1e-3),
+        "users_per_sec": job_users * args.steps / (total_ms * 1e-3),
         "clocks": clocks,
-        "e2e": {"value": positions * world * e2e_steps / e2e_s, "unit": UNIT,
+        "e2e": {"value": job_positions * e2e_steps / e2e_s, "unit": UNIT,
                 "h2d_bytes_per_step": q_host.numel() * q_host.element_size() + users.nbytes + q_off.nbytes,
                 "d2h_bytes_per_step": o_host.numel() * o_host.element_size(), "ms_per_step": 1e3 * e2e_s / e2e_steps},
         "gpu_launches": launches,

@@ -51,7 +51,7 @@ def _peaks():
 # from the ncu captures summarised under profiles/ (attend_*_kernel_<workload>.md).  cfg3 and cfg5
 # were captured on a cut of the workload and scaled by the number of users.  Set an entry to None
 # when its kernel changes after the capture.
-TRAFFIC_BYTES = {"cfg2": 191553536, "cfg3": 1084903424, "cfg4": 372967680, "cfg5": 1858093056}
+TRAFFIC_BYTES = {"cfg2": 190658560, "cfg3": 1090254848, "cfg4": 372389376, "cfg5": 1857857536}
 # transcendental evaluations per SM per clock (ex2 / tanh issue rate of the special-function unit)
 XU_PER_SM_CLK = 16
 

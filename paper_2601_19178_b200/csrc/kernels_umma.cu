@@ -73,7 +73,8 @@ constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColS = 0, kColP = 256, kColO = 384;  // S_bi at kColS + 64 (2b+i), P_bi at kColP + 32 (2b+i), O_b at kColO + 48 b
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kHeadroom = 64.0f;       // log2 units a score may exceed the reference maximum
-constexpr uint32_t kSpinLimit = 1u << 20;  // polls of a wait before the CTA gives up
+constexpr uint32_t kSpinLimit = 1u << 18;  // polls of a wait before the CTA gives up
+constexpr uint32_t kSuspendNs = 4000;      // how long one poll may stay suspended in hardware (longer hints wake later)
 static_assert(NS > kProducerWarps, "every producer warp holds one stage while it copies");
 
 // dynamic shared memory map
@@ -118,10 +119,10 @@ __device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const vola
         uint32_t ok;
         asm volatile(
             "{\n.reg .pred p;\n"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
             "selp.u32 %0, 1, 0, p;\n}\n"
             : "=r"(ok)
-            : "r"(bar), "r"(parity)
+            : "r"(bar), "r"(parity), "r"(kSuspendNs)
             : "memory");
         if (ok) return true;
         if ((i & 31u) == 31u && *abort_flag) return false;

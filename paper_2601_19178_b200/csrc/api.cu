@@ -68,7 +68,8 @@ struct ckv_ctx {
     // pool
     int n_entries = 0, d_shared = 0, d_user = 0, idx_bytes = 0;
     void* pool = nullptr;  // K rows then V rows, each [G][m][D]; then the two MMA-ordered copies
-    bool has_mma_pool = false;
+    bool has_mma_pool = false;    // the warp-level tensor-core family can run
+    bool mma_copies = false;      // ... and the pool allocation holds its two extra copies
     bool has_umma = false;
     int* d_err = nullptr;  // OR of error codes from kernels whose bounded waits ran out
     size_t pool_half = 0;  // bytes of one of them
@@ -236,7 +237,7 @@ int64_t auto_split_len(const ckv_ctx* ctx, int64_t total_positions, int family, 
         return std::min<int64_t>(std::max<int64_t>(c, 1024), 16384);
     }
     if (family == 2) {
-        const int qpw = mma_queries_per_warp(max_M);
+        const int qpw = mma_queries_per_warp(ctx->cfg.head_dim, max_M);
         c = total_positions * ctx->cfg.n_groups * ((max_M + qpw - 1) / qpw) / (ctx->n_sms * 32);
         c = (c + 63) / 64 * 64;
         return std::min<int64_t>(std::max<int64_t>(c, 256), 4096);
@@ -268,7 +269,8 @@ ckv_status build_plan(ckv_ctx* ctx, Plan& pl, int32_t n, const int64_t* users, c
     }
     pl.max_M = max_M;
     const bool can_mma = ctx->has_mma_pool;
-    if (ctx->opt_kernel == 0) pl.family = ctx->has_umma && max_M >= 48 ? 3 : (can_mma && max_M >= 9 ? 2 : 1);
+    const int mma_from = ctx->cfg.head_dim == 64 ? 1 : 9;  // queries per user from which the warp-level tensor-core kernel pays
+    if (ctx->opt_kernel == 0) pl.family = ctx->has_umma && max_M >= 48 ? 3 : (can_mma && max_M >= mma_from ? 2 : 1);
     else if (ctx->opt_kernel == 1) pl.family = 1;
     else if (ctx->opt_kernel == 2 && can_mma) pl.family = 2;
     else if (ctx->opt_kernel == 3 && ctx->has_umma) pl.family = 3;
@@ -460,19 +462,21 @@ ckv_status ckv_pool_load(ckv_ctx* ctx, const void* pool_K, const void* pool_V, i
     CK(sk.init(pool_K, src_bytes, s));
     CK(sv.init(pool_V, src_bytes, s));
     const bool mma = mma_supported(ctx->cfg.dtype, D, D - d_shared);
-    if (!ctx->pool || half != ctx->pool_half || mma != ctx->has_mma_pool) {
+    const bool copies = mma && mma_needs_pool_copies(D);
+    if (!ctx->pool || half != ctx->pool_half || copies != ctx->mma_copies) {
         void* np = nullptr;
-        CK(cudaMalloc(&np, (mma ? 4 : 2) * half));
+        CK(cudaMalloc(&np, (copies ? 4 : 2) * half));
         if (ctx->pool) cudaFree(ctx->pool);
         ctx->pool = np;
         ctx->pool_half = half;
-        ctx->has_mma_pool = mma;
+        ctx->mma_copies = copies;
     }
+    ctx->has_mma_pool = mma;
     ctx->has_umma = umma_supported(ctx->cfg.dtype, D, D - d_shared, n_entries <= 65536 ? 2 : 4);
     CK(launch_pool_layout(ctx->cfg.dtype, G, n_entries, d_shared, D, sk.dev, ctx->pool, s));
     CK(launch_pool_layout(ctx->cfg.dtype, G, n_entries, d_shared, D, sv.dev, (char*)ctx->pool + half, s));
-    if (mma)
-        CK(launch_pool_permute(G, n_entries, ctx->pool, (char*)ctx->pool + half, (char*)ctx->pool + 2 * half,
+    if (copies)
+        CK(launch_pool_permute(D, G, n_entries, ctx->pool, (char*)ctx->pool + half, (char*)ctx->pool + 2 * half,
                                (char*)ctx->pool + 3 * half, s));
     if (sk.owned || sv.owned) CK(cudaStreamSynchronize(s));
     if (ctx->users.empty() && (ctx->n_entries != n_entries || ctx->d_shared != d_shared)) {
@@ -636,8 +640,8 @@ ckv_status ckv_attend(ckv_ctx* ctx, int32_t n, const int64_t* users, const int32
         if (pl->family == 3)
             CK(launch_attend_umma(pl->max_M, a, ctx->n_sms, ctx->d_err, s));
         else if (pl->family == 2)
-            CK(launch_attend_mma(pl->max_M, a, (const char*)ctx->pool + 2 * ctx->pool_half,
-                                 (const char*)ctx->pool + 3 * ctx->pool_half, s));
+            CK(launch_attend_mma(D, pl->max_M, a, ctx->mma_copies ? (const char*)ctx->pool + 2 * ctx->pool_half : nullptr,
+                                 ctx->mma_copies ? (const char*)ctx->pool + 3 * ctx->pool_half : nullptr, s));
         else
             CK(launch_attend_simt(ctx->cfg.dtype, D, pl->max_M, a, s));
         ctx->st_launches++;
@@ -870,7 +874,7 @@ extern "C" ckv_status ckv_attend_static(ckv_ctx* ctx, int32_t n, const int64_t* 
         max_M = std::max(max_M, r.M);
     }
     int family;
-    if (ctx->opt_kernel == 0) family = ctx->has_mma_pool && max_M >= 9 ? 2 : 1;
+    if (ctx->opt_kernel == 0) family = ctx->has_mma_pool && max_M >= (D == 64 ? 1 : 9) ? 2 : 1;
     else if (ctx->opt_kernel == 1) family = 1;
     else if (ctx->opt_kernel == 2 && ctx->has_mma_pool) family = 2;
     else return CKV_ERR_UNSUPPORTED;
@@ -919,8 +923,8 @@ extern "C" ckv_status ckv_attend_static(ckv_ctx* ctx, int32_t n, const int64_t* 
     a.scale = ctx->scale;
     if (n_items > 0) {
         if (family == 2)
-            CK(launch_attend_mma(max_M, a, (const char*)ctx->pool + 2 * ctx->pool_half,
-                                 (const char*)ctx->pool + 3 * ctx->pool_half, s));
+            CK(launch_attend_mma(D, max_M, a, ctx->mma_copies ? (const char*)ctx->pool + 2 * ctx->pool_half : nullptr,
+                                 ctx->mma_copies ? (const char*)ctx->pool + 3 * ctx->pool_half : nullptr, s));
         else
             CK(launch_attend_simt(ctx->cfg.dtype, D, max_M, a, s));
     }

@@ -77,7 +77,7 @@ __device__ __forceinline__ void store_out(void* out, int64_t i, float v, int out
 }
 
 template <bool BF16, int D, int QB, int MODE>
-__global__ void __launch_bounds__(kWarps * 32) attend_simt_kernel(const AttendArgs a)
+__global__ void __launch_bounds__(kWarps * 32, QB == 1 ? 5 : 1) attend_simt_kernel(const AttendArgs a)
 {
     constexpr int ES = BF16 ? 2 : 4;
     constexpr int EPL = 16 / ES;         // elements per lane

@@ -67,9 +67,8 @@ struct ckv_ctx {
     int n_sms = 148;
     // pool
     int n_entries = 0, d_shared = 0, d_user = 0, idx_bytes = 0;
-    void* pool = nullptr;  // K rows then V rows, each [G][m][D]; then the two MMA-ordered copies
-    bool has_mma_pool = false;    // the warp-level tensor-core family can run
-    bool mma_copies = false;      // ... and the pool allocation holds its two extra copies
+    void* pool = nullptr;  // K rows then V rows, each [G][m][D]
+    bool has_mma = false;         // the warp-level tensor-core family can run
     bool has_umma = false;
     int* d_err = nullptr;  // OR of error codes from kernels whose bounded waits ran out
     size_t pool_half = 0;  // bytes of one of them
@@ -268,7 +267,7 @@ ckv_status build_plan(ckv_ctx* ctx, Plan& pl, int32_t n, const int64_t* users, c
         max_M = std::max(max_M, r.M);
     }
     pl.max_M = max_M;
-    const bool can_mma = ctx->has_mma_pool;
+    const bool can_mma = ctx->has_mma;
     const int mma_from = ctx->cfg.head_dim == 64 ? 1 : 9;  // queries per user from which the warp-level tensor-core kernel pays
     if (ctx->opt_kernel == 0) pl.family = ctx->has_umma && max_M >= 48 ? 3 : (can_mma && max_M >= mma_from ? 2 : 1);
     else if (ctx->opt_kernel == 1) pl.family = 1;
@@ -461,23 +460,17 @@ ckv_status ckv_pool_load(ckv_ctx* ctx, const void* pool_K, const void* pool_V, i
     Staged sk, sv;
     CK(sk.init(pool_K, src_bytes, s));
     CK(sv.init(pool_V, src_bytes, s));
-    const bool mma = mma_supported(ctx->cfg.dtype, D, D - d_shared);
-    const bool copies = mma && mma_needs_pool_copies(D);
-    if (!ctx->pool || half != ctx->pool_half || copies != ctx->mma_copies) {
+    if (!ctx->pool || half != ctx->pool_half) {
         void* np = nullptr;
-        CK(cudaMalloc(&np, (copies ? 4 : 2) * half));
+        CK(cudaMalloc(&np, 2 * half));
         if (ctx->pool) cudaFree(ctx->pool);
         ctx->pool = np;
         ctx->pool_half = half;
-        ctx->mma_copies = copies;
     }
-    ctx->has_mma_pool = mma;
+    ctx->has_mma = mma_supported(ctx->cfg.dtype, D, D - d_shared);
     ctx->has_umma = umma_supported(ctx->cfg.dtype, D, D - d_shared, n_entries <= 65536 ? 2 : 4);
     CK(launch_pool_layout(ctx->cfg.dtype, G, n_entries, d_shared, D, sk.dev, ctx->pool, s));
     CK(launch_pool_layout(ctx->cfg.dtype, G, n_entries, d_shared, D, sv.dev, (char*)ctx->pool + half, s));
-    if (copies)
-        CK(launch_pool_permute(D, G, n_entries, ctx->pool, (char*)ctx->pool + half, (char*)ctx->pool + 2 * half,
-                               (char*)ctx->pool + 3 * half, s));
     if (sk.owned || sv.owned) CK(cudaStreamSynchronize(s));
     if (ctx->users.empty() && (ctx->n_entries != n_entries || ctx->d_shared != d_shared)) {
         // index width or user width may change: restart the (empty) arena
@@ -640,8 +633,7 @@ ckv_status ckv_attend(ckv_ctx* ctx, int32_t n, const int64_t* users, const int32
         if (pl->family == 3)
             CK(launch_attend_umma(pl->max_M, a, ctx->n_sms, ctx->d_err, s));
         else if (pl->family == 2)
-            CK(launch_attend_mma(D, pl->max_M, a, ctx->mma_copies ? (const char*)ctx->pool + 2 * ctx->pool_half : nullptr,
-                                 ctx->mma_copies ? (const char*)ctx->pool + 3 * ctx->pool_half : nullptr, s));
+            CK(launch_attend_mma(D, pl->max_M, a, s));
         else
             CK(launch_attend_simt(ctx->cfg.dtype, D, pl->max_M, a, s));
         ctx->st_launches++;
@@ -874,9 +866,9 @@ extern "C" ckv_status ckv_attend_static(ckv_ctx* ctx, int32_t n, const int64_t* 
         max_M = std::max(max_M, r.M);
     }
     int family;
-    if (ctx->opt_kernel == 0) family = ctx->has_mma_pool && max_M >= (D == 64 ? 1 : 9) ? 2 : 1;
+    if (ctx->opt_kernel == 0) family = ctx->has_mma && max_M >= (D == 64 ? 1 : 9) ? 2 : 1;
     else if (ctx->opt_kernel == 1) family = 1;
-    else if (ctx->opt_kernel == 2 && ctx->has_mma_pool) family = 2;
+    else if (ctx->opt_kernel == 2 && ctx->has_mma) family = 2;
     else return CKV_ERR_UNSUPPORTED;
     const int64_t C = ctx->opt_split > 0 ? ctx->opt_split : auto_split_len(ctx, total_pos, family, max_M);
     const int64_t row_floats = (int64_t)G * (D + 2);
@@ -923,8 +915,7 @@ extern "C" ckv_status ckv_attend_static(ckv_ctx* ctx, int32_t n, const int64_t* 
     a.scale = ctx->scale;
     if (n_items > 0) {
         if (family == 2)
-            CK(launch_attend_mma(D, max_M, a, ctx->mma_copies ? (const char*)ctx->pool + 2 * ctx->pool_half : nullptr,
-                                 ctx->mma_copies ? (const char*)ctx->pool + 3 * ctx->pool_half : nullptr, s));
+            CK(launch_attend_mma(D, max_M, a, s));
         else
             CK(launch_attend_simt(ctx->cfg.dtype, D, max_M, a, s));
     }

@@ -88,13 +88,7 @@ cudaError_t launch_combine(int D, const AttendArgs& a, const int32_t* split_reqs
 // ---- kernels_mma.cu : warp-level tensor-core family (bf16, head_dim 32 or 64, d_user <= 8)
 bool mma_supported(int dtype, int head_dim, int d_user);
 int mma_queries_per_warp(int head_dim, int max_M);
-// Whether the family reads the two extra pool copies (row-internal element order of the MMA B fragments)
-// that launch_pool_permute builds; if not, launch_attend_mma ignores poolKp / poolVp.
-bool mma_needs_pool_copies(int head_dim);
-cudaError_t launch_pool_permute(int head_dim, int G, int m, const void* poolK, const void* poolV, void* poolKp, void* poolVp,
-                                cudaStream_t s);
-cudaError_t launch_attend_mma(int head_dim, int max_M, const AttendArgs& a, const void* poolKp, const void* poolVp,
-                              cudaStream_t s);
+cudaError_t launch_attend_mma(int head_dim, int max_M, const AttendArgs& a, cudaStream_t s);
 
 // ---- kernels_umma.cu : tcgen05 family (bf16, head_dim 32, d_user in {0, 1, 2, 4, 8}, 16-bit stored indices)
 bool umma_supported(int dtype, int head_dim, int d_user, int idx_bytes);

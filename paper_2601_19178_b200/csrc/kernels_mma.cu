@@ -1,22 +1,14 @@
-// Warp-level tensor-core gather-concat-attention kernels (bf16) for a moderate number of queries
-// per user.  One warp owns (work item, group, block of 16*MT queries) and walks the history chunk
-// 32 positions at a time with m16n8k16 MMAs: S = Q K^T, weights in registers, O += P V.
+// Warp-level tensor-core gather-concat-attention kernel (bf16, head_dim 32 or 64) for a moderate
+// number of queries per user (head_dim 64: also for a single query).
 //
-// head_dim 32 (attend_mma_kernel): K and V rows never pass through shared memory.  The pool is
-// kept in two extra copies whose element order inside a row matches the B-operand register
-// layout, so that
-//   - for S = Q K^T a lane reads 16 contiguous bytes of "its" K row and has both k-steps'
-//     B fragments,
-//   - for O += P V a lane reads 8 contiguous bytes of four V rows and builds the B
-//     fragments with byte permutes.
-// Which history position sits in which MMA slot is free (attention does not depend on the
-// order of positions): slot (n-tile nt, column n) of a 32-block holds position 4n + nt, which
-// makes a lane's four K positions (4g..4g+3) and eight V positions (8t..8t+7) contiguous in
-// the compressed cache -- one 8-byte and one 16-byte index load per 32 positions.
-// The user-specific leading elements (Eq. K) are patched into the owning register.
-//
-// head_dim 64 (attend_mma_staged_kernel, also for a single query per user): rows are staged in
-// a per-warp shared-memory ring by asynchronous copies and read with ldmatrix; see there.
+// One warp owns (work item, group, block of 16*MT queries) and walks the history chunk 32
+// positions at a time with m16n8k16 MMAs: S = Q K^T, weights in registers, O += P V.
+// K and V rows go from the pool into a per-warp ring of shared-memory tiles with 16-byte
+// asynchronous copies, NST tiles deep, and reach the MMA register layouts through ldmatrix
+// (transposing for V).  A whole row is fetched by adjacent lanes, so the L1 sees one line per
+// row, and the copies in flight cost no registers: a warp keeps NST - 1 tiles outstanding
+// while it computes.  The user-specific leading elements (Eq. K) are written over the head
+// of each staged row.  Positions keep their order: tile row r is position p0 + r.
 #include <cuda_bf16.h>
 #include <math_constants.h>
 
@@ -56,347 +48,6 @@ __device__ __forceinline__ float tanh_fast(float x)
     asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-
-template <bool IDX16, int N>
-__device__ __forceinline__ void load_indices(const void* base, int64_t unit, int (&out)[N])
-{
-    if constexpr (IDX16) {
-        if constexpr (N == 4) {
-            const uint2 r = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const uint16_t*>(base) + unit));
-            out[0] = r.x & 0xffff; out[1] = r.x >> 16; out[2] = r.y & 0xffff; out[3] = r.y >> 16;
-        } else {
-            const uint4 r = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const uint16_t*>(base) + unit));
-            out[0] = r.x & 0xffff; out[1] = r.x >> 16; out[2] = r.y & 0xffff; out[3] = r.y >> 16;
-            out[4] = r.z & 0xffff; out[5] = r.z >> 16; out[6] = r.w & 0xffff; out[7] = r.w >> 16;
-        }
-    } else {
-        const int4* p = reinterpret_cast<const int4*>(reinterpret_cast<const int32_t*>(base) + unit);
-#pragma unroll
-        for (int i = 0; i < N / 4; ++i) {
-            const int4 r = __ldg(p + i);
-            out[4 * i] = r.x; out[4 * i + 1] = r.y; out[4 * i + 2] = r.z; out[4 * i + 3] = r.w;
-        }
-    }
-}
-
-template <int D, int MT, int MODE, bool IDX16>
-__global__ void __launch_bounds__(128, MT == 1 ? (D == 32 ? 5 : 3) : 1) attend_mma_kernel(const AttendArgs a, const void* poolKp,
-                                                                                        const void* poolVp, int n_mb)
-{
-    constexpr int NTD = D / 8;   // n-tiles of the output
-    constexpr int KS = D / 16;   // k-steps of Q K^T
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int g = lane >> 2, t = lane & 3;
-    const int64_t wid = (int64_t)blockIdx.x * 4 + warp;
-    if (wid >= (int64_t)a.n_items * n_mb) return;
-    const Item it = a.items[wid / n_mb];
-    const int mb = (int)(wid % n_mb);
-    const Req rq = a.reqs[it.req];
-    const int row0 = mb * 16 * MT;
-    if (row0 >= rq.M) return;
-    const int grp = blockIdx.y, G = a.cv.n_groups, d_user = a.cv.d_user;
-
-    // Q as A fragments (row-major m16 x k16): rows g and g+8, columns 2t.. and 2t+8..
-    uint32_t qa[MT][KS][4];
-    const uint16_t* Q = reinterpret_cast<const uint16_t*>(a.queries);
-#pragma unroll
-    for (int mt = 0; mt < MT; ++mt) {
-        const int r_lo = row0 + 16 * mt + g, r_hi = r_lo + 8;
-        const uint16_t* q_lo = Q + ((int64_t)(rq.q0 + r_lo) * G + grp) * D;
-        const uint16_t* q_hi = Q + ((int64_t)(rq.q0 + r_hi) * G + grp) * D;
-#pragma unroll
-        for (int ks = 0; ks < KS; ++ks) {
-            const int c = 16 * ks + 2 * t;
-            qa[mt][ks][0] = r_lo < rq.M ? __ldg(reinterpret_cast<const uint32_t*>(q_lo + c)) : 0u;
-            qa[mt][ks][1] = r_hi < rq.M ? __ldg(reinterpret_cast<const uint32_t*>(q_hi + c)) : 0u;
-            qa[mt][ks][2] = r_lo < rq.M ? __ldg(reinterpret_cast<const uint32_t*>(q_lo + c + 8)) : 0u;
-            qa[mt][ks][3] = r_hi < rq.M ? __ldg(reinterpret_cast<const uint32_t*>(q_hi + c + 8)) : 0u;
-        }
-    }
-
-    float o[MT][NTD][4];
-    float m_run[MT][2], l_run[MT][2];
-#pragma unroll
-    for (int mt = 0; mt < MT; ++mt) {
-        m_run[mt][0] = m_run[mt][1] = -CUDART_INF_F;
-        l_run[mt][0] = l_run[mt][1] = 0.f;
-#pragma unroll
-        for (int j = 0; j < NTD; ++j)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) o[mt][j][e] = 0.f;
-    }
-
-    const char* pK = reinterpret_cast<const char*>(poolKp) + (int64_t)grp * a.cv.n_entries * (D * 2) + t * (D / 2);
-    const char* pV = reinterpret_cast<const char*>(poolVp) + (int64_t)grp * a.cv.n_entries * (D * 2) + g * (NTD * 2);
-    const int64_t unit0 = rq.base + (int64_t)grp * rq.Lpad;
-    const uint16_t* uK = reinterpret_cast<const uint16_t*>(a.cv.userK);
-    const uint16_t* uV = reinterpret_cast<const uint16_t*>(a.cv.userV);
-    const int end = it.begin + it.len;
-    const float sc = a.scale * (MODE == CKV_SOFTMAX ? kLog2e : 0.5f);
-    const bool patchK0 = 2 * t < d_user, patchK1 = 2 * t + 1 < d_user, patchV = g < d_user;
-
-    for (int p0 = it.begin; p0 < end; p0 += 32) {
-        int ik[4], iv[8];
-        const int64_t unitK = unit0 + p0 + 4 * g;   // this lane's four K positions
-        const int64_t unitV = unit0 + p0 + 8 * t;   // this lane's eight V positions
-        // (the user parts are requested first: they come from HBM like the indices, and a warp
-        // issues in order, so behind the gathers they would only start once the indices are back)
-        uint4 uk4[2], uv4[4];
-        if (d_user == 1) {
-            if (t == 0) {
-                const uint2 r = __ldg(reinterpret_cast<const uint2*>(uK + unitK));
-                uk4[0].x = r.x;
-                uk4[0].y = r.y;
-            }
-            if (g == 0) uv4[0] = __ldg(reinterpret_cast<const uint4*>(uV + unitV));
-        } else if (d_user == 2) {
-            if (t == 0) uk4[0] = __ldg(reinterpret_cast<const uint4*>(uK + unitK * 2));
-            if (g < 2) {
-                uv4[0] = __ldg(reinterpret_cast<const uint4*>(uV + unitV * 2));
-                uv4[1] = __ldg(reinterpret_cast<const uint4*>(uV + unitV * 2) + 1);
-            }
-        } else if (d_user == 4) {
-            if (t < 2) {
-                uk4[0] = __ldg(reinterpret_cast<const uint4*>(uK + unitK * 4));
-                uk4[1] = __ldg(reinterpret_cast<const uint4*>(uK + unitK * 4) + 1);
-            }
-            if (g < 4) {
-#pragma unroll
-                for (int jj = 0; jj < 4; ++jj) uv4[jj] = __ldg(reinterpret_cast<const uint4*>(uV + unitV * 4) + jj);
-            }
-        }
-        load_indices<IDX16, 4>(a.cv.idxK, unitK, ik);
-        load_indices<IDX16, 8>(a.cv.idxV, unitV, iv);
-        uint32_t kf[4][2 * KS];  // K rows: per k-step the two B-fragment registers of this lane
-        uint32_t vr[8][NTD / 2];  // V rows: element g of every n-tile, two per register
-#pragma unroll
-        for (int nt = 0; nt < 4; ++nt) {
-            const uint4* src = reinterpret_cast<const uint4*>(pK + (int64_t)ik[nt] * (D * 2));
-#pragma unroll
-            for (int h = 0; h < KS / 2; ++h) {
-                const uint4 r = __ldg(src + h);
-                kf[nt][4 * h] = r.x;
-                kf[nt][4 * h + 1] = r.y;
-                kf[nt][4 * h + 2] = r.z;
-                kf[nt][4 * h + 3] = r.w;
-            }
-        }
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            if constexpr (D == 32) {
-                const uint2 r = __ldg(reinterpret_cast<const uint2*>(pV + (int64_t)iv[j] * (D * 2)));
-                vr[j][0] = r.x;
-                vr[j][1] = r.y;
-            } else {
-                const uint4 r = __ldg(reinterpret_cast<const uint4*>(pV + (int64_t)iv[j] * (D * 2)));
-                vr[j][0] = r.x;
-                vr[j][1] = r.y;
-                vr[j][2] = r.z;
-                vr[j][3] = r.w;
-            }
-        }
-        // Eq. K: dims [0, d_user) come from the user-specific part.  The user parts of this lane's four K
-        // positions (and of its eight V positions) are contiguous in the cache: for the common widths
-        // they are fetched with one or two wide loads instead of one 2-byte load per element.
-        if (d_user == 1) {
-            if (t == 0) {
-                const uint2 r = make_uint2(uk4[0].x, uk4[0].y);
-                kf[0][0] = (kf[0][0] & 0xffff0000u) | (r.x & 0xffffu);
-                kf[1][0] = (kf[1][0] & 0xffff0000u) | (r.x >> 16);
-                kf[2][0] = (kf[2][0] & 0xffff0000u) | (r.y & 0xffffu);
-                kf[3][0] = (kf[3][0] & 0xffff0000u) | (r.y >> 16);
-            }
-            if (g == 0) {
-                const uint4 r = uv4[0];
-                const uint32_t w[4] = {r.x, r.y, r.z, r.w};
-#pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    vr[j][0] = (vr[j][0] & 0xffff0000u) | ((j & 1) ? w[j >> 1] >> 16 : w[j >> 1] & 0xffffu);
-            }
-        } else if (d_user == 2) {
-            if (t == 0) {
-                const uint4 r = uk4[0];
-                kf[0][0] = r.x;
-                kf[1][0] = r.y;
-                kf[2][0] = r.z;
-                kf[3][0] = r.w;
-            }
-            if (g < 2) {
-                const uint4 r0 = uv4[0], r1 = uv4[1];
-                const uint32_t w[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
-#pragma unroll
-                for (int j = 0; j < 8; ++j) vr[j][0] = (vr[j][0] & 0xffff0000u) | (g ? w[j] >> 16 : w[j] & 0xffffu);
-            }
-        } else if (d_user == 4) {
-            if (t < 2) {
-                const uint4 r0 = uk4[0], r1 = uk4[1];
-                kf[0][0] = t ? r0.y : r0.x;
-                kf[1][0] = t ? r0.w : r0.z;
-                kf[2][0] = t ? r1.y : r1.x;
-                kf[3][0] = t ? r1.w : r1.z;
-            }
-            if (g < 4) {
-#pragma unroll
-                for (int jj = 0; jj < 4; ++jj) {  // positions 2 jj and 2 jj + 1
-                    const uint4 r = uv4[jj];
-                    const uint32_t a0 = (g & 2) ? r.y : r.x, a1 = (g & 2) ? r.w : r.z;
-                    vr[2 * jj][0] = (vr[2 * jj][0] & 0xffff0000u) | ((g & 1) ? a0 >> 16 : a0 & 0xffffu);
-                    vr[2 * jj + 1][0] = (vr[2 * jj + 1][0] & 0xffff0000u) | ((g & 1) ? a1 >> 16 : a1 & 0xffffu);
-                }
-            }
-        } else {
-            if (patchK0) {
-#pragma unroll
-                for (int nt = 0; nt < 4; ++nt) {
-                    const uint16_t* u = uK + (unitK + nt) * d_user + 2 * t;
-                    uint32_t w = __ldg(u);
-                    w |= patchK1 ? (uint32_t)__ldg(u + 1) << 16 : (kf[nt][0] & 0xffff0000u);
-                    kf[nt][0] = w;
-                }
-            }
-            if (patchV) {
-#pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    vr[j][0] = (vr[j][0] & 0xffff0000u) | (uint32_t)__ldg(uV + (unitV + j) * d_user + g);
-            }
-        }
-        // V B-fragments: k-slots (2t, 2t+1, 2t+8, 2t+9) of block b are positions
-        // 8t + (2b, 4+2b, 2b+1, 5+2b)
-        uint32_t vb[2][NTD][2];
-#pragma unroll
-        for (int b = 0; b < 2; ++b)
-#pragma unroll
-            for (int j = 0; j < NTD; ++j) {
-                const uint32_t sel = (j & 1) ? 0x7632 : 0x5410;
-                vb[b][j][0] = __byte_perm(vr[2 * b][j >> 1], vr[4 + 2 * b][j >> 1], sel);
-                vb[b][j][1] = __byte_perm(vr[2 * b + 1][j >> 1], vr[5 + 2 * b][j >> 1], sel);
-            }
-        const bool tail = p0 + 32 > end;
-
-#pragma unroll
-        for (int mt = 0; mt < MT; ++mt) {
-            float s[4][4];
-#pragma unroll
-            for (int nt = 0; nt < 4; ++nt) {
-                s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
-#pragma unroll
-                for (int ks = 0; ks < KS; ++ks) mma_bf16(s[nt], qa[mt][ks], kf[nt][2 * ks], kf[nt][2 * ks + 1]);
-            }
-            // element (nt, e): column 2t + (e & 1) -> position p0 + 8t + 4 (e & 1) + nt
-            uint32_t pa[2][4];
-            if constexpr (MODE == CKV_SOFTMAX) {
-                if (tail) {
-#pragma unroll
-                    for (int nt = 0; nt < 4; ++nt) {
-                        if (p0 + 8 * t + nt >= end) s[nt][0] = s[nt][2] = -CUDART_INF_F;
-                        if (p0 + 8 * t + 4 + nt >= end) s[nt][1] = s[nt][3] = -CUDART_INF_F;
-                    }
-                }
-                float mx0 = s[0][0], mx1 = s[0][2];
-#pragma unroll
-                for (int nt = 0; nt < 4; ++nt) {
-                    mx0 = fmaxf(mx0, fmaxf(s[nt][0], s[nt][1]));
-                    mx1 = fmaxf(mx1, fmaxf(s[nt][2], s[nt][3]));
-                }
-                mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
-                mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
-                mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
-                mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
-                // the first position of a block is always valid, so mx is finite
-                const float mn0 = fmaxf(m_run[mt][0], mx0 * sc), mn1 = fmaxf(m_run[mt][1], mx1 * sc);
-                const float c0 = ex2(m_run[mt][0] - mn0), c1 = ex2(m_run[mt][1] - mn1);
-                m_run[mt][0] = mn0;
-                m_run[mt][1] = mn1;
-                float ps0 = 0.f, ps1 = 0.f;
-#pragma unroll
-                for (int nt = 0; nt < 4; ++nt) {
-                    const float p0v = ex2(fmaf(s[nt][0], sc, -mn0)), p1v = ex2(fmaf(s[nt][1], sc, -mn0));
-                    const float p2v = ex2(fmaf(s[nt][2], sc, -mn1)), p3v = ex2(fmaf(s[nt][3], sc, -mn1));
-                    ps0 += p0v + p1v;
-                    ps1 += p2v + p3v;
-                    pa[nt >> 1][(nt & 1) * 2] = pack_bf16(p0v, p1v);
-                    pa[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(p2v, p3v);
-                }
-                l_run[mt][0] = l_run[mt][0] * c0 + ps0;
-                l_run[mt][1] = l_run[mt][1] * c1 + ps1;
-#pragma unroll
-                for (int j = 0; j < NTD; ++j) {
-                    o[mt][j][0] *= c0; o[mt][j][1] *= c0;
-                    o[mt][j][2] *= c1; o[mt][j][3] *= c1;
-                }
-            } else {
-                // silu(x) = x sigmoid(x) = h (1 + tanh(h)), h = x / 2   (sc = scale / 2)
-#pragma unroll
-                for (int nt = 0; nt < 4; ++nt) {
-                    float w[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const float h = s[nt][e] * sc;
-                        w[e] = fmaf(h, tanh_fast(h), h);
-                    }
-                    if (tail) {
-                        if (p0 + 8 * t + nt >= end) w[0] = w[2] = 0.f;
-                        if (p0 + 8 * t + 4 + nt >= end) w[1] = w[3] = 0.f;
-                    }
-                    pa[nt >> 1][(nt & 1) * 2] = pack_bf16(w[0], w[1]);
-                    pa[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(w[2], w[3]);
-                }
-            }
-#pragma unroll
-            for (int b = 0; b < 2; ++b)
-#pragma unroll
-                for (int j = 0; j < NTD; ++j) mma_bf16(o[mt][j], pa[b], vb[b][j][0], vb[b][j][1]);
-        }
-    }
-
-    // epilogue: finish the row sums over the quad, then store outputs or partials
-#pragma unroll
-    for (int mt = 0; mt < MT; ++mt) {
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            float l = l_run[mt][h];
-            l += __shfl_xor_sync(0xffffffffu, l, 1);
-            l += __shfl_xor_sync(0xffffffffu, l, 2);
-            const int r = row0 + 16 * mt + g + 8 * h;
-            if (r >= rq.M) continue;
-            if (it.part_row < 0) {
-                float inv;
-                if constexpr (MODE == CKV_SOFTMAX) inv = l > 0.f ? 1.0f / l : 0.f;
-                else inv = rq.L > 0 ? 1.0f / (float)rq.L : 0.f;
-                const int64_t base = ((int64_t)(rq.q0 + r) * G + grp) * D;
-#pragma unroll
-                for (int j = 0; j < NTD; ++j) {
-                    const float x = o[mt][j][2 * h] * inv, y = o[mt][j][2 * h + 1] * inv;
-                    if (a.out_dtype == CKV_BF16)
-                        *reinterpret_cast<uint32_t*>(reinterpret_cast<uint16_t*>(a.out) + base + 8 * j + 2 * t) =
-                            pack_bf16(x, y);
-                    else
-                        *reinterpret_cast<float2*>(reinterpret_cast<float*>(a.out) + base + 8 * j + 2 * t) =
-                            make_float2(x, y);
-                }
-            } else {
-                float* pr = a.partials + ((int64_t)(it.part_row + r) * G + grp) * (D + 2);
-                if (t == 0) {
-                    pr[0] = m_run[mt][h];
-                    pr[1] = l;
-                }
-#pragma unroll
-                for (int j = 0; j < NTD; ++j)
-                    *reinterpret_cast<float2*>(pr + 2 + 8 * j + 2 * t) =
-                        make_float2(o[mt][j][2 * h], o[mt][j][2 * h + 1]);
-            }
-        }
-    }
-}
-
-// ---------------------------------------------------------------------------------------------
-// Staged variant: K and V rows go from the pool (in its plain layout) into a per-warp ring of
-// shared-memory tiles with 16-byte asynchronous copies, NST tiles deep, and reach the MMA
-// register layouts through ldmatrix.  A whole row is fetched by adjacent lanes, so the L1 sees
-// one line per row instead of one per (row, lane group), and the copies in flight cost no
-// registers: a warp keeps NST - 1 tiles (of 32 positions) outstanding while it computes.
-// The user-specific leading elements (Eq. K) are written over the head of each staged row.
-// Positions keep their order: tile row r is position p0 + r.
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -466,12 +117,12 @@ __device__ __forceinline__ void store_user_part(uint32_t addr, const uint4& r, i
 }
 
 template <int D, int MT>
-struct StagedCfg {
+struct MmaCfg {
     static constexpr int ROWB = D * 2;            // bytes per row
     static constexpr int CPR = ROWB / 16;         // 16-byte chunks per row
     static constexpr int RPI = 32 / CPR;          // rows one warp-wide copy instruction covers
     static constexpr int TILE_B = 32 * ROWB;      // one K or V tile of 32 positions
-    static constexpr int NST = D == 64 ? 3 : 4;   // ring depth
+    static constexpr int NST = D == 64 ? 3 : 2;   // ring depth (64-byte rows: more resident warps beat a deeper ring)
     static constexpr int WARPS = 4;
     static constexpr int SMEM = WARPS * NST * 2 * TILE_B;
     static constexpr int MIN_BLOCKS = MT == 1 ? (D == 64 ? 2 : 4) : 1;
@@ -486,10 +137,10 @@ __device__ __forceinline__ int swz(int r)
 }
 
 template <int D, int MT, int MODE, bool IDX16>
-__global__ void __launch_bounds__(128, StagedCfg<D, MT>::MIN_BLOCKS)
-    attend_mma_staged_kernel(const AttendArgs a, int n_mb)
+__global__ void __launch_bounds__(128, MmaCfg<D, MT>::MIN_BLOCKS)
+    attend_mma_kernel(const AttendArgs a, int n_mb)
 {
-    using C = StagedCfg<D, MT>;
+    using C = MmaCfg<D, MT>;
     constexpr int NTD = D / 8, KS = D / 16, ROWB = C::ROWB, CPR = C::CPR, RPI = C::RPI, NST = C::NST;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -776,66 +427,32 @@ __global__ void __launch_bounds__(128, StagedCfg<D, MT>::MIN_BLOCKS)
     }
 }
 
-// Row-internal element orders of the two extra pool copies (see the header comment).
-//   K copy: chunk t (head_dim / 2 bytes) holds, per k-step ks, elements 16ks + {2t, 2t+1, 2t+8, 2t+9}
-//   V copy: chunk g (head_dim / 4 bytes) holds elements g, g+8, g+16, ...
-template <int D>
-__global__ void pool_permute_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dstK,
-                                    uint16_t* __restrict__ dstV, const uint16_t* __restrict__ srcV, int64_t rows)
-{
-    constexpr int NTD = D / 8;
-    const int64_t total = rows * D;
-    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
-        const int64_t r = i / D;
-        const int c = (int)(i - r * D);
-        const int ks = c >> 4, rem = c & 15, hi = rem >> 3, tt = (rem & 7) >> 1, lo = rem & 1;
-        dstK[r * D + tt * (D / 4) + ks * 4 + hi * 2 + lo] = src[i];
-        dstV[r * D + (c & 7) * NTD + (c >> 3)] = srcV[i];
-    }
-}
-
-template <int D, int MT>
-cudaError_t launch_mt(const AttendArgs& a, const void* pKp, const void* pVp, int n_mb, cudaStream_t s)
-{
-    const int64_t warps = (int64_t)a.n_items * n_mb;
-    const dim3 grid((unsigned)((warps + 3) / 4), a.cv.n_groups);
-    const bool i16 = a.cv.idx_bytes == 2;
-    if (a.mode == CKV_SOFTMAX) {
-        if (i16) attend_mma_kernel<D, MT, CKV_SOFTMAX, true><<<grid, 128, 0, s>>>(a, pKp, pVp, n_mb);
-        else attend_mma_kernel<D, MT, CKV_SOFTMAX, false><<<grid, 128, 0, s>>>(a, pKp, pVp, n_mb);
-    } else {
-        if (i16) attend_mma_kernel<D, MT, CKV_SILU_OVER_L, true><<<grid, 128, 0, s>>>(a, pKp, pVp, n_mb);
-        else attend_mma_kernel<D, MT, CKV_SILU_OVER_L, false><<<grid, 128, 0, s>>>(a, pKp, pVp, n_mb);
-    }
-    return cudaGetLastError();
-}
-
 template <int D, int MT, int MODE, bool IDX16>
-cudaError_t launch_staged_one(const AttendArgs& a, int n_mb, dim3 grid, cudaStream_t s)
+cudaError_t launch_mma_one(const AttendArgs& a, int n_mb, dim3 grid, cudaStream_t s)
 {
-    using C = StagedCfg<D, MT>;
+    using C = MmaCfg<D, MT>;
     static bool configured = false;  // per instantiation; the attribute is idempotent
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(attend_mma_staged_kernel<D, MT, MODE, IDX16>,
+        cudaError_t e = cudaFuncSetAttribute(attend_mma_kernel<D, MT, MODE, IDX16>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    attend_mma_staged_kernel<D, MT, MODE, IDX16><<<grid, 128, C::SMEM, s>>>(a, n_mb);
+    attend_mma_kernel<D, MT, MODE, IDX16><<<grid, 128, C::SMEM, s>>>(a, n_mb);
     return cudaGetLastError();
 }
 
 template <int D, int MT>
-cudaError_t launch_staged(const AttendArgs& a, int n_mb, cudaStream_t s)
+cudaError_t launch_mma(const AttendArgs& a, int n_mb, cudaStream_t s)
 {
     const int64_t warps = (int64_t)a.n_items * n_mb;
     const dim3 grid((unsigned)((warps + 3) / 4), a.cv.n_groups);
     const bool i16 = a.cv.idx_bytes == 2;
     if (a.mode == CKV_SOFTMAX)
-        return i16 ? launch_staged_one<D, MT, CKV_SOFTMAX, true>(a, n_mb, grid, s)
-                   : launch_staged_one<D, MT, CKV_SOFTMAX, false>(a, n_mb, grid, s);
-    return i16 ? launch_staged_one<D, MT, CKV_SILU_OVER_L, true>(a, n_mb, grid, s)
-               : launch_staged_one<D, MT, CKV_SILU_OVER_L, false>(a, n_mb, grid, s);
+        return i16 ? launch_mma_one<D, MT, CKV_SOFTMAX, true>(a, n_mb, grid, s)
+                   : launch_mma_one<D, MT, CKV_SOFTMAX, false>(a, n_mb, grid, s);
+    return i16 ? launch_mma_one<D, MT, CKV_SILU_OVER_L, true>(a, n_mb, grid, s)
+               : launch_mma_one<D, MT, CKV_SILU_OVER_L, false>(a, n_mb, grid, s);
 }
 
 }  // namespace
@@ -845,37 +462,19 @@ bool mma_supported(int dtype, int head_dim, int d_user)
     return dtype == CKV_BF16 && (head_dim == 32 || head_dim == 64) && d_user <= 8;
 }
 
-bool mma_needs_pool_copies(int head_dim) { return head_dim == 32; }
-
-cudaError_t launch_pool_permute(int D, int G, int m, const void* poolK, const void* poolV, void* poolKp, void* poolVp,
-                                cudaStream_t s)
-{
-    const int64_t rows = (int64_t)G * m;
-    int grid = (int)((rows * D + 255) / 256);
-    if (grid > 148 * 16) grid = 148 * 16;
-    if (D == 32)
-        pool_permute_kernel<32><<<grid, 256, 0, s>>>((const uint16_t*)poolK, (uint16_t*)poolKp, (uint16_t*)poolVp,
-                                                     (const uint16_t*)poolV, rows);
-    else
-        pool_permute_kernel<64><<<grid, 256, 0, s>>>((const uint16_t*)poolK, (uint16_t*)poolKp, (uint16_t*)poolVp,
-                                                     (const uint16_t*)poolV, rows);
-    return cudaGetLastError();
-}
-
 // head_dim 64 rows keep a warp busy with one 16-query tile; 32-wide heads take up to four
 int mma_queries_per_warp(int D, int max_M) { return (D == 64 || max_M <= 16) ? 16 : (max_M <= 32 ? 32 : 64); }
 
-cudaError_t launch_attend_mma(int D, int max_M, const AttendArgs& a, const void* poolKp, const void* poolVp,
-                              cudaStream_t s)
+cudaError_t launch_attend_mma(int D, int max_M, const AttendArgs& a, cudaStream_t s)
 {
     if (a.n_items == 0) return cudaSuccess;
     const int qpw = mma_queries_per_warp(D, max_M);
     const int n_mb = (max_M + qpw - 1) / qpw;
-    if (D == 64) return launch_staged<64, 1>(a, n_mb, s);
+    if (D == 64) return launch_mma<64, 1>(a, n_mb, s);
     switch (qpw) {
-        case 16: return launch_mt<32, 1>(a, poolKp, poolVp, n_mb, s);
-        case 32: return launch_mt<32, 2>(a, poolKp, poolVp, n_mb, s);
-        default: return launch_mt<32, 4>(a, poolKp, poolVp, n_mb, s);
+        case 16: return launch_mma<32, 1>(a, n_mb, s);
+        case 32: return launch_mma<32, 2>(a, n_mb, s);
+        default: return launch_mma<32, 4>(a, n_mb, s);
     }
 }
 

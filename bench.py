@@ -51,9 +51,11 @@ def _peaks():
 # from the ncu captures summarised under profiles/ (attend_*_kernel_<workload>.md).  cfg3 and cfg5
 # were captured on a cut of the workload and scaled by the number of users.  Set an entry to None
 # when its kernel changes after the capture.
-TRAFFIC_BYTES = {"cfg2": 190658560, "cfg3": 1090254848, "cfg4": 372389376, "cfg5": 1857857536}
+TRAFFIC_BYTES = {"cfg2": 190658560, "cfg3": 1090254848, "cfg4": 372015872, "cfg5": 1854877696}
 # transcendental evaluations per SM per clock (ex2 / tanh issue rate of the special-function unit)
 XU_PER_SM_CLK = 16
+# bytes per SM per clock through the L1 / shared-memory data pipe (one 128-byte wavefront per clock)
+L1_PIPE_BYTES_PER_SM_CLK = 128
 
 
 def _traffic(workload: str, full_size: bool):
@@ -316,10 +318,22 @@ def run_ours(args, w):
         rate, dt, cores, n_u, pos = _oracle_rate(w, data, CPU_SAMPLE_USERS.get(w.name, w.n_users))
         cpu = {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle",
                "sample": f"first {n_u} of {w.n_users} users ({pos} positions), {dt:.1f} s"}
-    # One exp (softmax) or tanh (SiLU) per score: with many queries per user the special-function
-    # unit, not HBM, is the roof that binds.  Reported beside the HBM roofline the metric asks for.
+    # The roof that binds, reported beside the HBM roofline the metric asks for.
+    # Many queries per user (tcgen05 kernel): one exp (softmax) or tanh (SiLU) per score on the
+    # special-function unit.  Few queries (warp-level tensor-core kernel): every gathered pool row crosses
+    # the SM's L1 / shared-memory data pipe twice, once copied into the staging ring and once read
+    # out by ldmatrix; the pool rows come from L2, not HBM.
     binding = None
-    if w.n_queries >= 9 and clocks and clocks.get("sm_max_mhz"):
+    family = s.stat("kernel")
+    if family == 2 and clocks and clocks.get("sm_max_mhz"):
+        n_sms = torch.cuda.get_device_properties(local).multi_processor_count
+        pipe_bytes = float(positions) * w.n_groups * 2 * (w.head_dim * 2) * 2
+        peak_pipe = L1_PIPE_BYTES_PER_SM_CLK * n_sms * clocks["sm_max_mhz"] * 1e6 / 1e9
+        binding = {"bound": "l1_shared_data_pipe",
+                   "what": "K and V pool rows into the shared-memory ring and out through ldmatrix",
+                   "achieved": pipe_bytes / kern_s / 1e9, "peak": peak_pipe, "unit": "GB/s",
+                   "frac": pipe_bytes / kern_s / 1e9 / peak_pipe}
+    elif w.n_queries >= 9 and clocks and clocks.get("sm_max_mhz"):
         scores = float(positions) * w.n_groups * w.n_queries
         n_sms = torch.cuda.get_device_properties(local).multi_processor_count
         peak_xu = XU_PER_SM_CLK * n_sms * clocks["sm_max_mhz"] * 1e6 / 1e9

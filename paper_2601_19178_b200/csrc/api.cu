@@ -268,8 +268,9 @@ ckv_status build_plan(ckv_ctx* ctx, Plan& pl, int32_t n, const int64_t* users, c
     }
     pl.max_M = max_M;
     const bool can_mma = ctx->has_mma;
-    const int mma_from = ctx->cfg.head_dim == 64 ? 1 : 9;  // queries per user from which the warp-level tensor-core kernel pays
-    if (ctx->opt_kernel == 0) pl.family = ctx->has_umma && max_M >= 48 ? 3 : (can_mma && max_M >= mma_from ? 2 : 1);
+    // tcgen05 from three 16-query blocks on, else the warp-level tensor-core kernel (faster than the CUDA-core
+    // kernel from a single query on); the CUDA-core kernel serves what neither supports
+    if (ctx->opt_kernel == 0) pl.family = ctx->has_umma && max_M >= 48 ? 3 : (can_mma ? 2 : 1);
     else if (ctx->opt_kernel == 1) pl.family = 1;
     else if (ctx->opt_kernel == 2 && can_mma) pl.family = 2;
     else if (ctx->opt_kernel == 3 && ctx->has_umma) pl.family = 3;
@@ -866,7 +867,7 @@ extern "C" ckv_status ckv_attend_static(ckv_ctx* ctx, int32_t n, const int64_t* 
         max_M = std::max(max_M, r.M);
     }
     int family;
-    if (ctx->opt_kernel == 0) family = ctx->has_mma && max_M >= (D == 64 ? 1 : 9) ? 2 : 1;
+    if (ctx->opt_kernel == 0) family = ctx->has_mma ? 2 : 1;
     else if (ctx->opt_kernel == 1) family = 1;
     else if (ctx->opt_kernel == 2 && ctx->has_mma) family = 2;
     else return CKV_ERR_UNSUPPORTED;

@@ -186,6 +186,34 @@ CKV_API ckv_status ckv_attend_static(ckv_ctx* ctx, int32_t n, const int64_t* use
  */
 CKV_API ckv_status ckv_materialize(ckv_ctx* ctx, int64_t user, void* K_out, void* V_out, void* stream);
 
+/*
+ * Decode-stage load path (Sec. 4.4: T_load(s d_u + s) + T_index): a serving system keeps the
+ * compressed caches in host memory and loads the users of a request batch before attending.
+ * A blob is the packed form of n users' caches exactly as the library stores them, so loading it
+ * is four plain copies and no packing kernel.  Layout, for the users in the order given, with
+ * units(u) = n_groups * round_up(L_u, 32):
+ *     [ K indices of all users | V indices | user-specific K | user-specific V ]
+ * each section holding units(u) entries per user back to back, an entry being [group][position]
+ * within a user (2- or 4-byte indices as stored, d_user elements for the user parts; padding
+ * positions hold index 0 and zeros), each section starting at a multiple of 256 bytes.  A blob is only meaningful for a context with the same n_groups, head_dim, dtype and
+ * pool shape (n_entries, d_shared) as the one that exported it.
+ *
+ * ckv_cache_blob_bytes: size of the blob for histories of lengths L[0..n) (host array).
+ * ckv_cache_export: writes the blob of n cached users to `blob` (host or device memory, `bytes`
+ *   must equal ckv_cache_blob_bytes of their lengths); stream-ordered, synchronise before reading.
+ * ckv_cache_import: stores n users from `blob` (host -- pinned for an asynchronous copy -- or
+ *   device memory) under the given ids, replacing users that exist.  The stored indices are
+ *   range-checked on the device; the call returns after that check (it synchronises `stream`).
+ * Errors: INVALID_ARG (null pointers, n < 0, negative length, wrong `bytes`), STATE (no pool),
+ *   UNKNOWN_USER (export), INDEX_RANGE (import: an index >= n_entries; nothing is stored),
+ *   OOM, CUDA.
+ */
+CKV_API ckv_status ckv_cache_blob_bytes(ckv_ctx* ctx, int32_t n, const int32_t* L, int64_t* bytes);
+CKV_API ckv_status ckv_cache_export(ckv_ctx* ctx, int32_t n, const int64_t* users, void* blob, int64_t bytes,
+                                    void* stream);
+CKV_API ckv_status ckv_cache_import(ckv_ctx* ctx, int32_t n, const int64_t* users, const int32_t* L,
+                                    const void* blob, int64_t bytes, void* stream);
+
 /* History length of a cached user.  Errors: UNKNOWN_USER. */
 CKV_API ckv_status ckv_user_length(ckv_ctx* ctx, int64_t user, int64_t* L);
 

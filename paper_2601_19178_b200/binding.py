@@ -23,7 +23,7 @@ CKV_SOFTMAX, CKV_SILU_OVER_L = 0, 1
 EXPORTS = (
     "ckv_create", "ckv_destroy", "ckv_pool_load", "ckv_cache_put", "ckv_cache_put_batch",
     "ckv_cache_evict", "ckv_cache_clear", "ckv_attend", "ckv_attend_static", "ckv_materialize",
-    "ckv_user_length",
+    "ckv_user_length", "ckv_cache_blob_bytes", "ckv_cache_export", "ckv_cache_import",
     "ckv_cache_bytes", "ckv_set_option", "ckv_get_option", "ckv_last_stat", "ckv_strerror",
     "ckv_last_cuda_error", "ckv_version",
 )
@@ -62,6 +62,9 @@ def _load() -> ctypes.CDLL:
         "ckv_attend_static": (i32, [vp, i32, vp, vp, vp, vp, vp]),
         "ckv_materialize": (i32, [vp, i64, vp, vp, vp]),
         "ckv_user_length": (i32, [vp, i64, p64]),
+        "ckv_cache_blob_bytes": (i32, [vp, i32, vp, p64]),
+        "ckv_cache_export": (i32, [vp, i32, vp, vp, i64, vp]),
+        "ckv_cache_import": (i32, [vp, i32, vp, vp, vp, i64, vp]),
         "ckv_cache_bytes": (i32, [vp, p64, p64]),
         "ckv_set_option": (i32, [vp, cs, i64]),
         "ckv_get_option": (i32, [vp, cs, p64]),
@@ -190,6 +193,29 @@ def ckv_user_length(ctx, user: int) -> int:
     v = ctypes.c_int64()
     _check(ctx, lib.ckv_user_length(ctx, int(user), ctypes.byref(v)), "ckv_user_length")
     return v.value
+
+
+def ckv_cache_blob_bytes(ctx, L) -> int:
+    L = _host_i32(L)
+    v = ctypes.c_int64()
+    _check(ctx, lib.ckv_cache_blob_bytes(ctx, L.shape[0], L.ctypes.data, ctypes.byref(v)), "ckv_cache_blob_bytes")
+    return v.value
+
+
+def ckv_cache_export(ctx, users, blob, nbytes: int, stream=None) -> None:
+    """Writes the packed caches of `users` (host int64 [n]) to `blob` (host or device buffer of nbytes)."""
+    users = _host_i64(users)
+    _check(ctx, lib.ckv_cache_export(ctx, users.shape[0], users.ctypes.data, _ptr(blob), int(nbytes),
+                                     _stream(stream)), "ckv_cache_export")
+
+
+def ckv_cache_import(ctx, users, L, blob, nbytes: int, stream=None) -> None:
+    """Stores `users` (host int64 [n]) with history lengths L (host int32 [n]) from a packed blob."""
+    users, L = _host_i64(users), _host_i32(L)
+    if L.shape[0] != users.shape[0]:
+        raise ValueError("L must have len(users) entries")
+    _check(ctx, lib.ckv_cache_import(ctx, users.shape[0], users.ctypes.data, L.ctypes.data, _ptr(blob), int(nbytes),
+                                     _stream(stream)), "ckv_cache_import")
 
 
 def ckv_cache_bytes(ctx):

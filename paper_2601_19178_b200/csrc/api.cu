@@ -551,6 +551,117 @@ ckv_status ckv_cache_put(ckv_ctx* ctx, int64_t user, int32_t L, const int32_t* i
     return ckv_cache_put_batch(ctx, 1, &user, off, idx_K, idx_V, user_K, user_V, d_user, stream);
 }
 
+namespace {
+
+// Section offsets of a blob holding `total_units` units: K indices, V indices, user K, user V, end.
+void blob_sections(const ckv_ctx* ctx, int64_t total_units, int64_t (&off)[5])
+{
+    const int64_t ub = (int64_t)ctx->d_user * ctx->elem;
+    const int64_t sz[4] = {total_units * ctx->idx_bytes, total_units * ctx->idx_bytes, total_units * ub,
+                           total_units * ub};
+    off[0] = 0;
+    for (int i = 0; i < 4; ++i) off[i + 1] = (off[i] + sz[i] + 255) / 256 * 256;
+}
+
+int64_t units_of(const ckv_ctx* ctx, int64_t L) { return (int64_t)ctx->cfg.n_groups * ((L + 31) / 32 * 32); }
+
+}  // namespace
+
+ckv_status ckv_cache_blob_bytes(ckv_ctx* ctx, int32_t n, const int32_t* L, int64_t* bytes)
+{
+    if (!ctx || n < 0 || (n > 0 && !L) || !bytes) return CKV_ERR_INVALID_ARG;
+    if (!ctx->pool) return CKV_ERR_STATE;
+    int64_t total = 0;
+    for (int32_t k = 0; k < n; ++k) {
+        if (L[k] < 0 || L[k] > INT32_MAX - 32) return CKV_ERR_INVALID_ARG;
+        total += units_of(ctx, L[k]);
+    }
+    int64_t off[5];
+    blob_sections(ctx, total, off);
+    *bytes = off[4];
+    return CKV_OK;
+}
+
+ckv_status ckv_cache_export(ckv_ctx* ctx, int32_t n, const int64_t* users, void* blob, int64_t bytes, void* stream)
+{
+    if (!ctx || n < 0 || (n > 0 && (!users || !blob))) return CKV_ERR_INVALID_ARG;
+    if (!ctx->pool) return CKV_ERR_STATE;
+    int64_t total = 0;
+    for (int32_t k = 0; k < n; ++k) {
+        auto f = ctx->users.find(users[k]);
+        if (f == ctx->users.end()) return CKV_ERR_UNKNOWN_USER;
+        total += units_of(ctx, f->second.L);
+    }
+    int64_t off[5];
+    blob_sections(ctx, total, off);
+    if (bytes != off[4]) return CKV_ERR_INVALID_ARG;
+    DeviceGuard dg(ctx->cfg.device);
+    cudaStream_t s = (cudaStream_t)stream;
+    const int64_t ub = (int64_t)ctx->d_user * ctx->elem;  // no user sections without a user part
+    const int64_t eb[4] = {ctx->idx_bytes, ctx->idx_bytes, ub, ub};
+    const char* src[4] = {(const char*)ctx->a_idxK, (const char*)ctx->a_idxV, (const char*)ctx->a_userK,
+                          (const char*)ctx->a_userV};
+    int64_t done = 0;
+    for (int32_t k = 0; k < n; ++k) {
+        const UserEntry& e = ctx->users.find(users[k])->second;
+        const int64_t u = units_of(ctx, e.L);
+        for (int i = 0; i < 4 && u > 0; ++i)
+            if (eb[i] > 0)
+                CK(cudaMemcpyAsync((char*)blob + off[i] + done * eb[i], src[i] + e.base * eb[i], (size_t)(u * eb[i]),
+                               cudaMemcpyDefault, s));
+        done += u;
+    }
+    return CKV_OK;
+}
+
+ckv_status ckv_cache_import(ckv_ctx* ctx, int32_t n, const int64_t* users, const int32_t* L, const void* blob,
+                            int64_t bytes, void* stream)
+{
+    if (!ctx || n < 0 || (n > 0 && (!users || !L))) return CKV_ERR_INVALID_ARG;
+    if (!ctx->pool) return CKV_ERR_STATE;
+    if (n == 0) return CKV_OK;
+    std::vector<int64_t> unit_off((size_t)n + 1);
+    unit_off[0] = 0;
+    for (int32_t k = 0; k < n; ++k) {
+        if (L[k] < 0 || L[k] > INT32_MAX - 32) return CKV_ERR_INVALID_ARG;
+        unit_off[k + 1] = unit_off[k] + units_of(ctx, L[k]);
+    }
+    const int64_t total = unit_off[n];
+    int64_t off[5];
+    blob_sections(ctx, total, off);
+    if (bytes != off[4] || (total > 0 && !blob)) return CKV_ERR_INVALID_ARG;
+    DeviceGuard dg(ctx->cfg.device);
+    cudaStream_t s = (cudaStream_t)stream;
+    if (total > 0) {
+        ckv_status st = ensure_arena(ctx, total, s);
+        if (st != CKV_OK) return st;
+        const int64_t ub = (int64_t)ctx->d_user * ctx->elem;
+        const int64_t eb[4] = {ctx->idx_bytes, ctx->idx_bytes, ub, ub};
+        char* dst[4] = {(char*)ctx->a_idxK, (char*)ctx->a_idxV, (char*)ctx->a_userK, (char*)ctx->a_userV};
+        // the batch takes contiguous units behind what is stored: one copy per section
+        for (int i = 0; i < 4; ++i)
+            if (eb[i] > 0)
+                CK(cudaMemcpyAsync(dst[i] + ctx->used_units * eb[i], (const char*)blob + off[i],
+                                   (size_t)(total * eb[i]), cudaMemcpyDefault, s));
+        CK(cudaMemsetAsync(ctx->d_flag, 0, sizeof(int), s));
+        CK(launch_check_indices(ctx->idx_bytes, ctx->n_entries, dst[0] + ctx->used_units * eb[0],
+                                dst[1] + ctx->used_units * eb[1], total, ctx->d_flag, s));
+        int bad = 0;
+        CK(cudaMemcpyAsync(&bad, ctx->d_flag, sizeof(int), cudaMemcpyDeviceToHost, s));
+        CK(cudaStreamSynchronize(s));
+        if (bad) return CKV_ERR_INDEX_RANGE;  // used_units not advanced: nothing was stored
+    }
+    for (int32_t k = 0; k < n; ++k) {
+        auto f = ctx->users.find(users[k]);
+        if (f != ctx->users.end()) ctx->live_positions -= f->second.L;
+        ctx->users[users[k]] = UserEntry{ctx->used_units + unit_off[k], L[k], (L[k] + 31) / 32 * 32};
+        ctx->live_positions += L[k];
+    }
+    ctx->used_units += total;
+    ctx->generation++;
+    return CKV_OK;
+}
+
 ckv_status ckv_cache_evict(ckv_ctx* ctx, int64_t user)
 {
     if (!ctx) return CKV_ERR_INVALID_ARG;

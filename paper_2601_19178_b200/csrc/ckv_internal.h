@@ -79,6 +79,10 @@ cudaError_t launch_pack(int dtype, int G, int n_entries, int d_user, int idx_byt
 cudaError_t launch_materialize(int dtype, int D, const CacheView& cv, int64_t base, int L, int Lpad,
                                void* K_out, void* V_out, cudaStream_t s);
 
+// ORs 1 into *bad_flag (device int) if any of the n_units stored K or V indices is >= n_entries.
+cudaError_t launch_check_indices(int idx_bytes, int n_entries, const void* idxK, const void* idxV, int64_t n_units,
+                                 int* bad_flag, cudaStream_t s);
+
 // ---- kernels_simt.cu : CUDA-core family (any number of queries, best for few)
 cudaError_t launch_attend_simt(int dtype, int D, int max_M, const AttendArgs& a, cudaStream_t s);
 // Merges the partial results of split requests into `out`.

@@ -97,6 +97,17 @@ __global__ void materialize_kernel(int G, int n_entries, int d_user, int D,
     }
 }
 
+// Range check of stored indices that did not go through pack_kernel (imported blobs).
+template <typename I>
+__global__ void check_indices_kernel(const I* __restrict__ a, const I* __restrict__ b, int64_t n, uint32_t n_entries,
+                                     int* __restrict__ bad_flag)
+{
+    bool bad = false;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+        bad |= (uint32_t)a[i] >= n_entries || (uint32_t)b[i] >= n_entries;
+    if (__any_sync(0xffffffffu, bad) && (threadIdx.x & 31) == 0) atomicOr(bad_flag, 1);
+}
+
 inline int grid_for(int64_t total, int block)
 {
     int64_t g = (total + block - 1) / block;
@@ -159,6 +170,20 @@ cudaError_t launch_materialize(int dtype, int D, const CacheView& cv, int64_t ba
         if (cv.idx_bytes == 2) CKV_MAT(uint32_t, uint16_t); else CKV_MAT(uint32_t, int32_t);
     }
 #undef CKV_MAT
+    return cudaGetLastError();
+}
+
+cudaError_t launch_check_indices(int idx_bytes, int n_entries, const void* idxK, const void* idxV, int64_t n_units,
+                                 int* bad_flag, cudaStream_t s)
+{
+    if (n_units == 0) return cudaSuccess;
+    const int grid = grid_for(n_units, 256);
+    if (idx_bytes == 2)
+        check_indices_kernel<uint16_t><<<grid, 256, 0, s>>>((const uint16_t*)idxK, (const uint16_t*)idxV, n_units,
+                                                            (uint32_t)n_entries, bad_flag);
+    else
+        check_indices_kernel<int32_t><<<grid, 256, 0, s>>>((const int32_t*)idxK, (const int32_t*)idxV, n_units,
+                                                           (uint32_t)n_entries, bad_flag);
     return cudaGetLastError();
 }
 

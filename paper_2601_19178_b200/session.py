@@ -54,6 +54,20 @@ class CollectiveKV:
         B.ckv_attend(self.ctx, users, q_off, queries, out)
         return out
 
+    def export_blob(self, users) -> torch.Tensor:
+        """Packed caches of `users` as one pinned host buffer (the form a serving system keeps in
+        host memory and loads per request batch)."""
+        L = [B.ckv_user_length(self.ctx, int(u)) for u in users]
+        nbytes = B.ckv_cache_blob_bytes(self.ctx, L)
+        blob = torch.empty(max(nbytes, 1), dtype=torch.uint8).pin_memory()
+        B.ckv_cache_export(self.ctx, users, blob, nbytes)
+        torch.cuda.current_stream().synchronize()
+        return blob[:nbytes]
+
+    def import_blob(self, users, lengths, blob: torch.Tensor):
+        """Loads `users` (history lengths `lengths`) from a packed blob (host or device tensor)."""
+        B.ckv_cache_import(self.ctx, users, lengths, blob, blob.numel() * blob.element_size())
+
     def materialize(self, user: int):
         L = B.ckv_user_length(self.ctx, user)
         K = torch.empty((L, self.n_groups, self.head_dim), dtype=self.dtype, device=self.device)

@@ -371,6 +371,93 @@ def run_ours(args, w):
         dist.destroy_process_group()
 
 
+# Table 2 of the paper (A100, SIM model, Kuaivideo): latency in ms against batch size, for context only
+PAPER_TABLE2_A100_MS = {"batch": [1, 8, 32, 64, 128, 256, 512],
+                        "kv_cache": [0.099, 1.030, 1.808, 3.418, 6.679, 15.216, 32.991],
+                        "collectivekv": [0.084, 0.129, 0.136, 0.152, 0.222, 0.375, 0.695]}
+
+
+def run_load_path(args, w):
+    """Decode-stage load path (Sec. 4.4, Table 2): per request batch, the latency of bringing the
+    batch's cache from pinned host memory to the GPU.  Classical cache: one copy of the full-width
+    K/V bytes, T_load(s d_a).  Here: ckv_cache_import of the packed blob, T_load(s d_u + s), and
+    import + ckv_attend, which contains the on-GPU indexing T_index fused with the attention."""
+    import time
+    import torch
+    import paper_2601_19178_b200 as ckv
+    from paper_2601_19178_b200.session import as_device_tensor as dev
+
+    rank, _, local = rank_env()
+    if rank != 0:
+        return
+    torch.cuda.set_device(local)
+    batches = [b for b in (1, 8, 32, 64, 128, 256, 512) if b <= w.n_users]
+    data = synth.generate(w)
+    tdt = torch.float32 if w.dtype == "f32" else torch.bfloat16
+    e = 4 if w.dtype == "f32" else 2
+    src = ckv.CollectiveKV(w.n_groups, w.head_dim, tdt, w.mode, device=local)
+    src.pool_load(dev(data["pool_K"], w.dtype), dev(data["pool_V"], w.dtype))
+    src.cache_put_batch(data["users"], data["hist_off"], dev(data["idx_K"], "i"), dev(data["idx_V"], "i"),
+                        dev(data["user_K"], w.dtype), dev(data["user_V"], w.dtype))
+    lens = np.diff(data["hist_off"]).astype(np.int32)
+    blobs = {b: src.export_blob(data["users"][:b]) for b in batches}
+
+    dst = ckv.CollectiveKV(w.n_groups, w.head_dim, tdt, w.mode, device=local)
+    dst.pool_load(dev(data["pool_K"], w.dtype), dev(data["pool_V"], w.dtype))
+    q = dev(data["queries"], w.dtype)
+    out = torch.empty_like(q)
+    full_max = int(data["hist_off"][batches[-1]]) * w.n_groups * 2 * w.head_dim * e
+    host_full = torch.empty(full_max, dtype=torch.uint8).pin_memory()
+    dev_full = torch.empty(full_max, dtype=torch.uint8, device="cuda")
+    reps = max(args.steps, 5)
+
+    def med_ms(fn):
+        for _ in range(3):
+            fn()
+        ts = []
+        for _ in range(reps):
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            fn()
+            torch.cuda.synchronize()
+            ts.append(1e3 * (time.perf_counter() - t0))
+        return statistics.median(ts)
+
+    rows, ok = [], True
+    for b in batches:
+        users, L, blob = data["users"][:b], lens[:b], blobs[b]
+        q_off = data["q_off"][:b + 1]
+        nq = int(q_off[-1])
+        positions = int(data["hist_off"][b])
+        full_bytes = positions * w.n_groups * 2 * w.head_dim * e
+
+        def load_full():
+            dev_full[:full_bytes].copy_(host_full[:full_bytes], non_blocking=True)
+
+        def load_packed():
+            ckv.ckv_cache_clear(dst.ctx)
+            dst.import_blob(users, L, blob)
+
+        def load_and_attend():
+            load_packed()
+            dst.attend(users, q_off, q[:nq], out[:nq])
+
+        row = {"batch": b, "positions": positions, "full_kv_bytes": full_bytes, "packed_bytes": blob.numel(),
+               "kv_cache_load_ms": med_ms(load_full), "ckv_import_ms": med_ms(load_packed),
+               "ckv_import_attend_ms": med_ms(load_and_attend)}
+        # same users, same request shape: the resident cache must give the same bits
+        ok = ok and bool(torch.equal(out[:nq], src.attend(users, q_off, q[:nq])))
+        rows.append(row)
+    dst.close()
+    src.close()
+    line = {"mode": "load_path", "metric": "decode_load_latency_ms", "unit": "ms", "higher_is_better": False,
+            "n_gpus": 1, "repeats": reps, "timing": "host wall clock around call + device synchronise, median",
+            "data": "synthetic", "dtype": "f32" if w.dtype == "f32" else "bf16",
+            "config": {"workload": w.name, "describe": w.describe, "source": "pinned host memory"},
+            "rows": rows, "outputs_match_resident_cache": ok, "paper_table2_a100_ms": PAPER_TABLE2_A100_MS}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -383,12 +470,16 @@ def main():
     ap.add_argument("--split-len", type=int, default=0)
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-check", action="store_true", help="skip the sampled parity check")
+    ap.add_argument("--load-path", action="store_true",
+                    help="time the decode-stage load path per batch size (Sec. 4.4) instead of the attend step")
     args = ap.parse_args()
     w = synth.WORKLOADS[args.workload]
     if args.users:
         w = synth.scaled(w, n_users=args.users)
     if args.impl == "reference":
         run_reference(args, w)
+    elif args.load_path:
+        run_load_path(args, w)
     else:
         run_ours(args, w)
 

@@ -214,6 +214,8 @@ def run_ours(args, w):
         s.set_option("kernel", args.kernel)
     if args.split_len:
         s.set_option("split_len", args.split_len)
+    if args.mma_loader:
+        s.set_option("mma_loader", args.mma_loader)
     s.set_option("time_kernels", 1)
     users, q_off = data["users"], data["q_off"]
     q = dev(data["queries"], w.dtype)
@@ -347,7 +349,8 @@ def run_ours(args, w):
         "data": "synthetic",
         "config": {"workload": w.name, "describe": w.describe, "users": w.n_users, "positions": positions,
                    "l2": "flushed between timed steps (256 MiB overwrite)",
-                   "kernel_family": s.stat("kernel"), "work_items": s.stat("work_items"),
+                   "kernel_family": s.stat("kernel"), "mma_loader": s.stat("mma_loader"),
+                   "work_items": s.stat("work_items"),
                    "split_items": s.stat("split_items")},
         "users_per_sec": job_users * args.steps / (total_ms * 1e-3),
         "clocks": clocks,
@@ -468,6 +471,7 @@ def main():
     ap.add_argument("--users", type=int, default=0, help="override the user count (smaller captures)")
     ap.add_argument("--kernel", type=int, default=0)
     ap.add_argument("--split-len", type=int, default=0)
+    ap.add_argument("--mma-loader", type=int, default=0, help="1 = cp.async (default), 2 = TMA gathers")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-check", action="store_true", help="skip the sampled parity check")
     ap.add_argument("--load-path", action="store_true",

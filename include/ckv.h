@@ -230,6 +230,10 @@ CKV_API ckv_status ckv_cache_bytes(ckv_ctx* ctx, int64_t* compressed, int64_t* f
  *                  0 = choose automatically (default)
  *   "kernel"       0 = choose by queries per user (default); 1 = CUDA-core kernel;
  *                  2 = warp-level tensor-core kernel; 3 = tcgen05 kernel
+ *   "mma_loader"   how the warp-level tensor-core kernel brings pool rows into shared memory:
+ *                  0 or 1 = 16-byte asynchronous copies through L1 (default), 2 = TMA row gathers
+ *                  (UNSUPPORTED from ckv_attend if the driver cannot encode the tensor maps);
+ *                  the results are the same bits either way
  *   "l2_persist"   1 = ask for the pool to persist in L2 on the streams used (default), 0 = off
  *   "time_kernels" 1 = record CUDA events around the kernels of each ckv_attend (see ckv_last_stat)
  */
@@ -239,7 +243,8 @@ CKV_API ckv_status ckv_get_option(ckv_ctx* ctx, const char* name, int64_t* value
 /*
  * Introspection for tests and the benchmark.  Counters describe the most recent
  * ckv_attend: "launches" (kernels enqueued), "work_items", "split_items" (items that went
- * through the partial-result workspace), "kernel" (family that ran: 1, 2 or 3),
+ * through the partial-result workspace), "kernel" (family that ran: 1, 2 or 3), "mma_loader"
+ * (loader the last warp-level tensor-core launch used: 1 or 2),
  * "workspace_bytes", "plan_cache_hit"; with option "time_kernels" also "main_kernel_ns" and
  * "combine_kernel_ns" (device time of the attend kernel and of the split-merge kernel; the
  * query waits for that attend to finish; CKV_ERR_STATE if nothing was timed).

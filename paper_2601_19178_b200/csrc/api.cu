@@ -69,6 +69,8 @@ struct ckv_ctx {
     int n_entries = 0, d_shared = 0, d_user = 0, idx_bytes = 0;
     void* pool = nullptr;  // K rows then V rows, each [G][m][D]
     bool has_mma = false;         // the warp-level tensor-core family can run
+    bool has_tma = false;         // ... and its TMA-gather loader too (tensor maps of the pool encoded)
+    alignas(64) unsigned char tmaps[256] = {};  // two CUtensorMap: K pool, V pool
     bool has_umma = false;
     int* d_err = nullptr;  // OR of error codes from kernels whose bounded waits ran out
     size_t pool_half = 0;  // bytes of one of them
@@ -83,11 +85,11 @@ struct ckv_ctx {
     std::vector<Plan> plans;
     uint64_t tick = 0;
     // options
-    int64_t opt_split = 0, opt_kernel = 0, opt_l2 = 1, opt_time = 0;
+    int64_t opt_split = 0, opt_kernel = 0, opt_l2 = 1, opt_time = 0, opt_loader = 0;
     cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};  // around the main kernel and the combine
     bool ev_valid = false;
     // statistics of the last attend
-    int64_t st_launches = 0, st_items = 0, st_split = 0, st_kernel = 0, st_ws = 0, st_hit = 0;
+    int64_t st_launches = 0, st_items = 0, st_split = 0, st_kernel = 0, st_ws = 0, st_hit = 0, st_loader = 0;
     std::string cuda_err;
 
     ckv_status fail(cudaError_t e)
@@ -469,6 +471,8 @@ ckv_status ckv_pool_load(ckv_ctx* ctx, const void* pool_K, const void* pool_V, i
         ctx->pool_half = half;
     }
     ctx->has_mma = mma_supported(ctx->cfg.dtype, D, D - d_shared);
+    ctx->has_tma = ctx->has_mma && make_pool_tensor_maps(D, (int64_t)G * n_entries, ctx->pool,
+                                                         (const char*)ctx->pool + half, ctx->tmaps);
     ctx->has_umma = umma_supported(ctx->cfg.dtype, D, D - d_shared, n_entries <= 65536 ? 2 : 4);
     CK(launch_pool_layout(ctx->cfg.dtype, G, n_entries, d_shared, D, sk.dev, ctx->pool, s));
     CK(launch_pool_layout(ctx->cfg.dtype, G, n_entries, d_shared, D, sv.dev, (char*)ctx->pool + half, s));
@@ -684,6 +688,23 @@ ckv_status ckv_cache_clear(ckv_ctx* ctx)
     return CKV_OK;
 }
 
+namespace {
+
+// The warp-level tensor-core kernel with the loader the options ask for.  The cp.async loader is the default:
+// on B200 a warp spends about 100 clocks per TMA gather instruction it issues, so with the compute warps doing
+// their own gathers the TMA loader measured slower (cfg4: 607 against 522 us; cfg5, Zipf indices that profit
+// from L1, which TMA bypasses: 5.07 against 2.37 ms).  Both loaders give the same bits.
+ckv_status run_mma(ckv_ctx* ctx, int D, int max_M, const AttendArgs& a, cudaStream_t s)
+{
+    const int loader = ctx->opt_loader == 2 ? 2 : 1;
+    if (loader == 2 && !ctx->has_tma) return CKV_ERR_UNSUPPORTED;
+    ctx->st_loader = loader;
+    CK(launch_attend_mma(D, max_M, a, loader == 2 ? ctx->tmaps : nullptr, ctx->d_err, s));
+    return CKV_OK;
+}
+
+}  // namespace
+
 ckv_status ckv_attend(ckv_ctx* ctx, int32_t n, const int64_t* users, const int32_t* q_off,
                       const void* queries, void* out, void* stream)
 {
@@ -744,9 +765,10 @@ ckv_status ckv_attend(ckv_ctx* ctx, int32_t n, const int64_t* users, const int32
     if (pl->n_items > 0) {
         if (pl->family == 3)
             CK(launch_attend_umma(pl->max_M, a, ctx->n_sms, ctx->d_err, s));
-        else if (pl->family == 2)
-            CK(launch_attend_mma(D, pl->max_M, a, s));
-        else
+        else if (pl->family == 2) {
+            ckv_status st2 = run_mma(ctx, D, pl->max_M, a, s);
+            if (st2 != CKV_OK) return st2;
+        } else
             CK(launch_attend_simt(ctx->cfg.dtype, D, pl->max_M, a, s));
         ctx->st_launches++;
     }
@@ -826,6 +848,9 @@ ckv_status ckv_set_option(ckv_ctx* ctx, const char* name, int64_t value)
     } else if (!std::strcmp(name, "kernel")) {
         if (value < 0 || value > 3) return CKV_ERR_INVALID_ARG;
         ctx->opt_kernel = value;
+    } else if (!std::strcmp(name, "mma_loader")) {
+        if (value < 0 || value > 2) return CKV_ERR_INVALID_ARG;
+        ctx->opt_loader = value;
     } else if (!std::strcmp(name, "l2_persist")) {
         ctx->opt_l2 = value != 0;
     } else if (!std::strcmp(name, "time_kernels")) {
@@ -841,6 +866,7 @@ ckv_status ckv_get_option(ckv_ctx* ctx, const char* name, int64_t* value)
     if (!ctx || !name || !value) return CKV_ERR_INVALID_ARG;
     if (!std::strcmp(name, "split_len")) *value = ctx->opt_split;
     else if (!std::strcmp(name, "kernel")) *value = ctx->opt_kernel;
+    else if (!std::strcmp(name, "mma_loader")) *value = ctx->opt_loader;
     else if (!std::strcmp(name, "l2_persist")) *value = ctx->opt_l2;
     else if (!std::strcmp(name, "time_kernels")) *value = ctx->opt_time;
     else return CKV_ERR_INVALID_ARG;
@@ -854,6 +880,7 @@ ckv_status ckv_last_stat(ckv_ctx* ctx, const char* name, int64_t* value)
     else if (!std::strcmp(name, "work_items")) *value = ctx->st_items;
     else if (!std::strcmp(name, "split_items")) *value = ctx->st_split;
     else if (!std::strcmp(name, "kernel")) *value = ctx->st_kernel;
+    else if (!std::strcmp(name, "mma_loader")) *value = ctx->st_loader;
     else if (!std::strcmp(name, "workspace_bytes")) *value = ctx->st_ws;
     else if (!std::strcmp(name, "plan_cache_hit")) *value = ctx->st_hit;
     else if (!std::strcmp(name, "device_errors")) {
@@ -1027,7 +1054,7 @@ extern "C" ckv_status ckv_attend_static(ckv_ctx* ctx, int32_t n, const int64_t* 
     a.scale = ctx->scale;
     if (n_items > 0) {
         if (family == 2)
-            CK(launch_attend_mma(D, max_M, a, s));
+            CK(launch_attend_mma(D, max_M, a, nullptr, ctx->d_err, s));
         else
             CK(launch_attend_simt(ctx->cfg.dtype, D, max_M, a, s));
     }

@@ -92,7 +92,11 @@ cudaError_t launch_combine(int D, const AttendArgs& a, const int32_t* split_reqs
 // ---- kernels_mma.cu : warp-level tensor-core family (bf16, head_dim 32 or 64, d_user <= 8)
 bool mma_supported(int dtype, int head_dim, int d_user);
 int mma_queries_per_warp(int head_dim, int max_M);
-cudaError_t launch_attend_mma(int head_dim, int max_M, const AttendArgs& a, cudaStream_t s);
+// tensor_maps: null = fill the staging ring with cp.async copies; else the two maps of make_pool_tensor_maps =
+// fill it with TMA gathers (err_flag: device int, OR-ed with a code if a bounded wait for a tile ran out).
+cudaError_t launch_attend_mma(int head_dim, int max_M, const AttendArgs& a, const void* tensor_maps, int* err_flag,
+                              cudaStream_t s);
+bool make_pool_tensor_maps(int head_dim, int64_t rows, const void* poolK, const void* poolV, void* maps_out);
 
 // ---- kernels_umma.cu : tcgen05 family (bf16, head_dim 32, d_user in {0, 1, 2, 4, 8}, 16-bit stored indices)
 bool umma_supported(int dtype, int head_dim, int d_user, int idx_bytes);

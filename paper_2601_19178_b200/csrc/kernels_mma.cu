@@ -9,6 +9,13 @@
 // row, and the copies in flight cost no registers: a warp keeps NST - 1 tiles outstanding
 // while it computes.  The user-specific leading elements (Eq. K) are written over the head
 // of each staged row.  Positions keep their order: tile row r is position p0 + r.
+//
+// Two ways to fill the ring (template parameter TMA), same results bit for bit:
+//   - 16-byte cp.async copies through L1 (hot rows of skewed index distributions stay in L1, but every
+//     row crosses the L1 / shared-memory data pipe on the way in and again on the way out);
+//   - TMA tile::gather4 loads, four pool rows per instruction, completion on an mbarrier: the rows
+//     bypass L1 and that pipe; the hardware swizzle modes are the chunk order ldmatrix wants.
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <math_constants.h>
 
@@ -116,17 +123,33 @@ __device__ __forceinline__ void store_user_part(uint32_t addr, const uint4& r, i
     }
 }
 
-template <int D, int MT>
+template <int D, int MT, bool TMA>
 struct MmaCfg {
     static constexpr int ROWB = D * 2;            // bytes per row
     static constexpr int CPR = ROWB / 16;         // 16-byte chunks per row
     static constexpr int RPI = 32 / CPR;          // rows one warp-wide copy instruction covers
     static constexpr int TILE_B = 32 * ROWB;      // one K or V tile of 32 positions
-    static constexpr int NST = D == 64 ? 3 : 2;   // ring depth (64-byte rows: more resident warps beat a deeper ring)
+    // ring depth (more resident warps beat a deeper ring, except for cp.async with 128-byte rows)
+    static constexpr int NST = (D == 64 && !TMA) ? 3 : 2;
     static constexpr int WARPS = 4;
-    static constexpr int SMEM = WARPS * NST * 2 * TILE_B;
-    static constexpr int MIN_BLOCKS = MT == 1 ? (D == 64 ? 2 : 4) : 1;
+    // TMA: tiles on 1024-byte boundaries (the swizzle pattern follows the address), then one mbarrier per slot
+    static constexpr int SMEM = WARPS * NST * 2 * TILE_B + (TMA ? 1024 + WARPS * NST * 8 : 0);
+    static constexpr int MIN_BLOCKS = MT == 1 ? (D == 64 ? (TMA ? 3 : 2) : 4) : 1;
 };
+
+enum { ERR_MMA_LOAD = 16 };  // a bounded wait for a TMA tile ran out
+constexpr int kTmaSpinLimit = 1 << 22;
+
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
 
 // chunk c of tile row r sits at chunk c ^ swz(r): the eight rows of an 8x8 ldmatrix block fall into
 // eight different 16-byte bank groups
@@ -136,11 +159,12 @@ __device__ __forceinline__ int swz(int r)
     return D == 64 ? (r & 7) : ((r >> 1) & 3);
 }
 
-template <int D, int MT, int MODE, bool IDX16>
-__global__ void __launch_bounds__(128, MmaCfg<D, MT>::MIN_BLOCKS)
-    attend_mma_kernel(const AttendArgs a, int n_mb)
+template <int D, int MT, int MODE, bool IDX16, bool TMA>
+__global__ void __launch_bounds__(128, MmaCfg<D, MT, TMA>::MIN_BLOCKS)
+    attend_mma_kernel(const AttendArgs a, int n_mb, const __grid_constant__ CUtensorMap tmK,
+                      const __grid_constant__ CUtensorMap tmV, int* err_flag)
 {
-    using C = MmaCfg<D, MT>;
+    using C = MmaCfg<D, MT, TMA>;
     constexpr int NTD = D / 8, KS = D / 16, ROWB = C::ROWB, CPR = C::CPR, RPI = C::RPI, NST = C::NST;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -196,7 +220,19 @@ __global__ void __launch_bounds__(128, MmaCfg<D, MT>::MIN_BLOCKS)
     const int nsteps = (it.len + 31) >> 5;
     const float sc = a.scale * (MODE == CKV_SOFTMAX ? kLog2e : 0.5f);
 
-    const uint32_t ring = smem_u32(smem_raw) + warp * (NST * 2 * C::TILE_B);
+    uint32_t smem0 = smem_u32(smem_raw);
+    if constexpr (TMA) smem0 = (smem0 + 1023u) & ~1023u;
+    const uint32_t ring = smem0 + warp * (NST * 2 * C::TILE_B);
+    const uint32_t bars = smem0 + C::WARPS * (NST * 2 * C::TILE_B) + warp * (NST * 8);  // TMA only
+    if constexpr (TMA) {
+        if (lane == 0) {
+#pragma unroll
+            for (int i = 0; i < NST; ++i) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bars + 8 * i));
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        }
+        __syncwarp();
+    }
+    const int row_base = grp * a.cv.n_entries;  // TMA row coordinate of pool row 0 of this group
     // ldmatrix row addresses of this lane (matrix lane >> 3, row lane & 7)
     const int lr = lane & 7, lm = lane >> 3;
     uint32_t offK[KS / 2 > 0 ? KS / 2 : 1], offV[NTD / 2];
@@ -210,13 +246,47 @@ __global__ void __launch_bounds__(128, MmaCfg<D, MT>::MIN_BLOCKS)
     // copies of one tile: the indices of its 32 positions sit one per lane
     auto issue = [&](int step, int idx_k, int idx_v) {
         const uint32_t kt = ring + (step % NST) * (2 * C::TILE_B), vt = kt + C::TILE_B;
+        if constexpr (TMA) {
+            // lanes 0..7 fetch the K tile, lanes 8..15 the V tile, four rows (positions 4j .. 4j+3) each
+            const uint32_t bar = bars + 8 * (step % NST);
+            if (lane == 0)
+                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(2 * C::TILE_B)
+                             : "memory");
+            __syncwarp();
+            int r[4];
+            const int j4 = 4 * (lane & 7);
+            if constexpr (IDX16) {
+                const int both = idx_k | (idx_v << 16);
 #pragma unroll
-        for (int i = 0; i < 32 / RPI; ++i) {
-            const int r = i * RPI + cr;
-            const uint32_t off = r * ROWB + ((cc ^ swz<D>(r)) << 4);
-            const int rk = __shfl_sync(0xffffffffu, idx_k, r), rv = __shfl_sync(0xffffffffu, idx_v, r);
-            cp_async16(kt + off, pK + (int64_t)rk * ROWB);
-            cp_async16(vt + off, pV + (int64_t)rv * ROWB);
+                for (int j = 0; j < 4; ++j) {
+                    const int x = __shfl_sync(0xffffffffu, both, j4 + j);
+                    r[j] = row_base + (lane < 8 ? (x & 0xffff) : (int)((uint32_t)x >> 16));
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int xk = __shfl_sync(0xffffffffu, idx_k, j4 + j), xv = __shfl_sync(0xffffffffu, idx_v, j4 + j);
+                    r[j] = row_base + (lane < 8 ? xk : xv);
+                }
+            }
+            if (lane < 16) {
+                const CUtensorMap* tm = lane < 8 ? &tmK : &tmV;
+                const uint32_t dst = (lane < 8 ? kt : vt) + j4 * ROWB;
+                asm volatile(
+                    "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes "
+                    "[%0], [%1, {%2, %3, %4, %5, %6}], [%7];" ::"r"(dst),
+                    "l"(tm), "r"(0), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(bar)
+                    : "memory");
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 32 / RPI; ++i) {
+                const int r = i * RPI + cr;
+                const uint32_t off = r * ROWB + ((cc ^ swz<D>(r)) << 4);
+                const int rk = __shfl_sync(0xffffffffu, idx_k, r), rv = __shfl_sync(0xffffffffu, idx_v, r);
+                cp_async16(kt + off, pK + (int64_t)rk * ROWB);
+                cp_async16(vt + off, pV + (int64_t)rv * ROWB);
+            }
         }
     };
     auto fetch_idx = [&](int step, int& idx_k, int& idx_v) {
@@ -240,7 +310,7 @@ __global__ void __launch_bounds__(128, MmaCfg<D, MT>::MIN_BLOCKS)
     for (int s0 = 0; s0 < NST - 1; ++s0) {
         fetch_idx(s0, ikA, ivA);
         if (s0 < nsteps) issue(s0, ikA, ivA);
-        cp_async_commit();
+        if constexpr (!TMA) cp_async_commit();
     }
     fetch_idx(NST - 1, ikA, ivA);
     fetch_idx(NST, ikB, ivB);
@@ -250,13 +320,29 @@ __global__ void __launch_bounds__(128, MmaCfg<D, MT>::MIN_BLOCKS)
     fetch_user(0, ukA, uvA);
     fetch_user(1, ukB, uvB);
 
+    bool ok = true;
     for (int step = 0; step < nsteps; ++step) {
         const int p0 = it.begin + 32 * step;
         if (step + NST - 1 < nsteps) issue(step + NST - 1, ikA, ivA);
-        cp_async_commit();
+        if constexpr (!TMA) cp_async_commit();
         ikA = ikB; ivA = ivB; ikB = ikC; ivB = ivC;
         fetch_idx(step + NST + 2, ikC, ivC);
-        cp_async_wait<NST - 1>();
+        if constexpr (TMA) {
+            const uint32_t bar = bars + 8 * (step % NST), parity = (step / NST) & 1;
+            int spins = 0;
+            while (!mbar_try_wait(bar, parity)) {
+                if (++spins > kTmaSpinLimit) {
+                    ok = false;
+                    break;
+                }
+            }
+            if (!__all_sync(0xffffffffu, ok)) {  // give up: nothing more is issued, nothing is stored
+                ok = false;
+                break;
+            }
+        } else {
+            cp_async_wait<NST - 1>();
+        }
         __syncwarp();
         const uint32_t kt = ring + (step % NST) * (2 * C::TILE_B), vt = kt + C::TILE_B;
         // Eq. K: dims [0, d_user) of every row come from the user-specific part
@@ -383,9 +469,19 @@ __global__ void __launch_bounds__(128, MmaCfg<D, MT>::MIN_BLOCKS)
 #pragma unroll
                 for (int j = 0; j < NTD; ++j) mma_bf16(o[mt][j], pa[b], vb[b][j][0], vb[b][j][1]);
         }
-        __syncwarp();  // every lane is done reading this tile before the ring slot is refilled
+        // every lane is done with this tile before the ring slot is refilled (TMA: its ordinary stores
+        // and loads are ordered before the asynchronous-proxy writes of the refill)
+        if constexpr (TMA) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
     }
-    cp_async_wait<0>();
+    if constexpr (TMA) {
+        if (!ok) {
+            if (lane == 0) atomicOr(err_flag, ERR_MMA_LOAD);
+            return;
+        }
+    } else {
+        cp_async_wait<0>();
+    }
 
     // epilogue: finish the row sums over the quad, then store outputs or partials
 #pragma unroll
@@ -427,32 +523,36 @@ __global__ void __launch_bounds__(128, MmaCfg<D, MT>::MIN_BLOCKS)
     }
 }
 
-template <int D, int MT, int MODE, bool IDX16>
-cudaError_t launch_mma_one(const AttendArgs& a, int n_mb, dim3 grid, cudaStream_t s)
+template <int D, int MT, int MODE, bool IDX16, bool TMA>
+cudaError_t launch_mma_one(const AttendArgs& a, int n_mb, dim3 grid, const CUtensorMap* maps, int* err_flag,
+                           cudaStream_t s)
 {
-    using C = MmaCfg<D, MT>;
+    using C = MmaCfg<D, MT, TMA>;
     static bool configured = false;  // per instantiation; the attribute is idempotent
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(attend_mma_kernel<D, MT, MODE, IDX16>,
+        cudaError_t e = cudaFuncSetAttribute(attend_mma_kernel<D, MT, MODE, IDX16, TMA>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    attend_mma_kernel<D, MT, MODE, IDX16><<<grid, 128, C::SMEM, s>>>(a, n_mb);
+    static const CUtensorMap none{};
+    attend_mma_kernel<D, MT, MODE, IDX16, TMA>
+        <<<grid, 128, C::SMEM, s>>>(a, n_mb, TMA ? maps[0] : none, TMA ? maps[1] : none, err_flag);
     return cudaGetLastError();
 }
 
 template <int D, int MT>
-cudaError_t launch_mma(const AttendArgs& a, int n_mb, cudaStream_t s)
+cudaError_t launch_mma(const AttendArgs& a, int n_mb, const CUtensorMap* maps, int* err_flag, cudaStream_t s)
 {
     const int64_t warps = (int64_t)a.n_items * n_mb;
     const dim3 grid((unsigned)((warps + 3) / 4), a.cv.n_groups);
     const bool i16 = a.cv.idx_bytes == 2;
-    if (a.mode == CKV_SOFTMAX)
-        return i16 ? launch_mma_one<D, MT, CKV_SOFTMAX, true>(a, n_mb, grid, s)
-                   : launch_mma_one<D, MT, CKV_SOFTMAX, false>(a, n_mb, grid, s);
-    return i16 ? launch_mma_one<D, MT, CKV_SILU_OVER_L, true>(a, n_mb, grid, s)
-               : launch_mma_one<D, MT, CKV_SILU_OVER_L, false>(a, n_mb, grid, s);
+#define CKV_MMA_GO(MODE, I16)                                                                        \
+    (maps ? launch_mma_one<D, MT, MODE, I16, true>(a, n_mb, grid, maps, err_flag, s)                 \
+          : launch_mma_one<D, MT, MODE, I16, false>(a, n_mb, grid, maps, err_flag, s))
+    if (a.mode == CKV_SOFTMAX) return i16 ? CKV_MMA_GO(CKV_SOFTMAX, true) : CKV_MMA_GO(CKV_SOFTMAX, false);
+    return i16 ? CKV_MMA_GO(CKV_SILU_OVER_L, true) : CKV_MMA_GO(CKV_SILU_OVER_L, false);
+#undef CKV_MMA_GO
 }
 
 }  // namespace
@@ -465,17 +565,51 @@ bool mma_supported(int dtype, int head_dim, int d_user)
 // head_dim 64 rows keep a warp busy with one 16-query tile; 32-wide heads take up to four
 int mma_queries_per_warp(int D, int max_M) { return (D == 64 || max_M <= 16) ? 16 : (max_M <= 32 ? 32 : 64); }
 
-cudaError_t launch_attend_mma(int D, int max_M, const AttendArgs& a, cudaStream_t s)
+cudaError_t launch_attend_mma(int D, int max_M, const AttendArgs& a, const void* tensor_maps, int* err_flag,
+                              cudaStream_t s)
 {
     if (a.n_items == 0) return cudaSuccess;
+    const CUtensorMap* maps = reinterpret_cast<const CUtensorMap*>(tensor_maps);
     const int qpw = mma_queries_per_warp(D, max_M);
     const int n_mb = (max_M + qpw - 1) / qpw;
-    if (D == 64) return launch_mma<64, 1>(a, n_mb, s);
+    if (D == 64) return launch_mma<64, 1>(a, n_mb, maps, err_flag, s);
     switch (qpw) {
-        case 16: return launch_mma<32, 1>(a, n_mb, s);
-        case 32: return launch_mma<32, 2>(a, n_mb, s);
-        default: return launch_mma<32, 4>(a, n_mb, s);
+        case 16: return launch_mma<32, 1>(a, n_mb, maps, err_flag, s);
+        case 32: return launch_mma<32, 2>(a, n_mb, maps, err_flag, s);
+        default: return launch_mma<32, 4>(a, n_mb, maps, err_flag, s);
     }
+}
+
+// Tensor maps of the K and the V pool ([n_groups * n_entries] rows of head_dim bf16) for tile::gather4: a box of
+// one row, hardware swizzle of the row's 16-byte chunks (128-byte rows: chunk ^ (row & 7); 64-byte rows:
+// chunk ^ ((row >> 1) & 3)).  maps_out: 2 x 128 bytes, 64-byte aligned.  false if the driver cannot encode them.
+bool make_pool_tensor_maps(int D, int64_t rows, const void* poolK, const void* poolV, void* maps_out)
+{
+    typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                 const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                 CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    if ((D != 32 && D != 64) || rows < 1 || rows > INT32_MAX) return false;
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || !fn ||
+        q != cudaDriverEntryPointSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    CUtensorMap* maps = reinterpret_cast<CUtensorMap*>(maps_out);
+    const void* src[2] = {poolK, poolV};
+    for (int i = 0; i < 2; ++i) {
+        const cuuint64_t dims[2] = {(cuuint64_t)D, (cuuint64_t)rows};
+        const cuuint64_t strides[1] = {(cuuint64_t)D * 2};
+        const cuuint32_t box[2] = {(cuuint32_t)D, 1};
+        const cuuint32_t estr[2] = {1, 1};
+        const CUresult r = reinterpret_cast<EncodeFn>(fn)(
+            &maps[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(src[i]), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, D == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+            CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return false;
+    }
+    return true;
 }
 
 }  // namespace ckv

@@ -47,29 +47,49 @@ def test_every_kernel_family_matches_oracle(name, kernel):
     assert_close(got, oracle_attend(w, d), w.dtype, f"{name} kernel {kernel}")
 
 
-@pytest.mark.parametrize("kernel", [2, 3])
+@pytest.mark.parametrize("kernel,loader", [(2, 1), (2, 2), (3, 0)])
 @pytest.mark.parametrize("mode", ["softmax", "silu_over_l"])
 @pytest.mark.parametrize("d_user", [0, 1, 2, 4, 8])
-def test_tensor_core_kernels_user_widths_and_sharp_softmax(kernel, mode, d_user):
+def test_tensor_core_kernels_user_widths_and_sharp_softmax(kernel, loader, mode, d_user):
     w = synth.Workload("tc", 3, 32 - d_user, d_user, 300, 5, (1, 700), 70, mode, "bf16", 1.1, 1 / 32, 1 / 32, 21)
     d = synth.generate(w)
     scale = 8.0 / np.sqrt(32) if mode == "softmax" else 1.0
-    s = make_session(w, d, scale=scale, kernel=kernel, split_len=256)
+    s = make_session(w, d, scale=scale, kernel=kernel, split_len=256, mma_loader=loader)
     got = gpu_attend(w, d, session=s)
     assert s.stat("split_items") > 0 and s.stat("device_errors") == 0
     s.close()
     assert_close(got, oracle_attend(w, d, scale=scale), "bf16", f"d_user={d_user}")
 
 
+@pytest.mark.parametrize("name", ["cfg4", "cfg5", "cfg5_ragged", "cfg2_ragged", "cfg3_ragged"])
+def test_warp_mma_kernel_loaders_agree_bit_for_bit(name):
+    """The staging ring is filled by cp.async copies (loader 1) or TMA row gathers (loader 2); everything
+    after that is the same code, so the outputs must be the same bits.  Loader 0 is the default (cp.async)."""
+    w = SMALL[name]
+    d = synth.generate(w)
+    outs = {}
+    for loader in (1, 2, 0):
+        s = make_session(w, d, kernel=2, mma_loader=loader)
+        outs[loader] = gpu_attend(w, d, session=s)
+        again = gpu_attend(w, d, session=s)
+        assert s.stat("kernel") == 2 and s.stat("device_errors") == 0
+        assert s.stat("mma_loader") == (loader or 1)
+        s.close()
+        assert np.array_equal(outs[loader], again)
+    assert np.array_equal(outs[1], outs[2]) and np.array_equal(outs[0], outs[1])
+    assert_close(outs[2], oracle_attend(w, d), w.dtype, name)
+
+
+@pytest.mark.parametrize("loader", [1, 2])
 @pytest.mark.parametrize("n_queries", [1, 7, 20])
 @pytest.mark.parametrize("mode", ["softmax", "silu_over_l"])
 @pytest.mark.parametrize("d_user", [0, 1, 2, 4, 8])
-def test_warp_mma_kernel_head_dim_64(n_queries, mode, d_user):
+def test_warp_mma_kernel_head_dim_64(n_queries, mode, d_user, loader):
     """64-wide heads run on the warp-level tensor-core kernel from one query per user on."""
     w = synth.Workload("tc64", 3, 64 - d_user, d_user, 500, 6, (1, 900), n_queries, mode, "bf16", 1.1, 1 / 32, 1 / 32, 22)
     d = synth.generate(w)
     scale = 8.0 / np.sqrt(64) if mode == "softmax" else 1.0
-    s = make_session(w, d, scale=scale, split_len=256)
+    s = make_session(w, d, scale=scale, split_len=256, mma_loader=loader)
     got = gpu_attend(w, d, session=s)
     assert s.stat("kernel") == 2 and s.stat("split_items") > 0 and s.stat("device_errors") == 0
     s.close()

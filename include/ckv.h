@@ -229,7 +229,12 @@ CKV_API ckv_status ckv_cache_bytes(ckv_ctx* ctx, int64_t* compressed, int64_t* f
  *   "split_len"    positions per history chunk for the split-along-history reduction;
  *                  0 = choose automatically (default)
  *   "kernel"       0 = choose by queries per user (default); 1 = CUDA-core kernel;
- *                  2 = warp-level tensor-core kernel; 3 = tcgen05 kernel
+ *                  2 = warp-level tensor-core kernel; 3 = tcgen05 kernel; 4 = pool-side
+ *                  factorisation (one query per user: per-user score and weight tables over the
+ *                  pool replace the row gathers; chosen by default when histories are long against
+ *                  the pool; its weight histogram is summed with shared-memory atomics, so the last
+ *                  bits can differ from run to run).  ckv_attend returns UNSUPPORTED if the forced
+ *                  kernel cannot take the request.
  *   "mma_loader"   how the warp-level tensor-core kernel brings pool rows into shared memory:
  *                  0 or 1 = 16-byte asynchronous copies through L1 (default), 2 = TMA row gathers
  *                  (UNSUPPORTED from ckv_attend if the driver cannot encode the tensor maps);
@@ -243,7 +248,7 @@ CKV_API ckv_status ckv_get_option(ckv_ctx* ctx, const char* name, int64_t* value
 /*
  * Introspection for tests and the benchmark.  Counters describe the most recent
  * ckv_attend: "launches" (kernels enqueued), "work_items", "split_items" (items that went
- * through the partial-result workspace), "kernel" (family that ran: 1, 2 or 3), "mma_loader"
+ * through the partial-result workspace), "kernel" (family that ran: 1 to 4), "mma_loader"
  * (loader the last warp-level tensor-core launch used: 1 or 2),
  * "workspace_bytes", "plan_cache_hit"; with option "time_kernels" also "main_kernel_ns" and
  * "combine_kernel_ns" (device time of the attend kernel and of the split-merge kernel; the

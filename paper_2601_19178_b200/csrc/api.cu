@@ -36,7 +36,7 @@ struct Plan {
     Item* d_items = nullptr;
     int32_t* d_split = nullptr;
     Work* d_works = nullptr;
-    int32_t n_items = 0, n_split = 0, split_items = 0, max_M = 0, family = 1;
+    int32_t n_items = 0, n_split = 0, split_items = 0, max_M = 0, max_L = 0, n_req = 0, family = 1;
     int64_t part_rows = 0;
     uint64_t last_use = 0;
 };
@@ -252,8 +252,9 @@ ckv_status build_plan(ckv_ctx* ctx, Plan& pl, int32_t n, const int64_t* users, c
                       cudaStream_t s)
 {
     std::vector<Req> reqs((size_t)n);
-    int64_t total_pos = 0;
-    int32_t max_M = 0;
+    int64_t total_pos = 0, n_active = 0;
+    int32_t max_M = 0, max_L = 0;
+    bool all_single = true;
     for (int32_t k = 0; k < n; ++k) {
         auto f = ctx->users.find(users[k]);
         if (f == ctx->users.end()) return CKV_ERR_UNKNOWN_USER;
@@ -265,19 +266,40 @@ ckv_status build_plan(ckv_ctx* ctx, Plan& pl, int32_t n, const int64_t* users, c
         r.M = q_off[k + 1] - q_off[k];
         r.part0 = -1;
         r.n_chunks = 1;
-        if (r.M > 0) total_pos += r.L;
+        if (r.M > 0) {
+            total_pos += r.L;
+            max_L = std::max(max_L, r.L);
+            n_active++;
+            all_single = all_single && r.M == 1;
+        }
         max_M = std::max(max_M, r.M);
     }
     pl.max_M = max_M;
+    pl.max_L = max_L;
+    pl.n_req = n;
     const bool can_mma = ctx->has_mma;
     // tcgen05 from three 16-query blocks on, else the warp-level tensor-core kernel (faster than the CUDA-core
     // kernel from a single query on); the CUDA-core kernel serves what neither supports
-    if (ctx->opt_kernel == 0) pl.family = ctx->has_umma && max_M >= 48 ? 3 : (can_mma ? 2 : 1);
+    // One query per user and histories long against the pool: the pool-side factorisation trades the row gathers
+    // for two tables per (user, group) in HBM.  Break-even measured on B200 at a mean length of about a quarter
+    // of the pool's entries for 64-wide heads (the gathering kernel costs half as much per position at 32).
+    const bool can_fact = all_single && n_active > 0 &&
+                          fact_max_history(ctx->cfg.dtype, ctx->cfg.head_dim, ctx->d_user, ctx->n_entries,
+                                           ctx->cfg.mode) >= max_L;
+    const int64_t fact_ratio = ctx->cfg.head_dim == 64 ? 4 : 2;
+    if (ctx->opt_kernel == 0)
+        pl.family = ctx->has_umma && max_M >= 48                               ? 3
+                    : can_fact && total_pos * fact_ratio >= n_active * ctx->n_entries ? 4
+                    : can_mma                                                  ? 2
+                                                                               : 1;
+    else if (ctx->opt_kernel == 4 && can_fact) pl.family = 4;
     else if (ctx->opt_kernel == 1) pl.family = 1;
     else if (ctx->opt_kernel == 2 && can_mma) pl.family = 2;
     else if (ctx->opt_kernel == 3 && ctx->has_umma) pl.family = 3;
     else return CKV_ERR_UNSUPPORTED;
-    const int64_t C = ctx->opt_split > 0 ? ctx->opt_split : auto_split_len(ctx, total_pos, pl.family, max_M);
+    const int64_t C = pl.family == 4         ? (int64_t)INT32_MAX  // one CTA holds a whole history
+                      : ctx->opt_split > 0 ? ctx->opt_split
+                                           : auto_split_len(ctx, total_pos, pl.family, max_M);
     std::vector<Item> items;
     std::vector<int32_t> split;
     items.reserve((size_t)n);
@@ -740,7 +762,10 @@ ckv_status ckv_attend(ckv_ctx* ctx, int32_t n, const int64_t* users, const int32
         CK(grow(ctx->stage_out, o_bytes));
         d_out = ctx->stage_out.p;
     }
-    const size_t ws = (size_t)pl->part_rows * G * (D + 2) * sizeof(float);
+    // split-reduction partials, or the factorisation's tables (per request and group: n_entries + a few floats)
+    const size_t ws = pl->family == 4
+                          ? (size_t)pl->n_req * G * ((size_t)ctx->n_entries + fact_aux_floats()) * sizeof(float)
+                          : (size_t)pl->part_rows * G * (D + 2) * sizeof(float);
     if (ws) CK(grow(ctx->partials, ws));
     ctx->st_ws = (int64_t)ws;
 
@@ -763,7 +788,11 @@ ckv_status ckv_attend(ckv_ctx* ctx, int32_t n, const int64_t* users, const int32
         CK(cudaEventRecord(ctx->ev[0], s));
     }
     if (pl->n_items > 0) {
-        if (pl->family == 3)
+        if (pl->family == 4) {
+            float* tw = (float*)ctx->partials.p;
+            CK(launch_attend_fact(D, a, pl->n_req, pl->max_L, tw, tw + (size_t)pl->n_req * G * ctx->n_entries, s));
+            ctx->st_launches += 2;
+        } else if (pl->family == 3)
             CK(launch_attend_umma(pl->max_M, a, ctx->n_sms, ctx->d_err, s));
         else if (pl->family == 2) {
             ckv_status st2 = run_mma(ctx, D, pl->max_M, a, s);
@@ -846,7 +875,7 @@ ckv_status ckv_set_option(ckv_ctx* ctx, const char* name, int64_t value)
         if (value < 0) return CKV_ERR_INVALID_ARG;
         ctx->opt_split = value == 0 ? 0 : (value + 63) / 64 * 64;
     } else if (!std::strcmp(name, "kernel")) {
-        if (value < 0 || value > 3) return CKV_ERR_INVALID_ARG;
+        if (value < 0 || value > 4) return CKV_ERR_INVALID_ARG;
         ctx->opt_kernel = value;
     } else if (!std::strcmp(name, "mma_loader")) {
         if (value < 0 || value > 2) return CKV_ERR_INVALID_ARG;

@@ -98,6 +98,15 @@ cudaError_t launch_attend_mma(int head_dim, int max_M, const AttendArgs& a, cons
                               cudaStream_t s);
 bool make_pool_tensor_maps(int head_dim, int64_t rows, const void* poolK, const void* poolV, void* maps_out);
 
+// ---- kernels_fact.cu : pool-side factorisation for one query per user (bf16, head_dim 32 or 64, d_user <= 8)
+// Largest history the family can take for this shape (its tables and scores share one CTA's shared memory),
+// or -1 if the shape is not supported.
+int fact_max_history(int dtype, int head_dim, int d_user, int n_entries, int mode);
+int fact_aux_floats();
+// a.items: one unsplit item per request with a query.  tw: [n_req][G][n_entries] floats, aux: [n_req][G][fact_aux_floats()].
+cudaError_t launch_attend_fact(int head_dim, const AttendArgs& a, int n_req, int max_L, float* tw, float* aux,
+                               cudaStream_t s);
+
 // ---- kernels_umma.cu : tcgen05 family (bf16, head_dim 32, d_user in {0, 1, 2, 4, 8}, 16-bit stored indices)
 bool umma_supported(int dtype, int head_dim, int d_user, int idx_bytes);
 // err_flag: device int, OR-ed with a non-zero code if a bounded wait inside the kernel ran out.

@@ -89,7 +89,7 @@ def test_warp_mma_kernel_head_dim_64(n_queries, mode, d_user, loader):
     w = synth.Workload("tc64", 3, 64 - d_user, d_user, 500, 6, (1, 900), n_queries, mode, "bf16", 1.1, 1 / 32, 1 / 32, 22)
     d = synth.generate(w)
     scale = 8.0 / np.sqrt(64) if mode == "softmax" else 1.0
-    s = make_session(w, d, scale=scale, split_len=256, mma_loader=loader)
+    s = make_session(w, d, scale=scale, split_len=256, mma_loader=loader, kernel=2)
     got = gpu_attend(w, d, session=s)
     assert s.stat("kernel") == 2 and s.stat("split_items") > 0 and s.stat("device_errors") == 0
     s.close()
@@ -231,6 +231,73 @@ def test_empty_history_empty_query_list_and_repeated_user(kernel):
     o_rep = O.attend("bf16", "softmax", w.default_scale, d["pool_K"], d["pool_V"], d["hist_off"], d["idx_K"],
                      d["idx_V"], d["user_K"], d["user_V"], np.array([0, 3, 3, 3, 3]), d2["queries"])
     assert_close(out[9:12], o_rep, "bf16")
+
+
+@pytest.mark.parametrize("mode", ["softmax", "silu_over_l"])
+@pytest.mark.parametrize("head", [(64, 0), (63, 1), (62, 2), (60, 4), (56, 8), (28, 4), (29, 3)])
+def test_pool_side_factorisation_matches_oracle(mode, head):
+    """One query per user: score table T = P_k q and weight histogram w replace the row gathers (kernel 4)."""
+    dg, du = head
+    w = synth.Workload("fact", 3, dg, du, 333, 21, (1, 700), 1, mode, "bf16", 1.1, 1.0 / (dg + du), 1.0 / (dg + du), 31)
+    d = synth.generate(w)
+    scale = 8.0 / np.sqrt(dg + du) if mode == "softmax" else 1.0
+    s = make_session(w, d, scale=scale, kernel=4)
+    got = gpu_attend(w, d, session=s)
+    assert s.stat("kernel") == 4 and s.stat("launches") == 3 and s.stat("split_items") == 0
+    s.close()
+    want = oracle_attend(w, d, scale=scale)
+    assert_close(got, want, "bf16", f"{head} {mode}")
+    # the gathering tensor-core kernel on the same inputs: both within tolerance of the oracle, and of each other
+    other = gpu_attend(w, d, scale=scale, kernel=2)
+    assert np.abs(got - other).max() <= 2.0 ** -7 * np.abs(want).max()
+
+
+def test_pool_side_factorisation_is_chosen_for_long_histories_only_and_handles_edge_requests():
+    import paper_2601_19178_b200 as ckv
+    # histories long against the pool (mean length >= n_entries / 4): chosen by default
+    w = synth.Workload("fact_long", 2, 60, 4, 512, 6, (100, 2000), 1, "softmax", "bf16", None, 1 / 64, 1 / 64, 32)
+    d = synth.generate(w)
+    s = make_session(w, d)
+    got = gpu_attend(w, d, session=s)
+    assert s.stat("kernel") == 4
+    assert_close(got, oracle_attend(w, d), "bf16", "auto")
+    # request list with an empty query list and a repeated user: [u0, u1 (no query), u2, u0]
+    req = d["users"][[0, 1, 2, 0]]
+    q_off = np.array([0, 1, 1, 2, 3], dtype=np.int32)
+    q = to_dev(d["queries"][[0, 2, 0]], "bf16")
+    out = s.attend(req, q_off, q).float().cpu().numpy().astype(np.float64)
+    assert s.stat("kernel") == 4
+    assert_close(out[0], got[0], "bf16")
+    assert_close(out[1], got[2], "bf16")
+    assert_close(out[2], got[0], "bf16")
+    # more than one query for a user: the family cannot take it
+    s.set_option("kernel", 4)
+    with pytest.raises(ckv.CkvError) as e:
+        s.attend(d["users"][:2], np.array([0, 2, 3], dtype=np.int32), to_dev(d["queries"][:3], "bf16"))
+    assert e.value.status == ckv.CKV_ERR_UNSUPPORTED
+    s.close()
+    # short histories against a large pool: the gathering kernel stays
+    w2 = synth.Workload("fact_short", 2, 60, 4, 4096, 6, (10, 200), 1, "softmax", "bf16", None, 1 / 64, 1 / 64, 33)
+    d2 = synth.generate(w2)
+    s2 = make_session(w2, d2)
+    assert_close(gpu_attend(w2, d2, session=s2), oracle_attend(w2, d2), "bf16", "short")
+    assert s2.stat("kernel") == 2
+    s2.close()
+
+
+def test_pool_side_factorisation_empty_history_gives_zero_rows():
+    w = synth.Workload("fact_empty", 2, 30, 2, 64, 3, (40, 40), 1, "softmax", "bf16", None, 1 / 32, 1 / 32, 8)
+    d = synth.generate(w)
+    keep = np.r_[0:40, 80:120]
+    for k in ("idx_K", "idx_V", "user_K", "user_V"):
+        d[k] = np.ascontiguousarray(d[k][keep])
+    d["hist_off"] = np.array([0, 40, 40, 80], dtype=np.int64)
+    s = make_session(w, d, kernel=4)
+    got = gpu_attend(w, d, session=s)
+    assert s.stat("kernel") == 4
+    s.close()
+    assert np.all(got[1] == 0.0)
+    assert_close(got, oracle_attend(w, d), "bf16", "empty history")
 
 
 def test_host_buffers_go_through_the_same_path():

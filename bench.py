@@ -48,10 +48,11 @@ def _peaks():
 
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel,
-# from the ncu captures summarised under profiles/ (attend_*_kernel_<workload>.md).  cfg3 and cfg5
+# from the ncu captures summarised under profiles/ (attend_*_<workload>.md; cfg4: the three launches of
+# the factorised path together, which is also what the timed interval covers).  cfg3 and cfg5
 # were captured on a cut of the workload and scaled by the number of users.  Set an entry to None
 # when its kernel changes after the capture.
-TRAFFIC_BYTES = {"cfg2": 190658560, "cfg3": 1090254848, "cfg4": 372015872, "cfg5": 1854877696}
+TRAFFIC_BYTES = {"cfg2": 190658560, "cfg3": 1090254848, "cfg4": 821408256, "cfg5": 1852809216}
 # transcendental evaluations per SM per clock (ex2 / tanh issue rate of the special-function unit)
 XU_PER_SM_CLK = 16
 # bytes per SM per clock through the L1 / shared-memory data pipe (one 128-byte wavefront per clock)

@@ -300,6 +300,26 @@ def test_pool_side_factorisation_empty_history_gives_zero_rows():
     assert_close(got, oracle_attend(w, d), "bf16", "empty history")
 
 
+@pytest.mark.parametrize("name", ["cfg2", "cfg3", "cfg4", "cfg5"])
+def test_full_size_workloads_on_sampled_users(name):
+    """The benchmark workloads at full size, default options (the launch configuration bench.py times):
+    first, last, longest, shortest and two random users against the oracle."""
+    w = W[name]
+    d = synth.generate(w)
+    s = make_session(w, d)
+    out = s.attend(d["users"], d["q_off"], to_dev(d["queries"], w.dtype))
+    torch.cuda.synchronize()
+    assert s.stat("device_errors") == 0
+    s.close()
+    lens = np.diff(d["hist_off"])
+    rng = np.random.default_rng(11)
+    sel = sorted(set([0, w.n_users - 1, int(np.argmax(lens)), int(np.argmin(lens))] +
+                     rng.integers(0, w.n_users, size=2).tolist()))
+    rows = np.concatenate([np.arange(d["q_off"][u], d["q_off"][u + 1]) for u in sel])
+    got = out[torch.from_numpy(rows).cuda()].float().cpu().numpy().astype(np.float64)
+    assert_close(got, oracle_attend(w, d, sel=sel), w.dtype, name)
+
+
 def test_host_buffers_go_through_the_same_path():
     w = SMALL["cfg5_ragged"]
     d = synth.generate(w)

@@ -13,7 +13,7 @@
 //   fact_table_kernel  T[r][g][j] = q_r . P_k[g][j]          m16n8k16 MMAs, fp32 out
 //   fact_main_kernel   one CTA per (user, group): T row into shared memory, scores, max, weights, histogram w,
 //                      user-part output and row sum; w takes T's place in shared memory and in HBM
-//   fact_out_kernel    out[r][g][:] = (w[r][g] P_v[g] + user part) / l          MMAs, w rounded to bf16
+//   fact_out_kernel    out[r][g][:] = (w[r][g] P_v[g] + user part) / l          MMAs, w in bf16
 #include <cuda_bf16.h>
 #include <math_constants.h>
 
@@ -301,7 +301,13 @@ __global__ void __launch_bounds__(kMainThreads, 1)
 #pragma unroll
         for (int k = 0; k < 9; ++k) Sb[(tid >> 5) * 9 + k] = vals[k];
     }
-    for (int j = tid; j < m; j += kMainThreads) row[j] = Ws[j];
+    // w goes back to HBM rounded to bf16 (the precision the output product takes it in), two entries per word,
+    // over the head of the T row; an odd last entry is paired with a zero
+    {
+        uint32_t* wrow = reinterpret_cast<uint32_t*>(row);
+        for (int j2 = tid; 2 * j2 < m; j2 += kMainThreads)
+            wrow[j2] = pack_bf16(Ws[2 * j2], 2 * j2 + 1 < m ? Ws[2 * j2 + 1] : 0.f);
+    }
     __syncthreads();
     if (tid < 9) {
         float v = 0.f;
@@ -352,26 +358,25 @@ __global__ void __launch_bounds__(kOutWarps * 32, 1)
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
     };
-    // weights of one 32-entry chunk as A fragments' raw values: k-step b, (row lo/hi) x (cols 2t, 2t+1, 2t+8, 2t+9)
-    auto load_w = [&](int jc, float (&x)[16]) {
+    // weights of one 32-entry chunk as A fragments: k-step b, registers (row lo, row hi) x (cols 2t.., cols 2t+8..);
+    // a register is the bf16 pair the main kernel stored
+    auto load_w = [&](int jc, uint32_t (&x)[8]) {
 #pragma unroll
         for (int b = 0; b < 2; ++b)
 #pragma unroll
-            for (int h = 0; h < 2; ++h)
-#pragma unroll
-                for (int e = 0; e < 2; ++e) {
-                    const int j = jc + 16 * b + 8 * h + 2 * t + e;
-                    const bool in = j < jend;
-                    x[8 * b + 4 * h + 2 * e] = (in && v_lo) ? __ldg(w_lo + j) : 0.f;
-                    x[8 * b + 4 * h + 2 * e + 1] = (in && v_hi) ? __ldg(w_hi + j) : 0.f;
-                }
+            for (int h = 0; h < 2; ++h) {
+                const int j = jc + 16 * b + 8 * h + 2 * t;  // even; the pair (j, j + 1) ends inside this warp's span
+                const bool in = j < jend;
+                x[4 * b + 2 * h] = (in && v_lo) ? __ldg(reinterpret_cast<const uint32_t*>(w_lo) + (j >> 1)) : 0u;
+                x[4 * b + 2 * h + 1] = (in && v_hi) ? __ldg(reinterpret_cast<const uint32_t*>(w_hi) + (j >> 1)) : 0u;
+            }
     };
 
     float o[NTD][4];
 #pragma unroll
     for (int j = 0; j < NTD; ++j) o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f;
     const int nch = jbeg < jend ? (jend - jbeg + 31) / 32 : 0;
-    float wa[16], wb[16];
+    uint32_t wa[8], wb[8];
     if (nch > 0) {
         issue(jbeg, 0);
         load_w(jbeg, wa);
@@ -389,11 +394,7 @@ __global__ void __launch_bounds__(kOutWarps * 32, 1)
         const uint32_t vt = ring + (c & 1) * TILE_B;
 #pragma unroll
         for (int b = 0; b < 2; ++b) {
-            uint32_t pa[4];
-            pa[0] = pack_bf16(wa[8 * b], wa[8 * b + 2]);      // row lo, cols 2t, 2t+1
-            pa[1] = pack_bf16(wa[8 * b + 1], wa[8 * b + 3]);  // row hi
-            pa[2] = pack_bf16(wa[8 * b + 4], wa[8 * b + 6]);  // row lo, cols 2t+8, 2t+9
-            pa[3] = pack_bf16(wa[8 * b + 5], wa[8 * b + 7]);  // row hi
+            const uint32_t pa[4] = {wa[4 * b], wa[4 * b + 1], wa[4 * b + 2], wa[4 * b + 3]};
 #pragma unroll
             for (int jp = 0; jp < NTD / 2; ++jp) {
                 uint32_t v0, v1, v2, v3;
@@ -407,7 +408,7 @@ __global__ void __launch_bounds__(kOutWarps * 32, 1)
         }
         __syncwarp();  // every lane is done reading the slot that the next iteration refills
 #pragma unroll
-        for (int i = 0; i < 16; ++i) wa[i] = wb[i];
+        for (int i = 0; i < 8; ++i) wa[i] = wb[i];
     }
 
     // sum the warps' partial outputs in fixed order, add the user part, normalise, store

@@ -790,7 +790,8 @@ ckv_status ckv_attend(ckv_ctx* ctx, int32_t n, const int64_t* users, const int32
     if (pl->n_items > 0) {
         if (pl->family == 4) {
             float* tw = (float*)ctx->partials.p;
-            CK(launch_attend_fact(D, a, pl->n_req, pl->max_L, tw, tw + (size_t)pl->n_req * G * ctx->n_entries, s));
+            CK(launch_attend_fact(D, a, pl->n_req, pl->max_L, ctx->n_sms, tw,
+                                  tw + (size_t)pl->n_req * G * ctx->n_entries, s));
             ctx->st_launches += 2;
         } else if (pl->family == 3)
             CK(launch_attend_umma(pl->max_M, a, ctx->n_sms, ctx->d_err, s));

@@ -104,8 +104,8 @@ bool make_pool_tensor_maps(int head_dim, int64_t rows, const void* poolK, const 
 int fact_max_history(int dtype, int head_dim, int d_user, int n_entries, int mode);
 int fact_aux_floats();
 // a.items: one unsplit item per request with a query.  tw: [n_req][G][n_entries] floats, aux: [n_req][G][fact_aux_floats()].
-cudaError_t launch_attend_fact(int head_dim, const AttendArgs& a, int n_req, int max_L, float* tw, float* aux,
-                               cudaStream_t s);
+cudaError_t launch_attend_fact(int head_dim, const AttendArgs& a, int n_req, int max_L, int n_sms, float* tw,
+                               float* aux, cudaStream_t s);
 
 // ---- kernels_umma.cu : tcgen05 family (bf16, head_dim 32, d_user in {0, 1, 2, 4, 8}, 16-bit stored indices)
 bool umma_supported(int dtype, int head_dim, int d_user, int idx_bytes);

@@ -11,7 +11,7 @@
 //
 // Three launches:
 //   fact_table_kernel  T[r][g][j] = q_r . P_k[g][j]          m16n8k16 MMAs, fp32 out
-//   fact_main_kernel   one CTA per (user, group): T row into shared memory, scores, max, weights, histogram w,
+//   fact_main_kernel   persistent CTAs over the (user, group) pairs: T row into shared memory, scores, max, weights, histogram w,
 //                      user-part output and row sum; w takes T's place in shared memory and in HBM
 //   fact_out_kernel    out[r][g][:] = (w[r][g] P_v[g] + user part) / l          MMAs, w in bf16
 #include <cuda_bf16.h>
@@ -192,127 +192,166 @@ __device__ __forceinline__ float block_reduce(float v, bool is_max, float* red)
 
 constexpr int kAux = 16;  // floats per (request, group): [0] row sum l, [1..8] user-part output (not normalised)
 
+// Persistent: CTA c takes (item, group) pairs c, c + gridDim.x, ... of the list ordered longest history first
+// (pair = item * G + group, so neighbours in the list weigh about the same).  While a pair is processed, the T row
+// of the CTA's next pair is already on its way into the other table buffer.
 template <int D, int MODE, bool IDX16>
 __global__ void __launch_bounds__(kMainThreads, 1)
     fact_main_kernel(const AttendArgs a, float* __restrict__ tw, float* __restrict__ aux, int s_cap)
 {
     extern __shared__ __align__(16) float fsm[];
-    const int m = a.cv.n_entries, G = a.cv.n_groups, d_user = a.cv.d_user, grp = blockIdx.y;
-    const Item it = a.items[blockIdx.x];
-    const Req rq = a.reqs[it.req];
-    const int L = rq.L, tid = threadIdx.x;
-    float* Ts = fsm;                   // [m]     T row of this (user, group); dead after the scores
-    float* Ws = fsm;                   // [m]     weight histogram, in the same memory
-    float* Sb = fsm + m;               // [s_cap] scores (softmax), weights (SiLU)
-    float* red = Sb + s_cap;           // [32]
-    float* row = tw + ((int64_t)it.req * G + grp) * m;
-    const int64_t unit0 = rq.base + (int64_t)grp * rq.Lpad;
+    const int m = a.cv.n_entries, G = a.cv.n_groups, d_user = a.cv.d_user, tid = threadIdx.x;
+    const int n_pairs = a.n_items * G;
+    // fsm[0 .. 2m): two table buffers; a pair's T row, dead after the scores, then its weight histogram
+    float* Sb = fsm + 2 * (size_t)m;     // [s_cap] scores (softmax), half scores (SiLU); at the end the warps' sums
+    float* red = Sb + s_cap;             // [32]
     const uint16_t* uK = reinterpret_cast<const uint16_t*>(a.cv.userK);
     const uint16_t* uV = reinterpret_cast<const uint16_t*>(a.cv.userV);
     const float sc = a.scale * (MODE == CKV_SOFTMAX ? kLog2e : 0.5f);
     constexpr int B = 4;  // positions per thread whose loads are in flight together
     int ix[B];
     uint4 x[B];
-    auto load_batch = [&](const void* idx, const uint16_t* u, int i0) {
+
+    struct Pair {
+        int req, grp, L, q0;
+        int64_t unit0;
+    };
+    auto get_pair = [&](int p) {
+        Pair r;
+        const Item it = a.items[p / G];
+        const Req rq = a.reqs[it.req];
+        r.req = it.req;
+        r.grp = p - (p / G) * G;
+        r.L = rq.L;
+        r.q0 = rq.q0;
+        r.unit0 = rq.base + (int64_t)r.grp * rq.Lpad;
+        return r;
+    };
+    auto table_row = [&](const Pair& pr) { return tw + ((int64_t)pr.req * G + pr.grp) * m; };
+    auto fetch_table = [&](const Pair& pr, float* dstp) {  // all of the row in flight at once
+        const float* row = table_row(pr);
+        if ((m & 3) == 0) {
+            const uint32_t dst = smem_u32(dstp);
+            for (int j = 4 * tid; j < m; j += 4 * kMainThreads)
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + 4 * j), "l"(row + j) : "memory");
+        } else {
+            for (int j = tid; j < m; j += kMainThreads) dstp[j] = row[j];
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    auto load_batch = [&](const void* idx, const uint16_t* u, const Pair& pr, int i0) {
 #pragma unroll
         for (int b = 0; b < B; ++b) {
             const int i = i0 + b * kMainThreads;
             ix[b] = 0;
             x[b] = make_uint4(0, 0, 0, 0);
-            if (i < L) {
-                ix[b] = load_index<IDX16>(idx, unit0 + i);
-                x[b] = load_user(u, unit0 + i, d_user);
+            if (i < pr.L) {
+                ix[b] = load_index<IDX16>(idx, pr.unit0 + i);
+                x[b] = load_user(u, pr.unit0 + i, d_user);
             }
         }
     };
 
-    // T row into shared memory, all of it in flight at once, with the first batch of K-side loads behind it
-    if ((m & 3) == 0) {
-        const uint32_t dst = smem_u32(Ts);
-        for (int j = 4 * tid; j < m; j += 4 * kMainThreads)
-            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + 4 * j), "l"(row + j) : "memory");
-        asm volatile("cp.async.commit_group;" ::: "memory");
-    } else {
-        for (int j = tid; j < m; j += kMainThreads) Ts[j] = row[j];
-    }
-    float qu[8], ou[8];
-    {
-        const uint16_t* q = reinterpret_cast<const uint16_t*>(a.queries) + ((int64_t)rq.q0 * G + grp) * D;
+    int p = blockIdx.x, k = 0;
+    if (p >= n_pairs) return;
+    Pair cur = get_pair(p);
+    fetch_table(cur, fsm);
+    load_batch(a.cv.idxK, uK, cur, tid);
+    for (;;) {
+        float* Ts = fsm + (size_t)k * m;
+        float* Ws = Ts;
+        const int L = cur.L;
+        float qu[8], ou[8];
+        {
+            const uint16_t* q = reinterpret_cast<const uint16_t*>(a.queries) + ((int64_t)cur.q0 * G + cur.grp) * D;
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            qu[e] = e < d_user ? bf16_bits_to_float(__ldg(q + e)) : 0.f;
-            ou[e] = 0.f;
+            for (int e = 0; e < 8; ++e) {
+                qu[e] = e < d_user ? bf16_bits_to_float(__ldg(q + e)) : 0.f;
+                ou[e] = 0.f;
+            }
         }
-    }
-    load_batch(a.cv.idxK, uK, tid);
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
-    __syncthreads();
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        __syncthreads();  // T of this pair is in place; the other buffer's histogram has been written out
+        const int p_next = p + gridDim.x;
+        const bool more = p_next < n_pairs;
+        Pair nxt = cur;
+        if (more) {
+            nxt = get_pair(p_next);
+            fetch_table(nxt, fsm + (size_t)(k ^ 1) * m);
+        }
 
-    // scores: Sb[i] = scale * (q_u . K_u[i] + T[I_k[i]])   (softmax: in log2 units; SiLU: half the score)
-    float mx = -CUDART_INF_F, lsum = 0.f;
-    for (int i0 = tid; i0 < L;) {
+        // scores: Sb[i] = scale * (q_u . K_u[i] + T[I_k[i]])   (softmax: in log2 units; SiLU: half the score)
+        float mx = -CUDART_INF_F, lsum = 0.f;
+        for (int i0 = tid; i0 < L;) {
 #pragma unroll
-        for (int b = 0; b < B; ++b) {
-            const int i = i0 + b * kMainThreads;
-            if (i < L) {
-                const float sv = dot_user(qu, x[b], Ts[ix[b]]) * sc;
-                Sb[i] = sv;
-                mx = fmaxf(mx, sv);
-            }
-        }
-        i0 += B * kMainThreads;
-        if (i0 < L) load_batch(a.cv.idxK, uK, i0);
-    }
-    load_batch(a.cv.idxV, uV, tid);  // the first V-side batch travels during the reduction
-    if constexpr (MODE == CKV_SOFTMAX) mx = block_reduce(mx, true, red);
-    else __syncthreads();
-    // T is dead: the same memory becomes the histogram
-    for (int j = tid; j < m; j += kMainThreads) Ws[j] = 0.f;
-    __syncthreads();
-    // weights: p_i into w[I_v[i]], p_i V_u[i] into the user-part output (every thread reads back its own scores)
-    for (int i0 = tid; i0 < L;) {
-#pragma unroll
-        for (int b = 0; b < B; ++b) {
-            const int i = i0 + b * kMainThreads;
-            if (i < L) {
-                float p;
-                if constexpr (MODE == CKV_SOFTMAX) {
-                    p = ex2(Sb[i] - mx);
-                    lsum += p;
-                } else {
-                    const float h = Sb[i];  // silu(x) = x sigmoid(x) = h (1 + tanh(h)), h = x / 2
-                    p = fmaf(h, tanh_fast(h), h);
+            for (int b = 0; b < B; ++b) {
+                const int i = i0 + b * kMainThreads;
+                if (i < L) {
+                    const float sv = dot_user(qu, x[b], Ts[ix[b]]) * sc;
+                    Sb[i] = sv;
+                    mx = fmaxf(mx, sv);
                 }
-                atomicAdd(&Ws[ix[b]], p);
-                axpy_user(ou, p, x[b]);
             }
+            i0 += B * kMainThreads;
+            if (i0 < L) load_batch(a.cv.idxK, uK, cur, i0);
         }
-        i0 += B * kMainThreads;
-        if (i0 < L) load_batch(a.cv.idxV, uV, i0);
-    }
-    // row sum and user-part output: warp sums, then one thread per value adds the warps' sums in fixed order
-    float vals[9] = {lsum, ou[0], ou[1], ou[2], ou[3], ou[4], ou[5], ou[6], ou[7]};
+        load_batch(a.cv.idxV, uV, cur, tid);  // the first V-side batch travels during the reduction
+        if constexpr (MODE == CKV_SOFTMAX) mx = block_reduce(mx, true, red);
+        else __syncthreads();
+        // T is dead: the same memory becomes the histogram
+        for (int j = tid; j < m; j += kMainThreads) Ws[j] = 0.f;
+        __syncthreads();
+        // weights: p_i into w[I_v[i]], p_i V_u[i] into the user-part output (every thread reads back its own scores)
+        for (int i0 = tid; i0 < L;) {
 #pragma unroll
-    for (int k = 0; k < 9; ++k)
+            for (int b = 0; b < B; ++b) {
+                const int i = i0 + b * kMainThreads;
+                if (i < L) {
+                    float pw;
+                    if constexpr (MODE == CKV_SOFTMAX) {
+                        pw = ex2(Sb[i] - mx);
+                        lsum += pw;
+                    } else {
+                        const float h = Sb[i];  // silu(x) = x sigmoid(x) = h (1 + tanh(h)), h = x / 2
+                        pw = fmaf(h, tanh_fast(h), h);
+                    }
+                    atomicAdd(&Ws[ix[b]], pw);
+                    axpy_user(ou, pw, x[b]);
+                }
+            }
+            i0 += B * kMainThreads;
+            if (i0 < L) load_batch(a.cv.idxV, uV, cur, i0);
+        }
+        if (more) load_batch(a.cv.idxK, uK, nxt, tid);  // the next pair's first K-side batch travels during the write-out
+        // row sum and user-part output: warp sums, then one thread per value adds the warps' sums in fixed order
+        float vals[9] = {lsum, ou[0], ou[1], ou[2], ou[3], ou[4], ou[5], ou[6], ou[7]};
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) vals[k] += __shfl_xor_sync(0xffffffffu, vals[k], o);
-    __syncthreads();  // the histogram is complete; Sb is free
-    if ((tid & 31) == 0) {
+        for (int q9 = 0; q9 < 9; ++q9)
 #pragma unroll
-        for (int k = 0; k < 9; ++k) Sb[(tid >> 5) * 9 + k] = vals[k];
-    }
-    // w goes back to HBM rounded to bf16 (the precision the output product takes it in), two entries per word,
-    // over the head of the T row; an odd last entry is paired with a zero
-    {
-        uint32_t* wrow = reinterpret_cast<uint32_t*>(row);
-        for (int j2 = tid; 2 * j2 < m; j2 += kMainThreads)
-            wrow[j2] = pack_bf16(Ws[2 * j2], 2 * j2 + 1 < m ? Ws[2 * j2 + 1] : 0.f);
-    }
-    __syncthreads();
-    if (tid < 9) {
-        float v = 0.f;
-        for (int w = 0; w < kMainThreads / 32; ++w) v += Sb[w * 9 + tid];
-        aux[((int64_t)it.req * G + grp) * kAux + tid] = v;
+            for (int o = 16; o > 0; o >>= 1) vals[q9] += __shfl_xor_sync(0xffffffffu, vals[q9], o);
+        __syncthreads();  // the histogram is complete; Sb is free
+        if ((tid & 31) == 0) {
+#pragma unroll
+            for (int q9 = 0; q9 < 9; ++q9) Sb[(tid >> 5) * 9 + q9] = vals[q9];
+        }
+        // w goes back to HBM rounded to bf16 (the precision the output product takes it in), two entries per word,
+        // over the head of the T row; an odd last entry is paired with a zero
+        {
+            uint32_t* wrow = reinterpret_cast<uint32_t*>(table_row(cur));
+            for (int j2 = tid; 2 * j2 < m; j2 += kMainThreads)
+                wrow[j2] = pack_bf16(Ws[2 * j2], 2 * j2 + 1 < m ? Ws[2 * j2 + 1] : 0.f);
+        }
+        __syncthreads();
+        if (tid < 9) {
+            float v = 0.f;
+            for (int w = 0; w < kMainThreads / 32; ++w) v += Sb[w * 9 + tid];
+            aux[((int64_t)cur.req * G + cur.grp) * kAux + tid] = v;
+        }
+        if (!more) break;
+        __syncthreads();  // Sb (the warps' sums) is read before the next pair's scores overwrite it
+        cur = nxt;
+        p = p_next;
+        k ^= 1;
     }
 }
 
@@ -447,7 +486,7 @@ cudaError_t set_smem(K kernel, size_t bytes)
 }
 
 template <int D>
-cudaError_t launch_fact(const AttendArgs& a, int n_req, int max_L, float* tw, float* aux, cudaStream_t s)
+cudaError_t launch_fact(const AttendArgs& a, int n_req, int max_L, int n_sms, float* tw, float* aux, cudaStream_t s)
 {
     const int m = a.cv.n_entries, G = a.cv.n_groups;
     const bool i16 = a.cv.idx_bytes == 2, soft = a.mode == CKV_SOFTMAX;
@@ -455,8 +494,9 @@ cudaError_t launch_fact(const AttendArgs& a, int n_req, int max_L, float* tw, fl
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     const int s_cap = std::max((max_L + 31) / 32 * 32, 9 * (kMainThreads / 32));  // scores; later the warps' sums
-    const size_t smem_main = ((size_t)m + s_cap + 32) * sizeof(float);
-    const dim3 grid(a.n_items, G);
+    const size_t smem_main = (2 * (size_t)m + s_cap + 32) * sizeof(float);
+    const int n_pairs = a.n_items * G;
+    const dim3 grid(n_pairs < n_sms ? n_pairs : n_sms);
 #define CKV_FACT_MAIN(MODE, I16)                                                       \
     do {                                                                               \
         e = set_smem(fact_main_kernel<D, MODE, I16>, smem_main);                       \
@@ -485,7 +525,7 @@ int fact_max_history(int dtype, int head_dim, int d_user, int n_entries, int mod
 {
     if (dtype != CKV_BF16 || (head_dim != 32 && head_dim != 64) || d_user > 8) return -1;
     (void)mode;
-    const int64_t floats = 220 * 1024 / 4 - 32 - (int64_t)n_entries;  // one table + one score per position
+    const int64_t floats = 220 * 1024 / 4 - 32 - 2 * (int64_t)n_entries;  // two table buffers + one score per position
     if (floats < 9 * (kMainThreads / 32)) return -1;
     return (int)(floats / 32 * 32);
 }
@@ -494,10 +534,12 @@ int fact_aux_floats() { return kAux; }
 
 // Three launches; a.items holds one unsplit item per request with a query; tw: [n_req][G][n_entries] floats,
 // aux: [n_req][G][fact_aux_floats()] floats.
-cudaError_t launch_attend_fact(int D, const AttendArgs& a, int n_req, int max_L, float* tw, float* aux, cudaStream_t s)
+cudaError_t launch_attend_fact(int D, const AttendArgs& a, int n_req, int max_L, int n_sms, float* tw, float* aux,
+                               cudaStream_t s)
 {
     if (a.n_items == 0) return cudaSuccess;
-    return D == 64 ? launch_fact<64>(a, n_req, max_L, tw, aux, s) : launch_fact<32>(a, n_req, max_L, tw, aux, s);
+    return D == 64 ? launch_fact<64>(a, n_req, max_L, n_sms, tw, aux, s)
+                   : launch_fact<32>(a, n_req, max_L, n_sms, tw, aux, s);
 }
 
 }  // namespace ckv

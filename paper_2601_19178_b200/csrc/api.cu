@@ -764,7 +764,7 @@ ckv_status ckv_attend(ckv_ctx* ctx, int32_t n, const int64_t* users, const int32
     }
     // split-reduction partials, or the factorisation's tables (per request and group: n_entries + a few floats)
     const size_t ws = pl->family == 4
-                          ? (size_t)pl->n_req * G * ((size_t)ctx->n_entries + fact_aux_floats()) * sizeof(float)
+                          ? (size_t)pl->n_req * G * ((size_t)fact_row_floats(ctx->n_entries) + fact_aux_floats()) * sizeof(float)
                           : (size_t)pl->part_rows * G * (D + 2) * sizeof(float);
     if (ws) CK(grow(ctx->partials, ws));
     ctx->st_ws = (int64_t)ws;
@@ -791,7 +791,7 @@ ckv_status ckv_attend(ckv_ctx* ctx, int32_t n, const int64_t* users, const int32
         if (pl->family == 4) {
             float* tw = (float*)ctx->partials.p;
             CK(launch_attend_fact(D, a, pl->n_req, pl->max_L, ctx->n_sms, tw,
-                                  tw + (size_t)pl->n_req * G * ctx->n_entries, s));
+                                  tw + (size_t)pl->n_req * G * fact_row_floats(ctx->n_entries), s));
             ctx->st_launches += 2;
         } else if (pl->family == 3)
             CK(launch_attend_umma(pl->max_M, a, ctx->n_sms, ctx->d_err, s));

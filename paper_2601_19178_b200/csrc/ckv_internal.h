@@ -103,7 +103,9 @@ bool make_pool_tensor_maps(int head_dim, int64_t rows, const void* poolK, const 
 // or -1 if the shape is not supported.
 int fact_max_history(int dtype, int head_dim, int d_user, int n_entries, int mode);
 int fact_aux_floats();
-// a.items: one unsplit item per request with a query.  tw: [n_req][G][n_entries] floats, aux: [n_req][G][fact_aux_floats()].
+int fact_row_floats(int n_entries);
+// a.items: one unsplit item per request with a query.  tw: [n_req][G][fact_row_floats(n_entries)] floats,
+// aux: [n_req][G][fact_aux_floats()].
 cudaError_t launch_attend_fact(int head_dim, const AttendArgs& a, int n_req, int max_L, int n_sms, float* tw,
                                float* aux, cudaStream_t s);
 

@@ -58,45 +58,56 @@ __device__ __forceinline__ float bf16_bits_to_float(uint32_t b) { return __uint_
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 // ------------------------------------------------------------------------------------------------ T = P_k q
+// T / w rows in HBM are this many floats apart: 32-byte aligned rows, room for zero-filled bf16 pairs up to a
+// multiple of 8 entries
+__host__ __device__ __forceinline__ int row_floats(int n_entries) { return (n_entries + 7) & ~7; }
+
+constexpr int kTableMT = 4;  // 16-request tiles per warp: every pool row fetched serves 64 requests
+
 template <int D>
 __global__ void __launch_bounds__(128) fact_table_kernel(const AttendArgs a, int n_req, float* __restrict__ tw)
 {
-    constexpr int KS = D / 16;
+    constexpr int KS = D / 16, MT = kTableMT;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, gl = lane >> 2, t = lane & 3;
     const int m = a.cv.n_entries, G = a.cv.n_groups, grp = blockIdx.z;
-    const int j0 = blockIdx.x * 256 + warp * 64, r0 = blockIdx.y * 16;
+    const int j0 = blockIdx.x * 256 + warp * 64, r0 = blockIdx.y * (16 * MT);
     if (j0 >= m) return;
-    const int r_lo = r0 + gl, r_hi = r_lo + 8;
-    const bool v_lo = r_lo < n_req && a.reqs[r_lo].M > 0, v_hi = r_hi < n_req && a.reqs[r_hi].M > 0;
     // Which feature sits in which k-slot of the MMA is free as long as Q and the pool rows agree: a lane reads
     // D / 4 contiguous bytes of "its" rows, and k-step ks, slots (2t, 2t+1, 2t+8, 2t+9) hold features
     // (D / 4) t + 4 ks + (0, 1, 2, 3).
     constexpr int W = D / 8;  // 32-bit words per lane and row
     const uint16_t* Q = reinterpret_cast<const uint16_t*>(a.queries);
-    uint32_t q_lo[W], q_hi[W];
+    uint32_t qa[MT][KS][4];
+    bool v_lo[MT], v_hi[MT];
 #pragma unroll
-    for (int h = 0; h < W / 4; ++h) {
-        uint4 x = make_uint4(0, 0, 0, 0), y = x;
-        if (v_lo) x = __ldg(reinterpret_cast<const uint4*>(Q + ((int64_t)a.reqs[r_lo].q0 * G + grp) * D + 2 * W * t) + h);
-        if (v_hi) y = __ldg(reinterpret_cast<const uint4*>(Q + ((int64_t)a.reqs[r_hi].q0 * G + grp) * D + 2 * W * t) + h);
-        q_lo[4 * h] = x.x; q_lo[4 * h + 1] = x.y; q_lo[4 * h + 2] = x.z; q_lo[4 * h + 3] = x.w;
-        q_hi[4 * h] = y.x; q_hi[4 * h + 1] = y.y; q_hi[4 * h + 2] = y.z; q_hi[4 * h + 3] = y.w;
-    }
-    uint32_t qa[KS][4];
+    for (int mt = 0; mt < MT; ++mt) {
+        const int r_lo = r0 + 16 * mt + gl, r_hi = r_lo + 8;
+        v_lo[mt] = r_lo < n_req && a.reqs[r_lo].M > 0;
+        v_hi[mt] = r_hi < n_req && a.reqs[r_hi].M > 0;
+        uint32_t q_lo[W], q_hi[W];
 #pragma unroll
-    for (int ks = 0; ks < KS; ++ks) {
-        qa[ks][0] = q_lo[2 * ks];
-        qa[ks][1] = q_hi[2 * ks];
-        qa[ks][2] = q_lo[2 * ks + 1];
-        qa[ks][3] = q_hi[2 * ks + 1];
+        for (int h = 0; h < W / 4; ++h) {
+            uint4 x = make_uint4(0, 0, 0, 0), y = x;
+            if (v_lo[mt])
+                x = __ldg(reinterpret_cast<const uint4*>(Q + ((int64_t)a.reqs[r_lo].q0 * G + grp) * D + 2 * W * t) + h);
+            if (v_hi[mt])
+                y = __ldg(reinterpret_cast<const uint4*>(Q + ((int64_t)a.reqs[r_hi].q0 * G + grp) * D + 2 * W * t) + h);
+            q_lo[4 * h] = x.x; q_lo[4 * h + 1] = x.y; q_lo[4 * h + 2] = x.z; q_lo[4 * h + 3] = x.w;
+            q_hi[4 * h] = y.x; q_hi[4 * h + 1] = y.y; q_hi[4 * h + 2] = y.z; q_hi[4 * h + 3] = y.w;
+        }
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+            qa[mt][ks][0] = q_lo[2 * ks];
+            qa[mt][ks][1] = q_hi[2 * ks];
+            qa[mt][ks][2] = q_lo[2 * ks + 1];
+            qa[mt][ks][3] = q_hi[2 * ks + 1];
+        }
     }
     const uint16_t* P = reinterpret_cast<const uint16_t*>(a.cv.poolK) + (int64_t)grp * m * D;
-    float* t_lo = tw + ((int64_t)r_lo * G + grp) * m;
-    float* t_hi = tw + ((int64_t)r_hi * G + grp) * m;
-#pragma unroll 4
+    const int ms = row_floats(m);
+#pragma unroll 2
     for (int nt = 0; nt < 8; ++nt) {
         const int jb = j0 + 8 * nt + gl;  // pool entry whose row is this lane's B column
-        float c[4] = {0.f, 0.f, 0.f, 0.f};
         const uint4* row = reinterpret_cast<const uint4*>(P + (int64_t)(jb < m ? jb : m - 1) * D + 2 * W * t);
         uint32_t pw[W];
 #pragma unroll
@@ -104,21 +115,17 @@ __global__ void __launch_bounds__(128) fact_table_kernel(const AttendArgs a, int
             const uint4 x = __ldg(row + h);
             pw[4 * h] = x.x; pw[4 * h + 1] = x.y; pw[4 * h + 2] = x.z; pw[4 * h + 3] = x.w;
         }
-#pragma unroll
-        for (int ks = 0; ks < KS; ++ks) mma_bf16(c, qa[ks], pw[2 * ks], pw[2 * ks + 1]);
         const int jc = j0 + 8 * nt + 2 * t;  // columns of the accumulator fragment
-        if ((m & 1) == 0) {  // even rows: the two columns of a lane are one aligned 8-byte store
-            if (v_lo && jc < m) *reinterpret_cast<float2*>(t_lo + jc) = make_float2(c[0], c[1]);
-            if (v_hi && jc < m) *reinterpret_cast<float2*>(t_hi + jc) = make_float2(c[2], c[3]);
-        } else {
-            if (v_lo) {
-                if (jc < m) t_lo[jc] = c[0];
-                if (jc + 1 < m) t_lo[jc + 1] = c[1];
-            }
-            if (v_hi) {
-                if (jc < m) t_hi[jc] = c[2];
-                if (jc + 1 < m) t_hi[jc + 1] = c[3];
-            }
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+            float c[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int ks = 0; ks < KS; ++ks) mma_bf16(c, qa[mt][ks], pw[2 * ks], pw[2 * ks + 1]);
+            float* t_lo = tw + ((int64_t)(r0 + 16 * mt + gl) * G + grp) * ms;
+            float* t_hi = t_lo + (int64_t)8 * G * ms;
+            // the two columns of a lane are one aligned 8-byte store (a column past the last entry lands in the row's padding)
+            if (v_lo[mt] && jc < m) *reinterpret_cast<float2*>(t_lo + jc) = make_float2(c[0], c[1]);
+            if (v_hi[mt] && jc < m) *reinterpret_cast<float2*>(t_hi + jc) = make_float2(c[2], c[3]);
         }
     }
 }
@@ -227,7 +234,7 @@ __global__ void __launch_bounds__(kMainThreads, 1)
         r.unit0 = rq.base + (int64_t)r.grp * rq.Lpad;
         return r;
     };
-    auto table_row = [&](const Pair& pr) { return tw + ((int64_t)pr.req * G + pr.grp) * m; };
+    auto table_row = [&](const Pair& pr) { return tw + ((int64_t)pr.req * G + pr.grp) * row_floats(m); };
     auto fetch_table = [&](const Pair& pr, float* dstp) {  // all of the row in flight at once
         const float* row = table_row(pr);
         if ((m & 3) == 0) {
@@ -335,11 +342,11 @@ __global__ void __launch_bounds__(kMainThreads, 1)
             for (int q9 = 0; q9 < 9; ++q9) Sb[(tid >> 5) * 9 + q9] = vals[q9];
         }
         // w goes back to HBM rounded to bf16 (the precision the output product takes it in), two entries per word,
-        // over the head of the T row; an odd last entry is paired with a zero
+        // over the head of the T row, zero-filled up to a multiple of 8 entries
         {
             uint32_t* wrow = reinterpret_cast<uint32_t*>(table_row(cur));
-            for (int j2 = tid; 2 * j2 < m; j2 += kMainThreads)
-                wrow[j2] = pack_bf16(Ws[2 * j2], 2 * j2 + 1 < m ? Ws[2 * j2 + 1] : 0.f);
+            for (int j2 = tid; 2 * j2 < row_floats(m); j2 += kMainThreads)
+                wrow[j2] = pack_bf16(2 * j2 < m ? Ws[2 * j2] : 0.f, 2 * j2 + 1 < m ? Ws[2 * j2 + 1] : 0.f);
         }
         __syncthreads();
         if (tid < 9) {
@@ -358,10 +365,12 @@ __global__ void __launch_bounds__(kMainThreads, 1)
 // ------------------------------------------------------------------------------------------------ out = w P_v
 // One CTA per (16 requests, group); warp w covers pool entries [w, w + 1) * ceil32(m / 16).  P_v rows are
 // contiguous here: 32-row tiles through a two-slot cp.async ring per warp, fragments by transposing ldmatrix.
+// 16-byte chunk c of tile row r sits at chunk c ^ swz(r).  The eight rows of one ldmatrix block are rows
+// 8 t' + const + e (t' < 4, e < 2) here, see the k-slot order below: they must fall into eight different bank groups.
 template <int D>
 __device__ __forceinline__ int swz(int r)
 {
-    return D == 64 ? (r & 7) : ((r >> 1) & 3);
+    return D == 64 ? ((((r >> 3) & 3) << 1) | (r & 1)) : ((r >> 3) & 3);
 }
 
 template <int D>
@@ -376,15 +385,21 @@ __global__ void __launch_bounds__(kOutWarps * 32, 1)
     const int jbeg = warp * span, jend = min(m, jbeg + span);
     const int r_lo = r0 + gl, r_hi = r_lo + 8;
     const bool v_lo = r_lo < n_req && a.reqs[r_lo].M > 0, v_hi = r_hi < n_req && a.reqs[r_hi].M > 0;
-    const float* w_lo = tw + ((int64_t)(v_lo ? r_lo : 0) * G + grp) * m;
-    const float* w_hi = tw + ((int64_t)(v_hi ? r_hi : 0) * G + grp) * m;
+    const float* w_lo = tw + ((int64_t)(v_lo ? r_lo : 0) * G + grp) * row_floats(m);
+    const float* w_hi = tw + ((int64_t)(v_hi ? r_hi : 0) * G + grp) * row_floats(m);
     const char* pV = reinterpret_cast<const char*>(a.cv.poolV) + (int64_t)grp * m * ROWB;
     const uint32_t ring = smem_u32(osm) + warp * (2 * TILE_B);
     const int cr = lane / CPR, cc = lane % CPR, lr = lane & 7, lm = lane >> 3;
-    uint32_t offV[NTD / 2];
+    // Which pool entry sits in which k-slot is free as long as w and the V rows agree: a lane reads 8 consecutive
+    // weights of its two requests with one 16-byte load each, and k-step b, slots (2t, 2t+1, 2t+8, 2t+9) hold
+    // entries 8t + 4b + (0, 1, 2, 3) of the 32-entry chunk; the ldmatrix row addresses follow.
+    uint32_t offV[2][NTD / 2];
 #pragma unroll
-    for (int jp = 0; jp < NTD / 2; ++jp)
-        offV[jp] = ((lm & 1) * 8 + lr) * ROWB + (((2 * jp + (lm >> 1)) ^ swz<D>(lr)) << 4);
+    for (int b = 0; b < 2; ++b) {
+        const int r = 8 * (lr >> 1) + 4 * b + 2 * (lm & 1) + (lr & 1);  // chunk row of matrix row lr, matrix half lm & 1
+#pragma unroll
+        for (int jp = 0; jp < NTD / 2; ++jp) offV[b][jp] = r * ROWB + (((2 * jp + (lm >> 1)) ^ swz<D>(r)) << 4);
+    }
 
     auto issue = [&](int jc, int slot) {  // rows jc .. jc+31 of the V pool (clamped: their weights are zero)
 #pragma unroll
@@ -397,25 +412,22 @@ __global__ void __launch_bounds__(kOutWarps * 32, 1)
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
     };
-    // weights of one 32-entry chunk as A fragments: k-step b, registers (row lo, row hi) x (cols 2t.., cols 2t+8..);
-    // a register is the bf16 pair the main kernel stored
-    auto load_w = [&](int jc, uint32_t (&x)[8]) {
-#pragma unroll
-        for (int b = 0; b < 2; ++b)
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const int j = jc + 16 * b + 8 * h + 2 * t;  // even; the pair (j, j + 1) ends inside this warp's span
-                const bool in = j < jend;
-                x[4 * b + 2 * h] = (in && v_lo) ? __ldg(reinterpret_cast<const uint32_t*>(w_lo) + (j >> 1)) : 0u;
-                x[4 * b + 2 * h + 1] = (in && v_hi) ? __ldg(reinterpret_cast<const uint32_t*>(w_hi) + (j >> 1)) : 0u;
-            }
+    // weights of one 32-entry chunk: entries 8t .. 8t+7 of both requests, the bf16 pairs the main kernel stored
+    // (rows start at multiples of 32 bytes and are zero-filled behind the last entry up to a multiple of 8 entries)
+    auto load_w = [&](int jc, uint4 (&x)[2]) {
+        const int j = jc + 8 * t;
+        const bool in = j < jend;
+        x[0] = (in && v_lo) ? __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const uint32_t*>(w_lo) + (j >> 1)))
+                            : make_uint4(0, 0, 0, 0);
+        x[1] = (in && v_hi) ? __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const uint32_t*>(w_hi) + (j >> 1)))
+                            : make_uint4(0, 0, 0, 0);
     };
 
     float o[NTD][4];
 #pragma unroll
     for (int j = 0; j < NTD; ++j) o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f;
     const int nch = jbeg < jend ? (jend - jbeg + 31) / 32 : 0;
-    uint32_t wa[8], wb[8];
+    uint4 wa[2], wb[2];
     if (nch > 0) {
         issue(jbeg, 0);
         load_w(jbeg, wa);
@@ -433,13 +445,14 @@ __global__ void __launch_bounds__(kOutWarps * 32, 1)
         const uint32_t vt = ring + (c & 1) * TILE_B;
 #pragma unroll
         for (int b = 0; b < 2; ++b) {
-            const uint32_t pa[4] = {wa[4 * b], wa[4 * b + 1], wa[4 * b + 2], wa[4 * b + 3]};
+            const uint32_t pa[4] = {b ? wa[0].z : wa[0].x, b ? wa[1].z : wa[1].x, b ? wa[0].w : wa[0].y,
+                                    b ? wa[1].w : wa[1].y};
 #pragma unroll
             for (int jp = 0; jp < NTD / 2; ++jp) {
                 uint32_t v0, v1, v2, v3;
                 asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
                              : "=r"(v0), "=r"(v1), "=r"(v2), "=r"(v3)
-                             : "r"(vt + b * (16 * ROWB) + offV[jp])
+                             : "r"(vt + offV[b][jp])
                              : "memory");
                 mma_bf16(o[2 * jp], pa, v0, v1);
                 mma_bf16(o[2 * jp + 1], pa, v2, v3);
@@ -447,7 +460,7 @@ __global__ void __launch_bounds__(kOutWarps * 32, 1)
         }
         __syncwarp();  // every lane is done reading the slot that the next iteration refills
 #pragma unroll
-        for (int i = 0; i < 8; ++i) wa[i] = wb[i];
+        for (int i = 0; i < 2; ++i) wa[i] = wb[i];
     }
 
     // sum the warps' partial outputs in fixed order, add the user part, normalise, store
@@ -490,7 +503,8 @@ cudaError_t launch_fact(const AttendArgs& a, int n_req, int max_L, int n_sms, fl
 {
     const int m = a.cv.n_entries, G = a.cv.n_groups;
     const bool i16 = a.cv.idx_bytes == 2, soft = a.mode == CKV_SOFTMAX;
-    fact_table_kernel<D><<<dim3((m + 255) / 256, (n_req + 15) / 16, G), 128, 0, s>>>(a, n_req, tw);
+    fact_table_kernel<D><<<dim3((m + 255) / 256, (n_req + 16 * kTableMT - 1) / (16 * kTableMT), G), 128, 0, s>>>(
+        a, n_req, tw);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     const int s_cap = std::max((max_L + 31) / 32 * 32, 9 * (kMainThreads / 32));  // scores; later the warps' sums
@@ -531,8 +545,9 @@ int fact_max_history(int dtype, int head_dim, int d_user, int n_entries, int mod
 }
 
 int fact_aux_floats() { return kAux; }
+int fact_row_floats(int n_entries) { return row_floats(n_entries); }
 
-// Three launches; a.items holds one unsplit item per request with a query; tw: [n_req][G][n_entries] floats,
+// Three launches; a.items holds one unsplit item per request with a query; tw: [n_req][G][fact_row_floats()] floats,
 // aux: [n_req][G][fact_aux_floats()] floats.
 cudaError_t launch_attend_fact(int D, const AttendArgs& a, int n_req, int max_L, int n_sms, float* tw, float* aux,
                                cudaStream_t s)

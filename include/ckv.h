@@ -187,6 +187,18 @@ CKV_API ckv_status ckv_attend_static(ckv_ctx* ctx, int32_t n, const int64_t* use
 CKV_API ckv_status ckv_materialize(ckv_ctx* ctx, int64_t user, void* K_out, void* V_out, void* stream);
 
 /*
+ * Appends L_new positions (new interactions) behind a cached user's history; arguments as for
+ * ckv_cache_put, describing only the new positions.  The user's compressed cache moves to fresh
+ * storage holding the old and the new positions (storage is only reclaimed by ckv_cache_clear or
+ * when the last user is evicted).  Synchronises `stream`.
+ * Errors: INVALID_ARG, STATE (no pool), SHAPE (d_user), UNKNOWN_USER, INDEX_RANGE (an index
+ * outside [0, n_entries); the user keeps the old history), OOM, CUDA.
+ */
+CKV_API ckv_status ckv_cache_append(ckv_ctx* ctx, int64_t user, int32_t L_new, const int32_t* idx_K,
+                                    const int32_t* idx_V, const void* user_K, const void* user_V, int32_t d_user,
+                                    void* stream);
+
+/*
  * Decode-stage load path (Sec. 4.4: T_load(s d_u + s) + T_index): a serving system keeps the
  * compressed caches in host memory and loads the users of a request batch before attending.
  * A blob is the packed form of n users' caches exactly as the library stores them, so loading it

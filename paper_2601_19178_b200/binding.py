@@ -23,7 +23,7 @@ CKV_SOFTMAX, CKV_SILU_OVER_L = 0, 1
 EXPORTS = (
     "ckv_create", "ckv_destroy", "ckv_pool_load", "ckv_cache_put", "ckv_cache_put_batch",
     "ckv_cache_evict", "ckv_cache_clear", "ckv_attend", "ckv_attend_static", "ckv_materialize",
-    "ckv_user_length", "ckv_cache_blob_bytes", "ckv_cache_export", "ckv_cache_import",
+    "ckv_user_length", "ckv_cache_append", "ckv_cache_blob_bytes", "ckv_cache_export", "ckv_cache_import",
     "ckv_cache_bytes", "ckv_set_option", "ckv_get_option", "ckv_last_stat", "ckv_strerror",
     "ckv_last_cuda_error", "ckv_version",
 )
@@ -56,6 +56,7 @@ def _load() -> ctypes.CDLL:
         "ckv_pool_load": (i32, [vp, vp, vp, i32, i32, vp]),
         "ckv_cache_put": (i32, [vp, i64, i32, vp, vp, vp, vp, i32, vp]),
         "ckv_cache_put_batch": (i32, [vp, i32, vp, vp, vp, vp, vp, vp, i32, vp]),
+        "ckv_cache_append": (i32, [vp, i64, i32, vp, vp, vp, vp, i32, vp]),
         "ckv_cache_evict": (i32, [vp, i64]),
         "ckv_cache_clear": (i32, [vp]),
         "ckv_attend": (i32, [vp, i32, vp, vp, vp, vp, vp]),
@@ -151,6 +152,11 @@ def ckv_cache_put_batch(ctx, users, hist_off, idx_K, idx_V, user_K, user_V, d_us
     _check(ctx, lib.ckv_cache_put_batch(ctx, users.shape[0], users.ctypes.data, hist_off.ctypes.data,
                                         _ptr(idx_K), _ptr(idx_V), _ptr(user_K), _ptr(user_V), d_user,
                                         _stream(stream)), "ckv_cache_put_batch")
+
+
+def ckv_cache_append(ctx, user: int, L_new: int, idx_K, idx_V, user_K, user_V, d_user: int, stream=None) -> None:
+    _check(ctx, lib.ckv_cache_append(ctx, int(user), int(L_new), _ptr(idx_K), _ptr(idx_V), _ptr(user_K),
+                                     _ptr(user_V), d_user, _stream(stream)), "ckv_cache_append")
 
 
 def ckv_cache_evict(ctx, user: int) -> None:

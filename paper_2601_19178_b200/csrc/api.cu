@@ -577,6 +577,47 @@ ckv_status ckv_cache_put(ckv_ctx* ctx, int64_t user, int32_t L, const int32_t* i
     return ckv_cache_put_batch(ctx, 1, &user, off, idx_K, idx_V, user_K, user_V, d_user, stream);
 }
 
+ckv_status ckv_cache_append(ckv_ctx* ctx, int64_t user, int32_t L_new, const int32_t* idx_K, const int32_t* idx_V,
+                            const void* user_K, const void* user_V, int32_t d_user, void* stream)
+{
+    if (!ctx || L_new < 0) return CKV_ERR_INVALID_ARG;
+    if (!ctx->pool) return CKV_ERR_STATE;
+    if (d_user != ctx->d_user) return CKV_ERR_SHAPE;
+    auto f = ctx->users.find(user);
+    if (f == ctx->users.end()) return CKV_ERR_UNKNOWN_USER;
+    if (L_new == 0) return CKV_OK;
+    if (!idx_K || !idx_V || (d_user > 0 && (!user_K || !user_V))) return CKV_ERR_INVALID_ARG;
+    const UserEntry old = f->second;
+    if ((int64_t)old.L + L_new > INT32_MAX - 32) return CKV_ERR_INVALID_ARG;
+    const int G = ctx->cfg.n_groups;
+    const int32_t L_tot = old.L + L_new, Lpad_tot = (L_tot + 31) / 32 * 32;
+    const int64_t units = (int64_t)G * Lpad_tot;
+    DeviceGuard dg(ctx->cfg.device);
+    cudaStream_t s = (cudaStream_t)stream;
+    Staged sik, siv, suk, suv;
+    const size_t ib = (size_t)L_new * G * sizeof(int32_t), ubytes = (size_t)L_new * G * d_user * ctx->elem;
+    CK(sik.init(idx_K, ib, s));
+    if (idx_V == idx_K) siv.dev = sik.dev; else CK(siv.init(idx_V, ib, s));
+    CK(suk.init(user_K, ubytes, s));
+    CK(suv.init(user_V, ubytes, s));
+    // the longer history takes fresh units behind what is stored (the arena only grows until it is cleared)
+    ckv_status st = ensure_arena(ctx, units, s);
+    if (st != CKV_OK) return st;
+    CK(cudaMemsetAsync(ctx->d_flag, 0, sizeof(int), s));
+    CK(launch_append(ctx->cfg.dtype, G, ctx->n_entries, d_user, ctx->idx_bytes, old.base, old.L, old.Lpad,
+                     ctx->used_units, L_new, Lpad_tot, (const int32_t*)sik.dev, (const int32_t*)siv.dev, suk.dev,
+                     suv.dev, ctx->a_idxK, ctx->a_idxV, ctx->a_userK, ctx->a_userV, ctx->d_flag, s));
+    int bad = 0;
+    CK(cudaMemcpyAsync(&bad, ctx->d_flag, sizeof(int), cudaMemcpyDeviceToHost, s));
+    CK(cudaStreamSynchronize(s));
+    if (bad) return CKV_ERR_INDEX_RANGE;  // used_units not advanced: the user keeps the old history
+    f->second = UserEntry{ctx->used_units, L_tot, Lpad_tot};
+    ctx->live_positions += L_new;
+    ctx->used_units += units;
+    ctx->generation++;
+    return CKV_OK;
+}
+
 namespace {
 
 // Section offsets of a blob holding `total_units` units: K indices, V indices, user K, user V, end.

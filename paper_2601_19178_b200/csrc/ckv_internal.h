@@ -76,6 +76,12 @@ cudaError_t launch_pack(int dtype, int G, int n_entries, int d_user, int idx_byt
                         int64_t total_units, int64_t arena_base, const int32_t* idxK,
                         const int32_t* idxV, const void* userK, const void* userV, void* a_idxK,
                         void* a_idxV, void* a_userK, void* a_userV, int* bad_flag, cudaStream_t s);
+// Writes a user's units for L_old + L_new positions at arena unit dst_base: the first L_old positions copied from
+// the units at old_base (same arena), the rest packed from the new [L_new][G] indices and [L_new][G][d_user] parts.
+cudaError_t launch_append(int dtype, int G, int n_entries, int d_user, int idx_bytes, int64_t old_base, int L_old,
+                          int Lpad_old, int64_t dst_base, int L_new, int Lpad_tot, const int32_t* idxK,
+                          const int32_t* idxV, const void* userK, const void* userV, void* a_idxK, void* a_idxV,
+                          void* a_userK, void* a_userV, int* bad_flag, cudaStream_t s);
 cudaError_t launch_materialize(int dtype, int D, const CacheView& cv, int64_t base, int L, int Lpad,
                                void* K_out, void* V_out, cudaStream_t s);
 

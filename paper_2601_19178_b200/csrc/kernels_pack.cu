@@ -71,6 +71,52 @@ __global__ void pack_kernel(int G, int n_entries, int d_user, int n_users,
     }
 }
 
+// Append: units of one user with L_old + L_new positions at arena unit `dst_base`; position i < L_old is copied
+// from the user's old units, the rest comes from the new [L_new][G] inputs (range-checked like pack_kernel).
+template <typename E, typename I>
+__global__ void append_kernel(int G, int n_entries, int d_user, int64_t old_base, int L_old, int Lpad_old,
+                              int64_t dst_base, int L_new, int Lpad_tot, const int32_t* __restrict__ idxK,
+                              const int32_t* __restrict__ idxV, const E* __restrict__ userK,
+                              const E* __restrict__ userV, I* a_idxK, I* a_idxV, E* a_userK, E* a_userV,
+                              int* __restrict__ bad_flag)
+{
+    const int64_t total = (int64_t)G * Lpad_tot;
+    for (int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; t < total; t += (int64_t)gridDim.x * blockDim.x) {
+        const int g = (int)(t / Lpad_tot);
+        const int i = (int)(t - (int64_t)g * Lpad_tot);
+        const int64_t dst = dst_base + t;
+        if (i < L_old) {
+            const int64_t src = old_base + (int64_t)g * Lpad_old + i;
+            a_idxK[dst] = a_idxK[src];
+            a_idxV[dst] = a_idxV[src];
+            for (int c = 0; c < d_user; ++c) {
+                a_userK[dst * d_user + c] = a_userK[src * d_user + c];
+                a_userV[dst * d_user + c] = a_userV[src * d_user + c];
+            }
+        } else if (i < L_old + L_new) {
+            const int64_t src = (int64_t)(i - L_old) * G + g;
+            int32_t ik = idxK[src], iv = idxV[src];
+            if (ik < 0 || ik >= n_entries || iv < 0 || iv >= n_entries) {
+                atomicOr(bad_flag, 1);
+                ik = iv = 0;
+            }
+            a_idxK[dst] = (I)ik;
+            a_idxV[dst] = (I)iv;
+            for (int c = 0; c < d_user; ++c) {
+                a_userK[dst * d_user + c] = userK[src * d_user + c];
+                a_userV[dst * d_user + c] = userV[src * d_user + c];
+            }
+        } else {  // padding: a valid row index and a zero user part
+            a_idxK[dst] = (I)0;
+            a_idxV[dst] = (I)0;
+            for (int c = 0; c < d_user; ++c) {
+                a_userK[dst * d_user + c] = E(0);
+                a_userV[dst * d_user + c] = E(0);
+            }
+        }
+    }
+}
+
 template <typename E, typename I>
 __global__ void materialize_kernel(int G, int n_entries, int d_user, int D,
                                    const E* __restrict__ poolK, const E* __restrict__ poolV,
@@ -151,6 +197,27 @@ cudaError_t launch_pack(int dtype, int G, int n_entries, int d_user, int idx_byt
         if (idx_bytes == 2) CKV_PACK(uint32_t, uint16_t); else CKV_PACK(uint32_t, int32_t);
     }
 #undef CKV_PACK
+    return cudaGetLastError();
+}
+
+cudaError_t launch_append(int dtype, int G, int n_entries, int d_user, int idx_bytes, int64_t old_base, int L_old,
+                          int Lpad_old, int64_t dst_base, int L_new, int Lpad_tot, const int32_t* idxK,
+                          const int32_t* idxV, const void* userK, const void* userV, void* a_idxK, void* a_idxV,
+                          void* a_userK, void* a_userV, int* bad_flag, cudaStream_t s)
+{
+    const int64_t total = (int64_t)G * Lpad_tot;
+    if (total == 0) return cudaSuccess;
+    const int grid = grid_for(total, 256);
+#define CKV_APPEND(E, I)                                                                                       \
+    append_kernel<E, I><<<grid, 256, 0, s>>>(G, n_entries, d_user, old_base, L_old, Lpad_old, dst_base, L_new, \
+                                             Lpad_tot, idxK, idxV, (const E*)userK, (const E*)userV,          \
+                                             (I*)a_idxK, (I*)a_idxV, (E*)a_userK, (E*)a_userV, bad_flag)
+    if (dtype == CKV_BF16) {
+        if (idx_bytes == 2) CKV_APPEND(uint16_t, uint16_t); else CKV_APPEND(uint16_t, int32_t);
+    } else {
+        if (idx_bytes == 2) CKV_APPEND(uint32_t, uint16_t); else CKV_APPEND(uint32_t, int32_t);
+    }
+#undef CKV_APPEND
     return cudaGetLastError();
 }
 

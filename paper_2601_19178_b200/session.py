@@ -45,6 +45,10 @@ class CollectiveKV:
     def cache_put(self, user: int, idx_K, idx_V, user_K, user_V):
         B.ckv_cache_put(self.ctx, user, idx_K.shape[0], idx_K, idx_V, user_K, user_V, self.d_user)
 
+    def cache_append(self, user: int, idx_K, idx_V, user_K, user_V):
+        """New interactions behind a cached user's history (arguments describe the new positions only)."""
+        B.ckv_cache_append(self.ctx, user, idx_K.shape[0], idx_K, idx_V, user_K, user_V, self.d_user)
+
     def cache_put_batch(self, users, hist_off, idx_K, idx_V, user_K, user_V):
         B.ckv_cache_put_batch(self.ctx, users, hist_off, idx_K, idx_V, user_K, user_V, self.d_user)
 

@@ -110,3 +110,53 @@ def test_import_rejects_bad_blobs_and_leaves_the_cache_unchanged():
     # the original users are untouched
     assert_close(gpu_attend(w, d, session=s), oracle_attend(w, d), w.dtype, "after rejected import")
     s.close()
+
+
+@pytest.mark.parametrize("name", ["cfg1", "cfg4", "cfg5"])
+def test_append_equals_put_of_the_whole_history(name):
+    """New interactions appended in two steps: the packed cache and the attention output must be the bits that
+    a single put of the whole history gives."""
+    import paper_2601_19178_b200 as ckv
+    w = synth.scaled(CASES[name], hist_len=(40, 200))
+    d = synth.generate(w)
+    ref = make_session(w, d)
+    want_out = gpu_attend(w, d, session=ref)
+    want_blob = ref.export_blob(d["users"]).numpy().tobytes()
+    ref.close()
+
+    dt = torch.float32 if w.dtype == "f32" else torch.bfloat16
+    s = ckv.CollectiveKV(w.n_groups, w.head_dim, dt, w.mode)
+    s.pool_load(to_dev(d["pool_K"], w.dtype), to_dev(d["pool_V"], w.dtype))
+    ho = d["hist_off"]
+    cuts = [(3, 30), (0, 17), (39, 1)]                           # (first put, first append) positions; rest in the second append
+    for u in range(w.n_users):
+        a, b = int(ho[u]), int(ho[u + 1])
+        n0, n1 = cuts[u % len(cuts)]
+        c0, c1 = a + n0, a + n0 + n1
+        sl = lambda lo, hi: (to_dev(d["idx_K"][lo:hi], "i"), to_dev(d["idx_V"][lo:hi], "i"),
+                             to_dev(d["user_K"][lo:hi], w.dtype), to_dev(d["user_V"][lo:hi], w.dtype))
+        s.cache_put(int(d["users"][u]), *sl(a, c0))
+        s.cache_append(int(d["users"][u]), *sl(c0, c1))
+        # host inputs for the second append
+        ckv.ckv_cache_append(s.ctx, int(d["users"][u]), b - c1, np.ascontiguousarray(d["idx_K"][c1:b]),
+                             np.ascontiguousarray(d["idx_V"][c1:b]), np.ascontiguousarray(d["user_K"][c1:b]),
+                             np.ascontiguousarray(d["user_V"][c1:b]), w.d_user)
+        assert ckv.ckv_user_length(s.ctx, int(d["users"][u])) == b - a
+    assert s.export_blob(d["users"]).numpy().tobytes() == want_blob
+    assert np.array_equal(gpu_attend(w, d, session=s), want_out)
+    comp, _ = ckv.ckv_cache_bytes(s.ctx)
+    assert comp == int(ho[-1]) * w.n_groups * (2 * 2 + 2 * w.d_user * (4 if w.dtype == "f32" else 2))
+    # error paths: unknown user, index out of range (the user keeps the old history)
+    u0 = int(d["users"][0])
+    one = (np.zeros((1, w.n_groups), np.int32), np.zeros((1, w.n_groups), np.int32),
+           np.zeros((1, w.n_groups, w.d_user), d["user_K"].dtype), np.zeros((1, w.n_groups, w.d_user), d["user_K"].dtype))
+    with pytest.raises(ckv.CkvError) as e:
+        ckv.ckv_cache_append(s.ctx, 424242, 1, *one, w.d_user)
+    assert e.value.status == ckv.CKV_ERR_UNKNOWN_USER
+    bad = (np.full((1, w.n_groups), w.n_entries, np.int32),) + one[1:]
+    with pytest.raises(ckv.CkvError) as e:
+        ckv.ckv_cache_append(s.ctx, u0, 1, *bad, w.d_user)
+    assert e.value.status == ckv.CKV_ERR_INDEX_RANGE
+    assert ckv.ckv_user_length(s.ctx, u0) == int(ho[1] - ho[0])
+    assert np.array_equal(gpu_attend(w, d, session=s), want_out)
+    s.close()

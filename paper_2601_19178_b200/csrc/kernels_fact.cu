@@ -492,10 +492,14 @@ __global__ void __launch_bounds__(kOutWarps * 32, 1)
     }
 }
 
+// Opt-in to large dynamic shared memory, once per kernel (the most a CTA can have on this architecture).
 template <typename K>
-cudaError_t set_smem(K kernel, size_t bytes)
+cudaError_t set_smem(K kernel, bool& done)
 {
-    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (done) return cudaSuccess;
+    const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    done = e == cudaSuccess;
+    return e;
 }
 
 template <int D>
@@ -513,7 +517,8 @@ cudaError_t launch_fact(const AttendArgs& a, int n_req, int max_L, int n_sms, fl
     const dim3 grid(n_pairs < n_sms ? n_pairs : n_sms);
 #define CKV_FACT_MAIN(MODE, I16)                                                       \
     do {                                                                               \
-        e = set_smem(fact_main_kernel<D, MODE, I16>, smem_main);                       \
+        static bool done_main = false;                                                 \
+        e = set_smem(fact_main_kernel<D, MODE, I16>, done_main);                       \
         if (e != cudaSuccess) return e;                                                \
         fact_main_kernel<D, MODE, I16><<<grid, kMainThreads, smem_main, s>>>(a, tw, aux, s_cap); \
     } while (0)
@@ -526,7 +531,8 @@ cudaError_t launch_fact(const AttendArgs& a, int n_req, int max_L, int n_sms, fl
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     const size_t smem_out = std::max((size_t)kOutWarps * 2 * 32 * D * 2, (size_t)kOutWarps * 16 * D * sizeof(float));
-    e = set_smem(fact_out_kernel<D>, smem_out);
+    static bool done_out = false;
+    e = set_smem(fact_out_kernel<D>, done_out);
     if (e != cudaSuccess) return e;
     fact_out_kernel<D><<<dim3((n_req + 15) / 16, G), kOutWarps * 32, smem_out, s>>>(a, n_req, tw, aux);
     return cudaGetLastError();

@@ -320,6 +320,32 @@ def test_full_size_workloads_on_sampled_users(name):
     assert_close(got, oracle_attend(w, d, sel=sel), w.dtype, name)
 
 
+@pytest.mark.parametrize("seed", range(40))
+def test_random_shapes_against_the_oracle(seed):
+    """Seeded random workloads across head widths, user-part widths, pool sizes, ragged lengths (zero included),
+    query counts and both normalisations: whatever kernel the library picks must match the oracle."""
+    rng = np.random.default_rng(1000 + seed)
+    dtype = "f32" if seed % 5 == 0 else "bf16"
+    D = int(rng.choice([16, 32, 32, 64, 64, 128]))
+    du = int(rng.choice([0, 1, 2, 3, 4, 8, 12]))
+    du = min(du, D - 4)
+    m = int(rng.choice([1, 7, 100, 333, 2048, 5000]))
+    G = int(rng.integers(1, 5))
+    n_users = int(rng.integers(1, 9))
+    Lmax = int(rng.choice([1, 40, 300, 1500]))
+    M = int(rng.choice([1, 1, 2, 9, 33, 50, 130]))
+    mode = "softmax" if rng.integers(0, 2) else "silu_over_l"
+    zipf = None if rng.integers(0, 2) else 1.1
+    w = synth.Workload(f"rnd{seed}", G, D - du, du, m, n_users, (0, Lmax), M, mode, dtype, zipf, 1.0 / D, 1.0 / D, 500 + seed)
+    d = synth.generate(w)
+    s = make_session(w, d)
+    got = gpu_attend(w, d, session=s)
+    fam = s.stat("kernel")
+    assert s.stat("device_errors") == 0
+    s.close()
+    assert_close(got, oracle_attend(w, d), dtype, f"seed {seed}: D={D} du={du} m={m} G={G} M={M} {mode} family {fam}")
+
+
 def test_host_buffers_go_through_the_same_path():
     w = SMALL["cfg5_ragged"]
     d = synth.generate(w)

@@ -449,8 +449,10 @@ def run_load_path(args, w):
         row = {"batch": b, "positions": positions, "full_kv_bytes": full_bytes, "packed_bytes": blob.numel(),
                "kv_cache_load_ms": med_ms(load_full), "ckv_import_ms": med_ms(load_packed),
                "ckv_import_attend_ms": med_ms(load_and_attend)}
-        # same users, same request shape: the resident cache must give the same bits
-        ok = ok and bool(torch.equal(out[:nq], src.attend(users, q_off, q[:nq])))
+        # same users, same request shape: the resident cache gives the same result (the same bits from the
+        # gathering kernels; the factorised path sums its histogram with atomics: up to a bf16 ulp apart)
+        ref = src.attend(users, q_off, q[:nq]).float()
+        ok = ok and bool((out[:nq].float() - ref).abs().max() <= 2.0 ** -7 * ref.abs().max())
         rows.append(row)
     dst.close()
     src.close()

@@ -285,8 +285,7 @@ ckv_status build_plan(ckv_ctx* ctx, Plan& pl, int32_t n, const int64_t* users, c
     // of the pool's entries for 64-wide heads (the gathering kernel costs half as much per position at 32).
     // (its tables take n_entries floats per request and group: not beyond 2 GiB of workspace)
     const bool can_fact = all_single && n_active > 0 &&
-                          fact_max_history(ctx->cfg.dtype, ctx->cfg.head_dim, ctx->d_user, ctx->n_entries,
-                                           ctx->cfg.mode) >= max_L &&
+                          fact_max_history(ctx->cfg.dtype, ctx->cfg.head_dim, ctx->d_user, ctx->n_entries) >= max_L &&
                           (int64_t)n * ctx->cfg.n_groups * (fact_row_floats(ctx->n_entries) + fact_aux_floats()) *
                                   (int64_t)sizeof(float) <= ((int64_t)2 << 30);
     const int64_t fact_ratio = ctx->cfg.head_dim == 64 ? 4 : 2;

@@ -107,7 +107,7 @@ bool make_pool_tensor_maps(int head_dim, int64_t rows, const void* poolK, const 
 // ---- kernels_fact.cu : pool-side factorisation for one query per user (bf16, head_dim 32 or 64, d_user <= 8)
 // Largest history the family can take for this shape (its tables and scores share one CTA's shared memory),
 // or -1 if the shape is not supported.
-int fact_max_history(int dtype, int head_dim, int d_user, int n_entries, int mode);
+int fact_max_history(int dtype, int head_dim, int d_user, int n_entries);
 int fact_aux_floats();
 int fact_row_floats(int n_entries);
 // a.items: one unsplit item per request with a query.  tw: [n_req][G][fact_row_floats(n_entries)] floats,

@@ -541,10 +541,9 @@ cudaError_t launch_fact(const AttendArgs& a, int n_req, int max_L, int n_sms, fl
 }  // namespace
 
 // Largest history (positions) the main kernel can hold next to its two tables, or -1 if the shape is not supported.
-int fact_max_history(int dtype, int head_dim, int d_user, int n_entries, int mode)
+int fact_max_history(int dtype, int head_dim, int d_user, int n_entries)
 {
     if (dtype != CKV_BF16 || (head_dim != 32 && head_dim != 64) || d_user > 8) return -1;
-    (void)mode;
     const int64_t floats = 220 * 1024 / 4 - 32 - 2 * (int64_t)n_entries;  // two table buffers + one score per position
     if (floats < 9 * (kMainThreads / 32)) return -1;
     return (int)(floats / 32 * 32);

@@ -280,20 +280,29 @@ ckv_status build_plan(ckv_ctx* ctx, Plan& pl, int32_t n, const int64_t* users, c
     const bool can_mma = ctx->has_mma;
     // tcgen05 from three 16-query blocks on, else the warp-level tensor-core kernel (faster than the CUDA-core
     // kernel from a single query on); the CUDA-core kernel serves what neither supports
-    // One query per user and histories long against the pool: the pool-side factorisation trades the row gathers
-    // for two tables per (user, group) in HBM.  Break-even measured on B200 at a mean length of about a quarter
-    // of the pool's entries for 64-wide heads (the gathering kernel costs half as much per position at 32).
-    // (its tables take n_entries floats per request and group: not beyond 2 GiB of workspace)
+    // One query per user: the pool-side factorisation trades the row gathers for two tables per (user, group) in
+    // HBM (n_entries floats per request and group: not beyond 2 GiB of workspace).
     const bool can_fact = all_single && n_active > 0 &&
                           fact_max_history(ctx->cfg.dtype, ctx->cfg.head_dim, ctx->d_user, ctx->n_entries) >= max_L &&
                           (int64_t)n * ctx->cfg.n_groups * (fact_row_floats(ctx->n_entries) + fact_aux_floats()) *
                                   (int64_t)sizeof(float) <= ((int64_t)2 << 30);
-    const int64_t fact_ratio = ctx->cfg.head_dim == 64 ? 4 : 2;
+    // It pays when histories are long against the pool and there are enough (user, group) pairs to fill the SMs
+    // (one CTA holds a whole pair; the gathering kernel splits long histories over CTAs).  Cost lines fitted to
+    // B200 measurements, in microseconds of one SM: a pair costs a + b n_entries + c L on the factorised path,
+    // a position d on the gathering path.
+    bool fact_pays = false;
+    if (can_fact) {
+        const bool wide = ctx->cfg.head_dim == 64;
+        const double a = wide ? 4.8 : 4.7, b = wide ? 0.00032 : 0.00024, c = wide ? 0.0010 : 0.0008,
+                     d = wide ? 0.0047 : 0.0025;
+        const double pairs = (double)n_active * ctx->cfg.n_groups, mean_L = (double)total_pos / (double)n_active;
+        const double waves = std::ceil(pairs / ctx->n_sms);
+        const double t_fact = waves * (a + b * ctx->n_entries + c * mean_L);
+        const double t_gather = d * (double)total_pos * ctx->cfg.n_groups / ctx->n_sms;
+        fact_pays = t_fact < t_gather;
+    }
     if (ctx->opt_kernel == 0)
-        pl.family = ctx->has_umma && max_M >= 48                               ? 3
-                    : can_fact && total_pos * fact_ratio >= n_active * ctx->n_entries ? 4
-                    : can_mma                                                  ? 2
-                                                                               : 1;
+        pl.family = ctx->has_umma && max_M >= 48 ? 3 : fact_pays ? 4 : can_mma ? 2 : 1;
     else if (ctx->opt_kernel == 4 && can_fact) pl.family = 4;
     else if (ctx->opt_kernel == 1) pl.family = 1;
     else if (ctx->opt_kernel == 2 && can_mma) pl.family = 2;

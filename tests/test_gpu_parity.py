@@ -252,16 +252,21 @@ def test_pool_side_factorisation_matches_oracle(mode, head):
     assert np.abs(got - other).max() <= 2.0 ** -7 * np.abs(want).max()
 
 
-def test_pool_side_factorisation_is_chosen_for_long_histories_only_and_handles_edge_requests():
+def test_pool_side_factorisation_is_chosen_when_it_pays_and_handles_edge_requests():
     import paper_2601_19178_b200 as ckv
-    # histories long against the pool (mean length >= n_entries / 4): chosen by default
-    w = synth.Workload("fact_long", 2, 60, 4, 512, 6, (100, 2000), 1, "softmax", "bf16", None, 1 / 64, 1 / 64, 32)
+    # one wave of (user, group) pairs with histories long against the pool: chosen by default
+    w = synth.Workload("fact_long", 4, 60, 4, 512, 37, (1500, 3000), 1, "softmax", "bf16", None, 1 / 64, 1 / 64, 32)
     d = synth.generate(w)
     s = make_session(w, d)
     got = gpu_attend(w, d, session=s)
     assert s.stat("kernel") == 4
     assert_close(got, oracle_attend(w, d), "bf16", "auto")
-    # request list with an empty query list and a repeated user: [u0, u1 (no query), u2, u0]
+    # a handful of pairs cannot fill the SMs with one CTA per pair: the gathering kernel stays
+    few = s.attend(d["users"][:3], d["q_off"][:4], to_dev(d["queries"][:3], "bf16")).float().cpu().numpy().astype(np.float64)
+    assert s.stat("kernel") == 2
+    assert_close(few, got[:3], "bf16", "few pairs")
+    # forced: request list with an empty query list and a repeated user: [u0, u1 (no query), u2, u0]
+    s.set_option("kernel", 4)
     req = d["users"][[0, 1, 2, 0]]
     q_off = np.array([0, 1, 1, 2, 3], dtype=np.int32)
     q = to_dev(d["queries"][[0, 2, 0]], "bf16")
@@ -271,13 +276,12 @@ def test_pool_side_factorisation_is_chosen_for_long_histories_only_and_handles_e
     assert_close(out[1], got[2], "bf16")
     assert_close(out[2], got[0], "bf16")
     # more than one query for a user: the family cannot take it
-    s.set_option("kernel", 4)
     with pytest.raises(ckv.CkvError) as e:
         s.attend(d["users"][:2], np.array([0, 2, 3], dtype=np.int32), to_dev(d["queries"][:3], "bf16"))
     assert e.value.status == ckv.CKV_ERR_UNSUPPORTED
     s.close()
-    # short histories against a large pool: the gathering kernel stays
-    w2 = synth.Workload("fact_short", 2, 60, 4, 4096, 6, (10, 200), 1, "softmax", "bf16", None, 1 / 64, 1 / 64, 33)
+    # many pairs, but short histories against a large pool: the gathering kernel stays
+    w2 = synth.Workload("fact_short", 4, 60, 4, 4096, 40, (10, 200), 1, "softmax", "bf16", None, 1 / 64, 1 / 64, 33)
     d2 = synth.generate(w2)
     s2 = make_session(w2, d2)
     assert_close(gpu_attend(w2, d2, session=s2), oracle_attend(w2, d2), "bf16", "short")

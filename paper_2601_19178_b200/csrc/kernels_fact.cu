@@ -492,14 +492,11 @@ __global__ void __launch_bounds__(kOutWarps * 32, 1)
     }
 }
 
-// Opt-in to large dynamic shared memory, once per kernel (the most a CTA can have on this architecture).
+// Opt-in to large dynamic shared memory (per launch: the attribute belongs to the current device).
 template <typename K>
-cudaError_t set_smem(K kernel, bool& done)
+cudaError_t set_smem(K kernel, size_t bytes)
 {
-    if (done) return cudaSuccess;
-    const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-    done = e == cudaSuccess;
-    return e;
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
 }
 
 template <int D>
@@ -517,8 +514,7 @@ cudaError_t launch_fact(const AttendArgs& a, int n_req, int max_L, int n_sms, fl
     const dim3 grid(n_pairs < n_sms ? n_pairs : n_sms);
 #define CKV_FACT_MAIN(MODE, I16)                                                       \
     do {                                                                               \
-        static bool done_main = false;                                                 \
-        e = set_smem(fact_main_kernel<D, MODE, I16>, done_main);                       \
+        e = set_smem(fact_main_kernel<D, MODE, I16>, smem_main);                       \
         if (e != cudaSuccess) return e;                                                \
         fact_main_kernel<D, MODE, I16><<<grid, kMainThreads, smem_main, s>>>(a, tw, aux, s_cap); \
     } while (0)
@@ -531,8 +527,7 @@ cudaError_t launch_fact(const AttendArgs& a, int n_req, int max_L, int n_sms, fl
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     const size_t smem_out = std::max((size_t)kOutWarps * 2 * 32 * D * 2, (size_t)kOutWarps * 16 * D * sizeof(float));
-    static bool done_out = false;
-    e = set_smem(fact_out_kernel<D>, done_out);
+    e = set_smem(fact_out_kernel<D>, smem_out);
     if (e != cudaSuccess) return e;
     fact_out_kernel<D><<<dim3((n_req + 15) / 16, G), kOutWarps * 32, smem_out, s>>>(a, n_req, tw, aux);
     return cudaGetLastError();

@@ -528,13 +528,10 @@ cudaError_t launch_mma_one(const AttendArgs& a, int n_mb, dim3 grid, const CUten
                            cudaStream_t s)
 {
     using C = MmaCfg<D, MT, TMA>;
-    static bool configured = false;  // per instantiation; the attribute is idempotent
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(attend_mma_kernel<D, MT, MODE, IDX16, TMA>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
+    // per launch: the attribute belongs to the current device, and a context may sit on any of them
+    cudaError_t e = cudaFuncSetAttribute(attend_mma_kernel<D, MT, MODE, IDX16, TMA>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
+    if (e != cudaSuccess) return e;
     static const CUtensorMap none{};
     attend_mma_kernel<D, MT, MODE, IDX16, TMA>
         <<<grid, 128, C::SMEM, s>>>(a, n_mb, TMA ? maps[0] : none, TMA ? maps[1] : none, err_flag);

@@ -187,6 +187,22 @@ CKV_API ckv_status ckv_attend_static(ckv_ctx* ctx, int32_t n, const int64_t* use
 CKV_API ckv_status ckv_materialize(ckv_ctx* ctx, int64_t user, void* K_out, void* V_out, void* stream);
 
 /*
+ * Prefill router (Sec. 4.3): the global-pool entry each of n history positions selects,
+ *     idx_out[i][g] = the lowest j that maximises  x_i . W[g][j] + bias[g][j]
+ * (one router per group; the K and the V router are two calls).  The n x n_entries score matrix is
+ * never written.  Needs no context.
+ *   x        device, bf16 [n][d_in]             inputs of the positions (d_in in {32, 64, 128})
+ *   W        device, bf16 [n_groups][n_entries][d_in]   router weights, an entry's weights contiguous
+ *   bias     device, fp32 [n_groups][n_entries], or NULL for none
+ *   idx_out  device, int32 [n][n_groups]        what ckv_cache_put takes as idx_K / idx_V
+ * Products are exact, sums fp32; entries whose scores are equal in that arithmetic resolve to the
+ * lowest index.  Stream-ordered.
+ * Errors: INVALID_ARG (sizes, null or host pointers), UNSUPPORTED (d_in), CUDA.
+ */
+CKV_API ckv_status ckv_route(int32_t device, int32_t n, int32_t n_groups, int32_t d_in, int32_t n_entries,
+                             const void* x, const void* W, const float* bias, int32_t* idx_out, void* stream);
+
+/*
  * Appends L_new positions (new interactions) behind a cached user's history; arguments as for
  * ckv_cache_put, describing only the new positions.  The user's compressed cache moves to fresh
  * storage holding the old and the new positions (storage is only reclaimed by ckv_cache_clear or

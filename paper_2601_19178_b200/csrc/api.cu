@@ -921,6 +921,25 @@ ckv_status ckv_cache_bytes(ckv_ctx* ctx, int64_t* compressed, int64_t* full_widt
     return CKV_OK;
 }
 
+ckv_status ckv_route(int32_t device, int32_t n, int32_t n_groups, int32_t d_in, int32_t n_entries, const void* x,
+                     const void* W, const float* bias, int32_t* idx_out, void* stream)
+{
+    if (n < 0 || n_groups < 1 || n_entries < 1 || device < 0) return CKV_ERR_INVALID_ARG;
+    if (!route_supported(d_in)) return CKV_ERR_UNSUPPORTED;
+    if (n == 0) return CKV_OK;
+    if (!x || !W || !idx_out) return CKV_ERR_INVALID_ARG;
+    DeviceGuard dg(device);
+    if (!dg.ok) return CKV_ERR_CUDA;
+    if (!is_device_ptr(x) || !is_device_ptr(W) || !is_device_ptr(idx_out) || (bias && !is_device_ptr(bias)))
+        return CKV_ERR_INVALID_ARG;
+    const cudaError_t e = launch_route(d_in, x, W, bias, n, n_entries, n_groups, idx_out, (cudaStream_t)stream);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return CKV_ERR_CUDA;
+    }
+    return CKV_OK;
+}
+
 ckv_status ckv_set_option(ckv_ctx* ctx, const char* name, int64_t value)
 {
     if (!ctx || !name) return CKV_ERR_INVALID_ARG;

@@ -115,6 +115,13 @@ int fact_row_floats(int n_entries);
 cudaError_t launch_attend_fact(int head_dim, const AttendArgs& a, int n_req, int max_L, int n_sms, float* tw,
                                float* aux, cudaStream_t s);
 
+// ---- kernels_route.cu : prefill router, fused scores + row arg-max (bf16, d_in 32 / 64 / 128)
+bool route_supported(int d_in);
+// out[i][g] = lowest entry j maximising x_i . W[g][j] + bias[g][j]; x [n][d_in], W [G][n_entries][d_in] bf16 (device),
+// bias [G][n_entries] fp32 or null, out [n][G] int32.
+cudaError_t launch_route(int d_in, const void* x, const void* W, const float* bias, int n, int n_entries, int G,
+                         int32_t* out, cudaStream_t s);
+
 // ---- kernels_umma.cu : tcgen05 family (bf16, head_dim 32, d_user in {0, 1, 2, 4, 8}, 16-bit stored indices)
 bool umma_supported(int dtype, int head_dim, int d_user, int idx_bytes);
 // err_flag: device int, OR-ed with a non-zero code if a bounded wait inside the kernel ran out.

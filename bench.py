@@ -464,6 +464,65 @@ def run_load_path(args, w):
     print(json.dumps(line), flush=True)
 
 
+def run_route(args):
+    """Prefill router (Sec. 4.3) on a prefill-sized batch: n positions scored against every pool entry of every
+    group, arg-max per row.  Reported against the bf16 tensor-core peak (it is a dense contraction)."""
+    import torch
+    import paper_2601_19178_b200 as ckv
+    from oracle import route_oracle as R
+
+    rank, _, local = rank_env()
+    if rank != 0:
+        return
+    torch.cuda.set_device(local)
+    n, d_in, m, G = 1 << 20, 64, 16384, 4           # one million positions, the pool shape of cfg4
+    rng = np.random.default_rng(7)
+    x = synth.f32_to_bf16_bits((rng.standard_normal((n, d_in)) / np.sqrt(d_in)).astype(np.float32))
+    W = synth.f32_to_bf16_bits(rng.standard_normal((G, m, d_in)).astype(np.float32))
+    b = (0.1 * rng.standard_normal((G, m))).astype(np.float32)
+    xd = torch.from_numpy(x.view(np.int16)).view(torch.bfloat16).cuda()
+    Wd = torch.from_numpy(W.view(np.int16)).view(torch.bfloat16).cuda()
+    bd = torch.from_numpy(b).cuda()
+    out = torch.empty((n, G), dtype=torch.int32, device="cuda")
+    steps, warm = max(args.steps, 3), max(args.warmup, 3)
+    for _ in range(warm):
+        ckv.ckv_route(local, n, G, d_in, m, xd, Wd, bd, out)
+    torch.cuda.synchronize()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for e0, e1 in evs:
+        e0.record()
+        ckv.ckv_route(local, n, G, d_in, m, xd, Wd, bd, out)
+        e1.record()
+    torch.cuda.synchronize()
+    ms = statistics.mean(e0.elapsed_time(e1) for e0, e1 in evs)
+    # sampled parity: 512 positions against the float64 oracle (ties in fp32 may pick an equal-scoring entry)
+    sel = rng.integers(0, n, size=512)
+    M = R.scores(x[sel], W, b)
+    want = np.argmax(M, axis=2).T
+    got = out[torch.from_numpy(sel).cuda()].cpu().numpy()
+    gi, ii = np.meshgrid(np.arange(G), np.arange(len(sel)))
+    gap = M[gi, ii, want] - M[gi, ii, got]
+    ok = bool((gap <= 4 * d_in * 2.0 ** -24 * np.abs(M).max()).all())
+    flops = 2.0 * n * m * d_in * G
+    peak_tf, kind = 1590.0, "fallback"
+    pth = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(pth):
+        try:
+            peak_tf, kind = float(json.load(open(pth))["bf16_tflops"]), "measured"
+        except Exception:
+            pass
+    ach = flops / (ms * 1e-3) / 1e12
+    line = {"mode": "route", "metric": "router_positions_per_sec", "value": n / (ms * 1e-3), "unit": "positions/s",
+            "higher_is_better": True, "n_gpus": 1, "steps": steps, "warmup": warm, "ms_per_step": ms, "dtype": "bf16",
+            "data": "synthetic",
+            "config": {"positions": n, "d_in": d_in, "n_entries": m, "n_groups": G, "inputs": "larger than L2"},
+            "roofline": {"bound": "tensor", "achieved": ach, "peak": peak_tf, "unit": "TFLOP/s", "frac": ach / peak_tf,
+                         "peak_kind": kind, "traffic": None},
+            "parity": {"positions_checked": int(len(sel)), "ok": ok, "index_mismatches": int((got != want).sum())},
+            "gpu_launches": steps}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -477,6 +536,7 @@ def main():
     ap.add_argument("--mma-loader", type=int, default=0, help="1 = cp.async (default), 2 = TMA gathers")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-check", action="store_true", help="skip the sampled parity check")
+    ap.add_argument("--route", action="store_true", help="time the prefill router (Sec. 4.3) instead of the attend step")
     ap.add_argument("--load-path", action="store_true",
                     help="time the decode-stage load path per batch size (Sec. 4.4) instead of the attend step")
     args = ap.parse_args()
@@ -485,6 +545,8 @@ def main():
         w = synth.scaled(w, n_users=args.users)
     if args.impl == "reference":
         run_reference(args, w)
+    elif args.route:
+        run_route(args)
     elif args.load_path:
         run_load_path(args, w)
     else:

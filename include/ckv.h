@@ -203,6 +203,20 @@ CKV_API ckv_status ckv_route(int32_t device, int32_t n, int32_t n_groups, int32_
                              const void* x, const void* W, const float* bias, int32_t* idx_out, void* stream);
 
 /*
+ * Prefill, user-specific part (Sec. 4.2): the low-dimensional keys (or values) of n positions,
+ *     out[i][g][c] = x_i . W[g][c] + bias[g][c],      c < d_out
+ * (one call with the K weights, one with the V weights).  Needs no context.
+ *   x     device, bf16 [n][d_in]                    d_in a multiple of 8, at most 256
+ *   W     device, bf16 [n_groups][d_out][d_in]      d_out at most 16
+ *   bias  device, fp32 [n_groups][d_out], or NULL
+ *   out   device, bf16 [n][n_groups][d_out]         what ckv_cache_put takes as user_K / user_V
+ * fp32 sums, result rounded to nearest even.  Stream-ordered.
+ * Errors: INVALID_ARG, UNSUPPORTED (shape), CUDA.
+ */
+CKV_API ckv_status ckv_project(int32_t device, int32_t n, int32_t n_groups, int32_t d_in, int32_t d_out,
+                               const void* x, const void* W, const float* bias, void* out, void* stream);
+
+/*
  * Appends L_new positions (new interactions) behind a cached user's history; arguments as for
  * ckv_cache_put, describing only the new positions.  The user's compressed cache moves to fresh
  * storage holding the old and the new positions (storage is only reclaimed by ckv_cache_clear or

@@ -29,3 +29,13 @@ def scores(x, W, bias=None) -> np.ndarray:
 def route(x, W, bias=None) -> np.ndarray:
     """I [n][G] int32: lowest index of the row maximum of M."""
     return np.argmax(scores(x, W, bias), axis=2).T.astype(np.int32)
+
+
+def project(x, W, bias=None) -> np.ndarray:
+    """User-specific low-dimensional part (Sec. 4.2): y [n][G][d_out] float64 = x . W[g][c] + bias[g][c]
+    for x [n][d_in], W [G][d_out][d_in], bias [G][d_out] or None -- the linear layer written out."""
+    X, Wf = _f64(x), _f64(W)
+    y = np.einsum("nk,gck->ngc", X, Wf)
+    if bias is not None:
+        y = y + np.asarray(bias, dtype=np.float64)[None]
+    return y

@@ -25,7 +25,7 @@ EXPORTS = (
     "ckv_cache_evict", "ckv_cache_clear", "ckv_attend", "ckv_attend_static", "ckv_materialize",
     "ckv_user_length", "ckv_cache_append", "ckv_cache_blob_bytes", "ckv_cache_export", "ckv_cache_import",
     "ckv_cache_bytes", "ckv_set_option", "ckv_get_option", "ckv_last_stat", "ckv_strerror",
-    "ckv_last_cuda_error", "ckv_version", "ckv_route",
+    "ckv_last_cuda_error", "ckv_version", "ckv_route", "ckv_project",
 )
 
 
@@ -74,6 +74,7 @@ def _load() -> ctypes.CDLL:
         "ckv_last_cuda_error": (cs, [vp]),
         "ckv_version": (i32, []),
         "ckv_route": (i32, [i32, i32, i32, i32, i32, vp, vp, vp, vp, vp]),
+        "ckv_project": (i32, [i32, i32, i32, i32, i32, vp, vp, vp, vp, vp]),
     }
     for name, (res, args) in sig.items():
         f = getattr(L, name)
@@ -256,3 +257,10 @@ def ckv_route(device: int, n: int, n_groups: int, d_in: int, n_entries: int, x, 
     or None, idx_out [n][G] int32 (device)."""
     _check(None, lib.ckv_route(device, n, n_groups, d_in, n_entries, _ptr(x), _ptr(W), _ptr(bias), _ptr(idx_out),
                                _stream(stream)), "ckv_route")
+
+
+def ckv_project(device: int, n: int, n_groups: int, d_in: int, d_out: int, x, W, bias, out, stream=None) -> None:
+    """User-specific low-dimensional projection: x [n][d_in], W [G][d_out][d_in] (bf16, device), bias [G][d_out]
+    fp32 or None, out [n][G][d_out] bf16 (device)."""
+    _check(None, lib.ckv_project(device, n, n_groups, d_in, d_out, _ptr(x), _ptr(W), _ptr(bias), _ptr(out),
+                                 _stream(stream)), "ckv_project")

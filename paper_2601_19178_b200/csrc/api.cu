@@ -940,6 +940,25 @@ ckv_status ckv_route(int32_t device, int32_t n, int32_t n_groups, int32_t d_in, 
     return CKV_OK;
 }
 
+ckv_status ckv_project(int32_t device, int32_t n, int32_t n_groups, int32_t d_in, int32_t d_out, const void* x,
+                       const void* W, const float* bias, void* out, void* stream)
+{
+    if (n < 0 || n_groups < 1 || device < 0) return CKV_ERR_INVALID_ARG;
+    if (!project_supported(d_in, d_out, n_groups)) return CKV_ERR_UNSUPPORTED;
+    if (n == 0) return CKV_OK;
+    if (!x || !W || !out) return CKV_ERR_INVALID_ARG;
+    DeviceGuard dg(device);
+    if (!dg.ok) return CKV_ERR_CUDA;
+    if (!is_device_ptr(x) || !is_device_ptr(W) || !is_device_ptr(out) || (bias && !is_device_ptr(bias)))
+        return CKV_ERR_INVALID_ARG;
+    const cudaError_t e = launch_project(d_in, d_out, n_groups, x, W, bias, n, out, (cudaStream_t)stream);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return CKV_ERR_CUDA;
+    }
+    return CKV_OK;
+}
+
 ckv_status ckv_set_option(ckv_ctx* ctx, const char* name, int64_t value)
 {
     if (!ctx || !name) return CKV_ERR_INVALID_ARG;

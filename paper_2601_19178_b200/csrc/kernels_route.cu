@@ -176,6 +176,39 @@ cudaError_t launch_route_t(const void* x, const void* W, const float* bias, int 
     return cudaGetLastError();
 }
 
+// User-specific low-dimensional projection of the prefill (Sec. 4.2): y[i][g][c] = x_i . W[g][c] + b[g][c],
+// d_out <= 16 outputs per group.  Memory-bound: one thread per output element, the weights in shared memory
+// (rows padded by 16 bytes against bank conflicts), 16-byte loads of the input row, fp32 sums, bf16 result.
+__global__ void __launch_bounds__(256) project_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ W,
+                                                      const float* __restrict__ bias, int64_t total, int d_in, int gd,
+                                                      uint16_t* __restrict__ out)
+{
+    extern __shared__ __align__(16) unsigned char psm[];
+    const int wrow = d_in * 2 + 16;  // bytes per padded weight row
+    for (int q = threadIdx.x; q < gd * (d_in / 8); q += blockDim.x) {
+        const int r = q / (d_in / 8), c = q - r * (d_in / 8);
+        *reinterpret_cast<uint4*>(psm + r * wrow + c * 16) = __ldg(reinterpret_cast<const uint4*>(W + (int64_t)r * d_in) + c);
+    }
+    __syncthreads();
+    for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t i = e / gd;
+        const int r = (int)(e - i * gd);  // (group, output) row of W
+        const uint4* xr = reinterpret_cast<const uint4*>(x + i * d_in);
+        const unsigned char* wr = psm + r * wrow;
+        float acc = bias ? __ldg(bias + r) : 0.f;
+        for (int c = 0; c < d_in / 8; ++c) {
+            const uint4 a = __ldg(xr + c), b = *reinterpret_cast<const uint4*>(wr + c * 16);
+            const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                acc = fmaf(__uint_as_float(aw[k] << 16), __uint_as_float(bw[k] << 16), acc);
+                acc = fmaf(__uint_as_float(aw[k] & 0xffff0000u), __uint_as_float(bw[k] & 0xffff0000u), acc);
+            }
+        }
+        out[e] = __bfloat16_as_ushort(__float2bfloat16_rn(acc));
+    }
+}
+
 }  // namespace
 
 bool route_supported(int d_in) { return d_in == 32 || d_in == 64 || d_in == 128; }
@@ -189,6 +222,28 @@ cudaError_t launch_route(int d_in, const void* x, const void* W, const float* bi
         case 64: return launch_route_t<64>(x, W, bias, n, n_entries, G, out, s);
         default: return launch_route_t<128>(x, W, bias, n, n_entries, G, out, s);
     }
+}
+
+bool project_supported(int d_in, int d_out, int n_groups)
+{
+    return d_in >= 8 && d_in <= 256 && d_in % 8 == 0 && d_out >= 1 && d_out <= 16 &&
+           (size_t)n_groups * d_out * (d_in * 2 + 16) <= 96 * 1024;
+}
+
+cudaError_t launch_project(int d_in, int d_out, int G, const void* x, const void* W, const float* bias, int64_t n,
+                           void* out, cudaStream_t s)
+{
+    if (n == 0) return cudaSuccess;
+    const int gd = G * d_out;
+    const size_t smem = (size_t)gd * (d_in * 2 + 16);
+    cudaError_t e = cudaFuncSetAttribute(project_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    const int64_t total = n * gd;
+    int64_t blocks = (total + 255) / 256;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    project_kernel<<<(unsigned)blocks, 256, smem, s>>>((const uint16_t*)x, (const uint16_t*)W, bias, total, d_in, gd,
+                                                       (uint16_t*)out);
+    return cudaGetLastError();
 }
 
 }  // namespace ckv

@@ -486,12 +486,12 @@ def run_route(args):
     out = torch.empty((n, G), dtype=torch.int32, device="cuda")
     steps, warm = max(args.steps, 3), max(args.warmup, 3)
     for _ in range(warm):
-        ckv.ckv_route(local, n, G, d_in, m, xd, Wd, bd, out)
+        ckv.ckv_route(local, n, G, d_in, m, xd, Wd, bd, out, args.kernel if args.kernel in (1, 2) else 0)
     torch.cuda.synchronize()
     evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
     for e0, e1 in evs:
         e0.record()
-        ckv.ckv_route(local, n, G, d_in, m, xd, Wd, bd, out)
+        ckv.ckv_route(local, n, G, d_in, m, xd, Wd, bd, out, args.kernel if args.kernel in (1, 2) else 0)
         e1.record()
     torch.cuda.synchronize()
     ms = statistics.mean(e0.elapsed_time(e1) for e0, e1 in evs)
@@ -515,7 +515,8 @@ def run_route(args):
     line = {"mode": "route", "metric": "router_positions_per_sec", "value": n / (ms * 1e-3), "unit": "positions/s",
             "higher_is_better": True, "n_gpus": 1, "steps": steps, "warmup": warm, "ms_per_step": ms, "dtype": "bf16",
             "data": "synthetic",
-            "config": {"positions": n, "d_in": d_in, "n_entries": m, "n_groups": G, "inputs": "larger than L2"},
+            "config": {"positions": n, "d_in": d_in, "n_entries": m, "n_groups": G, "inputs": "larger than L2",
+                       "variant": "warp-level mma" if args.kernel == 1 else "tcgen05"},
             "roofline": {"bound": "tensor", "achieved": ach, "peak": peak_tf, "unit": "TFLOP/s", "frac": ach / peak_tf,
                          "peak_kind": kind, "traffic": None},
             "parity": {"positions_checked": int(len(sel)), "ok": ok, "index_mismatches": int((got != want).sum())},

@@ -195,12 +195,16 @@ CKV_API ckv_status ckv_materialize(ckv_ctx* ctx, int64_t user, void* K_out, void
  *   W        device, bf16 [n_groups][n_entries][d_in]   router weights, an entry's weights contiguous
  *   bias     device, fp32 [n_groups][n_entries], or NULL for none
  *   idx_out  device, int32 [n][n_groups]        what ckv_cache_put takes as idx_K / idx_V
+ *   variant  0 = default (tcgen05 kernel), 1 = warp-level tensor-core kernel, 2 = tcgen05 kernel
  * Products are exact, sums fp32; entries whose scores are equal in that arithmetic resolve to the
- * lowest index.  Stream-ordered.
- * Errors: INVALID_ARG (sizes, null or host pointers), UNSUPPORTED (d_in), CUDA.
+ * lowest index.  The tcgen05 kernel's waits are bounded; the call reads its error word back and
+ * therefore synchronises `stream` (variant 1 is only stream-ordered).
+ * Errors: INVALID_ARG (sizes, null or host pointers), UNSUPPORTED (d_in), OOM, CUDA (also: a wait
+ * inside the kernel ran out; idx_out is not valid then).
  */
 CKV_API ckv_status ckv_route(int32_t device, int32_t n, int32_t n_groups, int32_t d_in, int32_t n_entries,
-                             const void* x, const void* W, const float* bias, int32_t* idx_out, void* stream);
+                             const void* x, const void* W, const float* bias, int32_t* idx_out, int32_t variant,
+                             void* stream);
 
 /*
  * Prefill, user-specific part (Sec. 4.2): the low-dimensional keys (or values) of n positions,

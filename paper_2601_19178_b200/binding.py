@@ -73,7 +73,7 @@ def _load() -> ctypes.CDLL:
         "ckv_strerror": (cs, [i32]),
         "ckv_last_cuda_error": (cs, [vp]),
         "ckv_version": (i32, []),
-        "ckv_route": (i32, [i32, i32, i32, i32, i32, vp, vp, vp, vp, vp]),
+        "ckv_route": (i32, [i32, i32, i32, i32, i32, vp, vp, vp, vp, i32, vp]),
         "ckv_project": (i32, [i32, i32, i32, i32, i32, vp, vp, vp, vp, vp]),
     }
     for name, (res, args) in sig.items():
@@ -252,11 +252,12 @@ def ckv_version() -> int:
     return int(lib.ckv_version())
 
 
-def ckv_route(device: int, n: int, n_groups: int, d_in: int, n_entries: int, x, W, bias, idx_out, stream=None) -> None:
+def ckv_route(device: int, n: int, n_groups: int, d_in: int, n_entries: int, x, W, bias, idx_out, variant: int = 0,
+              stream=None) -> None:
     """Router indices of n positions: x [n][d_in], W [G][n_entries][d_in] (bf16, device), bias [G][n_entries] fp32
-    or None, idx_out [n][G] int32 (device)."""
+    or None, idx_out [n][G] int32 (device); variant 0 / 2 = tcgen05 kernel, 1 = warp-level tensor-core kernel."""
     _check(None, lib.ckv_route(device, n, n_groups, d_in, n_entries, _ptr(x), _ptr(W), _ptr(bias), _ptr(idx_out),
-                               _stream(stream)), "ckv_route")
+                               int(variant), _stream(stream)), "ckv_route")
 
 
 def ckv_project(device: int, n: int, n_groups: int, d_in: int, d_out: int, x, W, bias, out, stream=None) -> None:

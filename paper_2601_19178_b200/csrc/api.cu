@@ -921,10 +921,32 @@ ckv_status ckv_cache_bytes(ckv_ctx* ctx, int64_t* compressed, int64_t* full_widt
     return CKV_OK;
 }
 
-ckv_status ckv_route(int32_t device, int32_t n, int32_t n_groups, int32_t d_in, int32_t n_entries, const void* x,
-                     const void* W, const float* bias, int32_t* idx_out, void* stream)
+namespace {
+
+// one error word per device for the context-free tcgen05 router (allocated on first use, never freed)
+int* route_err_word(int device)
 {
-    if (n < 0 || n_groups < 1 || n_entries < 1 || device < 0) return CKV_ERR_INVALID_ARG;
+    static std::mutex mu;
+    static int* words[64] = {};
+    std::lock_guard<std::mutex> lock(mu);
+    if (device >= 64) return nullptr;
+    if (!words[device]) {
+        int* p = nullptr;
+        if (cudaMalloc(&p, sizeof(int)) != cudaSuccess || cudaMemset(p, 0, sizeof(int)) != cudaSuccess) {
+            cudaGetLastError();
+            return nullptr;
+        }
+        words[device] = p;
+    }
+    return words[device];
+}
+
+}  // namespace
+
+ckv_status ckv_route(int32_t device, int32_t n, int32_t n_groups, int32_t d_in, int32_t n_entries, const void* x,
+                     const void* W, const float* bias, int32_t* idx_out, int32_t variant, void* stream)
+{
+    if (n < 0 || n_groups < 1 || n_entries < 1 || device < 0 || variant < 0 || variant > 2) return CKV_ERR_INVALID_ARG;
     if (!route_supported(d_in)) return CKV_ERR_UNSUPPORTED;
     if (n == 0) return CKV_OK;
     if (!x || !W || !idx_out) return CKV_ERR_INVALID_ARG;
@@ -932,7 +954,22 @@ ckv_status ckv_route(int32_t device, int32_t n, int32_t n_groups, int32_t d_in, 
     if (!dg.ok) return CKV_ERR_CUDA;
     if (!is_device_ptr(x) || !is_device_ptr(W) || !is_device_ptr(idx_out) || (bias && !is_device_ptr(bias)))
         return CKV_ERR_INVALID_ARG;
-    const cudaError_t e = launch_route(d_in, x, W, bias, n, n_entries, n_groups, idx_out, (cudaStream_t)stream);
+    cudaStream_t s = (cudaStream_t)stream;
+    cudaError_t e;
+    if (variant == 1) {
+        e = launch_route(d_in, x, W, bias, n, n_entries, n_groups, idx_out, s);
+    } else {
+        int* word = route_err_word(device);
+        if (!word) return CKV_ERR_OOM;
+        e = launch_route_umma(d_in, x, W, bias, n, n_entries, n_groups, idx_out, word, s);
+        int bad = 0;
+        if (e == cudaSuccess) e = cudaMemcpyAsync(&bad, word, sizeof(int), cudaMemcpyDeviceToHost, s);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+        if (e == cudaSuccess && bad) {  // a bounded wait inside the kernel ran out: the output is not valid
+            cudaMemsetAsync(word, 0, sizeof(int), s);
+            return CKV_ERR_CUDA;
+        }
+    }
     if (e != cudaSuccess) {
         cudaGetLastError();
         return CKV_ERR_CUDA;

@@ -122,6 +122,11 @@ bool route_supported(int d_in);
 cudaError_t launch_route(int d_in, const void* x, const void* W, const float* bias, int n, int n_entries, int G,
                          int32_t* out, cudaStream_t s);
 
+// ---- kernels_route_umma.cu : the same router on tcgen05 (TMEM accumulators, warp-specialised)
+// err_flag: device int, OR-ed with a non-zero code if a bounded wait inside the kernel ran out (nothing is written then).
+cudaError_t launch_route_umma(int d_in, const void* x, const void* W, const float* bias, int n, int n_entries, int G,
+                              int32_t* out, int* err_flag, cudaStream_t s);
+
 // out[i][g][c] = x_i . W[g][c] + bias[g][c] (bf16 in and out, fp32 sums); W [G][d_out][d_in], bias [G][d_out] or null.
 bool project_supported(int d_in, int d_out, int n_groups);
 cudaError_t launch_project(int d_in, int d_out, int G, const void* x, const void* W, const float* bias, int64_t n,

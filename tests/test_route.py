@@ -56,7 +56,7 @@ def test_oracle_closed_forms():
     assert np.array_equal(R.route(_bf16(x), _bf16(Wr)), R.route(synth.bf16_bits_to_f32(_bf16(x)), synth.bf16_bits_to_f32(_bf16(Wr))))
 
 
-def _gpu_route(x_bits, W_bits, bias):
+def _gpu_route(x_bits, W_bits, bias, variant=0):
     import torch
     import paper_2601_19178_b200 as ckv
     from paper_2601_19178_b200.session import as_device_tensor as dev
@@ -65,13 +65,13 @@ def _gpu_route(x_bits, W_bits, bias):
     xd, Wd = dev(x_bits, "bf16"), dev(W_bits, "bf16")
     bd = torch.from_numpy(bias).cuda() if bias is not None else None
     out = torch.full((n, G), -1, dtype=torch.int32, device="cuda")
-    ckv.ckv_route(0, n, G, d, m, xd, Wd, bd, out)
+    ckv.ckv_route(0, n, G, d, m, xd, Wd, bd, out, variant)
     torch.cuda.synchronize()
     return out.cpu().numpy()
 
 
-def _check(x_bits, W_bits, bias, what):
-    got = _gpu_route(x_bits, W_bits, bias)
+def _check(x_bits, W_bits, bias, what, variant=0):
+    got = _gpu_route(x_bits, W_bits, bias, variant)
     M = R.scores(x_bits, W_bits, bias)                     # [G][n][m] float64
     want = np.argmax(M, axis=2).T
     n, G = want.shape
@@ -87,15 +87,16 @@ def _check(x_bits, W_bits, bias, what):
 
 
 @pytest.mark.gpu
+@pytest.mark.parametrize("variant", [1, 2])
 @pytest.mark.parametrize("d_in", [32, 64, 128])
 @pytest.mark.parametrize("n,m,G", [(1, 1, 1), (37, 5, 2), (300, 333, 3), (1000, 2048, 2), (513, 4100, 1)])
-def test_gpu_router_matches_oracle(d_in, n, m, G):
+def test_gpu_router_matches_oracle(d_in, n, m, G, variant):
     rng = np.random.default_rng(d_in + n + m)
     x = _bf16(rng.standard_normal((n, d_in)) / np.sqrt(d_in))
     W = _bf16(rng.standard_normal((G, m, d_in)))
     b = (0.1 * rng.standard_normal((G, m))).astype(np.float32)
-    _check(x, W, b, f"d_in={d_in} n={n} m={m} G={G}")
-    _check(x, W, None, f"no bias d_in={d_in} n={n} m={m} G={G}")
+    _check(x, W, b, f"d_in={d_in} n={n} m={m} G={G} variant={variant}", variant)
+    _check(x, W, None, f"no bias d_in={d_in} n={n} m={m} G={G} variant={variant}", variant)
 
 
 @pytest.mark.gpu
@@ -109,18 +110,19 @@ def test_gpu_router_exact_cases_and_errors():
     for j in range(m):
         W[0, j, j % d] = 1.0
     x = np.eye(d, dtype=np.float32)[np.arange(70) % d]
-    got = _gpu_route(_bf16(x), _bf16(W), None)
-    assert np.array_equal(got[:, 0], np.arange(70) % d)      # entries k, k + 32, ... tie: the first one
-    assert np.array_equal(got, R.route(_bf16(x), _bf16(W)))
+    for variant in (1, 2):
+        got = _gpu_route(_bf16(x), _bf16(W), None, variant)
+        assert np.array_equal(got[:, 0], np.arange(70) % d)      # entries k, k + 32, ... tie: the first one
+        assert np.array_equal(got, R.route(_bf16(x), _bf16(W)))
     # the output feeds ckv_cache_put as it is: indices in range, int32 [n][G]
     with pytest.raises(ckv.CkvError) as e:
         ckv.ckv_route(0, 4, 1, 48, 8, torch.zeros(4, 48, dtype=torch.bfloat16, device="cuda"),
                       torch.zeros(1, 8, 48, dtype=torch.bfloat16, device="cuda"), None,
-                      torch.zeros(4, 1, dtype=torch.int32, device="cuda"))
+                      torch.zeros(4, 1, dtype=torch.int32, device="cuda"), 0)
     assert e.value.status == ckv.CKV_ERR_UNSUPPORTED
     with pytest.raises(ckv.CkvError) as e:
         ckv.ckv_route(0, 4, 1, 32, 8, np.zeros((4, 32), np.uint16), torch.zeros(1, 8, 32, dtype=torch.bfloat16, device="cuda"),
-                      None, torch.zeros(4, 1, dtype=torch.int32, device="cuda"))
+                      None, torch.zeros(4, 1, dtype=torch.int32, device="cuda"), 0)
     assert e.value.status == ckv.CKV_ERR_INVALID_ARG
 
 

@@ -1,9 +1,10 @@
 // Prefill router (Sec. 4.3) on the tcgen05 tensor cores: I[i][g] = lowest j maximising x_i . W_g[j] + b_g[j].
 //
 // One CTA owns 128 positions of one group.  Their inputs sit in shared memory once (A operand, K-major core-matrix
-// layout); the group's weight rows stream through a four-stage ring in tiles of 128 entries (B operand, same
-// layout, 16-byte cp.async by four producer warps, each owning every fourth tile and therefore one stage).  One
-// thread issues the 128 x 128 x d_in product of a tile into one of two TMEM accumulators; two groups of four warps
+// layout); the group's weight rows stream through a ring of stages in tiles of 256 entries (B operand, same
+// layout, 16-byte cp.async by four producer warps, each bound to one stage).  A tcgen05 instruction costs
+// its issuing thread about 100 clocks whatever its size, hence the widest tile the accumulators allow.  One
+// thread issues the 128 x 256 x d_in product of a tile into one of two TMEM accumulators (all 512 columns); two groups of four warps
 // (thread = position = TMEM lane) take turns reading an accumulator, add the bias, and keep a running (best score,
 // entry) in registers, so the score matrix never leaves the SM.  The two groups' results are merged at the end.
 // Every wait is bounded: a time-out raises the CTA's abort flag, the CTA drains, frees its TMEM, reports through
@@ -16,13 +17,13 @@
 namespace ckv {
 namespace {
 
-constexpr int kRows = 128, kTileN = 128, kStages = 4, kBiasSlots = 8;
+constexpr int kRows = 128, kTileN = 256, kMaxStages = 4, kBiasSlots = 8;
 constexpr int kEpiWarps = 8, kIssueWarp = 8, kProdWarp0 = 9, kProdWarps = 4;
 constexpr int kThreadsRU = (kProdWarp0 + kProdWarps) * 32;
 constexpr uint32_t kSpin = 1u << 18, kSuspend = 4000;
 enum { ERR_ROUTE = 64 };
 
-enum Bar { B_FULL = 0, B_EMPTY = kStages, B_AFULL = 2 * kStages, B_AEMPTY = 2 * kStages + 2, B_DRAIN = 2 * kStages + 4, B_COUNT };
+enum Bar { B_FULL = 0, B_EMPTY = kMaxStages, B_AFULL = 2 * kMaxStages, B_AEMPTY = 2 * kMaxStages + 2, B_DRAIN = 2 * kMaxStages + 4, B_COUNT };
 
 __device__ __forceinline__ uint32_t s_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void bar_init(uint32_t bar, uint32_t count)
@@ -115,8 +116,11 @@ template <int DIN>
 struct RU {
     static constexpr int CPR = DIN / 8;              // 16-byte chunks per row
     static constexpr int SBO = CPR * 128;            // bytes per group of 8 rows
-    static constexpr int TILE = kRows * DIN * 2;     // bytes of a 128-row tile
-    static constexpr int OFF_X = 0, OFF_W = TILE, OFF_BIAS = OFF_W + kStages * TILE,
+    static constexpr int XTILE = kRows * DIN * 2;    // bytes of the positions' tile
+    static constexpr int TILE = kTileN * DIN * 2;    // bytes of a weight tile
+    static constexpr int STAGES = DIN == 128 ? 2 : 4;
+    static constexpr int PPT = kProdWarps / STAGES;  // producer warps that share one tile (each stage has its own warps)
+    static constexpr int OFF_X = 0, OFF_W = XTILE, OFF_BIAS = OFF_W + STAGES * TILE,
                          OFF_MERGE = OFF_BIAS + kBiasSlots * kTileN * 4, OFF_BAR = OFF_MERGE + kRows * 8,
                          OFF_ABORT = OFF_BAR + 16 * 8, SMEM = OFF_ABORT + 16;
 };
@@ -147,8 +151,8 @@ __global__ void __launch_bounds__(kThreadsRU, 1)
     const int n_tiles = (m + kTileN - 1) / kTileN;
 
     if (tid == 0) {
-        for (int s = 0; s < kStages; ++s) {
-            bar_init(bar(B_FULL + s), 1);
+        for (int s = 0; s < L::STAGES; ++s) {
+            bar_init(bar(B_FULL + s), L::PPT);
             bar_init(bar(B_EMPTY + s), 1);
         }
         for (int e = 0; e < 2; ++e) {
@@ -160,7 +164,7 @@ __global__ void __launch_bounds__(kThreadsRU, 1)
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == kIssueWarp) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s_u32(&tmem_slot)), "r"(256)
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s_u32(&tmem_slot)), "r"(512)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -220,17 +224,15 @@ __global__ void __launch_bounds__(kThreadsRU, 1)
                     arg = j0 + 32 * c4 + first;
                 }
             };
-            wait_ld32(va);
-            ld32(tacc + 32, vb);
-            block(va, 0);
-            wait_ld32(vb);
-            ld32(tacc + 64, va);
-            block(vb, 1);
-            wait_ld32(va);
-            ld32(tacc + 96, vb);
-            block(va, 2);
-            wait_ld32(vb);
-            block(vb, 3);
+#pragma unroll 1
+            for (int c4 = 0; c4 < kTileN / 32; c4 += 2) {
+                wait_ld32(va);
+                ld32(tacc + 32 * (c4 + 1), vb);
+                block(va, c4);
+                wait_ld32(vb);
+                if (c4 + 2 < kTileN / 32) ld32(tacc + 32 * (c4 + 2), va);
+                block(vb, c4 + 1);
+            }
             tc_before();
             bar_arrive(bar(B_AEMPTY + e));
         }
@@ -254,8 +256,8 @@ __global__ void __launch_bounds__(kThreadsRU, 1)
         if (lane == 0) {
             constexpr uint32_t idesc = idesc_bf16(kRows, kTileN);
             for (int t = 0; t < n_tiles && ok; ++t) {
-                const int s = t % kStages, a = t & 1;
-                ok = bar_wait(bar(B_FULL + s), (t / kStages) & 1, abort_flag);
+                const int s = t % L::STAGES, a = t & 1;
+                ok = bar_wait(bar(B_FULL + s), (t / L::STAGES) & 1, abort_flag);
                 if (ok && t >= 2) ok = bar_wait(bar(B_AEMPTY + a), ((t >> 1) - 1) & 1, abort_flag);
                 if (!ok) break;
                 tc_after();
@@ -274,22 +276,25 @@ __global__ void __launch_bounds__(kThreadsRU, 1)
         }
         __syncwarp();
     } else {
-        // ------------------------------------------------------------ producers: tiles p, p + 4, ... into stage p
-        const int p = warp - kProdWarp0;
+        // ------------------------------------------------------------ producers
+        // warp p works for stage p % STAGES only (its waits on that stage's barriers are then in phase order) and
+        // copies part p / STAGES of each of that stage's tiles
+        const int p = warp - kProdWarp0, part = p / L::STAGES;
+        constexpr int kPartRows = kTileN / L::PPT;
         float* bias_s = reinterpret_cast<float*>(usm + L::OFF_BIAS);
-        for (int t = p; t < n_tiles && ok; t += kProdWarps) {
-            const int s = t % kStages, j0 = t * kTileN;
-            if (t >= kStages) ok = bar_wait(bar(B_EMPTY + s), ((t / kStages) - 1) & 1, abort_flag);
+        for (int t = p % L::STAGES; t < n_tiles && ok; t += L::STAGES) {
+            const int s = t % L::STAGES, j0 = t * kTileN;
+            if (t >= L::STAGES) ok = bar_wait(bar(B_EMPTY + s), ((t / L::STAGES) - 1) & 1, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             const uint32_t dst = sb + L::OFF_W + s * L::TILE;
-            for (int q = lane; q < kRows * L::CPR; q += 32) {
-                const int r = (q & 7) + 8 * (q / (8 * L::CPR)), c = (q >> 3) % L::CPR;
+            for (int q = lane; q < kPartRows * L::CPR; q += 32) {
+                const int r = part * kPartRows + (q & 7) + 8 * (q / (8 * L::CPR)), c = (q >> 3) % L::CPR;
                 const int j = min(j0 + r, m - 1);
                 cp16(dst + tile_off<DIN>(r, c), Wg + (int64_t)j * DIN + c * 8, 16u);
             }
             asm volatile("cp.async.commit_group;" ::: "memory");
-            for (int k = lane; k < kTileN; k += 32) {
+            for (int k = part * kPartRows + lane; k < (part + 1) * kPartRows; k += 32) {
                 const int j = j0 + k;
                 bias_s[(t % kBiasSlots) * kTileN + k] = j < m ? (bg ? __ldg(bg + j) : 0.f) : -CUDART_INF_F;
             }
@@ -304,7 +309,7 @@ __global__ void __launch_bounds__(kThreadsRU, 1)
     __syncthreads();
     tc_after();
     if (warp == kIssueWarp)
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(256) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512) : "memory");
     if (tid == 0 && *abort_flag) atomicOr(err_flag, ERR_ROUTE);
 }
 

@@ -1,12 +1,12 @@
 // Prefill router (Sec. 4.3) on the tcgen05 tensor cores: I[i][g] = lowest j maximising x_i . W_g[j] + b_g[j].
 //
-// One CTA owns 128 positions of one group.  Their inputs sit in shared memory once (A operand, K-major core-matrix
-// layout); the group's weight rows stream through a ring of stages in tiles of 256 entries (B operand, same
-// layout, 16-byte cp.async by four producer warps, each bound to one stage).  A tcgen05 instruction costs
-// its issuing thread about 100 clocks whatever its size, hence the widest tile the accumulators allow.  One
-// thread issues the 128 x 256 x d_in product of a tile into one of two TMEM accumulators (all 512 columns); two groups of four warps
-// (thread = position = TMEM lane) take turns reading an accumulator, add the bias, and keep a running (best score,
-// entry) in registers, so the score matrix never leaves the SM.  The two groups' results are merged at the end.
+// One CTA owns 256 positions of one group, as two blocks of 128.  Their inputs sit in shared memory once (A operand,
+// K-major core-matrix layout); the group's weight rows stream through a four-stage ring in tiles of 128 entries
+// (B operand, same layout, 16-byte cp.async by four producer warps, each bound to one stage), and every tile is
+// multiplied with both blocks, which halves the weight traffic out of L2 per product.  One thread issues the two
+// 128 x 128 x d_in products of a tile into the tile's two TMEM accumulators (two per block, alternating: all 512
+// columns); two groups of four warps, one per block (thread = position = TMEM lane), read their accumulator, add
+// the bias, and keep a running (best score, entry) in registers, so the score matrix never leaves the SM.
 // Every wait is bounded: a time-out raises the CTA's abort flag, the CTA drains, frees its TMEM, reports through
 // the error word and writes nothing.
 #include <cuda_bf16.h>
@@ -17,13 +17,14 @@
 namespace ckv {
 namespace {
 
-constexpr int kRows = 128, kTileN = 256, kMaxStages = 4, kBiasSlots = 8;
+constexpr int kRows = 256, kTileN = 128, kMaxStages = 4, kBiasSlots = 8;
 constexpr int kEpiWarps = 8, kIssueWarp = 8, kProdWarp0 = 9, kProdWarps = 4;
 constexpr int kThreadsRU = (kProdWarp0 + kProdWarps) * 32;
 constexpr uint32_t kSpin = 1u << 18, kSuspend = 4000;
 enum { ERR_ROUTE = 64 };
 
-enum Bar { B_FULL = 0, B_EMPTY = kMaxStages, B_AFULL = 2 * kMaxStages, B_AEMPTY = 2 * kMaxStages + 2, B_DRAIN = 2 * kMaxStages + 4, B_COUNT };
+// B_AFULL / B_AEMPTY: [2 * block + buffer]
+enum Bar { B_FULL = 0, B_EMPTY = kMaxStages, B_AFULL = 2 * kMaxStages, B_AEMPTY = 2 * kMaxStages + 4, B_DRAIN = 2 * kMaxStages + 8, B_COUNT };
 
 __device__ __forceinline__ uint32_t s_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void bar_init(uint32_t bar, uint32_t count)
@@ -118,11 +119,11 @@ struct RU {
     static constexpr int SBO = CPR * 128;            // bytes per group of 8 rows
     static constexpr int XTILE = kRows * DIN * 2;    // bytes of the positions' tile
     static constexpr int TILE = kTileN * DIN * 2;    // bytes of a weight tile
-    static constexpr int STAGES = DIN == 128 ? 2 : 4;
+    static constexpr int STAGES = 4;
     static constexpr int PPT = kProdWarps / STAGES;  // producer warps that share one tile (each stage has its own warps)
     static constexpr int OFF_X = 0, OFF_W = XTILE, OFF_BIAS = OFF_W + STAGES * TILE,
-                         OFF_MERGE = OFF_BIAS + kBiasSlots * kTileN * 4, OFF_BAR = OFF_MERGE + kRows * 8,
-                         OFF_ABORT = OFF_BAR + 16 * 8, SMEM = OFF_ABORT + 16;
+                         OFF_BAR = OFF_BIAS + kBiasSlots * kTileN * 4,
+                         OFF_ABORT = OFF_BAR + 24 * 8, SMEM = OFF_ABORT + 16;
 };
 // byte offset of (row r, 16-byte chunk c) in the K-major core-matrix layout: 8 x 16-byte core matrices, chunks of a
 // row group 128 bytes apart, row groups SBO apart
@@ -155,7 +156,7 @@ __global__ void __launch_bounds__(kThreadsRU, 1)
             bar_init(bar(B_FULL + s), L::PPT);
             bar_init(bar(B_EMPTY + s), 1);
         }
-        for (int e = 0; e < 2; ++e) {
+        for (int e = 0; e < 4; ++e) {
             bar_init(bar(B_AFULL + e), 1);
             bar_init(bar(B_AEMPTY + e), 128);
         }
@@ -185,15 +186,17 @@ __global__ void __launch_bounds__(kThreadsRU, 1)
 
     if (warp < kEpiWarps) {
         // ------------------------------------------------------------ running arg-max, thread = position
-        const int e = warp >> 2, row = (warp & 3) * 32 + lane;
-        const uint32_t tacc = tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(kTileN * e);
+        const int e = warp >> 2, row = 128 * e + (warp & 3) * 32 + lane;  // block e, position row of the CTA
+        const uint32_t tacc0 = tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(2 * kTileN * e);
         float best = -CUDART_INF_F;
         int arg = 0;
-        for (int t = e; t < n_tiles && ok; t += 2) {
-            ok = bar_wait(bar(B_AFULL + e), (t >> 1) & 1, abort_flag);
+        for (int t = 0; t < n_tiles && ok; ++t) {
+            const int a = t & 1;
+            ok = bar_wait(bar(B_AFULL + 2 * e + a), (t >> 1) & 1, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_after();
+            const uint32_t tacc = tacc0 + (uint32_t)(kTileN * a);
             const float4* bs = reinterpret_cast<const float4*>(usm + L::OFF_BIAS) + (t % kBiasSlots) * (kTileN / 4);
             const int j0 = t * kTileN;
             // 32 columns at a time, the next 32 already on their way out of TMEM.  Only the maximum of a block is
@@ -234,39 +237,30 @@ __global__ void __launch_bounds__(kThreadsRU, 1)
                 block(vb, c4 + 1);
             }
             tc_before();
-            bar_arrive(bar(B_AEMPTY + e));
+            bar_arrive(bar(B_AEMPTY + 2 * e + a));
         }
-        // merge the two groups (they saw disjoint tiles): larger score, lowest entry among equals
-        float* mv = reinterpret_cast<float*>(usm + L::OFF_MERGE);
-        int* mi = reinterpret_cast<int*>(usm + L::OFF_MERGE + kRows * 4);
-        if (e == 1) {
-            mv[row] = best;
-            mi[row] = arg;
-        }
-        asm volatile("bar.sync 1, 256;" ::: "memory");
-        if (e == 0 && ok && !*abort_flag) {
-            const float v2 = mv[row];
-            const int i2 = mi[row];
-            if (v2 > best || (v2 == best && i2 < arg)) arg = i2;
-            if (row0 + row < n) out[(row0 + row) * G + grp] = arg;
-        }
+        if (ok && !*abort_flag && row0 + row < n) out[(row0 + row) * G + grp] = arg;
         if (!ok) *abort_flag = 1;
     } else if (warp == kIssueWarp) {
         // ------------------------------------------------------------ MMA issue
         if (lane == 0) {
-            constexpr uint32_t idesc = idesc_bf16(kRows, kTileN);
+            constexpr uint32_t idesc = idesc_bf16(128, kTileN);
             for (int t = 0; t < n_tiles && ok; ++t) {
                 const int s = t % L::STAGES, a = t & 1;
                 ok = bar_wait(bar(B_FULL + s), (t / L::STAGES) & 1, abort_flag);
-                if (ok && t >= 2) ok = bar_wait(bar(B_AEMPTY + a), ((t >> 1) - 1) & 1, abort_flag);
-                if (!ok) break;
-                tc_after();
+                for (int e = 0; e < 2 && ok; ++e) {
+                    if (t >= 2) ok = bar_wait(bar(B_AEMPTY + 2 * e + a), ((t >> 1) - 1) & 1, abort_flag);
+                    if (!ok) break;
+                    tc_after();
 #pragma unroll
-                for (int ks = 0; ks < DIN / 16; ++ks)
-                    mma_ss(tmem + (uint32_t)(kTileN * a), mat_desc(sb + L::OFF_X + ks * 256, 128, L::SBO),
-                           mat_desc(sb + L::OFF_W + s * L::TILE + ks * 256, 128, L::SBO), idesc, ks > 0 ? 1u : 0u);
+                    for (int ks = 0; ks < DIN / 16; ++ks)
+                        mma_ss(tmem + (uint32_t)(kTileN * (2 * e + a)),
+                               mat_desc(sb + L::OFF_X + e * 16 * L::SBO + ks * 256, 128, L::SBO),
+                               mat_desc(sb + L::OFF_W + s * L::TILE + ks * 256, 128, L::SBO), idesc, ks > 0 ? 1u : 0u);
+                    tc_commit_to(bar(B_AFULL + 2 * e + a));
+                }
+                if (!ok) break;
                 tc_commit_to(bar(B_EMPTY + s));
-                tc_commit_to(bar(B_AFULL + a));
             }
             if (!ok) *abort_flag = 1;
             // nothing of this CTA may still run on the tensor core at teardown

@@ -13,7 +13,7 @@
  *   target attention: every query is an independent 1 x d row):
  *     softmax mode : s_i = scale * <q, K[i]>,  p = softmax_i(s),  o = sum_i p_i V[i]
  *     pointwise    : o = (1/L_u) * sum_i silu(s_i) V[i],  silu(x) = x / (1 + exp(-x))
- *   A user with L_u = 0 yields a zero output row (reading chosen by this build).
+ *   A user with L_u = 0 yields a zero output row (the paper does not define the case).
  *
  * Inputs are taken at their stored precision (float32, or bfloat16 bit patterns
  * widened exactly); all arithmetic is double.  No blocking, no online softmax,

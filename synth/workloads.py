@@ -1,6 +1,6 @@
 """Workload shapes and the seeded generator of synthetic decode-stage inputs.
 
-The five named workloads follow the benchmark configurations of this build
+The five named workloads are the benchmark configurations of this library
 (SASRec-style target attention, an HSTU-style pointwise config, long ragged
 histories and a high-concurrency serving batch).  They stand in for the
 paper's MicroVideo / KuaiVideo / EBNeRD workloads (Sec. 5.1), which are not

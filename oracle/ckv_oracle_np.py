@@ -48,3 +48,36 @@ def attend(mode: str, scale: float, pool_K, pool_V, hist_off, idx_K, idx_V, user
                 W = S / (1.0 + np.exp(-S)) / L
             out[q0:q1, g] = W @ V[:, g]
     return out
+
+
+def attend_variants(mode: str, scale: float, d_a: int, pool_K, pool_V, hist_off, idx_K, idx_V, user_K, user_V,
+                    q_off, queries, vis=None) -> np.ndarray:
+    """The same second formulation for the variants: a side whose pool is None is taken as cached full-width
+    rows (sharing only keys or only values, Sec. 5.5), and `vis` gives every query row the number of leading
+    positions it may see (self-attention over the cached sequence, Sec. 2.1), applied as a boolean mask on the
+    full score matrix."""
+    G = queries.shape[1]
+    U = len(hist_off) - 1
+    out = np.zeros((int(q_off[-1]), G, d_a), dtype=np.float64)
+    qf = _f64(queries)
+    for u in range(U):
+        p0, L = int(hist_off[u]), int(hist_off[u + 1] - hist_off[u])
+        q0, q1 = int(q_off[u]), int(q_off[u + 1])
+        if L == 0 or q1 == q0:
+            continue
+        K = _f64(user_K[p0:p0 + L]) if pool_K is None else materialize_f64(pool_K, idx_K, user_K, p0, L)
+        V = _f64(user_V[p0:p0 + L]) if pool_V is None else materialize_f64(pool_V, idx_V, user_V, p0, L)
+        n_vis = np.full(q1 - q0, L) if vis is None else np.asarray(vis[q0:q1])
+        seen = np.arange(L)[None, :] < n_vis[:, None]        # [M, L]
+        for g in range(G):
+            S = scale * (qf[q0:q1, g] @ K[:, g].T)           # [M, L]
+            if mode == "softmax":
+                Sm = np.where(seen, S, -np.inf)
+                mx = Sm.max(axis=1, keepdims=True)
+                E = np.exp(Sm - np.where(np.isfinite(mx), mx, 0.0))   # exp(-inf) = 0 for what is not seen
+                Z = E.sum(axis=1, keepdims=True)
+                W = np.divide(E, Z, out=np.zeros_like(E), where=Z > 0)
+            else:
+                W = np.where(seen, S / (1.0 + np.exp(-S)), 0.0) / L
+            out[q0:q1, g] = W @ V[:, g]
+    return out

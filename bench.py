@@ -1,21 +1,31 @@
 #!/usr/bin/env python
 """Benchmark of the CollectiveKV decode path (one `ckv_attend` over all users of a workload).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload all|cfg2|...] [--impl ours|reference]
 
 Prints ONE JSON line.  A step = one pass of the whole hot path (compressed-cache read, pool
 gather, concat, scores, normalisation, weighted sum, split merge, store) over the workload,
 with pool and caches resident in HBM.  `value` is cached history positions per second over all
 ranks (device time, max over ranks); `e2e` is the same call fed with host buffers (query
-upload and output download inside the timed region).  Under torchrun each rank serves its own
+upload and output download inside the timed region), `e2e_fresh_plan` the same with a request
+list the library has not seen before on every call.  Under torchrun each rank serves its own
 users (weak scaling, no collective on the data path).
+
+With `--workload all` (the default) the four large workloads run one after the other in this
+process; the line's top-level figures are those of the largest one (cfg5: most positions and
+bytes) and `per_config` carries the figures of each.  Per workload: W warm-up steps, a sampled
+parity check, then at least one second of back-to-back steps (the SM clock settles to what it
+sustains under this load; every step is timed and the clock is sampled throughout), a
+synchronise, and the K timed steps of the headline figure.
 
 `--impl reference` times the CPU oracle, as it stands, on this machine's host cores.
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
+import math
 import os
 import statistics
 import sys
@@ -33,8 +43,17 @@ import synth  # noqa: E402
 METRIC = "cached_history_positions_per_sec"
 UNIT = "positions/s"
 HBM_FALLBACK_GBS = 6650.0
-# users of the workload the CPU oracle is timed on (about 10-30 s of host work)
-CPU_SAMPLE_USERS = {"cfg1": 64, "cfg2": 1024, "cfg3": 256, "cfg4": 690900000, "cfg5": 32768}
+ALL_WORKLOADS = ("cfg2", "cfg3", "cfg4", "cfg5")
+HEADLINE = "cfg5"            # the largest single-GPU workload: most positions and most bytes
+SUSTAIN_SECONDS = 1.0        # back-to-back load per workload before (and around) the timed steps
+CPU_SECONDS = {"headline": 15.0, "other": 4.0}   # host time the oracle leg may take per workload
+# transcendental evaluations per SM per clock (ex2 / tanh issue rate of the special-function unit)
+XU_PER_SM_CLK = 16
+# bytes per SM per clock through the L1 / shared-memory data pipe (one 128-byte wavefront per clock)
+L1_PIPE_BYTES_PER_SM_CLK = 128
+TRAFFIC_JSON = os.path.join(ROOT, "profiles", "traffic.json")
+CSRC = os.path.join(ROOT, "paper_2601_19178_b200", "csrc")
+KERNEL_SOURCES = {1: ["kernels_simt.cu"], 2: ["kernels_mma.cu"], 3: ["kernels_umma.cu"], 4: ["kernels_fact.cu"]}
 
 
 def _peaks():
@@ -47,20 +66,61 @@ def _peaks():
     return HBM_FALLBACK_GBS, "fallback"
 
 
-# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel,
-# from the ncu captures summarised under profiles/ (attend_*_<workload>.md; cfg4: the three launches of
-# the factorised path together, which is also what the timed interval covers).  cfg3 and cfg5
-# were captured on a cut of the workload and scaled by the number of users.  Set an entry to None
-# when its kernel changes after the capture.
-TRAFFIC_BYTES = {"cfg2": 190658560, "cfg3": 1090254848, "cfg4": 690900000, "cfg5": 1852809216}
-# transcendental evaluations per SM per clock (ex2 / tanh issue rate of the special-function unit)
-XU_PER_SM_CLK = 16
-# bytes per SM per clock through the L1 / shared-memory data pipe (one 128-byte wavefront per clock)
-L1_PIPE_BYTES_PER_SM_CLK = 128
+def source_hash(family: int) -> str:
+    """Hash of the source of a kernel family (and the shared device helpers): the DRAM-traffic record of a
+    kernel is only valid for the source it was captured from."""
+    h = hashlib.sha256()
+    for name in KERNEL_SOURCES.get(family, []) + ["ptx_helpers.cuh", "ckv_internal.h"]:
+        path = os.path.join(CSRC, name)
+        if os.path.exists(path):
+            h.update(open(path, "rb").read())
+    return h.hexdigest()[:16]
 
 
-def _traffic(workload: str, full_size: bool):
-    return TRAFFIC_BYTES.get(workload) if full_size else None
+def _traffic(entry: str, family: int, users: int):
+    """DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the workload's attend kernel(s),
+    from the record `--record-traffic` wrote after an ncu capture (profiles/traffic.json), scaled by the number
+    of users when the capture ran on a cut of the workload (users are independent: traffic grows in proportion).
+    None when there is no record or the kernel's source has changed since."""
+    try:
+        rec = json.load(open(TRAFFIC_JSON)).get(entry)
+    except Exception:
+        return None
+    if not rec or rec.get("source_hash") != source_hash(family) or rec.get("kernel_family") != family:
+        return None
+    return rec["dram_bytes"] * users / rec["users"]
+
+
+def record_traffic(args):
+    """Reads `ncu -i <rep> --page raw --csv` output and stores the DRAM bytes of the captured attend launch(es)
+    in profiles/traffic.json under the entry name given.  Runs here, without a GPU."""
+    import csv
+    rows = list(csv.reader(open(args.record_traffic)))
+    hdr = next(i for i, r in enumerate(rows) if "Kernel Name" in r)
+    cols = rows[hdr]
+    ci = {c: i for i, c in enumerate(cols)}
+    units = rows[hdr + 1]
+    total, names = 0.0, []
+    for r in rows[hdr + 2:]:
+        if len(r) != len(cols):
+            continue
+        name = r[ci["Kernel Name"]]
+        if not any(k in name for k in ("attend_", "fact_", "combine_kernel")):
+            continue
+        for m in ("dram__bytes_read.sum", "dram__bytes_write.sum"):
+            v = float(r[ci[m]].replace(",", ""))
+            u = units[ci[m]].lower()
+            total += v * {"byte": 1.0, "kbyte": 1e3, "mbyte": 1e6, "gbyte": 1e9}[u]
+        names.append(name.split("(")[0])
+    w = synth.WORKLOADS[args.workload if args.workload != "all" else HEADLINE]
+    data = {}
+    if os.path.exists(TRAFFIC_JSON):
+        data = json.load(open(TRAFFIC_JSON))
+    data[args.entry] = {"workload": w.name, "users": args.users or w.n_users, "kernel_family": args.family,
+                        "kernels": names, "dram_bytes": total, "source_hash": source_hash(args.family),
+                        "from": os.path.basename(args.record_traffic)}
+    json.dump(data, open(TRAFFIC_JSON, "w"), indent=1, sort_keys=True)
+    print(json.dumps(data[args.entry]))
 
 
 class ClockSampler(threading.Thread):
@@ -108,14 +168,19 @@ class ClockSampler(threading.Thread):
     def off(self):
         self._on.clear()
 
+    def take(self):
+        """Summary of the samples since the last call."""
+        s, r = self.samples, sorted(self.reasons)
+        self.samples, self.reasons = [], set()
+        return {"sm_mhz": statistics.median(s) if s else None, "sm_min_mhz": min(s) if s else None,
+                "sm_max_mhz": self.max_mhz, "reasons": r, "samples": len(s)}
+
     def finish(self):
         self._stop_evt.set()
-        return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
-                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
 def _oracle_rate(w, data, n_users: int, n_threads: int = 0):
-    """Times the CPU oracle on the first n_users users; returns (positions/s, seconds, cores)."""
+    """Times the CPU oracle on the first n_users users; returns (positions/s, seconds, cores, users, positions)."""
     from oracle import ckv_oracle as O
     n_users = min(n_users, w.n_users)
     sel = np.arange(n_users, dtype=np.int64)
@@ -126,6 +191,16 @@ def _oracle_rate(w, data, n_users: int, n_threads: int = 0):
     dt = time.perf_counter() - t0
     pos = int(data["hist_off"][n_users])
     return pos / dt, dt, O.max_threads(), n_users, pos
+
+
+def _oracle_sample(w, data, seconds: float):
+    """The oracle on a bounded sample of the workload: a short probe sizes the sample to about `seconds`."""
+    probe_users = max(1, min(w.n_users, 8))
+    _, probe_dt, _, _, _ = _oracle_rate(w, data, probe_users)
+    n_users = int(max(probe_users, min(w.n_users, seconds * probe_users / max(probe_dt, 1e-9))))
+    rate, dt, cores, n_u, pos = _oracle_rate(w, data, n_users)
+    return {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"first {n_u} of {w.n_users} users ({pos} positions), {dt:.1f} s"}
 
 
 def rank_env():
@@ -152,27 +227,45 @@ def reduce_over_ranks(elapsed, positions: int, users: int, dist=None, device="cp
     return float(t.item()), int(c[0].item()), int(c[1].item())
 
 
-def run_reference(args, w):
-    """The oracle, as it stands, on the host cores: each step is a bounded sample of users."""
+def workload_list(args):
+    names = ALL_WORKLOADS if args.workload == "all" else (args.workload,)
+    ws = []
+    for n in names:
+        w = synth.WORKLOADS[n]
+        if args.users:
+            w = synth.scaled(w, n_users=min(args.users, w.n_users))
+        ws.append(w)
+    return ws
+
+
+def run_reference(args):
+    """The oracle, as it stands, on the host cores: each step is a bounded sample of users of the headline
+    workload (the same workload the CUDA arm puts at the top level of its line)."""
     rank, _, _ = rank_env()
     if rank != 0:
         return
-    data = synth.generate(w)
+    ws = workload_list(args)
+    w = next((x for x in ws if x.name == HEADLINE), ws[-1])
+    # the oracle only touches the users it computes: generate a cut that holds the per-step sample
+    gen_users = min(w.n_users, 4096)
+    wg = synth.scaled(w, n_users=gen_users)
+    data = synth.generate(wg)
     # size the per-step sample from a short probe so the whole run stays within ~2 minutes
-    probe_users = max(1, min(w.n_users, 8))
-    _, probe_dt, cores, _, _ = _oracle_rate(w, data, probe_users)
+    probe_users = max(1, min(gen_users, 8))
+    _, probe_dt, cores, _, _ = _oracle_rate(wg, data, probe_users)
     per_user = probe_dt / probe_users
     budget = 100.0 / max(1, args.steps + args.warmup)
-    n_users = int(max(1, min(w.n_users, budget / max(per_user, 1e-9))))
+    n_users = int(max(1, min(gen_users, budget / max(per_user, 1e-9))))
     for _ in range(args.warmup):
-        _oracle_rate(w, data, n_users)
+        _oracle_rate(wg, data, n_users)
     times, pos = [], 0
     for _ in range(args.steps):
-        _, dt, cores, _, pos = _oracle_rate(w, data, n_users)
+        _, dt, cores, _, pos = _oracle_rate(wg, data, n_users)
         times.append(dt)
     total = sum(times)
     value = pos * args.steps / total
-    sample = f"first {n_users} of {w.n_users} users ({pos} positions) per step"
+    sample = (f"first {n_users} of {w.n_users} users ({pos} positions) per step; a rate over a sample of the "
+              f"workload, not a pass over all of it")
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
@@ -187,10 +280,228 @@ def run_reference(args, w):
     print(json.dumps(line), flush=True)
 
 
-def run_ours(args, w):
+class Measured:
+    """One workload loaded into a library context on this rank, and the measurements taken on it."""
+
+    def __init__(self, args, w, rank, local, dist, sampler):
+        import torch
+        import paper_2601_19178_b200 as ckv
+        from paper_2601_19178_b200.session import as_device_tensor as dev
+        self.torch, self.ckv, self.args, self.w, self.rank, self.local = torch, ckv, args, w, rank, local
+        self.dist, self.sampler = dist, sampler
+        # weak scaling: every rank serves its own users of the same workload shape
+        self.data = data = synth.generate(w, seed=rank_seed(w, rank))
+        tdt = torch.float32 if w.dtype == "f32" else torch.bfloat16
+        self.s = s = ckv.CollectiveKV(w.n_groups, w.head_dim, tdt, w.mode, device=local)
+        s.pool_load(dev(data["pool_K"], w.dtype), dev(data["pool_V"], w.dtype))
+        ik, iv = dev(data["idx_K"], "i"), dev(data["idx_V"], "i")
+        uk, uv = dev(data["user_K"], w.dtype), dev(data["user_V"], w.dtype)
+        s.cache_put_batch(data["users"], data["hist_off"], ik, iv, uk, uv)
+        del ik, iv, uk, uv
+        torch.cuda.empty_cache()
+        if args.split_len:
+            s.set_option("split_len", args.split_len)
+        if args.mma_loader:
+            s.set_option("mma_loader", args.mma_loader)
+        if args.l2_persist >= 0:
+            s.set_option("l2_persist", args.l2_persist)
+        s.set_option("time_kernels", 1)
+        self.users, self.q_off = data["users"], data["q_off"]
+        self.q = dev(data["queries"], w.dtype)
+        self.out = torch.empty_like(self.q)
+        self.positions = int(data["hist_off"][-1])
+        self.comp_bytes, self.full_bytes = ckv.ckv_cache_bytes(s.ctx)
+        self.qo_bytes = self.q.numel() * self.q.element_size() + self.out.numel() * self.out.element_size()
+        self.algo_bytes = self.comp_bytes + self.qo_bytes
+        # L2 flush between timed iterations: overwrite a buffer twice the size of L2
+        self.flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
+        self.stream = torch.cuda.current_stream()
+        self.q_host = self.o_host = None
+
+    def close(self):
+        self.s.close()
+        del self.q, self.out, self.flush, self.q_host, self.o_host, self.data
+        self.torch.cuda.empty_cache()
+
+    def step(self):
+        self.s.attend(self.users, self.q_off, self.q, self.out)
+
+    def parity(self):
+        from oracle import ckv_oracle as O
+        torch, w, data = self.torch, self.w, self.data
+        rng = np.random.default_rng(0)
+        lens = np.diff(data["hist_off"])
+        sel = sorted(set([0, w.n_users - 1, int(np.argmax(lens)), int(np.argmin(lens))] +
+                         rng.integers(0, w.n_users, size=4).tolist()))
+        want = O.attend(w.dtype, w.mode, w.default_scale, data["pool_K"], data["pool_V"], data["hist_off"],
+                        data["idx_K"], data["idx_V"], data["user_K"], data["user_V"], data["q_off"],
+                        data["queries"], sel=sel)
+        rows = np.concatenate([np.arange(self.q_off[u], self.q_off[u + 1]) for u in sel])
+        got = self.out[torch.from_numpy(rows).cuda()].float().cpu().numpy().astype(np.float64)
+        atol, rtol = (1e-5, 1e-5) if w.dtype == "f32" else (2e-3, 1e-2)
+        err = np.abs(got - want)
+        ok = bool((err <= atol + rtol * np.abs(want)).all())
+        rown = float((err.max(axis=-1) / np.maximum(np.abs(want).max(axis=-1), 1e-30)).max())
+        return {"users_checked": len(sel), "ok": ok, "max_abs_err": float(err.max()), "row_norm_err": rown}
+
+    def timed_steps(self, n_steps):
+        """n_steps back-to-back steps (L2 flushed before each), every step timed with CUDA events on the
+        launching stream; the library's own events around the attend kernel are read every 32nd step."""
+        torch, s = self.torch, self.s
+        ev0 = [torch.cuda.Event(enable_timing=True) for _ in range(n_steps)]
+        ev1 = [torch.cuda.Event(enable_timing=True) for _ in range(n_steps)]
+        kern_ns, comb_ns, launches = [], [], 0
+        for i in range(n_steps):
+            self.flush.zero_()
+            ev0[i].record(self.stream)
+            self.step()
+            ev1[i].record(self.stream)
+            launches += s.stat("launches")
+            if i % 32 == 31 or i == n_steps - 1:
+                kern_ns.append(s.stat("main_kernel_ns"))
+                comb_ns.append(s.stat("combine_kernel_ns"))
+        torch.cuda.synchronize()
+        step_ms = [a.elapsed_time(b) for a, b in zip(ev0, ev1)]
+        return step_ms, kern_ns, comb_ns, launches
+
+    def e2e(self, fresh_plans: bool):
+        """Host query buffer in, host output buffer out, through the same C-ABI call; host wall clock around
+        call + synchronise.  fresh_plans: every call carries a request list (a rotation through nine
+        permutations of the users) that is not among the plans the library keeps."""
+        torch, s = self.torch, self.s
+        if self.q_host is None:
+            self.q_host = torch.empty(self.q.shape, dtype=self.q.dtype).pin_memory()
+            self.q_host.copy_(self.q)
+            self.o_host = torch.empty(self.out.shape, dtype=self.out.dtype).pin_memory()
+        lists = [(self.users, self.q_off)]
+        if fresh_plans:
+            # all users of a workload have the same number of queries, so q_off stays as it is
+            rng = np.random.default_rng(11)
+            lists = [(np.ascontiguousarray(self.users[rng.permutation(self.w.n_users)]), self.q_off) for _ in range(9)]
+        n = max(3, min(self.args.steps, 20))
+        if fresh_plans:
+            n = max(n, len(lists))
+        for k in range(2 if not fresh_plans else len(lists)):
+            s.attend(lists[k % len(lists)][0], lists[k % len(lists)][1], self.q_host, self.o_host)
+        torch.cuda.synchronize()
+        if self.dist is not None:
+            self.dist.barrier()
+        hits = allocs = 0
+        t0 = time.perf_counter()
+        for k in range(n):
+            u, qo = lists[k % len(lists)]
+            s.attend(u, qo, self.q_host, self.o_host)
+            torch.cuda.synchronize()
+            hits += s.stat("plan_cache_hit")
+            allocs += s.stat("alloc_calls")
+        secs, pos, _ = reduce_over_ranks(time.perf_counter() - t0, self.positions, self.w.n_users, self.dist, "cuda")
+        return {"value": pos * n / secs, "unit": UNIT,
+                "h2d_bytes_per_step": self.q_host.numel() * self.q_host.element_size() + self.users.nbytes + self.q_off.nbytes,
+                "d2h_bytes_per_step": self.o_host.numel() * self.o_host.element_size(),
+                "ms_per_step": 1e3 * secs / n, "steps": n, "plan_cache_hits": hits, "alloc_calls": allocs}
+
+    def measure(self, entry: str, kernel: int, cpu_seconds: float):
+        """The whole protocol for one kernel choice on the loaded workload; returns the entry of `per_config`."""
+        torch, s, w, args = self.torch, self.s, self.w, self.args
+        s.set_option("kernel", kernel)
+        warm = max(args.warmup, 3)
+        t_probe = []
+        for _ in range(warm):
+            self.flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(self.stream)
+            self.step()
+            e1.record(self.stream)
+            t_probe.append((e0, e1))
+        torch.cuda.synchronize()
+        est_ms = max(1e-3, min(a.elapsed_time(b) for a, b in t_probe))
+        parity = self.parity() if (self.rank == 0 and not args.no_check) else None
+
+        # sustained load: at least SUSTAIN_SECONDS of back-to-back steps, then the K timed steps behind a synchronise
+        n_sustain = max(args.steps, int(math.ceil(1e3 * args.sustain / est_ms)))
+        if self.dist is not None:
+            self.dist.barrier()
+        torch.cuda.synchronize()
+        if self.sampler:
+            self.sampler.take()
+            self.sampler.on()
+        sus_ms, sus_kern, sus_comb, sus_launches = self.timed_steps(n_sustain)
+        if self.dist is not None:
+            self.dist.barrier()
+        torch.cuda.synchronize()
+        step_ms, kern_ns, comb_ns, launches = self.timed_steps(args.steps)
+        if self.sampler:
+            self.sampler.off()
+        if self.dist is not None:
+            self.dist.barrier()
+        clocks = self.sampler.take() if self.sampler else None
+        total_ms, job_pos, job_users = reduce_over_ranks(float(sum(step_ms)), self.positions, w.n_users, self.dist, "cuda")
+        sus_total_ms, _, _ = reduce_over_ranks(float(sum(sus_ms)), self.positions, w.n_users, self.dist, "cuda")
+        e2e = self.e2e(False)
+        e2e_fresh = self.e2e(True)
+        dev_err = s.stat("device_errors")
+        if dev_err:
+            raise SystemExit(f"{entry}: a kernel gave up on a bounded wait (device_errors = {dev_err})")
+        if self.rank != 0:
+            return None
+
+        peak, peak_kind = _peaks()
+        kern_s = statistics.mean(kern_ns) * 1e-9
+        sus_kern_s = statistics.mean(sus_kern) * 1e-9
+        family = s.stat("kernel")
+        achieved = self.algo_bytes / kern_s / 1e9
+        mhz = clocks["sm_mhz"] if clocks and clocks.get("sm_mhz") else None
+        cpu = None if args.no_cpu else _oracle_sample(w, self.data, cpu_seconds)
+        # The roof that binds, reported beside the HBM roofline the metric asks for.
+        # Many queries per user (tcgen05 kernel): one exp (softmax) or tanh (SiLU) per score on the
+        # special-function unit.  Few queries (warp-level tensor-core kernel): every gathered pool row crosses
+        # the SM's L1 / shared-memory data pipe twice, once copied into the staging ring and once read
+        # out by ldmatrix; the pool rows come from L2, not HBM.
+        binding = None
+        n_sms = torch.cuda.get_device_properties(self.local).multi_processor_count
+        max_mhz = clocks["sm_max_mhz"] if clocks and clocks.get("sm_max_mhz") else None
+        if family == 2 and max_mhz:
+            pipe_bytes = float(self.positions) * w.n_groups * 2 * (w.head_dim * 2) * 2
+            peak_pipe = L1_PIPE_BYTES_PER_SM_CLK * n_sms * max_mhz * 1e6 / 1e9
+            binding = {"bound": "l1_shared_data_pipe",
+                       "what": "K and V pool rows into the shared-memory ring and out through ldmatrix",
+                       "achieved": pipe_bytes / kern_s / 1e9, "peak": peak_pipe, "unit": "GB/s",
+                       "frac": pipe_bytes / kern_s / 1e9 / peak_pipe}
+        elif family == 3 and max_mhz:
+            scores = float(self.positions) * w.n_groups * w.n_queries
+            peak_xu = XU_PER_SM_CLK * n_sms * max_mhz * 1e6 / 1e9
+            binding = {"bound": "alu", "what": "one ex2/tanh per score on the special-function unit",
+                       "achieved": scores / kern_s / 1e9, "peak": peak_xu, "unit": "Gscore/s",
+                       "frac": scores / kern_s / 1e9 / peak_xu}
+        return {
+            "entry": entry, "workload": w.name, "describe": w.describe, "users": w.n_users, "positions": self.positions,
+            "value": job_pos * args.steps / (total_ms * 1e-3), "unit": UNIT,
+            "users_per_sec": job_users * args.steps / (total_ms * 1e-3),
+            "steps": args.steps, "ms_per_step": total_ms / args.steps,
+            "sustained": {"steps": n_sustain, "seconds": sus_total_ms * 1e-3, "ms_per_step": sus_total_ms / n_sustain,
+                          "value": job_pos * n_sustain / (sus_total_ms * 1e-3), "kernel_us": sus_kern_s * 1e6,
+                          "what": "back-to-back steps directly before the timed ones, every step timed"},
+            "kernel_family": family, "kernel_option": kernel, "mma_loader": s.stat("mma_loader"),
+            "work_items": s.stat("work_items"), "split_items": s.stat("split_items"),
+            "l2_window": s.stat("l2_window"),
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": _traffic(entry, family, w.n_users), "peak_kind": peak_kind,
+                         "algorithmic_bytes": self.algo_bytes, "kernel_us": kern_s * 1e6,
+                         "kernel_us_x_sm_mhz": kern_s * 1e6 * mhz if mhz else None,
+                         "combine_us": statistics.mean(comb_ns) * 1e-3, "frac_of_nominal_8TBs": achieved / 8000.0},
+            "roofline_binding": binding,
+            "clocks": clocks,
+            "e2e": e2e, "e2e_fresh_plan": e2e_fresh,
+            "gpu_launches": launches, "gpu_launches_sustained": sus_launches,
+            "cpu_baseline": cpu,
+            "parity": parity,
+            "compression": {"compressed_bytes": self.comp_bytes, "full_width_bytes": self.full_bytes,
+                            "ratio": self.comp_bytes / max(self.full_bytes, 1)},
+        }
+
+
+def run_ours(args):
     import torch
-    import paper_2601_19178_b200 as ckv
-    from paper_2601_19178_b200.session import as_device_tensor as dev
 
     rank, world, local = rank_env()
     if not torch.cuda.is_available():
@@ -200,63 +511,6 @@ def run_ours(args, w):
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-
-    # weak scaling: every rank serves its own users of the same workload shape
-    data = synth.generate(w, seed=rank_seed(w, rank))
-    tdt = torch.float32 if w.dtype == "f32" else torch.bfloat16
-    s = ckv.CollectiveKV(w.n_groups, w.head_dim, tdt, w.mode, device=local)
-    s.pool_load(dev(data["pool_K"], w.dtype), dev(data["pool_V"], w.dtype))
-    ik, iv = dev(data["idx_K"], "i"), dev(data["idx_V"], "i")
-    uk, uv = dev(data["user_K"], w.dtype), dev(data["user_V"], w.dtype)
-    s.cache_put_batch(data["users"], data["hist_off"], ik, iv, uk, uv)
-    del ik, iv, uk, uv
-    torch.cuda.empty_cache()
-    if args.kernel:
-        s.set_option("kernel", args.kernel)
-    if args.split_len:
-        s.set_option("split_len", args.split_len)
-    if args.mma_loader:
-        s.set_option("mma_loader", args.mma_loader)
-    s.set_option("time_kernels", 1)
-    users, q_off = data["users"], data["q_off"]
-    q = dev(data["queries"], w.dtype)
-    out = torch.empty_like(q)
-    positions = int(data["hist_off"][-1])
-    comp_bytes, full_bytes = ckv.ckv_cache_bytes(s.ctx)
-    qo_bytes = q.numel() * q.element_size() + out.numel() * out.element_size()
-    algo_bytes = comp_bytes + qo_bytes
-
-    # L2 flush between timed iterations: overwrite a buffer twice the size of L2
-    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
-    stream = torch.cuda.current_stream()
-
-    def step():
-        s.attend(users, q_off, q, out)
-
-    for _ in range(max(args.warmup, 3)):
-        flush.zero_()
-        step()
-    torch.cuda.synchronize()
-
-    # parity spot check on sampled users, in the launch configuration that is timed
-    parity = None
-    if rank == 0 and not args.no_check:
-        from oracle import ckv_oracle as O
-        rng = np.random.default_rng(0)
-        lens = np.diff(data["hist_off"])
-        sel = sorted(set([0, w.n_users - 1, int(np.argmax(lens)), int(np.argmin(lens))] +
-                         rng.integers(0, w.n_users, size=4).tolist()))
-        want = O.attend(w.dtype, w.mode, w.default_scale, data["pool_K"], data["pool_V"], data["hist_off"],
-                        data["idx_K"], data["idx_V"], data["user_K"], data["user_V"], data["q_off"],
-                        data["queries"], sel=sel)
-        rows = np.concatenate([np.arange(q_off[u], q_off[u + 1]) for u in sel])
-        got = out[torch.from_numpy(rows).cuda()].float().cpu().numpy().astype(np.float64)
-        atol, rtol = (1e-5, 1e-5) if w.dtype == "f32" else (2e-3, 1e-2)
-        err = np.abs(got - want)
-        ok = bool((err <= atol + rtol * np.abs(want)).all())
-        rown = float((err.max(axis=-1) / np.maximum(np.abs(want).max(axis=-1), 1e-30)).max())
-        parity = {"users_checked": len(sel), "ok": ok, "max_abs_err": float(err.max()), "row_norm_err": rown}
-
     sampler = None
     if rank == 0:
         try:
@@ -265,112 +519,54 @@ def run_ours(args, w):
         except Exception:
             sampler = None
 
-    ev0 = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
-    ev1 = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
-    kern_ns, comb_ns, launches = [], [], 0
-    if dist is not None:
-        dist.barrier()
-    torch.cuda.synchronize()
+    ws = workload_list(args)
+    head_name = HEADLINE if any(w.name == HEADLINE for w in ws) else ws[-1].name
+    per_config = []
+    for w in ws:
+        m = Measured(args, w, rank, local, dist, sampler)
+        runs = [(w.name, args.kernel)]
+        if w.name == "cfg4" and args.kernel == 0 and args.workload == "all":
+            # the gathering tensor-core kernel on the same workload: the path that splits the long histories
+            runs.append(("cfg4_gather", 2))
+        for entry, kernel in runs:
+            r = m.measure(entry, kernel, args.cpu_seconds or
+                          (CPU_SECONDS["headline"] if w.name == head_name else CPU_SECONDS["other"]))
+            if r is not None:
+                per_config.append(r)
+        m.close()
     if sampler:
-        sampler.on()
-    for i in range(args.steps):
-        flush.zero_()
-        ev0[i].record(stream)
-        step()
-        ev1[i].record(stream)
-        launches += s.stat("launches")
-        if i % 8 == 7 or i == args.steps - 1:   # keep the queue shallow; read the library's own events
-            kern_ns.append(s.stat("main_kernel_ns"))
-            comb_ns.append(s.stat("combine_kernel_ns"))
-    torch.cuda.synchronize()
-    if sampler:
-        sampler.off()
-    if dist is not None:
-        dist.barrier()
-    step_ms = [a.elapsed_time(b) for a, b in zip(ev0, ev1)]
-    total_ms, job_positions, job_users = reduce_over_ranks(float(sum(step_ms)), positions, w.n_users, dist, "cuda")
-
-    # end to end: host query buffer in, host output buffer out, through the same C-ABI call
-    q_host = torch.empty(q.shape, dtype=q.dtype).pin_memory()
-    q_host.copy_(q)
-    o_host = torch.empty(out.shape, dtype=out.dtype).pin_memory()
-    e2e_steps = max(3, min(args.steps, 20))
-    for _ in range(2):
-        s.attend(users, q_off, q_host, o_host)
-    torch.cuda.synchronize()
-    if dist is not None:
-        dist.barrier()
-    t0 = time.perf_counter()
-    for _ in range(e2e_steps):
-        s.attend(users, q_off, q_host, o_host)
-        torch.cuda.synchronize()
-    e2e_s, _, _ = reduce_over_ranks(time.perf_counter() - t0, positions, w.n_users, dist, "cuda")
-    clocks = sampler.finish() if sampler else None
-
+        sampler.finish()
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
         return
 
-    peak, peak_kind = _peaks()
-    kern_s = statistics.mean(kern_ns) * 1e-9
-    achieved = algo_bytes / kern_s / 1e9
-    value = job_positions * args.steps / (total_ms * 1e-3)
-    cpu = None
-    if not args.no_cpu:
-        rate, dt, cores, n_u, pos = _oracle_rate(w, data, CPU_SAMPLE_USERS.get(w.name, w.n_users))
-        cpu = {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle",
-               "sample": f"first {n_u} of {w.n_users} users ({pos} positions), {dt:.1f} s"}
-    # The roof that binds, reported beside the HBM roofline the metric asks for.
-    # Many queries per user (tcgen05 kernel): one exp (softmax) or tanh (SiLU) per score on the
-    # special-function unit.  Few queries (warp-level tensor-core kernel): every gathered pool row crosses
-    # the SM's L1 / shared-memory data pipe twice, once copied into the staging ring and once read
-    # out by ldmatrix; the pool rows come from L2, not HBM.
-    binding = None
-    family = s.stat("kernel")
-    if family == 2 and clocks and clocks.get("sm_max_mhz"):
-        n_sms = torch.cuda.get_device_properties(local).multi_processor_count
-        pipe_bytes = float(positions) * w.n_groups * 2 * (w.head_dim * 2) * 2
-        peak_pipe = L1_PIPE_BYTES_PER_SM_CLK * n_sms * clocks["sm_max_mhz"] * 1e6 / 1e9
-        binding = {"bound": "l1_shared_data_pipe",
-                   "what": "K and V pool rows into the shared-memory ring and out through ldmatrix",
-                   "achieved": pipe_bytes / kern_s / 1e9, "peak": peak_pipe, "unit": "GB/s",
-                   "frac": pipe_bytes / kern_s / 1e9 / peak_pipe}
-    elif w.n_queries >= 9 and clocks and clocks.get("sm_max_mhz"):
-        scores = float(positions) * w.n_groups * w.n_queries
-        n_sms = torch.cuda.get_device_properties(local).multi_processor_count
-        peak_xu = XU_PER_SM_CLK * n_sms * clocks["sm_max_mhz"] * 1e6 / 1e9
-        binding = {"bound": "alu", "what": "one ex2/tanh per score on the special-function unit",
-                   "achieved": scores / kern_s / 1e9, "peak": peak_xu, "unit": "Gscore/s",
-                   "frac": scores / kern_s / 1e9 / peak_xu}
+    head = next(r for r in per_config if r["entry"] == head_name)
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "f32" if w.dtype == "f32" else "bf16",
+        "metric": METRIC, "value": head["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": head["ms_per_step"], "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32" if synth.WORKLOADS[head["workload"]].dtype == "f32" else "bf16",
         "data": "synthetic",
-        "config": {"workload": w.name, "describe": w.describe, "users": w.n_users, "positions": positions,
+        "config": {"workload": head["workload"], "describe": head["describe"], "users": head["users"],
+                   "positions": head["positions"],
                    "l2": "flushed between timed steps (256 MiB overwrite)",
-                   "kernel_family": s.stat("kernel"), "mma_loader": s.stat("mma_loader"),
-                   "work_items": s.stat("work_items"),
-                   "split_items": s.stat("split_items")},
-        "users_per_sec": job_users * args.steps / (total_ms * 1e-3),
-        "clocks": clocks,
-        "e2e": {"value": job_positions * e2e_steps / e2e_s, "unit": UNIT,
-                "h2d_bytes_per_step": q_host.numel() * q_host.element_size() + users.nbytes + q_off.nbytes,
-                "d2h_bytes_per_step": o_host.numel() * o_host.element_size(), "ms_per_step": 1e3 * e2e_s / e2e_steps},
-        "gpu_launches": launches,
-        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": _traffic(w.name, not args.users), "peak_kind": peak_kind, "algorithmic_bytes": algo_bytes,
-                     "kernel_us": kern_s * 1e6, "combine_us": statistics.mean(comb_ns) * 1e-3,
-                     "frac_of_nominal_8TBs": achieved / 8000.0},
-        "roofline_binding": binding,
-        "cpu_baseline": cpu,
-        "parity": parity,
-        "compression": {"compressed_bytes": comp_bytes, "full_width_bytes": full_bytes,
-                        "ratio": comp_bytes / max(full_bytes, 1)},
+                   "protocol": f"per workload: warm-up, >= {args.sustain:g} s of back-to-back steps, synchronise, the timed steps",
+                   "sustained_steps_before_timed": head["sustained"]["steps"],
+                   "kernel_family": head["kernel_family"], "mma_loader": head["mma_loader"],
+                   "work_items": head["work_items"], "split_items": head["split_items"],
+                   "workloads_in_per_config": [r["entry"] for r in per_config]},
+        "users_per_sec": head["users_per_sec"],
+        "clocks": head["clocks"],
+        "e2e": head["e2e"], "e2e_fresh_plan": head["e2e_fresh_plan"],
+        "gpu_launches": sum(r["gpu_launches"] for r in per_config),
+        "roofline": head["roofline"],
+        "roofline_binding": head["roofline_binding"],
+        "cpu_baseline": head["cpu_baseline"],
+        "parity": head["parity"],
+        "compression": head["compression"],
+        "per_config": per_config,
     }
     print(json.dumps(line), flush=True)
-    s.close()
     if dist is not None:
         dist.destroy_process_group()
 
@@ -386,7 +582,6 @@ def run_load_path(args, w):
     batch's cache from pinned host memory to the GPU.  Classical cache: one copy of the full-width
     K/V bytes, T_load(s d_a).  Here: ckv_cache_import of the packed blob, T_load(s d_u + s), and
     import + ckv_attend, which contains the on-GPU indexing T_index fused with the attention."""
-    import time
     import torch
     import paper_2601_19178_b200 as ckv
     from paper_2601_19178_b200.session import as_device_tensor as dev
@@ -527,31 +722,42 @@ def run_route(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="cfg2", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--workload", default="all", choices=["all"] + sorted(synth.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--users", type=int, default=0, help="override the user count (smaller captures)")
     ap.add_argument("--kernel", type=int, default=0)
     ap.add_argument("--split-len", type=int, default=0)
     ap.add_argument("--mma-loader", type=int, default=0, help="1 = cp.async (default), 2 = TMA gathers")
+    ap.add_argument("--l2-persist", type=int, default=-1, help="0 / 1: the library's option of that name (default: leave it)")
+    ap.add_argument("--sustain", type=float, default=SUSTAIN_SECONDS,
+                    help="seconds of back-to-back steps before the timed ones (0: only the timed steps' own count)")
+    ap.add_argument("--cpu-seconds", type=float, default=0.0, help="host time of the CPU-oracle leg per workload")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-check", action="store_true", help="skip the sampled parity check")
     ap.add_argument("--route", action="store_true", help="time the prefill router (Sec. 4.3) instead of the attend step")
     ap.add_argument("--load-path", action="store_true",
                     help="time the decode-stage load path per batch size (Sec. 4.4) instead of the attend step")
+    ap.add_argument("--record-traffic", metavar="NCU_RAW_CSV",
+                    help="no GPU work: store the DRAM bytes of the attend launches of an `ncu --page raw --csv` dump "
+                         "in profiles/traffic.json (with --entry, --family, --workload, --users)")
+    ap.add_argument("--entry", default="", help="per_config entry the traffic record belongs to (cfg2, cfg4_gather, ...)")
+    ap.add_argument("--family", type=int, default=0, help="kernel family of the traffic record")
     args = ap.parse_args()
-    w = synth.WORKLOADS[args.workload]
-    if args.users:
-        w = synth.scaled(w, n_users=args.users)
-    if args.impl == "reference":
-        run_reference(args, w)
+    if args.record_traffic:
+        record_traffic(args)
+    elif args.impl == "reference":
+        run_reference(args)
     elif args.route:
         run_route(args)
     elif args.load_path:
+        w = synth.WORKLOADS["cfg4" if args.workload == "all" else args.workload]
+        if args.users:
+            w = synth.scaled(w, n_users=args.users)
         run_load_path(args, w)
     else:
-        run_ours(args, w)
+        run_ours(args)
 
 
 if __name__ == "__main__":

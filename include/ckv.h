@@ -28,7 +28,10 @@
  *   - Errors are return codes.  Nothing aborts, traps or throws across the boundary.  After
  *     any error the context is unchanged and stays usable (CKV_ERR_CUDA excepted: the CUDA
  *     context may be lost).
- *   - A context belongs to one device and may be used by one host thread at a time.
+ *   - A context belongs to one device and may be used by one host thread at a time.  All calls
+ *     on a context must be ordered on the GPU: pass the same stream, or chain the streams with
+ *     events.  The context's scratch buffers, its plan tables and the storage that evicted or
+ *     replaced users give back are reused by later calls in stream order only.
  */
 #ifndef CKV_H_
 #define CKV_H_
@@ -89,7 +92,10 @@ CKV_API ckv_status ckv_destroy(ckv_ctx* ctx);
  * memory at inference).
  *   pool_K, pool_V [any] : [n_groups][n_entries][d_shared], contiguous, ctx dtype.
  * The pool is copied into the library's own row layout (full head_dim-wide rows whose first
- * d_user slots are zero) and asked to persist in L2.  Fixes d_user = head_dim - d_shared and
+ * d_user slots are zero).  To keep it resident in L2 the call raises this process's persisting-L2
+ * carve-out on the device to the pool's size (cudaLimitPersistingL2CacheSize, capped by the device;
+ * put back when the last context on the device is destroyed); see option "l2_persist".  Fixes
+ * d_user = head_dim - d_shared and
  * the stored index width (16 bit when n_entries <= 65536, else 32 bit).  May be called again
  * with the same n_entries and d_shared to refresh the values; any other reload while users
  * are cached is CKV_ERR_SHAPE.
@@ -100,7 +106,8 @@ CKV_API ckv_status ckv_pool_load(ckv_ctx* ctx, const void* pool_K, const void* p
 
 /*
  * Store one user's compressed cache (Sec. 4.2, prefill output: global K/V indices plus
- * user-specific K/V), replacing any earlier entry of `user`.
+ * user-specific K/V), replacing any earlier entry of `user` (whose storage is reused by later
+ * puts, imports and appends).
  *   idx_K, idx_V   [any] : int32 [L][n_groups]  (may alias each other)
  *   user_K, user_V [any] : [L][n_groups][d_user], ctx dtype; may be NULL iff d_user == 0
  *   L >= 0 (a user with an empty history is legal and attends to a zero output).
@@ -123,7 +130,9 @@ CKV_API ckv_status ckv_cache_put_batch(ckv_ctx* ctx, int32_t n, const int64_t* u
                                const void* user_K, const void* user_V, int32_t d_user,
                                void* stream);
 
-/* Forget one user / all users (the pool stays).  Unknown user: CKV_ERR_UNKNOWN_USER. */
+/* Forget one user / all users (the pool stays).  Unknown user: CKV_ERR_UNKNOWN_USER.  The user's
+ * storage goes to a free list (neighbouring free runs merge) and is reused first-fit, so a cache that
+ * is updated continuously stays bounded by its live users plus fragmentation. */
 CKV_API ckv_status ckv_cache_evict(ckv_ctx* ctx, int64_t user);
 CKV_API ckv_status ckv_cache_clear(ckv_ctx* ctx);
 
@@ -137,8 +146,13 @@ CKV_API ckv_status ckv_cache_clear(ckv_ctx* ctx);
  *   queries [any]  : [q_off[n]][n_groups][head_dim], ctx dtype
  *   out     [any]  : [q_off[n]][n_groups][head_dim], ctx out_dtype, caller-allocated
  * A user with an empty history produces zero rows.  Results do not depend on how the
- * library splits long histories across thread blocks beyond fp32 rounding, and are bitwise
- * reproducible from call to call for the same context settings.
+ * library splits long histories across thread blocks beyond fp32 rounding.  With kernel
+ * families 1 to 3 (see option "kernel") they are bitwise reproducible from call to call for the
+ * same context settings; family 4, which the library picks by itself for one query per user over
+ * histories that are long against the pool, sums its weight histogram with shared-memory atomics
+ * and can differ in the last bits from run to run (set option "kernel" to 2 where that matters).
+ * A kernel whose internal bounded wait runs out cannot be reported by this (asynchronous) call:
+ * read ckv_last_stat("device_errors") after synchronising when that matters.
  * Errors: STATE, INVALID_ARG, UNKNOWN_USER, OOM (workspace), CUDA.
  */
 CKV_API ckv_status ckv_attend(ckv_ctx* ctx, int32_t n, const int64_t* users, const int32_t* q_off,
@@ -148,14 +162,13 @@ CKV_API ckv_status ckv_attend(ckv_ctx* ctx, int32_t n, const int64_t* users, con
  * Decode without any allocation.  (The paper has no counterpart: this is a deployment variant of
  * ckv_attend, not a different computation.)
  *
- * ckv_attend may call cudaMalloc/cudaFree: it grows a workspace for the partial results of
- * the split-along-history reduction and keeps per-request tables in device memory it
- * allocates.  Some callers cannot tolerate that: a serving thread inside a latency-critical
- * section (cudaMalloc and cudaFree synchronise the device), a process whose memory was handed
- * in full to another allocator, code running between cudaStreamBeginCapture and EndCapture
- * where allocation is not permitted.  For them this entry point computes exactly what
- * ckv_attend computes, with the same kernels, but keeps those tables and partial results in a
- * fixed array that is part of the library's device image:
+ * ckv_attend may call cudaMalloc/cudaFree and cudaMallocHost: it grows a workspace for the partial
+ * results of the split-along-history reduction and keeps per-request tables in device and pinned
+ * memory it allocates.  Some callers cannot tolerate that: a serving thread inside a
+ * latency-critical section (cudaMalloc and cudaFree synchronise the device), a process whose GPU
+ * memory was handed in full to another allocator.  For them this entry point computes what
+ * ckv_attend computes, but keeps those tables and partial results in a fixed array that is part
+ * of the library's device image:
  *   - CKV_STATIC_SCRATCH_BYTES (8 MiB) per GPU that loads the library, held until the
  *     process exits, shared by every context and every call on that GPU;
  *   - limits: n <= CKV_STATIC_MAX_USERS (256) users per call, at most 4096 history chunks, and
@@ -164,9 +177,19 @@ CKV_API ckv_status ckv_attend(ckv_ctx* ctx, int32_t n, const int64_t* users, con
  *     enqueues nothing.  ("split_len" controls the chunk count; 0 = automatic.)
  *   - queries and out must be device memory (staging host buffers would need an allocation);
  *     host pointers return CKV_ERR_INVALID_ARG.
- * It calls no cudaMalloc, cudaFree or other allocating routine.  The first call on a device
- * looks up the array's device address (once per device, with that device current); make that
- * first call outside any stream capture.
+ *   - kernels: only the CUDA-core family (1) and the warp-level tensor-core family (2) run here
+ *     (option "kernel" 0, 1 or 2; 3 and 4 return CKV_ERR_UNSUPPORTED: the tcgen05 kernel wants a
+ *     work list and the factorised path tables whose sizes follow the request).  For requests
+ *     that ckv_attend would give to family 3 or 4 the results agree within the usual tolerance,
+ *     not bit for bit.
+ * It calls no cudaMalloc, cudaFree or other allocating routine, and copies nothing from the
+ * caller's host memory asynchronously: the request tables travel as kernel arguments of a small
+ * kernel that writes them into the array (ceil(n / 80) launches of one thread block), followed by
+ * the attend kernel and, for split histories, the merge kernel.  The first call on a device
+ * looks up the array's device address (once per device, with that device current), which is also
+ * when the CUDA driver may load the part of the library's device image that holds the array (the
+ * 8 MiB leave the device's free memory at that moment, not later); make that first call during
+ * start-up and outside any stream capture.
  * The array keeps the previous call's contents.  Nothing in it needs clearing: every entry
  * a call reads it has written itself.  Because all calls on a GPU share the array, two
  * calls whose kernels may overlap on the GPU (different streams, or different host threads)
@@ -222,9 +245,9 @@ CKV_API ckv_status ckv_project(int32_t device, int32_t n, int32_t n_groups, int3
 
 /*
  * Appends L_new positions (new interactions) behind a cached user's history; arguments as for
- * ckv_cache_put, describing only the new positions.  The user's compressed cache moves to fresh
- * storage holding the old and the new positions (storage is only reclaimed by ckv_cache_clear or
- * when the last user is evicted).  Synchronises `stream`.
+ * ckv_cache_put, describing only the new positions.  The user's compressed cache moves to other
+ * storage holding the old and the new positions; the old storage is reused by later calls.
+ * Synchronises `stream`.
  * Errors: INVALID_ARG, STATE (no pool), SHAPE (d_user), UNKNOWN_USER, INDEX_RANGE (an index
  * outside [0, n_entries); the user keeps the old history), OOM, CUDA.
  */
@@ -285,7 +308,9 @@ CKV_API ckv_status ckv_cache_bytes(ckv_ctx* ctx, int64_t* compressed, int64_t* f
  *                  0 or 1 = 16-byte asynchronous copies through L1 (default), 2 = TMA row gathers
  *                  (UNSUPPORTED from ckv_attend if the driver cannot encode the tensor maps);
  *                  the results are the same bits either way
- *   "l2_persist"   1 = ask for the pool to persist in L2 on the streams used (default), 0 = off
+ *   "l2_persist"   1 (default) = every ckv_attend puts an access-policy window over the pool
+ *                  (persisting hits) on the caller's stream while it enqueues its kernels and restores
+ *                  the stream's previous window before it returns; 0 = leave the stream alone
  *   "time_kernels" 1 = record CUDA events around the kernels of each ckv_attend (see ckv_last_stat)
  */
 CKV_API ckv_status ckv_set_option(ckv_ctx* ctx, const char* name, int64_t value);
@@ -296,7 +321,11 @@ CKV_API ckv_status ckv_get_option(ckv_ctx* ctx, const char* name, int64_t* value
  * ckv_attend: "launches" (kernels enqueued), "work_items", "split_items" (items that went
  * through the partial-result workspace), "kernel" (family that ran: 1 to 4), "mma_loader"
  * (loader the last warp-level tensor-core launch used: 1 or 2),
- * "workspace_bytes", "plan_cache_hit"; with option "time_kernels" also "main_kernel_ns" and
+ * "workspace_bytes", "plan_cache_hit", "alloc_calls" (device or pinned-host allocations the call
+ * made: 0 once its buffers have reached their size), "l2_window" (1 if the pool's L2 window was on
+ * the stream for the call); "arena_capacity_units", "arena_used_units", "arena_free_runs" (state of
+ * the compressed-cache storage, in (position, group) units); with option "time_kernels" also
+ * "main_kernel_ns" and
  * "combine_kernel_ns" (device time of the attend kernel and of the split-merge kernel; the
  * query waits for that attend to finish; CKV_ERR_STATE if nothing was timed).
  * "device_errors" (not tied to the last call): non-zero once a kernel of this context gave up

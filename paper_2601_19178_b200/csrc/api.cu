@@ -3,10 +3,10 @@
 #include <algorithm>
 #include <cmath>
 #include <cstring>
+#include <map>
 #include <mutex>
 #include <new>
 #include <string>
-#include <unordered_map>
 #include <vector>
 
 #include "ckv_internal.h"
@@ -21,17 +21,116 @@ struct UserEntry {
     int32_t Lpad;
 };
 
+// User id -> cache entry: open addressing with linear probing and backward-shift deletion.  A decode
+// call looks up every user of its request list, so a lookup has to cost one cache line, not a node chase.
+class UserTable {
+    struct Slot {
+        int64_t key;
+        UserEntry e;
+        uint32_t used;
+    };
+    std::vector<Slot> slots_;
+    size_t n_ = 0, mask_ = 0;
+    static size_t hash(int64_t k)
+    {
+        uint64_t x = (uint64_t)k + 0x9e3779b97f4a7c15ull;
+        x = (x ^ (x >> 30)) * 0xbf58476d1ce4e5b9ull;
+        x = (x ^ (x >> 27)) * 0x94d049bb133111ebull;
+        return (size_t)(x ^ (x >> 31));
+    }
+    void rehash(size_t cap)
+    {
+        std::vector<Slot> old;
+        old.swap(slots_);
+        slots_.assign(cap, Slot{0, {0, 0, 0}, 0});
+        mask_ = cap - 1;
+        n_ = 0;
+        for (const Slot& sl : old)
+            if (sl.used) *insert(sl.key) = sl.e;
+    }
+
+public:
+    size_t size() const { return n_; }
+    bool empty() const { return n_ == 0; }
+    void clear()
+    {
+        slots_.clear();
+        n_ = mask_ = 0;
+    }
+    const UserEntry* find(int64_t key) const
+    {
+        if (n_ == 0) return nullptr;
+        for (size_t i = hash(key) & mask_;; i = (i + 1) & mask_) {
+            const Slot& sl = slots_[i];
+            if (!sl.used) return nullptr;
+            if (sl.key == key) return &sl.e;
+        }
+    }
+    UserEntry* find(int64_t key) { return const_cast<UserEntry*>(static_cast<const UserTable*>(this)->find(key)); }
+    // the entry of `key`, created (zeroed) if absent; may throw std::bad_alloc
+    UserEntry* insert(int64_t key)
+    {
+        if (slots_.empty() || (n_ + 1) * 2 > slots_.size()) rehash(slots_.empty() ? 64 : slots_.size() * 2);
+        for (size_t i = hash(key) & mask_;; i = (i + 1) & mask_) {
+            Slot& sl = slots_[i];
+            if (!sl.used) {
+                sl.used = 1;
+                sl.key = key;
+                sl.e = UserEntry{0, 0, 0};
+                ++n_;
+                return &sl.e;
+            }
+            if (sl.key == key) return &sl.e;
+        }
+    }
+    bool erase(int64_t key)
+    {
+        if (n_ == 0) return false;
+        size_t i = hash(key) & mask_;
+        for (;; i = (i + 1) & mask_) {
+            if (!slots_[i].used) return false;
+            if (slots_[i].key == key) break;
+        }
+        // close the gap: move back every follower whose home slot is not inside (i, j]
+        for (size_t j = (i + 1) & mask_; slots_[j].used; j = (j + 1) & mask_) {
+            const size_t h = hash(slots_[j].key) & mask_;
+            const bool stays = i <= j ? (h > i && h <= j) : (h > i || h <= j);
+            if (!stays) {
+                slots_[i] = slots_[j];
+                i = j;
+            }
+        }
+        slots_[i].used = 0;
+        --n_;
+        return true;
+    }
+    // room for `extra` more users, so that `insert` cannot fail half-way through a batch
+    void reserve_more(size_t extra)
+    {
+        size_t cap = slots_.empty() ? 64 : slots_.size();
+        while ((n_ + extra) * 2 > cap) cap *= 2;
+        if (cap != slots_.size()) rehash(cap);
+    }
+};
+
 struct DevBuf {  // grow-only device buffer
     void* p = nullptr;
     size_t cap = 0;
 };
 
+// A cached attend plan.  Its tables live in one pinned host block and one device block that the slot keeps
+// (grow-only) when another request list takes it over, so a new request list costs no allocation once the
+// blocks have reached their size.
 struct Plan {
+    bool live = false;
     std::vector<int64_t> users;
     std::vector<int32_t> q_off;
     uint64_t generation = 0;
     int64_t opt_split = 0, opt_kernel = 0;
-    void* dev = nullptr;  // one allocation: reqs | items | split list | works
+    DevBuf dev;              // reqs | items | split list | works
+    void* host = nullptr;    // pinned mirror the tables are built in
+    size_t host_cap = 0;
+    cudaEvent_t uploaded = nullptr;  // recorded behind the last upload from `host`
     Req* d_reqs = nullptr;
     Item* d_items = nullptr;
     int32_t* d_split = nullptr;
@@ -74,22 +173,31 @@ struct ckv_ctx {
     bool has_umma = false;
     int* d_err = nullptr;  // OR of error codes from kernels whose bounded waits ran out
     size_t pool_half = 0;  // bytes of one of them
-    // arena of compressed caches (units = (position, group) slots)
+    // arena of compressed caches (units = (position, group) slots).  Units [0, used_units) are handed out;
+    // runs inside that range given back by evicted, replaced or appended-to users wait in free_runs
+    // (first unit -> length, neighbours merged) and are reused first-fit.
     void *a_idxK = nullptr, *a_idxV = nullptr, *a_userK = nullptr, *a_userV = nullptr;
     int64_t cap_units = 0, used_units = 0, live_positions = 0;
-    std::unordered_map<int64_t, UserEntry> users;
+    std::map<int64_t, int64_t> free_runs;
+    UserTable users;
     uint64_t generation = 1;
     // scratch
     DevBuf stage_q, stage_out, partials;
     int* d_flag = nullptr;
-    std::vector<Plan> plans;
+    Plan plans[kMaxPlans];
     uint64_t tick = 0;
     // options
     int64_t opt_split = 0, opt_kernel = 0, opt_l2 = 1, opt_time = 0, opt_loader = 0;
     cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};  // around the main kernel and the combine
     bool ev_valid = false;
+    // L2 residency of the pool: an access-policy window over the pool allocation is put on the caller's
+    // stream around the kernels of a decode call and taken off again before the call returns
+    bool l2_ready = false;       // the persisting-L2 carve-out of this device was raised for this context
+    size_t l2_window = 0;        // bytes of the window (0: not available)
+    float l2_ratio = 1.f;
     // statistics of the last attend
-    int64_t st_launches = 0, st_items = 0, st_split = 0, st_kernel = 0, st_ws = 0, st_hit = 0, st_loader = 0;
+    int64_t st_launches = 0, st_items = 0, st_split = 0, st_kernel = 0, st_ws = 0, st_hit = 0, st_loader = 0,
+            st_allocs = 0, st_l2 = 0;
     std::string cuda_err;
 
     ckv_status fail(cudaError_t e)
@@ -139,9 +247,10 @@ struct Staged {
     }
 };
 
-cudaError_t grow(DevBuf& b, size_t bytes)
+cudaError_t grow(DevBuf& b, size_t bytes, int64_t* allocs = nullptr)
 {
     if (bytes <= b.cap) return cudaSuccess;
+    if (allocs) ++*allocs;
     if (b.p) {
         cudaError_t e = cudaFree(b.p);  // waits for work that may still use it
         b.p = nullptr;
@@ -162,14 +271,15 @@ cudaError_t grow(DevBuf& b, size_t bytes)
 
 void free_plan(Plan& p)
 {
-    if (p.dev) cudaFree(p.dev);
-    p.dev = nullptr;
+    if (p.dev.p) cudaFree(p.dev.p);
+    if (p.host) cudaFreeHost(p.host);
+    if (p.uploaded) cudaEventDestroy(p.uploaded);
+    p = Plan();
 }
 
 void drop_plans(ckv_ctx* ctx)
 {
     for (auto& p : ctx->plans) free_plan(p);
-    ctx->plans.clear();
 }
 
 CacheView view_of(const ckv_ctx* ctx)
@@ -188,11 +298,11 @@ CacheView view_of(const ckv_ctx* ctx)
     return v;
 }
 
-// Make room for `need` more units, keeping what is stored.
-ckv_status ensure_arena(ckv_ctx* ctx, int64_t need, cudaStream_t s)
+// Capacity for units [0, need_end), keeping what is stored.
+ckv_status ensure_arena(ckv_ctx* ctx, int64_t need_end, cudaStream_t s)
 {
-    if (ctx->used_units + need <= ctx->cap_units) return CKV_OK;
-    int64_t cap = std::max<int64_t>(ctx->cap_units * 2, ctx->used_units + need);
+    if (need_end <= ctx->cap_units) return CKV_OK;
+    int64_t cap = std::max<int64_t>(ctx->cap_units * 2, need_end);
     cap = (cap + 1023) / 1024 * 1024;
     const size_t ub = (size_t)std::max(ctx->d_user, 1) * ctx->elem;
     void* n[4] = {nullptr, nullptr, nullptr, nullptr};
@@ -227,6 +337,56 @@ ckv_status ensure_arena(ckv_ctx* ctx, int64_t need, cudaStream_t s)
     return CKV_OK;
 }
 
+// A run of `units` contiguous arena units: the first free run that is large enough, else fresh units behind
+// everything handed out so far (growing the arena if need be).
+ckv_status arena_take(ckv_ctx* ctx, int64_t units, cudaStream_t s, int64_t* base)
+{
+    for (auto it = ctx->free_runs.begin(); it != ctx->free_runs.end(); ++it) {
+        if (it->second < units) continue;
+        *base = it->first;
+        const int64_t rest = it->second - units;
+        ctx->free_runs.erase(it);
+        if (rest > 0) ctx->free_runs.emplace(*base + units, rest);
+        return CKV_OK;
+    }
+    ckv_status st = ensure_arena(ctx, ctx->used_units + units, s);
+    if (st != CKV_OK) return st;
+    *base = ctx->used_units;
+    ctx->used_units += units;
+    return CKV_OK;
+}
+
+// Gives a run back.  Work already enqueued on the context's stream may still read it; whatever reuses it is
+// enqueued behind that work on the same stream.
+void arena_give(ckv_ctx* ctx, int64_t base, int64_t units)
+{
+    if (units <= 0) return;
+    try {
+        auto it = ctx->free_runs.emplace(base, units).first;
+        auto nx = std::next(it);
+        if (nx != ctx->free_runs.end() && it->first + it->second == nx->first) {
+            it->second += nx->second;
+            ctx->free_runs.erase(nx);
+        }
+        if (it != ctx->free_runs.begin()) {
+            auto pv = std::prev(it);
+            if (pv->first + pv->second == it->first) {
+                pv->second += it->second;
+                ctx->free_runs.erase(it);
+                it = pv;
+            }
+        }
+        if (it->first + it->second == ctx->used_units) {  // the run touches the end: shrink instead of keeping it
+            ctx->used_units = it->first;
+            ctx->free_runs.erase(it);
+        }
+    } catch (const std::bad_alloc&) {
+        // the run is lost until the arena is cleared; nothing else depends on it
+    }
+}
+
+int64_t units_of_len(const ckv_ctx* ctx, int64_t L) { return (int64_t)ctx->cfg.n_groups * ((L + 31) / 32 * 32); }
+
 int64_t auto_split_len(const ckv_ctx* ctx, int64_t total_positions, int family, int max_M)
 {
     // Enough (chunk, group) blocks to fill the SMs several times over, but chunks long
@@ -248,6 +408,30 @@ int64_t auto_split_len(const ckv_ctx* ctx, int64_t total_positions, int family, 
     return std::min<int64_t>(std::max<int64_t>(c, 256), 2048);
 }
 
+// Orders item indices by descending chunk length, equal lengths in their original order (two 16-bit
+// counting passes over the complemented length: linear in the number of items).
+void order_longest_first(const std::vector<Item>& items, std::vector<uint32_t>& order)
+{
+    const size_t n = items.size();
+    order.resize(n);
+    bool same = true;
+    for (size_t i = 0; i < n; ++i) {
+        order[i] = (uint32_t)i;
+        same = same && items[i].len == items[0].len;
+    }
+    if (same || n < 2) return;
+    std::vector<uint32_t> tmp(n);
+    std::vector<uint32_t> count(65536 + 1);
+    for (int pass = 0; pass < 2; ++pass) {
+        const int shift = 16 * pass;
+        std::fill(count.begin(), count.end(), 0u);
+        for (size_t i = 0; i < n; ++i) ++count[((~(uint32_t)items[order[i]].len >> shift) & 0xffffu) + 1];
+        for (size_t d = 0; d < 65536; ++d) count[d + 1] += count[d];
+        for (size_t i = 0; i < n; ++i) tmp[count[(~(uint32_t)items[order[i]].len >> shift) & 0xffffu]++] = order[i];
+        order.swap(tmp);
+    }
+}
+
 ckv_status build_plan(ckv_ctx* ctx, Plan& pl, int32_t n, const int64_t* users, const int32_t* q_off,
                       cudaStream_t s)
 {
@@ -256,12 +440,12 @@ ckv_status build_plan(ckv_ctx* ctx, Plan& pl, int32_t n, const int64_t* users, c
     int32_t max_M = 0, max_L = 0;
     bool all_single = true;
     for (int32_t k = 0; k < n; ++k) {
-        auto f = ctx->users.find(users[k]);
-        if (f == ctx->users.end()) return CKV_ERR_UNKNOWN_USER;
+        const UserEntry* f = ctx->users.find(users[k]);
+        if (!f) return CKV_ERR_UNKNOWN_USER;
         Req& r = reqs[k];
-        r.base = f->second.base;
-        r.L = f->second.L;
-        r.Lpad = f->second.Lpad;
+        r.base = f->base;
+        r.L = f->L;
+        r.Lpad = f->Lpad;
         r.q0 = q_off[k];
         r.M = q_off[k + 1] - q_off[k];
         r.part0 = -1;
@@ -334,41 +518,54 @@ ckv_status build_plan(ckv_ctx* ctx, Plan& pl, int32_t n, const int64_t* users, c
         part_rows += nc * r.M;
     }
     // longest chunks first: the tail of the grid is made of short ones
-    std::stable_sort(items.begin(), items.end(), [](const Item& x, const Item& y) { return x.len > y.len; });
+    std::vector<uint32_t> order;
+    order_longest_first(items, order);
     pl.n_items = (int32_t)items.size();
     pl.n_split = (int32_t)split.size();
     pl.split_items = 0;
     for (const Item& it : items) pl.split_items += it.part_row >= 0;
     pl.part_rows = part_rows;
 
-    std::vector<Work> works;
-    if (pl.family == 3) {
-        works.resize(items.size());
-        for (size_t i = 0; i < items.size(); ++i) {
-            const Item& it = items[i];
-            const Req& r = reqs[it.req];
-            works[i] = Work{r.base, r.L, r.Lpad, r.q0, r.M, it.begin, it.len, it.part_row, {0, 0, 0}};
-        }
-    }
+    // the tables are laid out in the slot's pinned block and go to the device in one copy
+    const size_t n_works = pl.family == 3 ? items.size() : 0;
     const size_t b_req = sizeof(Req) * reqs.size(), b_item = sizeof(Item) * items.size(),
-                 b_split = sizeof(int32_t) * split.size(), b_work = sizeof(Work) * works.size();
+                 b_split = sizeof(int32_t) * split.size(), b_work = sizeof(Work) * n_works;
     const size_t o_item = (b_req + 255) / 256 * 256, o_split = o_item + (b_item + 255) / 256 * 256,
-                 o_work = o_split + (b_split + 255) / 256 * 256;
-    CK(cudaMalloc(&pl.dev, o_work + b_work + 256));
-    pl.d_reqs = (Req*)pl.dev;
-    pl.d_items = (Item*)((char*)pl.dev + o_item);
-    pl.d_split = (int32_t*)((char*)pl.dev + o_split);
-    pl.d_works = (Work*)((char*)pl.dev + o_work);
-    if (b_work) CK(cudaMemcpyAsync(pl.d_works, works.data(), b_work, cudaMemcpyHostToDevice, s));
-    if (b_req) CK(cudaMemcpyAsync(pl.d_reqs, reqs.data(), b_req, cudaMemcpyHostToDevice, s));
-    if (b_item) CK(cudaMemcpyAsync(pl.d_items, items.data(), b_item, cudaMemcpyHostToDevice, s));
-    if (b_split) CK(cudaMemcpyAsync(pl.d_split, split.data(), b_split, cudaMemcpyHostToDevice, s));
-    // the host vectors die at return: pageable copies have been staged by then
+                 o_work = o_split + (b_split + 255) / 256 * 256, total = o_work + b_work + 256;
+    if (pl.uploaded) CK(cudaEventSynchronize(pl.uploaded));  // the block's previous upload has left the host
+    else CK(cudaEventCreateWithFlags(&pl.uploaded, cudaEventDisableTiming));
+    if (total > pl.host_cap) {
+        ctx->st_allocs++;
+        if (pl.host) cudaFreeHost(pl.host);
+        pl.host = nullptr;
+        pl.host_cap = 0;
+        CK(cudaMallocHost(&pl.host, total + total / 4));
+        pl.host_cap = total + total / 4;
+    }
+    CK(grow(pl.dev, total, &ctx->st_allocs));
+    char* h = (char*)pl.host;
+    std::memcpy(h, reqs.data(), b_req);
+    Item* h_items = (Item*)(h + o_item);
+    for (size_t i = 0; i < items.size(); ++i) h_items[i] = items[order[i]];
+    if (b_split) std::memcpy(h + o_split, split.data(), b_split);
+    Work* h_works = (Work*)(h + o_work);
+    for (size_t i = 0; i < n_works; ++i) {
+        const Item& it = h_items[i];
+        const Req& r = reqs[it.req];
+        h_works[i] = Work{r.base, r.L, r.Lpad, r.q0, r.M, it.begin, it.len, it.part_row, {0, 0, 0}};
+    }
+    pl.d_reqs = (Req*)pl.dev.p;
+    pl.d_items = (Item*)((char*)pl.dev.p + o_item);
+    pl.d_split = (int32_t*)((char*)pl.dev.p + o_split);
+    pl.d_works = (Work*)((char*)pl.dev.p + o_work);
+    CK(cudaMemcpyAsync(pl.dev.p, h, o_work + b_work, cudaMemcpyHostToDevice, s));
+    CK(cudaEventRecord(pl.uploaded, s));
     pl.users.assign(users, users + n);
     pl.q_off.assign(q_off, q_off + n + 1);
     pl.generation = ctx->generation;
     pl.opt_split = ctx->opt_split;
     pl.opt_kernel = ctx->opt_kernel;
+    pl.live = true;
     return CKV_OK;
 }
 
@@ -376,9 +573,11 @@ ckv_status get_plan(ckv_ctx* ctx, int32_t n, const int64_t* users, const int32_t
                     Plan** out)
 {
     ctx->tick++;
+    Plan* victim = nullptr;
     for (auto& p : ctx->plans) {
-        if (p.generation == ctx->generation && p.opt_split == ctx->opt_split &&
-            p.opt_kernel == ctx->opt_kernel && (int32_t)p.users.size() == n &&
+        if (p.live && p.generation != ctx->generation) p.live = false;  // stale: the cache has changed since
+        if (p.live && p.opt_split == ctx->opt_split && p.opt_kernel == ctx->opt_kernel &&
+            (int32_t)p.users.size() == n &&
             std::memcmp(p.users.data(), users, sizeof(int64_t) * (size_t)n) == 0 &&
             std::memcmp(p.q_off.data(), q_off, sizeof(int32_t) * ((size_t)n + 1)) == 0) {
             p.last_use = ctx->tick;
@@ -386,35 +585,113 @@ ckv_status get_plan(ckv_ctx* ctx, int32_t n, const int64_t* users, const int32_t
             *out = &p;
             return CKV_OK;
         }
+        // the slot a new plan takes: a dead one, else the least recently used
+        if (!victim || (!p.live && victim->live) || (p.live == victim->live && p.last_use < victim->last_use))
+            victim = &p;
     }
     ctx->st_hit = 0;
-    // drop stale plans, then the least recently used one if the cache is full
-    for (size_t i = 0; i < ctx->plans.size();) {
-        if (ctx->plans[i].generation != ctx->generation) {
-            free_plan(ctx->plans[i]);
-            ctx->plans.erase(ctx->plans.begin() + i);
-        } else {
-            ++i;
-        }
+    victim->live = false;
+    ckv_status st;
+    try {
+        st = build_plan(ctx, *victim, n, users, q_off, s);
+    } catch (const std::bad_alloc&) {
+        st = CKV_ERR_OOM;
     }
-    if ((int)ctx->plans.size() >= kMaxPlans) {
-        size_t lru = 0;
-        for (size_t i = 1; i < ctx->plans.size(); ++i)
-            if (ctx->plans[i].last_use < ctx->plans[lru].last_use) lru = i;
-        free_plan(ctx->plans[lru]);
-        ctx->plans.erase(ctx->plans.begin() + lru);
-    }
-    Plan pl;
-    ckv_status st = build_plan(ctx, pl, n, users, q_off, s);
-    if (st != CKV_OK) {
-        free_plan(pl);
-        return st;
-    }
-    pl.last_use = ctx->tick;
-    ctx->plans.push_back(std::move(pl));
-    *out = &ctx->plans.back();
+    if (st != CKV_OK) return st;
+    victim->last_use = ctx->tick;
+    *out = victim;
     return CKV_OK;
 }
+
+// ---- L2 residency of the pool ------------------------------------------------------------------------
+// The pool is read by every work item of every decode call while the compressed caches stream through L2
+// once.  The device's persisting-L2 carve-out is raised to the pool's size (a per-process setting that ends
+// with the process; the previous value comes back when the last context on the device goes away), and each
+// decode call puts an access-policy window over the pool on the caller's stream while it enqueues its
+// kernels: pool lines are then kept in the carve-out and the streaming data cannot evict them.
+std::mutex g_l2_mu;
+int g_l2_users[64];
+size_t g_l2_prev[64];
+
+void l2_prepare(ckv_ctx* ctx)
+{
+    ctx->l2_window = 0;
+    const int dev = ctx->cfg.device;
+    if (dev >= 64) return;
+    int max_persist = 0, max_window = 0;
+    if (cudaDeviceGetAttribute(&max_persist, cudaDevAttrMaxPersistingL2CacheSize, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&max_window, cudaDevAttrMaxAccessPolicyWindowSize, dev) != cudaSuccess ||
+        max_persist <= 0 || max_window <= 0) {
+        cudaGetLastError();
+        return;
+    }
+    const size_t pool_bytes = 2 * ctx->pool_half;
+    const size_t want = std::min(pool_bytes, (size_t)max_persist);
+    std::lock_guard<std::mutex> lock(g_l2_mu);
+    size_t cur = 0;
+    if (cudaDeviceGetLimit(&cur, cudaLimitPersistingL2CacheSize) != cudaSuccess) {
+        cudaGetLastError();
+        return;
+    }
+    if (!ctx->l2_ready) {
+        if (g_l2_users[dev]++ == 0) g_l2_prev[dev] = cur;
+        ctx->l2_ready = true;
+    }
+    if (cur < want && cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, want) != cudaSuccess) {
+        cudaGetLastError();
+        return;
+    }
+    if (cur < want) cur = want;
+    ctx->l2_window = std::min(pool_bytes, (size_t)max_window);
+    ctx->l2_ratio = ctx->l2_window <= cur ? 1.0f : (float)((double)cur / (double)ctx->l2_window);
+}
+
+void l2_release(ckv_ctx* ctx)
+{
+    if (!ctx->l2_ready) return;
+    const int dev = ctx->cfg.device;
+    std::lock_guard<std::mutex> lock(g_l2_mu);
+    if (--g_l2_users[dev] == 0) {
+        cudaCtxResetPersistingL2Cache();
+        cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, g_l2_prev[dev]);
+        cudaGetLastError();
+    }
+    ctx->l2_ready = false;
+}
+
+// Puts the pool's window on a stream for the lifetime of the object and restores what the stream had.
+struct L2Window {
+    cudaStream_t s;
+    cudaStreamAttrValue prev;
+    bool on = false;
+    L2Window(ckv_ctx* ctx, cudaStream_t stream) : s(stream)
+    {
+        ctx->st_l2 = 0;
+        if (!ctx->opt_l2 || ctx->l2_window == 0) return;
+        if (cudaStreamGetAttribute(s, cudaStreamAttributeAccessPolicyWindow, &prev) != cudaSuccess) {
+            cudaGetLastError();
+            return;
+        }
+        cudaStreamAttrValue v;
+        std::memset(&v, 0, sizeof v);
+        v.accessPolicyWindow.base_ptr = ctx->pool;
+        v.accessPolicyWindow.num_bytes = ctx->l2_window;
+        v.accessPolicyWindow.hitRatio = ctx->l2_ratio;
+        v.accessPolicyWindow.hitProp = cudaAccessPropertyPersisting;
+        v.accessPolicyWindow.missProp = cudaAccessPropertyStreaming;
+        if (cudaStreamSetAttribute(s, cudaStreamAttributeAccessPolicyWindow, &v) != cudaSuccess) {
+            cudaGetLastError();
+            return;
+        }
+        on = true;
+        ctx->st_l2 = 1;
+    }
+    ~L2Window()
+    {
+        if (on && cudaStreamSetAttribute(s, cudaStreamAttributeAccessPolicyWindow, &prev) != cudaSuccess)
+            cudaGetLastError();
+    }
+};
 
 bool offsets_ok32(const int32_t* off, int32_t n)
 {
@@ -477,6 +754,7 @@ ckv_status ckv_destroy(ckv_ctx* ctx)
         if (b) cudaFree(b);
     for (auto& e : ctx->ev)
         if (e) cudaEventDestroy(e);
+    l2_release(ctx);
     cudaGetLastError();
     delete ctx;
     return CKV_OK;
@@ -510,6 +788,7 @@ ckv_status ckv_pool_load(ckv_ctx* ctx, const void* pool_K, const void* pool_V, i
     CK(launch_pool_layout(ctx->cfg.dtype, G, n_entries, d_shared, D, sk.dev, ctx->pool, s));
     CK(launch_pool_layout(ctx->cfg.dtype, G, n_entries, d_shared, D, sv.dev, (char*)ctx->pool + half, s));
     if (sk.owned || sv.owned) CK(cudaStreamSynchronize(s));
+    l2_prepare(ctx);
     if (ctx->users.empty() && (ctx->n_entries != n_entries || ctx->d_shared != d_shared)) {
         // index width or user width may change: restart the (empty) arena
         void* old[4] = {ctx->a_idxK, ctx->a_idxV, ctx->a_userK, ctx->a_userV};
@@ -517,6 +796,7 @@ ckv_status ckv_pool_load(ckv_ctx* ctx, const void* pool_K, const void* pool_V, i
             if (b) cudaFree(b);
         ctx->a_idxK = ctx->a_idxV = ctx->a_userK = ctx->a_userV = nullptr;
         ctx->cap_units = ctx->used_units = 0;
+        ctx->free_runs.clear();
     }
     ctx->n_entries = n_entries;
     ctx->d_shared = d_shared;
@@ -547,6 +827,12 @@ ckv_status ckv_cache_put_batch(ckv_ctx* ctx, int32_t n, const int64_t* users, co
 
     DeviceGuard dg(ctx->cfg.device);
     cudaStream_t s = (cudaStream_t)stream;
+    try {
+        ctx->users.reserve_more((size_t)n);
+    } catch (const std::bad_alloc&) {
+        return CKV_ERR_OOM;
+    }
+    int64_t base = 0;
     if (total_units > 0) {
         Staged sik, siv, suk, suv, sho, suo;
         const size_t ib = (size_t)P * G * sizeof(int32_t), ubytes = (size_t)P * G * d_user * ctx->elem;
@@ -556,26 +842,29 @@ ckv_status ckv_cache_put_batch(ckv_ctx* ctx, int32_t n, const int64_t* users, co
         CK(suv.init(user_V, ubytes, s));
         CK(sho.init(hist_off, sizeof(int64_t) * ((size_t)n + 1), s));
         CK(suo.init(unit_off.data(), sizeof(int64_t) * ((size_t)n + 1), s));
-        ckv_status st = ensure_arena(ctx, total_units, s);
+        ckv_status st = arena_take(ctx, total_units, s, &base);
         if (st != CKV_OK) return st;
-        CK(cudaMemsetAsync(ctx->d_flag, 0, sizeof(int), s));
-        CK(launch_pack(ctx->cfg.dtype, G, ctx->n_entries, d_user, ctx->idx_bytes, n, (const int64_t*)sho.dev,
-                       (const int64_t*)suo.dev, total_units, ctx->used_units, (const int32_t*)sik.dev,
-                       (const int32_t*)siv.dev, suk.dev, suv.dev, ctx->a_idxK, ctx->a_idxV, ctx->a_userK,
-                       ctx->a_userV, ctx->d_flag, s));
+        cudaError_t e = cudaMemsetAsync(ctx->d_flag, 0, sizeof(int), s);
+        if (e == cudaSuccess)
+            e = launch_pack(ctx->cfg.dtype, G, ctx->n_entries, d_user, ctx->idx_bytes, n, (const int64_t*)sho.dev,
+                            (const int64_t*)suo.dev, total_units, base, (const int32_t*)sik.dev,
+                            (const int32_t*)siv.dev, suk.dev, suv.dev, ctx->a_idxK, ctx->a_idxV, ctx->a_userK,
+                            ctx->a_userV, ctx->d_flag, s);
         int bad = 0;
-        CK(cudaMemcpyAsync(&bad, ctx->d_flag, sizeof(int), cudaMemcpyDeviceToHost, s));
-        CK(cudaStreamSynchronize(s));
-        if (bad) return CKV_ERR_INDEX_RANGE;  // used_units not advanced: nothing was stored
+        if (e == cudaSuccess) e = cudaMemcpyAsync(&bad, ctx->d_flag, sizeof(int), cudaMemcpyDeviceToHost, s);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+        if (e != cudaSuccess || bad) {  // nothing was stored: the units go back
+            arena_give(ctx, base, total_units);
+            return e != cudaSuccess ? ctx->fail(e) : CKV_ERR_INDEX_RANGE;
+        }
     }
     for (int32_t k = 0; k < n; ++k) {
         const int64_t L = hist_off[k + 1] - hist_off[k];
-        auto f = ctx->users.find(users[k]);
-        if (f != ctx->users.end()) ctx->live_positions -= f->second.L;
-        ctx->users[users[k]] = UserEntry{ctx->used_units + unit_off[k], (int32_t)L, (int32_t)((L + 31) / 32 * 32)};
-        ctx->live_positions += L;
+        UserEntry* f = ctx->users.insert(users[k]);
+        if (f->Lpad > 0) arena_give(ctx, f->base, (int64_t)G * f->Lpad);  // the entry this one replaces
+        ctx->live_positions += L - f->L;
+        *f = UserEntry{base + unit_off[k], (int32_t)L, (int32_t)((L + 31) / 32 * 32)};
     }
-    ctx->used_units += total_units;
     ctx->generation++;
     return CKV_OK;
 }
@@ -594,11 +883,11 @@ ckv_status ckv_cache_append(ckv_ctx* ctx, int64_t user, int32_t L_new, const int
     if (!ctx || L_new < 0) return CKV_ERR_INVALID_ARG;
     if (!ctx->pool) return CKV_ERR_STATE;
     if (d_user != ctx->d_user) return CKV_ERR_SHAPE;
-    auto f = ctx->users.find(user);
-    if (f == ctx->users.end()) return CKV_ERR_UNKNOWN_USER;
+    UserEntry* f = ctx->users.find(user);
+    if (!f) return CKV_ERR_UNKNOWN_USER;
     if (L_new == 0) return CKV_OK;
     if (!idx_K || !idx_V || (d_user > 0 && (!user_K || !user_V))) return CKV_ERR_INVALID_ARG;
-    const UserEntry old = f->second;
+    const UserEntry old = *f;
     if ((int64_t)old.L + L_new > INT32_MAX - 32) return CKV_ERR_INVALID_ARG;
     const int G = ctx->cfg.n_groups;
     const int32_t L_tot = old.L + L_new, Lpad_tot = (L_tot + 31) / 32 * 32;
@@ -611,20 +900,26 @@ ckv_status ckv_cache_append(ckv_ctx* ctx, int64_t user, int32_t L_new, const int
     if (idx_V == idx_K) siv.dev = sik.dev; else CK(siv.init(idx_V, ib, s));
     CK(suk.init(user_K, ubytes, s));
     CK(suv.init(user_V, ubytes, s));
-    // the longer history takes fresh units behind what is stored (the arena only grows until it is cleared)
-    ckv_status st = ensure_arena(ctx, units, s);
+    // the longer history is written to a run of its own (the old units are read while it is written) and the
+    // old run is given back afterwards
+    int64_t base = 0;
+    ckv_status st = arena_take(ctx, units, s, &base);
     if (st != CKV_OK) return st;
-    CK(cudaMemsetAsync(ctx->d_flag, 0, sizeof(int), s));
-    CK(launch_append(ctx->cfg.dtype, G, ctx->n_entries, d_user, ctx->idx_bytes, old.base, old.L, old.Lpad,
-                     ctx->used_units, L_new, Lpad_tot, (const int32_t*)sik.dev, (const int32_t*)siv.dev, suk.dev,
-                     suv.dev, ctx->a_idxK, ctx->a_idxV, ctx->a_userK, ctx->a_userV, ctx->d_flag, s));
+    cudaError_t e = cudaMemsetAsync(ctx->d_flag, 0, sizeof(int), s);
+    if (e == cudaSuccess)
+        e = launch_append(ctx->cfg.dtype, G, ctx->n_entries, d_user, ctx->idx_bytes, old.base, old.L, old.Lpad, base,
+                          L_new, Lpad_tot, (const int32_t*)sik.dev, (const int32_t*)siv.dev, suk.dev, suv.dev,
+                          ctx->a_idxK, ctx->a_idxV, ctx->a_userK, ctx->a_userV, ctx->d_flag, s);
     int bad = 0;
-    CK(cudaMemcpyAsync(&bad, ctx->d_flag, sizeof(int), cudaMemcpyDeviceToHost, s));
-    CK(cudaStreamSynchronize(s));
-    if (bad) return CKV_ERR_INDEX_RANGE;  // used_units not advanced: the user keeps the old history
-    f->second = UserEntry{ctx->used_units, L_tot, Lpad_tot};
+    if (e == cudaSuccess) e = cudaMemcpyAsync(&bad, ctx->d_flag, sizeof(int), cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess || bad) {  // the user keeps the old history
+        arena_give(ctx, base, units);
+        return e != cudaSuccess ? ctx->fail(e) : CKV_ERR_INDEX_RANGE;
+    }
+    arena_give(ctx, old.base, (int64_t)G * old.Lpad);
+    *f = UserEntry{base, L_tot, Lpad_tot};
     ctx->live_positions += L_new;
-    ctx->used_units += units;
     ctx->generation++;
     return CKV_OK;
 }
@@ -666,9 +961,9 @@ ckv_status ckv_cache_export(ckv_ctx* ctx, int32_t n, const int64_t* users, void*
     if (!ctx->pool) return CKV_ERR_STATE;
     int64_t total = 0;
     for (int32_t k = 0; k < n; ++k) {
-        auto f = ctx->users.find(users[k]);
-        if (f == ctx->users.end()) return CKV_ERR_UNKNOWN_USER;
-        total += units_of(ctx, f->second.L);
+        const UserEntry* f = ctx->users.find(users[k]);
+        if (!f) return CKV_ERR_UNKNOWN_USER;
+        total += units_of(ctx, f->L);
     }
     int64_t off[5];
     blob_sections(ctx, total, off);
@@ -681,7 +976,7 @@ ckv_status ckv_cache_export(ckv_ctx* ctx, int32_t n, const int64_t* users, void*
                           (const char*)ctx->a_userV};
     int64_t done = 0;
     for (int32_t k = 0; k < n; ++k) {
-        const UserEntry& e = ctx->users.find(users[k])->second;
+        const UserEntry& e = *ctx->users.find(users[k]);
         const int64_t u = units_of(ctx, e.L);
         for (int i = 0; i < 4 && u > 0; ++i)
             if (eb[i] > 0)
@@ -710,32 +1005,43 @@ ckv_status ckv_cache_import(ckv_ctx* ctx, int32_t n, const int64_t* users, const
     if (bytes != off[4] || (total > 0 && !blob)) return CKV_ERR_INVALID_ARG;
     DeviceGuard dg(ctx->cfg.device);
     cudaStream_t s = (cudaStream_t)stream;
+    try {
+        ctx->users.reserve_more((size_t)n);
+    } catch (const std::bad_alloc&) {
+        return CKV_ERR_OOM;
+    }
+    int64_t base = 0;
     if (total > 0) {
-        ckv_status st = ensure_arena(ctx, total, s);
+        ckv_status st = arena_take(ctx, total, s, &base);
         if (st != CKV_OK) return st;
         const int64_t ub = (int64_t)ctx->d_user * ctx->elem;
         const int64_t eb[4] = {ctx->idx_bytes, ctx->idx_bytes, ub, ub};
         char* dst[4] = {(char*)ctx->a_idxK, (char*)ctx->a_idxV, (char*)ctx->a_userK, (char*)ctx->a_userV};
-        // the batch takes contiguous units behind what is stored: one copy per section
-        for (int i = 0; i < 4; ++i)
+        // the batch takes one run of contiguous units: one copy per section
+        cudaError_t e = cudaSuccess;
+        for (int i = 0; i < 4 && e == cudaSuccess; ++i)
             if (eb[i] > 0)
-                CK(cudaMemcpyAsync(dst[i] + ctx->used_units * eb[i], (const char*)blob + off[i],
-                                   (size_t)(total * eb[i]), cudaMemcpyDefault, s));
-        CK(cudaMemsetAsync(ctx->d_flag, 0, sizeof(int), s));
-        CK(launch_check_indices(ctx->idx_bytes, ctx->n_entries, dst[0] + ctx->used_units * eb[0],
-                                dst[1] + ctx->used_units * eb[1], total, ctx->d_flag, s));
+                e = cudaMemcpyAsync(dst[i] + base * eb[i], (const char*)blob + off[i], (size_t)(total * eb[i]),
+                                    cudaMemcpyDefault, s);
+        if (e == cudaSuccess) e = cudaMemsetAsync(ctx->d_flag, 0, sizeof(int), s);
+        if (e == cudaSuccess)
+            e = launch_check_indices(ctx->idx_bytes, ctx->n_entries, dst[0] + base * eb[0], dst[1] + base * eb[1],
+                                     total, ctx->d_flag, s);
         int bad = 0;
-        CK(cudaMemcpyAsync(&bad, ctx->d_flag, sizeof(int), cudaMemcpyDeviceToHost, s));
-        CK(cudaStreamSynchronize(s));
-        if (bad) return CKV_ERR_INDEX_RANGE;  // used_units not advanced: nothing was stored
+        if (e == cudaSuccess) e = cudaMemcpyAsync(&bad, ctx->d_flag, sizeof(int), cudaMemcpyDeviceToHost, s);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+        if (e != cudaSuccess || bad) {  // nothing was stored: the units go back
+            arena_give(ctx, base, total);
+            return e != cudaSuccess ? ctx->fail(e) : CKV_ERR_INDEX_RANGE;
+        }
     }
+    const int G = ctx->cfg.n_groups;
     for (int32_t k = 0; k < n; ++k) {
-        auto f = ctx->users.find(users[k]);
-        if (f != ctx->users.end()) ctx->live_positions -= f->second.L;
-        ctx->users[users[k]] = UserEntry{ctx->used_units + unit_off[k], L[k], (L[k] + 31) / 32 * 32};
-        ctx->live_positions += L[k];
+        UserEntry* f = ctx->users.insert(users[k]);
+        if (f->Lpad > 0) arena_give(ctx, f->base, (int64_t)G * f->Lpad);  // the entry this one replaces
+        ctx->live_positions += L[k] - f->L;
+        *f = UserEntry{base + unit_off[k], L[k], (L[k] + 31) / 32 * 32};
     }
-    ctx->used_units += total;
     ctx->generation++;
     return CKV_OK;
 }
@@ -743,12 +1049,12 @@ ckv_status ckv_cache_import(ckv_ctx* ctx, int32_t n, const int64_t* users, const
 ckv_status ckv_cache_evict(ckv_ctx* ctx, int64_t user)
 {
     if (!ctx) return CKV_ERR_INVALID_ARG;
-    auto f = ctx->users.find(user);
-    if (f == ctx->users.end()) return CKV_ERR_UNKNOWN_USER;
-    ctx->live_positions -= f->second.L;
-    ctx->users.erase(f);
+    const UserEntry* f = ctx->users.find(user);
+    if (!f) return CKV_ERR_UNKNOWN_USER;
+    ctx->live_positions -= f->L;
+    arena_give(ctx, f->base, (int64_t)ctx->cfg.n_groups * f->Lpad);
+    ctx->users.erase(user);
     ctx->generation++;
-    if (ctx->users.empty()) ctx->used_units = 0;
     return CKV_OK;
 }
 
@@ -756,6 +1062,7 @@ ckv_status ckv_cache_clear(ckv_ctx* ctx)
 {
     if (!ctx) return CKV_ERR_INVALID_ARG;
     ctx->users.clear();
+    ctx->free_runs.clear();
     ctx->live_positions = 0;
     ctx->used_units = 0;
     ctx->generation++;
@@ -791,6 +1098,7 @@ ckv_status ckv_attend(ckv_ctx* ctx, int32_t n, const int64_t* users, const int32
     DeviceGuard dg(ctx->cfg.device);
     cudaStream_t s = (cudaStream_t)stream;
     ctx->st_launches = 0;
+    ctx->st_allocs = 0;
     Plan* pl = nullptr;
     ckv_status st = get_plan(ctx, n, users, q_off, s, &pl);
     if (st != CKV_OK) return st;
@@ -806,20 +1114,21 @@ ckv_status ckv_attend(ckv_ctx* ctx, int32_t n, const int64_t* users, const int32
     void* d_out = out;
     const bool q_host = !is_device_ptr(queries), o_host = !is_device_ptr(out);
     if (q_host) {
-        CK(grow(ctx->stage_q, q_bytes));
+        CK(grow(ctx->stage_q, q_bytes, &ctx->st_allocs));
         CK(cudaMemcpyAsync(ctx->stage_q.p, queries, q_bytes, cudaMemcpyHostToDevice, s));
         d_q = ctx->stage_q.p;
     }
     if (o_host) {
-        CK(grow(ctx->stage_out, o_bytes));
+        CK(grow(ctx->stage_out, o_bytes, &ctx->st_allocs));
         d_out = ctx->stage_out.p;
     }
     // split-reduction partials, or the factorisation's tables (per request and group: n_entries + a few floats)
     const size_t ws = pl->family == 4
                           ? (size_t)pl->n_req * G * ((size_t)fact_row_floats(ctx->n_entries) + fact_aux_floats()) * sizeof(float)
                           : (size_t)pl->part_rows * G * (D + 2) * sizeof(float);
-    if (ws) CK(grow(ctx->partials, ws));
+    if (ws) CK(grow(ctx->partials, ws, &ctx->st_allocs));
     ctx->st_ws = (int64_t)ws;
+    L2Window l2(ctx, s);
 
     AttendArgs a;
     a.cv = view_of(ctx);
@@ -871,9 +1180,9 @@ ckv_status ckv_materialize(ckv_ctx* ctx, int64_t user, void* K_out, void* V_out,
 {
     if (!ctx || !K_out || !V_out) return CKV_ERR_INVALID_ARG;
     if (!ctx->pool) return CKV_ERR_STATE;
-    auto f = ctx->users.find(user);
-    if (f == ctx->users.end()) return CKV_ERR_UNKNOWN_USER;
-    const UserEntry& e = f->second;
+    const UserEntry* f = ctx->users.find(user);
+    if (!f) return CKV_ERR_UNKNOWN_USER;
+    const UserEntry& e = *f;
     if (e.L == 0) return CKV_OK;
     DeviceGuard dg(ctx->cfg.device);
     cudaStream_t s = (cudaStream_t)stream;
@@ -906,9 +1215,9 @@ ckv_status ckv_materialize(ckv_ctx* ctx, int64_t user, void* K_out, void* V_out,
 ckv_status ckv_user_length(ckv_ctx* ctx, int64_t user, int64_t* L)
 {
     if (!ctx || !L) return CKV_ERR_INVALID_ARG;
-    auto f = ctx->users.find(user);
-    if (f == ctx->users.end()) return CKV_ERR_UNKNOWN_USER;
-    *L = f->second.L;
+    const UserEntry* f = ctx->users.find(user);
+    if (!f) return CKV_ERR_UNKNOWN_USER;
+    *L = f->L;
     return CKV_OK;
 }
 
@@ -1040,6 +1349,11 @@ ckv_status ckv_last_stat(ckv_ctx* ctx, const char* name, int64_t* value)
     else if (!std::strcmp(name, "mma_loader")) *value = ctx->st_loader;
     else if (!std::strcmp(name, "workspace_bytes")) *value = ctx->st_ws;
     else if (!std::strcmp(name, "plan_cache_hit")) *value = ctx->st_hit;
+    else if (!std::strcmp(name, "alloc_calls")) *value = ctx->st_allocs;
+    else if (!std::strcmp(name, "l2_window")) *value = ctx->st_l2;
+    else if (!std::strcmp(name, "arena_capacity_units")) *value = ctx->cap_units;
+    else if (!std::strcmp(name, "arena_used_units")) *value = ctx->used_units;
+    else if (!std::strcmp(name, "arena_free_runs")) *value = (int64_t)ctx->free_runs.size();
     else if (!std::strcmp(name, "device_errors")) {
         DeviceGuard dg(ctx->cfg.device);
         int v = 0;
@@ -1088,7 +1402,9 @@ int32_t ckv_version(void) { return 100; }
 // Everything ckv_attend would put into freshly allocated or grown device memory -- the
 // request/work-item tables and the partial results of the split-along-history reduction --
 // lives in one fixed array in the library's device image instead.  The array exists once per
-// GPU that loads the library and is shared by every call on that GPU.
+// GPU that loads the library and is shared by every call on that GPU.  The tables reach it as
+// kernel arguments of a small kernel that writes them out, so no host buffer has to outlive the
+// call and no copy from pageable memory is enqueued.
 // ------------------------------------------------------------------------------------------
 namespace {
 
@@ -1120,6 +1436,42 @@ cudaError_t static_scratch_address(int device, void** out)
     return cudaSuccess;
 }
 
+// One launch carries the plan rows of up to kStaticChunk requests as its argument (under the 4 KB that
+// kernel arguments may take) and thread t writes request t's row, its history chunks and its entry of
+// the split list into the array.
+constexpr int kStaticChunk = 80;
+struct StaticRow {
+    Req req;
+    int32_t item0;       // first work item of the request (-1: no queries, no items)
+    int32_t split_slot;  // position in the list of split requests, or -1
+    int32_t chunk_len;   // positions per history chunk
+};
+struct StaticRows {
+    int32_t first, count;
+    StaticRow row[kStaticChunk];
+};
+static_assert(sizeof(StaticRows) <= 4000, "kernel arguments");
+
+__global__ void static_plan_kernel(const StaticRows rows)
+{
+    const int t = threadIdx.x;
+    if (t >= rows.count) return;
+    const StaticRow& r = rows.row[t];
+    const int k = rows.first + t;
+    reinterpret_cast<Req*>(ckv_static_scratch)[k] = r.req;
+    if (r.item0 < 0) return;
+    Item* items = reinterpret_cast<Item*>(ckv_static_scratch + kOffItems) + r.item0;
+    if (r.split_slot < 0) {
+        items[0] = Item{k, 0, r.req.L, -1};
+        return;
+    }
+    reinterpret_cast<int32_t*>(ckv_static_scratch + kOffSplit)[r.split_slot] = k;
+    for (int c = 0; c < r.req.n_chunks; ++c) {
+        const int b = c * r.chunk_len;
+        items[c] = Item{k, b, min(r.chunk_len, r.req.L - b), r.req.part0 + c * r.req.M};
+    }
+}
+
 }  // namespace
 
 extern "C" ckv_status ckv_attend_static(ckv_ctx* ctx, int32_t n, const int64_t* users, const int32_t* q_off,
@@ -1140,20 +1492,18 @@ extern "C" ckv_status ckv_attend_static(ckv_ctx* ctx, int32_t n, const int64_t* 
     void* scratch = nullptr;
     CK(static_scratch_address(ctx->cfg.device, &scratch));
 
-    // the plan, in fixed-size host arrays
-    Req reqs[kStaticMaxReqs];
-    Item items[kStaticMaxItems];
-    int32_t split[kStaticMaxReqs];
+    // the plan, in fixed-size host arrays; nothing is enqueued before the request is known to fit
+    StaticRow rows[kStaticMaxReqs];
     const int D = ctx->cfg.head_dim, G = ctx->cfg.n_groups;
     int64_t total_pos = 0;
     int32_t max_M = 0;
     for (int32_t k = 0; k < n; ++k) {
-        auto f = ctx->users.find(users[k]);
-        if (f == ctx->users.end()) return CKV_ERR_UNKNOWN_USER;
-        Req& r = reqs[k];
-        r.base = f->second.base;
-        r.L = f->second.L;
-        r.Lpad = f->second.Lpad;
+        const UserEntry* f = ctx->users.find(users[k]);
+        if (!f) return CKV_ERR_UNKNOWN_USER;
+        Req& r = rows[k].req;
+        r.base = f->base;
+        r.L = f->L;
+        r.Lpad = f->Lpad;
         r.q0 = q_off[k];
         r.M = q_off[k + 1] - q_off[k];
         r.part0 = -1;
@@ -1172,31 +1522,33 @@ extern "C" ckv_status ckv_attend_static(ckv_ctx* ctx, int32_t n, const int64_t* 
     int32_t n_items = 0, n_split = 0;
     int64_t part_rows = 0;
     for (int32_t k = 0; k < n; ++k) {
-        Req& r = reqs[k];
+        StaticRow& row = rows[k];
+        Req& r = row.req;
+        row.item0 = row.split_slot = -1;
+        row.chunk_len = (int32_t)std::min<int64_t>(C, INT32_MAX);
         if (r.M <= 0) continue;
         const int64_t nc = r.L == 0 ? 1 : (r.L + C - 1) / C;
         if (n_items + nc > kStaticMaxItems) return CKV_ERR_TOO_LARGE;
         r.n_chunks = (int32_t)nc;
-        if (nc == 1) {
-            items[n_items++] = Item{k, 0, r.L, -1};
-            continue;
-        }
+        row.item0 = n_items;
+        n_items += (int32_t)nc;
+        if (nc == 1) continue;
         if (part_rows + nc * r.M > cap_rows) return CKV_ERR_TOO_LARGE;
         r.part0 = (int32_t)part_rows;
-        split[n_split++] = k;
-        for (int64_t c = 0; c < nc; ++c) {
-            const int32_t b = (int32_t)(c * C);
-            items[n_items++] = Item{k, b, (int32_t)std::min<int64_t>(C, r.L - b), (int32_t)(part_rows + c * r.M)};
-        }
+        row.split_slot = n_split++;
         part_rows += nc * r.M;
     }
-    std::stable_sort(items, items + n_items, [](const Item& x, const Item& y) { return x.len > y.len; });
+
+    for (int32_t k0 = 0; k0 < n; k0 += kStaticChunk) {
+        StaticRows arg;
+        arg.first = k0;
+        arg.count = std::min<int32_t>(kStaticChunk, n - k0);
+        std::memcpy(arg.row, rows + k0, sizeof(StaticRow) * (size_t)arg.count);
+        static_plan_kernel<<<1, kStaticChunk, 0, s>>>(arg);
+        CK(cudaGetLastError());
+    }
 
     char* base = (char*)scratch;
-    CK(cudaMemcpyAsync(base, reqs, sizeof(Req) * (size_t)n, cudaMemcpyHostToDevice, s));
-    if (n_items) CK(cudaMemcpyAsync(base + kOffItems, items, sizeof(Item) * (size_t)n_items, cudaMemcpyHostToDevice, s));
-    if (n_split) CK(cudaMemcpyAsync(base + kOffSplit, split, sizeof(int32_t) * (size_t)n_split, cudaMemcpyHostToDevice, s));
-
     AttendArgs a;
     a.cv = view_of(ctx);
     a.reqs = (const Req*)base;

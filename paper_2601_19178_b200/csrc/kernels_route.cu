@@ -12,6 +12,7 @@
 #include <math_constants.h>
 
 #include "ckv_internal.h"
+#include "ptx_helpers.cuh"
 
 namespace ckv {
 namespace {
@@ -20,16 +21,6 @@ constexpr int kRouteWarps = 8, kRouteChunk = 64;
 // 16-position tiles per warp: every weight fragment read from shared memory serves that many MMAs
 __host__ __device__ constexpr int route_mt(int) { return 2; }  // (four measured no faster: 334 against 342 TFLOP/s)
 __host__ __device__ constexpr int route_rows(int d_in) { return kRouteWarps * 16 * route_mt(d_in); }  // positions per CTA
-
-__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
-{
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
-        "{%0,%1,%2,%3};\n"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 // 16-byte chunk c of ring row r sits at chunk c ^ swz(r): the eight rows of an ldmatrix block (consecutive
 // entries) fall into eight different bank groups

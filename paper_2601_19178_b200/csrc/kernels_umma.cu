@@ -45,11 +45,9 @@
 // returns.
 #include <cuda_bf16.h>
 #include <math_constants.h>
-#ifdef CKV_STAGE_TIMERS
-#include <cstdio>
-#endif
 
 #include "ckv_internal.h"
+#include "ptx_helpers.cuh"
 
 namespace ckv {
 namespace {
@@ -101,8 +99,6 @@ static_assert(BAR_COUNT * 8 <= 320, "barrier area");
 
 // error codes OR-ed into the context's device error word
 enum { ERR_NORMALISE = 1, ERR_MMA = 2, ERR_DRAIN = 4, ERR_PRODUCER = 8 };
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
 {
@@ -246,43 +242,12 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
         : "memory");
 }
 
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
-{
-    uint32_t r;
-    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-    return r;
-}
-__device__ __forceinline__ float ex2(float x)
-{
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-__device__ __forceinline__ float tanh_fast(float x)
-{
-    float y;
-    asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
 __device__ __forceinline__ float max3(float a, float b, float c)
 {
     float r;
     asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
     return r;
 }
-
-// Optional stage timers (debug builds with -DCKV_STAGE_TIMERS): one thread per role of CTA 0
-// accumulates clock64 intervals per stage and prints them when the kernel ends.
-#ifdef CKV_STAGE_TIMERS
-__device__ __forceinline__ unsigned long long t_global_ns() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
-#define T_DECL(n) long long tmr_[n] = {}; long long tmr_last_ = clock64(); const long long tmr_start_ = tmr_last_; const unsigned long long tmr_ns0_ = t_global_ns()
-#define T_MHZ() (1e3 * (double)(clock64() - tmr_start_) / (double)(t_global_ns() - tmr_ns0_))
-#define T_ACC(i) do { const long long t_now_ = clock64(); tmr_[i] += t_now_ - tmr_last_; tmr_last_ = t_now_; } while (0)
-#define T_TOTAL() (clock64() - tmr_start_)
-#else
-#define T_DECL(n) do {} while (0)
-#define T_ACC(i) do {} while (0)
-#endif
 
 // byte offset of (row r, 16-byte chunk c) inside a K/Q tile and inside a V tile
 __device__ __forceinline__ uint32_t k_off(int r, int c) { return (uint32_t)((r >> 3) * 512 + c * 128 + (r & 7) * 16); }
@@ -615,11 +580,9 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
         int ocnt = 0;   // units in which this group had tiles
         int xcnt = 0;   // units exchanged between the groups
         bool ok = true;
-        T_DECL(8);  // 0 other, 1 wait S, 2 wait PFREE, 3 read O, 4 tile, 5 wait O, 6 exchange wait, 7 next unit
         Stream<true> sn;
         sn.init(a, n_mb, n_work);
         for (; sn.valid && ok; sn.next_unit()) {
-            T_ACC(7);  // (time since the end of the previous unit's body: next_unit)
             const Unit& u = sn.u;
             const int r = u.row0 + row;
             const int64_t out_base = ((int64_t)(u.wk.q0 + r) * G + u.grp) * D;
@@ -642,13 +605,10 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                 if (valid <= 0) continue;  // only the second half of a unit's last tile can be empty
                 const int i = cnt & 1;     // buffer pair of this step
                 const uint32_t tS = tS0 + 64u * i, tP = tP0 + 32u * i;
-                T_ACC(0);
                 ok = mbar_wait(bar(BAR_SFULL + 2 * b + i), (cnt >> 1) & 1, abort_flag);
-                T_ACC(1);
                 // P_bi is free once the weighted sum of two steps ago has been computed
                 if (ok && cnt >= 2) ok = mbar_wait(bar(BAR_PFREE + 2 * b + i), ((cnt >> 1) - 1) & 1, abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
-                T_ACC(2);
                 if (!ok) break;
                 tc_fence_after();
                 const bool tail = valid < TH;
@@ -680,7 +640,6 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                 tc_wait_st();
                 tc_fence_before();
                 mbar_arrive(bar(BAR_PREADY + 2 * b + i));
-                T_ACC(4);
                 ++cnt;
                 ++mine;
             }
@@ -688,11 +647,9 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
 
             // ---- the unit's epilogue: fetch O_b, merge the two groups, store
             float o[32], l = 0.f;
-            T_ACC(0);
             if (mine > 0) {
                 ok = mbar_wait(bar(BAR_OFULL + b), ocnt & 1, abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
-                T_ACC(5);
                 if (!ok) break;
                 ++ocnt;
                 tc_fence_after();
@@ -703,16 +660,13 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                 for (int e = 0; e < 32; ++e) o[e] = __uint_as_float(raw[e]);
                 if constexpr (MODE == CKV_SOFTMAX) l = __uint_as_float(tmem_ld1(tO + 32));
                 tc_fence_before();
-                T_ACC(3);
             } else {
 #pragma unroll
                 for (int e = 0; e < 32; ++e) o[e] = 0.f;
             }
             if (b == 1) {
-                T_ACC(0);
                 if (xcnt > 0) ok = mbar_wait(bar(BAR_XEMPTY), (xcnt - 1) & 1, abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
-                T_ACC(6);
                 if (!ok) break;
                 xch[row] = m_ref;
                 xch[128 + row] = l;
@@ -721,10 +675,8 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                 mbar_arrive(bar(BAR_XFULL));
                 ++xcnt;
             } else {
-                T_ACC(0);
                 ok = mbar_wait(bar(BAR_XFULL), xcnt & 1, abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
-                T_ACC(6);
                 if (!ok) break;
                 ++xcnt;
                 const float m1 = xch[row], l1 = xch[128 + row];
@@ -773,14 +725,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                     }
                 }
             }
-            T_ACC(0);
         }
-        T_ACC(0);
-#ifdef CKV_STAGE_TIMERS
-        if (blockIdx.x == 0 && row == 0)
-            printf("group %d: %.0f MHz total %lld | other %lld waitS %lld waitPfree %lld tile %lld waitO %lld readO %lld xchg %lld nextunit %lld | tiles %d\n", b,
-                   T_MHZ(), T_TOTAL(), tmr_[0], tmr_[1], tmr_[2], tmr_[4], tmr_[5], tmr_[3], tmr_[6], tmr_[7], cnt);
-#endif
         if (!ok) {
             *abort_flag = 1;
             if (lane == 0) atomicOr(err_flag, ERR_NORMALISE);
@@ -794,18 +739,14 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
             ss.init(a, n_mb, n_work);
             int cnt = 0;  // half tiles issued
             bool ok = true;
-            T_DECL(3);  // 0 issue, 1 wait FULL, 2 wait PREADY
             for (; ok && ss.valid; ss.advance()) {
                 const int s = ss.g % NS;
                 const bool last = ss.j == ss.u.n_tiles - 1;
                 if ((last ? ss.u.last_valid : TK) > TH * b) {  // else: empty second half
                     const int i = cnt & 1;
-                    T_ACC(0);
                     ok = mbar_wait(bar(BAR_FULL + s), (ss.g / NS) & 1, abort_flag);
-                    T_ACC(1);
                     // S_bi is free once the group has read the half tile of two steps ago
                     if (ok && cnt >= 2) ok = mbar_wait(bar(BAR_PREADY + 2 * b + i), ((cnt >> 1) - 1) & 1, abort_flag);
-                    T_ACC(2);
                     if (!ok) break;
                     tc_fence_after();
                     ++cnt;
@@ -826,11 +767,6 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                     tc_commit(bar(BAR_QEMPTY + ss.useq % NQ));
                 }
             }
-            T_ACC(0);
-#ifdef CKV_STAGE_TIMERS
-            if (blockIdx.x == 0)
-                printf("S issue %d: total %lld | issue %lld waitFULL %lld waitPREADY %lld | tiles %d\n", b, T_TOTAL(), tmr_[0], tmr_[1], tmr_[2], cnt);
-#endif
             if (!ok) {
                 *abort_flag = 1;
                 atomicOr(err_flag, ERR_MMA);
@@ -850,7 +786,6 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
             sp.init(a, n_mb, n_work);
             int cnt = 0;
             bool ok = true;
-            T_DECL(2);  // 0 issue, 1 wait PREADY
             for (; ok && sp.valid; sp.advance()) {
                 const int s = sp.g % NS;
                 const int valid = (sp.j == sp.u.n_tiles - 1 ? sp.u.last_valid : TK) - TH * b;
@@ -860,10 +795,8 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                     continue;
                 }
                 const int i = cnt & 1;
-                T_ACC(0);
                 ok = mbar_wait(bar(BAR_PREADY + 2 * b + i), (cnt >> 1) & 1, abort_flag);
                 if (ok) ok = mbar_wait(bar(BAR_FULL + s), (sp.g / NS) & 1, abort_flag);  // completed long ago: makes the V tile visible here
-                T_ACC(1);
                 if (!ok) break;
                 ++cnt;
                 tc_fence_after();
@@ -877,11 +810,6 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                 tc_commit(bar(BAR_PFREE + 2 * b + i));
                 if (last) tc_commit(bar(BAR_OFULL + b));  // the group's last step of the unit
             }
-            T_ACC(0);
-#ifdef CKV_STAGE_TIMERS
-            if (blockIdx.x == 0)
-                printf("PV issue %d: total %lld | issue %lld waitPREADY %lld | tiles %d\n", b, T_TOTAL(), tmr_[0], tmr_[1], cnt);
-#endif
             if (!ok) {
                 *abort_flag = 1;
                 atomicOr(err_flag, ERR_MMA);
@@ -936,7 +864,6 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
             }
         };
         fetch();
-        T_DECL(6);  // 0 other, 1 wait copies, 2 wait EMPTY, 3 wait QEMPTY, 4 patch+publish, 5 copy issue
         while (st.valid && ok) {
             const int s = st.g % NS;
             UserPart<DUB> uk[4], uv[4];
@@ -948,12 +875,10 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
             *reinterpret_cast<uint2*>(sidxK + 4 * lane) = xk;
             *reinterpret_cast<uint2*>(sidxV + 4 * lane) = xv;
             __syncwarp();
-            T_ACC(0);
             if (st.g >= NS) {
                 if (lane == 0) ok = mbar_wait(bar(BAR_EMPTY + s), ((st.g / NS) - 1) & 1, abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
             }
-            T_ACC(2);
             if (!ok) break;
             if (st.j == 0) {  // a new unit: stage its Q block (rows beyond M are zero)
                 if (st.useq >= NQ) {
@@ -961,7 +886,6 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                 }
-                T_ACC(3);
                 const uint32_t qdst = sbase + kOffQ + (st.useq % NQ) * kTileK + kv_lane;
                 const int rows_in = st.u.wk.M - st.u.row0;
                 const uint16_t* qsrc = Q + ((int64_t)(st.u.wk.q0 + st.u.row0 + q) * G + st.u.grp) * D + chunk * 8;
@@ -983,14 +907,11 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                 cp_async16(vdst + kVGroup * it, pv + (size_t)sidxV[pos] * (D * 2), nb);
             }
             cp_async_commit();
-            T_ACC(5);
             // what this warp's next tile needs travels while the copies land
             for (int i = 0; i < kProducerWarps && st.valid; ++i) st.advance();
             fetch();
-            T_ACC(0);
             cp_async_wait<0>();
             __syncwarp();  // a row's chunks were copied by four lanes of this warp
-            T_ACC(1);
             if constexpr (DUB > 0) {
 #pragma unroll
                 for (int rb = 0; rb < 4; ++rb) {
@@ -1003,15 +924,8 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
             fence_proxy_async();  // by the writing threads themselves: a fence on the reading side alone is not enough
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(BAR_FULL + s));
-            T_ACC(4);
         }
         cp_async_wait<0>();
-        T_ACC(0);
-#ifdef CKV_STAGE_TIMERS
-        if (blockIdx.x == 0 && lane == 0)
-            printf("producer %d: total %lld | other %lld waitcopies %lld waitEMPTY %lld waitQEMPTY %lld publish %lld copies %lld\n", pw, T_TOTAL(),
-                   tmr_[0], tmr_[1], tmr_[2], tmr_[3], tmr_[4], tmr_[5]);
-#endif
         if (!ok) {
             *abort_flag = 1;
             if (lane == 0) atomicOr(err_flag, ERR_PRODUCER);

@@ -23,6 +23,7 @@ round-to-nearest-even).
 """
 from __future__ import annotations
 
+import concurrent.futures
 import dataclasses
 from dataclasses import dataclass
 from typing import Dict, Optional, Tuple
@@ -114,11 +115,20 @@ def _indices(rng: np.random.Generator, P: int, G: int, m: int, zipf_s: Optional[
     cdf = np.cumsum(w)
     cdf /= cdf[-1]
     out = np.empty((P, G), dtype=np.int32)
-    for g in range(G):
-        perm = rng.permutation(m).astype(np.int32)
-        ranks = np.searchsorted(cdf, rng.random(P), side="left")
+
+    def fill(g, perm, u):
+        ranks = np.searchsorted(cdf, u, side="left")
         np.minimum(ranks, m - 1, out=ranks)
         out[:, g] = perm[ranks]
+
+    # the draws stay in the stream's order (group by group); only the table look-ups run side by side
+    with concurrent.futures.ThreadPoolExecutor(max_workers=min(G, 4)) as ex:
+        pending = []
+        for g in range(G):
+            perm = rng.permutation(m).astype(np.int32)
+            pending.append(ex.submit(fill, g, perm, rng.random(P)))
+        for f in pending:
+            f.result()
     return out
 
 
@@ -136,17 +146,25 @@ def generate(w: Workload, seed: Optional[int] = None) -> Dict[str, np.ndarray]:
     P = int(hist_off[-1])
     q_off = (np.arange(U + 1, dtype=np.int64) * M).astype(np.int32)
     Q = int(q_off[-1])
-    data = {
-        "pool_K": _normal(s_pk, (G, m, dg), w.pool_var, w.dtype),
-        "pool_V": _normal(s_pv, (G, m, dg), w.pool_var, w.dtype),
-        "idx_K": _indices(s_ik, P, G, m, w.zipf_s),
-        "idx_V": _indices(s_iv, P, G, m, w.zipf_s),
-        "user_K": _normal(s_uk, (P, G, du), w.user_var, w.dtype),
-        "user_V": _normal(s_uv, (P, G, du), w.user_var, w.dtype),
-        "hist_off": hist_off,
-        "queries": _normal(s_q, (Q, G, d), 1.0, w.dtype),
-        "q_off": q_off,
-        # distinct, non-contiguous ids so that a lookup bug cannot hide behind id == slot
-        "users": (s_id.permutation(U).astype(np.int64) * 7919 + 1000003),
+    # every tensor has a random stream of its own, so the draws can run side by side (numpy releases the
+    # interpreter lock inside them) without changing a single value
+    jobs = {
+        "pool_K": lambda: _normal(s_pk, (G, m, dg), w.pool_var, w.dtype),
+        "pool_V": lambda: _normal(s_pv, (G, m, dg), w.pool_var, w.dtype),
+        "idx_K": lambda: _indices(s_ik, P, G, m, w.zipf_s),
+        "idx_V": lambda: _indices(s_iv, P, G, m, w.zipf_s),
+        "user_K": lambda: _normal(s_uk, (P, G, du), w.user_var, w.dtype),
+        "user_V": lambda: _normal(s_uv, (P, G, du), w.user_var, w.dtype),
+        "queries": lambda: _normal(s_q, (Q, G, d), 1.0, w.dtype),
     }
+    if P * G >= 1 << 20:
+        with concurrent.futures.ThreadPoolExecutor(max_workers=len(jobs)) as ex:
+            futures = {k: ex.submit(f) for k, f in jobs.items()}
+            data = {k: f.result() for k, f in futures.items()}
+    else:
+        data = {k: f() for k, f in jobs.items()}
+    data["hist_off"] = hist_off
+    data["q_off"] = q_off
+    # distinct, non-contiguous ids so that a lookup bug cannot hide behind id == slot
+    data["users"] = s_id.permutation(U).astype(np.int64) * 7919 + 1000003
     return data

@@ -160,3 +160,45 @@ def test_append_equals_put_of_the_whole_history(name):
     assert ckv.ckv_user_length(s.ctx, u0) == int(ho[1] - ho[0])
     assert np.array_equal(gpu_attend(w, d, session=s), want_out)
     s.close()
+
+
+def test_storage_of_replaced_and_evicted_users_is_reused():
+    """A cache that is updated continuously must not grow: replacing one user a thousand times, cycling
+    import / evict over a batch and appending to a user all hand their old storage back."""
+    import paper_2601_19178_b200 as B
+    w = synth.scaled(synth.WORKLOADS["cfg5"], n_users=24, hist_len=(40, 700))
+    d = synth.generate(w)
+    s = make_session(w, d)
+    cap0 = s.stat("arena_capacity_units")
+    G = w.n_groups
+    ho = d["hist_off"]
+    ik, iv = to_dev(d["idx_K"], "i"), to_dev(d["idx_V"], "i")
+    uk, uv = to_dev(d["user_K"], w.dtype), to_dev(d["user_V"], w.dtype)
+    want = gpu_attend(w, d, session=s)
+    # one user replaced 1000 times by histories of the other users' lengths
+    target = int(d["users"][3])
+    for r in range(1000):
+        u = r % w.n_users
+        sl = slice(int(ho[u]), int(ho[u + 1]))
+        s.cache_put(target, ik[sl], iv[sl], uk[sl], uv[sl])
+    sl = slice(int(ho[3]), int(ho[4]))
+    s.cache_put(target, ik[sl], iv[sl], uk[sl], uv[sl])
+    assert s.stat("arena_capacity_units") <= 2 * cap0
+    assert np.array_equal(gpu_attend(w, d, session=s), want)
+    # import / evict cycles of half the users
+    half = d["users"][: w.n_users // 2]
+    lens = np.diff(ho)[: w.n_users // 2].astype(np.int32)
+    blob = s.export_blob(half)
+    used = []
+    for _ in range(50):
+        for u in half:
+            B.ckv_cache_evict(s.ctx, int(u))
+        s.import_blob(half, lens, blob)
+        used.append(s.stat("arena_used_units"))
+    assert s.stat("arena_capacity_units") <= 2 * cap0 and max(used) <= 2 * cap0
+    assert np.array_equal(gpu_attend(w, d, session=s), want)
+    # everything evicted: nothing stays in use
+    for u in d["users"]:
+        B.ckv_cache_evict(s.ctx, int(u))
+    assert s.stat("arena_used_units") == 0 and s.stat("arena_free_runs") == 0
+    s.close()

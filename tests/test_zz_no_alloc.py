@@ -21,11 +21,12 @@ def _run(fn, s, users, q_off, q):
     return out.float().cpu().numpy().astype(np.float64)
 
 
-@pytest.mark.parametrize("name,kw", [
-    ("cfg4", dict(n_users=5, hist_len=(1, 5000), n_queries=2)),      # CUDA-core kernel, split histories
-    ("cfg5", dict(n_users=40, hist_len=(1, 900))),                   # tensor-core kernel
+@pytest.mark.parametrize("name,kw,family", [
+    ("cfg4", dict(n_users=5, hist_len=(1, 5000), n_queries=2), 2),   # warp-level tensor-core kernel, 64-wide heads
+    ("cfg5", dict(n_users=40, hist_len=(1, 900)), 2),                # warp-level tensor-core kernel, 32-wide heads
+    ("cfg1", dict(n_users=90, hist_len=(1, 1500), n_queries=3), 1),  # fp32: CUDA-core kernel; two table launches
 ])
-def test_static_entry_point_matches_ckv_attend_twice_in_a_row(name, kw):
+def test_static_entry_point_matches_ckv_attend_twice_in_a_row(name, kw, family):
     import paper_2601_19178_b200 as ckv
     w = synth.scaled(synth.WORKLOADS[name], **kw)
     d = synth.generate(w)
@@ -33,11 +34,17 @@ def test_static_entry_point_matches_ckv_attend_twice_in_a_row(name, kw):
     q = to_dev(d["queries"], w.dtype)
     want = _run(ckv.ckv_attend, s, d["users"], d["q_off"], q)
     assert s.stat("split_items") > 0, "the case must exercise the scratch memory"
+    assert s.stat("kernel") == family
+    # the first call on a device does the set-up (the driver may only now load the part of the library's device
+    # image that holds the array); from then on the device's free memory must not move (the output tensor of
+    # _run comes out of torch's cache, which the earlier runs of the same shape have filled)
     first = _run(ckv.ckv_attend_static, s, d["users"], d["q_off"], q)
+    free_before = torch.cuda.mem_get_info()[0]
     # a different request in between leaves other contents in the shared array
     half = w.n_users // 2
     _run(ckv.ckv_attend_static, s, d["users"][:half], d["q_off"][:half + 1], q[: int(d["q_off"][half])])
     second = _run(ckv.ckv_attend_static, s, d["users"], d["q_off"], q)
+    assert torch.cuda.mem_get_info()[0] == free_before, "ckv_attend_static changed the device's free memory"
     assert_close(first, want, w.dtype, "first call")
     assert_close(second, want, w.dtype, "second call")
     assert np.array_equal(first, second)

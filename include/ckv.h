@@ -105,6 +105,25 @@ CKV_API ckv_status ckv_pool_load(ckv_ctx* ctx, const void* pool_K, const void* p
                          int32_t n_entries, int32_t d_shared, void* stream);
 
 /*
+ * Sharing only the keys or only the values (ablation on sharing keys or values, Sec. 5.5: "CollectiveK"
+ * shares the keys and keeps classical values, "CollectiveV" the reverse).  As ckv_pool_load, with a shared
+ * width per side:
+ *   d_shared_k, d_shared_v : 0 = that side is not shared: it has no pool (its pool pointer is ignored and may be
+ *       NULL) and no indices, and the cache calls take its full head_dim-wide rows as the "user" array of that
+ *       side (user_K or user_V : [L][n_groups][head_dim]; idx_K or idx_V is ignored and may be NULL).
+ *       Otherwise 1..head_dim as for ckv_pool_load; when both are non-zero they must be equal.
+ *   The d_user argument of the cache calls is head_dim - max(d_shared_k, d_shared_v), the user-specific width
+ *   of the shared side(s) (head_dim if no side is shared, which is a classical KV cache).
+ * The blob of ckv_cache_export / ckv_cache_import then has an empty index section for a side that is not shared
+ * and head_dim elements per entry in that side's user section; ckv_cache_bytes counts what is stored.
+ * Decode runs on the CUDA-core and the warp-level tensor-core kernels (option "kernel" 0, 1 or 2; the
+ * warp-level kernel's TMA loader is not available).
+ * Errors: as ckv_pool_load; SHAPE also for unequal non-zero widths.
+ */
+CKV_API ckv_status ckv_pool_load_sides(ckv_ctx* ctx, const void* pool_K, const void* pool_V, int32_t n_entries,
+                                       int32_t d_shared_k, int32_t d_shared_v, void* stream);
+
+/*
  * Store one user's compressed cache (Sec. 4.2, prefill output: global K/V indices plus
  * user-specific K/V), replacing any earlier entry of `user` (whose storage is reused by later
  * puts, imports and appends).
@@ -145,6 +164,11 @@ CKV_API ckv_status ckv_cache_clear(ckv_ctx* ctx);
  *                    q_off[k] .. q_off[k+1]-1
  *   queries [any]  : [q_off[n]][n_groups][head_dim], ctx dtype
  *   out     [any]  : [q_off[n]][n_groups][head_dim], ctx out_dtype, caller-allocated
+ * With host memory for both `queries` and `out` and a few MB or more of queries, the request list
+ * is cut into four ranges of consecutive users whose upload, kernels and download run on streams
+ * of the library's own, so that the three overlap (pinned host memory is what makes the copies
+ * asynchronous); `stream` is ordered before the first and behind the last of them, and the
+ * results are the same bits.
  * A user with an empty history produces zero rows.  Results do not depend on how the
  * library splits long histories across thread blocks beyond fp32 rounding.  With kernel
  * families 1 to 3 (see option "kernel") they are bitwise reproducible from call to call for the
@@ -157,6 +181,21 @@ CKV_API ckv_status ckv_cache_clear(ckv_ctx* ctx);
  */
 CKV_API ckv_status ckv_attend(ckv_ctx* ctx, int32_t n, const int64_t* users, const int32_t* q_off,
                       const void* queries, void* out, void* stream);
+
+/*
+ * Decode with a visible length per query: self-attention over the cached sequence (Sec. 2.1: in self-attention
+ * models the s queries are projected from the sequence itself).  The paper does not restate the mask; this call
+ * takes, for every query row, the number of leading history positions it attends:
+ *   vis [any] : int32 [q_off[n]], row r of user k attends positions 0 .. vis[r]-1 of that user's history
+ *               (values are clamped to [0, L_k]; causal self-attention over the whole history is
+ *               vis = 1, 2, ..., L_k for the user's L_k queries; vis = 0 gives a zero row).
+ * CKV_SOFTMAX normalises over the attended positions; CKV_SILU_OVER_L sums over them and still divides by the
+ * user's history length L_k.  Everything else as ckv_attend; the CUDA-core and the warp-level tensor-core
+ * kernels serve this call (option "kernel" 0, 1 or 2).
+ * Errors: as ckv_attend; INVALID_ARG also for vis == NULL with queries present.
+ */
+CKV_API ckv_status ckv_attend_visible(ckv_ctx* ctx, int32_t n, const int64_t* users, const int32_t* q_off,
+                                      const int32_t* vis, const void* queries, void* out, void* stream);
 
 /*
  * Decode without any allocation.  (The paper has no counterpart: this is a deployment variant of
@@ -323,7 +362,7 @@ CKV_API ckv_status ckv_get_option(ckv_ctx* ctx, const char* name, int64_t* value
  * (loader the last warp-level tensor-core launch used: 1 or 2),
  * "workspace_bytes", "plan_cache_hit", "alloc_calls" (device or pinned-host allocations the call
  * made: 0 once its buffers have reached their size), "l2_window" (1 if the pool's L2 window was on
- * the stream for the call); "arena_capacity_units", "arena_used_units", "arena_free_runs" (state of
+ * the stream for the call), "pipeline_ranges" (ranges of users a host-buffer call was cut into: 1 or 4); "arena_capacity_units", "arena_used_units", "arena_free_runs" (state of
  * the compressed-cache storage, in (position, group) units); with option "time_kernels" also
  * "main_kernel_ns" and
  * "combine_kernel_ns" (device time of the attend kernel and of the split-merge kernel; the

@@ -25,7 +25,7 @@ EXPORTS = (
     "ckv_cache_evict", "ckv_cache_clear", "ckv_attend", "ckv_attend_static", "ckv_materialize",
     "ckv_user_length", "ckv_cache_append", "ckv_cache_blob_bytes", "ckv_cache_export", "ckv_cache_import",
     "ckv_cache_bytes", "ckv_set_option", "ckv_get_option", "ckv_last_stat", "ckv_strerror",
-    "ckv_last_cuda_error", "ckv_version", "ckv_route", "ckv_project",
+    "ckv_last_cuda_error", "ckv_version", "ckv_route", "ckv_project", "ckv_pool_load_sides", "ckv_attend_visible",
 )
 
 
@@ -54,6 +54,8 @@ def _load() -> ctypes.CDLL:
         "ckv_create": (i32, [ctypes.POINTER(ckv_config), ctypes.POINTER(vp)]),
         "ckv_destroy": (i32, [vp]),
         "ckv_pool_load": (i32, [vp, vp, vp, i32, i32, vp]),
+        "ckv_pool_load_sides": (i32, [vp, vp, vp, i32, i32, i32, vp]),
+        "ckv_attend_visible": (i32, [vp, i32, vp, vp, vp, vp, vp, vp]),
         "ckv_cache_put": (i32, [vp, i64, i32, vp, vp, vp, vp, i32, vp]),
         "ckv_cache_put_batch": (i32, [vp, i32, vp, vp, vp, vp, vp, vp, i32, vp]),
         "ckv_cache_append": (i32, [vp, i64, i32, vp, vp, vp, vp, i32, vp]),
@@ -142,6 +144,12 @@ def ckv_pool_load(ctx, pool_K, pool_V, n_entries: int, d_shared: int, stream=Non
            "ckv_pool_load")
 
 
+def ckv_pool_load_sides(ctx, pool_K, pool_V, n_entries: int, d_shared_k: int, d_shared_v: int, stream=None) -> None:
+    """ckv_pool_load with a shared width per side; 0 = that side is not shared (its pool may be None)."""
+    _check(ctx, lib.ckv_pool_load_sides(ctx, _ptr(pool_K), _ptr(pool_V), n_entries, d_shared_k, d_shared_v,
+                                        _stream(stream)), "ckv_pool_load_sides")
+
+
 def ckv_cache_put(ctx, user: int, L: int, idx_K, idx_V, user_K, user_V, d_user: int, stream=None) -> None:
     _check(ctx, lib.ckv_cache_put(ctx, int(user), int(L), _ptr(idx_K), _ptr(idx_V), _ptr(user_K),
                                   _ptr(user_V), d_user, _stream(stream)), "ckv_cache_put")
@@ -176,6 +184,17 @@ def ckv_attend(ctx, users, q_off, queries, out, stream=None) -> None:
         raise ValueError("q_off must have len(users) + 1 entries")
     _check(ctx, lib.ckv_attend(ctx, users.shape[0], users.ctypes.data, q_off.ctypes.data, _ptr(queries),
                                _ptr(out), _stream(stream)), "ckv_attend")
+
+
+def ckv_attend_visible(ctx, users, q_off, vis, queries, out, stream=None) -> None:
+    """ckv_attend with a visible length per query row: vis int32 [q_off[n]] (host array or device tensor)."""
+    users, q_off = _host_i64(users), _host_i32(q_off)
+    if q_off.shape[0] != users.shape[0] + 1:
+        raise ValueError("q_off must have len(users) + 1 entries")
+    if isinstance(vis, np.ndarray):
+        vis = _host_i32(vis)
+    _check(ctx, lib.ckv_attend_visible(ctx, users.shape[0], users.ctypes.data, q_off.ctypes.data, _ptr(vis),
+                                       _ptr(queries), _ptr(out), _stream(stream)), "ckv_attend_visible")
 
 
 def ckv_attend_static(ctx, users, q_off, queries, out, stream=None) -> None:

@@ -67,6 +67,12 @@ public:
         }
     }
     UserEntry* find(int64_t key) { return const_cast<UserEntry*>(static_cast<const UserTable*>(this)->find(key)); }
+    // a hint that `key` is about to be looked up (a request list names tens of thousands of users whose slots
+    // are scattered over a table larger than the host's caches)
+    void prefetch(int64_t key) const
+    {
+        if (n_) __builtin_prefetch(&slots_[hash(key) & mask_]);
+    }
     // the entry of `key`, created (zeroed) if absent; may throw std::bad_alloc
     UserEntry* insert(int64_t key)
     {
@@ -113,6 +119,8 @@ public:
     }
 };
 
+constexpr int kMaxRanges = 4;
+
 struct DevBuf {  // grow-only device buffer
     void* p = nullptr;
     size_t cap = 0;
@@ -127,6 +135,11 @@ struct Plan {
     std::vector<int32_t> q_off;
     uint64_t generation = 0;
     int64_t opt_split = 0, opt_kernel = 0;
+    bool with_vis = false;   // planned for a call with visible lengths (other kernel choice)
+    // The request list cut into n_ranges runs of consecutive users (host-buffer calls are pipelined range by
+    // range): items and the split list are grouped by range, r_item / r_split give each range's slice.
+    int32_t n_ranges = 1;
+    int32_t r_user[kMaxRanges + 1] = {}, r_item[kMaxRanges + 1] = {}, r_split[kMaxRanges + 1] = {};
     DevBuf dev;              // reqs | items | split list | works
     void* host = nullptr;    // pinned mirror the tables are built in
     size_t host_cap = 0;
@@ -166,13 +179,15 @@ struct ckv_ctx {
     int n_sms = 148;
     // pool
     int n_entries = 0, d_shared = 0, d_user = 0, idx_bytes = 0;
-    void* pool = nullptr;  // K rows then V rows, each [G][m][D]
+    bool full_k = false, full_v = false;  // the side is not shared: cached full width, no pool, no indices
+    void* pool = nullptr;  // K rows then V rows, each [G][m][D] (a side that is not shared has none)
     bool has_mma = false;         // the warp-level tensor-core family can run
     bool has_tma = false;         // ... and its TMA-gather loader too (tensor maps of the pool encoded)
     alignas(64) unsigned char tmaps[256] = {};  // two CUtensorMap: K pool, V pool
     bool has_umma = false;
     int* d_err = nullptr;  // OR of error codes from kernels whose bounded waits ran out
-    size_t pool_half = 0;  // bytes of one of them
+    size_t pool_half = 0;  // bytes of one side's rows
+    int n_pool_sides = 2;  // sides that have a pool
     // arena of compressed caches (units = (position, group) slots).  Units [0, used_units) are handed out;
     // runs inside that range given back by evicted, replaced or appended-to users wait in free_runs
     // (first unit -> length, neighbours merged) and are reused first-fit.
@@ -182,7 +197,7 @@ struct ckv_ctx {
     UserTable users;
     uint64_t generation = 1;
     // scratch
-    DevBuf stage_q, stage_out, partials;
+    DevBuf stage_q, stage_out, stage_vis, partials;
     int* d_flag = nullptr;
     Plan plans[kMaxPlans];
     uint64_t tick = 0;
@@ -190,6 +205,11 @@ struct ckv_ctx {
     int64_t opt_split = 0, opt_kernel = 0, opt_l2 = 1, opt_time = 0, opt_loader = 0;
     cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};  // around the main kernel and the combine
     bool ev_valid = false;
+    // host-buffer calls: one internal stream per range of users, so that the upload of one range, the kernels of
+    // another and the download of a third overlap; events tie them to the caller's stream at both ends
+    cudaStream_t pipe_stream[kMaxRanges] = {};
+    cudaEvent_t pipe_start = nullptr, pipe_plan = nullptr, pipe_h2d[kMaxRanges] = {}, pipe_done[kMaxRanges] = {};
+    bool pipe_ready = false;
     // L2 residency of the pool: an access-policy window over the pool allocation is put on the caller's
     // stream around the kernels of a decode call and taken off again before the call returns
     bool l2_ready = false;       // the persisting-L2 carve-out of this device was raised for this context
@@ -197,7 +217,7 @@ struct ckv_ctx {
     float l2_ratio = 1.f;
     // statistics of the last attend
     int64_t st_launches = 0, st_items = 0, st_split = 0, st_kernel = 0, st_ws = 0, st_hit = 0, st_loader = 0,
-            st_allocs = 0, st_l2 = 0;
+            st_allocs = 0, st_l2 = 0, st_ranges = 1;
     std::string cuda_err;
 
     ckv_status fail(cudaError_t e)
@@ -285,8 +305,8 @@ void drop_plans(ckv_ctx* ctx)
 CacheView view_of(const ckv_ctx* ctx)
 {
     CacheView v;
-    v.poolK = ctx->pool;
-    v.poolV = (const char*)ctx->pool + ctx->pool_half;
+    v.poolK = ctx->full_k ? nullptr : ctx->pool;
+    v.poolV = ctx->full_v ? nullptr : (const char*)ctx->pool + (ctx->full_k ? 0 : ctx->pool_half);
     v.idxK = ctx->a_idxK;
     v.idxV = ctx->a_idxV;
     v.userK = ctx->a_userK;
@@ -295,7 +315,20 @@ CacheView view_of(const ckv_ctx* ctx)
     v.n_entries = ctx->n_entries;
     v.d_user = ctx->d_user;
     v.idx_bytes = ctx->idx_bytes;
+    v.full_k = ctx->full_k;
+    v.full_v = ctx->full_v;
     return v;
+}
+
+// Bytes one unit takes in the four arena arrays: K indices, V indices, K user part, V user part.  A side that
+// is not shared keeps no index and the whole head_dim-wide row.
+void unit_bytes(const ckv_ctx* ctx, int64_t (&eb)[4])
+{
+    const int64_t D = ctx->cfg.head_dim;
+    eb[0] = ctx->full_k ? 0 : ctx->idx_bytes;
+    eb[1] = ctx->full_v ? 0 : ctx->idx_bytes;
+    eb[2] = (ctx->full_k ? D : ctx->d_user) * ctx->elem;
+    eb[3] = (ctx->full_v ? D : ctx->d_user) * ctx->elem;
 }
 
 // Capacity for units [0, need_end), keeping what is stored.
@@ -304,25 +337,25 @@ ckv_status ensure_arena(ckv_ctx* ctx, int64_t need_end, cudaStream_t s)
     if (need_end <= ctx->cap_units) return CKV_OK;
     int64_t cap = std::max<int64_t>(ctx->cap_units * 2, need_end);
     cap = (cap + 1023) / 1024 * 1024;
-    const size_t ub = (size_t)std::max(ctx->d_user, 1) * ctx->elem;
+    int64_t eb[4];
+    unit_bytes(ctx, eb);
     void* n[4] = {nullptr, nullptr, nullptr, nullptr};
-    const size_t bytes[4] = {(size_t)cap * ctx->idx_bytes, (size_t)cap * ctx->idx_bytes, (size_t)cap * ub,
-                             (size_t)cap * ub};
     void* old[4] = {ctx->a_idxK, ctx->a_idxV, ctx->a_userK, ctx->a_userV};
     for (int i = 0; i < 4; ++i) {
-        cudaError_t e = cudaMalloc(&n[i], bytes[i]);
+        if (eb[i] == 0) continue;  // nothing is stored there (no user part, or no indices on a side that is not shared)
+        cudaError_t e = cudaMalloc(&n[i], (size_t)cap * eb[i]);
         if (e != cudaSuccess) {
-            for (int j = 0; j < i; ++j) cudaFree(n[j]);
+            for (int j = 0; j < i; ++j)
+                if (n[j]) cudaFree(n[j]);
             return ctx->fail(e);
         }
     }
-    const size_t used[4] = {(size_t)ctx->used_units * ctx->idx_bytes, (size_t)ctx->used_units * ctx->idx_bytes,
-                            (size_t)ctx->used_units * ub, (size_t)ctx->used_units * ub};
     for (int i = 0; i < 4; ++i)
-        if (used[i]) {
-            cudaError_t e = cudaMemcpyAsync(n[i], old[i], used[i], cudaMemcpyDeviceToDevice, s);
+        if (eb[i] && ctx->used_units) {
+            cudaError_t e = cudaMemcpyAsync(n[i], old[i], (size_t)ctx->used_units * eb[i], cudaMemcpyDeviceToDevice, s);
             if (e != cudaSuccess) {
-                for (int j = 0; j < 4; ++j) cudaFree(n[j]);
+                for (int j = 0; j < 4; ++j)
+                    if (n[j]) cudaFree(n[j]);
                 return ctx->fail(e);
             }
         }
@@ -408,38 +441,40 @@ int64_t auto_split_len(const ckv_ctx* ctx, int64_t total_positions, int family, 
     return std::min<int64_t>(std::max<int64_t>(c, 256), 2048);
 }
 
-// Orders item indices by descending chunk length, equal lengths in their original order (two 16-bit
-// counting passes over the complemented length: linear in the number of items).
-void order_longest_first(const std::vector<Item>& items, std::vector<uint32_t>& order)
+// Orders the item indices [begin, end) by descending chunk length, equal lengths in their original order (two
+// 16-bit counting passes over the complemented length: linear in the number of items).
+void order_longest_first(const std::vector<Item>& items, size_t begin, size_t end, std::vector<uint32_t>& order,
+                         std::vector<uint32_t>& tmp, std::vector<uint32_t>& count)
 {
-    const size_t n = items.size();
-    order.resize(n);
+    const size_t n = end - begin;
     bool same = true;
-    for (size_t i = 0; i < n; ++i) {
+    for (size_t i = begin; i < end; ++i) {
         order[i] = (uint32_t)i;
-        same = same && items[i].len == items[0].len;
+        same = same && items[i].len == items[begin].len;
     }
     if (same || n < 2) return;
-    std::vector<uint32_t> tmp(n);
-    std::vector<uint32_t> count(65536 + 1);
+    tmp.resize(items.size());
+    count.resize(65536 + 1);
     for (int pass = 0; pass < 2; ++pass) {
         const int shift = 16 * pass;
         std::fill(count.begin(), count.end(), 0u);
-        for (size_t i = 0; i < n; ++i) ++count[((~(uint32_t)items[order[i]].len >> shift) & 0xffffu) + 1];
+        for (size_t i = begin; i < end; ++i) ++count[((~(uint32_t)items[order[i]].len >> shift) & 0xffffu) + 1];
         for (size_t d = 0; d < 65536; ++d) count[d + 1] += count[d];
-        for (size_t i = 0; i < n; ++i) tmp[count[(~(uint32_t)items[order[i]].len >> shift) & 0xffffu]++] = order[i];
-        order.swap(tmp);
+        for (size_t i = begin; i < end; ++i)
+            tmp[begin + count[(~(uint32_t)items[order[i]].len >> shift) & 0xffffu]++] = order[i];
+        std::copy(tmp.begin() + begin, tmp.begin() + end, order.begin() + begin);
     }
 }
 
-ckv_status build_plan(ckv_ctx* ctx, Plan& pl, int32_t n, const int64_t* users, const int32_t* q_off,
-                      cudaStream_t s)
+ckv_status build_plan(ckv_ctx* ctx, Plan& pl, int32_t n, const int64_t* users, const int32_t* q_off, bool with_vis,
+                      int n_ranges, const int32_t* r_user, cudaStream_t s)
 {
     std::vector<Req> reqs((size_t)n);
     int64_t total_pos = 0, n_active = 0;
     int32_t max_M = 0, max_L = 0;
     bool all_single = true;
     for (int32_t k = 0; k < n; ++k) {
+        if (k + 12 < n) ctx->users.prefetch(users[k + 12]);
         const UserEntry* f = ctx->users.find(users[k]);
         if (!f) return CKV_ERR_UNKNOWN_USER;
         Req& r = reqs[k];
@@ -462,11 +497,15 @@ ckv_status build_plan(ckv_ctx* ctx, Plan& pl, int32_t n, const int64_t* users, c
     pl.max_L = max_L;
     pl.n_req = n;
     const bool can_mma = ctx->has_mma;
+    // visible lengths and sides that are not shared are served by the CUDA-core and the warp-level tensor-core
+    // kernels only
+    const bool plain = !with_vis && !ctx->full_k && !ctx->full_v;
+    const bool can_umma = ctx->has_umma && plain;
     // tcgen05 from three 16-query blocks on, else the warp-level tensor-core kernel (faster than the CUDA-core
     // kernel from a single query on); the CUDA-core kernel serves what neither supports
     // One query per user: the pool-side factorisation trades the row gathers for two tables per (user, group) in
     // HBM (n_entries floats per request and group: not beyond 2 GiB of workspace).
-    const bool can_fact = all_single && n_active > 0 &&
+    const bool can_fact = plain && all_single && n_active > 0 &&
                           fact_max_history(ctx->cfg.dtype, ctx->cfg.head_dim, ctx->d_user, ctx->n_entries) >= max_L &&
                           (int64_t)n * ctx->cfg.n_groups * (fact_row_floats(ctx->n_entries) + fact_aux_floats()) *
                                   (int64_t)sizeof(float) <= ((int64_t)2 << 30);
@@ -486,11 +525,11 @@ ckv_status build_plan(ckv_ctx* ctx, Plan& pl, int32_t n, const int64_t* users, c
         fact_pays = t_fact < t_gather;
     }
     if (ctx->opt_kernel == 0)
-        pl.family = ctx->has_umma && max_M >= 48 ? 3 : fact_pays ? 4 : can_mma ? 2 : 1;
+        pl.family = can_umma && max_M >= 48 ? 3 : fact_pays ? 4 : can_mma ? 2 : 1;
     else if (ctx->opt_kernel == 4 && can_fact) pl.family = 4;
     else if (ctx->opt_kernel == 1) pl.family = 1;
     else if (ctx->opt_kernel == 2 && can_mma) pl.family = 2;
-    else if (ctx->opt_kernel == 3 && ctx->has_umma) pl.family = 3;
+    else if (ctx->opt_kernel == 3 && can_umma) pl.family = 3;
     else return CKV_ERR_UNSUPPORTED;
     const int64_t C = pl.family == 4         ? (int64_t)INT32_MAX  // one CTA holds a whole history
                       : ctx->opt_split > 0 ? ctx->opt_split
@@ -499,7 +538,16 @@ ckv_status build_plan(ckv_ctx* ctx, Plan& pl, int32_t n, const int64_t* users, c
     std::vector<int32_t> split;
     items.reserve((size_t)n);
     int64_t part_rows = 0;
-    for (int32_t k = 0; k < n; ++k) {
+    if (pl.family == 4) n_ranges = 1;  // its three launches work on all requests at once
+    pl.n_ranges = n_ranges;
+    for (int32_t k = 0, rg = 0; k <= n; ++k) {
+        while (rg <= n_ranges && (n_ranges == 1 ? (rg == 0 ? 0 : n) : r_user[rg]) == k) {
+            pl.r_user[rg] = k;
+            pl.r_item[rg] = (int32_t)items.size();
+            pl.r_split[rg] = (int32_t)split.size();
+            ++rg;
+        }
+        if (k == n) break;
         Req& r = reqs[k];
         if (r.M <= 0) continue;
         const int64_t nc = r.L == 0 ? 1 : (r.L + C - 1) / C;
@@ -517,9 +565,10 @@ ckv_status build_plan(ckv_ctx* ctx, Plan& pl, int32_t n, const int64_t* users, c
         }
         part_rows += nc * r.M;
     }
-    // longest chunks first: the tail of the grid is made of short ones
-    std::vector<uint32_t> order;
-    order_longest_first(items, order);
+    // longest chunks first (inside every range): the tail of a grid is made of short ones
+    std::vector<uint32_t> order(items.size()), tmp, count;
+    for (int rg = 0; rg < n_ranges; ++rg)
+        order_longest_first(items, (size_t)pl.r_item[rg], (size_t)pl.r_item[rg + 1], order, tmp, count);
     pl.n_items = (int32_t)items.size();
     pl.n_split = (int32_t)split.size();
     pl.split_items = 0;
@@ -565,19 +614,20 @@ ckv_status build_plan(ckv_ctx* ctx, Plan& pl, int32_t n, const int64_t* users, c
     pl.generation = ctx->generation;
     pl.opt_split = ctx->opt_split;
     pl.opt_kernel = ctx->opt_kernel;
+    pl.with_vis = with_vis;
     pl.live = true;
     return CKV_OK;
 }
 
-ckv_status get_plan(ckv_ctx* ctx, int32_t n, const int64_t* users, const int32_t* q_off, cudaStream_t s,
-                    Plan** out)
+ckv_status get_plan(ckv_ctx* ctx, int32_t n, const int64_t* users, const int32_t* q_off, bool with_vis,
+                    int n_ranges, const int32_t* r_user, cudaStream_t s, Plan** out)
 {
     ctx->tick++;
     Plan* victim = nullptr;
     for (auto& p : ctx->plans) {
         if (p.live && p.generation != ctx->generation) p.live = false;  // stale: the cache has changed since
-        if (p.live && p.opt_split == ctx->opt_split && p.opt_kernel == ctx->opt_kernel &&
-            (int32_t)p.users.size() == n &&
+        if (p.live && p.opt_split == ctx->opt_split && p.opt_kernel == ctx->opt_kernel && p.with_vis == with_vis &&
+            (p.n_ranges == n_ranges || (p.family == 4 && p.n_ranges == 1)) && (int32_t)p.users.size() == n &&
             std::memcmp(p.users.data(), users, sizeof(int64_t) * (size_t)n) == 0 &&
             std::memcmp(p.q_off.data(), q_off, sizeof(int32_t) * ((size_t)n + 1)) == 0) {
             p.last_use = ctx->tick;
@@ -593,7 +643,7 @@ ckv_status get_plan(ckv_ctx* ctx, int32_t n, const int64_t* users, const int32_t
     victim->live = false;
     ckv_status st;
     try {
-        st = build_plan(ctx, *victim, n, users, q_off, s);
+        st = build_plan(ctx, *victim, n, users, q_off, with_vis, n_ranges, r_user, s);
     } catch (const std::bad_alloc&) {
         st = CKV_ERR_OOM;
     }
@@ -625,7 +675,8 @@ void l2_prepare(ckv_ctx* ctx)
         cudaGetLastError();
         return;
     }
-    const size_t pool_bytes = 2 * ctx->pool_half;
+    const size_t pool_bytes = (size_t)ctx->n_pool_sides * ctx->pool_half;
+    if (pool_bytes == 0) return;
     const size_t want = std::min(pool_bytes, (size_t)max_persist);
     std::lock_guard<std::mutex> lock(g_l2_mu);
     size_t cur = 0;
@@ -749,48 +800,66 @@ ckv_status ckv_destroy(ckv_ctx* ctx)
     DeviceGuard dg(ctx->cfg.device);
     drop_plans(ctx);
     void* bufs[] = {ctx->pool,    ctx->a_idxK,     ctx->a_idxV,      ctx->a_userK,   ctx->a_userV,
-                    ctx->d_flag,  ctx->stage_q.p,  ctx->stage_out.p, ctx->partials.p};
+                    ctx->d_flag,  ctx->stage_q.p,  ctx->stage_out.p, ctx->partials.p, ctx->stage_vis.p};
     for (void* b : bufs)
         if (b) cudaFree(b);
     for (auto& e : ctx->ev)
         if (e) cudaEventDestroy(e);
+    for (int r = 0; r < kMaxRanges; ++r) {
+        if (ctx->pipe_stream[r]) cudaStreamDestroy(ctx->pipe_stream[r]);
+        if (ctx->pipe_h2d[r]) cudaEventDestroy(ctx->pipe_h2d[r]);
+        if (ctx->pipe_done[r]) cudaEventDestroy(ctx->pipe_done[r]);
+    }
+    if (ctx->pipe_start) cudaEventDestroy(ctx->pipe_start);
+    if (ctx->pipe_plan) cudaEventDestroy(ctx->pipe_plan);
     l2_release(ctx);
     cudaGetLastError();
     delete ctx;
     return CKV_OK;
 }
 
-ckv_status ckv_pool_load(ckv_ctx* ctx, const void* pool_K, const void* pool_V, int32_t n_entries,
-                         int32_t d_shared, void* stream)
+ckv_status ckv_pool_load_sides(ckv_ctx* ctx, const void* pool_K, const void* pool_V, int32_t n_entries,
+                               int32_t d_shared_k, int32_t d_shared_v, void* stream)
 {
-    if (!ctx || !pool_K || !pool_V || n_entries < 1) return CKV_ERR_INVALID_ARG;
+    if (!ctx || n_entries < 1) return CKV_ERR_INVALID_ARG;
     const int D = ctx->cfg.head_dim, G = ctx->cfg.n_groups;
-    if (d_shared < 1 || d_shared > D) return CKV_ERR_SHAPE;
-    if (!ctx->users.empty() && (n_entries != ctx->n_entries || d_shared != ctx->d_shared)) return CKV_ERR_SHAPE;
+    if (d_shared_k < 0 || d_shared_k > D || d_shared_v < 0 || d_shared_v > D) return CKV_ERR_SHAPE;
+    if (d_shared_k > 0 && d_shared_v > 0 && d_shared_k != d_shared_v) return CKV_ERR_SHAPE;
+    const bool full_k = d_shared_k == 0, full_v = d_shared_v == 0;
+    if ((!full_k && !pool_K) || (!full_v && !pool_V)) return CKV_ERR_INVALID_ARG;
+    const int d_shared = std::max(d_shared_k, d_shared_v);  // of the shared side(s); 0: no side is shared
+    if (!ctx->users.empty() && (n_entries != ctx->n_entries || d_shared != ctx->d_shared || full_k != ctx->full_k ||
+                                full_v != ctx->full_v))
+        return CKV_ERR_SHAPE;
     DeviceGuard dg(ctx->cfg.device);
     cudaStream_t s = (cudaStream_t)stream;
     const size_t half = (size_t)G * n_entries * D * ctx->elem;
     const size_t src_bytes = (size_t)G * n_entries * d_shared * ctx->elem;
+    const int n_sides = (full_k ? 0 : 1) + (full_v ? 0 : 1);
     Staged sk, sv;
-    CK(sk.init(pool_K, src_bytes, s));
-    CK(sv.init(pool_V, src_bytes, s));
-    if (!ctx->pool || half != ctx->pool_half) {
+    if (!full_k) CK(sk.init(pool_K, src_bytes, s));
+    if (!full_v) CK(sv.init(pool_V, src_bytes, s));
+    const bool layout_changes = ctx->n_entries != n_entries || ctx->d_shared != d_shared || ctx->full_k != full_k ||
+                                ctx->full_v != full_v || !ctx->pool;
+    if (layout_changes || half != ctx->pool_half) {
         void* np = nullptr;
-        CK(cudaMalloc(&np, 2 * half));
+        CK(cudaMalloc(&np, std::max<size_t>((size_t)n_sides * half, 256)));
         if (ctx->pool) cudaFree(ctx->pool);
         ctx->pool = np;
         ctx->pool_half = half;
     }
-    ctx->has_mma = mma_supported(ctx->cfg.dtype, D, D - d_shared);
-    ctx->has_tma = ctx->has_mma && make_pool_tensor_maps(D, (int64_t)G * n_entries, ctx->pool,
-                                                         (const char*)ctx->pool + half, ctx->tmaps);
-    ctx->has_umma = umma_supported(ctx->cfg.dtype, D, D - d_shared, n_entries <= 65536 ? 2 : 4);
-    CK(launch_pool_layout(ctx->cfg.dtype, G, n_entries, d_shared, D, sk.dev, ctx->pool, s));
-    CK(launch_pool_layout(ctx->cfg.dtype, G, n_entries, d_shared, D, sv.dev, (char*)ctx->pool + half, s));
+    void* dst_k = ctx->pool;
+    void* dst_v = (char*)ctx->pool + (full_k ? 0 : half);
+    const int du = D - d_shared;  // user-specific width of the shared side(s)
+    ctx->has_mma = mma_supported(ctx->cfg.dtype, D, n_sides ? du : 0);
+    ctx->has_tma = ctx->has_mma && n_sides == 2 &&
+                   make_pool_tensor_maps(D, (int64_t)G * n_entries, dst_k, dst_v, ctx->tmaps);
+    ctx->has_umma = umma_supported(ctx->cfg.dtype, D, n_sides ? du : 0, n_entries <= 65536 ? 2 : 4);
+    if (!full_k) CK(launch_pool_layout(ctx->cfg.dtype, G, n_entries, d_shared, D, sk.dev, dst_k, s));
+    if (!full_v) CK(launch_pool_layout(ctx->cfg.dtype, G, n_entries, d_shared, D, sv.dev, dst_v, s));
     if (sk.owned || sv.owned) CK(cudaStreamSynchronize(s));
-    l2_prepare(ctx);
-    if (ctx->users.empty() && (ctx->n_entries != n_entries || ctx->d_shared != d_shared)) {
-        // index width or user width may change: restart the (empty) arena
+    if (ctx->users.empty() && layout_changes) {
+        // index width or the sides' widths may change: restart the (empty) arena
         void* old[4] = {ctx->a_idxK, ctx->a_idxV, ctx->a_userK, ctx->a_userV};
         for (void* b : old)
             if (b) cudaFree(b);
@@ -801,8 +870,20 @@ ckv_status ckv_pool_load(ckv_ctx* ctx, const void* pool_K, const void* pool_V, i
     ctx->n_entries = n_entries;
     ctx->d_shared = d_shared;
     ctx->d_user = D - d_shared;
+    ctx->full_k = full_k;
+    ctx->full_v = full_v;
     ctx->idx_bytes = n_entries <= 65536 ? 2 : 4;
+    ctx->n_pool_sides = n_sides;
+    l2_prepare(ctx);
     return CKV_OK;
+}
+
+ckv_status ckv_pool_load(ckv_ctx* ctx, const void* pool_K, const void* pool_V, int32_t n_entries,
+                         int32_t d_shared, void* stream)
+{
+    if (!ctx || !pool_K || !pool_V || n_entries < 1) return CKV_ERR_INVALID_ARG;
+    if (d_shared < 1 || d_shared > ctx->cfg.head_dim) return CKV_ERR_SHAPE;
+    return ckv_pool_load_sides(ctx, pool_K, pool_V, n_entries, d_shared, d_shared, stream);
 }
 
 ckv_status ckv_cache_put_batch(ckv_ctx* ctx, int32_t n, const int64_t* users, const int64_t* hist_off,
@@ -823,7 +904,10 @@ ckv_status ckv_cache_put_batch(ckv_ctx* ctx, int32_t n, const int64_t* users, co
         unit_off[k + 1] = unit_off[k] + (int64_t)G * ((L + 31) / 32 * 32);
     }
     const int64_t P = hist_off[n], total_units = unit_off[n];
-    if (P > 0 && (!idx_K || !idx_V || (d_user > 0 && (!user_K || !user_V)))) return CKV_ERR_INVALID_ARG;
+    int64_t eb[4];
+    unit_bytes(ctx, eb);
+    if (P > 0 && ((eb[0] && !idx_K) || (eb[1] && !idx_V) || (eb[2] && !user_K) || (eb[3] && !user_V)))
+        return CKV_ERR_INVALID_ARG;
 
     DeviceGuard dg(ctx->cfg.device);
     cudaStream_t s = (cudaStream_t)stream;
@@ -835,21 +919,22 @@ ckv_status ckv_cache_put_batch(ckv_ctx* ctx, int32_t n, const int64_t* users, co
     int64_t base = 0;
     if (total_units > 0) {
         Staged sik, siv, suk, suv, sho, suo;
-        const size_t ib = (size_t)P * G * sizeof(int32_t), ubytes = (size_t)P * G * d_user * ctx->elem;
-        CK(sik.init(idx_K, ib, s));
-        if (idx_V == idx_K) siv.dev = sik.dev; else CK(siv.init(idx_V, ib, s));
-        CK(suk.init(user_K, ubytes, s));
-        CK(suv.init(user_V, ubytes, s));
+        const size_t ib = (size_t)P * G * sizeof(int32_t);
+        if (eb[0]) CK(sik.init(idx_K, ib, s));
+        if (eb[1]) {
+            if (idx_V == idx_K && eb[0]) siv.dev = sik.dev; else CK(siv.init(idx_V, ib, s));
+        }
+        CK(suk.init(user_K, (size_t)P * G * eb[2], s));
+        CK(suv.init(user_V, (size_t)P * G * eb[3], s));
         CK(sho.init(hist_off, sizeof(int64_t) * ((size_t)n + 1), s));
         CK(suo.init(unit_off.data(), sizeof(int64_t) * ((size_t)n + 1), s));
         ckv_status st = arena_take(ctx, total_units, s, &base);
         if (st != CKV_OK) return st;
         cudaError_t e = cudaMemsetAsync(ctx->d_flag, 0, sizeof(int), s);
         if (e == cudaSuccess)
-            e = launch_pack(ctx->cfg.dtype, G, ctx->n_entries, d_user, ctx->idx_bytes, n, (const int64_t*)sho.dev,
+            e = launch_pack(ctx->cfg.dtype, G, ctx->n_entries, ctx->idx_bytes, n, (const int64_t*)sho.dev,
                             (const int64_t*)suo.dev, total_units, base, (const int32_t*)sik.dev,
-                            (const int32_t*)siv.dev, suk.dev, suv.dev, ctx->a_idxK, ctx->a_idxV, ctx->a_userK,
-                            ctx->a_userV, ctx->d_flag, s);
+                            (const int32_t*)siv.dev, suk.dev, suv.dev, view_of(ctx), ctx->cfg.head_dim, ctx->d_flag, s);
         int bad = 0;
         if (e == cudaSuccess) e = cudaMemcpyAsync(&bad, ctx->d_flag, sizeof(int), cudaMemcpyDeviceToHost, s);
         if (e == cudaSuccess) e = cudaStreamSynchronize(s);
@@ -886,7 +971,9 @@ ckv_status ckv_cache_append(ckv_ctx* ctx, int64_t user, int32_t L_new, const int
     UserEntry* f = ctx->users.find(user);
     if (!f) return CKV_ERR_UNKNOWN_USER;
     if (L_new == 0) return CKV_OK;
-    if (!idx_K || !idx_V || (d_user > 0 && (!user_K || !user_V))) return CKV_ERR_INVALID_ARG;
+    int64_t eb[4];
+    unit_bytes(ctx, eb);
+    if ((eb[0] && !idx_K) || (eb[1] && !idx_V) || (eb[2] && !user_K) || (eb[3] && !user_V)) return CKV_ERR_INVALID_ARG;
     const UserEntry old = *f;
     if ((int64_t)old.L + L_new > INT32_MAX - 32) return CKV_ERR_INVALID_ARG;
     const int G = ctx->cfg.n_groups;
@@ -895,11 +982,13 @@ ckv_status ckv_cache_append(ckv_ctx* ctx, int64_t user, int32_t L_new, const int
     DeviceGuard dg(ctx->cfg.device);
     cudaStream_t s = (cudaStream_t)stream;
     Staged sik, siv, suk, suv;
-    const size_t ib = (size_t)L_new * G * sizeof(int32_t), ubytes = (size_t)L_new * G * d_user * ctx->elem;
-    CK(sik.init(idx_K, ib, s));
-    if (idx_V == idx_K) siv.dev = sik.dev; else CK(siv.init(idx_V, ib, s));
-    CK(suk.init(user_K, ubytes, s));
-    CK(suv.init(user_V, ubytes, s));
+    const size_t ib = (size_t)L_new * G * sizeof(int32_t);
+    if (eb[0]) CK(sik.init(idx_K, ib, s));
+    if (eb[1]) {
+        if (idx_V == idx_K && eb[0]) siv.dev = sik.dev; else CK(siv.init(idx_V, ib, s));
+    }
+    CK(suk.init(user_K, (size_t)L_new * G * eb[2], s));
+    CK(suv.init(user_V, (size_t)L_new * G * eb[3], s));
     // the longer history is written to a run of its own (the old units are read while it is written) and the
     // old run is given back afterwards
     int64_t base = 0;
@@ -907,9 +996,9 @@ ckv_status ckv_cache_append(ckv_ctx* ctx, int64_t user, int32_t L_new, const int
     if (st != CKV_OK) return st;
     cudaError_t e = cudaMemsetAsync(ctx->d_flag, 0, sizeof(int), s);
     if (e == cudaSuccess)
-        e = launch_append(ctx->cfg.dtype, G, ctx->n_entries, d_user, ctx->idx_bytes, old.base, old.L, old.Lpad, base,
+        e = launch_append(ctx->cfg.dtype, G, ctx->n_entries, ctx->idx_bytes, old.base, old.L, old.Lpad, base,
                           L_new, Lpad_tot, (const int32_t*)sik.dev, (const int32_t*)siv.dev, suk.dev, suv.dev,
-                          ctx->a_idxK, ctx->a_idxV, ctx->a_userK, ctx->a_userV, ctx->d_flag, s);
+                          view_of(ctx), ctx->cfg.head_dim, ctx->d_flag, s);
     int bad = 0;
     if (e == cudaSuccess) e = cudaMemcpyAsync(&bad, ctx->d_flag, sizeof(int), cudaMemcpyDeviceToHost, s);
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);
@@ -929,11 +1018,10 @@ namespace {
 // Section offsets of a blob holding `total_units` units: K indices, V indices, user K, user V, end.
 void blob_sections(const ckv_ctx* ctx, int64_t total_units, int64_t (&off)[5])
 {
-    const int64_t ub = (int64_t)ctx->d_user * ctx->elem;
-    const int64_t sz[4] = {total_units * ctx->idx_bytes, total_units * ctx->idx_bytes, total_units * ub,
-                           total_units * ub};
+    int64_t eb[4];
+    unit_bytes(ctx, eb);
     off[0] = 0;
-    for (int i = 0; i < 4; ++i) off[i + 1] = (off[i] + sz[i] + 255) / 256 * 256;
+    for (int i = 0; i < 4; ++i) off[i + 1] = (off[i] + total_units * eb[i] + 255) / 256 * 256;
 }
 
 int64_t units_of(const ckv_ctx* ctx, int64_t L) { return (int64_t)ctx->cfg.n_groups * ((L + 31) / 32 * 32); }
@@ -970,8 +1058,8 @@ ckv_status ckv_cache_export(ckv_ctx* ctx, int32_t n, const int64_t* users, void*
     if (bytes != off[4]) return CKV_ERR_INVALID_ARG;
     DeviceGuard dg(ctx->cfg.device);
     cudaStream_t s = (cudaStream_t)stream;
-    const int64_t ub = (int64_t)ctx->d_user * ctx->elem;  // no user sections without a user part
-    const int64_t eb[4] = {ctx->idx_bytes, ctx->idx_bytes, ub, ub};
+    int64_t eb[4];  // a section is empty where nothing is stored (no user part; no indices of a side that is not shared)
+    unit_bytes(ctx, eb);
     const char* src[4] = {(const char*)ctx->a_idxK, (const char*)ctx->a_idxV, (const char*)ctx->a_userK,
                           (const char*)ctx->a_userV};
     int64_t done = 0;
@@ -1014,8 +1102,8 @@ ckv_status ckv_cache_import(ckv_ctx* ctx, int32_t n, const int64_t* users, const
     if (total > 0) {
         ckv_status st = arena_take(ctx, total, s, &base);
         if (st != CKV_OK) return st;
-        const int64_t ub = (int64_t)ctx->d_user * ctx->elem;
-        const int64_t eb[4] = {ctx->idx_bytes, ctx->idx_bytes, ub, ub};
+        int64_t eb[4];
+        unit_bytes(ctx, eb);
         char* dst[4] = {(char*)ctx->a_idxK, (char*)ctx->a_idxV, (char*)ctx->a_userK, (char*)ctx->a_userV};
         // the batch takes one run of contiguous units: one copy per section
         cudaError_t e = cudaSuccess;
@@ -1025,8 +1113,8 @@ ckv_status ckv_cache_import(ckv_ctx* ctx, int32_t n, const int64_t* users, const
                                     cudaMemcpyDefault, s);
         if (e == cudaSuccess) e = cudaMemsetAsync(ctx->d_flag, 0, sizeof(int), s);
         if (e == cudaSuccess)
-            e = launch_check_indices(ctx->idx_bytes, ctx->n_entries, dst[0] + base * eb[0], dst[1] + base * eb[1],
-                                     total, ctx->d_flag, s);
+            e = launch_check_indices(ctx->idx_bytes, ctx->n_entries, eb[0] ? dst[0] + base * eb[0] : nullptr,
+                                     eb[1] ? dst[1] + base * eb[1] : nullptr, total, ctx->d_flag, s);
         int bad = 0;
         if (e == cudaSuccess) e = cudaMemcpyAsync(&bad, ctx->d_flag, sizeof(int), cudaMemcpyDeviceToHost, s);
         if (e == cudaSuccess) e = cudaStreamSynchronize(s);
@@ -1078,7 +1166,8 @@ namespace {
 ckv_status run_mma(ckv_ctx* ctx, int D, int max_M, const AttendArgs& a, cudaStream_t s)
 {
     const int loader = ctx->opt_loader == 2 ? 2 : 1;
-    if (loader == 2 && !ctx->has_tma) return CKV_ERR_UNSUPPORTED;
+    // the TMA loader serves the plain form only (both sides shared, no visible lengths)
+    if (loader == 2 && (!ctx->has_tma || a.cv.full_k || a.cv.full_v || a.vis)) return CKV_ERR_UNSUPPORTED;
     ctx->st_loader = loader;
     CK(launch_attend_mma(D, max_M, a, loader == 2 ? ctx->tmaps : nullptr, ctx->d_err, s));
     return CKV_OK;
@@ -1086,69 +1175,38 @@ ckv_status run_mma(ckv_ctx* ctx, int D, int max_M, const AttendArgs& a, cudaStre
 
 }  // namespace
 
-ckv_status ckv_attend(ckv_ctx* ctx, int32_t n, const int64_t* users, const int32_t* q_off,
-                      const void* queries, void* out, void* stream)
+}  // extern "C"
+
+namespace {
+
+constexpr size_t kPipeMinBytes = size_t(4) << 20;  // host query buffers below this are not worth pipelining
+
+cudaError_t pipe_prepare(ckv_ctx* ctx)
 {
-    if (!ctx || n < 0 || (n > 0 && (!users || !q_off))) return CKV_ERR_INVALID_ARG;
-    if (!ctx->pool) return CKV_ERR_STATE;
-    if (n == 0) return CKV_OK;
-    if (!offsets_ok32(q_off, n)) return CKV_ERR_INVALID_ARG;
-    const int64_t Q = q_off[n];
-    if (Q > 0 && (!queries || !out)) return CKV_ERR_INVALID_ARG;
-    DeviceGuard dg(ctx->cfg.device);
-    cudaStream_t s = (cudaStream_t)stream;
-    ctx->st_launches = 0;
-    ctx->st_allocs = 0;
-    Plan* pl = nullptr;
-    ckv_status st = get_plan(ctx, n, users, q_off, s, &pl);
-    if (st != CKV_OK) return st;
-    ctx->st_items = pl->n_items;
-    ctx->st_split = pl->split_items;
-    ctx->st_kernel = pl->family;
-    if (Q == 0) return CKV_OK;
+    if (ctx->pipe_ready) return cudaSuccess;
+    cudaError_t e = cudaSuccess;
+    for (int r = 0; r < kMaxRanges && e == cudaSuccess; ++r) {
+        if (!ctx->pipe_stream[r]) e = cudaStreamCreateWithFlags(&ctx->pipe_stream[r], cudaStreamNonBlocking);
+        if (e == cudaSuccess && !ctx->pipe_h2d[r]) e = cudaEventCreateWithFlags(&ctx->pipe_h2d[r], cudaEventDisableTiming);
+        if (e == cudaSuccess && !ctx->pipe_done[r]) e = cudaEventCreateWithFlags(&ctx->pipe_done[r], cudaEventDisableTiming);
+    }
+    if (e == cudaSuccess && !ctx->pipe_start) e = cudaEventCreateWithFlags(&ctx->pipe_start, cudaEventDisableTiming);
+    if (e == cudaSuccess && !ctx->pipe_plan) e = cudaEventCreateWithFlags(&ctx->pipe_plan, cudaEventDisableTiming);
+    ctx->pipe_ready = e == cudaSuccess;
+    return e;
+}
 
+// The kernels of one slice of a plan (items [i0, i1), split requests [s0, s1)) on stream s.
+ckv_status launch_slice(ckv_ctx* ctx, const Plan* pl, AttendArgs a, int i0, int i1, int s0, int s1, bool time_it,
+                        cudaStream_t s)
+{
     const int D = ctx->cfg.head_dim, G = ctx->cfg.n_groups;
-    const size_t q_bytes = (size_t)Q * G * D * ctx->elem;
-    const size_t o_bytes = (size_t)Q * G * D * (ctx->cfg.out_dtype == CKV_BF16 ? 2 : 4);
-    const void* d_q = queries;
-    void* d_out = out;
-    const bool q_host = !is_device_ptr(queries), o_host = !is_device_ptr(out);
-    if (q_host) {
-        CK(grow(ctx->stage_q, q_bytes, &ctx->st_allocs));
-        CK(cudaMemcpyAsync(ctx->stage_q.p, queries, q_bytes, cudaMemcpyHostToDevice, s));
-        d_q = ctx->stage_q.p;
-    }
-    if (o_host) {
-        CK(grow(ctx->stage_out, o_bytes, &ctx->st_allocs));
-        d_out = ctx->stage_out.p;
-    }
-    // split-reduction partials, or the factorisation's tables (per request and group: n_entries + a few floats)
-    const size_t ws = pl->family == 4
-                          ? (size_t)pl->n_req * G * ((size_t)fact_row_floats(ctx->n_entries) + fact_aux_floats()) * sizeof(float)
-                          : (size_t)pl->part_rows * G * (D + 2) * sizeof(float);
-    if (ws) CK(grow(ctx->partials, ws, &ctx->st_allocs));
-    ctx->st_ws = (int64_t)ws;
+    a.items = pl->d_items + i0;
+    a.works = pl->d_works ? pl->d_works + i0 : nullptr;
+    a.n_items = i1 - i0;
     L2Window l2(ctx, s);
-
-    AttendArgs a;
-    a.cv = view_of(ctx);
-    a.reqs = pl->d_reqs;
-    a.items = pl->d_items;
-    a.works = pl->d_works;
-    a.n_items = pl->n_items;
-    a.queries = d_q;
-    a.out = d_out;
-    a.partials = (float*)ctx->partials.p;
-    a.out_dtype = ctx->cfg.out_dtype;
-    a.mode = ctx->cfg.mode;
-    a.scale = ctx->scale;
-    ctx->ev_valid = false;
-    if (ctx->opt_time) {
-        for (auto& e : ctx->ev)
-            if (!e) CK(cudaEventCreate(&e));
-        CK(cudaEventRecord(ctx->ev[0], s));
-    }
-    if (pl->n_items > 0) {
+    if (time_it) CK(cudaEventRecord(ctx->ev[0], s));
+    if (a.n_items > 0) {
         if (pl->family == 4) {
             float* tw = (float*)ctx->partials.p;
             CK(launch_attend_fact(D, a, pl->n_req, pl->max_L, ctx->n_sms, tw,
@@ -1163,17 +1221,185 @@ ckv_status ckv_attend(ckv_ctx* ctx, int32_t n, const int64_t* users, const int32
             CK(launch_attend_simt(ctx->cfg.dtype, D, pl->max_M, a, s));
         ctx->st_launches++;
     }
-    if (ctx->opt_time) CK(cudaEventRecord(ctx->ev[1], s));
-    if (pl->n_split > 0) {
-        CK(launch_combine(D, a, pl->d_split, pl->n_split, s));
+    if (time_it) CK(cudaEventRecord(ctx->ev[1], s));
+    if (s1 > s0) {
+        CK(launch_combine(D, a, pl->d_split + s0, s1 - s0, s));
         ctx->st_launches++;
     }
-    if (ctx->opt_time) {
-        CK(cudaEventRecord(ctx->ev[2], s));
-        ctx->ev_valid = true;
-    }
-    if (o_host) CK(cudaMemcpyAsync(out, d_out, o_bytes, cudaMemcpyDeviceToHost, s));
+    if (time_it) CK(cudaEventRecord(ctx->ev[2], s));
     return CKV_OK;
+}
+
+// ckv_attend (vis null) and ckv_attend_visible
+ckv_status attend_impl(ckv_ctx* ctx, int32_t n, const int64_t* users, const int32_t* q_off, const int32_t* vis,
+                       const void* queries, void* out, void* stream)
+{
+    if (!ctx || n < 0 || (n > 0 && (!users || !q_off))) return CKV_ERR_INVALID_ARG;
+    if (!ctx->pool) return CKV_ERR_STATE;
+    if (n == 0) return CKV_OK;
+    if (!offsets_ok32(q_off, n)) return CKV_ERR_INVALID_ARG;
+    const int64_t Q = q_off[n];
+    if (Q > 0 && (!queries || !out)) return CKV_ERR_INVALID_ARG;
+    DeviceGuard dg(ctx->cfg.device);
+    cudaStream_t s = (cudaStream_t)stream;
+    ctx->st_launches = 0;
+    ctx->st_allocs = 0;
+    ctx->st_ranges = 1;
+    const int D = ctx->cfg.head_dim, G = ctx->cfg.n_groups;
+    const size_t q_row = (size_t)G * D * ctx->elem, o_row = (size_t)G * D * (ctx->cfg.out_dtype == CKV_BF16 ? 2 : 4);
+    const size_t q_bytes = (size_t)Q * q_row, o_bytes = (size_t)Q * o_row;
+    const bool q_host = Q > 0 && !is_device_ptr(queries), o_host = Q > 0 && !is_device_ptr(out);
+
+    // Host buffers on both sides and enough of them: the request list is cut into ranges of consecutive users
+    // with about equal numbers of query rows, and every range gets a stream of its own for its upload, its
+    // kernels and its download.  The uploads are enqueued before the plan is looked up or built, so that host
+    // work overlaps them too.
+    int n_ranges = 1;
+    int32_t r_user[kMaxRanges + 1] = {0, n, n, n, n};
+    if (q_host && o_host && q_bytes >= kPipeMinBytes && n >= 2 * kMaxRanges && pipe_prepare(ctx) == cudaSuccess) {
+        n_ranges = kMaxRanges;
+        int32_t k = 0;
+        for (int r = 1; r < n_ranges; ++r) {
+            const int64_t want = Q * r / n_ranges;
+            while (k < n && q_off[k] < want) ++k;
+            r_user[r] = k;
+        }
+        r_user[n_ranges] = n;
+    }
+    const void* d_q = queries;
+    void* d_out = out;
+    if (q_host) {
+        CK(grow(ctx->stage_q, q_bytes, &ctx->st_allocs));
+        d_q = ctx->stage_q.p;
+    }
+    if (o_host) {
+        CK(grow(ctx->stage_out, o_bytes, &ctx->st_allocs));
+        d_out = ctx->stage_out.p;
+    }
+    const int32_t* d_vis = vis;
+    if (vis && Q > 0 && !is_device_ptr(vis)) {
+        CK(grow(ctx->stage_vis, (size_t)Q * sizeof(int32_t), &ctx->st_allocs));
+        CK(cudaMemcpyAsync(ctx->stage_vis.p, vis, (size_t)Q * sizeof(int32_t), cudaMemcpyHostToDevice, s));
+        d_vis = (const int32_t*)ctx->stage_vis.p;
+    }
+    // The first range's upload goes out before the plan is looked up or built, so that the host work overlaps
+    // it; the other ranges follow the plan's own (small) upload, which would otherwise queue behind all of them
+    // on the copy engine and hold back the first kernels.
+    auto upload_range = [&](int r) -> cudaError_t {
+        cudaStream_t ps = ctx->pipe_stream[r];
+        cudaError_t e = cudaStreamWaitEvent(ps, ctx->pipe_start, 0);
+        const size_t r0 = (size_t)q_off[r_user[r]], r1 = (size_t)q_off[r_user[r + 1]];
+        if (e == cudaSuccess && r1 > r0)
+            e = cudaMemcpyAsync((char*)ctx->stage_q.p + r0 * q_row, (const char*)queries + r0 * q_row, (r1 - r0) * q_row,
+                                cudaMemcpyHostToDevice, ps);
+        if (e == cudaSuccess) e = cudaEventRecord(ctx->pipe_h2d[r], ps);
+        return e;
+    };
+    if (n_ranges > 1) {
+        CK(cudaEventRecord(ctx->pipe_start, s));
+        CK(upload_range(0));
+    } else if (q_host) {
+        CK(cudaMemcpyAsync(ctx->stage_q.p, queries, q_bytes, cudaMemcpyHostToDevice, s));
+    }
+
+    Plan* pl = nullptr;
+    ckv_status st = get_plan(ctx, n, users, q_off, vis != nullptr, n_ranges, r_user, s, &pl);
+    if (st != CKV_OK) {
+        if (n_ranges > 1) cudaStreamWaitEvent(s, ctx->pipe_h2d[0], 0);  // the upload already enqueued stays inside the call
+        return st;
+    }
+    if (n_ranges > 1) {
+        CK(cudaEventRecord(ctx->pipe_plan, s));
+        for (int r = 1; r < n_ranges; ++r) CK(upload_range(r));
+    }
+    ctx->st_items = pl->n_items;
+    ctx->st_split = pl->split_items;
+    ctx->st_kernel = pl->family;
+    if (Q == 0) return CKV_OK;
+
+    // split-reduction partials, or the factorisation's tables (per request and group: n_entries + a few floats)
+    const size_t ws = pl->family == 4
+                          ? (size_t)pl->n_req * G * ((size_t)fact_row_floats(ctx->n_entries) + fact_aux_floats()) * sizeof(float)
+                          : (size_t)pl->part_rows * G * (D + 2) * sizeof(float);
+    if (ws) CK(grow(ctx->partials, ws, &ctx->st_allocs));
+    ctx->st_ws = (int64_t)ws;
+
+    AttendArgs a;
+    a.cv = view_of(ctx);
+    a.reqs = pl->d_reqs;
+    a.items = pl->d_items;
+    a.works = pl->d_works;
+    a.n_items = pl->n_items;
+    a.queries = d_q;
+    a.vis = d_vis;
+    a.out = d_out;
+    a.partials = (float*)ctx->partials.p;
+    a.out_dtype = ctx->cfg.out_dtype;
+    a.mode = ctx->cfg.mode;
+    a.scale = ctx->scale;
+    ctx->ev_valid = false;
+
+    if (n_ranges == 1) {
+        const bool time_it = ctx->opt_time != 0;
+        if (time_it)
+            for (auto& e : ctx->ev)
+                if (!e) CK(cudaEventCreate(&e));
+        st = launch_slice(ctx, pl, a, 0, pl->n_items, 0, pl->n_split, time_it, s);
+        if (st != CKV_OK) return st;
+        ctx->ev_valid = time_it;
+        if (o_host) CK(cudaMemcpyAsync(out, d_out, o_bytes, cudaMemcpyDeviceToHost, s));
+        return CKV_OK;
+    }
+
+    // pipelined: the plan's tables (uploaded on the caller's stream if the plan is new) come first on every stream
+    ctx->st_ranges = n_ranges;
+    ckv_status result = CKV_OK;
+    if (pl->n_ranges == 1) {
+        // a plan that is not cut into ranges (pool-side factorisation): one pass on the first stream behind all uploads
+        cudaStream_t ps = ctx->pipe_stream[0];
+        CK(cudaStreamWaitEvent(ps, ctx->pipe_plan, 0));
+        for (int r = 1; r < n_ranges; ++r) CK(cudaStreamWaitEvent(ps, ctx->pipe_h2d[r], 0));
+        result = launch_slice(ctx, pl, a, 0, pl->n_items, 0, pl->n_split, false, ps);
+        if (result == CKV_OK) {
+            cudaError_t e = cudaMemcpyAsync(out, d_out, o_bytes, cudaMemcpyDeviceToHost, ps);
+            if (e != cudaSuccess) result = ctx->fail(e);
+        }
+    } else {
+        for (int r = 0; r < n_ranges && result == CKV_OK; ++r) {
+            cudaStream_t ps = ctx->pipe_stream[r];
+            CK(cudaStreamWaitEvent(ps, ctx->pipe_plan, 0));
+            result = launch_slice(ctx, pl, a, pl->r_item[r], pl->r_item[r + 1], pl->r_split[r], pl->r_split[r + 1], false, ps);
+            const size_t r0 = (size_t)q_off[r_user[r]], r1 = (size_t)q_off[r_user[r + 1]];
+            if (result == CKV_OK && r1 > r0) {
+                cudaError_t e = cudaMemcpyAsync((char*)out + r0 * o_row, (const char*)d_out + r0 * o_row, (r1 - r0) * o_row,
+                                                cudaMemcpyDeviceToHost, ps);
+                if (e != cudaSuccess) result = ctx->fail(e);
+            }
+        }
+    }
+    // whatever happened, the caller's stream continues behind everything that was enqueued on the internal ones
+    for (int r = 0; r < n_ranges; ++r) {
+        cudaEventRecord(ctx->pipe_done[r], ctx->pipe_stream[r]);
+        cudaStreamWaitEvent(s, ctx->pipe_done[r], 0);
+    }
+    return result;
+}
+
+}  // namespace
+
+extern "C" {
+
+ckv_status ckv_attend(ckv_ctx* ctx, int32_t n, const int64_t* users, const int32_t* q_off,
+                      const void* queries, void* out, void* stream)
+{
+    return attend_impl(ctx, n, users, q_off, nullptr, queries, out, stream);
+}
+
+ckv_status ckv_attend_visible(ckv_ctx* ctx, int32_t n, const int64_t* users, const int32_t* q_off, const int32_t* vis,
+                              const void* queries, void* out, void* stream)
+{
+    if (n > 0 && q_off && q_off[n] > 0 && !vis) return CKV_ERR_INVALID_ARG;
+    return attend_impl(ctx, n, users, q_off, vis, queries, out, stream);
 }
 
 ckv_status ckv_materialize(ckv_ctx* ctx, int64_t user, void* K_out, void* V_out, void* stream)
@@ -1225,7 +1451,9 @@ ckv_status ckv_cache_bytes(ckv_ctx* ctx, int64_t* compressed, int64_t* full_widt
 {
     if (!ctx || !compressed || !full_width) return CKV_ERR_INVALID_ARG;
     const int64_t pg = ctx->live_positions * ctx->cfg.n_groups;
-    *compressed = pg * (2 * (int64_t)ctx->idx_bytes + 2 * (int64_t)ctx->d_user * ctx->elem);
+    int64_t eb[4] = {0, 0, 0, 0};
+    if (ctx->pool) unit_bytes(ctx, eb);
+    *compressed = pg * (eb[0] + eb[1] + eb[2] + eb[3]);
     *full_width = pg * 2 * (int64_t)ctx->cfg.head_dim * ctx->elem;
     return CKV_OK;
 }
@@ -1351,6 +1579,7 @@ ckv_status ckv_last_stat(ckv_ctx* ctx, const char* name, int64_t* value)
     else if (!std::strcmp(name, "plan_cache_hit")) *value = ctx->st_hit;
     else if (!std::strcmp(name, "alloc_calls")) *value = ctx->st_allocs;
     else if (!std::strcmp(name, "l2_window")) *value = ctx->st_l2;
+    else if (!std::strcmp(name, "pipeline_ranges")) *value = ctx->st_ranges;
     else if (!std::strcmp(name, "arena_capacity_units")) *value = ctx->cap_units;
     else if (!std::strcmp(name, "arena_used_units")) *value = ctx->used_units;
     else if (!std::strcmp(name, "arena_free_runs")) *value = (int64_t)ctx->free_runs.size();
@@ -1556,6 +1785,7 @@ extern "C" ckv_status ckv_attend_static(ckv_ctx* ctx, int32_t n, const int64_t* 
     a.works = nullptr;
     a.n_items = n_items;
     a.queries = queries;
+    a.vis = nullptr;
     a.out = out;
     a.partials = (float*)(base + kOffPartials);  // every entry that is read was written by this call
     a.out_dtype = ctx->cfg.out_dtype;

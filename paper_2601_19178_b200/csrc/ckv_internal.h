@@ -48,8 +48,12 @@ struct CacheView {
     const void* userV;
     int32_t n_groups;
     int32_t n_entries;
-    int32_t d_user;
+    int32_t d_user;      // user-specific elements per unit of a shared side
     int32_t idx_bytes;   // 2 or 4
+    // Sharing only keys or only values: a side that is not shared has no pool and no indices (poolX, idxX
+    // null); its userX array holds the full head_dim-wide row of every unit.
+    int32_t full_k;
+    int32_t full_v;
 };
 
 struct AttendArgs {
@@ -59,6 +63,7 @@ struct AttendArgs {
     const Work* works;     // one per item, same order (tcgen05 family only, else null)
     int32_t n_items;
     const void* queries;   // [Q][G][D]
+    const int32_t* vis;    // null, or per query row the number of leading history positions it attends [Q]
     void* out;             // [Q][G][D]
     float* partials;       // [part rows][G][D + 2]  (m, l, acc[D])
     int32_t out_dtype;     // ckv_dtype
@@ -71,21 +76,23 @@ cudaError_t launch_pool_layout(int dtype, int G, int m, int d_shared, int D, con
                                void* dst, cudaStream_t s);
 // Packs n users' [P][G] indices and [P][G][d_user] user parts into arena units and
 // validates index range; *bad_flag (device int) is OR-ed with 1 on a bad index.
-cudaError_t launch_pack(int dtype, int G, int n_entries, int d_user, int idx_bytes, int n_users,
+// The arena arrays and the sides' widths come from `cv` (head_dim D).
+cudaError_t launch_pack(int dtype, int G, int n_entries, int idx_bytes, int n_users,
                         const int64_t* hist_off_dev, const int64_t* unit_off_dev,
                         int64_t total_units, int64_t arena_base, const int32_t* idxK,
-                        const int32_t* idxV, const void* userK, const void* userV, void* a_idxK,
-                        void* a_idxV, void* a_userK, void* a_userV, int* bad_flag, cudaStream_t s);
+                        const int32_t* idxV, const void* userK, const void* userV, const CacheView& cv, int D,
+                        int* bad_flag, cudaStream_t s);
 // Writes a user's units for L_old + L_new positions at arena unit dst_base: the first L_old positions copied from
 // the units at old_base (same arena), the rest packed from the new [L_new][G] indices and [L_new][G][d_user] parts.
-cudaError_t launch_append(int dtype, int G, int n_entries, int d_user, int idx_bytes, int64_t old_base, int L_old,
+cudaError_t launch_append(int dtype, int G, int n_entries, int idx_bytes, int64_t old_base, int L_old,
                           int Lpad_old, int64_t dst_base, int L_new, int Lpad_tot, const int32_t* idxK,
-                          const int32_t* idxV, const void* userK, const void* userV, void* a_idxK, void* a_idxV,
-                          void* a_userK, void* a_userV, int* bad_flag, cudaStream_t s);
+                          const int32_t* idxV, const void* userK, const void* userV, const CacheView& cv, int D,
+                          int* bad_flag, cudaStream_t s);
 cudaError_t launch_materialize(int dtype, int D, const CacheView& cv, int64_t base, int L, int Lpad,
                                void* K_out, void* V_out, cudaStream_t s);
 
-// ORs 1 into *bad_flag (device int) if any of the n_units stored K or V indices is >= n_entries.
+// ORs 1 into *bad_flag (device int) if any of the n_units stored K or V indices is >= n_entries (idxK or idxV may be
+// null: that side is not checked).
 cudaError_t launch_check_indices(int idx_bytes, int n_entries, const void* idxK, const void* idxV, int64_t n_units,
                                  int* bad_flag, cudaStream_t s);
 
@@ -96,7 +103,7 @@ cudaError_t launch_combine(int D, const AttendArgs& a, const int32_t* split_reqs
                            cudaStream_t s);
 
 // ---- kernels_mma.cu : warp-level tensor-core family (bf16, head_dim 32 or 64, d_user <= 8)
-bool mma_supported(int dtype, int head_dim, int d_user);
+bool mma_supported(int dtype, int head_dim, int d_user);  // d_user of the shared side(s)
 int mma_queries_per_warp(int head_dim, int max_M);
 // tensor_maps: null = fill the staging ring with cp.async copies; else the two maps of make_pool_tensor_maps =
 // fill it with TMA gathers (err_flag: device int, OR-ed with a code if a bounded wait for a tile ran out).

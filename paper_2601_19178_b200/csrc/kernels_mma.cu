@@ -9,6 +9,9 @@
 // row, and the copies in flight cost no registers: a warp keeps NST - 1 tiles outstanding
 // while it computes.  The user-specific leading elements (Eq. K) are written over the head
 // of each staged row.  Positions keep their order: tile row r is position p0 + r.
+// A side that is not shared (sharing only keys or only values) has its full-width rows in the
+// arena; they are copied into the ring in place of pool rows (cp.async loader only) and nothing is
+// patched.  With visible lengths a query row only takes the positions before its own limit.
 //
 // Two ways to fill the ring (template parameter TMA), same results bit for bit:
 //   - 16-byte cp.async copies through L1 (hot rows of skewed index distributions stay in L1, but every
@@ -128,7 +131,9 @@ __device__ __forceinline__ int swz(int r)
     return D == 64 ? (r & 7) : ((r >> 1) & 3);
 }
 
-template <int D, int MT, int MODE, bool IDX16, bool TMA>
+// VAR = false: both sides shared and no visible lengths (the hot configurations); the code for the variants is
+// compiled out.
+template <int D, int MT, int MODE, bool IDX16, bool TMA, bool VAR>
 __global__ void __launch_bounds__(128, MmaCfg<D, MT, TMA>::MIN_BLOCKS)
     attend_mma_kernel(const AttendArgs a, int n_mb, const __grid_constant__ CUtensorMap tmK,
                       const __grid_constant__ CUtensorMap tmV, int* err_flag)
@@ -146,6 +151,7 @@ __global__ void __launch_bounds__(128, MmaCfg<D, MT, TMA>::MIN_BLOCKS)
     const int row0 = mb * 16 * MT;
     if (row0 >= rq.M) return;
     const int grp = blockIdx.y, G = a.cv.n_groups, d_user = a.cv.d_user;
+    const bool full_k = VAR && a.cv.full_k != 0, full_v = VAR && a.cv.full_v != 0;  // the side's rows are cached full width
     const bool wide_user = d_user == 1 || d_user == 2 || d_user == 4 || d_user == 8;
 
     uint32_t qa[MT][KS][4];
@@ -166,6 +172,29 @@ __global__ void __launch_bounds__(128, MmaCfg<D, MT, TMA>::MIN_BLOCKS)
     }
     // rows 8..15 of the only query tile are all padding when the user has at most 8 queries
     const bool has_hi = MT > 1 || row0 + 8 < rq.M;
+    // positions a query row attends: [0, lim); rows beyond the user's queries take none
+    int lim[MT][2], lim_max = rq.L, lim_min = rq.L;
+    if constexpr (VAR) {
+        lim_max = 0;
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int r = row0 + 16 * mt + g + 8 * h;
+                int v = 0;
+                if (r < rq.M) {
+                    v = a.vis ? min(max(__ldg(a.vis + rq.q0 + r), 0), rq.L) : rq.L;
+                    lim_min = min(lim_min, v);
+                }
+                lim[mt][h] = v;
+                lim_max = max(lim_max, v);
+            }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            lim_max = max(lim_max, __shfl_xor_sync(0xffffffffu, lim_max, o));
+            lim_min = min(lim_min, __shfl_xor_sync(0xffffffffu, lim_min, o));
+        }
+    }
 
     float o[MT][NTD][4];
     float m_run[MT][2], l_run[MT][2];
@@ -185,8 +214,13 @@ __global__ void __launch_bounds__(128, MmaCfg<D, MT, TMA>::MIN_BLOCKS)
     const int64_t unit0 = rq.base + (int64_t)grp * rq.Lpad + it.begin + lane;  // this lane's position of step 0
     const uint16_t* uK = reinterpret_cast<const uint16_t*>(a.cv.userK);
     const uint16_t* uV = reinterpret_cast<const uint16_t*>(a.cv.userV);
-    const int end = it.begin + it.len;
-    const int nsteps = (it.len + 31) >> 5;
+    const int end = VAR ? min(it.begin + it.len, lim_max) : it.begin + it.len;  // nothing behind the last visible position is touched
+    const int nsteps = VAR ? (end > it.begin ? (end - it.begin + 31) >> 5 : 0) : (it.len + 31) >> 5;
+    const int full_end = VAR ? min(end, lim_min) : end;  // up to here every row of this warp sees every position
+    // A side that is not shared: its rows are the chunk's own units in the arena, and what stands in for the pool
+    // index of the position in lane l of tile `step` is its offset 32 step + l from the chunk's first unit.
+    if (full_k) pK = reinterpret_cast<const char*>(a.cv.userK) + (unit0 - lane) * ROWB + cc * 16;
+    if (full_v) pV = reinterpret_cast<const char*>(a.cv.userV) + (unit0 - lane) * ROWB + cc * 16;
     const float sc = a.scale * (MODE == CKV_SOFTMAX ? kLog2e : 0.5f);
 
     uint32_t smem0 = smem_u32(smem_raw);
@@ -260,16 +294,16 @@ __global__ void __launch_bounds__(128, MmaCfg<D, MT, TMA>::MIN_BLOCKS)
     };
     auto fetch_idx = [&](int step, int& idx_k, int& idx_v) {
         if (step < nsteps) {
-            idx_k = load_index<IDX16>(a.cv.idxK, unit0 + 32 * step);
-            idx_v = load_index<IDX16>(a.cv.idxV, unit0 + 32 * step);
+            idx_k = full_k ? 32 * step + lane : load_index<IDX16>(a.cv.idxK, unit0 + 32 * step);
+            idx_v = full_v ? 32 * step + lane : load_index<IDX16>(a.cv.idxV, unit0 + 32 * step);
         } else {
             idx_k = idx_v = 0;
         }
     };
     auto fetch_user = [&](int step, uint4& k, uint4& v) {
         if (wide_user && step < nsteps) {
-            k = load_user_part(uK, unit0 + 32 * step, d_user);
-            v = load_user_part(uV, unit0 + 32 * step, d_user);
+            if (!full_k) k = load_user_part(uK, unit0 + 32 * step, d_user);
+            if (!full_v) v = load_user_part(uV, unit0 + 32 * step, d_user);
         }
     };
 
@@ -316,20 +350,24 @@ __global__ void __launch_bounds__(128, MmaCfg<D, MT, TMA>::MIN_BLOCKS)
         const uint32_t kt = ring + (step % NST) * (2 * C::TILE_B), vt = kt + C::TILE_B;
         // Eq. K: dims [0, d_user) of every row come from the user-specific part
         if (wide_user) {
-            store_user_part(kt + offU, ukA, d_user);
-            store_user_part(vt + offU, uvA, d_user);
+            if (!full_k) store_user_part(kt + offU, ukA, d_user);
+            if (!full_v) store_user_part(vt + offU, uvA, d_user);
             ukA = ukB; uvA = uvB;
             fetch_user(step + 2, ukB, uvB);
-        } else if (d_user > 0) {
+        } else if (d_user > 0 && !(full_k && full_v)) {
             for (int e = 0; e < d_user; ++e) {
-                const uint16_t xk = __ldg(uK + (unit0 + 32 * step) * d_user + e);
-                const uint16_t xv = __ldg(uV + (unit0 + 32 * step) * d_user + e);
-                asm volatile("st.shared.u16 [%0], %1;" ::"r"(kt + offU + 2 * e), "h"(xk) : "memory");
-                asm volatile("st.shared.u16 [%0], %1;" ::"r"(vt + offU + 2 * e), "h"(xv) : "memory");
+                if (!full_k) {
+                    const uint16_t xk = __ldg(uK + (unit0 + 32 * step) * d_user + e);
+                    asm volatile("st.shared.u16 [%0], %1;" ::"r"(kt + offU + 2 * e), "h"(xk) : "memory");
+                }
+                if (!full_v) {
+                    const uint16_t xv = __ldg(uV + (unit0 + 32 * step) * d_user + e);
+                    asm volatile("st.shared.u16 [%0], %1;" ::"r"(vt + offU + 2 * e), "h"(xv) : "memory");
+                }
             }
         }
         __syncwarp();
-        const bool tail = p0 + 32 > end;
+        const bool tail = p0 + 32 > full_end;  // some (row, position) pair of this tile is not attended
 
         uint32_t kf[4][2 * KS];
 #pragma unroll
@@ -364,10 +402,14 @@ __global__ void __launch_bounds__(128, MmaCfg<D, MT, TMA>::MIN_BLOCKS)
             uint32_t pa[2][4];
             if constexpr (MODE == CKV_SOFTMAX) {
                 if (tail) {
+                    const int e_lo = VAR ? min(end, lim[mt][0]) : end, e_hi = VAR ? min(end, lim[mt][1]) : end;
 #pragma unroll
                     for (int nt = 0; nt < 4; ++nt) {
-                        if (p0 + 8 * nt + 2 * t >= end) s[nt][0] = s[nt][2] = -CUDART_INF_F;
-                        if (p0 + 8 * nt + 2 * t + 1 >= end) s[nt][1] = s[nt][3] = -CUDART_INF_F;
+                        const int pc = p0 + 8 * nt + 2 * t;
+                        if (pc >= e_lo) s[nt][0] = -CUDART_INF_F;
+                        if (pc + 1 >= e_lo) s[nt][1] = -CUDART_INF_F;
+                        if (pc >= e_hi) s[nt][2] = -CUDART_INF_F;
+                        if (pc + 1 >= e_hi) s[nt][3] = -CUDART_INF_F;
                     }
                 }
                 float mx0 = s[0][0], mx1 = s[0][2];
@@ -382,13 +424,16 @@ __global__ void __launch_bounds__(128, MmaCfg<D, MT, TMA>::MIN_BLOCKS)
                     mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
                     mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
                 }
-                // the first position of a tile is always valid, so mx is finite
+                // a row may not see any position of this tile (or of any tile so far): its maximum is then -inf
+                // and must not enter the exponent arguments
                 const float mn0 = fmaxf(m_run[mt][0], mx0 * sc);
                 const float mn1 = has_hi ? fmaxf(m_run[mt][1], mx1 * sc) : 0.f;
+                // (without visible lengths the first position of a tile is always attended and the maxima are finite)
+                const float ms0 = VAR && mn0 == -CUDART_INF_F ? 0.f : mn0, ms1 = VAR && mn1 == -CUDART_INF_F ? 0.f : mn1;
                 // the running maxima settle after a few tiles: rescale only when one of them moved
                 const bool moved = mn0 != m_run[mt][0] || (has_hi && mn1 != m_run[mt][1]);
                 if (__any_sync(0xffffffffu, moved)) {
-                    const float c0 = ex2(m_run[mt][0] - mn0), c1 = has_hi ? ex2(m_run[mt][1] - mn1) : 1.f;
+                    const float c0 = ex2(m_run[mt][0] - ms0), c1 = has_hi ? ex2(m_run[mt][1] - ms1) : 1.f;
                     m_run[mt][0] = mn0;
                     if (has_hi) m_run[mt][1] = mn1;
                     l_run[mt][0] *= c0;
@@ -402,11 +447,11 @@ __global__ void __launch_bounds__(128, MmaCfg<D, MT, TMA>::MIN_BLOCKS)
                 float ps0 = 0.f, ps1 = 0.f;
 #pragma unroll
                 for (int nt = 0; nt < 4; ++nt) {
-                    const float p0v = ex2(fmaf(s[nt][0], sc, -mn0)), p1v = ex2(fmaf(s[nt][1], sc, -mn0));
+                    const float p0v = ex2(fmaf(s[nt][0], sc, -ms0)), p1v = ex2(fmaf(s[nt][1], sc, -ms0));
                     ps0 += p0v + p1v;
                     pa[nt >> 1][(nt & 1) * 2] = pack_bf16(p0v, p1v);
                     if (has_hi) {
-                        const float p2v = ex2(fmaf(s[nt][2], sc, -mn1)), p3v = ex2(fmaf(s[nt][3], sc, -mn1));
+                        const float p2v = ex2(fmaf(s[nt][2], sc, -ms1)), p3v = ex2(fmaf(s[nt][3], sc, -ms1));
                         ps1 += p2v + p3v;
                         pa[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(p2v, p3v);
                     } else {
@@ -426,8 +471,12 @@ __global__ void __launch_bounds__(128, MmaCfg<D, MT, TMA>::MIN_BLOCKS)
                         w[e] = (e < 2 || has_hi) ? fmaf(h, tanh_fast(h), h) : 0.f;
                     }
                     if (tail) {
-                        if (p0 + 8 * nt + 2 * t >= end) w[0] = w[2] = 0.f;
-                        if (p0 + 8 * nt + 2 * t + 1 >= end) w[1] = w[3] = 0.f;
+                        const int e_lo = VAR ? min(end, lim[mt][0]) : end, e_hi = VAR ? min(end, lim[mt][1]) : end,
+                                  pc = p0 + 8 * nt + 2 * t;
+                        if (pc >= e_lo) w[0] = 0.f;
+                        if (pc + 1 >= e_lo) w[1] = 0.f;
+                        if (pc >= e_hi) w[2] = 0.f;
+                        if (pc + 1 >= e_hi) w[3] = 0.f;
                     }
                     pa[nt >> 1][(nt & 1) * 2] = pack_bf16(w[0], w[1]);
                     pa[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(w[2], w[3]);
@@ -492,17 +541,17 @@ __global__ void __launch_bounds__(128, MmaCfg<D, MT, TMA>::MIN_BLOCKS)
     }
 }
 
-template <int D, int MT, int MODE, bool IDX16, bool TMA>
+template <int D, int MT, int MODE, bool IDX16, bool TMA, bool VAR>
 cudaError_t launch_mma_one(const AttendArgs& a, int n_mb, dim3 grid, const CUtensorMap* maps, int* err_flag,
                            cudaStream_t s)
 {
     using C = MmaCfg<D, MT, TMA>;
     // per launch: the attribute belongs to the current device, and a context may sit on any of them
-    cudaError_t e = cudaFuncSetAttribute(attend_mma_kernel<D, MT, MODE, IDX16, TMA>,
+    cudaError_t e = cudaFuncSetAttribute(attend_mma_kernel<D, MT, MODE, IDX16, TMA, VAR>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
     if (e != cudaSuccess) return e;
     static const CUtensorMap none{};
-    attend_mma_kernel<D, MT, MODE, IDX16, TMA>
+    attend_mma_kernel<D, MT, MODE, IDX16, TMA, VAR>
         <<<grid, 128, C::SMEM, s>>>(a, n_mb, TMA ? maps[0] : none, TMA ? maps[1] : none, err_flag);
     return cudaGetLastError();
 }
@@ -513,9 +562,11 @@ cudaError_t launch_mma(const AttendArgs& a, int n_mb, const CUtensorMap* maps, i
     const int64_t warps = (int64_t)a.n_items * n_mb;
     const dim3 grid((unsigned)((warps + 3) / 4), a.cv.n_groups);
     const bool i16 = a.cv.idx_bytes == 2;
+    const bool var = a.vis != nullptr || a.cv.full_k || a.cv.full_v;  // the TMA loader is never asked for with these
 #define CKV_MMA_GO(MODE, I16)                                                                        \
-    (maps ? launch_mma_one<D, MT, MODE, I16, true>(a, n_mb, grid, maps, err_flag, s)                 \
-          : launch_mma_one<D, MT, MODE, I16, false>(a, n_mb, grid, maps, err_flag, s))
+    (maps  ? launch_mma_one<D, MT, MODE, I16, true, false>(a, n_mb, grid, maps, err_flag, s)         \
+     : var ? launch_mma_one<D, MT, MODE, I16, false, true>(a, n_mb, grid, maps, err_flag, s)         \
+           : launch_mma_one<D, MT, MODE, I16, false, false>(a, n_mb, grid, maps, err_flag, s))
     if (a.mode == CKV_SOFTMAX) return i16 ? CKV_MMA_GO(CKV_SOFTMAX, true) : CKV_MMA_GO(CKV_SOFTMAX, false);
     return i16 ? CKV_MMA_GO(CKV_SILU_OVER_L, true) : CKV_MMA_GO(CKV_SILU_OVER_L, false);
 #undef CKV_MMA_GO

@@ -21,17 +21,44 @@ __global__ void pool_layout_kernel(const E* __restrict__ src, E* __restrict__ ds
     }
 }
 
+// The two sides of a cache entry (K and V) are stored alike but may differ in width: a shared side keeps a pool
+// index and d_user user-specific elements per unit, a side that is not shared (sharing only keys or only values)
+// keeps the whole head_dim-wide row and no index.
+struct SideDst {
+    void* idx;     // arena indices, null for a side that is not shared
+    void* user;    // arena user parts / full rows
+    int width;     // elements per unit in `user`
+};
+
+template <typename E, typename I>
+__device__ __forceinline__ void store_unit(const SideDst& d, int64_t dst, const int32_t* idx_src, const E* user_src,
+                                           int64_t src, bool real, int n_entries, int* bad_flag)
+{
+    E* du = reinterpret_cast<E*>(d.user);
+    if (real) {
+        for (int c = 0; c < d.width; ++c) du[dst * d.width + c] = user_src[src * d.width + c];
+    } else {  // padding: a valid row index and zeros
+        for (int c = 0; c < d.width; ++c) du[dst * d.width + c] = E(0);
+    }
+    if (d.idx) {
+        int32_t j = real ? idx_src[src] : 0;
+        if (j < 0 || j >= n_entries) {
+            atomicOr(bad_flag, 1);
+            j = 0;
+        }
+        reinterpret_cast<I*>(d.idx)[dst] = (I)j;
+    }
+}
+
 // One thread per arena unit of the batch.  unit_off[u] = sum over earlier users of
 // G * Lpad; the unit of (user u, group g, position i) is unit_off[u] + g * Lpad_u + i.
 template <typename E, typename I>
-__global__ void pack_kernel(int G, int n_entries, int d_user, int n_users,
+__global__ void pack_kernel(int G, int n_entries, int n_users,
                             const int64_t* __restrict__ hist_off,
                             const int64_t* __restrict__ unit_off, int64_t total_units,
                             int64_t arena_base, const int32_t* __restrict__ idxK,
                             const int32_t* __restrict__ idxV, const E* __restrict__ userK,
-                            const E* __restrict__ userV, I* __restrict__ a_idxK,
-                            I* __restrict__ a_idxV, E* __restrict__ a_userK,
-                            E* __restrict__ a_userV, int* __restrict__ bad_flag)
+                            const E* __restrict__ userV, SideDst dK, SideDst dV, int* __restrict__ bad_flag)
 {
     for (int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; t < total_units;
          t += (int64_t)gridDim.x * blockDim.x) {
@@ -47,38 +74,27 @@ __global__ void pack_kernel(int G, int n_entries, int d_user, int n_users,
         const int64_t i = local - g * Lpad;
         const int64_t L = hist_off[u + 1] - hist_off[u];
         const int64_t dst = arena_base + t;
-        int32_t ik = 0, iv = 0;
-        if (i < L) {
-            const int64_t src = (hist_off[u] + i) * G + g;
-            ik = idxK[src];
-            iv = idxV[src];
-            if (ik < 0 || ik >= n_entries || iv < 0 || iv >= n_entries) {
-                atomicOr(bad_flag, 1);
-                ik = iv = 0;
-            }
-            for (int c = 0; c < d_user; ++c) {
-                a_userK[dst * d_user + c] = userK[src * d_user + c];
-                a_userV[dst * d_user + c] = userV[src * d_user + c];
-            }
-        } else {  // padding: a valid row index and a zero user part
-            for (int c = 0; c < d_user; ++c) {
-                a_userK[dst * d_user + c] = E(0);
-                a_userV[dst * d_user + c] = E(0);
-            }
-        }
-        a_idxK[dst] = (I)ik;
-        a_idxV[dst] = (I)iv;
+        const int64_t src = (hist_off[u] + i) * G + g;
+        store_unit<E, I>(dK, dst, idxK, userK, src, i < L, n_entries, bad_flag);
+        store_unit<E, I>(dV, dst, idxV, userV, src, i < L, n_entries, bad_flag);
     }
+}
+
+template <typename E, typename I>
+__device__ __forceinline__ void copy_unit(const SideDst& d, int64_t dst, int64_t src)
+{
+    E* du = reinterpret_cast<E*>(d.user);
+    for (int c = 0; c < d.width; ++c) du[dst * d.width + c] = du[src * d.width + c];
+    if (d.idx) reinterpret_cast<I*>(d.idx)[dst] = reinterpret_cast<I*>(d.idx)[src];
 }
 
 // Append: units of one user with L_old + L_new positions at arena unit `dst_base`; position i < L_old is copied
 // from the user's old units, the rest comes from the new [L_new][G] inputs (range-checked like pack_kernel).
 template <typename E, typename I>
-__global__ void append_kernel(int G, int n_entries, int d_user, int64_t old_base, int L_old, int Lpad_old,
+__global__ void append_kernel(int G, int n_entries, int64_t old_base, int L_old, int Lpad_old,
                               int64_t dst_base, int L_new, int Lpad_tot, const int32_t* __restrict__ idxK,
                               const int32_t* __restrict__ idxV, const E* __restrict__ userK,
-                              const E* __restrict__ userV, I* a_idxK, I* a_idxV, E* a_userK, E* a_userV,
-                              int* __restrict__ bad_flag)
+                              const E* __restrict__ userV, SideDst dK, SideDst dV, int* __restrict__ bad_flag)
 {
     const int64_t total = (int64_t)G * Lpad_tot;
     for (int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; t < total; t += (int64_t)gridDim.x * blockDim.x) {
@@ -87,44 +103,28 @@ __global__ void append_kernel(int G, int n_entries, int d_user, int64_t old_base
         const int64_t dst = dst_base + t;
         if (i < L_old) {
             const int64_t src = old_base + (int64_t)g * Lpad_old + i;
-            a_idxK[dst] = a_idxK[src];
-            a_idxV[dst] = a_idxV[src];
-            for (int c = 0; c < d_user; ++c) {
-                a_userK[dst * d_user + c] = a_userK[src * d_user + c];
-                a_userV[dst * d_user + c] = a_userV[src * d_user + c];
-            }
-        } else if (i < L_old + L_new) {
+            copy_unit<E, I>(dK, dst, src);
+            copy_unit<E, I>(dV, dst, src);
+        } else {
             const int64_t src = (int64_t)(i - L_old) * G + g;
-            int32_t ik = idxK[src], iv = idxV[src];
-            if (ik < 0 || ik >= n_entries || iv < 0 || iv >= n_entries) {
-                atomicOr(bad_flag, 1);
-                ik = iv = 0;
-            }
-            a_idxK[dst] = (I)ik;
-            a_idxV[dst] = (I)iv;
-            for (int c = 0; c < d_user; ++c) {
-                a_userK[dst * d_user + c] = userK[src * d_user + c];
-                a_userV[dst * d_user + c] = userV[src * d_user + c];
-            }
-        } else {  // padding: a valid row index and a zero user part
-            a_idxK[dst] = (I)0;
-            a_idxV[dst] = (I)0;
-            for (int c = 0; c < d_user; ++c) {
-                a_userK[dst * d_user + c] = E(0);
-                a_userV[dst * d_user + c] = E(0);
-            }
+            const bool real = i < L_old + L_new;
+            store_unit<E, I>(dK, dst, idxK, userK, src, real, n_entries, bad_flag);
+            store_unit<E, I>(dV, dst, idxV, userV, src, real, n_entries, bad_flag);
         }
     }
 }
 
 template <typename E, typename I>
-__global__ void materialize_kernel(int G, int n_entries, int d_user, int D,
-                                   const E* __restrict__ poolK, const E* __restrict__ poolV,
-                                   const I* __restrict__ idxK, const I* __restrict__ idxV,
-                                   const E* __restrict__ userK, const E* __restrict__ userV,
-                                   int64_t base, int L, int Lpad, E* __restrict__ K_out,
-                                   E* __restrict__ V_out)
+__global__ void materialize_kernel(int G, int n_entries, int D, CacheView cv, int64_t base, int L, int Lpad,
+                                   E* __restrict__ K_out, E* __restrict__ V_out)
 {
+    const E* poolK = reinterpret_cast<const E*>(cv.poolK);
+    const E* poolV = reinterpret_cast<const E*>(cv.poolV);
+    const I* idxK = reinterpret_cast<const I*>(cv.idxK);
+    const I* idxV = reinterpret_cast<const I*>(cv.idxV);
+    const E* userK = reinterpret_cast<const E*>(cv.userK);
+    const E* userV = reinterpret_cast<const E*>(cv.userV);
+    const int duk = cv.full_k ? D : cv.d_user, duv = cv.full_v ? D : cv.d_user;
     const int64_t total = (int64_t)L * G * D;
     for (int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; t < total;
          t += (int64_t)gridDim.x * blockDim.x) {
@@ -133,13 +133,8 @@ __global__ void materialize_kernel(int G, int n_entries, int d_user, int D,
         const int g = (int)(ig % G);
         const int64_t i = ig / G;
         const int64_t unit = base + (int64_t)g * Lpad + i;
-        if (c < d_user) {
-            K_out[t] = userK[unit * d_user + c];
-            V_out[t] = userV[unit * d_user + c];
-        } else {
-            K_out[t] = poolK[((int64_t)g * n_entries + (int64_t)idxK[unit]) * D + c];
-            V_out[t] = poolV[((int64_t)g * n_entries + (int64_t)idxV[unit]) * D + c];
-        }
+        K_out[t] = c < duk ? userK[unit * duk + c] : poolK[((int64_t)g * n_entries + (int64_t)idxK[unit]) * D + c];
+        V_out[t] = c < duv ? userV[unit * duv + c] : poolV[((int64_t)g * n_entries + (int64_t)idxV[unit]) * D + c];
     }
 }
 
@@ -150,7 +145,7 @@ __global__ void check_indices_kernel(const I* __restrict__ a, const I* __restric
 {
     bool bad = false;
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
-        bad |= (uint32_t)a[i] >= n_entries || (uint32_t)b[i] >= n_entries;
+        bad |= (a && (uint32_t)a[i] >= n_entries) || (b && (uint32_t)b[i] >= n_entries);
     if (__any_sync(0xffffffffu, bad) && (threadIdx.x & 31) == 0) atomicOr(bad_flag, 1);
 }
 
@@ -178,19 +173,20 @@ cudaError_t launch_pool_layout(int dtype, int G, int m, int d_shared, int D, con
     return cudaGetLastError();
 }
 
-cudaError_t launch_pack(int dtype, int G, int n_entries, int d_user, int idx_bytes, int n_users,
+cudaError_t launch_pack(int dtype, int G, int n_entries, int idx_bytes, int n_users,
                         const int64_t* hist_off_dev, const int64_t* unit_off_dev,
                         int64_t total_units, int64_t arena_base, const int32_t* idxK,
-                        const int32_t* idxV, const void* userK, const void* userV, void* a_idxK,
-                        void* a_idxV, void* a_userK, void* a_userV, int* bad_flag, cudaStream_t s)
+                        const int32_t* idxV, const void* userK, const void* userV, const CacheView& cv, int D,
+                        int* bad_flag, cudaStream_t s)
 {
     if (total_units == 0) return cudaSuccess;
     const int grid = grid_for(total_units, 256);
+    const SideDst dK{cv.full_k ? nullptr : const_cast<void*>(cv.idxK), const_cast<void*>(cv.userK), cv.full_k ? D : cv.d_user};
+    const SideDst dV{cv.full_v ? nullptr : const_cast<void*>(cv.idxV), const_cast<void*>(cv.userV), cv.full_v ? D : cv.d_user};
 #define CKV_PACK(E, I)                                                                          \
-    pack_kernel<E, I><<<grid, 256, 0, s>>>(G, n_entries, d_user, n_users, hist_off_dev,          \
-                                           unit_off_dev, total_units, arena_base, idxK, idxV,    \
-                                           (const E*)userK, (const E*)userV, (I*)a_idxK,         \
-                                           (I*)a_idxV, (E*)a_userK, (E*)a_userV, bad_flag)
+    pack_kernel<E, I><<<grid, 256, 0, s>>>(G, n_entries, n_users, hist_off_dev, unit_off_dev,   \
+                                           total_units, arena_base, idxK, idxV, (const E*)userK, \
+                                           (const E*)userV, dK, dV, bad_flag)
     if (dtype == CKV_BF16) {
         if (idx_bytes == 2) CKV_PACK(uint16_t, uint16_t); else CKV_PACK(uint16_t, int32_t);
     } else {
@@ -200,18 +196,20 @@ cudaError_t launch_pack(int dtype, int G, int n_entries, int d_user, int idx_byt
     return cudaGetLastError();
 }
 
-cudaError_t launch_append(int dtype, int G, int n_entries, int d_user, int idx_bytes, int64_t old_base, int L_old,
+cudaError_t launch_append(int dtype, int G, int n_entries, int idx_bytes, int64_t old_base, int L_old,
                           int Lpad_old, int64_t dst_base, int L_new, int Lpad_tot, const int32_t* idxK,
-                          const int32_t* idxV, const void* userK, const void* userV, void* a_idxK, void* a_idxV,
-                          void* a_userK, void* a_userV, int* bad_flag, cudaStream_t s)
+                          const int32_t* idxV, const void* userK, const void* userV, const CacheView& cv, int D,
+                          int* bad_flag, cudaStream_t s)
 {
     const int64_t total = (int64_t)G * Lpad_tot;
     if (total == 0) return cudaSuccess;
     const int grid = grid_for(total, 256);
+    const SideDst dK{cv.full_k ? nullptr : const_cast<void*>(cv.idxK), const_cast<void*>(cv.userK), cv.full_k ? D : cv.d_user};
+    const SideDst dV{cv.full_v ? nullptr : const_cast<void*>(cv.idxV), const_cast<void*>(cv.userV), cv.full_v ? D : cv.d_user};
 #define CKV_APPEND(E, I)                                                                                       \
-    append_kernel<E, I><<<grid, 256, 0, s>>>(G, n_entries, d_user, old_base, L_old, Lpad_old, dst_base, L_new, \
-                                             Lpad_tot, idxK, idxV, (const E*)userK, (const E*)userV,          \
-                                             (I*)a_idxK, (I*)a_idxV, (E*)a_userK, (E*)a_userV, bad_flag)
+    append_kernel<E, I><<<grid, 256, 0, s>>>(G, n_entries, old_base, L_old, Lpad_old, dst_base, L_new,        \
+                                             Lpad_tot, idxK, idxV, (const E*)userK, (const E*)userV, dK, dV,  \
+                                             bad_flag)
     if (dtype == CKV_BF16) {
         if (idx_bytes == 2) CKV_APPEND(uint16_t, uint16_t); else CKV_APPEND(uint16_t, int32_t);
     } else {
@@ -227,10 +225,8 @@ cudaError_t launch_materialize(int dtype, int D, const CacheView& cv, int64_t ba
     if (L == 0) return cudaSuccess;
     const int grid = grid_for((int64_t)L * cv.n_groups * D, 256);
 #define CKV_MAT(E, I)                                                                            \
-    materialize_kernel<E, I><<<grid, 256, 0, s>>>(                                               \
-        cv.n_groups, cv.n_entries, cv.d_user, D, (const E*)cv.poolK, (const E*)cv.poolV,         \
-        (const I*)cv.idxK, (const I*)cv.idxV, (const E*)cv.userK, (const E*)cv.userV, base, L,   \
-        Lpad, (E*)K_out, (E*)V_out)
+    materialize_kernel<E, I><<<grid, 256, 0, s>>>(cv.n_groups, cv.n_entries, D, cv, base, L, Lpad, \
+                                                  (E*)K_out, (E*)V_out)
     if (dtype == CKV_BF16) {
         if (cv.idx_bytes == 2) CKV_MAT(uint16_t, uint16_t); else CKV_MAT(uint16_t, int32_t);
     } else {

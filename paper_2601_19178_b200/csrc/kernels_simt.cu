@@ -8,6 +8,9 @@
 // rows therefore only ever exist in registers.  Scores are reduced over the LPR lanes
 // with shuffles, the softmax is the running-max form, and partial results of the
 // sub-warps / warps / history chunks are merged with the usual (m, l, acc) rule.
+// A side that is not shared (sharing only keys or only values) has its full-width rows in the
+// arena: they are read in place of the pool rows, coalesced, and nothing is patched.  With
+// visible lengths a query row only takes the positions before its own limit.
 #include <cuda_bf16.h>
 #include <math_constants.h>
 
@@ -99,11 +102,14 @@ __global__ void __launch_bounds__(kWarps * 32, QB == 1 ? 5 : 1) attend_simt_kern
     const int64_t unit0 = rq.base + (int64_t)g * rq.Lpad;
     const char* poolK = (const char*)cv.poolK + (int64_t)g * cv.n_entries * D * ES + ch * 16;
     const char* poolV = (const char*)cv.poolV + (int64_t)g * cv.n_entries * D * ES + ch * 16;
-    const bool owns_user = ch * EPL < d_user;
+    const bool full_k = cv.full_k != 0, full_v = cv.full_v != 0;  // the side's rows are cached full width
+    const char* rowsK = (const char*)cv.userK + ch * 16;
+    const char* rowsV = (const char*)cv.userV + ch * 16;
+    const bool owns_user = ch * EPL < d_user && !(full_k && full_v);
     // user part of a position in one load of at most 8 bytes: it fits the row's first lane and its size is a power of two
     const int user_bytes = d_user * ES;
     const bool wide_user = d_user <= EPL && (user_bytes == 2 || user_bytes == 4 || user_bytes == 8);
-    const int end = it.begin + it.len;
+    const int chunk_end = it.begin + it.len;
     const float qscale = a.scale * (MODE == CKV_SOFTMAX ? kLog2e : 1.0f);
 
     for (int qb = 0; qb < rq.M; qb += QB) {
@@ -120,6 +126,15 @@ __global__ void __launch_bounds__(kWarps * 32, QB == 1 ? 5 : 1) attend_simt_kern
                 for (int e = 0; e < EPL; ++e) q[r][e] = 0.f;
             }
         }
+        // positions query row r attends: [0, lim[r]); the block of rows stops at the largest limit
+        int lim[QB], end = 0;
+#pragma unroll
+        for (int r = 0; r < QB; ++r) {
+            lim[r] = 0;
+            if (qb + r < rq.M) lim[r] = a.vis ? min(max(__ldg(a.vis + rq.q0 + qb + r), 0), rq.L) : rq.L;
+            end = max(end, lim[r]);
+        }
+        end = min(end, chunk_end);
         float m_run[QB], l_run[QB], acc[QB][EPL];
 #pragma unroll
         for (int r = 0; r < QB; ++r) {
@@ -141,31 +156,31 @@ __global__ void __launch_bounds__(kWarps * 32, QB == 1 ? 5 : 1) attend_simt_kern
             for (int l = 0; l < NL; ++l) {
                 const int my_p = p0 + l * 32 + lane;
                 const int64_t my_unit = unit0 + ((l * 32 + lane < PPW * UNR && my_p < end) ? my_p : it.begin);
-                my_ik[l] = load_idx(cv.idxK, my_unit, idx_bytes);
-                my_iv[l] = load_idx(cv.idxV, my_unit, idx_bytes);
+                my_ik[l] = full_k ? 0 : load_idx(cv.idxK, my_unit, idx_bytes);
+                my_iv[l] = full_v ? 0 : load_idx(cv.idxV, my_unit, idx_bytes);
+                my_uk[l] = my_uv[l] = make_uint2(0, 0);
                 if (wide_user) {
-                    my_uk[l] = load_user(cv.userK, my_unit, user_bytes);
-                    my_uv[l] = load_user(cv.userV, my_unit, user_bytes);
+                    if (!full_k) my_uk[l] = load_user(cv.userK, my_unit, user_bytes);
+                    if (!full_v) my_uv[l] = load_user(cv.userV, my_unit, user_bytes);
                 }
             }
         };
         if (it.begin + warp * (PPW * UNR) < end) request_indices(it.begin + warp * (PPW * UNR));
         for (int p0 = it.begin + warp * (PPW * UNR); p0 < end; p0 += kWarps * PPW * UNR) {
-            bool valid[UNR];
+            int pos[UNR];
             uint4 kraw[UNR], vraw[UNR];
             int64_t unit[UNR];
 #pragma unroll
             for (int j = 0; j < UNR; ++j) {
-                const int p = p0 + j * PPW + sub;
-                valid[j] = p < end;
-                unit[j] = unit0 + (valid[j] ? p : it.begin);
+                pos[j] = p0 + j * PPW + sub;
+                unit[j] = unit0 + (pos[j] < end ? pos[j] : it.begin);
             }
 #pragma unroll
             for (int j = 0; j < UNR; ++j) {
                 const int src = (j * PPW) % 32 + sub;
                 const int ik = __shfl_sync(0xffffffffu, my_ik[(j * PPW) / 32], src), iv = __shfl_sync(0xffffffffu, my_iv[(j * PPW) / 32], src);
-                kraw[j] = ldg16(poolK + (int64_t)ik * (D * ES));
-                vraw[j] = ldg16(poolV + (int64_t)iv * (D * ES));
+                kraw[j] = full_k ? ldg16(rowsK + unit[j] * (D * ES)) : ldg16(poolK + (int64_t)ik * (D * ES));
+                vraw[j] = full_v ? ldg16(rowsV + unit[j] * (D * ES)) : ldg16(poolV + (int64_t)iv * (D * ES));
             }
             uint2 cur_uk[NL], cur_uv[NL];  // this step's user parts: the next request overwrites my_uk, my_uv
 #pragma unroll
@@ -198,8 +213,8 @@ __global__ void __launch_bounds__(kWarps * 32, QB == 1 ? 5 : 1) attend_simt_kern
 #pragma unroll
                         for (int e = 0; e < EPL; ++e) {
                             if (e < d_user) {
-                                k[e] = ku[e];
-                                v[j][e] = vu[e];
+                                if (!full_k) k[e] = ku[e];
+                                if (!full_v) v[j][e] = vu[e];
                             }
                         }
                     }
@@ -208,8 +223,8 @@ __global__ void __launch_bounds__(kWarps * 32, QB == 1 ? 5 : 1) attend_simt_kern
                     for (int e = 0; e < EPL; ++e) {
                         if (ch * EPL + e < d_user) {
                             const int64_t ui = unit[j] * d_user + ch * EPL + e;
-                            k[e] = load_elem<BF16>(cv.userK, ui);
-                            v[j][e] = load_elem<BF16>(cv.userV, ui);
+                            if (!full_k) k[e] = load_elem<BF16>(cv.userK, ui);
+                            if (!full_v) v[j][e] = load_elem<BF16>(cv.userV, ui);
                         }
                     }
                 }
@@ -235,7 +250,7 @@ __global__ void __launch_bounds__(kWarps * 32, QB == 1 ? 5 : 1) attend_simt_kern
                     float mn = m_run[r];
 #pragma unroll
                     for (int j = 0; j < UNR; ++j)
-                        if (valid[j]) mn = fmaxf(mn, s[j][r]);
+                        if (pos[j] < min(end, lim[r])) mn = fmaxf(mn, s[j][r]);
                     const float ms = mn == -CUDART_INF_F ? 0.f : mn;
                     const float corr = exp2f(m_run[r] - ms);
                     m_run[r] = mn;
@@ -244,7 +259,7 @@ __global__ void __launch_bounds__(kWarps * 32, QB == 1 ? 5 : 1) attend_simt_kern
                     for (int e = 0; e < EPL; ++e) acc[r][e] *= corr;
 #pragma unroll
                     for (int j = 0; j < UNR; ++j) {
-                        const float p = valid[j] ? exp2f(s[j][r] - ms) : 0.f;
+                        const float p = pos[j] < min(end, lim[r]) ? exp2f(s[j][r] - ms) : 0.f;
                         l_run[r] += p;
 #pragma unroll
                         for (int e = 0; e < EPL; ++e) acc[r][e] = fmaf(p, v[j][e], acc[r][e]);
@@ -253,7 +268,7 @@ __global__ void __launch_bounds__(kWarps * 32, QB == 1 ? 5 : 1) attend_simt_kern
 #pragma unroll
                     for (int j = 0; j < UNR; ++j) {
                         const float x = s[j][r];
-                        const float w = valid[j] ? x / (1.0f + expf(-x)) : 0.f;
+                        const float w = pos[j] < min(end, lim[r]) ? x / (1.0f + expf(-x)) : 0.f;
 #pragma unroll
                         for (int e = 0; e < EPL; ++e) acc[r][e] = fmaf(w, v[j][e], acc[r][e]);
                     }

@@ -12,13 +12,19 @@
 //               tile; the owner of a unit's first tile also stages Q
 //
 // A tile (128 positions) is split into two halves of 64 positions; half b belongs to group b,
-// which has two score buffers and two weight buffers in TMEM and uses them alternately:
+// which has three score buffers in TMEM and uses them in turn; the weights of a half tile are
+// written over the head of the scores they were computed from (32 columns of bf16 pairs over
+// 64 columns of fp32):
 //   S_bi  = Q K_half^T                UMMA 128 x 64 x 32, A = Q smem, B = half K tile smem (K-major)
-//   P_bi  = exp2(S_bi c - m) | silu   group b: tcgen05.ld -> math -> bf16 -> tcgen05.st
+//   P_bi  = exp2(S_bi c - m) | silu   group b: tcgen05.ld -> math -> bf16 -> tcgen05.st, in place
 //   O_b  += P_bi [V_half | 1]         UMMA 128 x 48 x 64, A = P from TMEM, B = half V tile (MN-major)
-// While group b normalises its half of tile t, its scores of tile t+1 are already being
-// computed into the other buffer, the other group works on its own half, and the producers
-// gather tiles t+2...; nothing drains between work units.  The two groups keep separate
+// A buffer is free again when the weighted sum that read it has finished.  With three of them
+// the scores of step t+2 are issued while step t is being normalised: the round trip of a
+// hand-off through the tensor core (issue, a chain of K = 16 instructions, commit, the waiting
+// thread waking up: about a thousand clocks) is longer than one normalisation step, and with two
+// buffers both the normalisation threads and the issuing threads kept waiting for each other.
+// The other group works on its own half at the same time and the producers gather tiles
+// further ahead; nothing drains between work units.  The two groups keep separate
 // accumulators O_0, O_1 with separate reference maxima and merge them through shared memory
 // when a unit ends.
 //
@@ -30,10 +36,11 @@
 //
 // Softmax bookkeeping.  The V tile carries sixteen extra columns of which the first is all
 // ones, so column 32 of O_b accumulates the row sum l of exactly the bf16-rounded P that
-// multiplies V.  The reference maximum m of a row is the largest of the first 32 scores of the
-// group's first tile of the unit and stays fixed: later scores may exceed it by up to 2^64
-// (fp32 accumulators and bf16 P have the exponent range for that); only when a tile exceeds
-// that bound is O_b rescaled (TMEM read-modify-write) and the tile redone.
+// multiplies V.  The reference maximum m of a row is the largest score of the group's first
+// half tile of the unit and stays fixed: later scores may exceed it by up to 2^64 (fp32
+// accumulators and bf16 P have the exponent range for that).  The row maximum of every half
+// tile is taken from the registers before any weight is written; only when it exceeds that
+// bound is the reference moved and O_b rescaled first (TMEM read-modify-write).
 //
 // Shared-memory tiles use the no-swizzle UMMA canonical layout: groups of 8 rows, inside a
 // group one 128-byte core matrix per 16-byte row chunk, inside a core matrix row r%8 at 16 r.
@@ -68,7 +75,9 @@ constexpr int kVGroup = 768;             // bytes of one 8-row group of a V tile
 constexpr int kTileV = (TK / 8) * kVGroup;  // 12 KB
 constexpr int kNV = 48;                  // columns of [V | 1 | 0...]
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kColS = 0, kColP = 256, kColO = 384;  // S_bi at kColS + 64 (2b+i), P_bi at kColP + 32 (2b+i), O_b at kColO + 48 b
+constexpr int NB = 3;                    // score / weight buffers per group
+constexpr uint32_t kColS = 0, kColO = 384;  // S_bi (and P_bi over its head) at kColS + 64 (NB b + i), O_b at kColO + 48 b
+static_assert(kColS + 64 * NB * 2 <= kColO && kColO + 2 * kNV <= kTmemCols, "TMEM columns");
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kHeadroom = 64.0f;       // log2 units a score may exceed the reference maximum
 constexpr uint32_t kSpinLimit = 1u << 18;  // polls of a wait before the CTA gives up
@@ -82,20 +91,20 @@ constexpr int kOffV = kOffK + NS * kTileK;
 constexpr int kOffX = kOffV + NS * kTileV;          // exchange between the groups: [34][128] floats
 constexpr int kOffIdx = kOffX + 34 * 128 * 4;        // per producer warp: K and V row indices of its tile, 16 bit
 constexpr int kOffBar = kOffIdx + kProducerWarps * 2 * TK * 2;
-constexpr int kOffAbort = kOffBar + 320;
+constexpr int kOffAbort = kOffBar + 384;
 constexpr int kSmemBytes = kOffAbort + 16;
 
 // barrier slots (8 bytes each) behind kOffBar
 enum {
     BAR_FULL = 0, BAR_EMPTY = NS, BAR_QEMPTY = 2 * NS,
-    BAR_SFULL = 2 * NS + NQ,      // [2b + i]
-    BAR_PREADY = BAR_SFULL + 4,   // [2b + i]
-    BAR_PFREE = BAR_SFULL + 8,    // [2b + i]
-    BAR_OFULL = BAR_SFULL + 12,   // [b]
-    BAR_XFULL = BAR_SFULL + 14, BAR_XEMPTY, BAR_DRAIN,
+    BAR_SFULL = 2 * NS + NQ,            // [NB b + i]
+    BAR_PREADY = BAR_SFULL + 2 * NB,    // [NB b + i]
+    BAR_PFREE = BAR_SFULL + 4 * NB,     // [NB b + i]
+    BAR_OFULL = BAR_SFULL + 6 * NB,     // [b]
+    BAR_XFULL = BAR_OFULL + 2, BAR_XEMPTY, BAR_DRAIN,
     BAR_COUNT = BAR_DRAIN + 4
 };
-static_assert(BAR_COUNT * 8 <= 320, "barrier area");
+static_assert(BAR_COUNT * 8 <= 384, "barrier area");
 
 // error codes OR-ed into the context's device error word
 enum { ERR_NORMALISE = 1, ERR_MMA = 2, ERR_DRAIN = 4, ERR_PRODUCER = 8 };
@@ -125,6 +134,19 @@ __device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const vola
     }
     return false;
 }
+// One poll of a phase parity: true if that phase has completed.
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
 // 16-byte copy global -> shared; src_bytes = 0 fills the destination with zeros instead.
 // Pool rows go through L1 (with skewed indices the hot rows then stop hammering a few L2 lines
 // from every SM at once); rows that are read once bypass it.
@@ -147,6 +169,7 @@ __device__ __forceinline__ void tc_commit(uint32_t bar)
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // D[tmem] (+)= A[smem] * B[smem]
 __device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc)
@@ -261,68 +284,6 @@ __device__ __forceinline__ uint32_t v_off(int r, int c) { return (uint32_t)((r >
 __device__ __forceinline__ int pos_of_col(int c, int e) { return 32 * c + 4 * (e & 7) + (e >> 3); }
 
 // ---- normalisation of one 128 x 64 score half tile by its group (thread = query row = TMEM lane) ----
-// `valid` counts the real positions of the half (1..64); column (c, e) of the half holds position
-// pos_of_col(c, e) of the half.
-// TAIL = false: all 64 columns are real positions; the two 32-column chunks are double-buffered
-// in registers so that the second tcgen05.ld is in flight during the arithmetic of the first.
-// TAIL = true (end of a history, at most once per unit and group): compact code, masked columns.
-
-// p = exp2(s c - m) as bf16 into P; returns the largest exponent argument of the row.  With
-// `first` the row's reference m is set from its first 32 scores (column 0 is the half's position 0,
-// always a real one).
-template <bool TAIL>
-__device__ __forceinline__ float softmax_tile(uint32_t tS, uint32_t tP, float sc, int valid, bool first, float& m_ref)
-{
-    float nm = -m_ref;
-    float mx = -CUDART_INF_F, mx2 = -CUDART_INF_F;
-    auto chunk = [&](const uint32_t (&cur)[32], int c) {
-        if (c == 0 && first) {
-            float t0 = -CUDART_INF_F, t1 = -CUDART_INF_F;
-#pragma unroll
-            for (int e = 0; e < 32; e += 4) {
-                float x[4];
-#pragma unroll
-                for (int i = 0; i < 4; ++i)
-                    x[i] = (TAIL && pos_of_col(0, e + i) >= valid) ? -CUDART_INF_F : __uint_as_float(cur[e + i]);
-                t0 = max3(t0, x[0], x[1]);
-                t1 = max3(t1, x[2], x[3]);
-            }
-            m_ref = fmaxf(t0, t1) * sc;
-            nm = -m_ref;
-        }
-        uint32_t p[16];
-#pragma unroll
-        for (int e = 0; e < 32; e += 2) {
-            float x0 = fmaf(__uint_as_float(cur[e]), sc, nm), x1 = fmaf(__uint_as_float(cur[e + 1]), sc, nm);
-            if (TAIL) {
-                if (pos_of_col(c, e) >= valid) x0 = -CUDART_INF_F;
-                if (pos_of_col(c, e + 1) >= valid) x1 = -CUDART_INF_F;
-            }
-            if (e & 2) mx = max3(mx, x0, x1);
-            else mx2 = max3(mx2, x0, x1);
-            p[e >> 1] = pack_bf16(ex2(x0), ex2(x1));
-        }
-        tmem_st16(tP + 16 * c, p);
-    };
-    if constexpr (TAIL) {
-#pragma unroll 1
-        for (int c = 0; c < 2; ++c) {
-            uint32_t cur[32];
-            tmem_ld32(tS + 32 * c, cur);
-            tmem_wait_ld32(cur);
-            chunk(cur, c);
-        }
-    } else {
-        uint32_t sa[32], sb[32];
-        tmem_ld32(tS, sa);
-        tmem_wait_ld32(sa);
-        tmem_ld32(tS + 32, sb);
-        chunk(sa, 0);
-        tmem_wait_ld32(sb);
-        chunk(sb, 1);
-    }
-    return fmaxf(mx, mx2);
-}
 
 // Multiplies this thread's row of O (32 columns and the row sum in column 32) by f.
 __device__ __noinline__ void rescale_row(uint32_t tO, float f)
@@ -337,41 +298,120 @@ __device__ __noinline__ void rescale_row(uint32_t tO, float f)
     tmem_st1(tO + 32, __float_as_uint(__uint_as_float(l) * f));
 }
 
-// p = silu(x) = x sigmoid(x) = h (1 + tanh(h)), h = x / 2, as bf16 into P   (sc = scale / 2)
-template <bool TAIL>
-__device__ __forceinline__ void silu_tile(uint32_t tS, uint32_t tP, float sc, int valid)
+// Multiplies the 32 weights (16 columns of bf16 pairs) this thread wrote for the first chunk of the current half
+// tile by f, a power of two: exact unless a weight drops below the smallest bf16.
+__device__ __noinline__ void rescale_weights(uint32_t tP, float f)
 {
-    auto chunk = [&](const uint32_t (&cur)[32], int c) {
-        uint32_t p[16];
-#pragma unroll
-        for (int e = 0; e < 32; e += 2) {
-            const float h0 = __uint_as_float(cur[e]) * sc, h1 = __uint_as_float(cur[e + 1]) * sc;
-            float w0 = fmaf(h0, tanh_fast(h0), h0), w1 = fmaf(h1, tanh_fast(h1), h1);
-            if (TAIL) {
-                if (pos_of_col(c, e) >= valid) w0 = 0.f;
-                if (pos_of_col(c, e + 1) >= valid) w1 = 0.f;
-            }
-            p[e >> 1] = pack_bf16(w0, w1);
-        }
-        tmem_st16(tP + 16 * c, p);
-    };
-    if constexpr (TAIL) {
-#pragma unroll 1
-        for (int c = 0; c < 2; ++c) {
-            uint32_t cur[32];
-            tmem_ld32(tS + 32 * c, cur);
-            tmem_wait_ld32(cur);
-            chunk(cur, c);
-        }
-    } else {
-        uint32_t sa[32], sb[32];
-        tmem_ld32(tS, sa);
-        tmem_wait_ld32(sa);
-        tmem_ld32(tS + 32, sb);
-        chunk(sa, 0);
-        tmem_wait_ld32(sb);
-        chunk(sb, 1);
+    for (int c = 0; c < 16; ++c) {
+        const uint32_t w = tmem_ld1(tP + c);
+        tmem_st1(tP + c, pack_bf16(__uint_as_float(w << 16) * f, __uint_as_float(w & 0xffff0000u) * f));
     }
+}
+
+// The weights of one 32-column chunk once more, from scores the caller has put into local memory (only used on
+// the rare path that moves a row's reference; kept out of line so that it costs the common path nothing).
+template <bool TAIL>
+__device__ __noinline__ void rewrite_weights(uint32_t tP, const uint32_t* cur, float sc, float nm, int valid, int c)
+{
+    uint32_t p[16];
+#pragma unroll
+    for (int e = 0; e < 32; e += 2) {
+        float x0 = fmaf(__uint_as_float(cur[e]), sc, nm), x1 = fmaf(__uint_as_float(cur[e + 1]), sc, nm);
+        if (TAIL) {
+            if (pos_of_col(c, e) >= valid) x0 = -CUDART_INF_F;
+            if (pos_of_col(c, e + 1) >= valid) x1 = -CUDART_INF_F;
+        }
+        p[e >> 1] = pack_bf16(ex2(x0), ex2(x1));
+    }
+    tmem_st16(tP, p);
+}
+
+// Softmax weights of one 32-column chunk (c = 0, 1) of a 128 x 64 score half tile: p = exp2(s c - m) as bf16
+// pairs written over the head of the scores (columns 0..31 of the buffer; chunk 1 of the scores, columns 32..63,
+// is in the registers or still to be read when chunk 0's weights land on columns 0..15, and chunk 1's weights
+// land on columns 16..31, whose scores have been consumed).  With `first` (chunk 0 of the group's first half
+// tile of a unit) the row's reference m is set from these 32 scores (column 0 is the half's position 0, always a
+// real one).  A chunk whose largest exponent argument leaves the headroom moves the reference up by a whole
+// number of octaves and is written again from the scores still in the registers; what O_b holds so far
+// (`have_o`; wait_prev() waits for the previous step's MMAs) and, for chunk 1, the weights of chunk 0 are
+// multiplied by the same power of two.  Returns false if that wait ran out.
+// `valid` counts the real positions of the half (1..64); column (c, e) of the half holds position
+// pos_of_col(c, e) of the half.  TAIL = true (end of a history, at most once per unit and group) masks the
+// columns beyond.
+template <bool TAIL, typename WaitPrev>
+__device__ __forceinline__ bool softmax_chunk(const uint32_t (&cur)[32], int c, uint32_t tS, uint32_t tO, float sc,
+                                              int valid, bool first, bool have_o, float& m_ref, WaitPrev&& wait_prev)
+{
+    if (c == 0 && first) {
+        float t0 = -CUDART_INF_F, t1 = -CUDART_INF_F;
+#pragma unroll
+        for (int e = 0; e < 32; e += 4) {
+            float x[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                x[i] = (TAIL && pos_of_col(0, e + i) >= valid) ? -CUDART_INF_F : __uint_as_float(cur[e + i]);
+            t0 = max3(t0, x[0], x[1]);
+            t1 = max3(t1, x[2], x[3]);
+        }
+        m_ref = fmaxf(t0, t1) * sc;
+    }
+    float nm = -m_ref;
+    float mx = -CUDART_INF_F, mx2 = -CUDART_INF_F;
+    uint32_t p[16];
+#pragma unroll
+    for (int e = 0; e < 32; e += 2) {
+        float x0 = fmaf(__uint_as_float(cur[e]), sc, nm), x1 = fmaf(__uint_as_float(cur[e + 1]), sc, nm);
+        if (TAIL) {
+            if (pos_of_col(c, e) >= valid) x0 = -CUDART_INF_F;
+            if (pos_of_col(c, e + 1) >= valid) x1 = -CUDART_INF_F;
+        }
+        if (e & 2) mx = max3(mx, x0, x1);
+        else mx2 = max3(mx2, x0, x1);
+        p[e >> 1] = pack_bf16(ex2(x0), ex2(x1));
+    }
+    tmem_st16(tS + 16 * c, p);
+    mx = fmaxf(mx, mx2);
+    if (__any_sync(0xffffffffu, mx > kHeadroom)) {
+        // rare: some row of this warp left the headroom and its weights just written may have overflowed.
+        // The chunk's scores are still in the registers: move the reference, bring what was accumulated and
+        // written before into the new scale, and write the chunk's weights again.
+        const float shift = mx > kHeadroom ? ceilf(mx) : 0.f;
+        const float f = ex2(-shift);
+        m_ref += shift;
+        nm = -m_ref;
+        tc_wait_st();
+        if (have_o) {
+            if (!wait_prev()) return false;
+            tc_fence_after();
+            rescale_row(tO, f);
+        }
+        if (c == 1) rescale_weights(tS, f);
+        uint32_t again[32];
+#pragma unroll
+        for (int e = 0; e < 32; ++e) again[e] = cur[e];
+        rewrite_weights<TAIL>(tS + 16 * c, again, sc, nm, valid, c);
+        tc_wait_st();
+    }
+    return true;
+}
+
+// p = silu(x) = x sigmoid(x) = h (1 + tanh(h)), h = x / 2, as bf16 pairs over the head of the scores like the
+// softmax weights   (sc = scale / 2)
+template <bool TAIL>
+__device__ __forceinline__ void silu_chunk(const uint32_t (&cur)[32], int c, uint32_t tS, float sc, int valid)
+{
+    uint32_t p[16];
+#pragma unroll
+    for (int e = 0; e < 32; e += 2) {
+        const float h0 = __uint_as_float(cur[e]) * sc, h1 = __uint_as_float(cur[e + 1]) * sc;
+        float w0 = fmaf(h0, tanh_fast(h0), h0), w1 = fmaf(h1, tanh_fast(h1), h1);
+        if (TAIL) {
+            if (pos_of_col(c, e) >= valid) w0 = 0.f;
+            if (pos_of_col(c, e + 1) >= valid) w1 = 0.f;
+        }
+        p[e >> 1] = pack_bf16(w0, w1);
+    }
+    tmem_st16(tS + 16 * c, p);
 }
 
 // The user-specific leading elements of one row (DUB = 2 d_user bytes), as the producers carry
@@ -538,7 +578,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
             mbar_init(bar(BAR_EMPTY + s), 2);  // one arrival per half
         }
         for (int q = 0; q < NQ; ++q) mbar_init(bar(BAR_QEMPTY + q), 2);  // both score issuers
-        for (int bi = 0; bi < 4; ++bi) {
+        for (int bi = 0; bi < 2 * NB; ++bi) {
             mbar_init(bar(BAR_SFULL + bi), 1);
             mbar_init(bar(BAR_PREADY + bi), kGroupThreads);
             mbar_init(bar(BAR_PFREE + bi), 1);
@@ -572,14 +612,15 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
         const int b = warp >> 2;                    // group = score buffer
         const int row = tid & (kGroupThreads - 1);  // query row inside the block = TMEM lane
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t tS0 = tmem + lane_base + kColS + 128u * b, tP0 = tmem + lane_base + kColP + 64u * b,
-                       tO = tmem + lane_base + kColO + (uint32_t)kNV * b;
+        const uint32_t tS0 = tmem + lane_base + kColS + 64u * NB * b, tO = tmem + lane_base + kColO + (uint32_t)kNV * b;
         const float sc = a.scale * (MODE == CKV_SOFTMAX ? kLog2e : 0.5f);
         float* xch = reinterpret_cast<float*>(smem + kOffX);
         int cnt = 0;    // half tiles this group has normalised
         int ocnt = 0;   // units in which this group had tiles
         int xcnt = 0;   // units exchanged between the groups
         bool ok = true;
+        uint32_t sa[32], sb[32];  // the two chunks of a half tile's scores
+        bool have_sa = false;     // sa is already receiving the first chunk of the coming step's scores
         Stream<true> sn;
         sn.init(a, n_mb, n_work);
         for (; sn.valid && ok; sn.next_unit()) {
@@ -603,43 +644,64 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
             for (int j = 0; j < u.n_tiles && ok; ++j) {
                 const int valid = (j == u.n_tiles - 1 ? u.last_valid : TK) - TH * b;  // real positions of this group's half
                 if (valid <= 0) continue;  // only the second half of a unit's last tile can be empty
-                const int i = cnt & 1;     // buffer pair of this step
-                const uint32_t tS = tS0 + 64u * i, tP = tP0 + 32u * i;
-                ok = mbar_wait(bar(BAR_SFULL + 2 * b + i), (cnt >> 1) & 1, abort_flag);
-                // P_bi is free once the weighted sum of two steps ago has been computed
-                if (ok && cnt >= 2) ok = mbar_wait(bar(BAR_PFREE + 2 * b + i), ((cnt >> 1) - 1) & 1, abort_flag);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-                tc_fence_after();
-                const bool tail = valid < TH;
-                if constexpr (MODE == CKV_SOFTMAX) {
-                    for (int attempt = 0; attempt < 2; ++attempt) {
-                        const bool first = mine == 0 && attempt == 0;
-                        const float mx = tail ? softmax_tile<true>(tS, tP, sc, valid, first, m_ref)
-                                              : softmax_tile<false>(tS, tP, sc, valid, first, m_ref);
-                        if (!__any_sync(0xffffffffu, mx > kHeadroom)) break;
-                        // some row of this warp left the headroom: move its reference, rescale what
-                        // O_b holds so far (once the previous step's MMAs have finished too) and redo
-                        const float shift = mx > kHeadroom ? mx : 0.f;
-                        const float f = ex2(-shift);
-                        m_ref += shift;
-                        if (mine > 0) {
-                            ok = mbar_wait(bar(BAR_PFREE + 2 * b + (i ^ 1)), ((cnt - 1) >> 1) & 1, abort_flag);
-                            ok = __all_sync(0xffffffffu, ok);
-                            if (!ok) break;
-                            tc_fence_after();
-                            rescale_row(tO, f);
-                        }
-                        tc_wait_st();
-                    }
+                const int i = cnt % NB;    // buffer of this step
+                const uint32_t tS = tS0 + 64u * i;
+                if (!have_sa) {
+                    // the scores arrive in a buffer whose previous weights the tensor core has finished reading
+                    ok = mbar_wait(bar(BAR_SFULL + NB * b + i), (cnt / NB) & 1, abort_flag);
+                    ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
-                } else {
-                    if (tail) silu_tile<true>(tS, tP, sc, valid);
-                    else silu_tile<false>(tS, tP, sc, valid);
+                    tc_fence_after();
                 }
+                // (softmax, only taken when a row leaves the headroom) the previous step's MMAs must have finished
+                // before O_b is rescaled
+                auto wait_prev = [&]() {
+                    bool w = mbar_wait(bar(BAR_PFREE + NB * b + (cnt - 1) % NB), ((cnt - 1) / NB) & 1, abort_flag);
+                    return __all_sync(0xffffffffu, w);
+                };
+                if (valid < TH) {
+                    // end of a history (at most once per unit and group): compact code, masked columns, chunk by chunk
+#pragma unroll 1
+                    for (int c = 0; c < 2 && ok; ++c) {
+                        tmem_ld32(tS + 32 * c, sa);
+                        tmem_wait_ld32(sa);
+                        if constexpr (MODE == CKV_SOFTMAX)
+                            ok = softmax_chunk<true>(sa, c, tS, tO, sc, valid, mine == 0, mine > 0, m_ref, wait_prev);
+                        else
+                            silu_chunk<true>(sa, c, tS, sc, valid);
+                    }
+                } else {
+                    // all 64 columns are real positions.  The two 32-column chunks are double-buffered in registers:
+                    // the second tcgen05.ld is in flight during the arithmetic of the first, and the first chunk of
+                    // this group's NEXT step, if its scores are there already, during the arithmetic of the second
+                    // (a TMEM load takes a few hundred clocks to return, as long as the arithmetic of a chunk).
+                    if (!have_sa) tmem_ld32(tS, sa);
+                    tmem_wait_ld32(sa);
+                    tmem_ld32(tS + 32, sb);
+                    if constexpr (MODE == CKV_SOFTMAX)
+                        ok = softmax_chunk<false>(sa, 0, tS, tO, sc, valid, mine == 0, mine > 0, m_ref, wait_prev);
+                    else
+                        silu_chunk<false>(sa, 0, tS, sc, valid);
+                    tmem_wait_ld32(sb);
+                    have_sa = false;
+                    if (ok && j + 1 < u.n_tiles && (j + 1 == u.n_tiles - 1 ? u.last_valid : TK) - TH * b >= TH) {
+                        const int i2 = (cnt + 1) % NB;
+                        if (__all_sync(0xffffffffu, mbar_test(bar(BAR_SFULL + NB * b + i2), ((cnt + 1) / NB) & 1))) {
+                            tc_fence_after();
+                            tmem_ld32(tS0 + 64u * i2, sa);
+                            have_sa = true;
+                        }
+                    }
+                    if constexpr (MODE == CKV_SOFTMAX) {
+                        if (ok) ok = softmax_chunk<false>(sb, 1, tS, tO, sc, valid, false, mine > 0, m_ref, wait_prev);
+                    } else {
+                        silu_chunk<false>(sb, 1, tS, sc, valid);
+                    }
+                }
+                if (!ok) break;
                 tc_wait_st();
                 tc_fence_before();
-                mbar_arrive(bar(BAR_PREADY + 2 * b + i));
+                mbar_arrive(bar(BAR_PREADY + NB * b + i));
                 ++cnt;
                 ++mine;
             }
@@ -726,6 +788,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                 }
             }
         }
+        tc_wait_ld();  // a load issued ahead may still be in flight when a wait has run out
         if (!ok) {
             *abort_flag = 1;
             if (lane == 0) atomicOr(err_flag, ERR_NORMALISE);
@@ -743,10 +806,10 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                 const int s = ss.g % NS;
                 const bool last = ss.j == ss.u.n_tiles - 1;
                 if ((last ? ss.u.last_valid : TK) > TH * b) {  // else: empty second half
-                    const int i = cnt & 1;
+                    const int i = cnt % NB;
                     ok = mbar_wait(bar(BAR_FULL + s), (ss.g / NS) & 1, abort_flag);
-                    // S_bi is free once the group has read the half tile of two steps ago
-                    if (ok && cnt >= 2) ok = mbar_wait(bar(BAR_PREADY + 2 * b + i), ((cnt >> 1) - 1) & 1, abort_flag);
+                    // S_bi is free once the weighted sum of NB steps ago, which read its weights out of it, has finished
+                    if (ok && cnt >= NB) ok = mbar_wait(bar(BAR_PFREE + NB * b + i), ((cnt / NB) - 1) & 1, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
                     ++cnt;
@@ -754,9 +817,9 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                                    k_addr = sbase + kOffK + s * kTileK + b * (TH / 8) * 512;
 #pragma unroll
                     for (int ks = 0; ks < D / 16; ++ks)
-                        umma_ss(tmem + kColS + 64u * (2 * b + i), smem_desc(q_addr + ks * 256, 128, 512),
+                        umma_ss(tmem + kColS + 64u * (NB * b + i), smem_desc(q_addr + ks * 256, 128, 512),
                                 smem_desc(k_addr + ks * 256, 128, 512), idesc_s, ks > 0 ? 1u : 0u);
-                    tc_commit(bar(BAR_SFULL + 2 * b + i));
+                    tc_commit(bar(BAR_SFULL + NB * b + i));
                 }
                 if (last) {
                     // This issuer no longer reads the unit's Q buffer.  It must have seen the unit's last
@@ -794,8 +857,8 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                     if (ok) mbar_arrive(bar(BAR_EMPTY + s));
                     continue;
                 }
-                const int i = cnt & 1;
-                ok = mbar_wait(bar(BAR_PREADY + 2 * b + i), (cnt >> 1) & 1, abort_flag);
+                const int i = cnt % NB;
+                ok = mbar_wait(bar(BAR_PREADY + NB * b + i), (cnt / NB) & 1, abort_flag);
                 if (ok) ok = mbar_wait(bar(BAR_FULL + s), (sp.g / NS) & 1, abort_flag);  // completed long ago: makes the V tile visible here
                 if (!ok) break;
                 ++cnt;
@@ -804,10 +867,10 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                 const bool last = sp.j == sp.u.n_tiles - 1 || (sp.j == sp.u.n_tiles - 2 && sp.u.last_valid <= TH * b);
 #pragma unroll
                 for (int kk = 0; kk < TH / 16; ++kk)  // sixteen positions per instruction
-                    umma_ts(tmem + kColO + (uint32_t)kNV * b, tmem + kColP + 32u * (2 * b + i) + 8 * kk,
+                    umma_ts(tmem + kColO + (uint32_t)kNV * b, tmem + kColS + 64u * (NB * b + i) + 8 * kk,
                             smem_desc(v_addr + kk * 2 * kVGroup, kVGroup, 128), idesc_pv, (sp.j > 0 || kk > 0) ? 1u : 0u);
                 tc_commit(bar(BAR_EMPTY + s));
-                tc_commit(bar(BAR_PFREE + 2 * b + i));
+                tc_commit(bar(BAR_PFREE + NB * b + i));
                 if (last) tc_commit(bar(BAR_OFULL + b));  // the group's last step of the unit
             }
             if (!ok) {

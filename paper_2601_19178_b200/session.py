@@ -42,6 +42,16 @@ class CollectiveKV:
         B.ckv_pool_load(self.ctx, pool_K, pool_V, m, dg)
         self.d_user = self.head_dim - dg
 
+    def pool_load_sides(self, pool_K: Optional[torch.Tensor], pool_V: Optional[torch.Tensor]):
+        """Sharing only keys or only values: None for the side that is not shared (its rows are then cached full
+        width and handed to the cache calls as that side's user part)."""
+        shared = [p for p in (pool_K, pool_V) if p is not None]
+        m = shared[0].shape[1] if shared else 1
+        dk = 0 if pool_K is None else pool_K.shape[2]
+        dv = 0 if pool_V is None else pool_V.shape[2]
+        B.ckv_pool_load_sides(self.ctx, pool_K, pool_V, m, dk, dv)
+        self.d_user = self.head_dim - max(dk, dv)
+
     def cache_put(self, user: int, idx_K, idx_V, user_K, user_V):
         B.ckv_cache_put(self.ctx, user, idx_K.shape[0], idx_K, idx_V, user_K, user_V, self.d_user)
 
@@ -56,6 +66,13 @@ class CollectiveKV:
         if out is None:
             out = torch.empty(queries.shape, dtype=self.out_dtype, device=queries.device)
         B.ckv_attend(self.ctx, users, q_off, queries, out)
+        return out
+
+    def attend_visible(self, users, q_off, vis, queries: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """attend with a visible length per query row (self-attention over the cached sequence)."""
+        if out is None:
+            out = torch.empty(queries.shape, dtype=self.out_dtype, device=queries.device)
+        B.ckv_attend_visible(self.ctx, users, q_off, vis, queries, out)
         return out
 
     def export_blob(self, users) -> torch.Tensor:

@@ -363,6 +363,42 @@ def test_host_buffers_go_through_the_same_path():
     assert np.array_equal(o_host.float().numpy().astype(np.float64), dev)
 
 
+@pytest.mark.parametrize("name,kw", [
+    ("cfg2", dict(n_users=96, hist_len=(100, 400))),                 # tcgen05 kernel, 4.9 MB of queries
+    ("cfg5", dict(n_users=5000, hist_len=(1, 90))),                  # warp-level tensor-core kernel, 20 MB
+    ("cfg4", dict(n_users=48, hist_len=(3000, 9000), n_queries=200, n_entries=2048)),  # split histories, merge per range
+])
+def test_large_host_buffers_are_pipelined_and_give_the_same_bits(name, kw):
+    """Host query / output buffers of a few MB and more: the request list is cut into ranges of users whose
+    upload, kernels and download run on internal streams.  Same bits as the device-buffer call, the caller's
+    stream is ordered behind everything, and a second call (plan cached) and a permuted request agree too."""
+    w = synth.scaled(synth.WORKLOADS[name], **kw)
+    d = synth.generate(w)
+    s = make_session(w, d)
+    q_dev = to_dev(d["queries"], w.dtype)
+    dev = s.attend(d["users"], d["q_off"], q_dev).clone()
+    assert s.stat("pipeline_ranges") == 1
+    q_host = torch.from_numpy(d["queries"].view(np.int16)).view(torch.bfloat16).pin_memory()
+    o_host = torch.full(q_host.shape, float("nan"), dtype=torch.bfloat16).pin_memory()
+    for _ in range(2):
+        o_host.fill_(float("nan"))
+        s.attend(d["users"], d["q_off"], q_host, o_host)
+        assert s.stat("pipeline_ranges") == 4
+        torch.cuda.current_stream().synchronize()          # only the caller's stream: it must cover the internal ones
+        assert torch.equal(o_host, dev.cpu())
+    # users in another order, queries moved along
+    perm = np.random.default_rng(1).permutation(w.n_users)
+    M = w.n_queries
+    rows = (perm[:, None] * M + np.arange(M)[None, :]).reshape(-1)
+    q_perm = q_host[torch.from_numpy(rows)].contiguous().pin_memory()
+    o_perm = torch.empty_like(q_perm).pin_memory()
+    s.attend(d["users"][perm], d["q_off"], q_perm, o_perm)
+    torch.cuda.current_stream().synchronize()
+    assert torch.equal(o_perm, dev.cpu()[torch.from_numpy(rows)])
+    assert s.stat("device_errors") == 0
+    s.close()
+
+
 @pytest.mark.parametrize("kernel,tol", [(1, 1e-5), (2, 2.0 ** -8)])
 def test_permuting_a_history_keeps_the_output(kernel, tol):
     """Attention does not depend on the order of the history.  The CUDA-core kernel keeps the

@@ -92,26 +92,35 @@ def _traffic(entry: str, family: int, users: int):
 
 
 def record_traffic(args):
-    """Reads `ncu -i <rep> --page raw --csv` output and stores the DRAM bytes of the captured attend launch(es)
-    in profiles/traffic.json under the entry name given.  Runs here, without a GPU."""
+    """Reads an ncu CSV (`ncu -i <rep> --page raw --csv`, one row per launch, or the log of
+    `ncu --metrics ...,dram__bytes_read.sum,dram__bytes_write.sum --csv`, one row per launch and metric) and stores
+    the DRAM bytes of the captured attend launch(es) in profiles/traffic.json under the entry name given.
+    Runs here, without a GPU."""
     import csv
     rows = list(csv.reader(open(args.record_traffic)))
     hdr = next(i for i, r in enumerate(rows) if "Kernel Name" in r)
     cols = rows[hdr]
     ci = {c: i for i, c in enumerate(cols)}
-    units = rows[hdr + 1]
+    scale = {"byte": 1.0, "kbyte": 1e3, "mbyte": 1e6, "gbyte": 1e9}
+    wanted = ("attend_", "fact_", "combine_kernel")
     total, names = 0.0, []
-    for r in rows[hdr + 2:]:
-        if len(r) != len(cols):
-            continue
-        name = r[ci["Kernel Name"]]
-        if not any(k in name for k in ("attend_", "fact_", "combine_kernel")):
-            continue
-        for m in ("dram__bytes_read.sum", "dram__bytes_write.sum"):
-            v = float(r[ci[m]].replace(",", ""))
-            u = units[ci[m]].lower()
-            total += v * {"byte": 1.0, "kbyte": 1e3, "mbyte": 1e6, "gbyte": 1e9}[u]
-        names.append(name.split("(")[0])
+    if "Metric Name" in ci:      # one row per (launch, metric)
+        for r in rows[hdr + 1:]:
+            if len(r) != len(cols) or not any(k in r[ci["Kernel Name"]] for k in wanted):
+                continue
+            if r[ci["Metric Name"]] in ("dram__bytes_read.sum", "dram__bytes_write.sum"):
+                total += float(r[ci["Metric Value"]].replace(",", "")) * scale[r[ci["Metric Unit"]].lower()]
+                name = r[ci["Kernel Name"]].split("(")[0]
+                if name not in names:
+                    names.append(name)
+    else:                        # one row per launch, units in the row below the header
+        units = rows[hdr + 1]
+        for r in rows[hdr + 2:]:
+            if len(r) != len(cols) or not any(k in r[ci["Kernel Name"]] for k in wanted):
+                continue
+            for m in ("dram__bytes_read.sum", "dram__bytes_write.sum"):
+                total += float(r[ci[m]].replace(",", "")) * scale[units[ci[m]].lower()]
+            names.append(r[ci["Kernel Name"]].split("(")[0])
     w = synth.WORKLOADS[args.workload if args.workload != "all" else HEADLINE]
     data = {}
     if os.path.exists(TRAFFIC_JSON):
@@ -437,8 +446,8 @@ class Measured:
         clocks = self.sampler.take() if self.sampler else None
         total_ms, job_pos, job_users = reduce_over_ranks(float(sum(step_ms)), self.positions, w.n_users, self.dist, "cuda")
         sus_total_ms, _, _ = reduce_over_ranks(float(sum(sus_ms)), self.positions, w.n_users, self.dist, "cuda")
-        e2e = self.e2e(False)
-        e2e_fresh = self.e2e(True)
+        e2e = None if args.no_e2e else self.e2e(False)
+        e2e_fresh = None if args.no_e2e else self.e2e(True)
         dev_err = s.stat("device_errors")
         if dev_err:
             raise SystemExit(f"{entry}: a kernel gave up on a bounded wait (device_errors = {dev_err})")
@@ -736,6 +745,7 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=0.0, help="host time of the CPU-oracle leg per workload")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-check", action="store_true", help="skip the sampled parity check")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer legs (profiling runs)")
     ap.add_argument("--route", action="store_true", help="time the prefill router (Sec. 4.3) instead of the attend step")
     ap.add_argument("--load-path", action="store_true",
                     help="time the decode-stage load path per batch size (Sec. 4.4) instead of the attend step")

@@ -116,8 +116,8 @@ CKV_API ckv_status ckv_pool_load(ckv_ctx* ctx, const void* pool_K, const void* p
  *   of the shared side(s) (head_dim if no side is shared, which is a classical KV cache).
  * The blob of ckv_cache_export / ckv_cache_import then has an empty index section for a side that is not shared
  * and head_dim elements per entry in that side's user section; ckv_cache_bytes counts what is stored.
- * Decode runs on the CUDA-core and the warp-level tensor-core kernels (option "kernel" 0, 1 or 2; the
- * warp-level kernel's TMA loader is not available).
+ * Decode runs on the CUDA-core, the warp-level tensor-core and the tcgen05 kernels (option "kernel" 0 to 3; the
+ * warp-level kernel's TMA loader and the pool-side factorisation are not available).
  * Errors: as ckv_pool_load; SHAPE also for unequal non-zero widths.
  */
 CKV_API ckv_status ckv_pool_load_sides(ckv_ctx* ctx, const void* pool_K, const void* pool_V, int32_t n_entries,
@@ -369,6 +369,9 @@ CKV_API ckv_status ckv_get_option(ckv_ctx* ctx, const char* name, int64_t* value
  * query waits for that attend to finish; CKV_ERR_STATE if nothing was timed).
  * "device_errors" (not tied to the last call): non-zero once a kernel of this context gave up
  * on one of its internal bounded waits -- its outputs are then invalid; synchronises the device.
+ * In the range-checked build of the library (build.py --bounds) bit 32 of it reports an index, row
+ * or shared-memory offset that a kernel found outside its bound (the access is then redirected, not
+ * performed).
  */
 CKV_API ckv_status ckv_last_stat(ckv_ctx* ctx, const char* name, int64_t* value);
 

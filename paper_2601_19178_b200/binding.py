@@ -12,7 +12,8 @@ from typing import Optional, Sequence
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libckv.so")
+# CKV_LIBRARY names another build of the same library (the range-checked libckv_bounds.so of build.py --bounds)
+LIB_PATH = os.environ.get("CKV_LIBRARY") or os.path.join(_HERE, "libckv.so")
 
 CKV_F32, CKV_BF16 = 0, 1
 CKV_SOFTMAX, CKV_SILU_OVER_L = 0, 1

@@ -1,6 +1,6 @@
 """Builds libckv.so (sm_100a) next to this file with nvcc.  No GPU is needed to build.
 
-    python paper_2601_19178_b200/build.py [--force] [--verbose]     (or: python __graft_entry__.py)
+    python paper_2601_19178_b200/build.py [--force] [--verbose] [--bounds]     (or: python __graft_entry__.py)
 """
 from __future__ import annotations
 
@@ -15,6 +15,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 OBJ = os.path.join(ROOT, "_build")
 LIB = os.path.join(PKG, "libckv.so")
+LIB_BOUNDS = os.path.join(PKG, "libckv_bounds.so")
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -34,19 +35,23 @@ def _newest(paths) -> float:
     return max(os.path.getmtime(p) for p in paths)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, bounds: bool = False) -> str:
+    """bounds=True builds libckv_bounds.so instead: the same library with every index, row and shared-memory
+    offset the kernels compute range-checked into the context's error word (-DCKV_BOUNDS)."""
     sources = sorted(glob.glob(os.path.join(CSRC, "*.cu")))
     headers = glob.glob(os.path.join(CSRC, "*.h")) + glob.glob(os.path.join(CSRC, "*.cuh")) + \
         glob.glob(os.path.join(ROOT, "include", "*.h"))
     if not sources:
         raise RuntimeError("no CUDA sources under " + CSRC)
-    os.makedirs(OBJ, exist_ok=True)
+    obj_dir = OBJ + ("_bounds" if bounds else "")
+    lib = LIB_BOUNDS if bounds else LIB
+    os.makedirs(obj_dir, exist_ok=True)
     nvcc = _nvcc()
-    extra = ["-Xptxas", "-v"] if verbose else []
+    extra = (["-Xptxas", "-v"] if verbose else []) + (["-DCKV_BOUNDS"] if bounds else [])
     hdr_time = _newest(headers) if headers else 0.0
 
     def compile_one(src: str) -> str:
-        obj = os.path.join(OBJ, os.path.basename(src)[:-3] + ".o")
+        obj = os.path.join(obj_dir, os.path.basename(src)[:-3] + ".o")
         if force or not os.path.exists(obj) or os.path.getmtime(obj) < max(os.path.getmtime(src), hdr_time):
             cmd = [nvcc, *NVCC_FLAGS, *extra, "-c", src, "-o", obj]
             r = subprocess.run(cmd, capture_output=True, text=True)
@@ -58,16 +63,16 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
     with concurrent.futures.ThreadPoolExecutor(max_workers=min(8, len(sources))) as ex:
         objs = list(ex.map(compile_one, sources))
-    if force or not os.path.exists(LIB) or os.path.getmtime(LIB) < _newest(objs):
-        tmp = LIB + f".tmp{os.getpid()}"
+    if force or not os.path.exists(lib) or os.path.getmtime(lib) < _newest(objs):
+        tmp = lib + f".tmp{os.getpid()}"
         cmd = [nvcc, "-shared", "-o", tmp, *objs, "-Xlinker", "--exclude-libs,ALL"]
         r = subprocess.run(cmd, capture_output=True, text=True)
         if r.returncode != 0:
             sys.stderr.write(r.stdout + r.stderr)
             raise RuntimeError("link failed")
-        os.replace(tmp, LIB)
-    return LIB
+        os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv, bounds="--bounds" in sys.argv))

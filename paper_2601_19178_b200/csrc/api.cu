@@ -497,10 +497,10 @@ ckv_status build_plan(ckv_ctx* ctx, Plan& pl, int32_t n, const int64_t* users, c
     pl.max_L = max_L;
     pl.n_req = n;
     const bool can_mma = ctx->has_mma;
-    // visible lengths and sides that are not shared are served by the CUDA-core and the warp-level tensor-core
-    // kernels only
+    // visible lengths are served by the CUDA-core and the warp-level tensor-core kernels only; sides that are not
+    // shared by those and the tcgen05 kernel
     const bool plain = !with_vis && !ctx->full_k && !ctx->full_v;
-    const bool can_umma = ctx->has_umma && plain;
+    const bool can_umma = ctx->has_umma && !with_vis;
     // tcgen05 from three 16-query blocks on, else the warp-level tensor-core kernel (faster than the CUDA-core
     // kernel from a single query on); the CUDA-core kernel serves what neither supports
     // One query per user: the pool-side factorisation trades the row gathers for two tables per (user, group) in
@@ -1337,6 +1337,10 @@ ckv_status attend_impl(ckv_ctx* ctx, int32_t n, const int64_t* users, const int3
     a.out_dtype = ctx->cfg.out_dtype;
     a.mode = ctx->cfg.mode;
     a.scale = ctx->scale;
+    a.arena_units = ctx->cap_units;
+    a.q_rows = Q;
+    a.part_rows = pl->family == 4 ? 0 : pl->part_rows;
+    a.err = ctx->d_err;
     ctx->ev_valid = false;
 
     if (n_ranges == 1) {
@@ -1791,6 +1795,10 @@ extern "C" ckv_status ckv_attend_static(ckv_ctx* ctx, int32_t n, const int64_t* 
     a.out_dtype = ctx->cfg.out_dtype;
     a.mode = ctx->cfg.mode;
     a.scale = ctx->scale;
+    a.arena_units = ctx->cap_units;
+    a.q_rows = Q;
+    a.part_rows = part_rows;
+    a.err = ctx->d_err;
     if (n_items > 0) {
         if (family == 2)
             CK(launch_attend_mma(D, max_M, a, nullptr, ctx->d_err, s));

@@ -69,6 +69,11 @@ struct AttendArgs {
     int32_t out_dtype;     // ckv_dtype
     int32_t mode;          // ckv_mode
     float scale;
+    // What the range-checked build (-DCKV_BOUNDS) compares against; unused otherwise.
+    int64_t arena_units;   // units the arena arrays hold
+    int64_t q_rows;        // rows of `queries` and `out`
+    int64_t part_rows;     // rows of `partials`
+    int* err;              // device error word (the context's)
 };
 
 // ---- kernels_pack.cu

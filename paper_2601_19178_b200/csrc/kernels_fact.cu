@@ -226,7 +226,7 @@ __global__ void __launch_bounds__(kMainThreads, 1)
             ix[b] = 0;
             x[b] = make_uint4(0, 0, 0, 0);
             if (i < pr.L) {
-                ix[b] = load_index<IDX16>(idx, pr.unit0 + i);
+                ix[b] = load_index<IDX16>(idx, CKV_CLAMP(pr.unit0 + i, a.arena_units, a.err));
                 x[b] = load_user(u, pr.unit0 + i, d_user);
             }
         }
@@ -267,7 +267,7 @@ __global__ void __launch_bounds__(kMainThreads, 1)
             for (int b = 0; b < B; ++b) {
                 const int i = i0 + b * kMainThreads;
                 if (i < L) {
-                    const float sv = dot_user(qu, x[b], Ts[ix[b]]) * sc;
+                    const float sv = dot_user(qu, x[b], Ts[CKV_CLAMP(ix[b], m, a.err)]) * sc;
                     Sb[i] = sv;
                     mx = fmaxf(mx, sv);
                 }
@@ -295,7 +295,7 @@ __global__ void __launch_bounds__(kMainThreads, 1)
                         const float h = Sb[i];  // silu(x) = x sigmoid(x) = h (1 + tanh(h)), h = x / 2
                         pw = fmaf(h, tanh_fast(h), h);
                     }
-                    atomicAdd(&Ws[ix[b]], pw);
+                    atomicAdd(&Ws[CKV_CLAMP(ix[b], m, a.err)], pw);
                     axpy_user(ou, pw, x[b]);
                 }
             }

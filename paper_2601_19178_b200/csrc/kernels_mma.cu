@@ -161,6 +161,8 @@ __global__ void __launch_bounds__(128, MmaCfg<D, MT, TMA>::MIN_BLOCKS)
         const int r_lo = row0 + 16 * mt + g, r_hi = r_lo + 8;
         const uint16_t* q_lo = Q + ((int64_t)(rq.q0 + r_lo) * G + grp) * D;
         const uint16_t* q_hi = Q + ((int64_t)(rq.q0 + r_hi) * G + grp) * D;
+        if (r_lo < rq.M) (void)CKV_CLAMP((int64_t)(rq.q0 + r_lo), a.q_rows, err_flag);
+        if (r_hi < rq.M) (void)CKV_CLAMP((int64_t)(rq.q0 + r_hi), a.q_rows, err_flag);
 #pragma unroll
         for (int ks = 0; ks < KS; ++ks) {
             const int c = 16 * ks + 2 * t;
@@ -212,6 +214,7 @@ __global__ void __launch_bounds__(128, MmaCfg<D, MT, TMA>::MIN_BLOCKS)
     const char* pK = reinterpret_cast<const char*>(a.cv.poolK) + (int64_t)grp * a.cv.n_entries * ROWB + cc * 16;
     const char* pV = reinterpret_cast<const char*>(a.cv.poolV) + (int64_t)grp * a.cv.n_entries * ROWB + cc * 16;
     const int64_t unit0 = rq.base + (int64_t)grp * rq.Lpad + it.begin + lane;  // this lane's position of step 0
+    (void)CKV_CLAMP(unit0 - lane + ((it.len + 31) & ~31) - 1, a.arena_units, err_flag);  // the chunk's last (padded) unit
     const uint16_t* uK = reinterpret_cast<const uint16_t*>(a.cv.userK);
     const uint16_t* uV = reinterpret_cast<const uint16_t*>(a.cv.userV);
     const int end = VAR ? min(it.begin + it.len, lim_max) : it.begin + it.len;  // nothing behind the last visible position is touched
@@ -286,7 +289,11 @@ __global__ void __launch_bounds__(128, MmaCfg<D, MT, TMA>::MIN_BLOCKS)
             for (int i = 0; i < 32 / RPI; ++i) {
                 const int r = i * RPI + cr;
                 const uint32_t off = r * ROWB + ((cc ^ swz<D>(r)) << 4);
-                const int rk = __shfl_sync(0xffffffffu, idx_k, r), rv = __shfl_sync(0xffffffffu, idx_v, r);
+                // (range-checked build: a pool index below n_entries, or, for a side that is not shared, an offset
+                // inside the user's padded history; the ring slot inside this block's shared memory)
+                const int rk = CKV_CLAMP(__shfl_sync(0xffffffffu, idx_k, r), full_k ? rq.Lpad - it.begin : a.cv.n_entries, err_flag),
+                          rv = CKV_CLAMP(__shfl_sync(0xffffffffu, idx_v, r), full_v ? rq.Lpad - it.begin : a.cv.n_entries, err_flag);
+                (void)CKV_CLAMP((int)(vt + off - smem_u32(smem_raw)), C::SMEM - 15, err_flag);
                 cp_async16(kt + off, pK + (int64_t)rk * ROWB);
                 cp_async16(vt + off, pV + (int64_t)rv * ROWB);
             }
@@ -527,7 +534,7 @@ __global__ void __launch_bounds__(128, MmaCfg<D, MT, TMA>::MIN_BLOCKS)
                             make_float2(x, y);
                 }
             } else {
-                float* pr = a.partials + ((int64_t)(it.part_row + r) * G + grp) * (D + 2);
+                float* pr = a.partials + (CKV_CLAMP((int64_t)(it.part_row + r), a.part_rows, err_flag) * G + grp) * (D + 2);
                 if (t == 0) {
                     pr[0] = m_run[mt][h];
                     pr[1] = l;

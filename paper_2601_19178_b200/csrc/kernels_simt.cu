@@ -15,6 +15,7 @@
 #include <math_constants.h>
 
 #include "ckv_internal.h"
+#include "ptx_helpers.cuh"
 
 namespace ckv {
 namespace {
@@ -117,7 +118,7 @@ __global__ void __launch_bounds__(kWarps * 32, QB == 1 ? 5 : 1) attend_simt_kern
 #pragma unroll
         for (int r = 0; r < QB; ++r) {
             if (qb + r < rq.M) {
-                const int64_t row = ((int64_t)(rq.q0 + qb + r) * G + g) * D;
+                const int64_t row = (CKV_CLAMP((int64_t)(rq.q0 + qb + r), a.q_rows, a.err) * G + g) * D;
                 unpack16<BF16>(ldg16((const char*)a.queries + (row + ch * EPL) * ES), q[r]);
 #pragma unroll
                 for (int e = 0; e < EPL; ++e) q[r][e] *= qscale;
@@ -155,7 +156,8 @@ __global__ void __launch_bounds__(kWarps * 32, QB == 1 ? 5 : 1) attend_simt_kern
 #pragma unroll
             for (int l = 0; l < NL; ++l) {
                 const int my_p = p0 + l * 32 + lane;
-                const int64_t my_unit = unit0 + ((l * 32 + lane < PPW * UNR && my_p < end) ? my_p : it.begin);
+                const int64_t my_unit = CKV_CLAMP(unit0 + ((l * 32 + lane < PPW * UNR && my_p < end) ? my_p : it.begin),
+                                                  a.arena_units, a.err);
                 my_ik[l] = full_k ? 0 : load_idx(cv.idxK, my_unit, idx_bytes);
                 my_iv[l] = full_v ? 0 : load_idx(cv.idxV, my_unit, idx_bytes);
                 my_uk[l] = my_uv[l] = make_uint2(0, 0);
@@ -173,12 +175,13 @@ __global__ void __launch_bounds__(kWarps * 32, QB == 1 ? 5 : 1) attend_simt_kern
 #pragma unroll
             for (int j = 0; j < UNR; ++j) {
                 pos[j] = p0 + j * PPW + sub;
-                unit[j] = unit0 + (pos[j] < end ? pos[j] : it.begin);
+                unit[j] = CKV_CLAMP(unit0 + (pos[j] < end ? pos[j] : it.begin), a.arena_units, a.err);
             }
 #pragma unroll
             for (int j = 0; j < UNR; ++j) {
                 const int src = (j * PPW) % 32 + sub;
-                const int ik = __shfl_sync(0xffffffffu, my_ik[(j * PPW) / 32], src), iv = __shfl_sync(0xffffffffu, my_iv[(j * PPW) / 32], src);
+                const int ik = CKV_CLAMP(__shfl_sync(0xffffffffu, my_ik[(j * PPW) / 32], src), cv.n_entries, a.err),
+                          iv = CKV_CLAMP(__shfl_sync(0xffffffffu, my_iv[(j * PPW) / 32], src), cv.n_entries, a.err);
                 kraw[j] = full_k ? ldg16(rowsK + unit[j] * (D * ES)) : ldg16(poolK + (int64_t)ik * (D * ES));
                 vraw[j] = full_v ? ldg16(rowsV + unit[j] * (D * ES)) : ldg16(poolV + (int64_t)iv * (D * ES));
             }
@@ -335,9 +338,9 @@ __global__ void __launch_bounds__(kWarps * 32, QB == 1 ? 5 : 1) attend_simt_kern
                 float res;
                 if constexpr (MODE == CKV_SOFTMAX) res = lt > 0.f ? o / lt : 0.f;
                 else res = rq.L > 0 ? o / (float)rq.L : 0.f;
-                store_out(a.out, ((int64_t)(rq.q0 + qb + r) * G + g) * D + c, res, a.out_dtype);
+                store_out(a.out, (CKV_CLAMP((int64_t)(rq.q0 + qb + r), a.q_rows, a.err) * G + g) * D + c, res, a.out_dtype);
             } else {
-                float* pr = a.partials + ((int64_t)(it.part_row + qb + r) * G + g) * (D + 2);
+                float* pr = a.partials + (CKV_CLAMP((int64_t)(it.part_row + qb + r), a.part_rows, a.err) * G + g) * (D + 2);
                 if (c == 0) {
                     pr[0] = mt;
                     pr[1] = lt;
@@ -363,7 +366,7 @@ __global__ void __launch_bounds__(128) combine_kernel(const AttendArgs a, const 
         if constexpr (MODE == CKV_SOFTMAX) {
             float mt = -CUDART_INF_F;
             for (int k = 0; k < rq.n_chunks; ++k)
-                mt = fmaxf(mt, a.partials[((int64_t)(rq.part0 + k * rq.M + r) * G + g) * W]);
+                mt = fmaxf(mt, a.partials[(CKV_CLAMP((int64_t)(rq.part0 + k * rq.M + r), a.part_rows, a.err) * G + g) * W]);
             const float ms = mt == -CUDART_INF_F ? 0.f : mt;
             float lt = 0.f, o = 0.f;
             for (int k = 0; k < rq.n_chunks; ++k) {
@@ -379,7 +382,7 @@ __global__ void __launch_bounds__(128) combine_kernel(const AttendArgs a, const 
                 o += a.partials[((int64_t)(rq.part0 + k * rq.M + r) * G + g) * W + 2 + c];
             res = rq.L > 0 ? o / (float)rq.L : 0.f;
         }
-        store_out(a.out, ((int64_t)(rq.q0 + r) * G + g) * D + c, res, a.out_dtype);
+        store_out(a.out, (CKV_CLAMP((int64_t)(rq.q0 + r), a.q_rows, a.err) * G + g) * D + c, res, a.out_dtype);
     }
 }
 

@@ -9,7 +9,8 @@
 //   warps 10-11 issue the weighted-sum MMAs of group 0 and 1 (one thread each)
 //   warps 12-15 producers, one tile each in turn: gather pool rows into shared memory with
 //               16-byte cp.async, patch the user-specific leading elements (Eq. K), publish the
-//               tile; the owner of a unit's first tile also stages Q
+//               tile; the owner of a unit's first tile also stages Q.  (A side that is not shared --
+//               sharing only keys or only values -- is copied from the user's full-width rows instead.)
 //
 // A tile (128 positions) is split into two halves of 64 positions; half b belongs to group b,
 // which has three score buffers in TMEM and uses them in turn; the weights of a half tile are
@@ -626,6 +627,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
         for (; sn.valid && ok; sn.next_unit()) {
             const Unit& u = sn.u;
             const int r = u.row0 + row;
+            if (r < u.wk.M) (void)CKV_CLAMP((int64_t)(u.wk.q0 + r), a.q_rows, err_flag);
             const int64_t out_base = ((int64_t)(u.wk.q0 + r) * G + u.grp) * D;
             if (u.n_tiles == 0) {  // empty history: zero output rows
                 if (b == 0 && r < u.wk.M && u.wk.part_row < 0) {
@@ -779,7 +781,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                                                       o[4 * q4 + 3] * inv);
                         }
                     } else {
-                        float* pr = a.partials + ((int64_t)(u.wk.part_row + r) * G + u.grp) * (D + 2);
+                        float* pr = a.partials + (CKV_CLAMP((int64_t)(u.wk.part_row + r), a.part_rows, err_flag) * G + u.grp) * (D + 2);
                         pr[0] = m_ref;
                         pr[1] = l;
 #pragma unroll
@@ -897,6 +899,11 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
         const char* poolK0 = reinterpret_cast<const char*>(a.cv.poolK) + chunk * 16;
         const char* poolV0 = reinterpret_cast<const char*>(a.cv.poolV) + chunk * 16;
         const uint16_t* Q = reinterpret_cast<const uint16_t*>(a.queries);
+        // A side that is not shared (sharing only keys or only values): its rows are the tile's own units in the
+        // arena, the position inside the tile stands in for the pool index, and nothing is patched.
+        const bool full_k = a.cv.full_k != 0, full_v = a.cv.full_v != 0;
+        const char* rowsK0 = reinterpret_cast<const char*>(a.cv.userK) + chunk * 16;
+        const char* rowsV0 = reinterpret_cast<const char*>(a.cv.userV) + chunk * 16;
         uint16_t* sidxK = reinterpret_cast<uint16_t*>(smem + kOffIdx) + pw * 2 * TK;  // this warp's row indices of a tile
         uint16_t* sidxV = sidxK + TK;
         Stream<false> st;
@@ -910,18 +917,21 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
             if (!st.valid) return;
             const int pos0 = st.u.wk.begin + st.j * TK;
             const int64_t unit0 = st.u.wk.base + (int64_t)st.u.grp * st.u.wk.Lpad + pos0;  // arena unit of the tile's position 0
+            (void)CKV_CLAMP(unit0, a.arena_units, err_flag);
             const int valid = st.j == st.u.n_tiles - 1 ? st.u.last_valid : TK;
             xk = xv = make_uint2(0, 0);
             if (pos0 + 4 * lane < st.u.wk.Lpad) {  // the arena is padded to 32 positions per user
-                xk = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const uint16_t*>(a.cv.idxK) + unit0 + 4 * lane));
-                xv = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const uint16_t*>(a.cv.idxV) + unit0 + 4 * lane));
+                if (!full_k) xk = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const uint16_t*>(a.cv.idxK) + unit0 + 4 * lane));
+                if (!full_v) xv = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const uint16_t*>(a.cv.idxV) + unit0 + 4 * lane));
             }
+            if (full_k) xk = make_uint2((4 * lane) | ((4 * lane + 1) << 16), (4 * lane + 2) | ((4 * lane + 3) << 16));
+            if (full_v) xv = make_uint2((4 * lane) | ((4 * lane + 1) << 16), (4 * lane + 2) | ((4 * lane + 3) << 16));
             if constexpr (DUB > 0) {
 #pragma unroll
                 for (int rb = 0; rb < 4; ++rb) {
                     if (32 * rb + patch_pos < valid) {
-                        uk_n[rb].load(reinterpret_cast<const char*>(a.cv.userK) + (unit0 + 32 * rb + patch_pos) * DUB);
-                        uv_n[rb].load(reinterpret_cast<const char*>(a.cv.userV) + (unit0 + 32 * rb + patch_pos) * DUB);
+                        if (!full_k) uk_n[rb].load(reinterpret_cast<const char*>(a.cv.userK) + (unit0 + 32 * rb + patch_pos) * DUB);
+                        if (!full_v) uv_n[rb].load(reinterpret_cast<const char*>(a.cv.userV) + (unit0 + 32 * rb + patch_pos) * DUB);
                     }
                 }
             }
@@ -958,16 +968,20 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                     cp_async16_once(qdst + 512 * rr, in ? qsrc + (int64_t)8 * rr * G * D : Q, in ? 16u : 0u);
                 }
             }
-            const char* pk = poolK0 + st.u.grp * pool_stride;
-            const char* pv = poolV0 + st.u.grp * pool_stride;
+            const int64_t tile_unit0 = st.u.wk.base + (int64_t)st.u.grp * st.u.wk.Lpad + st.u.wk.begin + st.j * TK;
+            const char* pk = full_k ? rowsK0 + tile_unit0 * (D * 2) : poolK0 + st.u.grp * pool_stride;
+            const char* pv = full_v ? rowsV0 + tile_unit0 * (D * 2) : poolV0 + st.u.grp * pool_stride;
             const uint32_t kdst = sbase + kOffK + s * kTileK + kv_lane, vdst = sbase + kOffV + s * kTileV + kv_lane;
             const int valid = st.j == st.u.n_tiles - 1 ? st.u.last_valid : TK;
 #pragma unroll 2
             for (int it = 0; it < 16; ++it) {  // rb = it / 4, i = it % 4: position 32 rb + 4 q + i -> tile row 32 rb + 8 i + q
                 const int pos = 32 * (it >> 2) + 4 * q + (it & 3);
                 const uint32_t nb = pos < valid ? 16u : 0u;  // rows of positions beyond the history are zero
-                cp_async16(kdst + 512 * it, pk + (size_t)sidxK[pos] * (D * 2), nb);
-                cp_async16(vdst + kVGroup * it, pv + (size_t)sidxV[pos] * (D * 2), nb);
+                // (range-checked build: pool indices below n_entries, destinations inside the stage)
+                (void)CKV_CLAMP((int)(512 * it + kv_lane), kTileK - 15, err_flag);
+                (void)CKV_CLAMP((int)(kVGroup * it + kv_lane), kTileV - 15, err_flag);
+                cp_async16(kdst + 512 * it, pk + (size_t)CKV_CLAMP((int)sidxK[pos], full_k ? TK : a.cv.n_entries, err_flag) * (D * 2), nb);
+                cp_async16(vdst + kVGroup * it, pv + (size_t)CKV_CLAMP((int)sidxV[pos], full_v ? TK : a.cv.n_entries, err_flag) * (D * 2), nb);
             }
             cp_async_commit();
             // what this warp's next tile needs travels while the copies land
@@ -979,8 +993,8 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
 #pragma unroll
                 for (int rb = 0; rb < 4; ++rb) {
                     if (32 * rb + patch_pos < valid) {  // zero rows beyond the history stay zero
-                        uk[rb].store(smem + kOffK + s * kTileK + k_off(32 * rb + lane, 0));
-                        uv[rb].store(smem + kOffV + s * kTileV + v_off(32 * rb + lane, 0));
+                        if (!full_k) uk[rb].store(smem + kOffK + s * kTileK + k_off(32 * rb + lane, 0));
+                        if (!full_v) uv[rb].store(smem + kOffV + s * kTileV + v_off(32 * rb + lane, 0));
                     }
                 }
             }
@@ -1025,7 +1039,7 @@ cudaError_t launch_attend_umma(int max_M, const AttendArgs& a, int n_sms, int* e
         return cudaGetLastError();
     };
     const bool sm = a.mode == CKV_SOFTMAX;
-    switch (a.cv.d_user) {
+    switch (a.cv.full_k && a.cv.full_v ? 0 : a.cv.d_user) {  // the user-specific width of the shared side(s)
         case 0: return sm ? go(attend_umma_kernel<CKV_SOFTMAX, 0>) : go(attend_umma_kernel<CKV_SILU_OVER_L, 0>);
         case 1: return sm ? go(attend_umma_kernel<CKV_SOFTMAX, 2>) : go(attend_umma_kernel<CKV_SILU_OVER_L, 2>);
         case 2: return sm ? go(attend_umma_kernel<CKV_SOFTMAX, 4>) : go(attend_umma_kernel<CKV_SILU_OVER_L, 4>);

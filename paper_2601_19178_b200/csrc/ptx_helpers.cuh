@@ -40,4 +40,23 @@ __device__ __forceinline__ float tanh_fast(float x)
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
+// Range checks of the debug build (-DCKV_BOUNDS, the stand-in for a memory checker where none can run): every
+// index taken from the compressed cache, every unit, query / output / partial row and shared-memory offset a
+// kernel computes is compared with its bound; a violation ORs kErrBounds into the context's error word
+// (ckv_last_stat "device_errors") and the access is redirected to element 0 -- nothing traps, nothing faults.
+// In the normal build CKV_CLAMP is the identity and costs nothing.
+constexpr int kErrBounds = 32;
+#ifdef CKV_BOUNDS
+template <typename T, typename B>
+__device__ __forceinline__ T ckv_clamp(T v, B bound, int* err)
+{
+    if (v >= (T)0 && v < (T)bound) return v;
+    if (err) atomicOr(err, kErrBounds);
+    return (T)0;
+}
+#define CKV_CLAMP(v, bound, err) ::ckv::ckv_clamp((v), (bound), (err))
+#else
+#define CKV_CLAMP(v, bound, err) (v)
+#endif
+
 }  // namespace ckv

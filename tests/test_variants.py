@@ -79,6 +79,23 @@ def test_one_sided_sharing_matches_oracle(name, share, kernel, loader):
     s.close()
 
 
+@pytest.mark.parametrize("name,kw", [("cfg2", dict(n_users=5, hist_len=(1, 900))),
+                                     ("cfg3", dict(n_users=3, hist_len=(100, 1400)))])
+@pytest.mark.parametrize("share", [(True, False), (False, True), (False, False)], ids=["K_only", "V_only", "none"])
+def test_one_sided_sharing_on_the_tcgen05_kernel(name, kw, share):
+    """Many queries per user: the library's choice for these shapes is the tcgen05 kernel, whose producers copy a
+    side that is not shared from the user's full-width rows."""
+    w = synth.scaled(W[name], **kw)
+    d = synth.generate(w)
+    s, uk, uv = side_session(w, d, *share, split_len=512)
+    out = s.attend(d["users"], d["q_off"], to_dev(d["queries"], w.dtype))
+    torch.cuda.synchronize()
+    assert s.stat("kernel") == 3 and s.stat("device_errors") == 0
+    assert_close(out.float().cpu().numpy().astype(np.float64), oracle_sides(w, d, *share, uk, uv), w.dtype,
+                 f"{name} share={share}")
+    s.close()
+
+
 def test_one_sided_sharing_survives_export_import_and_append():
     w = synth.scaled(W["cfg5"], n_users=8, hist_len=(5, 300))
     d = synth.generate(w)

@@ -203,11 +203,14 @@ def _oracle_rate(w, data, n_users: int, n_threads: int = 0):
 
 
 def _oracle_sample(w, data, seconds: float):
-    """The oracle on a bounded sample of the workload: a short probe sizes the sample to about `seconds`."""
-    probe_users = max(1, min(w.n_users, 8))
-    _, probe_dt, _, _, _ = _oracle_rate(w, data, probe_users)
-    n_users = int(max(probe_users, min(w.n_users, seconds * probe_users / max(probe_dt, 1e-9))))
-    rate, dt, cores, n_u, pos = _oracle_rate(w, data, n_users)
+    """The oracle on a bounded sample of the workload: the first users of it, as many as take about `seconds`
+    (a short run sizes the next one; the last run is the one reported; the whole workload if that is quicker)."""
+    n_users = max(1, min(w.n_users, 64))
+    while True:
+        rate, dt, cores, n_u, pos = _oracle_rate(w, data, n_users)
+        if n_u >= w.n_users or dt >= 0.5 * seconds:
+            break
+        n_users = int(min(w.n_users, max(2 * n_u, n_u * seconds / max(dt, 1e-3))))
     return {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": f"first {n_u} of {w.n_users} users ({pos} positions), {dt:.1f} s"}
 

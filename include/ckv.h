@@ -190,8 +190,9 @@ CKV_API ckv_status ckv_attend(ckv_ctx* ctx, int32_t n, const int64_t* users, con
  *               (values are clamped to [0, L_k]; causal self-attention over the whole history is
  *               vis = 1, 2, ..., L_k for the user's L_k queries; vis = 0 gives a zero row).
  * CKV_SOFTMAX normalises over the attended positions; CKV_SILU_OVER_L sums over them and still divides by the
- * user's history length L_k.  Everything else as ckv_attend; the CUDA-core and the warp-level tensor-core
- * kernels serve this call (option "kernel" 0, 1 or 2).
+ * user's history length L_k.  Everything else as ckv_attend; every gathering kernel serves this call (option
+ * "kernel" 0 to 3; not the pool-side factorisation).  The tcgen05 kernel skips what lies behind the largest limit
+ * of each block of 128 queries of a user, so causal self-attention costs about half of full attention.
  * Errors: as ckv_attend; INVALID_ARG also for vis == NULL with queries present.
  */
 CKV_API ckv_status ckv_attend_visible(ckv_ctx* ctx, int32_t n, const int64_t* users, const int32_t* q_off,

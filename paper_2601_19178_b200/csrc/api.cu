@@ -148,7 +148,7 @@ struct Plan {
     Item* d_items = nullptr;
     int32_t* d_split = nullptr;
     Work* d_works = nullptr;
-    int32_t n_items = 0, n_split = 0, split_items = 0, max_M = 0, max_L = 0, n_req = 0, family = 1;
+    int32_t n_items = 0, n_split = 0, split_items = 0, max_M = 0, max_L = 0, n_req = 0, family = 1, n_vblocks = 0;
     int64_t part_rows = 0;
     uint64_t last_use = 0;
 };
@@ -197,7 +197,7 @@ struct ckv_ctx {
     UserTable users;
     uint64_t generation = 1;
     // scratch
-    DevBuf stage_q, stage_out, stage_vis, partials;
+    DevBuf stage_q, stage_out, stage_vis, vmax, partials;
     int* d_flag = nullptr;
     Plan plans[kMaxPlans];
     uint64_t tick = 0;
@@ -497,10 +497,10 @@ ckv_status build_plan(ckv_ctx* ctx, Plan& pl, int32_t n, const int64_t* users, c
     pl.max_L = max_L;
     pl.n_req = n;
     const bool can_mma = ctx->has_mma;
-    // visible lengths are served by the CUDA-core and the warp-level tensor-core kernels only; sides that are not
-    // shared by those and the tcgen05 kernel
+    // visible lengths and sides that are not shared are served by every gathering kernel, not by the pool-side
+    // factorisation
     const bool plain = !with_vis && !ctx->full_k && !ctx->full_v;
-    const bool can_umma = ctx->has_umma && !with_vis;
+    const bool can_umma = ctx->has_umma;
     // tcgen05 from three 16-query blocks on, else the warp-level tensor-core kernel (faster than the CUDA-core
     // kernel from a single query on); the CUDA-core kernel serves what neither supports
     // One query per user: the pool-side factorisation trades the row gathers for two tables per (user, group) in
@@ -598,10 +598,17 @@ ckv_status build_plan(ckv_ctx* ctx, Plan& pl, int32_t n, const int64_t* users, c
     for (size_t i = 0; i < items.size(); ++i) h_items[i] = items[order[i]];
     if (b_split) std::memcpy(h + o_split, split.data(), b_split);
     Work* h_works = (Work*)(h + o_work);
+    // where each request's blocks of 128 queries start in the table of largest visible lengths
+    std::vector<int32_t> vb_off(n_works ? reqs.size() : 0);
+    pl.n_vblocks = 0;
+    for (size_t k = 0; k < vb_off.size(); ++k) {
+        vb_off[k] = pl.n_vblocks;
+        pl.n_vblocks += (reqs[k].M + 127) / 128;
+    }
     for (size_t i = 0; i < n_works; ++i) {
         const Item& it = h_items[i];
         const Req& r = reqs[it.req];
-        h_works[i] = Work{r.base, r.L, r.Lpad, r.q0, r.M, it.begin, it.len, it.part_row, {0, 0, 0}};
+        h_works[i] = Work{r.base, r.L, r.Lpad, r.q0, r.M, it.begin, it.len, it.part_row, {vb_off[it.req], 0, 0}};
     }
     pl.d_reqs = (Req*)pl.dev.p;
     pl.d_items = (Item*)((char*)pl.dev.p + o_item);
@@ -800,7 +807,7 @@ ckv_status ckv_destroy(ckv_ctx* ctx)
     DeviceGuard dg(ctx->cfg.device);
     drop_plans(ctx);
     void* bufs[] = {ctx->pool,    ctx->a_idxK,     ctx->a_idxV,      ctx->a_userK,   ctx->a_userV,
-                    ctx->d_flag,  ctx->stage_q.p,  ctx->stage_out.p, ctx->partials.p, ctx->stage_vis.p};
+                    ctx->d_flag,  ctx->stage_q.p,  ctx->stage_out.p, ctx->partials.p, ctx->stage_vis.p, ctx->vmax.p};
     for (void* b : bufs)
         if (b) cudaFree(b);
     for (auto& e : ctx->ev)
@@ -1332,6 +1339,7 @@ ckv_status attend_impl(ckv_ctx* ctx, int32_t n, const int64_t* users, const int3
     a.n_items = pl->n_items;
     a.queries = d_q;
     a.vis = d_vis;
+    a.vmax = nullptr;
     a.out = d_out;
     a.partials = (float*)ctx->partials.p;
     a.out_dtype = ctx->cfg.out_dtype;
@@ -1342,6 +1350,17 @@ ckv_status attend_impl(ckv_ctx* ctx, int32_t n, const int64_t* users, const int3
     a.part_rows = pl->family == 4 ? 0 : pl->part_rows;
     a.err = ctx->d_err;
     ctx->ev_valid = false;
+    if (d_vis && pl->family == 3 && pl->n_items > 0) {
+        // the tcgen05 kernel's roles skip what lies behind every row's limit: the largest limit per block of queries
+        CK(grow(ctx->vmax, (size_t)std::max(pl->n_vblocks, 1) * sizeof(int32_t), &ctx->st_allocs));
+        cudaStream_t vs = n_ranges > 1 ? ctx->pipe_stream[0] : s;
+        if (n_ranges > 1) CK(cudaStreamWaitEvent(vs, ctx->pipe_plan, 0));
+        CK(launch_vis_block_max(a, (int32_t*)ctx->vmax.p, vs));
+        a.vmax = (const int32_t*)ctx->vmax.p;
+        if (n_ranges > 1) {  // every range's kernels need the whole table
+            CK(cudaEventRecord(ctx->pipe_plan, vs));
+        }
+    }
 
     if (n_ranges == 1) {
         const bool time_it = ctx->opt_time != 0;
@@ -1790,6 +1809,7 @@ extern "C" ckv_status ckv_attend_static(ckv_ctx* ctx, int32_t n, const int64_t* 
     a.n_items = n_items;
     a.queries = queries;
     a.vis = nullptr;
+    a.vmax = nullptr;
     a.out = out;
     a.partials = (float*)(base + kOffPartials);  // every entry that is read was written by this call
     a.out_dtype = ctx->cfg.out_dtype;

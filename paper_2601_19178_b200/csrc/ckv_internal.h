@@ -35,7 +35,7 @@ struct Work {
     int32_t L, Lpad;   // Req::L, Req::Lpad
     int32_t q0, M;     // Req::q0, Req::M
     int32_t begin, len, part_row;  // Item::begin, Item::len, Item::part_row
-    int32_t pad[3];
+    int32_t pad[3];    // [0]: with visible lengths, where the request's query blocks start in AttendArgs::vmax
 };
 
 // Everything a kernel needs to find the compressed cache and the pool.
@@ -64,6 +64,7 @@ struct AttendArgs {
     int32_t n_items;
     const void* queries;   // [Q][G][D]
     const int32_t* vis;    // null, or per query row the number of leading history positions it attends [Q]
+    const int32_t* vmax;   // tcgen05 family with visible lengths: largest limit per (request, block of 128 queries)
     void* out;             // [Q][G][D]
     float* partials;       // [part rows][G][D + 2]  (m, l, acc[D])
     int32_t out_dtype;     // ckv_dtype
@@ -149,5 +150,7 @@ bool umma_supported(int dtype, int head_dim, int d_user, int idx_bytes);
 // err_flag: device int, OR-ed with a non-zero code if a bounded wait inside the kernel ran out.
 // Persistent: one CTA per SM (n_sms of them at most).
 cudaError_t launch_attend_umma(int max_M, const AttendArgs& a, int n_sms, int* err_flag, cudaStream_t s);
+// Fills vmax (one int per request and block of 128 queries, at Work::pad[0] + block) from a.vis; a.works as for the attend.
+cudaError_t launch_vis_block_max(const AttendArgs& a, int32_t* vmax, cudaStream_t s);
 
 }  // namespace ckv

@@ -339,18 +339,20 @@ __device__ __noinline__ void rewrite_weights(uint32_t tP, const uint32_t* cur, f
 // `valid` counts the real positions of the half (1..64); column (c, e) of the half holds position
 // pos_of_col(c, e) of the half.  TAIL = true (end of a history, at most once per unit and group) masks the
 // columns beyond.
-template <bool TAIL, typename WaitPrev>
+// VIS (visible lengths): `valid` differs from thread to thread and may be zero or negative (the row sees nothing
+// of this half tile); a row's reference is then set by the first chunk in which it sees a position.
+template <bool TAIL, bool VIS, typename WaitPrev>
 __device__ __forceinline__ bool softmax_chunk(const uint32_t (&cur)[32], int c, uint32_t tS, uint32_t tO, float sc,
                                               int valid, bool first, bool have_o, float& m_ref, WaitPrev&& wait_prev)
 {
-    if (c == 0 && first) {
+    if ((c == 0 && first) || (VIS && m_ref == -CUDART_INF_F)) {
         float t0 = -CUDART_INF_F, t1 = -CUDART_INF_F;
 #pragma unroll
         for (int e = 0; e < 32; e += 4) {
             float x[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i)
-                x[i] = (TAIL && pos_of_col(0, e + i) >= valid) ? -CUDART_INF_F : __uint_as_float(cur[e + i]);
+                x[i] = (TAIL && pos_of_col(c, e + i) >= valid) ? -CUDART_INF_F : __uint_as_float(cur[e + i]);
             t0 = max3(t0, x[0], x[1]);
             t1 = max3(t1, x[2], x[3]);
         }
@@ -472,6 +474,7 @@ __device__ __forceinline__ Work load_work(const Work* p)
 template <bool KEEP_EMPTY>
 struct Stream {
     const Work* works;
+    const int32_t* vmax;         // visible lengths: per (request, query block) the largest limit of its rows, else null
     uint32_t n_mb, n_groups;
     uint32_t w, n_work;          // the host keeps n_work + gridDim.x below 2^32
     uint32_t item, grp, mb;      // coordinates of unit w
@@ -507,8 +510,11 @@ struct Stream {
             uint32_t ni = item, ng = grp, nm = mb;
             step(ni, ng, nm);
             if (wn < n_work) nxt = load_work(works + ni);
-            u.n_tiles = u.row0 < u.wk.M ? (u.wk.len + TK - 1) / TK : -1;
-            u.last_valid = u.wk.len - (u.n_tiles - 1) * TK;
+            // with visible lengths nothing behind the block's largest limit is touched (every role decodes the same)
+            int len = u.wk.len;
+            if (vmax != nullptr && u.row0 < u.wk.M) len = min(len, max(__ldg(vmax + u.wk.pad[0] + mb) - u.wk.begin, 0));
+            u.n_tiles = u.row0 < u.wk.M ? (len + TK - 1) / TK : -1;
+            u.last_valid = len - (u.n_tiles - 1) * TK;
             if (u.n_tiles > 0 || (KEEP_EMPTY && u.n_tiles == 0)) {
                 valid = true;
                 j = 0;
@@ -529,6 +535,7 @@ struct Stream {
     __device__ __forceinline__ void init(const AttendArgs& a, int n_mb_, int64_t n_work_)
     {
         works = a.works;
+        vmax = a.vmax;
         n_mb = (uint32_t)n_mb_;
         n_groups = (uint32_t)a.cv.n_groups;
         n_work = (uint32_t)n_work_;
@@ -560,7 +567,8 @@ struct Stream {
     }
 };
 
-template <int MODE, int DUB>
+// VIS: visible lengths (a.vis, a.vmax); the plain instantiations carry none of that code.
+template <int MODE, int DUB, bool VIS>
 __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendArgs a, int n_mb, int64_t n_work, int* err_flag)
 {
     extern __shared__ __align__(1024) unsigned char smem[];
@@ -629,9 +637,13 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
             const int r = u.row0 + row;
             if (r < u.wk.M) (void)CKV_CLAMP((int64_t)(u.wk.q0 + r), a.q_rows, err_flag);
             const int64_t out_base = ((int64_t)(u.wk.q0 + r) * G + u.grp) * D;
-            if (u.n_tiles == 0) {  // empty history: zero output rows
-                if (b == 0 && r < u.wk.M && u.wk.part_row < 0) {
-                    if (a.out_dtype == CKV_BF16) {
+            if (u.n_tiles == 0) {  // empty history, or a chunk behind every row's visible length: zero rows
+                if (b == 0 && r < u.wk.M) {
+                    if (u.wk.part_row >= 0) {  // (only with visible lengths) an empty partial result
+                        float* pr = a.partials + (CKV_CLAMP((int64_t)(u.wk.part_row + r), a.part_rows, err_flag) * G + u.grp) * (D + 2);
+                        pr[0] = -CUDART_INF_F;
+                        for (int e = 1; e < D + 2; ++e) pr[e] = 0.f;
+                    } else if (a.out_dtype == CKV_BF16) {
                         uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(a.out) + out_base);
                         for (int q4 = 0; q4 < 4; ++q4) dst[q4] = make_uint4(0, 0, 0, 0);
                     } else {
@@ -641,6 +653,9 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                 }
                 continue;
             }
+            // positions this thread's query row attends: [0, lim); rows beyond the user's queries take none
+            int lim = u.wk.L;
+            if constexpr (VIS) lim = r < u.wk.M ? min(max(__ldg(a.vis + u.wk.q0 + r), 0), u.wk.L) : 0;
             float m_ref = -CUDART_INF_F;
             int mine = 0;  // half tiles of this unit normalised by this group
             for (int j = 0; j < u.n_tiles && ok; ++j) {
@@ -661,16 +676,24 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                     bool w = mbar_wait(bar(BAR_PFREE + NB * b + (cnt - 1) % NB), ((cnt - 1) / NB) & 1, abort_flag);
                     return __all_sync(0xffffffffu, w);
                 };
-                if (valid < TH) {
-                    // end of a history (at most once per unit and group): compact code, masked columns, chunk by chunk
+                // real (and, with visible lengths, attended) positions of this thread's row in the half tile
+                int valid_r = valid;
+                bool tail = valid < TH;
+                if constexpr (VIS) {
+                    valid_r = min(valid, lim - (u.wk.begin + j * TK + TH * b));
+                    tail = __any_sync(0xffffffffu, valid_r < TH);
+                }
+                if (tail) {
+                    // end of a history (at most once per unit and group) or of some row's visible positions: compact
+                    // code, masked columns, chunk by chunk
 #pragma unroll 1
                     for (int c = 0; c < 2 && ok; ++c) {
                         tmem_ld32(tS + 32 * c, sa);
                         tmem_wait_ld32(sa);
                         if constexpr (MODE == CKV_SOFTMAX)
-                            ok = softmax_chunk<true>(sa, c, tS, tO, sc, valid, mine == 0, mine > 0, m_ref, wait_prev);
+                            ok = softmax_chunk<true, VIS>(sa, c, tS, tO, sc, valid_r, mine == 0, mine > 0, m_ref, wait_prev);
                         else
-                            silu_chunk<true>(sa, c, tS, sc, valid);
+                            silu_chunk<true>(sa, c, tS, sc, valid_r);
                     }
                 } else {
                     // all 64 columns are real positions.  The two 32-column chunks are double-buffered in registers:
@@ -681,12 +704,12 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                     tmem_wait_ld32(sa);
                     tmem_ld32(tS + 32, sb);
                     if constexpr (MODE == CKV_SOFTMAX)
-                        ok = softmax_chunk<false>(sa, 0, tS, tO, sc, valid, mine == 0, mine > 0, m_ref, wait_prev);
+                        ok = softmax_chunk<false, VIS>(sa, 0, tS, tO, sc, valid, mine == 0, mine > 0, m_ref, wait_prev);
                     else
                         silu_chunk<false>(sa, 0, tS, sc, valid);
                     tmem_wait_ld32(sb);
                     have_sa = false;
-                    if (ok && j + 1 < u.n_tiles && (j + 1 == u.n_tiles - 1 ? u.last_valid : TK) - TH * b >= TH) {
+                    if (ok && !VIS && j + 1 < u.n_tiles && (j + 1 == u.n_tiles - 1 ? u.last_valid : TK) - TH * b >= TH) {
                         const int i2 = (cnt + 1) % NB;
                         if (__all_sync(0xffffffffu, mbar_test(bar(BAR_SFULL + NB * b + i2), ((cnt + 1) / NB) & 1))) {
                             tc_fence_after();
@@ -695,7 +718,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                         }
                     }
                     if constexpr (MODE == CKV_SOFTMAX) {
-                        if (ok) ok = softmax_chunk<false>(sb, 1, tS, tO, sc, valid, false, mine > 0, m_ref, wait_prev);
+                        if (ok) ok = softmax_chunk<false, VIS>(sb, 1, tS, tO, sc, valid, false, mine > 0, m_ref, wait_prev);
                     } else {
                         silu_chunk<false>(sb, 1, tS, sc, valid);
                     }
@@ -1025,6 +1048,35 @@ bool umma_supported(int dtype, int head_dim, int d_user, int idx_bytes)
            (d_user == 0 || d_user == 1 || d_user == 2 || d_user == 4 || d_user == 8);
 }
 
+namespace {
+
+// vmax[off(req) + mb] = largest visible length (clamped to the history) among the rows of query block mb of a
+// request; off(req) is pad[0] of the request's work records.  One block per work item (its request's blocks are
+// written once per item: the same values).
+__global__ void vis_block_max_kernel(const Work* __restrict__ works, int n_items, const int32_t* __restrict__ vis,
+                                     int32_t* __restrict__ vmax)
+{
+    const Work w = works[blockIdx.x];
+    const int n_mb = (w.M + 127) / 128;
+    for (int mb = threadIdx.x >> 5; mb < n_mb; mb += blockDim.x >> 5) {
+        int m = 0;
+        for (int r = 128 * mb + (threadIdx.x & 31); r < min(w.M, 128 * mb + 128); r += 32)
+            m = max(m, min(max(__ldg(vis + w.q0 + r), 0), w.L));
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
+        if ((threadIdx.x & 31) == 0) vmax[w.pad[0] + mb] = m;
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_vis_block_max(const AttendArgs& a, int32_t* vmax, cudaStream_t s)
+{
+    if (a.n_items == 0) return cudaSuccess;
+    vis_block_max_kernel<<<a.n_items, 128, 0, s>>>(a.works, a.n_items, a.vis, vmax);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_attend_umma(int max_M, const AttendArgs& a, int n_sms, int* err_flag, cudaStream_t s)
 {
     if (a.n_items == 0) return cudaSuccess;
@@ -1038,14 +1090,19 @@ cudaError_t launch_attend_umma(int max_M, const AttendArgs& a, int n_sms, int* e
         kernel<<<grid, kThreads, kSmemBytes, s>>>(a, n_mb, n_work, err_flag);
         return cudaGetLastError();
     };
-    const bool sm = a.mode == CKV_SOFTMAX;
+    const bool sm = a.mode == CKV_SOFTMAX, vis = a.vis != nullptr;
+    if (vis && a.vmax == nullptr) return cudaErrorInvalidValue;
+#define CKV_UMMA_GO(DUB)                                                                                          \
+    (vis ? (sm ? go(attend_umma_kernel<CKV_SOFTMAX, DUB, true>) : go(attend_umma_kernel<CKV_SILU_OVER_L, DUB, true>)) \
+         : (sm ? go(attend_umma_kernel<CKV_SOFTMAX, DUB, false>) : go(attend_umma_kernel<CKV_SILU_OVER_L, DUB, false>)))
     switch (a.cv.full_k && a.cv.full_v ? 0 : a.cv.d_user) {  // the user-specific width of the shared side(s)
-        case 0: return sm ? go(attend_umma_kernel<CKV_SOFTMAX, 0>) : go(attend_umma_kernel<CKV_SILU_OVER_L, 0>);
-        case 1: return sm ? go(attend_umma_kernel<CKV_SOFTMAX, 2>) : go(attend_umma_kernel<CKV_SILU_OVER_L, 2>);
-        case 2: return sm ? go(attend_umma_kernel<CKV_SOFTMAX, 4>) : go(attend_umma_kernel<CKV_SILU_OVER_L, 4>);
-        case 4: return sm ? go(attend_umma_kernel<CKV_SOFTMAX, 8>) : go(attend_umma_kernel<CKV_SILU_OVER_L, 8>);
-        case 8: return sm ? go(attend_umma_kernel<CKV_SOFTMAX, 16>) : go(attend_umma_kernel<CKV_SILU_OVER_L, 16>);
+        case 0: return CKV_UMMA_GO(0);
+        case 1: return CKV_UMMA_GO(2);
+        case 2: return CKV_UMMA_GO(4);
+        case 4: return CKV_UMMA_GO(8);
+        case 8: return CKV_UMMA_GO(16);
     }
+#undef CKV_UMMA_GO
     return cudaErrorInvalidValue;
 }
 

@@ -143,6 +143,8 @@ def _vis_for(w, d, kind, rng):
         M = w.n_queries
         if kind == "causal_tail":          # the last M positions as queries of a causal self-attention
             out.append(np.clip(np.arange(L - M + 1, L + 1), 0, L))
+        elif kind == "causal_spread":      # M queries spread over the history, each seeing what lies before it
+            out.append(np.clip(np.linspace(0, L, M).astype(np.int64), 0, L))
         elif kind == "random":
             out.append(rng.integers(0, L + 1, size=M))
         else:                              # everything visible: must equal ckv_attend
@@ -178,6 +180,36 @@ def test_visible_lengths_match_oracle(name, kind, kernel, loader):
     want = O.attend_variants(w.dtype, w.mode, w.default_scale, w.head_dim, d["pool_K"], d["pool_V"], d["hist_off"],
                              d["idx_K"], d["idx_V"], d["user_K"], d["user_V"], d["q_off"], d["queries"], vis=vis)
     assert_close(out.float().cpu().numpy().astype(np.float64), want, w.dtype, f"{name} {kind}")
+    s.close()
+
+
+@pytest.mark.parametrize("name,kw", [
+    ("cfg2", dict(n_users=4, hist_len=(1, 1500), n_queries=100)),      # softmax, one block of queries, tails
+    ("cfg2", dict(n_users=3, hist_len=(300, 2500), n_queries=300)),    # three blocks of queries per user
+    ("cfg3", dict(n_users=3, hist_len=(100, 1700), n_queries=128)),    # SiLU
+])
+@pytest.mark.parametrize("kind", ["causal_tail", "causal_spread", "random", "all"])
+@pytest.mark.parametrize("split_len", [0, 512])
+def test_visible_lengths_on_the_tcgen05_kernel(name, kw, kind, split_len):
+    """Many queries per user (self-attention over the cached sequence is the case with as many queries as
+    positions): the tcgen05 kernel masks per query row and skips the tiles behind the largest limit of a block of
+    128 queries; with split histories a chunk that no row of the block sees yields an empty partial result."""
+    from ckv_testlib import make_session
+    w = synth.scaled(W[name], **kw)
+    d = synth.generate(w)
+    vis = _vis_for(w, d, kind, np.random.default_rng(5))
+    s = make_session(w, d, split_len=split_len)
+    q = to_dev(d["queries"], w.dtype)
+    out = s.attend_visible(d["users"], d["q_off"], vis, q)
+    torch.cuda.synchronize()
+    assert s.stat("kernel") == 3 and s.stat("device_errors") == 0
+    if split_len:
+        assert s.stat("split_items") > 0
+    want = O.attend_variants(w.dtype, w.mode, w.default_scale, w.head_dim, d["pool_K"], d["pool_V"], d["hist_off"],
+                             d["idx_K"], d["idx_V"], d["user_K"], d["user_V"], d["q_off"], d["queries"], vis=vis)
+    assert_close(out.float().cpu().numpy().astype(np.float64), want, w.dtype, f"{name} {kind}")
+    if kind == "all":
+        assert torch.equal(out, s.attend(d["users"], d["q_off"], q))
     s.close()
 
 

@@ -63,7 +63,7 @@ namespace {
 constexpr int D = 32;
 constexpr int TK = 128;                  // positions per tile (one shared-memory stage)
 constexpr int TH = 64;                   // positions per half tile = one MMA / normalisation step of a group
-constexpr int NS = 6;                    // K/V stages
+constexpr int NS = 9;                    // K/V stages
 constexpr int NQ = 3;                    // Q buffers
 constexpr int kGroupThreads = 128;       // one normalisation group
 constexpr int kMmaWarp = 8;              // warps 8, 9 issue S = Q K^T of group 0, 1; warp 8 owns the TMEM allocation
@@ -471,10 +471,10 @@ __device__ __forceinline__ Work load_work(const Work* p)
 // (item, group, query block) = (w / n_mb / G, w / n_mb % G, w % n_mb); the coordinates are
 // stepped with carries instead of divided out each time.
 // KEEP_EMPTY: also stop at units with an empty history (the role that writes their zero rows).
-template <bool KEEP_EMPTY>
+template <bool KEEP_EMPTY, bool VIS>
 struct Stream {
     const Work* works;
-    const int32_t* vmax;         // visible lengths: per (request, query block) the largest limit of its rows, else null
+    const int32_t* vmax;         // VIS: per (request, query block) the largest visible length of its rows
     uint32_t n_mb, n_groups;
     uint32_t w, n_work;          // the host keeps n_work + gridDim.x below 2^32
     uint32_t item, grp, mb;      // coordinates of unit w
@@ -512,7 +512,9 @@ struct Stream {
             if (wn < n_work) nxt = load_work(works + ni);
             // with visible lengths nothing behind the block's largest limit is touched (every role decodes the same)
             int len = u.wk.len;
-            if (vmax != nullptr && u.row0 < u.wk.M) len = min(len, max(__ldg(vmax + u.wk.pad[0] + mb) - u.wk.begin, 0));
+            if constexpr (VIS) {
+                if (u.row0 < u.wk.M) len = min(len, max(__ldg(vmax + u.wk.pad[0] + mb) - u.wk.begin, 0));
+            }
             u.n_tiles = u.row0 < u.wk.M ? (len + TK - 1) / TK : -1;
             u.last_valid = len - (u.n_tiles - 1) * TK;
             if (u.n_tiles > 0 || (KEEP_EMPTY && u.n_tiles == 0)) {
@@ -535,7 +537,7 @@ struct Stream {
     __device__ __forceinline__ void init(const AttendArgs& a, int n_mb_, int64_t n_work_)
     {
         works = a.works;
-        vmax = a.vmax;
+        if constexpr (VIS) vmax = a.vmax;
         n_mb = (uint32_t)n_mb_;
         n_groups = (uint32_t)a.cv.n_groups;
         n_work = (uint32_t)n_work_;
@@ -630,7 +632,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
         bool ok = true;
         uint32_t sa[32], sb[32];  // the two chunks of a half tile's scores
         bool have_sa = false;     // sa is already receiving the first chunk of the coming step's scores
-        Stream<true> sn;
+        Stream<true, VIS> sn;
         sn.init(a, n_mb, n_work);
         for (; sn.valid && ok; sn.next_unit()) {
             const Unit& u = sn.u;
@@ -823,7 +825,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
         if (lane == 0) {
             const int b = warp - kMmaWarp;
             constexpr uint32_t idesc_s = make_idesc(128, TH, false);
-            Stream<false> ss;
+            Stream<false, VIS> ss;
             ss.init(a, n_mb, n_work);
             int cnt = 0;  // half tiles issued
             bool ok = true;
@@ -870,7 +872,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
         if (lane == 0) {
             const int b = warp - kPvWarp0;
             constexpr uint32_t idesc_pv = make_idesc(128, MODE == CKV_SOFTMAX ? kNV : D, true);
-            Stream<false> sp;
+            Stream<false, VIS> sp;
             sp.init(a, n_mb, n_work);
             int cnt = 0;
             bool ok = true;
@@ -929,7 +931,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
         const char* rowsV0 = reinterpret_cast<const char*>(a.cv.userV) + chunk * 16;
         uint16_t* sidxK = reinterpret_cast<uint16_t*>(smem + kOffIdx) + pw * 2 * TK;  // this warp's row indices of a tile
         uint16_t* sidxV = sidxK + TK;
-        Stream<false> st;
+        Stream<false, VIS> st;
         st.init(a, n_mb, n_work);
         for (int i = 0; i < pw && st.valid; ++i) st.advance();
         bool ok = true;

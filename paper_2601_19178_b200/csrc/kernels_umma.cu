@@ -2,51 +2,41 @@
 //
 // Persistent: one CTA per SM walks a static round-robin share of the work units, where a unit
 // is (work item = history chunk of one user, group, block of up to 128 queries).  The history
-// chunk is processed in tiles of 128 positions.  Roles (warp-specialised, 16 warps):
-//   warps 0-3   normalisation group 0: thread i owns query row i = TMEM lane i, first half of every tile
-//   warps 4-7   normalisation group 1: the same rows, second half of every tile
-//   warps 8-9   issue the score MMAs of group 0 and 1 (one thread each); warp 8 owns the TMEM allocation
-//   warps 10-11 issue the weighted-sum MMAs of group 0 and 1 (one thread each)
-//   warps 12-15 producers, one tile each in turn: gather pool rows into shared memory with
+// chunk is processed in tiles of 128 positions, each split into two halves of 64 positions.
+// Roles (warp-specialised, 20 warps):
+//   warps 0-11  three normalisation groups of four warps: thread i of a group owns query row i = TMEM lane i
+//   warps 12-14 one issuing thread per group: the score MMAs and the weighted-sum MMAs of that group's halves;
+//               warp 12 owns the TMEM allocation
+//   warps 15-19 producers, one tile each in turn: gather pool rows into shared memory with
 //               16-byte cp.async, patch the user-specific leading elements (Eq. K), publish the
 //               tile; the owner of a unit's first tile also stages Q.  (A side that is not shared --
 //               sharing only keys or only values -- is copied from the user's full-width rows instead.)
 //
-// A tile (128 positions) is split into two halves of 64 positions; half b belongs to group b,
-// which has three score buffers in TMEM and uses them in turn; the weights of a half tile are
-// written over the head of the scores they were computed from (32 columns of bf16 pairs over
-// 64 columns of fp32):
+// The halves of the CTA's tile stream go to the groups in turn (half h to group h mod 3).  A group has two score
+// buffers in TMEM; the weights of a half are written over the head of the scores they were computed from (32
+// columns of bf16 pairs over 64 columns of fp32):
 //   S_bi  = Q K_half^T                UMMA 128 x 64 x 32, A = Q smem, B = half K tile smem (K-major)
 //   P_bi  = exp2(S_bi c - m) | silu   group b: tcgen05.ld -> math -> bf16 -> tcgen05.st, in place
-//   O_b  += P_bi [V_half | 1]         UMMA 128 x 48 x 64, A = P from TMEM, B = half V tile (MN-major)
-// A buffer is free again when the weighted sum that read it has finished.  With three of them
-// the scores of step t+2 are issued while step t is being normalised: the round trip of a
-// hand-off through the tensor core (issue, a chain of K = 16 instructions, commit, the waiting
-// thread waking up: about a thousand clocks) is longer than one normalisation step, and with two
-// buffers both the normalisation threads and the issuing threads kept waiting for each other.
-// The other group works on its own half at the same time and the producers gather tiles
-// further ahead; nothing drains between work units.  The two groups keep separate
-// accumulators O_0, O_1 with separate reference maxima and merge them through shared memory
-// when a unit ends.
+//   O_b  += P_bi V_half               UMMA 128 x 32 x 64, A = P from TMEM, B = half V tile (MN-major)
+// One thread issues both kinds of MMA of its group, in the order weighted sum of step t, scores of step t + 2
+// (into the buffer the weighted sum has just read): the tensor core runs one thread's instructions in order, so
+// the buffer needs no completion hand-off in between, and the scores of step t + 1 are there while the group
+// normalises step t.  Why three groups: the normalisation of a half is a chain of dependent work for its warp
+// (wait for the scores, TMEM load, arithmetic, TMEM store, publish; at a unit's end the accumulator read-out and
+// the merge) during most of which the special-function unit of the warp's sub-partition is idle; measured on a
+// stripped-down pipeline, two groups keep that unit 70 % busy, three 85 %, and registers (65536 / 640 threads =
+// 96 each, enough for one 32-column chunk of scores at a time) and TMEM (3 x (2 x 64 + 32) = 480 columns) admit
+// no fourth.  The groups keep separate accumulators O_b with separate reference maxima and row sums and merge
+// them through shared memory when a unit ends; nothing drains between work units.
 //
-// Why four issuing warps: one thread hands a tcgen05.mma to the tensor core about every
-// hundred cycles whatever the instruction's size, and a tile needs ten of these small ones
-// (K = 16 per instruction), twelve with the halves.  Why one producer warp per tile: the bookkeeping of a tile (stream
-// position, waits, index and user-part loads) is a serial chain of a few hundred instructions;
-// paid by every producer warp for every tile it was the bottleneck of the whole pipeline.
+// Softmax bookkeeping.  The reference maximum m of a row is the largest of the first 32 scores of the group's
+// first half of the unit and stays fixed: later scores may exceed it by up to 2^64 (fp32 accumulators and bf16
+// P have the exponent range for that).  The largest exponent argument of every chunk is taken from the registers
+// with the weights; only when it exceeds that bound is the reference moved, O_b and the row sum rescaled (TMEM
+// read-modify-write) and the chunk written again.  The row sum l is added up by the row's thread in fp32.
 //
-// Softmax bookkeeping.  The V tile carries sixteen extra columns of which the first is all
-// ones, so column 32 of O_b accumulates the row sum l of exactly the bf16-rounded P that
-// multiplies V.  The reference maximum m of a row is the largest score of the group's first
-// half tile of the unit and stays fixed: later scores may exceed it by up to 2^64 (fp32
-// accumulators and bf16 P have the exponent range for that).  The row maximum of every half
-// tile is taken from the registers before any weight is written; only when it exceeds that
-// bound is the reference moved and O_b rescaled first (TMEM read-modify-write).
-//
-// Shared-memory tiles use the no-swizzle UMMA canonical layout: groups of 8 rows, inside a
+// Shared-memory tiles use the no-swizzle UMMA canonical layout: groups of 8 rows (512 bytes), inside a
 // group one 128-byte core matrix per 16-byte row chunk, inside a core matrix row r%8 at 16 r.
-// K tiles and Q use 512-byte groups (4 chunks); V tiles 768-byte groups (4 data chunks + 2
-// chunks holding the ones column).
 //
 // Every wait in this kernel is bounded: on time-out the CTA records an error code, raises a
 // CTA-wide abort flag that ends every other wait, drains its own copies, frees its TMEM and
@@ -63,49 +53,53 @@ namespace {
 constexpr int D = 32;
 constexpr int TK = 128;                  // positions per tile (one shared-memory stage)
 constexpr int TH = 64;                   // positions per half tile = one MMA / normalisation step of a group
-constexpr int NS = 9;                    // K/V stages
+constexpr int NG = 3;                    // normalisation groups
+constexpr int NS = 10;                   // K/V stages
 constexpr int NQ = 3;                    // Q buffers
 constexpr int kGroupThreads = 128;       // one normalisation group
-constexpr int kMmaWarp = 8;              // warps 8, 9 issue S = Q K^T of group 0, 1; warp 8 owns the TMEM allocation
-constexpr int kPvWarp0 = 10;             // warps 10, 11 issue the weighted sums of group 0, 1
-constexpr int kProducerWarp0 = 12;
-constexpr int kProducerWarps = 4;        // each owns every fourth tile of the stream
-constexpr int kThreads = 2 * kGroupThreads + 4 * 32 + kProducerWarps * 32;  // 512
+constexpr int kIssueWarp0 = 4 * NG;      // warps 12..14 issue the MMAs of group 0..2; warp 12 owns the TMEM allocation
+constexpr int kProducerWarp0 = kIssueWarp0 + NG;
+constexpr int kProducerWarps = 5;        // each owns every fifth tile of the stream
+constexpr int kThreads = (kProducerWarp0 + kProducerWarps) * 32;  // 640
 constexpr int kTileK = TK * D * 2;       // 8 KB, also the Q tile
-constexpr int kVGroup = 768;             // bytes of one 8-row group of a V tile
-constexpr int kTileV = (TK / 8) * kVGroup;  // 12 KB
-constexpr int kNV = 48;                  // columns of [V | 1 | 0...]
+constexpr int kVGroup = 512;             // bytes of one 8-row group of a V tile
+constexpr int kTileV = (TK / 8) * kVGroup;  // 8 KB
 constexpr uint32_t kTmemCols = 512;
-constexpr int NB = 3;                    // score / weight buffers per group
-constexpr uint32_t kColS = 0, kColO = 384;  // S_bi (and P_bi over its head) at kColS + 64 (NB b + i), O_b at kColO + 48 b
-static_assert(kColS + 64 * NB * 2 <= kColO && kColO + 2 * kNV <= kTmemCols, "TMEM columns");
+constexpr int NB = 2;                    // score / weight buffers per group
+constexpr uint32_t kColGroup = 64 * NB + D;  // group b: S_bi (and P_bi over its head) at kColGroup b + 64 i, O_b behind them
+static_assert(kColGroup * NG <= kTmemCols, "TMEM columns");
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kHeadroom = 64.0f;       // log2 units a score may exceed the reference maximum
 constexpr uint32_t kSpinLimit = 1u << 18;  // polls of a wait before the CTA gives up
 constexpr uint32_t kSuspendNs = 4000;      // how long one poll may stay suspended in hardware (longer hints wake later)
 static_assert(NS > kProducerWarps, "every producer warp holds one stage while it copies");
+static_assert(NS % kProducerWarps == 0, "a stage is always filled by the same producer warp, one use after the other");
 
 // dynamic shared memory map
 constexpr int kOffQ = 0;
 constexpr int kOffK = kOffQ + NQ * kTileK;
 constexpr int kOffV = kOffK + NS * kTileK;
-constexpr int kOffX = kOffV + NS * kTileV;          // exchange between the groups: [34][128] floats
-constexpr int kOffIdx = kOffX + 34 * 128 * 4;        // per producer warp: K and V row indices of its tile, 16 bit
+constexpr int kOffX = kOffV + NS * kTileV;          // what groups 1.. hand to group 0 when a unit ends: [NG - 1][34][128] floats
+constexpr int kOffIdx = kOffX + (NG - 1) * 34 * 128 * 4;        // per producer warp: K and V row indices of its tile, 16 bit
 constexpr int kOffBar = kOffIdx + kProducerWarps * 2 * TK * 2;
-constexpr int kOffAbort = kOffBar + 384;
-constexpr int kSmemBytes = kOffAbort + 16;
+constexpr int kOffAbort = kOffBar + 448;
+constexpr int kSmemBytes = kOffAbort + 32;
 
 // barrier slots (8 bytes each) behind kOffBar
 enum {
-    BAR_FULL = 0, BAR_EMPTY = NS, BAR_QEMPTY = 2 * NS,
-    BAR_SFULL = 2 * NS + NQ,            // [NB b + i]
-    BAR_PREADY = BAR_SFULL + 2 * NB,    // [NB b + i]
-    BAR_PFREE = BAR_SFULL + 4 * NB,     // [NB b + i]
-    BAR_OFULL = BAR_SFULL + 6 * NB,     // [b]
-    BAR_XFULL = BAR_OFULL + 2, BAR_XEMPTY, BAR_DRAIN,
-    BAR_COUNT = BAR_DRAIN + 4
+    BAR_FULL = 0, BAR_EMPTY = NS, BAR_QEMPTY = 2 * NS, BAR_QFULL = 2 * NS + NQ,
+    BAR_SFULL = 2 * NS + 2 * NQ,          // [NB b + i]
+    BAR_PREADY = BAR_SFULL + NG * NB,     // [NB b + i]
+    BAR_PFREE = BAR_PREADY + NG * NB,     // [NB b + i]
+    BAR_OFULL = BAR_PFREE + NG * NB,      // [b]
+    BAR_XFULL = BAR_OFULL + NG,           // [b - 1]
+    BAR_XEMPTY = BAR_XFULL + NG - 1,      // [b - 1]
+    BAR_DRAIN = BAR_XEMPTY + NG - 1,      // [b]
+    BAR_COUNT = BAR_DRAIN + NG
 };
-static_assert(BAR_COUNT * 8 <= 384, "barrier area");
+static_assert(BAR_COUNT * 8 <= 448, "barrier area");
+static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
+
 
 // error codes OR-ed into the context's device error word
 enum { ERR_NORMALISE = 1, ERR_MMA = 2, ERR_DRAIN = 4, ERR_PRODUCER = 8 };
@@ -119,7 +113,17 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar)
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 // Bounded wait on a phase parity.  Returns false on time-out or when the CTA is aborting.
-__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const volatile int* abort_flag)
+// A wait that runs out (rather than being ended by the abort flag) leaves its site code in the word behind the flag;
+// the first one stays, and the kernel reports it in bits 8.. of the error word.
+enum {
+    SITE_SFULL = 1, SITE_OFULL, SITE_XEMPTY, SITE_XFULL, SITE_PFREE, SITE_TILE, SITE_Q, SITE_PREADY, SITE_TAIL_TILE,
+    SITE_STAGE, SITE_QBUF, SITE_DRAIN, SITE_QTURN
+};
+__device__ __forceinline__ void note_site(const volatile int* abort_flag, int site)
+{
+    atomicCAS(const_cast<int*>(abort_flag) + 1, 0, site);
+}
+__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const volatile int* abort_flag, int site)
 {
     for (uint32_t i = 0; i < kSpinLimit; ++i) {
         uint32_t ok;
@@ -133,10 +137,11 @@ __device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const vola
         if (ok) return true;
         if ((i & 31u) == 31u && *abort_flag) return false;
     }
+    note_site(abort_flag, site);
     return false;
 }
-// One poll of a phase parity: true if that phase has completed.
-__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity)
+// The bounded wait with its first poll inline: most waits of the issuing threads find their phase complete.
+__device__ __forceinline__ bool mbar_wait_fast(uint32_t bar, uint32_t parity, const volatile int* abort_flag, int site)
 {
     uint32_t ok;
     asm volatile(
@@ -146,7 +151,7 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity)
         : "=r"(ok)
         : "r"(bar), "r"(parity)
         : "memory");
-    return ok != 0;
+    return ok != 0 || mbar_wait(bar, parity, abort_flag, site);
 }
 // 16-byte copy global -> shared; src_bytes = 0 fills the destination with zeros instead.
 // Pool rows go through L1 (with skewed indices the hot rows then stop hammering a few L2 lines
@@ -286,7 +291,7 @@ __device__ __forceinline__ int pos_of_col(int c, int e) { return 32 * c + 4 * (e
 
 // ---- normalisation of one 128 x 64 score half tile by its group (thread = query row = TMEM lane) ----
 
-// Multiplies this thread's row of O (32 columns and the row sum in column 32) by f.
+// Multiplies this thread's row of O (32 columns) by f.
 __device__ __noinline__ void rescale_row(uint32_t tO, float f)
 {
     uint32_t o[32];
@@ -295,8 +300,6 @@ __device__ __noinline__ void rescale_row(uint32_t tO, float f)
 #pragma unroll
     for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * f);
     tmem_st32(tO, o);
-    const uint32_t l = tmem_ld1(tO + 32);
-    tmem_st1(tO + 32, __float_as_uint(__uint_as_float(l) * f));
 }
 
 // Multiplies the 32 weights (16 columns of bf16 pairs) this thread wrote for the first chunk of the current half
@@ -309,12 +312,13 @@ __device__ __noinline__ void rescale_weights(uint32_t tP, float f)
     }
 }
 
-// The weights of one 32-column chunk once more, from scores the caller has put into local memory (only used on
+// The weights of one 32-column chunk once more (returns their sum), from scores the caller has put into local memory (only used on
 // the rare path that moves a row's reference; kept out of line so that it costs the common path nothing).
 template <bool TAIL>
-__device__ __noinline__ void rewrite_weights(uint32_t tP, const uint32_t* cur, float sc, float nm, int valid, int c)
+__device__ __noinline__ float rewrite_weights(uint32_t tP, const uint32_t* cur, float sc, float nm, int valid, int c)
 {
     uint32_t p[16];
+    float sum = 0.f;
 #pragma unroll
     for (int e = 0; e < 32; e += 2) {
         float x0 = fmaf(__uint_as_float(cur[e]), sc, nm), x1 = fmaf(__uint_as_float(cur[e + 1]), sc, nm);
@@ -322,15 +326,18 @@ __device__ __noinline__ void rewrite_weights(uint32_t tP, const uint32_t* cur, f
             if (pos_of_col(c, e) >= valid) x0 = -CUDART_INF_F;
             if (pos_of_col(c, e + 1) >= valid) x1 = -CUDART_INF_F;
         }
-        p[e >> 1] = pack_bf16(ex2(x0), ex2(x1));
+        const float e0 = ex2(x0), e1 = ex2(x1);
+        sum += e0 + e1;
+        p[e >> 1] = pack_bf16(e0, e1);
     }
     tmem_st16(tP, p);
+    return sum;
 }
 
 // Softmax weights of one 32-column chunk (c = 0, 1) of a 128 x 64 score half tile: p = exp2(s c - m) as bf16
 // pairs written over the head of the scores (columns 0..31 of the buffer; chunk 1 of the scores, columns 32..63,
-// is in the registers or still to be read when chunk 0's weights land on columns 0..15, and chunk 1's weights
-// land on columns 16..31, whose scores have been consumed).  With `first` (chunk 0 of the group's first half
+// is still to be read when chunk 0's weights land on columns 0..15, and chunk 1's weights
+// land on columns 16..31, whose scores have been consumed).  The chunk's weights are added to the row sum l.  With `first` (chunk 0 of the group's first half
 // tile of a unit) the row's reference m is set from these 32 scores (column 0 is the half's position 0, always a
 // real one).  A chunk whose largest exponent argument leaves the headroom moves the reference up by a whole
 // number of octaves and is written again from the scores still in the registers; what O_b holds so far
@@ -343,7 +350,7 @@ __device__ __noinline__ void rewrite_weights(uint32_t tP, const uint32_t* cur, f
 // of this half tile); a row's reference is then set by the first chunk in which it sees a position.
 template <bool TAIL, bool VIS, typename WaitPrev>
 __device__ __forceinline__ bool softmax_chunk(const uint32_t (&cur)[32], int c, uint32_t tS, uint32_t tO, float sc,
-                                              int valid, bool first, bool have_o, float& m_ref, WaitPrev&& wait_prev)
+                                              int valid, bool first, bool have_o, float& m_ref, float& l, WaitPrev&& wait_prev)
 {
     if ((c == 0 && first) || (VIS && m_ref == -CUDART_INF_F)) {
         float t0 = -CUDART_INF_F, t1 = -CUDART_INF_F;
@@ -360,6 +367,7 @@ __device__ __forceinline__ bool softmax_chunk(const uint32_t (&cur)[32], int c, 
     }
     float nm = -m_ref;
     float mx = -CUDART_INF_F, mx2 = -CUDART_INF_F;
+    float ls0 = 0.f, ls1 = 0.f;  // this chunk's share of the row sum
     uint32_t p[16];
 #pragma unroll
     for (int e = 0; e < 32; e += 2) {
@@ -370,19 +378,24 @@ __device__ __forceinline__ bool softmax_chunk(const uint32_t (&cur)[32], int c, 
         }
         if (e & 2) mx = max3(mx, x0, x1);
         else mx2 = max3(mx2, x0, x1);
-        p[e >> 1] = pack_bf16(ex2(x0), ex2(x1));
+        const float e0 = ex2(x0), e1 = ex2(x1);
+        ls0 += e0;
+        ls1 += e1;
+        p[e >> 1] = pack_bf16(e0, e1);
     }
-    tmem_st16(tS + 16 * c, p);
     mx = fmaxf(mx, mx2);
-    if (__any_sync(0xffffffffu, mx > kHeadroom)) {
-        // rare: some row of this warp left the headroom and its weights just written may have overflowed.
-        // The chunk's scores are still in the registers: move the reference, bring what was accumulated and
-        // written before into the new scale, and write the chunk's weights again.
+    if (!__any_sync(0xffffffffu, mx > kHeadroom)) {
+        tmem_st16(tS + 16 * c, p);
+    } else {
+        // rare: some row of this warp left the headroom and its weights may have overflowed.  Nothing of this
+        // chunk has been written yet, so its scores are still in TMEM: move the reference, bring what was
+        // accumulated and written before into the new scale, and work the chunk out again from there.
         const float shift = mx > kHeadroom ? ceilf(mx) : 0.f;
         const float f = ex2(-shift);
         m_ref += shift;
         nm = -m_ref;
         tc_wait_st();
+        l *= f;
         if (have_o) {
             if (!wait_prev()) return false;
             tc_fence_after();
@@ -390,11 +403,13 @@ __device__ __forceinline__ bool softmax_chunk(const uint32_t (&cur)[32], int c, 
         }
         if (c == 1) rescale_weights(tS, f);
         uint32_t again[32];
-#pragma unroll
-        for (int e = 0; e < 32; ++e) again[e] = cur[e];
-        rewrite_weights<TAIL>(tS + 16 * c, again, sc, nm, valid, c);
+        tmem_ld32(tS + 32 * c, again);
+        tmem_wait_ld32(again);
+        ls0 = rewrite_weights<TAIL>(tS + 16 * c, again, sc, nm, valid, c);
+        ls1 = 0.f;
         tc_wait_st();
     }
+    l += ls0 + ls1;
     return true;
 }
 
@@ -450,6 +465,13 @@ struct Unit {
     int n_tiles;     // > 0: tiles to process; 0: empty history (zero output rows); < 0: nothing at all
     int last_valid;  // real positions in the last tile
 };
+
+// Which group takes a unit's first half (half p goes to group (p + rotation) mod NG).  A function of the unit
+// alone -- not of its place in a CTA's stream -- so that results do not depend on what else a call processes.
+__device__ __forceinline__ int unit_rotation(const Unit& u)
+{
+    return (int)((uint32_t)(u.grp + (u.row0 >> 7) + (u.wk.begin >> 6)) % (uint32_t)NG);
+}
 
 __device__ __forceinline__ Work load_work(const Work* p)
 {
@@ -585,53 +607,56 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
 
     if (tid == 0) {
         for (int s = 0; s < NS; ++s) {
-            mbar_init(bar(BAR_FULL + s), 1);  // lane 0 of the producer warp that owns the tile
+            mbar_init(bar(BAR_FULL + s), 1);   // lane 0 of the producer warp that owns the tile
             mbar_init(bar(BAR_EMPTY + s), 2);  // one arrival per half
         }
-        for (int q = 0; q < NQ; ++q) mbar_init(bar(BAR_QEMPTY + q), 2);  // both score issuers
-        for (int bi = 0; bi < 2 * NB; ++bi) {
+        for (int q = 0; q < NQ; ++q) {
+            mbar_init(bar(BAR_QEMPTY + q), NG);  // every issuer
+            mbar_init(bar(BAR_QFULL + q), 1);    // lane 0 of the producer warp that staged the unit's Q block
+        }
+        for (int bi = 0; bi < NG * NB; ++bi) {
             mbar_init(bar(BAR_SFULL + bi), 1);
             mbar_init(bar(BAR_PREADY + bi), kGroupThreads);
             mbar_init(bar(BAR_PFREE + bi), 1);
         }
-        for (int b = 0; b < 2; ++b) mbar_init(bar(BAR_OFULL + b), 1);
-        mbar_init(bar(BAR_XFULL), kGroupThreads);
-        mbar_init(bar(BAR_XEMPTY), kGroupThreads);
-        for (int i = 0; i < 4; ++i) mbar_init(bar(BAR_DRAIN + i), 1);
-        *abort_flag = 0;
+        for (int b = 0; b < NG; ++b) {
+            mbar_init(bar(BAR_OFULL + b), 1);
+            mbar_init(bar(BAR_DRAIN + b), 1);
+        }
+        for (int b = 0; b < NG - 1; ++b) {
+            mbar_init(bar(BAR_XFULL + b), kGroupThreads);
+            mbar_init(bar(BAR_XEMPTY + b), kGroupThreads);
+        }
+        abort_flag[0] = 0;  // raised by the first role that gives up
+        abort_flag[1] = 0;  // site of the first wait that ran out
+        abort_flag[4] = 0;  // units whose Q block has a producer at work on it (see the producers)
+        abort_flag[2] = 0;  // never raised: the flag of the teardown wait, which must not be cut short
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == kMmaWarp) {
+    if (warp == kIssueWarp0) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
                      "r"(kTmemCols)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    // the constant chunks 4 and 5 of every V stage: column 32 is one, columns 33..47 are zero
-    for (int i = tid; i < NS * TK * 2; i += kThreads) {
-        const int s = i / (TK * 2), r = (i >> 1) & (TK - 1), c = 4 + (i & 1);
-        *reinterpret_cast<uint4*>(smem + kOffV + s * kTileV + v_off(r, c)) = make_uint4(c == 4 ? 0x3f80u : 0u, 0u, 0u, 0u);
-    }
-    fence_proxy_async();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = tmem_base_slot;
 
-    if (warp < 8) {
+    if (warp < kIssueWarp0) {
         // --------------------------------------------------------------- normalisation groups
-        const int b = warp >> 2;                    // group = score buffer
+        const int b = warp >> 2;                    // group
         const int row = tid & (kGroupThreads - 1);  // query row inside the block = TMEM lane
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t tS0 = tmem + lane_base + kColS + 64u * NB * b, tO = tmem + lane_base + kColO + (uint32_t)kNV * b;
+        const uint32_t tS0 = tmem + lane_base + kColGroup * b, tO = tS0 + 64u * NB;
         const float sc = a.scale * (MODE == CKV_SOFTMAX ? kLog2e : 0.5f);
         float* xch = reinterpret_cast<float*>(smem + kOffX);
-        int cnt = 0;    // half tiles this group has normalised
-        int ocnt = 0;   // units in which this group had tiles
+        int cnt = 0;    // halves this group has normalised
+        int ocnt = 0;   // units in which this group had halves
         int xcnt = 0;   // units exchanged between the groups
         bool ok = true;
-        uint32_t sa[32], sb[32];  // the two chunks of a half tile's scores
-        bool have_sa = false;     // sa is already receiving the first chunk of the coming step's scores
+        uint32_t sa[32];  // one 32-column chunk of a half's scores
         Stream<true, VIS> sn;
         sn.init(a, n_mb, n_work);
         for (; sn.valid && ok; sn.next_unit()) {
@@ -658,71 +683,53 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
             // positions this thread's query row attends: [0, lim); rows beyond the user's queries take none
             int lim = u.wk.L;
             if constexpr (VIS) lim = r < u.wk.M ? min(max(__ldg(a.vis + u.wk.q0 + r), 0), u.wk.L) : 0;
-            float m_ref = -CUDART_INF_F;
-            int mine = 0;  // half tiles of this unit normalised by this group
-            for (int j = 0; j < u.n_tiles && ok; ++j) {
-                const int valid = (j == u.n_tiles - 1 ? u.last_valid : TK) - TH * b;  // real positions of this group's half
-                if (valid <= 0) continue;  // only the second half of a unit's last tile can be empty
-                const int i = cnt % NB;    // buffer of this step
+            float m_ref = -CUDART_INF_F, l = 0.f;
+            int mine = 0;  // halves of this unit normalised by this group
+            // The unit's non-empty halves are p = 2 j + half < n_half (only the second half of the last tile can be
+            // empty); half p goes to group (p + unit_rotation) mod NG.
+            const int n_half = 2 * u.n_tiles - (u.last_valid <= TH ? 1 : 0);
+            for (int p = (b + NG - unit_rotation(u)) % NG; p < n_half && ok; p += NG) {
+                const int j = p >> 1, half = p & 1;
+                const int valid = (j == u.n_tiles - 1 ? u.last_valid : TK) - TH * half;  // real positions of the half
+                const int i = cnt % NB;                                                   // buffer of this step
                 const uint32_t tS = tS0 + 64u * i;
-                if (!have_sa) {
-                    // the scores arrive in a buffer whose previous weights the tensor core has finished reading
-                    ok = mbar_wait(bar(BAR_SFULL + NB * b + i), (cnt / NB) & 1, abort_flag);
-                    ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) break;
-                    tc_fence_after();
-                }
+                ok = mbar_wait_fast(bar(BAR_SFULL + NB * b + i), (cnt / NB) & 1, abort_flag, SITE_SFULL);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after();
                 // (softmax, only taken when a row leaves the headroom) the previous step's MMAs must have finished
                 // before O_b is rescaled
                 auto wait_prev = [&]() {
-                    bool w = mbar_wait(bar(BAR_PFREE + NB * b + (cnt - 1) % NB), ((cnt - 1) / NB) & 1, abort_flag);
+                    bool w = mbar_wait(bar(BAR_PFREE + NB * b + (cnt - 1) % NB), ((cnt - 1) / NB) & 1, abort_flag, SITE_PFREE);
                     return __all_sync(0xffffffffu, w);
                 };
-                // real (and, with visible lengths, attended) positions of this thread's row in the half tile
+                // real (and, with visible lengths, attended) positions of this thread's row in the half
                 int valid_r = valid;
                 bool tail = valid < TH;
                 if constexpr (VIS) {
-                    valid_r = min(valid, lim - (u.wk.begin + j * TK + TH * b));
+                    valid_r = min(valid, lim - (u.wk.begin + j * TK + TH * half));
                     tail = __any_sync(0xffffffffu, valid_r < TH);
                 }
-                if (tail) {
-                    // end of a history (at most once per unit and group) or of some row's visible positions: compact
-                    // code, masked columns, chunk by chunk
+                // One 32-column chunk at a time: the other groups' warps on this sub-partition cover the TMEM load.
+                if (tail) {  // end of a history or of some row's visible positions: masked columns
 #pragma unroll 1
                     for (int c = 0; c < 2 && ok; ++c) {
                         tmem_ld32(tS + 32 * c, sa);
                         tmem_wait_ld32(sa);
                         if constexpr (MODE == CKV_SOFTMAX)
-                            ok = softmax_chunk<true, VIS>(sa, c, tS, tO, sc, valid_r, mine == 0, mine > 0, m_ref, wait_prev);
+                            ok = softmax_chunk<true, VIS>(sa, c, tS, tO, sc, valid_r, mine == 0, mine > 0, m_ref, l, wait_prev);
                         else
                             silu_chunk<true>(sa, c, tS, sc, valid_r);
                     }
                 } else {
-                    // all 64 columns are real positions.  The two 32-column chunks are double-buffered in registers:
-                    // the second tcgen05.ld is in flight during the arithmetic of the first, and the first chunk of
-                    // this group's NEXT step, if its scores are there already, during the arithmetic of the second
-                    // (a TMEM load takes a few hundred clocks to return, as long as the arithmetic of a chunk).
-                    if (!have_sa) tmem_ld32(tS, sa);
-                    tmem_wait_ld32(sa);
-                    tmem_ld32(tS + 32, sb);
-                    if constexpr (MODE == CKV_SOFTMAX)
-                        ok = softmax_chunk<false, VIS>(sa, 0, tS, tO, sc, valid, mine == 0, mine > 0, m_ref, wait_prev);
-                    else
-                        silu_chunk<false>(sa, 0, tS, sc, valid);
-                    tmem_wait_ld32(sb);
-                    have_sa = false;
-                    if (ok && !VIS && j + 1 < u.n_tiles && (j + 1 == u.n_tiles - 1 ? u.last_valid : TK) - TH * b >= TH) {
-                        const int i2 = (cnt + 1) % NB;
-                        if (__all_sync(0xffffffffu, mbar_test(bar(BAR_SFULL + NB * b + i2), ((cnt + 1) / NB) & 1))) {
-                            tc_fence_after();
-                            tmem_ld32(tS0 + 64u * i2, sa);
-                            have_sa = true;
-                        }
-                    }
-                    if constexpr (MODE == CKV_SOFTMAX) {
-                        if (ok) ok = softmax_chunk<false, VIS>(sb, 1, tS, tO, sc, valid, false, mine > 0, m_ref, wait_prev);
-                    } else {
-                        silu_chunk<false>(sb, 1, tS, sc, valid);
+#pragma unroll 1
+                    for (int c = 0; c < 2 && ok; ++c) {
+                        tmem_ld32(tS + 32 * c, sa);
+                        tmem_wait_ld32(sa);
+                        if constexpr (MODE == CKV_SOFTMAX)
+                            ok = softmax_chunk<false, VIS>(sa, c, tS, tO, sc, valid, mine == 0, mine > 0, m_ref, l, wait_prev);
+                        else
+                            silu_chunk<false>(sa, c, tS, sc, valid);
                     }
                 }
                 if (!ok) break;
@@ -734,10 +741,10 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
             }
             if (!ok) break;
 
-            // ---- the unit's epilogue: fetch O_b, merge the two groups, store
-            float o[32], l = 0.f;
+            // ---- the unit's epilogue: fetch O_b, merge the groups, store
+            float o[32];
             if (mine > 0) {
-                ok = mbar_wait(bar(BAR_OFULL + b), ocnt & 1, abort_flag);
+                ok = mbar_wait(bar(BAR_OFULL + b), ocnt & 1, abort_flag, SITE_OFULL);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 ++ocnt;
@@ -747,41 +754,46 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                 tmem_wait_ld32(raw);
 #pragma unroll
                 for (int e = 0; e < 32; ++e) o[e] = __uint_as_float(raw[e]);
-                if constexpr (MODE == CKV_SOFTMAX) l = __uint_as_float(tmem_ld1(tO + 32));
                 tc_fence_before();
             } else {
 #pragma unroll
                 for (int e = 0; e < 32; ++e) o[e] = 0.f;
             }
-            if (b == 1) {
-                if (xcnt > 0) ok = mbar_wait(bar(BAR_XEMPTY), (xcnt - 1) & 1, abort_flag);
+            if (b > 0) {
+                float* x = xch + (b - 1) * 34 * 128;
+                if (xcnt > 0) ok = mbar_wait(bar(BAR_XEMPTY + b - 1), (xcnt - 1) & 1, abort_flag, SITE_XEMPTY);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
-                xch[row] = m_ref;
-                xch[128 + row] = l;
+                x[row] = m_ref;
+                x[128 + row] = l;
 #pragma unroll
-                for (int e = 0; e < 32; ++e) xch[(2 + e) * 128 + row] = o[e];
-                mbar_arrive(bar(BAR_XFULL));
+                for (int e = 0; e < 32; ++e) x[(2 + e) * 128 + row] = o[e];
+                mbar_arrive(bar(BAR_XFULL + b - 1));
                 ++xcnt;
             } else {
-                ok = mbar_wait(bar(BAR_XFULL), xcnt & 1, abort_flag);
-                ok = __all_sync(0xffffffffu, ok);
+#pragma unroll 1
+                for (int g2 = 1; g2 < NG && ok; ++g2) {
+                    const float* x = xch + (g2 - 1) * 34 * 128;
+                    ok = mbar_wait(bar(BAR_XFULL + g2 - 1), xcnt & 1, abort_flag, SITE_XFULL);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    const float m1 = x[row], l1 = x[128 + row];
+                    if constexpr (MODE == CKV_SOFTMAX) {
+                        const float mt = fmaxf(m_ref, m1);
+                        const float ms = mt == -CUDART_INF_F ? 0.f : mt;
+                        const float c0 = ex2(m_ref - ms), c1 = ex2(m1 - ms);
+                        l = l * c0 + l1 * c1;
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) o[e] = o[e] * c0 + x[(2 + e) * 128 + row] * c1;
+                        m_ref = mt;
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) o[e] += x[(2 + e) * 128 + row];
+                    }
+                    mbar_arrive(bar(BAR_XEMPTY + g2 - 1));
+                }
                 if (!ok) break;
                 ++xcnt;
-                const float m1 = xch[row], l1 = xch[128 + row];
-                if constexpr (MODE == CKV_SOFTMAX) {
-                    const float mt = fmaxf(m_ref, m1);
-                    const float ms = mt == -CUDART_INF_F ? 0.f : mt;
-                    const float c0 = ex2(m_ref - ms), c1 = ex2(m1 - ms);
-                    l = l * c0 + l1 * c1;
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) o[e] = o[e] * c0 + xch[(2 + e) * 128 + row] * c1;
-                    m_ref = mt;
-                } else {
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) o[e] += xch[(2 + e) * 128 + row];
-                }
-                mbar_arrive(bar(BAR_XEMPTY));
                 if (r < u.wk.M) {
                     if (u.wk.part_row < 0) {
                         float inv;
@@ -815,98 +827,141 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                 }
             }
         }
-        tc_wait_ld();  // a load issued ahead may still be in flight when a wait has run out
+        tc_wait_ld();
         if (!ok) {
             *abort_flag = 1;
             if (lane == 0) atomicOr(err_flag, ERR_NORMALISE);
         }
-    } else if (warp < kPvWarp0) {
-        // --------------------------------------------------------------------- S_bi = Q K_half^T issue
+    } else if (warp < kProducerWarp0) {
+        // --------------------------------------------------------------------- MMA issue for one group
+        // One thread per group, and its loop is the pipeline's pacemaker: it is a chain of dependent instructions
+        // of a single thread, so everything that can be kept out of it is (descriptors are a constant plus an
+        // offset, the two pending weighted sums live in named registers, waits poll once inline before they call).
         if (lane == 0) {
-            const int b = warp - kMmaWarp;
-            constexpr uint32_t idesc_s = make_idesc(128, TH, false);
+            const int b = warp - kIssueWarp0;
+            constexpr uint32_t idesc_s = make_idesc(128, TH, false), idesc_pv = make_idesc(128, D, true);
+            const uint32_t tS0 = tmem + kColGroup * b, tO = tS0 + 64u * NB;
+            const uint64_t dq0 = smem_desc(sbase + kOffQ, 128, 512), dk0 = smem_desc(sbase + kOffK, 128, 512),
+                           dv0 = smem_desc(sbase + kOffV, kVGroup, 128);
+            auto at = [](uint64_t d, uint32_t byte_off) { return d + (uint64_t)(byte_off >> 4); };  // no carry out of the address field
+            static_assert(NB == 2, "two pending weighted sums");
             Stream<false, VIS> ss;
             ss.init(a, n_mb, n_work);
-            int cnt = 0;  // half tiles issued
+            int cnt = 0;   // steps whose scores have been issued
+            int done = 0;  // steps whose weighted sum has been issued
+            // what the weighted sums of the (at most two) steps in flight need, oldest first: byte offset of the half V
+            // tile, stage to release, flags (bit 0: O_b already holds the unit's earlier halves; bit 1: the group's
+            // last half of the unit)
+            uint32_t pv_off0 = 0, pv_off1 = 0;
+            int pv_s0 = 0, pv_s1 = 0, pv_f0 = 0, pv_f1 = 0;
+            int pv_t0 = 0, pv_t1 = 0;  // their tiles' places in the stream
+            int gs = 0, gp = 0;  // stage and phase parity of the unit's first tile: g % NS, (g / NS) & 1
             bool ok = true;
-            for (; ok && ss.valid; ss.advance()) {
-                const int s = ss.g % NS;
-                const bool last = ss.j == ss.u.n_tiles - 1;
-                if ((last ? ss.u.last_valid : TK) > TH * b) {  // else: empty second half
-                    const int i = cnt % NB;
-                    ok = mbar_wait(bar(BAR_FULL + s), (ss.g / NS) & 1, abort_flag);
-                    // S_bi is free once the weighted sum of NB steps ago, which read its weights out of it, has finished
-                    if (ok && cnt >= NB) ok = mbar_wait(bar(BAR_PFREE + NB * b + i), ((cnt / NB) - 1) & 1, abort_flag);
+            // O_b += P_bi V_half for step `done`, whose group has written P_bi
+            auto do_pv = [&]() {
+                const int i = done & 1;
+                tc_fence_after();
+                const uint64_t dv = at(dv0, pv_off0);
+#pragma unroll
+                for (int kk = 0; kk < TH / 16; ++kk)  // sixteen positions per instruction
+                    umma_ts(tO, tS0 + 64u * i + 8 * kk, at(dv, kk * 2 * kVGroup), idesc_pv, ((pv_f0 & 1) || kk > 0) ? 1u : 0u);
+                tc_commit(bar(BAR_EMPTY + pv_s0));
+                tc_commit(bar(BAR_PFREE + NB * b + i));
+                if (pv_f0 & 2) tc_commit(bar(BAR_OFULL + b));
+                pv_off0 = pv_off1;
+                pv_s0 = pv_s1;
+                pv_f0 = pv_f1;
+                pv_t0 = pv_t1;
+                ++done;
+            };
+            // ... waiting for the weights first (used where the thread can do nothing else)
+            auto issue_pv = [&]() {
+                if (!mbar_wait_fast(bar(BAR_PREADY + NB * b + (done & 1)), (done >> 1) & 1, abort_flag, SITE_PREADY)) return false;
+                do_pv();
+                return true;
+            };
+            // A weighted sum is normally issued when its buffer is wanted for the scores two steps on.  Where the
+            // group's halves lie far apart (short units whose halves go to the other groups) that could be never: the
+            // weighted sum releases a stage, and the tile this thread waits for next may need that very stage.  So
+            // before waiting for tile `t_now` of the stream, the weighted sums of steps kMaxLag or more tiles back are
+            // issued first (in the regular rhythm of one half in three a pending step is at most five tiles back, so
+            // this never delays the scores there).  With every issuer keeping to that, the tile the hindmost issuer
+            // waits for only needs stages of tiles NS back, which nobody holds any more.
+            constexpr int kMaxLag = 7;
+            static_assert(kMaxLag < NS, "a held stage must never be the one the awaited tile goes to");
+            auto catch_up = [&](int t_now) {
+                bool w = true;
+                while (w && done < cnt && t_now - pv_t0 >= kMaxLag) w = issue_pv();
+                return w;
+            };
+            for (; ok && ss.valid; ss.next_unit()) {
+                const Unit& u = ss.u;
+                const int n_half = 2 * u.n_tiles - (u.last_valid <= TH ? 1 : 0);
+                const int rot = unit_rotation(u);
+                const uint32_t q_off = (uint32_t)(ss.useq % NQ) * kTileK;
+                bool q_seen = false;  // this thread has seen the unit's Q block staged
+                for (int p = (b + NG - rot) % NG; p < n_half; p += NG) {
+                    const int t = gs + (p >> 1), half = p & 1;
+                    const int s = t % NS, par = gp ^ ((t / NS) & 1);
+                    ok = catch_up(ss.g + (p >> 1)) && mbar_wait_fast(bar(BAR_FULL + s), par, abort_flag, SITE_TILE);
+                    // buffer i still holds the weights of step cnt - NB: its weighted sum goes first.  The tensor core
+                    // runs this thread's instructions in order, so the scores below need not wait for it to finish.
+                    if (ok && cnt - done == NB) ok = issue_pv();
+                    if (ok && !q_seen) {  // first scores of a unit: its Q block must have landed
+                        ok = mbar_wait_fast(bar(BAR_QFULL + ss.useq % NQ), (ss.useq / NQ) & 1, abort_flag, SITE_Q);
+                        q_seen = true;
+                    }
                     if (!ok) break;
                     tc_fence_after();
-                    ++cnt;
-                    const uint32_t q_addr = sbase + kOffQ + (ss.useq % NQ) * kTileK,
-                                   k_addr = sbase + kOffK + s * kTileK + b * (TH / 8) * 512;
+                    const int i = cnt & 1;
+                    const uint64_t dq = at(dq0, q_off), dk = at(dk0, (uint32_t)s * kTileK + half * (TH / 8) * 512);
 #pragma unroll
                     for (int ks = 0; ks < D / 16; ++ks)
-                        umma_ss(tmem + kColS + 64u * (NB * b + i), smem_desc(q_addr + ks * 256, 128, 512),
-                                smem_desc(k_addr + ks * 256, 128, 512), idesc_s, ks > 0 ? 1u : 0u);
+                        umma_ss(tS0 + 64u * i, at(dq, ks * 256), at(dk, ks * 256), idesc_s, ks > 0 ? 1u : 0u);
                     tc_commit(bar(BAR_SFULL + NB * b + i));
+                    const uint32_t off = (uint32_t)s * kTileV + half * (TH / 8) * kVGroup;
+                    const int f = (p >= NG ? 1 : 0) | (p + NG >= n_half ? 2 : 0);
+                    if (cnt == done) {
+                        pv_off0 = off;
+                        pv_s0 = s;
+                        pv_f0 = f;
+                        pv_t0 = ss.g + (p >> 1);
+                    } else {
+                        pv_off1 = off;
+                        pv_s1 = s;
+                        pv_f1 = f;
+                        pv_t1 = ss.g + (p >> 1);
+                    }
+                    ++cnt;
                 }
-                if (last) {
-                    // This issuer no longer reads the unit's Q buffer.  It must have seen the unit's last
-                    // tile published even if it issued nothing for it, or it could run units ahead of
-                    // the other issuer and complete a later use of the same barrier in its place.
-                    ok = mbar_wait(bar(BAR_FULL + s), (ss.g / NS) & 1, abort_flag);
+                if (!ok) break;
+                ok = catch_up(ss.g + u.n_tiles - 1);
+                if (!ok) break;
+                const int t_last = gs + u.n_tiles - 1;
+                if (u.last_valid <= TH && (2 * u.n_tiles - 1 + rot) % NG == b) {
+                    // the empty second half of the unit's last tile is this group's: nothing to compute, but the
+                    // stage needs this half's release
+                    ok = mbar_wait_fast(bar(BAR_FULL + t_last % NS), gp ^ ((t_last / NS) & 1), abort_flag, SITE_TAIL_TILE);
                     if (!ok) break;
-                    tc_commit(bar(BAR_QEMPTY + ss.useq % NQ));
+                    mbar_arrive(bar(BAR_EMPTY + t_last % NS));
                 }
+                // This issuer no longer reads the unit's Q buffer.  It observes every staging of a buffer,
+                // whether it has halves in the unit or not: the buffer is staged again only after all
+                // issuers have released it, so no issuer can run a use ahead of another on these barriers.
+                if (!q_seen) ok = mbar_wait_fast(bar(BAR_QFULL + ss.useq % NQ), (ss.useq / NQ) & 1, abort_flag, SITE_Q);
+                if (!ok) break;
+                tc_commit(bar(BAR_QEMPTY + ss.useq % NQ));
+                gp ^= ((t_last + 1) / NS) & 1;
+                gs = (t_last + 1) % NS;
             }
+            while (ok && done < cnt) ok = issue_pv();
             if (!ok) {
                 *abort_flag = 1;
                 atomicOr(err_flag, ERR_MMA);
             }
             // nothing of this CTA may still be running on the tensor core at teardown
             tc_commit(bar(BAR_DRAIN + b));
-            volatile int never = 0;
-            if (!mbar_wait(bar(BAR_DRAIN + b), 0, &never)) atomicOr(err_flag, ERR_DRAIN);
-        }
-        __syncwarp();
-    } else if (warp < kProducerWarp0) {
-        // --------------------------------------------------------------------- O_b += P_b [V | 1] issue
-        if (lane == 0) {
-            const int b = warp - kPvWarp0;
-            constexpr uint32_t idesc_pv = make_idesc(128, MODE == CKV_SOFTMAX ? kNV : D, true);
-            Stream<false, VIS> sp;
-            sp.init(a, n_mb, n_work);
-            int cnt = 0;
-            bool ok = true;
-            for (; ok && sp.valid; sp.advance()) {
-                const int s = sp.g % NS;
-                const int valid = (sp.j == sp.u.n_tiles - 1 ? sp.u.last_valid : TK) - TH * b;
-                if (valid <= 0) {  // empty second half: nothing to add, but the stage still needs this half's release
-                    ok = mbar_wait(bar(BAR_FULL + s), (sp.g / NS) & 1, abort_flag);
-                    if (ok) mbar_arrive(bar(BAR_EMPTY + s));
-                    continue;
-                }
-                const int i = cnt % NB;
-                ok = mbar_wait(bar(BAR_PREADY + NB * b + i), (cnt / NB) & 1, abort_flag);
-                if (ok) ok = mbar_wait(bar(BAR_FULL + s), (sp.g / NS) & 1, abort_flag);  // completed long ago: makes the V tile visible here
-                if (!ok) break;
-                ++cnt;
-                tc_fence_after();
-                const uint32_t v_addr = sbase + kOffV + s * kTileV + b * (TH / 8) * kVGroup;
-                const bool last = sp.j == sp.u.n_tiles - 1 || (sp.j == sp.u.n_tiles - 2 && sp.u.last_valid <= TH * b);
-#pragma unroll
-                for (int kk = 0; kk < TH / 16; ++kk)  // sixteen positions per instruction
-                    umma_ts(tmem + kColO + (uint32_t)kNV * b, tmem + kColS + 64u * (NB * b + i) + 8 * kk,
-                            smem_desc(v_addr + kk * 2 * kVGroup, kVGroup, 128), idesc_pv, (sp.j > 0 || kk > 0) ? 1u : 0u);
-                tc_commit(bar(BAR_EMPTY + s));
-                tc_commit(bar(BAR_PFREE + NB * b + i));
-                if (last) tc_commit(bar(BAR_OFULL + b));  // the group's last step of the unit
-            }
-            if (!ok) {
-                *abort_flag = 1;
-                atomicOr(err_flag, ERR_MMA);
-            }
-            tc_commit(bar(BAR_DRAIN + 2 + b));
-            volatile int never = 0;
-            if (!mbar_wait(bar(BAR_DRAIN + 2 + b), 0, &never)) atomicOr(err_flag, ERR_DRAIN);
+            if (!mbar_wait(bar(BAR_DRAIN + b), 0, abort_flag + 2, SITE_DRAIN)) atomicOr(err_flag, ERR_DRAIN);
         }
         __syncwarp();
     } else {
@@ -974,16 +1029,33 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
             *reinterpret_cast<uint2*>(sidxV + 4 * lane) = xv;
             __syncwarp();
             if (st.g >= NS) {
-                if (lane == 0) ok = mbar_wait(bar(BAR_EMPTY + s), ((st.g / NS) - 1) & 1, abort_flag);
+                if (lane == 0) ok = mbar_wait(bar(BAR_EMPTY + s), ((st.g / NS) - 1) & 1, abort_flag, SITE_STAGE);
                 ok = __all_sync(0xffffffffu, ok);
             }
             if (!ok) break;
+            const int q_slot = st.j == 0 ? st.useq % NQ : -1;
             if (st.j == 0) {  // a new unit: stage its Q block (rows beyond M are zero)
-                if (st.useq >= NQ) {
-                    if (lane == 0) ok = mbar_wait(bar(BAR_QEMPTY + st.useq % NQ), ((st.useq / NQ) - 1) & 1, abort_flag);
-                    ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) break;
+                // Q blocks are taken up in unit order.  A parity wait cannot tell "this buffer's previous use has been
+                // released" from "not even the use before that has": with short units the producers work on five
+                // consecutive units at once, so the warp staging unit u could otherwise overtake the one still
+                // waiting to stage unit u - NQ.
+                if (lane == 0) {
+                    ok = false;
+                    for (uint32_t it = 0; it < (kSpinLimit << 3); ++it) {
+                        if (abort_flag[4] == st.useq) {
+                            ok = true;
+                            break;
+                        }
+                        if ((it & 63u) == 63u && *abort_flag) break;
+                        __nanosleep(64);
+                    }
+                    if (!ok && !*abort_flag) note_site(abort_flag, SITE_QTURN);
+                    if (ok && st.useq >= NQ)
+                        ok = mbar_wait(bar(BAR_QEMPTY + st.useq % NQ), ((st.useq / NQ) - 1) & 1, abort_flag, SITE_QBUF);
+                    if (ok) abort_flag[4] = st.useq + 1;
                 }
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
                 const uint32_t qdst = sbase + kOffQ + (st.useq % NQ) * kTileK + kv_lane;
                 const int rows_in = st.u.wk.M - st.u.row0;
                 const uint16_t* qsrc = Q + ((int64_t)(st.u.wk.q0 + st.u.row0 + q) * G + st.u.grp) * D + chunk * 8;
@@ -1025,7 +1097,10 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
             }
             fence_proxy_async();  // by the writing threads themselves: a fence on the reading side alone is not enough
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar(BAR_FULL + s));
+            if (lane == 0) {
+                if (q_slot >= 0) mbar_arrive(bar(BAR_QFULL + q_slot));
+                mbar_arrive(bar(BAR_FULL + s));
+            }
         }
         cp_async_wait<0>();
         if (!ok) {
@@ -1036,7 +1111,8 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
 
     tc_fence_before();
     __syncthreads();
-    if (warp == kMmaWarp) {
+    if (tid == 0 && abort_flag[1] != 0) atomicOr(err_flag, abort_flag[1] << 8);
+    if (warp == kIssueWarp0) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
     }

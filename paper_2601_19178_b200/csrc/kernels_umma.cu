@@ -80,8 +80,7 @@ constexpr int kOffQ = 0;
 constexpr int kOffK = kOffQ + NQ * kTileK;
 constexpr int kOffV = kOffK + NS * kTileK;
 constexpr int kOffX = kOffV + NS * kTileV;          // what groups 1.. hand to group 0 when a unit ends: [NG - 1][34][128] floats
-constexpr int kOffIdx = kOffX + (NG - 1) * 34 * 128 * 4;        // per producer warp: K and V row indices of its tile, 16 bit
-constexpr int kOffBar = kOffIdx + kProducerWarps * 2 * TK * 2;
+constexpr int kOffBar = kOffX + (NG - 1) * 34 * 128 * 4;
 constexpr int kOffAbort = kOffBar + 448;
 constexpr int kSmemBytes = kOffAbort + 32;
 
@@ -589,6 +588,18 @@ struct Stream {
             to_next_unit();
         }
     }
+    // n tiles on
+    __device__ __forceinline__ void advance_by(int n)
+    {
+        g += n;
+        j += n;
+        while (valid && j >= u.n_tiles) {
+            const int over = j - u.n_tiles;
+            ++useq;
+            to_next_unit();  // sets j = 0
+            j = over;
+        }
+    }
 };
 
 // VIS: visible lengths (a.vis, a.vmax); the plain instantiations carry none of that code.
@@ -984,8 +995,6 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
         const bool full_k = a.cv.full_k != 0, full_v = a.cv.full_v != 0;
         const char* rowsK0 = reinterpret_cast<const char*>(a.cv.userK) + chunk * 16;
         const char* rowsV0 = reinterpret_cast<const char*>(a.cv.userV) + chunk * 16;
-        uint16_t* sidxK = reinterpret_cast<uint16_t*>(smem + kOffIdx) + pw * 2 * TK;  // this warp's row indices of a tile
-        uint16_t* sidxV = sidxK + TK;
         Stream<false, VIS> st;
         st.init(a, n_mb, n_work);
         for (int i = 0; i < pw && st.valid; ++i) st.advance();
@@ -1025,9 +1034,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                 uk[rb] = uk_n[rb];
                 uv[rb] = uv_n[rb];
             }
-            *reinterpret_cast<uint2*>(sidxK + 4 * lane) = xk;
-            *reinterpret_cast<uint2*>(sidxV + 4 * lane) = xv;
-            __syncwarp();
+            const uint2 xk_cur = xk, xv_cur = xv;  // this tile's indices (fetch() below refills xk, xv for the next)
             if (st.g >= NS) {
                 if (lane == 0) ok = mbar_wait(bar(BAR_EMPTY + s), ((st.g / NS) - 1) & 1, abort_flag, SITE_STAGE);
                 ok = __all_sync(0xffffffffu, ok);
@@ -1070,19 +1077,31 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
             const char* pv = full_v ? rowsV0 + tile_unit0 * (D * 2) : poolV0 + st.u.grp * pool_stride;
             const uint32_t kdst = sbase + kOffK + s * kTileK + kv_lane, vdst = sbase + kOffV + s * kTileV + kv_lane;
             const int valid = st.j == st.u.n_tiles - 1 ? st.u.last_valid : TK;
-#pragma unroll 2
+            // The indices of positions 32 rb + 4 q .. + 3 are with lane 8 rb + q (it fetched them as one 8-byte
+            // word per side); all sixteen of a side come over by shuffles before the first copy is issued, so that
+            // the copies are not strung out between dependent loads.
+            uint32_t ik[8], iv[8];
+#pragma unroll
+            for (int rb = 0; rb < 4; ++rb) {
+                ik[2 * rb] = __shfl_sync(0xffffffffu, xk_cur.x, 8 * rb + q);
+                ik[2 * rb + 1] = __shfl_sync(0xffffffffu, xk_cur.y, 8 * rb + q);
+                iv[2 * rb] = __shfl_sync(0xffffffffu, xv_cur.x, 8 * rb + q);
+                iv[2 * rb + 1] = __shfl_sync(0xffffffffu, xv_cur.y, 8 * rb + q);
+            }
+#pragma unroll
             for (int it = 0; it < 16; ++it) {  // rb = it / 4, i = it % 4: position 32 rb + 4 q + i -> tile row 32 rb + 8 i + q
                 const int pos = 32 * (it >> 2) + 4 * q + (it & 3);
                 const uint32_t nb = pos < valid ? 16u : 0u;  // rows of positions beyond the history are zero
+                const int jk = (int)((ik[it >> 1] >> (16 * (it & 1))) & 0xffffu), jv = (int)((iv[it >> 1] >> (16 * (it & 1))) & 0xffffu);
                 // (range-checked build: pool indices below n_entries, destinations inside the stage)
                 (void)CKV_CLAMP((int)(512 * it + kv_lane), kTileK - 15, err_flag);
                 (void)CKV_CLAMP((int)(kVGroup * it + kv_lane), kTileV - 15, err_flag);
-                cp_async16(kdst + 512 * it, pk + (size_t)CKV_CLAMP((int)sidxK[pos], full_k ? TK : a.cv.n_entries, err_flag) * (D * 2), nb);
-                cp_async16(vdst + kVGroup * it, pv + (size_t)CKV_CLAMP((int)sidxV[pos], full_v ? TK : a.cv.n_entries, err_flag) * (D * 2), nb);
+                cp_async16(kdst + 512 * it, pk + (size_t)CKV_CLAMP(jk, full_k ? TK : a.cv.n_entries, err_flag) * (D * 2), nb);
+                cp_async16(vdst + kVGroup * it, pv + (size_t)CKV_CLAMP(jv, full_v ? TK : a.cv.n_entries, err_flag) * (D * 2), nb);
             }
             cp_async_commit();
             // what this warp's next tile needs travels while the copies land
-            for (int i = 0; i < kProducerWarps && st.valid; ++i) st.advance();
+            st.advance_by(kProducerWarps);
             fetch();
             cp_async_wait<0>();
             __syncwarp();  // a row's chunks were copied by four lanes of this warp

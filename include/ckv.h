@@ -370,6 +370,8 @@ CKV_API ckv_status ckv_get_option(ckv_ctx* ctx, const char* name, int64_t* value
  * query waits for that attend to finish; CKV_ERR_STATE if nothing was timed).
  * "device_errors" (not tied to the last call): non-zero once a kernel of this context gave up
  * on one of its internal bounded waits -- its outputs are then invalid; synchronises the device.
+ * (Diagnostics of the tcgen05 kernel: bits 0-3 name the roles that gave up, bits 8-11 the wait
+ * that ran out first.)
  * In the range-checked build of the library (build.py --bounds) bit 32 of it reports an index, row
  * or shared-memory offset that a kernel found outside its bound (the access is then redirected, not
  * performed).

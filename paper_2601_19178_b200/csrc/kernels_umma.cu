@@ -100,7 +100,8 @@ static_assert(BAR_COUNT * 8 <= 448, "barrier area");
 static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
 
 
-// error codes OR-ed into the context's device error word
+// error codes OR-ed into the context's device error word: which role gave up (bits 0..3); bits 8..11 carry the
+// site code of the first wait that ran out (see SITE_*)
 enum { ERR_NORMALISE = 1, ERR_MMA = 2, ERR_DRAIN = 4, ERR_PRODUCER = 8 };
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
@@ -981,8 +982,9 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
         // copies, so the per-tile bookkeeping is paid by one warp while the others work on their own
         // tiles.  Lane (q = lane / 4, chunk = lane % 4) copies chunk `chunk` of the pool rows of
         // positions 32 rb + 4 q + i (rb, i < 4) into tile rows 32 rb + 8 i + q, and patches the
-        // user-specific leading elements of tile rows 32 rb + lane.  The loops are kept rolled on
-        // purpose: the kernel's speed depends on how little code its roles execute.
+        // user-specific leading elements of tile rows 32 rb + lane.  A producer is one warp running a chain of
+        // dependent instructions per tile: five of them keep the stage ring ahead of three groups only because a
+        // tile's 32 copies per lane are issued back to back, with nothing that waits between them.
         const int pw = warp - kProducerWarp0, q = lane >> 2, chunk = lane & 3;
         const int patch_pos = 4 * (lane & 7) + (lane >> 3);  // position (inside a 32-block) held by row `lane`
         const uint32_t kv_lane = (uint32_t)(chunk * 128 + q * 16);

@@ -79,7 +79,7 @@ static_assert(NS % kProducerWarps == 0, "a stage is always filled by the same pr
 constexpr int kOffQ = 0;
 constexpr int kOffK = kOffQ + NQ * kTileK;
 constexpr int kOffV = kOffK + NS * kTileK;
-constexpr int kOffX = kOffV + NS * kTileV;          // what groups 1.. hand to group 0 when a unit ends: [NG - 1][34][128] floats
+constexpr int kOffX = kOffV + NS * kTileV;          // what the other groups hand to the merging one when a unit ends: [NG - 1][34][128] floats
 constexpr int kOffBar = kOffX + (NG - 1) * 34 * 128 * 4;
 constexpr int kOffAbort = kOffBar + 448;
 constexpr int kSmemBytes = kOffAbort + 32;
@@ -91,8 +91,8 @@ enum {
     BAR_PREADY = BAR_SFULL + NG * NB,     // [NB b + i]
     BAR_PFREE = BAR_PREADY + NG * NB,     // [NB b + i]
     BAR_OFULL = BAR_PFREE + NG * NB,      // [b]
-    BAR_XFULL = BAR_OFULL + NG,           // [b - 1]
-    BAR_XEMPTY = BAR_XFULL + NG - 1,      // [b - 1]
+    BAR_XFULL = BAR_OFULL + NG,           // [slot]
+    BAR_XEMPTY = BAR_XFULL + NG - 1,      // [slot]
     BAR_DRAIN = BAR_XEMPTY + NG - 1,      // [b]
     BAR_COUNT = BAR_DRAIN + NG
 };
@@ -771,22 +771,26 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
 #pragma unroll
                 for (int e = 0; e < 32; ++e) o[e] = 0.f;
             }
-            if (b > 0) {
-                float* x = xch + (b - 1) * 34 * 128;
-                if (xcnt > 0) ok = mbar_wait(bar(BAR_XEMPTY + b - 1), (xcnt - 1) & 1, abort_flag, SITE_XEMPTY);
+            // The group that has the unit's last half merges and stores: it is the last to finish anyway, and what
+            // the other two hand over (slot 0: the group after it, slot 1: the one after that) is there by then.
+            const int merger = (n_half - 1 + unit_rotation(u)) % NG;
+            if (b != merger) {
+                const int slot = (b + NG - merger - 1) % NG;
+                float* x = xch + slot * 34 * 128;
+                if (xcnt > 0) ok = mbar_wait(bar(BAR_XEMPTY + slot), (xcnt - 1) & 1, abort_flag, SITE_XEMPTY);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 x[row] = m_ref;
                 x[128 + row] = l;
 #pragma unroll
                 for (int e = 0; e < 32; ++e) x[(2 + e) * 128 + row] = o[e];
-                mbar_arrive(bar(BAR_XFULL + b - 1));
+                mbar_arrive(bar(BAR_XFULL + slot));
                 ++xcnt;
             } else {
 #pragma unroll 1
-                for (int g2 = 1; g2 < NG && ok; ++g2) {
-                    const float* x = xch + (g2 - 1) * 34 * 128;
-                    ok = mbar_wait(bar(BAR_XFULL + g2 - 1), xcnt & 1, abort_flag, SITE_XFULL);
+                for (int slot = 0; slot < NG - 1 && ok; ++slot) {
+                    const float* x = xch + slot * 34 * 128;
+                    ok = mbar_wait(bar(BAR_XFULL + slot), xcnt & 1, abort_flag, SITE_XFULL);
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                     const float m1 = x[row], l1 = x[128 + row];
@@ -802,7 +806,7 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
 #pragma unroll
                         for (int e = 0; e < 32; ++e) o[e] += x[(2 + e) * 128 + row];
                     }
-                    mbar_arrive(bar(BAR_XEMPTY + g2 - 1));
+                    mbar_arrive(bar(BAR_XEMPTY + slot));
                 }
                 if (!ok) break;
                 ++xcnt;
@@ -915,10 +919,12 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                 for (int p = (b + NG - rot) % NG; p < n_half; p += NG) {
                     const int t = gs + (p >> 1), half = p & 1;
                     const int s = t % NS, par = gp ^ ((t / NS) & 1);
-                    ok = catch_up(ss.g + (p >> 1)) && mbar_wait_fast(bar(BAR_FULL + s), par, abort_flag, SITE_TILE);
-                    // buffer i still holds the weights of step cnt - NB: its weighted sum goes first.  The tensor core
-                    // runs this thread's instructions in order, so the scores below need not wait for it to finish.
+                    ok = catch_up(ss.g + (p >> 1));
+                    // buffer i still holds the weights of step cnt - NB: its weighted sum goes first (and before the
+                    // wait for the tile: at a unit's end the group is waiting for exactly this weighted sum).  The tensor
+                    // core runs this thread's instructions in order, so the scores below need not wait for it to finish.
                     if (ok && cnt - done == NB) ok = issue_pv();
+                    if (ok) ok = mbar_wait_fast(bar(BAR_FULL + s), par, abort_flag, SITE_TILE);
                     if (ok && !q_seen) {  // first scores of a unit: its Q block must have landed
                         ok = mbar_wait_fast(bar(BAR_QFULL + ss.useq % NQ), (ss.useq / NQ) & 1, abort_flag, SITE_Q);
                         q_seen = true;

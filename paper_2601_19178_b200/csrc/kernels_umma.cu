@@ -771,11 +771,11 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
 #pragma unroll
                 for (int e = 0; e < 32; ++e) o[e] = 0.f;
             }
-            // The group that has the unit's last half merges and stores: it is the last to finish anyway, and what
-            // the other two hand over (slot 0: the group after it, slot 1: the one after that) is there by then.
-            const int merger = (n_half - 1 + unit_rotation(u)) % NG;
-            if (b != merger) {
-                const int slot = (b + NG - merger - 1) % NG;
+            // Group 0 merges and stores, always: a barrier of the hand-over is then waited on by the same threads use
+            // after use.  (With the merging passed round -- to the group that has the unit's last half -- a group
+            // could come to wait for a use while the one before was still open, and a parity wait cannot tell.)
+            if (b != 0) {
+                const int slot = b - 1;
                 float* x = xch + slot * 34 * 128;
                 if (xcnt > 0) ok = mbar_wait(bar(BAR_XEMPTY + slot), (xcnt - 1) & 1, abort_flag, SITE_XEMPTY);
                 ok = __all_sync(0xffffffffu, ok);
@@ -870,7 +870,6 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
             // last half of the unit)
             uint32_t pv_off0 = 0, pv_off1 = 0;
             int pv_s0 = 0, pv_s1 = 0, pv_f0 = 0, pv_f1 = 0;
-            int pv_t0 = 0, pv_t1 = 0;  // their tiles' places in the stream
             int gs = 0, gp = 0;  // stage and phase parity of the unit's first tile: g % NS, (g / NS) & 1
             bool ok = true;
             // O_b += P_bi V_half for step `done`, whose group has written P_bi
@@ -887,7 +886,6 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                 pv_off0 = pv_off1;
                 pv_s0 = pv_s1;
                 pv_f0 = pv_f1;
-                pv_t0 = pv_t1;
                 ++done;
             };
             // ... waiting for the weights first (used where the thread can do nothing else)
@@ -895,20 +893,6 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                 if (!mbar_wait_fast(bar(BAR_PREADY + NB * b + (done & 1)), (done >> 1) & 1, abort_flag, SITE_PREADY)) return false;
                 do_pv();
                 return true;
-            };
-            // A weighted sum is normally issued when its buffer is wanted for the scores two steps on.  Where the
-            // group's halves lie far apart (short units whose halves go to the other groups) that could be never: the
-            // weighted sum releases a stage, and the tile this thread waits for next may need that very stage.  So
-            // before waiting for tile `t_now` of the stream, the weighted sums of steps kMaxLag or more tiles back are
-            // issued first (in the regular rhythm of one half in three a pending step is at most five tiles back, so
-            // this never delays the scores there).  With every issuer keeping to that, the tile the hindmost issuer
-            // waits for only needs stages of tiles NS back, which nobody holds any more.
-            constexpr int kMaxLag = 7;
-            static_assert(kMaxLag < NS, "a held stage must never be the one the awaited tile goes to");
-            auto catch_up = [&](int t_now) {
-                bool w = true;
-                while (w && done < cnt && t_now - pv_t0 >= kMaxLag) w = issue_pv();
-                return w;
             };
             for (; ok && ss.valid; ss.next_unit()) {
                 const Unit& u = ss.u;
@@ -919,7 +903,6 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                 for (int p = (b + NG - rot) % NG; p < n_half; p += NG) {
                     const int t = gs + (p >> 1), half = p & 1;
                     const int s = t % NS, par = gp ^ ((t / NS) & 1);
-                    ok = catch_up(ss.g + (p >> 1));
                     // buffer i still holds the weights of step cnt - NB: its weighted sum goes first (and before the
                     // wait for the tile: at a unit's end the group is waiting for exactly this weighted sum).  The tensor
                     // core runs this thread's instructions in order, so the scores below need not wait for it to finish.
@@ -943,20 +926,27 @@ __global__ void __launch_bounds__(kThreads, 1) attend_umma_kernel(const AttendAr
                         pv_off0 = off;
                         pv_s0 = s;
                         pv_f0 = f;
-                        pv_t0 = ss.g + (p >> 1);
                     } else {
                         pv_off1 = off;
                         pv_s1 = s;
                         pv_f1 = f;
-                        pv_t1 = ss.g + (p >> 1);
                     }
                     ++cnt;
                 }
                 if (!ok) break;
-                ok = catch_up(ss.g + u.n_tiles - 1);
-                if (!ok) break;
                 const int t_last = gs + u.n_tiles - 1;
-                if (u.last_valid <= TH && (2 * u.n_tiles - 1 + rot) % NG == b) {
+                const bool empty_tail = u.last_valid <= TH && (2 * u.n_tiles - 1 + rot) % NG == b;
+                // A weighted sum is normally issued when its buffer is wanted for the scores two steps on.  In a run of
+                // short units whose halves go to the other groups that could be many units on -- while the other groups
+                // wait, at the end of the unit it belongs to, for this group's accumulator, the issuing threads behind
+                // them stop releasing Q blocks and stages, and the tile or Q block this thread is waiting for never comes.
+                // So where this thread passes a unit in which it issued nothing (or has only the empty tail to release),
+                // whatever it still holds is issued first; waiting for the weights there cannot block on anything this
+                // thread does later.  Units in which the group has halves keep their lead of two steps.
+                if (!q_seen || empty_tail)
+                    while (ok && done < cnt) ok = issue_pv();
+                if (!ok) break;
+                if (empty_tail) {
                     // the empty second half of the unit's last tile is this group's: nothing to compute, but the
                     // stage needs this half's release
                     ok = mbar_wait_fast(bar(BAR_FULL + t_last % NS), gp ^ ((t_last / NS) & 1), abort_flag, SITE_TAIL_TILE);

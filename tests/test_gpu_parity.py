@@ -442,3 +442,38 @@ def test_replacing_and_evicting_users():
     assert full == 2 * (2 * L0) * w.n_groups * w.head_dim * 4
     assert comp == (2 * L0) * w.n_groups * (2 * 2 + 2 * w.d_user * 4)
     s.close()
+
+
+def _cut_histories(d, new_lens):
+    """The generated data with user k's history cut to its first new_lens[k] positions."""
+    off = d["hist_off"]
+    keep = np.concatenate([np.arange(off[k], off[k] + n) for k, n in enumerate(new_lens)]).astype(np.int64)
+    out = dict(d)
+    for key in ("idx_K", "idx_V", "user_K", "user_V"):
+        out[key] = np.ascontiguousarray(d[key][keep])
+    out["hist_off"] = np.concatenate([[0], np.cumsum(new_lens)]).astype(np.int64)
+    return out
+
+
+@pytest.mark.parametrize("mode", ["softmax", "silu_over_l"])
+@pytest.mark.parametrize("n_groups", [1, 4])
+def test_tcgen05_kernel_long_units_followed_by_many_short_ones(mode, n_groups):
+    """A few long histories and many of at most two half tiles.  The planner puts the long ones first, so every
+    CTA of the tcgen05 kernel ends its stream with a run of units in which a normalisation group may own no half
+    for many tiles while it still has weighted sums to issue for the long unit; with one or four groups the
+    rotation that deals the halves out is the same for all units of a CTA, which makes such runs as long as
+    they get.  Nothing may run out of its bounded waits, and the results must match."""
+    rng = np.random.default_rng(5)
+    n_users = 700
+    w = synth.Workload("mixed", n_groups, 30, 2, 500, n_users, (1900, 1900), 64, mode, "bf16", 1.1, 1 / 32, 1 / 32, 77)
+    d = synth.generate(w)
+    # (SiLU: h (1 + tanh h) with the hardware's tanh cancels for strongly negative scores -- absolute error up to
+    # about 5e-4 |h| per term; a row made of one or two such terms alone would fail the row-normalised bound)
+    lens = rng.integers(1 if mode == "softmax" else 17, 129, size=n_users)
+    lens[rng.choice(n_users, 40, replace=False)] = rng.integers(1200, 1901, size=40)
+    d = _cut_histories(d, lens)
+    s = make_session(w, d, kernel=3)
+    got = gpu_attend(w, d, session=s)
+    assert s.stat("kernel") == 3 and s.stat("device_errors") == 0
+    s.close()
+    assert_close(got, oracle_attend(w, d), "bf16", f"{mode} G={n_groups}")

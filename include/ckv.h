@@ -165,7 +165,8 @@ CKV_API ckv_status ckv_cache_clear(ckv_ctx* ctx);
  *   queries [any]  : [q_off[n]][n_groups][head_dim], ctx dtype
  *   out     [any]  : [q_off[n]][n_groups][head_dim], ctx out_dtype, caller-allocated
  * With host memory for both `queries` and `out` and a few MB or more of queries, the request list
- * is cut into four ranges of consecutive users whose upload, kernels and download run on streams
+ * is cut into four ranges of consecutive users (eight from about 100 MB of queries on) whose upload,
+ * kernels and download run on streams
  * of the library's own, so that the three overlap (pinned host memory is what makes the copies
  * asynchronous); `stream` is ordered before the first and behind the last of them, and the
  * results are the same bits.
@@ -363,7 +364,7 @@ CKV_API ckv_status ckv_get_option(ckv_ctx* ctx, const char* name, int64_t* value
  * (loader the last warp-level tensor-core launch used: 1 or 2),
  * "workspace_bytes", "plan_cache_hit", "alloc_calls" (device or pinned-host allocations the call
  * made: 0 once its buffers have reached their size), "l2_window" (1 if the pool's L2 window was on
- * the stream for the call), "pipeline_ranges" (ranges of users a host-buffer call was cut into: 1 or 4); "arena_capacity_units", "arena_used_units", "arena_free_runs" (state of
+ * the stream for the call), "pipeline_ranges" (ranges of users a host-buffer call was cut into: 1, 4 or 8); "arena_capacity_units", "arena_used_units", "arena_free_runs" (state of
  * the compressed-cache storage, in (position, group) units); with option "time_kernels" also
  * "main_kernel_ns" and
  * "combine_kernel_ns" (device time of the attend kernel and of the split-merge kernel; the

@@ -119,7 +119,7 @@ public:
     }
 };
 
-constexpr int kMaxRanges = 4;
+constexpr int kMaxRanges = 8;
 
 struct DevBuf {  // grow-only device buffer
     void* p = nullptr;
@@ -1187,6 +1187,7 @@ ckv_status run_mma(ckv_ctx* ctx, int D, int max_M, const AttendArgs& a, cudaStre
 namespace {
 
 constexpr size_t kPipeMinBytes = size_t(4) << 20;  // host query buffers below this are not worth pipelining
+constexpr size_t kPipeManyBytes = size_t(96) << 20;  // from here on: eight ranges instead of four
 
 cudaError_t pipe_prepare(ckv_ctx* ctx)
 {
@@ -1262,9 +1263,13 @@ ckv_status attend_impl(ckv_ctx* ctx, int32_t n, const int64_t* users, const int3
     // kernels and its download.  The uploads are enqueued before the plan is looked up or built, so that host
     // work overlaps them too.
     int n_ranges = 1;
-    int32_t r_user[kMaxRanges + 1] = {0, n, n, n, n};
-    if (q_host && o_host && q_bytes >= kPipeMinBytes && n >= 2 * kMaxRanges && pipe_prepare(ctx) == cudaSuccess) {
-        n_ranges = kMaxRanges;
+    int32_t r_user[kMaxRanges + 1];
+    r_user[0] = 0;
+    for (int r = 1; r <= kMaxRanges; ++r) r_user[r] = n;
+    if (q_host && o_host && q_bytes >= kPipeMinBytes && n >= 8 && pipe_prepare(ctx) == cudaSuccess) {
+        // four ranges; eight once a range is still tens of MB (the first upload and the last download, which
+        // nothing overlaps, are then an eighth of the traffic instead of a quarter)
+        n_ranges = (q_bytes >= kPipeManyBytes && n >= 2 * kMaxRanges) ? kMaxRanges : 4;
         int32_t k = 0;
         for (int r = 1; r < n_ranges; ++r) {
             const int64_t want = Q * r / n_ranges;

@@ -1294,9 +1294,9 @@ ckv_status attend_impl(ckv_ctx* ctx, int32_t n, const int64_t* users, const int3
         CK(cudaMemcpyAsync(ctx->stage_vis.p, vis, (size_t)Q * sizeof(int32_t), cudaMemcpyHostToDevice, s));
         d_vis = (const int32_t*)ctx->stage_vis.p;
     }
-    // The first range's upload goes out before the plan is looked up or built, so that the host work overlaps
-    // it; the other ranges follow the plan's own (small) upload, which would otherwise queue behind all of them
-    // on the copy engine and hold back the first kernels.
+    // The first range's upload (the first two for long request lists) goes out before the plan is looked up or built, so that
+    // the host work overlaps it; the other ranges follow the plan's own (small) upload, which would otherwise
+    // queue behind all of them on the copy engine and hold back the first kernels.
     auto upload_range = [&](int r) -> cudaError_t {
         cudaStream_t ps = ctx->pipe_stream[r];
         cudaError_t e = cudaStreamWaitEvent(ps, ctx->pipe_start, 0);
@@ -1307,9 +1307,10 @@ ckv_status attend_impl(ckv_ctx* ctx, int32_t n, const int64_t* users, const int3
         if (e == cudaSuccess) e = cudaEventRecord(ctx->pipe_h2d[r], ps);
         return e;
     };
+    const int n_early = (n_ranges > 4 && n >= 8192) ? 2 : 1;  // planning thousands of users takes about as long as two uploads
     if (n_ranges > 1) {
         CK(cudaEventRecord(ctx->pipe_start, s));
-        CK(upload_range(0));
+        for (int r = 0; r < n_early; ++r) CK(upload_range(r));
     } else if (q_host) {
         CK(cudaMemcpyAsync(ctx->stage_q.p, queries, q_bytes, cudaMemcpyHostToDevice, s));
     }
@@ -1317,12 +1318,13 @@ ckv_status attend_impl(ckv_ctx* ctx, int32_t n, const int64_t* users, const int3
     Plan* pl = nullptr;
     ckv_status st = get_plan(ctx, n, users, q_off, vis != nullptr, n_ranges, r_user, s, &pl);
     if (st != CKV_OK) {
-        if (n_ranges > 1) cudaStreamWaitEvent(s, ctx->pipe_h2d[0], 0);  // the upload already enqueued stays inside the call
+        if (n_ranges > 1)  // the uploads already enqueued stay inside the call
+            for (int r = 0; r < n_early; ++r) cudaStreamWaitEvent(s, ctx->pipe_h2d[r], 0);
         return st;
     }
     if (n_ranges > 1) {
         CK(cudaEventRecord(ctx->pipe_plan, s));
-        for (int r = 1; r < n_ranges; ++r) CK(upload_range(r));
+        for (int r = n_early; r < n_ranges; ++r) CK(upload_range(r));
     }
     ctx->st_items = pl->n_items;
     ctx->st_split = pl->split_items;

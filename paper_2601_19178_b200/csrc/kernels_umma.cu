@@ -70,6 +70,7 @@ constexpr uint32_t kColGroup = 64 * NB + D;  // group b: S_bi (and P_bi over its
 static_assert(kColGroup * NG <= kTmemCols, "TMEM columns");
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kHeadroom = 64.0f;       // log2 units a score may exceed the reference maximum
+constexpr float kSumLimit = 1180591620717411303424.0f;  // 2^70: a chunk's sum beyond it gives the excess away
 constexpr uint32_t kSpinLimit = 1u << 18;  // polls of a wait before the CTA gives up
 constexpr uint32_t kSuspendNs = 4000;      // how long one poll may stay suspended in hardware (longer hints wake later)
 static_assert(NS > kProducerWarps, "every producer warp holds one stage while it copies");
@@ -334,6 +335,19 @@ __device__ __noinline__ float rewrite_weights(uint32_t tP, const uint32_t* cur, 
     return sum;
 }
 
+// Largest exponent argument of one 32-column chunk (rare path only, like rewrite_weights).
+template <bool TAIL>
+__device__ __noinline__ float chunk_max(const uint32_t* cur, float sc, float nm, int valid, int c)
+{
+    float mx = -CUDART_INF_F;
+#pragma unroll
+    for (int e = 0; e < 32; ++e) {
+        const float x = fmaf(__uint_as_float(cur[e]), sc, nm);
+        if (!TAIL || pos_of_col(c, e) < valid) mx = fmaxf(mx, x);
+    }
+    return mx;
+}
+
 // Softmax weights of one 32-column chunk (c = 0, 1) of a 128 x 64 score half tile: p = exp2(s c - m) as bf16
 // pairs written over the head of the scores (columns 0..31 of the buffer; chunk 1 of the scores, columns 32..63,
 // is still to be read when chunk 0's weights land on columns 0..15, and chunk 1's weights
@@ -366,7 +380,6 @@ __device__ __forceinline__ bool softmax_chunk(const uint32_t (&cur)[32], int c, 
         m_ref = fmaxf(t0, t1) * sc;
     }
     float nm = -m_ref;
-    float mx = -CUDART_INF_F, mx2 = -CUDART_INF_F;
     float ls0 = 0.f, ls1 = 0.f;  // this chunk's share of the row sum
     uint32_t p[16];
 #pragma unroll
@@ -376,20 +389,24 @@ __device__ __forceinline__ bool softmax_chunk(const uint32_t (&cur)[32], int c, 
             if (pos_of_col(c, e) >= valid) x0 = -CUDART_INF_F;
             if (pos_of_col(c, e + 1) >= valid) x1 = -CUDART_INF_F;
         }
-        if (e & 2) mx = max3(mx, x0, x1);
-        else mx2 = max3(mx2, x0, x1);
         const float e0 = ex2(x0), e1 = ex2(x1);
         ls0 += e0;
         ls1 += e1;
         p[e >> 1] = pack_bf16(e0, e1);
     }
-    mx = fmaxf(mx, mx2);
-    if (!__any_sync(0xffffffffu, mx > kHeadroom)) {
+    // Leaving the headroom shows in the chunk's sum: 32 weights of at most 2^64 add up to at most 2^69, so a sum
+    // beyond kSumLimit = 2^70 (or one that is not a number) means some weight of this row is beyond 2^65.  That
+    // costs one comparison here instead of a running maximum over the arguments.
+    if (!__any_sync(0xffffffffu, !(ls0 + ls1 <= kSumLimit))) {
         tmem_st16(tS + 16 * c, p);
     } else {
         // rare: some row of this warp left the headroom and its weights may have overflowed.  Nothing of this
         // chunk has been written yet, so its scores are still in TMEM: move the reference, bring what was
         // accumulated and written before into the new scale, and work the chunk out again from there.
+        uint32_t again[32];
+        tmem_ld32(tS + 32 * c, again);
+        tmem_wait_ld32(again);
+        const float mx = chunk_max<TAIL>(again, sc, nm, valid, c);
         const float shift = mx > kHeadroom ? ceilf(mx) : 0.f;
         const float f = ex2(-shift);
         m_ref += shift;
@@ -402,9 +419,6 @@ __device__ __forceinline__ bool softmax_chunk(const uint32_t (&cur)[32], int c, 
             rescale_row(tO, f);
         }
         if (c == 1) rescale_weights(tS, f);
-        uint32_t again[32];
-        tmem_ld32(tS + 32 * c, again);
-        tmem_wait_ld32(again);
         ls0 = rewrite_weights<TAIL>(tS + 16 * c, again, sc, nm, valid, c);
         ls1 = 0.f;
         tc_wait_st();

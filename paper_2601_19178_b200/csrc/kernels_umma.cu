@@ -279,6 +279,40 @@ __device__ __forceinline__ float max3(float a, float b, float c)
     return r;
 }
 
+// Two fp32 operations in one instruction (packed pairs): the normalisation is short of issue slots, not of FMA lanes.
+// (d0, d1) = (a0, a1) * b + c
+__device__ __forceinline__ void fma2_scalar(float& d0, float& d1, float a0, float a1, float b, float c)
+{
+    asm("{\n.reg .b64 ra, rb, rc, rd;\nmov.b64 ra, {%2, %3};\nmov.b64 rb, {%4, %4};\nmov.b64 rc, {%5, %5};\n"
+        "fma.rn.f32x2 rd, ra, rb, rc;\nmov.b64 {%0, %1}, rd;\n}\n"
+        : "=f"(d0), "=f"(d1)
+        : "f"(a0), "f"(a1), "f"(b), "f"(c));
+}
+// (d0, d1) = (a0, a1) * (b0, b1) + (c0, c1)
+__device__ __forceinline__ void fma2(float& d0, float& d1, float a0, float a1, float b0, float b1, float c0, float c1)
+{
+    asm("{\n.reg .b64 ra, rb, rc, rd;\nmov.b64 ra, {%2, %3};\nmov.b64 rb, {%4, %5};\nmov.b64 rc, {%6, %7};\n"
+        "fma.rn.f32x2 rd, ra, rb, rc;\nmov.b64 {%0, %1}, rd;\n}\n"
+        : "=f"(d0), "=f"(d1)
+        : "f"(a0), "f"(a1), "f"(b0), "f"(b1), "f"(c0), "f"(c1));
+}
+// (d0, d1) += (a0, a1)
+__device__ __forceinline__ void add2(float& d0, float& d1, float a0, float a1)
+{
+    asm("{\n.reg .b64 ra, rd;\nmov.b64 rd, {%0, %1};\nmov.b64 ra, {%2, %3};\nadd.rn.f32x2 rd, rd, ra;\n"
+        "mov.b64 {%0, %1}, rd;\n}\n"
+        : "+f"(d0), "+f"(d1)
+        : "f"(a0), "f"(a1));
+}
+// (d0, d1) = (a0, a1) * b
+__device__ __forceinline__ void mul2_scalar(float& d0, float& d1, float a0, float a1, float b)
+{
+    asm("{\n.reg .b64 ra, rb, rd;\nmov.b64 ra, {%2, %3};\nmov.b64 rb, {%4, %4};\nmul.rn.f32x2 rd, ra, rb;\n"
+        "mov.b64 {%0, %1}, rd;\n}\n"
+        : "=f"(d0), "=f"(d1)
+        : "f"(a0), "f"(a1), "f"(b));
+}
+
 // byte offset of (row r, 16-byte chunk c) inside a K/Q tile and inside a V tile
 __device__ __forceinline__ uint32_t k_off(int r, int c) { return (uint32_t)((r >> 3) * 512 + c * 128 + (r & 7) * 16); }
 __device__ __forceinline__ uint32_t v_off(int r, int c) { return (uint32_t)((r >> 3) * kVGroup + c * 128 + (r & 7) * 16); }
@@ -384,14 +418,14 @@ __device__ __forceinline__ bool softmax_chunk(const uint32_t (&cur)[32], int c, 
     uint32_t p[16];
 #pragma unroll
     for (int e = 0; e < 32; e += 2) {
-        float x0 = fmaf(__uint_as_float(cur[e]), sc, nm), x1 = fmaf(__uint_as_float(cur[e + 1]), sc, nm);
+        float x0, x1;
+        fma2_scalar(x0, x1, __uint_as_float(cur[e]), __uint_as_float(cur[e + 1]), sc, nm);
         if (TAIL) {
             if (pos_of_col(c, e) >= valid) x0 = -CUDART_INF_F;
             if (pos_of_col(c, e + 1) >= valid) x1 = -CUDART_INF_F;
         }
         const float e0 = ex2(x0), e1 = ex2(x1);
-        ls0 += e0;
-        ls1 += e1;
+        add2(ls0, ls1, e0, e1);
         p[e >> 1] = pack_bf16(e0, e1);
     }
     // Leaving the headroom shows in the chunk's sum: 32 weights of at most 2^64 add up to at most 2^69, so a sum
@@ -435,8 +469,9 @@ __device__ __forceinline__ void silu_chunk(const uint32_t (&cur)[32], int c, uin
     uint32_t p[16];
 #pragma unroll
     for (int e = 0; e < 32; e += 2) {
-        const float h0 = __uint_as_float(cur[e]) * sc, h1 = __uint_as_float(cur[e + 1]) * sc;
-        float w0 = fmaf(h0, tanh_fast(h0), h0), w1 = fmaf(h1, tanh_fast(h1), h1);
+        float h0, h1, w0, w1;
+        mul2_scalar(h0, h1, __uint_as_float(cur[e]), __uint_as_float(cur[e + 1]), sc);
+        fma2(w0, w1, h0, h1, tanh_fast(h0), tanh_fast(h1), h0, h1);
         if (TAIL) {
             if (pos_of_col(c, e) >= valid) w0 = 0.f;
             if (pos_of_col(c, e + 1) >= valid) w1 = 0.f;

@@ -31,9 +31,9 @@
 //
 // Softmax bookkeeping.  The reference maximum m of a row is the largest of the first 32 scores of the group's
 // first half of the unit and stays fixed: later scores may exceed it by up to 2^64 (fp32 accumulators and bf16
-// P have the exponent range for that).  The largest exponent argument of every chunk is taken from the registers
-// with the weights; only when it exceeds that bound is the reference moved, O_b and the row sum rescaled (TMEM
-// read-modify-write) and the chunk written again.  The row sum l is added up by the row's thread in fp32.
+// P have the exponent range for that).  The row sum l is added up by the row's thread in fp32, chunk by chunk, and
+// a chunk's share of it also tells when a row has left that bound (32 weights within it sum to at most 2^69); only
+// then is the reference moved, O_b and the row sum rescaled (TMEM read-modify-write) and the chunk worked out again.
 //
 // Shared-memory tiles use the no-swizzle UMMA canonical layout: groups of 8 rows (512 bytes), inside a
 // group one 128-byte core matrix per 16-byte row chunk, inside a core matrix row r%8 at 16 r.
